@@ -1,0 +1,125 @@
+"""Second, structurally different float64 DeepPoly (TEST INFRASTRUCTURE).
+
+Where the C oracle walks one neuron's expression at a time with scalar sign
+tests, this file uses the layer-level form the paper's rewrites arrive at
+(Section 4.3: the Matmul rewrite turns map(c*n[L]) into a matrix product, the
+ternary/clamp rewrites turn `c >= 0 ? c*L : c*U` into
+clamp(c, min=0)*L + clamp(c, max=0)*U).  Conv layers are expanded to dense
+matrices by index arithmetic.  It exists to cross-check the C oracle; it
+imports neither the C oracle nor the CUDA package.
+"""
+from __future__ import annotations
+
+import numpy as np
+
+
+def dense_matrix(layer) -> np.ndarray:
+    """[n_out, n_in] float64 matrix of an affine layer (conv: cross-correlation, zero padding)."""
+    w = np.asarray(layer.weight, dtype=np.float64)
+    if layer.kind == "fc":
+        return w
+    c_out, c_in, kh, kw = w.shape
+    _, h, wd = layer.in_shape
+    s, p = layer.stride, layer.pad
+    ho, wo = (h + 2 * p - kh) // s + 1, (wd + 2 * p - kw) // s + 1
+    m = np.zeros((c_out, ho, wo, c_in, h, wd), dtype=np.float64)
+    oy, ox = np.meshgrid(np.arange(ho), np.arange(wo), indexing="ij")
+    for ky in range(kh):
+        for kx in range(kw):
+            iy, ix = oy * s - p + ky, ox * s - p + kx
+            ok = (iy >= 0) & (iy < h) & (ix >= 0) & (ix < wd)
+            for co in range(c_out):
+                for ci in range(c_in):
+                    m[co, oy[ok], ox[ok], ci, iy[ok], ix[ok]] = w[co, ci, ky, kx]
+    return m.reshape(c_out * ho * wo, c_in * h * wd)
+
+
+def dense_bias(layer) -> np.ndarray:
+    b = np.asarray(layer.bias, dtype=np.float64)
+    if layer.kind == "fc":
+        return b
+    n_out = dense_matrix_rows(layer)
+    return np.repeat(b, n_out // b.shape[0])
+
+
+def dense_matrix_rows(layer) -> int:
+    if layer.kind == "fc":
+        return layer.weight.shape[0]
+    c_out, _, kh, kw = layer.weight.shape
+    _, h, wd = layer.in_shape
+    s, p = layer.stride, layer.pad
+    return c_out * ((h + 2 * p - kh) // s + 1) * ((wd + 2 * p - kw) // s + 1)
+
+
+def box(centers, eps, clip_lo, clip_hi):
+    c = np.asarray(centers, dtype=np.float32)
+    e = np.float32(eps)
+    l0 = np.maximum(c - e, np.float32(clip_lo)).astype(np.float64)
+    u0 = np.minimum(c + e, np.float32(clip_hi)).astype(np.float64)
+    return l0, u0
+
+
+def deeppoly_matrix(layers, centers, eps, clip_lo=0.0, clip_hi=1.0, decision_fp32=True):
+    """Returns lb, ub [batch, n_total] float64 and codes [batch, n_relu] uint8."""
+    A = [dense_matrix(l) for l in layers]
+    bias = [dense_bias(l) for l in layers]
+    L0, U0 = box(centers, eps, clip_lo, clip_hi)
+    batch = L0.shape[0]
+    n_total = sum(a.shape[0] for a in A)
+    n_relu = sum(a.shape[0] for a, l in zip(A, layers) if l.relu_after)
+    lb_all = np.empty((batch, n_total))
+    ub_all = np.empty((batch, n_total))
+    codes_all = np.empty((batch, n_relu), dtype=np.uint8)
+    for b in range(batch):
+        l0, u0 = L0[b], U0[b]
+        lam_l, lam_u, nu_u = [], [], []
+        off, coff = 0, 0
+        for k, layer in enumerate(layers):
+            Cl, Cu = A[k].copy(), A[k].copy()
+            dl, du = bias[k].copy(), bias[k].copy()
+            for j in range(k - 1, -1, -1):
+                if layers[j].relu_after:
+                    Clp, Clm = np.clip(Cl, 0.0, None), np.clip(Cl, None, 0.0)
+                    Cup, Cum = np.clip(Cu, 0.0, None), np.clip(Cu, None, 0.0)
+                    dl = dl + Clm @ nu_u[j]
+                    du = du + Cup @ nu_u[j]
+                    Cl = Clp * lam_l[j] + Clm * lam_u[j]
+                    Cu = Cup * lam_u[j] + Cum * lam_l[j]
+                dl = dl + Cl @ bias[j]
+                du = du + Cu @ bias[j]
+                Cl = Cl @ A[j]
+                Cu = Cu @ A[j]
+            lb = np.clip(Cl, 0.0, None) @ l0 + np.clip(Cl, None, 0.0) @ u0 + dl
+            ub = np.clip(Cu, 0.0, None) @ u0 + np.clip(Cu, None, 0.0) @ l0 + du
+            n_k = lb.shape[0]
+            lb_all[b, off:off + n_k], ub_all[b, off:off + n_k] = lb, ub
+            off += n_k
+            if layer.relu_after:
+                if decision_fp32:
+                    lf, uf = lb.astype(np.float32), ub.astype(np.float32)
+                    active, inactive, pick = lf >= 0, uf <= 0, (lf + uf) >= 0
+                else:
+                    active, inactive, pick = lb >= 0, ub <= 0, (lb + ub) >= 0
+                unstable = ~active & ~inactive
+                den = np.where(unstable, ub - lb, 1.0)
+                lam_u.append(np.where(active, 1.0, np.where(inactive, 0.0, ub / den)))
+                nu_u.append(np.where(unstable, -(ub * lb) / den, 0.0))
+                lam_l.append(np.where(pick, 1.0, 0.0))
+                codes_all[b, coff:coff + n_k] = np.where(active, 1, np.where(inactive, 0, 2 + pick))
+                coff += n_k
+            else:
+                lam_l.append(None); lam_u.append(None); nu_u.append(None)
+    return lb_all, ub_all, codes_all
+
+
+def forward_preactivations(layers, x):
+    """Plain float64 forward pass; x [m, n0]; returns [m, n_total] pre-activations."""
+    A = [dense_matrix(l) for l in layers]
+    bias = [dense_bias(l) for l in layers]
+    a = np.asarray(x, dtype=np.float64)
+    outs = []
+    for k, layer in enumerate(layers):
+        z = a @ A[k].T + bias[k]
+        outs.append(z)
+        a = np.maximum(z, 0.0) if layer.relu_after else z
+    return np.concatenate(outs, axis=1)

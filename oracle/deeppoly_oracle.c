@@ -1,0 +1,352 @@
+/*
+ * DeepPoly oracle: TEST INFRASTRUCTURE, not the product.
+ *
+ * A plain, slow, float64 CPU implementation of the DeepPoly certifier as the
+ * paper's DeepPoly specification (Appendix C, listing "DeepPoly") defines it,
+ * neuron by neuron.  Only tests, the smoke check and the benchmark's CPU
+ * baseline leg may build or call this file.  It shares no code, header, table
+ * or helper with the CUDA library.
+ *
+ * What follows which passage (Appendix C, DeepPoly listing, unless noted):
+ *   - input box: the abstract shape of an input neuron is its concrete
+ *     interval [l,u] (Section 2, "Concrete Bounds"); an L-infinity ball of
+ *     radius eps around a centre, intersected with the clip range.
+ *   - Affine transformer: L = U = prev.dot(weight) + bias, and
+ *     l = backsubs_lower(L), u = backsubs_upper(U).
+ *   - backsubs_*: traverse backward, highest layer first (priority2 =
+ *     -layer), never stopping early (stop_traverse = false), replacing every
+ *     (neuron, coefficient) pair with replace_lower / replace_upper; then
+ *     map(simplify_lower / simplify_upper) against concrete bounds.
+ *   - replace_lower(n,c) = c >= 0 ? c*n[L] : c*n[U]   (upper: swapped)
+ *   - simplify_lower(n,c) = c >= 0 ? c*n[l] : c*n[u]  (upper: swapped)
+ *   - Relu transformer: l = relu(prev[l]), u = relu(prev[u]),
+ *     L = relu_n(prev) = (l+u >= 0 ? prev : 0),
+ *     U = compute_upper(prev) = l >= 0 ? prev
+ *                             : u <= 0 ? 0
+ *                             : u/(u-l) * prev - u*l/(u-l).
+ *
+ * Readings taken where the paper is silent:
+ *   - the traversal ends when the expression is over input neurons (they
+ *     have no L/U), and simplify_* then uses the box;
+ *   - ReLU and Affine are separate layers, so one traversal round replaces
+ *     all neurons of the highest remaining layer;
+ *   - a back-substituted bound is NOT intersected with any other bound;
+ *   - conv layers are cross-correlations with zero padding,
+ *     out = floor((in + 2*pad - k)/stride) + 1, flattened (c,h,w) row-major;
+ *   - the three sign tests of the Relu transformer are taken on l and u
+ *     rounded to binary32 and (for l+u) added in binary32 when
+ *     decision_fp32 != 0, so that exact ties resolve as in a binary32
+ *     implementation; with decision_fp32 == 0 they are taken in float64.
+ *     The slopes and intercepts are always computed in float64 from the
+ *     float64 l and u.
+ *
+ * Parity with the paper's own executables is unpinned (they are not
+ * available); the pins are the tests under tests/ marked "not gpu".
+ *
+ * Branch codes per hidden (ReLU) neuron:
+ *   0 = stable inactive (u <= 0), 1 = stable active (l >= 0),
+ *   2 = unstable with lower slope 0, 3 = unstable with lower slope 1.
+ */
+#include <math.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+typedef struct {
+    int kind;        /* 0 = fully connected, 1 = conv2d                       */
+    int relu_after;  /* 1 = a ReLU layer follows this affine layer            */
+    int in_features, out_features;              /* FC: weight [out][in]      */
+    int c_in, h_in, w_in, c_out, kh, kw, stride, pad; /* conv: [co][ci][kh][kw] */
+    const float *weight;
+    const float *bias;
+} oracle_layer_t;
+
+static int conv_out(int in, int k, int s, int p) { return (in + 2 * p - k) / s + 1; }
+
+static int layer_n_in(const oracle_layer_t *L)
+{
+    return L->kind == 0 ? L->in_features : L->c_in * L->h_in * L->w_in;
+}
+
+static int layer_n_out(const oracle_layer_t *L)
+{
+    if (L->kind == 0) return L->out_features;
+    return L->c_out * conv_out(L->h_in, L->kh, L->stride, L->pad) *
+           conv_out(L->w_in, L->kw, L->stride, L->pad);
+}
+
+/* The polyhedral expression of affine neuron i over the layer's inputs:
+ * coef = row i of the layer's linear map, *d = its bias
+ * ("prev.dot(curr[weight]) + curr[bias]").                                   */
+static void affine_row(const oracle_layer_t *L, int i, double *coef, double *d)
+{
+    int n_in = layer_n_in(L);
+    if (L->kind == 0) {
+        for (int s = 0; s < n_in; ++s) coef[s] = (double)L->weight[(size_t)i * n_in + s];
+    } else {
+        int ho = conv_out(L->h_in, L->kh, L->stride, L->pad);
+        int wo = conv_out(L->w_in, L->kw, L->stride, L->pad);
+        int co = i / (ho * wo), oy = (i / wo) % ho, ox = i % wo;
+        for (int s = 0; s < n_in; ++s) coef[s] = 0.0;
+        for (int ci = 0; ci < L->c_in; ++ci)
+            for (int ky = 0; ky < L->kh; ++ky)
+                for (int kx = 0; kx < L->kw; ++kx) {
+                    int iy = oy * L->stride - L->pad + ky;
+                    int ix = ox * L->stride - L->pad + kx;
+                    if (iy < 0 || iy >= L->h_in || ix < 0 || ix >= L->w_in) continue;
+                    coef[((size_t)ci * L->h_in + iy) * L->w_in + ix] =
+                        (double)L->weight[(((size_t)co * L->c_in + ci) * L->kh + ky) * L->kw + kx];
+                }
+        i = co;                                  /* one bias per output channel */
+    }
+    *d = (double)L->bias[i];
+}
+
+/* Replace every neuron t of affine layer L in the expression (coef over the
+ * layer's outputs) by its polyhedral bound.  For an affine neuron L = U =
+ * w.prev + b, so both branches of replace_* give coef[t]*(w_t.prev + b_t).   */
+static void replace_through_affine(const oracle_layer_t *L, const double *coef,
+                                   double *next, double *d)
+{
+    int n_in = layer_n_in(L), n_out = layer_n_out(L);
+    for (int s = 0; s < n_in; ++s) next[s] = 0.0;
+    if (L->kind == 0) {
+        for (int t = 0; t < n_out; ++t) {
+            double c = coef[t];
+            if (c == 0.0) continue;
+            const float *w = L->weight + (size_t)t * n_in;
+            for (int s = 0; s < n_in; ++s) next[s] += c * (double)w[s];
+            *d += c * (double)L->bias[t];
+        }
+    } else {
+        int ho = conv_out(L->h_in, L->kh, L->stride, L->pad);
+        int wo = conv_out(L->w_in, L->kw, L->stride, L->pad);
+        for (int t = 0; t < n_out; ++t) {
+            double c = coef[t];
+            if (c == 0.0) continue;
+            int co = t / (ho * wo), oy = (t / wo) % ho, ox = t % wo;
+            for (int ci = 0; ci < L->c_in; ++ci)
+                for (int ky = 0; ky < L->kh; ++ky)
+                    for (int kx = 0; kx < L->kw; ++kx) {
+                        int iy = oy * L->stride - L->pad + ky;
+                        int ix = ox * L->stride - L->pad + kx;
+                        if (iy < 0 || iy >= L->h_in || ix < 0 || ix >= L->w_in) continue;
+                        next[((size_t)ci * L->h_in + iy) * L->w_in + ix] +=
+                            c * (double)L->weight[(((size_t)co * L->c_in + ci) * L->kh + ky) * L->kw + kx];
+                    }
+            *d += c * (double)L->bias[co];
+        }
+    }
+}
+
+/* Replace every ReLU neuron t by its polyhedral bound over the affine neuron
+ * below it: L_t = lamL[t]*z_t, U_t = lamU[t]*z_t + nuU[t].
+ * upper == 0: replace_lower; upper == 1: replace_upper.                      */
+static void replace_through_relu(int n, int upper, const double *lamL, const double *lamU,
+                                 const double *nuU, double *coef, double *d)
+{
+    for (int t = 0; t < n; ++t) {
+        double c = coef[t];
+        int use_L = upper ? !(c >= 0.0) : (c >= 0.0);
+        if (use_L) {
+            coef[t] = c * lamL[t];
+        } else {
+            coef[t] = c * lamU[t];
+            *d += c * nuU[t];
+        }
+    }
+}
+
+/* simplify_lower / simplify_upper summed over the input neurons. */
+static double concretize(int n, int upper, const double *coef, double d,
+                         const double *l0, const double *u0)
+{
+    double acc = d;
+    for (int s = 0; s < n; ++s) {
+        double c = coef[s];
+        if (c >= 0.0) acc += c * (upper ? u0[s] : l0[s]);
+        else          acc += c * (upper ? l0[s] : u0[s]);
+    }
+    return acc;
+}
+
+/* The Relu transformer for one neuron with concrete bounds (l,u) of the
+ * affine neuron below it. */
+static void relu_relaxation(double l, double u, int decision_fp32, double *lamL, double *lamU,
+                            double *nuU, unsigned char *code, double *margin)
+{
+    int active, inactive, pick_one;
+    if (decision_fp32) {
+        float lf = (float)l, uf = (float)u;
+        volatile float sum = lf + uf;
+        active = lf >= 0.0f;
+        inactive = uf <= 0.0f;
+        pick_one = sum >= 0.0f;
+    } else {
+        active = l >= 0.0;
+        inactive = u <= 0.0;
+        pick_one = (l + u) >= 0.0;
+    }
+    *lamL = pick_one ? 1.0 : 0.0;                        /* relu_n          */
+    if (active)        { *lamU = 1.0; *nuU = 0.0; *code = 1; }   /* compute_upper */
+    else if (inactive) { *lamU = 0.0; *nuU = 0.0; *code = 0; }
+    else {
+        *lamU = u / (u - l);
+        *nuU = -(u * l) / (u - l);
+        *code = (unsigned char)(2 + pick_one);
+    }
+    double m = fabs(l);
+    if (fabs(u) < m) m = fabs(u);
+    if (fabs(l + u) < m) m = fabs(l + u);
+    double scale = fabs(l) > fabs(u) ? fabs(l) : fabs(u);
+    *margin = m / (1.0 + scale);
+}
+
+/* One box: bounds of every affine neuron, layer after layer
+ * (flow(forward, priority = layer)). */
+static int one_box(const oracle_layer_t *layers, int n_layers, const float *center, float eps,
+                   float clip_lo, float clip_hi, int decision_fp32, int max_backsteps,
+                   double *lb, double *ub, unsigned char *codes, double *margins)
+{
+    int n0 = layer_n_in(&layers[0]);
+    int n_max = n0, n_total = 0;
+    for (int k = 0; k < n_layers; ++k) {
+        int n = layer_n_out(&layers[k]);
+        if (n > n_max) n_max = n;
+        n_total += n;
+    }
+    double *l0 = malloc(sizeof(double) * n0), *u0 = malloc(sizeof(double) * n0);
+    double *coef = malloc(sizeof(double) * n_max), *next = malloc(sizeof(double) * n_max);
+    double *lamL = malloc(sizeof(double) * n_total), *lamU = malloc(sizeof(double) * n_total);
+    double *nuU = malloc(sizeof(double) * n_total);
+    int *off = malloc(sizeof(int) * (n_layers + 1));
+    if (!l0 || !u0 || !coef || !next || !lamL || !lamU || !nuU || !off) return 1;
+
+    /* The box endpoints are binary32 values: fl(c -/+ eps) clipped. */
+    for (int s = 0; s < n0; ++s) {
+        volatile float lo = center[s] - eps, hi = center[s] + eps;
+        float lo_c = lo < clip_lo ? clip_lo : lo;
+        float hi_c = hi > clip_hi ? clip_hi : hi;
+        l0[s] = (double)lo_c;
+        u0[s] = (double)hi_c;
+    }
+    off[0] = 0;
+    for (int k = 0; k < n_layers; ++k) off[k + 1] = off[k] + layer_n_out(&layers[k]);
+
+    int code_off = 0;
+    for (int k = 0; k < n_layers; ++k) {
+        int n_k = layer_n_out(&layers[k]);
+        for (int i = 0; i < n_k; ++i) {
+            for (int upper = 0; upper < 2; ++upper) {
+                double d;
+                affine_row(&layers[k], i, coef, &d);
+                int steps = 0;
+                int j = k - 1;                 /* coef is over the outputs of layer j */
+                for (; j >= 0; --j) {
+                    if (max_backsteps >= 0 && steps >= max_backsteps) break;
+                    if (layers[j].relu_after)
+                        replace_through_relu(layer_n_out(&layers[j]), upper, lamL + off[j],
+                                             lamU + off[j], nuU + off[j], coef, &d);
+                    replace_through_affine(&layers[j], coef, next, &d);
+                    double *tmp = coef; coef = next; next = tmp;
+                    ++steps;
+                }
+                double v;
+                if (j < 0) {
+                    v = concretize(n0, upper, coef, d, l0, u0);
+                } else {
+                    /* Stopped early (DeepPoly_p, Section 6.2): simplify against the
+                     * concrete bounds of the neurons reached: relu(l), relu(u) of
+                     * layer j when a ReLU follows it, else its own l, u. */
+                    int n_j = layer_n_out(&layers[j]);
+                    double *lj = next, *uj = malloc(sizeof(double) * n_j);
+                    if (!uj) return 1;
+                    for (int t = 0; t < n_j; ++t) {
+                        double l = lb[off[j] + t], u = ub[off[j] + t];
+                        if (layers[j].relu_after) { l = l >= 0.0 ? l : 0.0; u = u >= 0.0 ? u : 0.0; }
+                        lj[t] = l; uj[t] = u;
+                    }
+                    v = concretize(n_j, upper, coef, d, lj, uj);
+                    free(uj);
+                }
+                if (upper) ub[off[k] + i] = v; else lb[off[k] + i] = v;
+            }
+        }
+        if (layers[k].relu_after) {
+            for (int t = 0; t < n_k; ++t) {
+                unsigned char code; double margin;
+                relu_relaxation(lb[off[k] + t], ub[off[k] + t], decision_fp32, &lamL[off[k] + t],
+                                &lamU[off[k] + t], &nuU[off[k] + t], &code, &margin);
+                if (codes) codes[code_off + t] = code;
+                if (margins) margins[code_off + t] = margin;
+            }
+            code_off += n_k;
+        }
+    }
+    free(l0); free(u0); free(coef); free(next); free(lamL); free(lamU); free(nuU); free(off);
+    return 0;
+}
+
+/* Number of affine neurons (sum over layers) and of ReLU neurons. */
+int oracle_num_neurons(const oracle_layer_t *layers, int n_layers)
+{
+    int n = 0;
+    for (int k = 0; k < n_layers; ++k) n += layer_n_out(&layers[k]);
+    return n;
+}
+
+int oracle_num_relu_neurons(const oracle_layer_t *layers, int n_layers)
+{
+    int n = 0;
+    for (int k = 0; k < n_layers; ++k)
+        if (layers[k].relu_after) n += layer_n_out(&layers[k]);
+    return n;
+}
+
+/*
+ * lb, ub: [batch][n_total] float64, affine layers concatenated in order.
+ * codes, margins (optional, may be NULL): [batch][n_relu].
+ * max_backsteps < 0: full DeepPoly.  max_backsteps = p >= 0: DeepPoly_p.
+ * n_threads: boxes are independent and are the only parallel axis.
+ * Returns 0, or 1 on allocation failure, 2 on a malformed network.
+ */
+int oracle_deeppoly(const oracle_layer_t *layers, int n_layers, const float *centers, float eps,
+                    int batch, float clip_lo, float clip_hi, int decision_fp32, int max_backsteps,
+                    int n_threads, double *lb, double *ub, unsigned char *codes, double *margins)
+{
+    if (n_layers < 1 || batch < 0) return 2;
+    for (int k = 1; k < n_layers; ++k)
+        if (layer_n_in(&layers[k]) != layer_n_out(&layers[k - 1])) return 2;
+    int n0 = layer_n_in(&layers[0]);
+    int n_total = oracle_num_neurons(layers, n_layers);
+    int n_relu = oracle_num_relu_neurons(layers, n_layers);
+    int err = 0;
+#ifdef _OPENMP
+    if (n_threads > 0) omp_set_num_threads(n_threads);
+#else
+    (void)n_threads;
+#endif
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int b = 0; b < batch; ++b) {
+        int e = one_box(layers, n_layers, centers + (size_t)b * n0, eps, clip_lo, clip_hi,
+                        decision_fp32, max_backsteps, lb + (size_t)b * n_total,
+                        ub + (size_t)b * n_total, codes ? codes + (size_t)b * n_relu : NULL,
+                        margins ? margins + (size_t)b * n_relu : NULL);
+        if (e) {
+#pragma omp atomic write
+            err = e;
+        }
+    }
+    return err;
+}
+
+int oracle_max_threads(void)
+{
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
