@@ -1,0 +1,299 @@
+#!/usr/bin/env python
+"""Benchmark: input boxes/sec fully bounded by DeepPoly on B200.
+
+One step = one cert_deeppoly_bounds call over one batch of synthetic boxes
+(every layer's back-substitution, concretisation and relaxation).
+Prints one JSON line (rank 0).  `--impl reference` times the float64 CPU
+oracle on the host cores instead (a reported baseline, not a target).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+
+from paper_2507_20055_b200 import workloads as wl
+
+METRIC = "input boxes/sec fully bounded (DeepPoly)"
+UNIT = "boxes/s"
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return {"hbm_gbs": d["hbm_gbs"], "bf16_tflops": d["bf16_tflops"],
+                "bf16_tflops_sustained": d["bf16_tflops_sustained"], "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.rows, self.proc, self.gpu = [], None, gpu_index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-i", str(self.gpu), "-lms", "100"], stdout=subprocess.PIPE,
+                                         stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[1])); mx.append(float(r[2]))
+                for n, v in zip(names, r[5:9]):
+                    if v.lower().startswith("active"):
+                        reasons.add(n)
+            except Exception:
+                pass
+        # under load = the upper half of the samples
+        load = sorted(sm)[len(sm) // 2:] if sm else []
+        return {"sm_mhz": statistics.median(load) if load else None,
+                "sm_max_mhz": max(mx) if mx else None, "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def oracle_sample(w, n_boxes, threads=None):
+    """Times the oracle, as it stands, on the first n_boxes boxes of the workload."""
+    from oracle import deeppoly_oracle as orc
+    orc.build()
+    cores = threads or orc.max_threads()
+    c = w.centers[:n_boxes]
+    t0 = time.perf_counter()
+    orc.deeppoly(w.layers, c, w.eps, w.clip_lo, w.clip_hi, n_threads=cores)
+    dt = time.perf_counter() - t0
+    return {"value": n_boxes / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": f"first {n_boxes} of {w.batch} boxes of {w.name}, one box per thread, {dt:.1f} s wall"}, dt
+
+
+def run_reference(args, w):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import deeppoly_oracle as orc
+    orc.build()
+    cores = orc.max_threads()
+    per = {0: 1, 1: 4 * cores, 2: 2 * cores, 3: cores, 4: cores}
+    n_boxes = min(w.batch, args.ref_boxes or per[args.config])
+    if args.config == 4 and not args.ref_boxes:
+        n_boxes = max(1, min(cores, 16) // 2)     # about 11 s per box per core
+    times = []
+    for i in range(args.warmup + args.steps):
+        base, dt = oracle_sample(w, n_boxes)
+        if i >= args.warmup:
+            times.append(dt)
+    ms = 1000.0 * sum(times) / len(times)
+    val = n_boxes / (ms / 1000.0)
+    base["value"] = val
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "boxes_per_step": n_boxes, "eps": w.eps,
+                   "note": "each step bounds a sample of the workload's boxes on the host cores"},
+        "cpu_baseline": base,
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", type=int, default=4, help="0..4: index into the benchmark configurations")
+    ap.add_argument("--batch", type=int, default=None)
+    ap.add_argument("--contraction", default="auto", choices=["auto", "ffma", "tc"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--ref-boxes", type=int, default=None)
+    args = ap.parse_args()
+
+    w = wl.make_config(args.config, batch=args.batch)
+    if args.impl == "reference":
+        run_reference(args, w)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2507_20055_b200 import build
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if args.warmup < 3:
+        args.warmup = 3
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    if rank == 0:
+        build.build()
+    if world > 1:
+        dist.barrier()
+    from paper_2507_20055_b200 import binding
+
+    # Boxes are independent: each rank bounds its own batch of the same shape (weak scaling),
+    # with its own seed; the weights are replicated.  No collective on the data path.
+    if world > 1:
+        w = wl.make_config(args.config, batch=args.batch)
+        w.centers = wl.centers_uniform(w.batch, w.centers.shape[1], seed=0, stream=1000 + rank)
+    B = w.batch
+    net = binding.CertNet(w.layers, B, w.clip_lo, w.clip_hi)
+    mode = {"auto": binding.CONTRACTION_AUTO, "ffma": binding.CONTRACTION_FFMA, "tc": binding.CONTRACTION_TC3XTF32}
+    net.set_contraction(mode[args.contraction])
+    stream = torch.cuda.Stream()
+    centers = torch.from_numpy(w.centers).cuda()
+    lb = torch.empty((B, net.n_total), dtype=torch.float32, device="cuda")
+    ub = torch.empty_like(lb)
+    flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device="cuda")   # > 126 MB L2
+    torch.cuda.synchronize()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def step_device():
+        net.deeppoly_bounds(centers, w.eps, lb, ub, stream=stream)
+
+    # ---- device-resident timing: K steps, each bracketed by events on the launching stream,
+    #      L2 flushed between steps outside the bracket ----
+    with torch.cuda.stream(stream):
+        for _ in range(args.warmup):
+            step_device()
+    barrier()
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    barrier()
+    t_wall0 = time.perf_counter()
+    with torch.cuda.stream(stream):
+        for i in range(args.steps):
+            flush.fill_(i & 0xFF)
+            evs[i][0].record(stream)
+            step_device()
+            evs[i][1].record(stream)
+    barrier()
+    t_wall = time.perf_counter() - t_wall0
+    step_ms = [a.elapsed_time(b) for a, b in evs]
+    total_ms = sum(step_ms)
+    launches = net.last_launch_count() * args.steps
+    assert net.last_status(stream.cuda_stream) == 0, "device-side status is not OK"
+
+    # ---- per-kernel-class times over the same K steps (events inside the library) ----
+    net.set_profiling(True)
+    cls_ms, cls_n = {}, {}
+    with torch.cuda.stream(stream):
+        for i in range(args.steps):
+            flush.fill_(i & 0xFF)
+            step_device()
+            stream.synchronize()
+            for name, (ms, n) in net.profile().items():
+                cls_ms[name] = cls_ms.get(name, 0.0) + ms
+                cls_n[name] = cls_n.get(name, 0) + n
+    net.set_profiling(False)
+    clocks = sampler.stop() if rank == 0 else None
+
+    # ---- end to end through the host-buffer entry point (pinned buffers, copies timed) ----
+    centers_pin = torch.from_numpy(w.centers).pin_memory()
+    lb_pin = torch.empty((B, net.n_total), dtype=torch.float32).pin_memory()
+    ub_pin = torch.empty((B, net.n_total), dtype=torch.float32).pin_memory()
+    c_np, lb_np, ub_np = centers_pin.numpy(), lb_pin.numpy(), ub_pin.numpy()
+    for _ in range(2):
+        net.deeppoly_bounds_host(c_np, w.eps, lb_np, ub_np, stream.cuda_stream)
+    barrier()
+    e2e_steps = max(3, min(args.steps, 10))
+    t0 = time.perf_counter()
+    for _ in range(e2e_steps):
+        net.deeppoly_bounds_host(c_np, w.eps, lb_np, ub_np, stream.cuda_stream)   # returns after the D2H copy
+    torch.cuda.synchronize()
+    e2e_s = time.perf_counter() - t0
+
+    # ---- max over ranks ----
+    t = torch.tensor([total_ms, e2e_s * 1000.0], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    total_ms_max, e2e_ms_max = float(t[0]), float(t[1])
+    value = world * B * args.steps / (total_ms_max / 1000.0)
+    e2e_value = world * B * e2e_steps / (e2e_ms_max / 1000.0)
+
+    if rank == 0:
+        peaks = load_peaks()
+        flops_call = net.backstep_flops(B)
+        con_ms = cls_ms.get("affine", 0.0) + cls_ms.get("conv", 0.0)
+        con_n = cls_n.get("affine", 0) + cls_n.get("conv", 0)
+        dom = "affine" if cls_ms.get("affine", 0.0) >= cls_ms.get("conv", 0.0) else "conv"
+        achieved = flops_call * args.steps / (con_ms / 1000.0) / 1e12 if con_ms > 0 else None
+        sm_max = (clocks or {}).get("sm_max_mhz") or 1965.0
+        ffma_peak = 148 * 128 * 2 * sm_max * 1e6 / 1e12
+        # fp32-accurate work on the tensor cores costs three TF32 products per multiply-add;
+        # TF32 dense peak = measured bf16 (sustained: the kernel runs inside a long step) x 1/2 (nominal ratio)
+        tc_peak = peaks["bf16_tflops_sustained"] * 0.5 / 3.0
+        used_tc = bool(net.last_contraction_paths() & 2)
+        roof = {"bound": "tensor" if used_tc else "alu",
+                "achieved": achieved, "peak": tc_peak if used_tc else ffma_peak, "unit": "TFLOP/s",
+                "frac": (achieved / (tc_peak if used_tc else ffma_peak)) if achieved else None,
+                "traffic": None,
+                "kernel": dom + " back-step", "launches_per_step": con_n // max(1, args.steps),
+                "avg_launch_ms": con_ms / con_n if con_n else None,
+                "flops_per_step": flops_call, "peak_source": peaks["source"],
+                "peak_note": ("bf16_tflops_sustained/2/3 (3xTF32)" if used_tc else "148 SM x 128 FMA x 2 x sm_max_mhz"),
+                "class_ms_per_step": {k: v / args.steps for k, v in cls_ms.items()}}
+        out = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": total_ms_max / args.steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": w.name, "boxes_per_gpu": B, "eps": w.eps,
+                       "net": "->".join(str(x) for x in [w.layers[0].n_in] + [l.n_out for l in w.layers]),
+                       "contraction": args.contraction, "parallelism": f"replicas over boxes x{world}",
+                       "l2": "256 MiB flush write between timed steps; per-step coefficient traffic exceeds L2"},
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(B * net.n0 * 4),
+                    "d2h_bytes_per_step": int(2 * B * net.n_total * 4), "steps": e2e_steps},
+            "gpu_launches": launches, "wall_s_timed_region": t_wall, "roofline": roof, "clocks": clocks,
+        }
+        if world == 1 and not args.no_cpu_baseline:
+            n_boxes = {0: 1, 1: 64, 2: 32, 3: 16, 4: 16}[args.config]
+            from oracle import deeppoly_oracle as orc
+            orc.build()
+            n_boxes = min(n_boxes, B) if args.config != 4 else min(B, orc.max_threads(), 16)
+            out["cpu_baseline"], _ = oracle_sample(w, n_boxes)
+        print(json.dumps(out))
+    net.destroy()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,163 @@
+/*
+ * cert.h - C ABI of the B200 DeepPoly back-substitution library.
+ *
+ * The calls follow the paper's problem statement (Section 2, "DNN
+ * Certification"): a ReLU network, a set of input regions given as concrete
+ * per-neuron bounds, and an abstract shape (here the concrete bounds l, u)
+ * out for every neuron, computed by the DeepPoly certifier (Appendix C,
+ * DeepPoly listing): polyhedral back-substitution at every affine layer
+ * (traverse + replace_lower/upper), concretisation against the input box
+ * (map(simplify_lower/upper)), and the ReLU relaxation chosen from the
+ * resulting bounds (Relu transformer: relu_n, compute_upper).
+ *
+ * All compute runs in CUDA kernels for sm_100a on the current device; there
+ * is no CPU fallback.  No function throws, aborts or traps: every failure is
+ * a return code.
+ */
+#ifndef CERT_H_
+#define CERT_H_
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct cert_net cert_net_t; /* opaque; owns device copies of the weights and a workspace */
+
+typedef enum {
+    CERT_OK = 0,
+    CERT_ERR_INVALID_ARG = 1,     /* null pointer, bad size, non-finite eps, layer chain mismatch */
+    CERT_ERR_UNSUPPORTED = 2,     /* a geometry the kernels do not cover                         */
+    CERT_ERR_OOM = 3,             /* device or host allocation failed                            */
+    CERT_ERR_BATCH_TOO_LARGE = 4, /* batch > max_batch given at create                           */
+    CERT_ERR_CUDA = 5,            /* a CUDA runtime or driver call failed                        */
+    CERT_ERR_TIMEOUT = 6          /* a bounded device-side wait ran out (see cert_net_last_status) */
+} cert_status_t;
+
+enum { CERT_LAYER_FC = 0, CERT_LAYER_CONV2D = 1 };
+
+/*
+ * One affine layer of the network, optionally followed by a ReLU layer
+ * (the paper treats Affine and Relu as separate layers; relu_after = 1 means
+ * a Relu layer sits on top of this affine layer).
+ *   FC:     z = W a + b, weight[out_features][in_features] row-major.
+ *   CONV2D: cross-correlation with zero padding on an input of shape
+ *           (c_in, h_in, w_in), weight[c_out][c_in][kh][kw], one bias per
+ *           output channel, output size floor((in + 2*pad - k)/stride) + 1;
+ *           neurons are flattened (channel, row, column) row-major.
+ * weight and bias are HOST pointers to float32; they are copied during
+ * cert_net_create and may be freed afterwards.
+ */
+typedef struct {
+    int kind;       /* CERT_LAYER_FC or CERT_LAYER_CONV2D */
+    int relu_after; /* 0 or 1 */
+    int in_features, out_features;                    /* FC only   */
+    int c_in, h_in, w_in, c_out, kh, kw, stride, pad; /* CONV only */
+    const float *weight;
+    const float *bias;
+} cert_layer_desc_t;
+
+/*
+ * Builds a network object on the current CUDA device: validates the
+ * descriptors, uploads the weights (and the operand forms the contraction
+ * kernels want), and allocates a workspace large enough for max_batch boxes.
+ * Input boxes are intersected with [clip_lo, clip_hi] (pass -INFINITY and
+ * INFINITY for no clipping).  On success *out receives the handle, which the
+ * caller releases with cert_net_destroy.  Synchronous.
+ */
+cert_status_t cert_net_create(const cert_layer_desc_t *layers, int n_layers, int max_batch,
+                              float clip_lo, float clip_hi, cert_net_t **out);
+
+/*
+ * DeepPoly bounds of every affine neuron for `batch` L-infinity boxes.
+ *   centers  DEVICE float32 [batch][n0]; box b is
+ *            [max(c - eps, clip_lo), min(c + eps, clip_hi)] per coordinate,
+ *            with c -/+ eps rounded to float32.
+ *   lb_out, ub_out  DEVICE float32 [batch][n_total], n_total =
+ *            cert_net_num_neurons(): the pre-activation neurons of affine
+ *            layer 1, 2, ... K concatenated in order.  (The bounds of a Relu
+ *            layer's neurons are max(l,0), max(u,0) of the layer below and
+ *            are not stored.)
+ *   stream   a cudaStream_t (NULL = the default stream).
+ * The work is enqueued on `stream` and the call returns without waiting; it
+ * allocates nothing.  Calls on the same net must not overlap on the device
+ * (they share the workspace).  Caller owns centers, lb_out and ub_out.
+ */
+cert_status_t cert_deeppoly_bounds(cert_net_t *net, const float *centers, float eps, int batch,
+                                   float *lb_out, float *ub_out, void *stream);
+
+/* Same, with HOST buffers (pageable or pinned): copies centers to the device,
+ * runs cert_deeppoly_bounds, copies the bounds back and waits for the stream. */
+cert_status_t cert_deeppoly_bounds_host(cert_net_t *net, const float *centers_host, float eps,
+                                        int batch, float *lb_host, float *ub_host, void *stream);
+
+/* Frees the device and host memory of the net.  Synchronises the device. */
+cert_status_t cert_net_destroy(cert_net_t *net);
+
+/* ---- helpers (not part of the paper's problem statement) ---- */
+
+/* n_total: number of affine neurons, summed over layers; -1 for a null net. */
+int cert_net_num_neurons(const cert_net_t *net);
+/* Number of neurons of affine layers that have a ReLU on top; -1 for null. */
+int cert_net_num_relu_neurons(const cert_net_t *net);
+
+/*
+ * Relaxation branch of every ReLU neuron in the most recent
+ * cert_deeppoly_bounds call (Relu transformer of the DeepPoly listing):
+ *   0 stable inactive (u <= 0), 1 stable active (l >= 0),
+ *   2 unstable with lower slope 0 (l + u < 0), 3 unstable with lower slope 1.
+ * codes_out: DEVICE uint8 [batch][n_relu], ReLU layers concatenated in
+ * order; copied on `stream`.
+ */
+cert_status_t cert_net_branch_codes(cert_net_t *net, unsigned char *codes_out, void *stream);
+
+/*
+ * Sticky device-side status.  Waits `stream`, then returns CERT_ERR_TIMEOUT
+ * if any kernel of an earlier call on this net gave up a bounded wait (its
+ * results are then invalid), CERT_ERR_CUDA if the stream reports an error,
+ * else CERT_OK.  Clears the flag.
+ */
+cert_status_t cert_net_last_status(cert_net_t *net, void *stream);
+
+/*
+ * Which kernel carries the affine back-step C' = C * W (Section 4.3, Matmul
+ * rewrite).  AUTO picks the tensor-core path where the shape allows it.
+ *   FFMA:    fp32 FMA units, unfused ReLU step and concretisation kernels.
+ *   TC3XTF32: tcgen05 tensor cores with a 3-term TF32 split (fp32-accurate),
+ *            ReLU back-step and concretisation fused into the epilogue.
+ */
+enum { CERT_CONTRACTION_AUTO = 0, CERT_CONTRACTION_FFMA = 1, CERT_CONTRACTION_TC3XTF32 = 2 };
+cert_status_t cert_net_set_contraction(cert_net_t *net, int mode);
+/* Which contraction kernels the most recent call ran: bit 0 = FFMA, bit 1 = TC3XTF32. */
+int cert_net_last_contraction_paths(const cert_net_t *net);
+
+/*
+ * Per-kernel-class device times.  With profiling on, cert_deeppoly_bounds
+ * records a CUDA event on `stream` after every launch (the events are created
+ * by cert_net_set_profiling, not in the hot call).  cert_net_profile waits for
+ * the most recent call and returns, per class, the summed time in ms between
+ * consecutive events and the number of launches.  Classes follow the steps of
+ * the DeepPoly listing: building the box and the first layer's bounds, the
+ * Relu transformer, replace_* through a ReLU layer (and the start of a
+ * traversal), replace_* through an FC layer, through a conv layer, and
+ * map(simplify_*).  Kernels that fuse steps count under the contraction.
+ */
+enum { CERT_CLASS_INPUT = 0, CERT_CLASS_RELAX = 1, CERT_CLASS_RELU_STEP = 2, CERT_CLASS_AFFINE = 3,
+       CERT_CLASS_CONV = 4, CERT_CLASS_CONCRETIZE = 5, CERT_N_CLASSES = 6 };
+cert_status_t cert_net_set_profiling(cert_net_t *net, int on);
+cert_status_t cert_net_profile(cert_net_t *net, float *ms_out /* HOST [CERT_N_CLASSES] */,
+                               int *launches_out /* HOST [CERT_N_CLASSES] */);
+
+/* Number of kernels the most recent cert_deeppoly_bounds call enqueued. */
+int cert_net_last_launch_count(const cert_net_t *net);
+
+/* Floating-point operations of the affine/conv back-steps of one call for
+ * `batch` boxes (2 per multiply-add, both bound sides, dense coefficient
+ * maps), as the benchmark's roofline numerator. */
+double cert_net_backstep_flops(const cert_net_t *net, int batch);
+
+const char *cert_status_string(cert_status_t s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CERT_H_ */

@@ -1,0 +1,213 @@
+"""Thin ctypes binding of libcert_b200.so (argument marshalling only).
+
+Every step of the path runs in the library's CUDA kernels.  PyTorch is used
+for device memory and streams.  There is no CPU fallback: if the library is
+missing or cannot be loaded, import of this module raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Sequence
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libcert_b200.so")
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError(
+        f"{LIB_PATH} is missing: build it with `python -m paper_2507_20055_b200.build` "
+        "(nvcc, sm_100a); there is no CPU fallback")
+
+_lib = ctypes.CDLL(LIB_PATH)
+
+CERT_OK = 0
+CONTRACTION_AUTO, CONTRACTION_FFMA, CONTRACTION_TC3XTF32 = 0, 1, 2
+
+EXPORTS = [
+    "cert_net_create", "cert_deeppoly_bounds", "cert_deeppoly_bounds_host", "cert_net_destroy",
+    "cert_net_num_neurons", "cert_net_num_relu_neurons", "cert_net_branch_codes",
+    "cert_net_last_status", "cert_net_set_contraction", "cert_net_last_launch_count",
+    "cert_net_backstep_flops", "cert_status_string", "cert_net_set_profiling", "cert_net_profile",
+    "cert_net_last_contraction_paths",
+]
+CLASS_NAMES = ["input", "relax", "relu_step", "affine", "conv", "concretize"]
+
+
+class cert_layer_desc_t(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int) for n in
+                ("kind", "relu_after", "in_features", "out_features",
+                 "c_in", "h_in", "w_in", "c_out", "kh", "kw", "stride", "pad")] + \
+               [("weight", ctypes.c_void_p), ("bias", ctypes.c_void_p)]
+
+
+_vp, _i, _f = ctypes.c_void_p, ctypes.c_int, ctypes.c_float
+_lib.cert_net_create.argtypes = [ctypes.POINTER(cert_layer_desc_t), _i, _i, _f, _f, ctypes.POINTER(_vp)]
+_lib.cert_net_create.restype = _i
+_lib.cert_deeppoly_bounds.argtypes = [_vp, _vp, _f, _i, _vp, _vp, _vp]
+_lib.cert_deeppoly_bounds.restype = _i
+_lib.cert_deeppoly_bounds_host.argtypes = [_vp, _vp, _f, _i, _vp, _vp, _vp]
+_lib.cert_deeppoly_bounds_host.restype = _i
+_lib.cert_net_destroy.argtypes = [_vp]
+_lib.cert_net_destroy.restype = _i
+_lib.cert_net_num_neurons.argtypes = [_vp]
+_lib.cert_net_num_neurons.restype = _i
+_lib.cert_net_num_relu_neurons.argtypes = [_vp]
+_lib.cert_net_num_relu_neurons.restype = _i
+_lib.cert_net_branch_codes.argtypes = [_vp, _vp, _vp]
+_lib.cert_net_branch_codes.restype = _i
+_lib.cert_net_last_status.argtypes = [_vp, _vp]
+_lib.cert_net_last_status.restype = _i
+_lib.cert_net_set_contraction.argtypes = [_vp, _i]
+_lib.cert_net_set_contraction.restype = _i
+_lib.cert_net_last_launch_count.argtypes = [_vp]
+_lib.cert_net_last_launch_count.restype = _i
+_lib.cert_net_backstep_flops.argtypes = [_vp, _i]
+_lib.cert_net_backstep_flops.restype = ctypes.c_double
+_lib.cert_net_last_contraction_paths.argtypes = [_vp]
+_lib.cert_net_last_contraction_paths.restype = _i
+_lib.cert_net_set_profiling.argtypes = [_vp, _i]
+_lib.cert_net_set_profiling.restype = _i
+_lib.cert_net_profile.argtypes = [_vp, _vp, _vp]
+_lib.cert_net_profile.restype = _i
+_lib.cert_status_string.argtypes = [_i]
+_lib.cert_status_string.restype = ctypes.c_char_p
+
+
+class CertError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {_lib.cert_status_string(code).decode()} (status {code})")
+
+
+def _check(code: int, where: str):
+    if code != CERT_OK:
+        raise CertError(code, where)
+
+
+def marshal_layers(layers: Sequence):
+    """ctypes array of cert_layer_desc_t from objects with kind/weight/bias/relu_after(/stride/pad/in_shape)."""
+    arr = (cert_layer_desc_t * len(layers))()
+    keep = []
+    for i, l in enumerate(layers):
+        w = np.ascontiguousarray(l.weight, dtype=np.float32)
+        b = np.ascontiguousarray(l.bias, dtype=np.float32)
+        keep += [w, b]
+        d = arr[i]
+        d.relu_after = int(bool(l.relu_after))
+        d.weight, d.bias = w.ctypes.data, b.ctypes.data
+        if l.kind == "fc":
+            d.kind = 0
+            d.out_features, d.in_features = w.shape
+        elif l.kind == "conv":
+            d.kind = 1
+            d.c_out, d.c_in, d.kh, d.kw = w.shape
+            _, d.h_in, d.w_in = l.in_shape
+            d.stride, d.pad = int(l.stride), int(l.pad)
+        else:
+            raise ValueError(f"unknown layer kind {l.kind!r}")
+    return arr, keep
+
+
+class CertNet:
+    """Owns a cert_net_t handle; the three calls of the C ABI plus the helpers."""
+
+    def __init__(self, layers: Sequence, max_batch: int, clip_lo: float = 0.0, clip_hi: float = 1.0):
+        arr, keep = marshal_layers(layers)
+        h = _vp()
+        _check(_lib.cert_net_create(arr, len(layers), int(max_batch), float(clip_lo), float(clip_hi),
+                                    ctypes.byref(h)), "cert_net_create")
+        self._h = h
+        self.max_batch = int(max_batch)
+        self.n0 = int(layers[0].n_in)
+        self.n_total = int(_lib.cert_net_num_neurons(h))
+        self.n_relu = int(_lib.cert_net_num_relu_neurons(h))
+
+    # -- raw-pointer form (what the C ABI takes) --
+    def deeppoly_bounds_ptr(self, centers_ptr: int, eps: float, batch: int, lb_ptr: int, ub_ptr: int,
+                            stream_ptr: int = 0):
+        _check(_lib.cert_deeppoly_bounds(self._h, centers_ptr, float(eps), int(batch), lb_ptr, ub_ptr,
+                                         stream_ptr), "cert_deeppoly_bounds")
+
+    # -- torch tensors on the device --
+    def deeppoly_bounds(self, centers, eps: float, lb_out=None, ub_out=None, stream=None):
+        import torch
+        assert centers.is_cuda and centers.dtype == torch.float32 and centers.is_contiguous()
+        batch = centers.shape[0]
+        assert centers.shape[1] == self.n0
+        if lb_out is None:
+            lb_out = torch.empty((batch, self.n_total), dtype=torch.float32, device=centers.device)
+        if ub_out is None:
+            ub_out = torch.empty((batch, self.n_total), dtype=torch.float32, device=centers.device)
+        st = stream if stream is not None else torch.cuda.current_stream(centers.device)
+        self.deeppoly_bounds_ptr(centers.data_ptr(), eps, batch, lb_out.data_ptr(), ub_out.data_ptr(),
+                                 st.cuda_stream)
+        return lb_out, ub_out
+
+    # -- host numpy arrays (copies inside the library) --
+    def deeppoly_bounds_host(self, centers: np.ndarray, eps: float, lb: Optional[np.ndarray] = None,
+                             ub: Optional[np.ndarray] = None, stream_ptr: int = 0):
+        centers = np.ascontiguousarray(centers, dtype=np.float32)
+        batch = centers.shape[0]
+        if lb is None:
+            lb = np.empty((batch, self.n_total), dtype=np.float32)
+        if ub is None:
+            ub = np.empty((batch, self.n_total), dtype=np.float32)
+        _check(_lib.cert_deeppoly_bounds_host(self._h, centers.ctypes.data, float(eps), batch,
+                                              lb.ctypes.data, ub.ctypes.data, stream_ptr),
+               "cert_deeppoly_bounds_host")
+        return lb, ub
+
+    def set_profiling(self, on: bool):
+        _check(_lib.cert_net_set_profiling(self._h, int(bool(on))), "cert_net_set_profiling")
+
+    def profile(self):
+        """dict class name -> (ms, launches) of the most recent call (profiling must be on)."""
+        ms = (ctypes.c_float * len(CLASS_NAMES))()
+        cnt = (ctypes.c_int * len(CLASS_NAMES))()
+        _check(_lib.cert_net_profile(self._h, ctypes.addressof(ms), ctypes.addressof(cnt)), "cert_net_profile")
+        return {n: (float(ms[i]), int(cnt[i])) for i, n in enumerate(CLASS_NAMES)}
+
+    def branch_codes(self, batch: int, stream=None):
+        import torch
+        if self.n_relu == 0:
+            return torch.empty((batch, 0), dtype=torch.uint8, device="cuda")
+        codes = torch.empty((batch, self.n_relu), dtype=torch.uint8, device="cuda")
+        st = stream if stream is not None else torch.cuda.current_stream()
+        _check(_lib.cert_net_branch_codes(self._h, codes.data_ptr(), st.cuda_stream), "cert_net_branch_codes")
+        return codes
+
+    def last_status(self, stream_ptr: int = 0) -> int:
+        return int(_lib.cert_net_last_status(self._h, stream_ptr))
+
+    def set_contraction(self, mode: int):
+        _check(_lib.cert_net_set_contraction(self._h, int(mode)), "cert_net_set_contraction")
+
+    def last_contraction_paths(self) -> int:
+        return int(_lib.cert_net_last_contraction_paths(self._h))
+
+    def last_launch_count(self) -> int:
+        return int(_lib.cert_net_last_launch_count(self._h))
+
+    def backstep_flops(self, batch: int) -> float:
+        return float(_lib.cert_net_backstep_flops(self._h, int(batch)))
+
+    def destroy(self):
+        if getattr(self, "_h", None):
+            _check(_lib.cert_net_destroy(self._h), "cert_net_destroy")
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass
+
+
+# C-ABI names, as plain functions
+cert_net_create = _lib.cert_net_create
+cert_deeppoly_bounds = _lib.cert_deeppoly_bounds
+cert_deeppoly_bounds_host = _lib.cert_deeppoly_bounds_host
+cert_net_destroy = _lib.cert_net_destroy
+lib = _lib

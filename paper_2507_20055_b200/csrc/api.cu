@@ -1,0 +1,475 @@
+// C ABI of the library: network object, workspace, and the per-call schedule
+// of kernel launches that realises the DeepPoly flow (Appendix C, DeepPoly
+// listing): flow(forward) over layers; at each affine layer a traversal
+// backward through every earlier layer; concretisation at the input; then
+// the Relu transformer picks the relaxation used by later traversals.
+#include <cmath>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "common.cuh"
+
+struct cert_net {
+    int n_layers = 0, max_batch = 0;
+    float clip_lo = 0, clip_hi = 0;
+    int n0 = 0, ld0 = 0, n_total = 0, n_relu = 0;
+    int device = 0;
+    int contraction = CERT_CONTRACTION_AUTO;
+    std::vector<cert::LayerDev> layers;
+    std::vector<void *> allocs;   // every device allocation, for destroy
+    float *l0 = nullptr, *u0 = nullptr;      // [max_batch][ld0]
+    float *buf[2] = {nullptr, nullptr};      // ping-pong coefficient matrices
+    float *d = nullptr;                      // [max rows] constants of the expressions
+    unsigned char *codes = nullptr;          // [max_batch][n_relu]
+    int *status_dev = nullptr;               // sticky device status word
+    // host staging for cert_deeppoly_bounds_host
+    float *centers_dev = nullptr, *lb_dev = nullptr, *ub_dev = nullptr;
+    int last_batch = 0;
+    int last_launches = 0;
+    int last_paths = 0;              // bit 0: an FFMA contraction ran, bit 1: a tensor-core one
+    // optional per-launch event timing (events are created when profiling is switched on)
+    bool profiling = false;
+    std::vector<cudaEvent_t> prof_events;
+    std::vector<int> prof_class;   // class of the launch between event i and i+1
+    int prof_marks = 0;
+};
+
+namespace cert {
+size_t convt_smem_bytes(const LayerDev &L);
+void convt_prepare();
+}  // namespace cert
+
+namespace {
+
+using cert::LayerDev;
+using cert::kPad;
+using cert::round_up;
+
+bool dev_alloc(cert_net *net, void **p, size_t bytes) {
+    if (bytes == 0) bytes = 256;
+    if (cudaMalloc(p, bytes) != cudaSuccess) {
+        cudaGetLastError();
+        *p = nullptr;
+        return false;
+    }
+    net->allocs.push_back(*p);
+    return true;
+}
+
+template <typename T>
+bool dev_alloc_zero(cert_net *net, T **p, size_t count) {
+    if (!dev_alloc(net, reinterpret_cast<void **>(p), count * sizeof(T))) return false;
+    return cudaMemset(*p, 0, (count ? count : 1) * sizeof(T)) == cudaSuccess;
+}
+
+void free_net(cert_net *net) {
+    if (!net) return;
+    for (cudaEvent_t e : net->prof_events) cudaEventDestroy(e);
+    for (void *p : net->allocs) cudaFree(p);
+    delete net;
+}
+
+cert_status_t validate(const cert_layer_desc_t *layers, int n_layers, int max_batch, float clip_lo,
+                       float clip_hi) {
+    if (!layers || n_layers < 1 || max_batch < 1) return CERT_ERR_INVALID_ARG;
+    if (std::isnan(clip_lo) || std::isnan(clip_hi) || clip_lo > clip_hi) return CERT_ERR_INVALID_ARG;
+    long long prev_out = -1;
+    for (int k = 0; k < n_layers; ++k) {
+        const cert_layer_desc_t &L = layers[k];
+        if (!L.weight || !L.bias) return CERT_ERR_INVALID_ARG;
+        if (L.relu_after != 0 && L.relu_after != 1) return CERT_ERR_INVALID_ARG;
+        long long n_in, n_out;
+        if (L.kind == CERT_LAYER_FC) {
+            if (L.in_features < 1 || L.out_features < 1) return CERT_ERR_INVALID_ARG;
+            n_in = L.in_features;
+            n_out = L.out_features;
+        } else if (L.kind == CERT_LAYER_CONV2D) {
+            if (L.c_in < 1 || L.h_in < 1 || L.w_in < 1 || L.c_out < 1 || L.kh < 1 || L.kw < 1 ||
+                L.stride < 1 || L.pad < 0)
+                return CERT_ERR_INVALID_ARG;
+            if (L.h_in + 2 * L.pad < L.kh || L.w_in + 2 * L.pad < L.kw) return CERT_ERR_INVALID_ARG;
+            int ho = (L.h_in + 2 * L.pad - L.kh) / L.stride + 1, wo = (L.w_in + 2 * L.pad - L.kw) / L.stride + 1;
+            n_in = (long long)L.c_in * L.h_in * L.w_in;
+            n_out = (long long)L.c_out * ho * wo;
+        } else {
+            return CERT_ERR_INVALID_ARG;
+        }
+        if (n_in > (1 << 20) || n_out > (1 << 20)) return CERT_ERR_UNSUPPORTED;
+        if (prev_out >= 0 && n_in != prev_out) return CERT_ERR_INVALID_ARG;
+        prev_out = n_out;
+    }
+    return CERT_OK;
+}
+
+// Counts launches; with profiling on, drops an event after each so that the
+// time between consecutive events is that launch's device time.
+struct Recorder {
+    cert_net *net;
+    cudaStream_t st;
+    int launches = 0, marks = 0;
+    Recorder(cert_net *n, cudaStream_t s) : net(n), st(s) {
+        if (net->profiling && !net->prof_events.empty()) cudaEventRecord(net->prof_events[0], st);
+    }
+    void mark(int cls) {
+        ++launches;
+        if (!net->profiling) return;
+        if (marks + 1 >= (int)net->prof_events.size()) return;
+        net->prof_class[marks] = cls;
+        ++marks;
+        cudaEventRecord(net->prof_events[marks], st);
+    }
+};
+
+}  // namespace
+
+extern "C" {
+
+const char *cert_status_string(cert_status_t s) {
+    switch (s) {
+        case CERT_OK: return "ok";
+        case CERT_ERR_INVALID_ARG: return "invalid argument";
+        case CERT_ERR_UNSUPPORTED: return "unsupported";
+        case CERT_ERR_OOM: return "out of memory";
+        case CERT_ERR_BATCH_TOO_LARGE: return "batch larger than max_batch";
+        case CERT_ERR_CUDA: return "CUDA error";
+        case CERT_ERR_TIMEOUT: return "device-side wait timed out";
+    }
+    return "unknown";
+}
+
+cert_status_t cert_net_create(const cert_layer_desc_t *layers, int n_layers, int max_batch, float clip_lo,
+                              float clip_hi, cert_net_t **out) {
+    if (!out) return CERT_ERR_INVALID_ARG;
+    *out = nullptr;
+    cert_status_t v = validate(layers, n_layers, max_batch, clip_lo, clip_hi);
+    if (v != CERT_OK) return v;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return CERT_ERR_CUDA; }
+
+    cert_net *net = new (std::nothrow) cert_net;
+    if (!net) return CERT_ERR_OOM;
+    net->device = dev;
+    net->n_layers = n_layers;
+    net->max_batch = max_batch;
+    net->clip_lo = clip_lo;
+    net->clip_hi = clip_hi;
+    net->layers.resize(n_layers);
+
+    cert_status_t fail = CERT_OK;
+    int out_off = 0, relu_off = 0;
+    std::vector<float> host;
+    for (int k = 0; k < n_layers && fail == CERT_OK; ++k) {
+        const cert_layer_desc_t &D = layers[k];
+        LayerDev &L = net->layers[k];
+        std::memset(&L, 0, sizeof(L));
+        L.kind = D.kind;
+        L.relu_after = D.relu_after;
+        if (D.kind == CERT_LAYER_FC) {
+            L.n_in = D.in_features;
+            L.n_out = D.out_features;
+        } else {
+            L.c_in = D.c_in; L.h_in = D.h_in; L.w_in = D.w_in; L.c_out = D.c_out;
+            L.kh = D.kh; L.kw = D.kw; L.stride = D.stride; L.pad = D.pad;
+            L.h_out = (D.h_in + 2 * D.pad - D.kh) / D.stride + 1;
+            L.w_out = (D.w_in + 2 * D.pad - D.kw) / D.stride + 1;
+            L.n_in = D.c_in * D.h_in * D.w_in;
+            L.n_out = D.c_out * L.h_out * L.w_out;
+        }
+        L.ld_in = round_up(L.n_in, kPad);
+        L.ld_out = round_up(L.n_out, kPad);
+        L.out_off = out_off;
+        out_off += L.n_out;
+        L.relu_off = relu_off;
+        if (L.relu_after) relu_off += L.n_out;
+
+        // per-neuron bias, zero padded
+        host.assign(L.ld_out, 0.0f);
+        if (D.kind == CERT_LAYER_FC) {
+            for (int i = 0; i < L.n_out; ++i) host[i] = D.bias[i];
+        } else {
+            int hw = L.h_out * L.w_out;
+            for (int i = 0; i < L.n_out; ++i) host[i] = D.bias[i / hw];
+        }
+        if (!dev_alloc(net, (void **)&L.bias_n, host.size() * sizeof(float))) { fail = CERT_ERR_OOM; break; }
+        if (cudaMemcpy(L.bias_n, host.data(), host.size() * sizeof(float), cudaMemcpyHostToDevice) != cudaSuccess) {
+            fail = CERT_ERR_CUDA; break;
+        }
+
+        if (D.kind == CERT_LAYER_FC) {
+            size_t rows_pad = round_up(L.n_out, kPad);
+            host.assign(rows_pad * L.ld_in, 0.0f);
+            for (int i = 0; i < L.n_out; ++i)
+                std::memcpy(&host[(size_t)i * L.ld_in], D.weight + (size_t)i * L.n_in, sizeof(float) * L.n_in);
+            if (!dev_alloc(net, (void **)&L.W, host.size() * sizeof(float))) { fail = CERT_ERR_OOM; break; }
+            if (cudaMemcpy(L.W, host.data(), host.size() * sizeof(float), cudaMemcpyHostToDevice) != cudaSuccess) {
+                fail = CERT_ERR_CUDA; break;
+            }
+        } else {
+            size_t nw = (size_t)L.c_out * L.c_in * L.kh * L.kw;
+            if (!dev_alloc(net, (void **)&L.W, nw * sizeof(float))) { fail = CERT_ERR_OOM; break; }
+            if (cudaMemcpy(L.W, D.weight, nw * sizeof(float), cudaMemcpyHostToDevice) != cudaSuccess) {
+                fail = CERT_ERR_CUDA; break;
+            }
+            host.assign(nw, 0.0f);
+            for (int co = 0; co < L.c_out; ++co)
+                for (int ci = 0; ci < L.c_in; ++ci)
+                    for (int ky = 0; ky < L.kh; ++ky)
+                        for (int kx = 0; kx < L.kw; ++kx)
+                            host[(((size_t)co * L.kh + ky) * L.kw + kx) * L.c_in + ci] =
+                                D.weight[(((size_t)co * L.c_in + ci) * L.kh + ky) * L.kw + kx];
+            if (!dev_alloc(net, (void **)&L.Wct, nw * sizeof(float))) { fail = CERT_ERR_OOM; break; }
+            if (cudaMemcpy(L.Wct, host.data(), nw * sizeof(float), cudaMemcpyHostToDevice) != cudaSuccess) {
+                fail = CERT_ERR_CUDA; break;
+            }
+            if (cert::convt_smem_bytes(L) > 200 * 1024) { fail = CERT_ERR_UNSUPPORTED; break; }
+        }
+        if (L.relu_after) {
+            size_t n = (size_t)max_batch * L.ld_out;
+            if (!dev_alloc_zero(net, &L.lamL, n) || !dev_alloc_zero(net, &L.lamU, n) ||
+                !dev_alloc_zero(net, &L.nuU, n)) { fail = CERT_ERR_OOM; break; }
+        }
+    }
+    if (fail == CERT_OK) {
+        net->n0 = net->layers[0].n_in;
+        net->ld0 = net->layers[0].ld_in;
+        net->n_total = out_off;
+        net->n_relu = relu_off;
+        // workspace: the largest coefficient matrix any traversal holds
+        size_t max_elems = 1, max_rows = 1;
+        for (int k = 1; k < n_layers; ++k) {
+            size_t rows = 2ull * max_batch * net->layers[k].n_out;
+            int ld_max = 0;
+            for (int j = 0; j < k; ++j) {
+                ld_max = std::max(ld_max, net->layers[j].ld_out);
+                ld_max = std::max(ld_max, net->layers[j].ld_in);
+            }
+            max_elems = std::max(max_elems, rows * (size_t)ld_max);
+            max_rows = std::max(max_rows, rows);
+        }
+        size_t b = (size_t)max_batch;
+        bool ok = dev_alloc_zero(net, &net->l0, b * net->ld0) && dev_alloc_zero(net, &net->u0, b * net->ld0) &&
+                  dev_alloc_zero(net, &net->buf[0], max_elems) && dev_alloc_zero(net, &net->buf[1], max_elems) &&
+                  dev_alloc_zero(net, &net->d, max_rows) &&
+                  dev_alloc_zero(net, &net->codes, b * std::max(1, net->n_relu)) &&
+                  dev_alloc_zero(net, &net->status_dev, 1) &&
+                  dev_alloc_zero(net, &net->centers_dev, b * net->n0) &&
+                  dev_alloc_zero(net, &net->lb_dev, b * net->n_total) &&
+                  dev_alloc_zero(net, &net->ub_dev, b * net->n_total);
+        if (!ok) fail = CERT_ERR_OOM;
+    }
+    if (fail == CERT_OK) {
+        cert::convt_prepare();
+        if (cudaDeviceSynchronize() != cudaSuccess) fail = CERT_ERR_CUDA;
+    }
+    if (fail != CERT_OK) {
+        cudaGetLastError();
+        free_net(net);
+        return fail;
+    }
+    *out = net;
+    return CERT_OK;
+}
+
+cert_status_t cert_deeppoly_bounds(cert_net_t *net, const float *centers, float eps, int batch, float *lb_out,
+                                   float *ub_out, void *stream) {
+    if (!net || !centers || !lb_out || !ub_out) return CERT_ERR_INVALID_ARG;
+    if (batch < 1 || !(eps >= 0.0f) || std::isinf(eps)) return CERT_ERR_INVALID_ARG;
+    if (batch > net->max_batch) return CERT_ERR_BATCH_TOO_LARGE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int K = net->n_layers;
+    const int n_total = net->n_total;
+    Recorder rec(net, st);
+    int paths = 0;
+
+    cert::launch_box(centers, eps, net->clip_lo, net->clip_hi, batch, net->n0, net->ld0, net->l0, net->u0, st);
+    rec.mark(CERT_CLASS_INPUT);
+    cert::launch_first_layer_bounds(net->layers[0], net->l0, net->u0, net->ld0, batch, lb_out, ub_out, n_total, st);
+    rec.mark(CERT_CLASS_INPUT);
+    if (net->layers[0].relu_after) {
+        cert::launch_relax(net->layers[0], lb_out, ub_out, n_total, batch, net->codes, net->n_relu, st);
+        rec.mark(CERT_CLASS_RELAX);
+    }
+    for (int k = 1; k < K; ++k) {
+        const LayerDev &Lk = net->layers[k];
+        const long long rows = 2LL * batch * Lk.n_out;
+        int cur = 0;
+        // expression over the outputs of layer k-1, pushed through its ReLU
+        cert::launch_init_expr(Lk, net->layers[k - 1], batch, net->buf[cur], net->d, st);
+        rec.mark(CERT_CLASS_RELU_STEP);
+        for (int j = k - 1; j >= 0; --j) {
+            const LayerDev &Lj = net->layers[j];
+            float *Q = net->buf[cur], *P = net->buf[cur ^ 1];
+            if (Lj.kind == CERT_LAYER_FC) {
+                cert::launch_gemm_ffma(Q, Lj.ld_out, Lj.W, Lj.ld_in, P, Lj.ld_in, rows, Lj.n_in, Lj.n_out, st);
+                rec.mark(CERT_CLASS_AFFINE);
+                paths |= 1;
+            } else {
+                cert::launch_convt_ffma(Lj, Q, P, rows, st);
+                rec.mark(CERT_CLASS_CONV);
+            }
+            cur ^= 1;
+            if (j > 0) {
+                cert::launch_relu_step(net->layers[j - 1], batch, Lk.n_out, P, net->d, st);
+                rec.mark(CERT_CLASS_RELU_STEP);
+            } else {
+                cert::launch_concretize(P, net->d, net->l0, net->u0, net->n0, net->ld0, batch, Lk.n_out, lb_out,
+                                        ub_out, n_total, Lk.out_off, st);
+                rec.mark(CERT_CLASS_CONCRETIZE);
+            }
+        }
+        if (Lk.relu_after) {
+            cert::launch_relax(Lk, lb_out, ub_out, n_total, batch, net->codes, net->n_relu, st);
+            rec.mark(CERT_CLASS_RELAX);
+        }
+    }
+    net->last_batch = batch;
+    net->last_launches = rec.launches;
+    net->last_paths = paths;
+    net->prof_marks = rec.marks;
+    if (cudaPeekAtLastError() != cudaSuccess) {
+        cudaGetLastError();
+        return CERT_ERR_CUDA;
+    }
+    return CERT_OK;
+}
+
+cert_status_t cert_deeppoly_bounds_host(cert_net_t *net, const float *centers_host, float eps, int batch,
+                                        float *lb_host, float *ub_host, void *stream) {
+    if (!net || !centers_host || !lb_host || !ub_host) return CERT_ERR_INVALID_ARG;
+    if (batch < 1) return CERT_ERR_INVALID_ARG;
+    if (batch > net->max_batch) return CERT_ERR_BATCH_TOO_LARGE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    size_t in_bytes = (size_t)batch * net->n0 * sizeof(float);
+    size_t out_bytes = (size_t)batch * net->n_total * sizeof(float);
+    if (cudaMemcpyAsync(net->centers_dev, centers_host, in_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) {
+        cudaGetLastError();
+        return CERT_ERR_CUDA;
+    }
+    cert_status_t s = cert_deeppoly_bounds(net, net->centers_dev, eps, batch, net->lb_dev, net->ub_dev, stream);
+    if (s != CERT_OK) return s;
+    if (cudaMemcpyAsync(lb_host, net->lb_dev, out_bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+        cudaMemcpyAsync(ub_host, net->ub_dev, out_bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+        cudaStreamSynchronize(st) != cudaSuccess) {
+        cudaGetLastError();
+        return CERT_ERR_CUDA;
+    }
+    return CERT_OK;
+}
+
+cert_status_t cert_net_destroy(cert_net_t *net) {
+    if (!net) return CERT_ERR_INVALID_ARG;
+    cudaError_t e = cudaDeviceSynchronize();
+    free_net(net);
+    if (e != cudaSuccess) {
+        cudaGetLastError();
+        return CERT_ERR_CUDA;
+    }
+    return CERT_OK;
+}
+
+int cert_net_num_neurons(const cert_net_t *net) { return net ? net->n_total : -1; }
+int cert_net_num_relu_neurons(const cert_net_t *net) { return net ? net->n_relu : -1; }
+
+cert_status_t cert_net_branch_codes(cert_net_t *net, unsigned char *codes_out, void *stream) {
+    if (!net) return CERT_ERR_INVALID_ARG;
+    if (net->last_batch < 1) return CERT_ERR_INVALID_ARG;
+    size_t bytes = (size_t)net->last_batch * net->n_relu;
+    if (bytes == 0) return CERT_OK;
+    if (!codes_out) return CERT_ERR_INVALID_ARG;
+    if (cudaMemcpyAsync(codes_out, net->codes, bytes, cudaMemcpyDeviceToDevice,
+                        static_cast<cudaStream_t>(stream)) != cudaSuccess) {
+        cudaGetLastError();
+        return CERT_ERR_CUDA;
+    }
+    return CERT_OK;
+}
+
+cert_status_t cert_net_last_status(cert_net_t *net, void *stream) {
+    if (!net) return CERT_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int flag = 0;
+    if (cudaMemcpyAsync(&flag, net->status_dev, sizeof(int), cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+        cudaStreamSynchronize(st) != cudaSuccess) {
+        cudaGetLastError();
+        return CERT_ERR_CUDA;
+    }
+    if (flag != 0) {
+        cudaMemsetAsync(net->status_dev, 0, sizeof(int), st);
+        cudaStreamSynchronize(st);
+        return CERT_ERR_TIMEOUT;
+    }
+    return CERT_OK;
+}
+
+cert_status_t cert_net_set_contraction(cert_net_t *net, int mode) {
+    if (!net) return CERT_ERR_INVALID_ARG;
+    if (mode == CERT_CONTRACTION_TC3XTF32) return CERT_ERR_UNSUPPORTED;
+    if (mode != CERT_CONTRACTION_AUTO && mode != CERT_CONTRACTION_FFMA) return CERT_ERR_INVALID_ARG;
+    net->contraction = mode;
+    return CERT_OK;
+}
+
+cert_status_t cert_net_set_profiling(cert_net_t *net, int on) {
+    if (!net) return CERT_ERR_INVALID_ARG;
+    if (on && net->prof_events.empty()) {
+        // one event per launch of the longest schedule, plus the opening one
+        int K = net->n_layers;
+        int n = 4 + K + K * (K + 1) + 8;
+        net->prof_events.resize(n);
+        net->prof_class.assign(n, 0);
+        for (int i = 0; i < n; ++i)
+            if (cudaEventCreate(&net->prof_events[i]) != cudaSuccess) {
+                cudaGetLastError();
+                for (int j = 0; j < i; ++j) cudaEventDestroy(net->prof_events[j]);
+                net->prof_events.clear();
+                return CERT_ERR_CUDA;
+            }
+    }
+    net->profiling = on != 0;
+    net->prof_marks = 0;
+    return CERT_OK;
+}
+
+cert_status_t cert_net_profile(cert_net_t *net, float *ms_out, int *launches_out) {
+    if (!net || !ms_out || !launches_out) return CERT_ERR_INVALID_ARG;
+    for (int c = 0; c < CERT_N_CLASSES; ++c) { ms_out[c] = 0.0f; launches_out[c] = 0; }
+    if (net->prof_marks == 0) return CERT_OK;
+    if (cudaEventSynchronize(net->prof_events[net->prof_marks]) != cudaSuccess) {
+        cudaGetLastError();
+        return CERT_ERR_CUDA;
+    }
+    for (int i = 0; i < net->prof_marks; ++i) {
+        float ms = 0.0f;
+        if (cudaEventElapsedTime(&ms, net->prof_events[i], net->prof_events[i + 1]) != cudaSuccess) {
+            cudaGetLastError();
+            return CERT_ERR_CUDA;
+        }
+        ms_out[net->prof_class[i]] += ms;
+        launches_out[net->prof_class[i]] += 1;
+    }
+    return CERT_OK;
+}
+
+int cert_net_last_contraction_paths(const cert_net_t *net) { return net ? net->last_paths : -1; }
+
+int cert_net_last_launch_count(const cert_net_t *net) { return net ? net->last_launches : -1; }
+
+double cert_net_backstep_flops(const cert_net_t *net, int batch) {
+    if (!net || batch < 1) return 0.0;
+    double f = 0.0;
+    for (int k = 1; k < net->n_layers; ++k) {
+        double rows = 2.0 * batch * net->layers[k].n_out;
+        for (int j = 0; j < k; ++j) {
+            const LayerDev &L = net->layers[j];
+            double per_row = L.kind == CERT_LAYER_FC
+                                 ? 2.0 * L.n_out * L.n_in
+                                 : 2.0 * L.n_out * (double)L.c_in * L.kh * L.kw;
+            f += rows * per_row;
+        }
+    }
+    return f;
+}
+
+}  // extern "C"

@@ -1,0 +1,84 @@
+// Shared declarations of the library's translation units (device structs,
+// launch wrappers, error helpers).  Notation follows the paper: an affine
+// layer k computes z_k = W_k a_{k-1} + b_k; `curr` neurons index rows of W_k,
+// `prev` neurons its columns (Section 3.2).
+#pragma once
+#include <cuda_runtime.h>
+#include <cstdint>
+#include <cstdio>
+#include "../../include/cert.h"
+
+namespace cert {
+
+constexpr int kPad = 32;  // every row of a coefficient / weight / relaxation array is padded to 32 floats
+
+inline int round_up(int x, int m) { return (x + m - 1) / m * m; }
+inline long long ceil_div_ll(long long a, long long b) { return (a + b - 1) / b; }
+
+// One affine layer on the device.
+struct LayerDev {
+    int kind, relu_after;
+    int n_in, n_out;         // neurons below / of this layer
+    int ld_in, ld_out;       // padded to kPad
+    int c_in, h_in, w_in, c_out, kh, kw, stride, pad, h_out, w_out;
+    float *W;                // FC: [round_up(n_out,kPad)][ld_in], zero padded.  CONV: [c_out][c_in][kh][kw]
+    float *Wt_hi, *Wt_lo;    // FC only: TF32 split of W transposed, [round_up(n_in,kPad)][ld_out] (rows = prev neuron)
+    float *Wct;              // CONV only: [c_out][kh][kw][c_in] (c_in innermost) for the transposed-conv kernel
+    float *bias_n;           // [ld_out] one bias per neuron (conv: per-channel bias expanded), zero padded
+    int out_off;             // offset of this layer's neurons in lb_out / ub_out rows
+    int relu_off;            // offset in the branch-code rows (valid if relu_after)
+    // relaxation of the ReLU on top (valid if relu_after): [max_batch][ld_out]
+    float *lamL, *lamU, *nuU;
+};
+
+// Conv geometry handed to kernels by value.
+struct ConvGeom {
+    int c_in, h_in, w_in, c_out, kh, kw, stride, pad, h_out, w_out;
+};
+
+inline ConvGeom geom_of(const LayerDev &L) {
+    return ConvGeom{L.c_in, L.h_in, L.w_in, L.c_out, L.kh, L.kw, L.stride, L.pad, L.h_out, L.w_out};
+}
+
+// ---- launch wrappers (each enqueues exactly one kernel on `st`) ----
+
+// l0 = max(c - eps, lo), u0 = min(c + eps, hi); rows padded with zeros.
+void launch_box(const float *centers, float eps, float lo, float hi, int batch, int n0, int ld0,
+                float *l0, float *u0, cudaStream_t st);
+
+// Bounds of the first affine layer: the expression is already over the input
+// (empty traversal), so they are simplify_lower/upper of the layer's rows.
+void launch_first_layer_bounds(const LayerDev &L, const float *l0, const float *u0, int ld0, int batch,
+                               float *lb_out, float *ub_out, int n_total, cudaStream_t st);
+
+// Relu transformer: relaxation (lamL, lamU, nuU) and branch code from (l, u).
+void launch_relax(const LayerDev &L, const float *lb_out, const float *ub_out, int n_total, int batch,
+                  unsigned char *codes, int n_relu, cudaStream_t st);
+
+// Start of the back-substitution for layer k: the expression of neuron i is
+// row i of W_k (the same for every box and both sides) and the constant b_k[i];
+// it is pushed through the ReLU below (if any) right away, and the constant
+// picks up Q.b of the affine layer below, through which the next step goes.
+//   Q  [rows][ld] with rows = batch*2*n_k ordered (box, side, neuron)
+void launch_init_expr(const LayerDev &Lk, const LayerDev &Lbelow, int batch, float *Q, float *d,
+                      cudaStream_t st);
+
+// ReLU back-step in place on P [rows][ld] (expression over the outputs of
+// layer `Lj`, i.e. over its ReLU neurons if it has one), plus d += Q.b_j.
+void launch_relu_step(const LayerDev &Lj, int batch, int n_k, float *P, float *d, cudaStream_t st);
+
+// map(simplify_lower/upper): rows of P [rows][ld0] against the box.
+void launch_concretize(const float *P, const float *d, const float *l0, const float *u0, int n0, int ld0,
+                       int batch, int n_k, float *lb_out, float *ub_out, int n_total, int out_off,
+                       cudaStream_t st);
+
+// C[M][ldc] = A[M][lda] * B[K][ldb]  (fp32 FMA units).  Columns up to ldc are
+// written (B is zero padded), so padded outputs are zero.
+void launch_gemm_ffma(const float *A, int lda, const float *B, int ldb, float *C, int ldc, long long M,
+                      int N, int K, cudaStream_t st);
+
+// P[r][(ci,iy,ix)] = sum over (co,ky,kx) of Q[r][(co,oy,ox)] * W[co][ci][ky][kx]: the exact
+// transpose of the conv layer applied to every row's coefficient map.
+void launch_convt_ffma(const LayerDev &L, const float *Q, float *P, long long rows, cudaStream_t st);
+
+}  // namespace cert

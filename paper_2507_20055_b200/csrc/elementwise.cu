@@ -1,0 +1,239 @@
+// Bandwidth-bound steps of the DeepPoly path: box construction, first-layer
+// interval bounds, ReLU relaxation, start of a back-substitution, the unfused
+// ReLU back-step and the unfused concretisation.  One warp owns one row of a
+// coefficient matrix; row sums are warp-shuffle trees, so every result is
+// deterministic.
+#include "common.cuh"
+
+namespace cert {
+
+namespace {
+
+constexpr int kWarpsPerBlock = 8;
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+// replace_lower / replace_upper through a ReLU neuron whose bounds are
+// L = lamL*z and U = lamU*z + nuU (Appendix C, DeepPoly listing).  Returns the
+// coefficient over z and adds the constant part to dacc.
+__device__ __forceinline__ float relu_backstep(float c, int upper, float lamL, float lamU, float nuU,
+                                               float &dacc) {
+    const bool nonneg = (c >= 0.0f);
+    const bool use_lower = upper ? !nonneg : nonneg;
+    if (use_lower) return c * lamL;
+    dacc = fmaf(c, nuU, dacc);
+    return c * lamU;
+}
+
+__global__ void box_kernel(const float *__restrict__ centers, float eps, float lo, float hi, int batch,
+                           int n0, int ld0, float *__restrict__ l0, float *__restrict__ u0) {
+    long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= (long long)batch * ld0) return;
+    int b = (int)(idx / ld0), s = (int)(idx % ld0);
+    float l = 0.0f, u = 0.0f;
+    if (s < n0) {
+        float c = centers[(size_t)b * n0 + s];
+        l = fmaxf(__fsub_rn(c, eps), lo);
+        u = fminf(__fadd_rn(c, eps), hi);
+    }
+    l0[idx] = l;
+    u0[idx] = u;
+}
+
+// One warp per (box, neuron of the first layer).
+__global__ void first_layer_kernel(const float *__restrict__ W, const float *__restrict__ bias_n, int kind,
+                                   ConvGeom g, int n_in, int ld_in, int n_out, const float *__restrict__ l0,
+                                   const float *__restrict__ u0, int ld0, int batch, float *__restrict__ lb_out,
+                                   float *__restrict__ ub_out, int n_total, int out_off) {
+    long long warp = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    int lane = threadIdx.x & 31;
+    if (warp >= (long long)batch * n_out) return;
+    int b = (int)(warp / n_out), i = (int)(warp % n_out);
+    const float *lrow = l0 + (size_t)b * ld0, *urow = u0 + (size_t)b * ld0;
+    float lo = 0.0f, hi = 0.0f;
+    if (kind == CERT_LAYER_FC) {
+        const float *w = W + (size_t)i * ld_in;
+        for (int s = lane; s < n_in; s += 32) {
+            float c = w[s], l = lrow[s], u = urow[s];
+            bool nn = (c >= 0.0f);
+            lo = fmaf(c, nn ? l : u, lo);
+            hi = fmaf(c, nn ? u : l, hi);
+        }
+    } else {
+        int hw = g.h_out * g.w_out;
+        int co = i / hw, oy = (i / g.w_out) % g.h_out, ox = i % g.w_out;
+        int taps = g.c_in * g.kh * g.kw;
+        for (int q = lane; q < taps; q += 32) {
+            int ci = q / (g.kh * g.kw), ky = (q / g.kw) % g.kh, kx = q % g.kw;
+            int iy = oy * g.stride - g.pad + ky, ix = ox * g.stride - g.pad + kx;
+            if (iy < 0 || iy >= g.h_in || ix < 0 || ix >= g.w_in) continue;
+            int s = (ci * g.h_in + iy) * g.w_in + ix;
+            float c = W[(size_t)co * taps + q], l = lrow[s], u = urow[s];
+            bool nn = (c >= 0.0f);
+            lo = fmaf(c, nn ? l : u, lo);
+            hi = fmaf(c, nn ? u : l, hi);
+        }
+    }
+    lo = warp_sum(lo);
+    hi = warp_sum(hi);
+    if (lane == 0) {
+        float bb = bias_n[i];
+        lb_out[(size_t)b * n_total + out_off + i] = lo + bb;
+        ub_out[(size_t)b * n_total + out_off + i] = hi + bb;
+    }
+}
+
+// Relu transformer.  One thread per (box, padded neuron).
+__global__ void relax_kernel(const float *__restrict__ lb_out, const float *__restrict__ ub_out, int n_total,
+                             int out_off, int n, int ld, int batch, float *__restrict__ lamL,
+                             float *__restrict__ lamU, float *__restrict__ nuU,
+                             unsigned char *__restrict__ codes, int n_relu, int relu_off) {
+    long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= (long long)batch * ld) return;
+    int b = (int)(idx / ld), t = (int)(idx % ld);
+    float ll = 0.0f, lu = 0.0f, nu = 0.0f;
+    if (t < n) {
+        float l = lb_out[(size_t)b * n_total + out_off + t];
+        float u = ub_out[(size_t)b * n_total + out_off + t];
+        bool pick_one = (__fadd_rn(l, u) >= 0.0f);   // relu_n
+        ll = pick_one ? 1.0f : 0.0f;
+        unsigned char code;
+        if (l >= 0.0f) {                              // compute_upper, first test
+            lu = 1.0f; code = 1;
+        } else if (u <= 0.0f) {                       // second test
+            lu = 0.0f; code = 0;
+        } else {
+            float den = __fsub_rn(u, l);
+            lu = __fdiv_rn(u, den);
+            nu = -__fdiv_rn(__fmul_rn(u, l), den);
+            code = (unsigned char)(2 + (pick_one ? 1 : 0));
+        }
+        codes[(size_t)b * n_relu + relu_off + t] = code;
+    }
+    lamL[idx] = ll;
+    lamU[idx] = lu;
+    nuU[idx] = nu;
+}
+
+// Coefficient of prev-neuron t in the expression of neuron i of layer L.
+__device__ __forceinline__ float weight_elem(const float *__restrict__ W, int kind, const ConvGeom &g,
+                                             int ld_in, int i, int t) {
+    if (kind == CERT_LAYER_FC) return W[(size_t)i * ld_in + t];
+    int hw = g.h_out * g.w_out;
+    int co = i / hw, oy = (i / g.w_out) % g.h_out, ox = i % g.w_out;
+    int ci = t / (g.h_in * g.w_in), iy = (t / g.w_in) % g.h_in, ix = t % g.w_in;
+    int ky = iy - (oy * g.stride - g.pad), kx = ix - (ox * g.stride - g.pad);
+    if (ky < 0 || ky >= g.kh || kx < 0 || kx >= g.kw) return 0.0f;
+    return W[(((size_t)co * g.c_in + ci) * g.kh + ky) * g.kw + kx];
+}
+
+// FROM_WEIGHTS: source is row i of W_k (start of a back-substitution), else P in place.
+template <bool FROM_WEIGHTS>
+__global__ void relu_step_kernel(const float *__restrict__ Wk, int kind_k, ConvGeom gk, int ldw_k,
+                                 const float *__restrict__ bias_k, float *__restrict__ P, float *__restrict__ d,
+                                 long long rows, int n_k, int n, int ld, int has_relu,
+                                 const float *__restrict__ lamL, const float *__restrict__ lamU,
+                                 const float *__restrict__ nuU, const float *__restrict__ bias_below) {
+    long long r = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    int lane = threadIdx.x & 31;
+    if (r >= rows) return;
+    int b = (int)(r / (2LL * n_k));
+    int upper = (int)((r / n_k) & 1);
+    int i = (int)(r % n_k);
+    float *prow = P + (size_t)r * ld;
+    const float *ll = lamL + (size_t)b * ld, *lu = lamU + (size_t)b * ld, *nu = nuU + (size_t)b * ld;
+    float dacc = 0.0f;
+    for (int t = lane; t < ld; t += 32) {
+        float q = 0.0f;
+        if (t < n) {
+            float c = FROM_WEIGHTS ? weight_elem(Wk, kind_k, gk, ldw_k, i, t) : prow[t];
+            q = has_relu ? relu_backstep(c, upper, ll[t], lu[t], nu[t], dacc) : c;
+            dacc = fmaf(q, bias_below[t], dacc);
+        }
+        prow[t] = q;
+    }
+    dacc = warp_sum(dacc);
+    if (lane == 0) d[r] = (FROM_WEIGHTS ? bias_k[i] : d[r]) + dacc;
+}
+
+__global__ void concretize_kernel(const float *__restrict__ P, const float *__restrict__ d,
+                                  const float *__restrict__ l0, const float *__restrict__ u0, int n0, int ld0,
+                                  long long rows, int n_k, float *__restrict__ lb_out, float *__restrict__ ub_out,
+                                  int n_total, int out_off) {
+    long long r = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    int lane = threadIdx.x & 31;
+    if (r >= rows) return;
+    int b = (int)(r / (2LL * n_k));
+    int upper = (int)((r / n_k) & 1);
+    int i = (int)(r % n_k);
+    const float *prow = P + (size_t)r * ld0;
+    const float *lrow = l0 + (size_t)b * ld0, *urow = u0 + (size_t)b * ld0;
+    float acc = 0.0f;
+    for (int s = lane; s < n0; s += 32) {
+        float c = prow[s], l = lrow[s], u = urow[s];
+        bool nn = (c >= 0.0f);
+        acc = fmaf(c, (nn != (upper != 0)) ? l : u, acc);   // lower: c>=0 -> l ; upper: c>=0 -> u
+    }
+    acc = warp_sum(acc);
+    if (lane == 0) {
+        float v = d[r] + acc;
+        (upper ? ub_out : lb_out)[(size_t)b * n_total + out_off + i] = v;
+    }
+}
+
+inline unsigned grid_for_warps(long long warps) {
+    return (unsigned)ceil_div_ll(warps, kWarpsPerBlock);
+}
+
+}  // namespace
+
+void launch_box(const float *centers, float eps, float lo, float hi, int batch, int n0, int ld0, float *l0,
+                float *u0, cudaStream_t st) {
+    long long n = (long long)batch * ld0;
+    box_kernel<<<(unsigned)ceil_div_ll(n, 256), 256, 0, st>>>(centers, eps, lo, hi, batch, n0, ld0, l0, u0);
+}
+
+void launch_first_layer_bounds(const LayerDev &L, const float *l0, const float *u0, int ld0, int batch,
+                               float *lb_out, float *ub_out, int n_total, cudaStream_t st) {
+    long long warps = (long long)batch * L.n_out;
+    first_layer_kernel<<<grid_for_warps(warps), kWarpsPerBlock * 32, 0, st>>>(
+        L.W, L.bias_n, L.kind, geom_of(L), L.n_in, L.ld_in, L.n_out, l0, u0, ld0, batch, lb_out, ub_out,
+        n_total, L.out_off);
+}
+
+void launch_relax(const LayerDev &L, const float *lb_out, const float *ub_out, int n_total, int batch,
+                  unsigned char *codes, int n_relu, cudaStream_t st) {
+    long long n = (long long)batch * L.ld_out;
+    relax_kernel<<<(unsigned)ceil_div_ll(n, 256), 256, 0, st>>>(lb_out, ub_out, n_total, L.out_off, L.n_out,
+                                                               L.ld_out, batch, L.lamL, L.lamU, L.nuU, codes,
+                                                               n_relu, L.relu_off);
+}
+
+void launch_init_expr(const LayerDev &Lk, const LayerDev &Lb, int batch, float *Q, float *d,
+                      cudaStream_t st) {
+    long long rows = 2LL * batch * Lk.n_out;
+    relu_step_kernel<true><<<grid_for_warps(rows), kWarpsPerBlock * 32, 0, st>>>(
+        Lk.W, Lk.kind, geom_of(Lk), Lk.ld_in, Lk.bias_n, Q, d, rows, Lk.n_out, Lb.n_out, Lb.ld_out,
+        Lb.relu_after, Lb.lamL, Lb.lamU, Lb.nuU, Lb.bias_n);
+}
+
+void launch_relu_step(const LayerDev &Lj, int batch, int n_k, float *P, float *d, cudaStream_t st) {
+    long long rows = 2LL * batch * n_k;
+    relu_step_kernel<false><<<grid_for_warps(rows), kWarpsPerBlock * 32, 0, st>>>(
+        nullptr, 0, ConvGeom{}, 0, nullptr, P, d, rows, n_k, Lj.n_out, Lj.ld_out, Lj.relu_after, Lj.lamL,
+        Lj.lamU, Lj.nuU, Lj.bias_n);
+}
+
+void launch_concretize(const float *P, const float *d, const float *l0, const float *u0, int n0, int ld0,
+                       int batch, int n_k, float *lb_out, float *ub_out, int n_total, int out_off,
+                       cudaStream_t st) {
+    long long rows = 2LL * batch * n_k;
+    concretize_kernel<<<grid_for_warps(rows), kWarpsPerBlock * 32, 0, st>>>(P, d, l0, u0, n0, ld0, rows, n_k,
+                                                                          lb_out, ub_out, n_total, out_off);
+}
+
+}  // namespace cert

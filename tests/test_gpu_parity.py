@@ -1,0 +1,130 @@
+"""GPU parity: the CUDA library (through its C ABI) against the float64 oracle,
+element by element, on the same seeded inputs."""
+import numpy as np
+import pytest
+
+from oracle import deeppoly_oracle as orc
+from paper_2507_20055_b200 import workloads as wl
+from parity_util import compare, run_gpu
+
+pytestmark = pytest.mark.gpu
+
+
+def _oracle(w, boxes=None):
+    c = w.centers if boxes is None else w.centers[np.asarray(boxes)]
+    return orc.deeppoly(w.layers, c, w.eps, w.clip_lo, w.clip_hi)
+
+
+@pytest.mark.parametrize("idx", [0, 1, 2, 3])
+def test_config_full_batch(idx):
+    w = wl.make_config(idx)
+    compare(run_gpu(w), _oracle(w), label=w.name)
+
+
+def test_config5_sampled_boxes():
+    """784 -> 1024 x 6 -> 10, 128 boxes on the GPU; the oracle bounds a sample of boxes
+    (boxes are independent, so each sampled box's oracle result is exact)."""
+    w = wl.make_config(4)
+    boxes = [0, 17, 42, 63, 64, 99, 120, 127]
+    compare(run_gpu(w), _oracle(w, boxes), boxes=boxes, label=w.name)
+
+
+SMALL = {
+    "ragged_widths": lambda: wl.small_fc([37, 50, 33, 70, 10], batch=5, eps=0.03, seed=61),
+    "one_hidden": lambda: wl.small_fc([20, 45, 7], batch=3, eps=0.1, seed=62),
+    "single_layer": lambda: wl.small_fc([30, 12], batch=4, eps=0.1, seed=63),
+    "wide_then_narrow": lambda: wl.small_fc([64, 300, 130, 257, 3], batch=9, eps=0.02, seed=64),
+    "relu_on_last": lambda: wl.small_fc([16, 40, 40, 8], batch=2, eps=0.05, seed=65, relu_last=True),
+    "conv_small": lambda: wl.small_conv((2, 9, 7), [(5, 3, 2, 1), (6, 3, 1, 1)], [20, 4], batch=3, eps=0.02, seed=66),
+    "conv_k4s2": lambda: wl.small_conv((3, 12, 12), [(8, 4, 2, 1), (12, 4, 2, 1)], [30, 5], batch=4, eps=0.01, seed=67),
+    "conv_only_then_fc": lambda: wl.small_conv((1, 10, 10), [(20, 5, 1, 0)], [6], batch=2, eps=0.05, seed=68),
+    "conv_stride3": lambda: wl.small_conv((2, 11, 13), [(4, 3, 3, 2)], [9, 3], batch=2, eps=0.05, seed=69),
+}
+
+
+@pytest.mark.parametrize("name", sorted(SMALL))
+def test_small_and_ragged(name):
+    w = SMALL[name]()
+    compare(run_gpu(w), _oracle(w), label=name)
+
+
+def test_missing_relu_in_the_middle():
+    w = wl.small_fc([24, 40, 36, 40, 6], batch=3, eps=0.05, seed=71)
+    w.layers[1].relu_after = False
+    compare(run_gpu(w), _oracle(w), label="no_relu_mid")
+
+
+def test_eps_zero_degenerate_box():
+    w = wl.small_fc([24, 40, 40, 6], batch=3, eps=0.0, seed=72)
+    g, r = run_gpu(w), _oracle(w)
+    assert set(np.unique(g["codes"])) <= {0, 1}
+    np.testing.assert_allclose(g["lb"], g["ub"], rtol=0, atol=1e-5)
+    compare(g, r, label="eps0")
+
+
+def test_no_clipping_and_large_eps():
+    w = wl.small_fc([12, 30, 30, 5], batch=2, eps=0.7, seed=73, clip=(-float("inf"), float("inf")))
+    compare(run_gpu(w), _oracle(w), label="noclip")
+
+
+def test_batch_smaller_than_max_batch_and_reuse():
+    import torch
+    from paper_2507_20055_b200 import binding
+    w = wl.small_fc([33, 64, 64, 10], batch=6, eps=0.04, seed=74)
+    r = _oracle(w)
+    net = binding.CertNet(w.layers, 16)
+    try:
+        c = torch.from_numpy(w.centers).cuda()
+        for batch in (6, 2, 6):          # the workspace is reused across calls
+            lb, ub = net.deeppoly_bounds(c[:batch].contiguous(), w.eps)
+            torch.cuda.synchronize()
+            g = {"lb": lb.cpu().numpy(), "ub": ub.cpu().numpy(),
+                 "codes": net.branch_codes(batch).cpu().numpy(), "status": net.last_status()}
+            sub = {k: v[:batch] for k, v in r.items()}
+            compare(g, sub, label=f"reuse_b{batch}")
+    finally:
+        net.destroy()
+
+
+def test_host_buffer_entry_point():
+    w = wl.small_fc([33, 64, 64, 10], batch=4, eps=0.04, seed=75)
+    compare(run_gpu(w, host_api=True), _oracle(w), label="host_api")
+
+
+def test_non_default_stream():
+    import torch
+    from paper_2507_20055_b200 import binding
+    w = wl.small_fc([33, 64, 64, 10], batch=4, eps=0.04, seed=76)
+    r = _oracle(w)
+    net = binding.CertNet(w.layers, w.batch)
+    try:
+        s = torch.cuda.Stream()
+        c = torch.from_numpy(w.centers).cuda()
+        torch.cuda.synchronize()
+        with torch.cuda.stream(s):
+            lb, ub = net.deeppoly_bounds(c, w.eps, stream=s)
+            codes = net.branch_codes(w.batch, stream=s)
+        s.synchronize()
+        g = {"lb": lb.cpu().numpy(), "ub": ub.cpu().numpy(), "codes": codes.cpu().numpy(),
+             "status": net.last_status(s.cuda_stream)}
+        compare(g, r, label="stream")
+    finally:
+        net.destroy()
+
+
+def test_error_codes_on_device():
+    import torch
+    from paper_2507_20055_b200 import binding
+    w = wl.small_fc([8, 8, 4], batch=2, eps=0.1, seed=77)
+    net = binding.CertNet(w.layers, 2)
+    try:
+        c = torch.zeros((3, 8), device="cuda")
+        out = torch.empty((3, net.n_total), device="cuda")
+        L = binding.lib
+        assert L.cert_deeppoly_bounds(net._h, c.data_ptr(), 0.1, 3, out.data_ptr(), out.data_ptr(), None) == 4
+        assert L.cert_deeppoly_bounds(net._h, None, 0.1, 1, out.data_ptr(), out.data_ptr(), None) == 1
+        assert L.cert_deeppoly_bounds(net._h, c.data_ptr(), -1.0, 1, out.data_ptr(), out.data_ptr(), None) == 1
+        assert L.cert_deeppoly_bounds(net._h, c.data_ptr(), float("nan"), 1, out.data_ptr(), out.data_ptr(), None) == 1
+        assert L.cert_deeppoly_bounds(net._h, c.data_ptr(), 0.1, 0, out.data_ptr(), out.data_ptr(), None) == 1
+    finally:
+        net.destroy()
