@@ -10,6 +10,17 @@
 #include <vector>
 
 #include "common.cuh"
+#include "gemm_tc.cuh"
+
+// Tensor-core operands of the back-step through one FC layer j: B = W_j transposed
+// (rows = neurons below, K-major), A = the coefficient matrix over layer j's neurons
+// in either ping-pong buffer.
+struct TcLayer {
+    bool usable = false;
+    cert::TcMap b_hi, b_lo;
+    cert::TcMap a_hi[2], a_lo[2];
+    int bn = 0, bn_pad = 0, n_tiles = 0, stages = 0, tmem_cols = 0, smem = 0;
+};
 
 struct cert_net {
     int n_layers = 0, max_batch = 0;
@@ -20,7 +31,10 @@ struct cert_net {
     std::vector<cert::LayerDev> layers;
     std::vector<void *> allocs;   // every device allocation, for destroy
     float *l0 = nullptr, *u0 = nullptr;      // [max_batch][ld0]
-    float *buf[2] = {nullptr, nullptr};      // ping-pong coefficient matrices
+    float *buf[2] = {nullptr, nullptr};      // ping-pong coefficient matrices (fp32, or the TF32 hi parts)
+    float *buf_lo[2] = {nullptr, nullptr};   // TF32 lo parts for the tensor-core contraction
+    bool tc_ok = false;                      // tensor-core path usable on this net
+    std::vector<TcLayer> tc;                 // per layer: operand maps and tile plan
     float *d = nullptr;                      // [max rows] constants of the expressions
     unsigned char *codes = nullptr;          // [max_batch][n_relu]
     int *status_dev = nullptr;               // sticky device status word
@@ -100,6 +114,64 @@ cert_status_t validate(const cert_layer_desc_t *layers, int n_layers, int max_ba
         if (prev_out >= 0 && n_in != prev_out) return CERT_ERR_INVALID_ARG;
         prev_out = n_out;
     }
+    return CERT_OK;
+}
+
+// TF32 with round-to-nearest, ties away from zero (what cvt.rna.tf32.f32 does), for finite inputs.
+float host_tf32(float x) {
+    uint32_t u;
+    std::memcpy(&u, &x, 4);
+    u = (u + 0x1000u) & 0xFFFFE000u;
+    float r;
+    std::memcpy(&r, &u, 4);
+    return r;
+}
+
+// Uploads the TF32 split of every FC layer's transposed weights and encodes the TMA
+// descriptors.  Failure to reach the driver entry point leaves the FFMA path in use.
+cert_status_t setup_tensor_core_path(cert_net *net, const cert_layer_desc_t *descs, size_t max_elems) {
+    const int K = net->n_layers;
+    net->tc.assign(K, TcLayer());
+    net->tc_ok = false;
+    if (K < 2) return CERT_OK;
+    if (!cert::tc_driver_init() || !cert::tc_prepare_kernels()) return CERT_OK;
+    if (!dev_alloc_zero(net, &net->buf_lo[0], max_elems) || !dev_alloc_zero(net, &net->buf_lo[1], max_elems))
+        return CERT_ERR_OOM;
+    std::vector<float> hi, lo;
+    for (int j = 0; j < K - 1; ++j) {
+        LayerDev &L = net->layers[j];
+        if (L.kind != CERT_LAYER_FC) continue;
+        TcLayer &T = net->tc[j];
+        // W_j transposed: row s (neuron below), column t (neuron of layer j), pitch ld_out
+        size_t rows_pad = round_up(L.n_in, kPad);
+        hi.assign(rows_pad * L.ld_out, 0.0f);
+        lo.assign(rows_pad * L.ld_out, 0.0f);
+        for (int t = 0; t < L.n_out; ++t)
+            for (int s2 = 0; s2 < L.n_in; ++s2) {
+                float w = descs[j].weight[(size_t)t * L.n_in + s2];
+                float h = host_tf32(w);
+                hi[(size_t)s2 * L.ld_out + t] = h;
+                lo[(size_t)s2 * L.ld_out + t] = host_tf32(w - h);
+            }
+        if (!dev_alloc(net, (void **)&L.Wt_hi, hi.size() * sizeof(float)) ||
+            !dev_alloc(net, (void **)&L.Wt_lo, lo.size() * sizeof(float)))
+            return CERT_ERR_OOM;
+        if (cudaMemcpy(L.Wt_hi, hi.data(), hi.size() * sizeof(float), cudaMemcpyHostToDevice) != cudaSuccess ||
+            cudaMemcpy(L.Wt_lo, lo.data(), lo.size() * sizeof(float), cudaMemcpyHostToDevice) != cudaSuccess)
+            return CERT_ERR_CUDA;
+        cert::tc_tile_plan(L.n_in, &T.bn, &T.bn_pad, &T.n_tiles, &T.stages, &T.tmem_cols, &T.smem);
+        if (T.stages < 2) continue;
+        bool ok = cert::tc_make_map(&T.b_hi, L.Wt_hi, L.n_out, L.n_in, L.ld_out, T.bn) &&
+                  cert::tc_make_map(&T.b_lo, L.Wt_lo, L.n_out, L.n_in, L.ld_out, T.bn);
+        // rows of the largest layer above j
+        long long rows_max = 0;
+        for (int k = j + 1; k < K; ++k) rows_max = std::max(rows_max, 2LL * net->max_batch * net->layers[k].n_out);
+        for (int p = 0; p < 2 && ok; ++p)
+            ok = cert::tc_make_map(&T.a_hi[p], net->buf[p], L.n_out, rows_max, L.ld_out, 128) &&
+                 cert::tc_make_map(&T.a_lo[p], net->buf_lo[p], L.n_out, rows_max, L.ld_out, 128);
+        T.usable = ok;
+    }
+    net->tc_ok = true;
     return CERT_OK;
 }
 
@@ -258,6 +330,7 @@ cert_status_t cert_net_create(const cert_layer_desc_t *layers, int n_layers, int
                   dev_alloc_zero(net, &net->lb_dev, b * net->n_total) &&
                   dev_alloc_zero(net, &net->ub_dev, b * net->n_total);
         if (!ok) fail = CERT_ERR_OOM;
+        if (ok) fail = setup_tensor_core_path(net, layers, max_elems);
     }
     if (fail == CERT_OK) {
         cert::convt_prepare();
@@ -295,12 +368,43 @@ cert_status_t cert_deeppoly_bounds(cert_net_t *net, const float *centers, float 
         const LayerDev &Lk = net->layers[k];
         const long long rows = 2LL * batch * Lk.n_out;
         int cur = 0;
+        // Does the back-step through layer j run on the tensor cores?  Its input must then be a TF32 pair.
+        auto on_tc = [&](int j) {
+            return net->contraction != CERT_CONTRACTION_FFMA && net->tc_ok && net->tc[j].usable;
+        };
         // expression over the outputs of layer k-1, pushed through its ReLU
-        cert::launch_init_expr(Lk, net->layers[k - 1], batch, net->buf[cur], net->d, st);
+        cert::launch_init_expr(Lk, net->layers[k - 1], batch, net->buf[cur],
+                               on_tc(k - 1) ? net->buf_lo[cur] : nullptr, net->d, st);
         rec.mark(CERT_CLASS_RELU_STEP);
         for (int j = k - 1; j >= 0; --j) {
             const LayerDev &Lj = net->layers[j];
             float *Q = net->buf[cur], *P = net->buf[cur ^ 1];
+            float *P_lo = (j > 0 && on_tc(j - 1)) ? net->buf_lo[cur ^ 1] : nullptr;
+            if (on_tc(j)) {
+                const TcLayer &T = net->tc[j];
+                cert::TcArgs a;
+                std::memset(&a, 0, sizeof(a));
+                a.M = rows; a.K = Lj.n_out; a.n_k = Lk.n_out; a.ld_n = Lj.ld_in;
+                a.bn = T.bn; a.bn_pad = T.bn_pad; a.n_tiles = T.n_tiles; a.stages = T.stages;
+                a.tmem_cols = T.tmem_cols;
+                a.d = net->d; a.status = net->status_dev;
+                if (j > 0) {
+                    const LayerDev &Lb = net->layers[j - 1];
+                    a.has_relu = Lb.relu_after;
+                    a.out_hi = P; a.out_lo = P_lo;
+                    a.lamL = Lb.lamL; a.lamU = Lb.lamU; a.nuU = Lb.nuU; a.bias_below = Lb.bias_n;
+                    cert::launch_gemm_tc(cert::TC_EPI_RELU, T.a_hi[cur], T.a_lo[cur], T.b_hi, T.b_lo, a, T.smem, st);
+                } else {
+                    a.l0 = net->l0; a.u0 = net->u0; a.lb_out = lb_out; a.ub_out = ub_out;
+                    a.n_total = n_total; a.out_off = Lk.out_off;
+                    cert::launch_gemm_tc(cert::TC_EPI_CONCRETIZE, T.a_hi[cur], T.a_lo[cur], T.b_hi, T.b_lo, a, T.smem,
+                                         st);
+                }
+                rec.mark(CERT_CLASS_AFFINE);
+                paths |= 2;
+                cur ^= 1;
+                continue;
+            }
             if (Lj.kind == CERT_LAYER_FC) {
                 cert::launch_gemm_ffma(Q, Lj.ld_out, Lj.W, Lj.ld_in, P, Lj.ld_in, rows, Lj.n_in, Lj.n_out, st);
                 rec.mark(CERT_CLASS_AFFINE);
@@ -311,7 +415,7 @@ cert_status_t cert_deeppoly_bounds(cert_net_t *net, const float *centers, float 
             }
             cur ^= 1;
             if (j > 0) {
-                cert::launch_relu_step(net->layers[j - 1], batch, Lk.n_out, P, net->d, st);
+                cert::launch_relu_step(net->layers[j - 1], batch, Lk.n_out, P, P_lo, net->d, st);
                 rec.mark(CERT_CLASS_RELU_STEP);
             } else {
                 cert::launch_concretize(P, net->d, net->l0, net->u0, net->n0, net->ld0, batch, Lk.n_out, lb_out,
@@ -405,8 +509,9 @@ cert_status_t cert_net_last_status(cert_net_t *net, void *stream) {
 
 cert_status_t cert_net_set_contraction(cert_net_t *net, int mode) {
     if (!net) return CERT_ERR_INVALID_ARG;
-    if (mode == CERT_CONTRACTION_TC3XTF32) return CERT_ERR_UNSUPPORTED;
-    if (mode != CERT_CONTRACTION_AUTO && mode != CERT_CONTRACTION_FFMA) return CERT_ERR_INVALID_ARG;
+    if (mode != CERT_CONTRACTION_AUTO && mode != CERT_CONTRACTION_FFMA && mode != CERT_CONTRACTION_TC3XTF32)
+        return CERT_ERR_INVALID_ARG;
+    if (mode == CERT_CONTRACTION_TC3XTF32 && !net->tc_ok) return CERT_ERR_UNSUPPORTED;
     net->contraction = mode;
     return CERT_OK;
 }

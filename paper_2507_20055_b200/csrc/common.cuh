@@ -60,12 +60,14 @@ void launch_relax(const LayerDev &L, const float *lb_out, const float *ub_out, i
 // it is pushed through the ReLU below (if any) right away, and the constant
 // picks up Q.b of the affine layer below, through which the next step goes.
 //   Q  [rows][ld] with rows = batch*2*n_k ordered (box, side, neuron)
-void launch_init_expr(const LayerDev &Lk, const LayerDev &Lbelow, int batch, float *Q, float *d,
+//   Q_lo != nullptr: Q is written as a TF32 pair (hi in Q, lo in Q_lo) for the tensor-core contraction
+void launch_init_expr(const LayerDev &Lk, const LayerDev &Lbelow, int batch, float *Q, float *Q_lo, float *d,
                       cudaStream_t st);
 
 // ReLU back-step in place on P [rows][ld] (expression over the outputs of
 // layer `Lj`, i.e. over its ReLU neurons if it has one), plus d += Q.b_j.
-void launch_relu_step(const LayerDev &Lj, int batch, int n_k, float *P, float *d, cudaStream_t st);
+void launch_relu_step(const LayerDev &Lj, int batch, int n_k, float *P, float *P_lo, float *d,
+                      cudaStream_t st);
 
 // map(simplify_lower/upper): rows of P [rows][ld0] against the box.
 void launch_concretize(const float *P, const float *d, const float *l0, const float *u0, int n0, int ld0,

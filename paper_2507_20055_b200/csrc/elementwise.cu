@@ -11,6 +11,12 @@ namespace {
 
 constexpr int kWarpsPerBlock = 8;
 
+__device__ __forceinline__ float tf32_round(float x) {
+    uint32_t r;
+    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(x));
+    return __uint_as_float(r);
+}
+
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
@@ -134,7 +140,8 @@ __device__ __forceinline__ float weight_elem(const float *__restrict__ W, int ki
 // FROM_WEIGHTS: source is row i of W_k (start of a back-substitution), else P in place.
 template <bool FROM_WEIGHTS>
 __global__ void relu_step_kernel(const float *__restrict__ Wk, int kind_k, ConvGeom gk, int ldw_k,
-                                 const float *__restrict__ bias_k, float *__restrict__ P, float *__restrict__ d,
+                                 const float *__restrict__ bias_k, float *__restrict__ P,
+                                 float *__restrict__ P_lo, float *__restrict__ d,
                                  long long rows, int n_k, int n, int ld, int has_relu,
                                  const float *__restrict__ lamL, const float *__restrict__ lamU,
                                  const float *__restrict__ nuU, const float *__restrict__ bias_below) {
@@ -154,7 +161,14 @@ __global__ void relu_step_kernel(const float *__restrict__ Wk, int kind_k, ConvG
             q = has_relu ? relu_backstep(c, upper, ll[t], lu[t], nu[t], dacc) : c;
             dacc = fmaf(q, bias_below[t], dacc);
         }
-        prow[t] = q;
+        if (P_lo) {
+            // operand form of the tensor-core contraction: q = hi + lo, both TF32
+            float h = tf32_round(q);
+            prow[t] = h;
+            P_lo[(size_t)r * ld + t] = tf32_round(q - h);
+        } else {
+            prow[t] = q;
+        }
     }
     dacc = warp_sum(dacc);
     if (lane == 0) d[r] = (FROM_WEIGHTS ? bias_k[i] : d[r]) + dacc;
@@ -213,18 +227,19 @@ void launch_relax(const LayerDev &L, const float *lb_out, const float *ub_out, i
                                                                n_relu, L.relu_off);
 }
 
-void launch_init_expr(const LayerDev &Lk, const LayerDev &Lb, int batch, float *Q, float *d,
+void launch_init_expr(const LayerDev &Lk, const LayerDev &Lb, int batch, float *Q, float *Q_lo, float *d,
                       cudaStream_t st) {
     long long rows = 2LL * batch * Lk.n_out;
     relu_step_kernel<true><<<grid_for_warps(rows), kWarpsPerBlock * 32, 0, st>>>(
-        Lk.W, Lk.kind, geom_of(Lk), Lk.ld_in, Lk.bias_n, Q, d, rows, Lk.n_out, Lb.n_out, Lb.ld_out,
+        Lk.W, Lk.kind, geom_of(Lk), Lk.ld_in, Lk.bias_n, Q, Q_lo, d, rows, Lk.n_out, Lb.n_out, Lb.ld_out,
         Lb.relu_after, Lb.lamL, Lb.lamU, Lb.nuU, Lb.bias_n);
 }
 
-void launch_relu_step(const LayerDev &Lj, int batch, int n_k, float *P, float *d, cudaStream_t st) {
+void launch_relu_step(const LayerDev &Lj, int batch, int n_k, float *P, float *P_lo, float *d,
+                      cudaStream_t st) {
     long long rows = 2LL * batch * n_k;
     relu_step_kernel<false><<<grid_for_warps(rows), kWarpsPerBlock * 32, 0, st>>>(
-        nullptr, 0, ConvGeom{}, 0, nullptr, P, d, rows, n_k, Lj.n_out, Lj.ld_out, Lj.relu_after, Lj.lamL,
+        nullptr, 0, ConvGeom{}, 0, nullptr, P, P_lo, d, rows, n_k, Lj.n_out, Lj.ld_out, Lj.relu_after, Lj.lamL,
         Lj.lamU, Lj.nuU, Lj.bias_n);
 }
 

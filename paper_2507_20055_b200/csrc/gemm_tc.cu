@@ -1,0 +1,446 @@
+// Affine back-step on the 5th-generation tensor cores (tcgen05), fp32-accurate
+// through a three-term TF32 split, with the ReLU back-step or the
+// concretisation fused into the epilogue.
+//
+//   P = Q * W_j                    (Section 4.3, Matmul rewrite of the traversal step)
+//   Q' = P+ * lam_a + P- * lam_b   (replace_lower/upper through the ReLU below,
+//   d += P(+/-) . nuU + Q' . b       clamp form of Section 4.3), or
+//   bound = P+ . l0 + P- . u0 + d  (map(simplify_lower/upper) at the input)
+//
+// Every fp32 operand x is held as hi = tf32(x) and lo = tf32(x - hi); the
+// product is hi*hi + lo*hi + hi*lo accumulated in fp32 in tensor memory.
+//
+// One CTA owns a panel of 128 rows and walks the column tiles of W_j, so the
+// thread that owns a row (its TMEM lane) carries that row's constant across
+// all columns in a register: no atomics, fixed summation order.
+// Warp roles: warp 0 = TMA producer, warp 1 = MMA issuer and TMEM owner,
+// warps 2..5 = epilogue (one TMEM lane quarter each).
+#include <cuda.h>
+
+#include "common.cuh"
+#include "gemm_tc.cuh"
+
+namespace cert {
+
+namespace {
+
+constexpr int BM = 128;
+constexpr int kThreads = 192;
+constexpr unsigned long long kWaitCycles = 2000000000ull;   // about a second
+
+// ---------------------------------------------------------------- PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void *p) {
+    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t *bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes)
+                 : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t *bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait: gives up after kWaitCycles and reports false.
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    while (!mbar_try_wait(bar, parity)) {
+        if ((unsigned long long)(clock64() - t0) > kWaitCycles) return false;
+    }
+    return true;
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, uint64_t *bar, int x, int y) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst), "l"(map), "r"(smem_u32(bar)), "r"(x), "r"(y)
+        : "memory");
+}
+__device__ __forceinline__ void tcgen05_fence_before() {
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+}
+__device__ __forceinline__ void tcgen05_fence_after() {
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+}
+__device__ __forceinline__ void tcgen05_commit(uint64_t *bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
+                 : "memory");
+}
+__device__ __forceinline__ void mma_tf32(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                         uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+          "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
+          "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
+          "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+__device__ __forceinline__ float tf32_round(float x) {
+    uint32_t r;
+    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(x));
+    return __uint_as_float(r);
+}
+
+// Shared-memory matrix descriptor: K-major tile, rows of 128 bytes, 128-byte swizzle,
+// 8-row groups 1024 bytes apart.
+__device__ __forceinline__ uint64_t make_desc_sw128(uint32_t smem_addr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((smem_addr >> 4) & 0x3FFF);
+    d |= (uint64_t)1 << 16;             // leading byte offset (unused for swizzled K-major), in 16-byte units
+    d |= (uint64_t)(1024 >> 4) << 32;   // stride byte offset between 8-row groups
+    d |= (uint64_t)1 << 46;             // descriptor version for sm_100
+    d |= (uint64_t)2 << 61;             // SWIZZLE_128B
+    return d;
+}
+
+struct __align__(8) Barriers {
+    uint64_t full[8];
+    uint64_t empty[8];
+    uint64_t acc_full[2];
+    uint64_t acc_empty[2];
+    uint32_t tmem_base;
+    uint32_t abort_flag;
+};
+
+template <int EPI>
+__global__ void __launch_bounds__(kThreads, 1)
+gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_constant__ CUtensorMap map_a_lo,
+               const __grid_constant__ CUtensorMap map_b_hi, const __grid_constant__ CUtensorMap map_b_lo,
+               const TcArgs a) {
+    extern __shared__ uint8_t smem_raw[];
+    // tiles need 1024-byte alignment for the 128-byte swizzle
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    const int BN = a.bn;
+    const int stages = a.stages;
+    const uint32_t a_tile_bytes = BM * 128;
+    const uint32_t b_tile_bytes = (uint32_t)BN * 128;
+    const uint32_t stage_bytes = 2 * a_tile_bytes + 2 * b_tile_bytes;
+    Barriers *bars = reinterpret_cast<Barriers *>(smem + (size_t)stages * stage_bytes);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const long long row0 = (long long)blockIdx.x * BM;
+    const int num_kb = (a.K + 31) / 32;
+    const int n_tiles = a.n_tiles;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < stages; ++s) {
+            mbar_init(&bars->full[s], 1);
+            mbar_init(&bars->empty[s], 1);
+        }
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(&bars->acc_full[i], 1);
+            mbar_init(&bars->acc_empty[i], 4);
+        }
+        bars->abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
+                         smem_u32(&bars->tmem_base)),
+                     "r"((uint32_t)a.tmem_cols)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tcgen05_fence_before();
+    __syncthreads();
+    tcgen05_fence_after();
+    const uint32_t tmem_base = bars->tmem_base;
+    volatile uint32_t *abort_flag = &bars->abort_flag;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            int s = 0;
+            uint32_t phase = 0;
+            bool ok = true;
+            int armed = 0;      // stages whose loads were issued
+            for (int nt = 0; nt < n_tiles && ok; ++nt) {
+                for (int kb = 0; kb < num_kb; ++kb) {
+                    if (!mbar_wait(&bars->empty[s], phase ^ 1) || *abort_flag) { ok = false; break; }
+                    uint8_t *st = smem + (size_t)s * stage_bytes;
+                    mbar_arrive_expect_tx(&bars->full[s], stage_bytes);
+                    const int kx = kb * 32;
+                    tma_load_2d(smem_u32(st), &map_a_hi, &bars->full[s], kx, (int)row0);
+                    tma_load_2d(smem_u32(st + a_tile_bytes), &map_a_lo, &bars->full[s], kx, (int)row0);
+                    tma_load_2d(smem_u32(st + 2 * a_tile_bytes), &map_b_hi, &bars->full[s], kx, nt * BN);
+                    tma_load_2d(smem_u32(st + 2 * a_tile_bytes + b_tile_bytes), &map_b_lo, &bars->full[s], kx,
+                                nt * BN);
+                    ++armed;
+                    if (++s == stages) { s = 0; phase ^= 1; }
+                }
+            }
+            if (!ok) {
+                *abort_flag = 1;
+                atomicExch(a.status, 1);
+                // let the copies already in flight land before the CTA gives its shared memory back
+                int back = armed < stages ? armed : stages;
+                int ss = s;
+                uint32_t ph = phase;
+                for (int i = 0; i < back; ++i) {
+                    if (--ss < 0) { ss = stages - 1; ph ^= 1; }
+                    mbar_wait(&bars->full[ss], ph);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(BN >> 3) << 17) |
+                                   ((uint32_t)(BM >> 4) << 24);
+            int s = 0;
+            uint32_t phase = 0;
+            bool ok = true;
+            for (int nt = 0; nt < n_tiles && ok; ++nt) {
+                const int acc = nt & 1;
+                const uint32_t acc_phase = (nt >> 1) & 1;
+                if (!mbar_wait(&bars->acc_empty[acc], acc_phase ^ 1) || *abort_flag) { ok = false; break; }
+                tcgen05_fence_after();
+                const uint32_t d_tmem = tmem_base + (uint32_t)(acc * a.bn_pad);
+                for (int kb = 0; kb < num_kb; ++kb) {
+                    if (!mbar_wait(&bars->full[s], phase) || *abort_flag) { ok = false; break; }
+                    tcgen05_fence_after();
+                    const uint32_t st = smem_u32(smem + (size_t)s * stage_bytes);
+                    const uint64_t da_hi = make_desc_sw128(st);
+                    const uint64_t da_lo = make_desc_sw128(st + a_tile_bytes);
+                    const uint64_t db_hi = make_desc_sw128(st + 2 * a_tile_bytes);
+                    const uint64_t db_lo = make_desc_sw128(st + 2 * a_tile_bytes + b_tile_bytes);
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        const uint64_t ko = (uint64_t)(k * 2);   // 8 floats = 32 bytes = 2 x 16-byte units
+                        mma_tf32(d_tmem, da_lo + ko, db_hi + ko, idesc, (kb | k) ? 1u : 0u);
+                        mma_tf32(d_tmem, da_hi + ko, db_lo + ko, idesc, 1u);
+                        mma_tf32(d_tmem, da_hi + ko, db_hi + ko, idesc, 1u);
+                    }
+                    tcgen05_commit(&bars->empty[s]);     // frees the stage when these MMAs retire
+                    if (++s == stages) { s = 0; phase ^= 1; }
+                }
+                if (ok) tcgen05_commit(&bars->acc_full[acc]);
+            }
+            if (!ok) {
+                *abort_flag = 1;
+                atomicExch(a.status, 1);
+            }
+        }
+    } else {
+        // ------------------------------------------------------------ epilogue
+        const int quarter = warp & 3;                       // TMEM lane quarter this warp may read
+        const long long r = row0 + quarter * 32 + lane;
+        const bool row_ok = r < a.M;
+        const long long rr = row_ok ? r : 0;
+        const int b = (int)(rr / (2LL * a.n_k));
+        const int upper = (int)((rr / a.n_k) & 1);
+        const int i = (int)(rr % a.n_k);
+        float dacc = 0.0f;
+        bool ok = true;
+        const size_t relax_row = (size_t)b * a.ld_n;
+        for (int nt = 0; nt < n_tiles && ok; ++nt) {
+            const int acc = nt & 1;
+            const uint32_t acc_phase = (nt >> 1) & 1;
+            if (!mbar_wait(&bars->acc_full[acc], acc_phase) || *abort_flag) { ok = false; break; }
+            tcgen05_fence_after();
+            const uint32_t t_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * a.bn_pad);
+            for (int c0 = 0; c0 < BN; c0 += 32) {
+                const int col0 = nt * BN + c0;
+                if (col0 >= a.ld_n) break;                  // warp-uniform
+                uint32_t v[32];
+                __syncwarp();
+                tmem_ld32(t_addr + (uint32_t)c0, v);
+                tmem_ld_wait();
+                const int col_end = min((nt + 1) * BN, a.ld_n);   // columns this tile owns
+                if (!row_ok) {
+                    // rows past the end of the matrix: nothing to store
+                } else if (EPI == TC_EPI_RELU) {
+                    float *qh = a.out_hi + (size_t)r * a.ld_n + col0;
+                    float *ql = a.out_lo ? a.out_lo + (size_t)r * a.ld_n + col0 : nullptr;
+#pragma unroll
+                    for (int g = 0; g < 8; ++g) {
+                        const int col = col0 + g * 4;
+                        if (col >= col_end) break;
+                        float q[4];
+                        const float4 bz = *reinterpret_cast<const float4 *>(a.bias_below + col);
+                        if (a.has_relu) {
+                            const float4 ll = *reinterpret_cast<const float4 *>(a.lamL + relax_row + col);
+                            const float4 lu = *reinterpret_cast<const float4 *>(a.lamU + relax_row + col);
+                            const float4 nu = *reinterpret_cast<const float4 *>(a.nuU + relax_row + col);
+                            const float l4[4] = {ll.x, ll.y, ll.z, ll.w}, u4[4] = {lu.x, lu.y, lu.z, lu.w},
+                                        n4[4] = {nu.x, nu.y, nu.z, nu.w};
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                const float c = __uint_as_float(v[g * 4 + e]);
+                                const bool nonneg = (c >= 0.0f);
+                                const bool use_lower = upper ? !nonneg : nonneg;
+                                q[e] = c * (use_lower ? l4[e] : u4[e]);
+                                dacc = fmaf(c, use_lower ? 0.0f : n4[e], dacc);
+                            }
+                        } else {
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) q[e] = __uint_as_float(v[g * 4 + e]);
+                        }
+                        dacc = fmaf(q[0], bz.x, dacc);
+                        dacc = fmaf(q[1], bz.y, dacc);
+                        dacc = fmaf(q[2], bz.z, dacc);
+                        dacc = fmaf(q[3], bz.w, dacc);
+                        if (ql) {
+                            float h[4], l[4];
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                h[e] = tf32_round(q[e]);
+                                l[e] = tf32_round(q[e] - h[e]);
+                            }
+                            *reinterpret_cast<float4 *>(qh + g * 4) = make_float4(h[0], h[1], h[2], h[3]);
+                            *reinterpret_cast<float4 *>(ql + g * 4) = make_float4(l[0], l[1], l[2], l[3]);
+                        } else {
+                            *reinterpret_cast<float4 *>(qh + g * 4) = make_float4(q[0], q[1], q[2], q[3]);
+                        }
+                    }
+                } else {
+                    const float *lrow = a.l0 + (size_t)b * a.ld_n + col0;
+                    const float *urow = a.u0 + (size_t)b * a.ld_n + col0;
+#pragma unroll
+                    for (int g = 0; g < 8; ++g) {
+                        const int col = col0 + g * 4;
+                        if (col >= col_end) break;
+                        const float4 l4 = *reinterpret_cast<const float4 *>(lrow + g * 4);
+                        const float4 u4 = *reinterpret_cast<const float4 *>(urow + g * 4);
+                        const float lo4[4] = {l4.x, l4.y, l4.z, l4.w}, up4[4] = {u4.x, u4.y, u4.z, u4.w};
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const float c = __uint_as_float(v[g * 4 + e]);
+                            const bool nonneg = (c >= 0.0f);
+                            dacc = fmaf(c, (nonneg != (upper != 0)) ? lo4[e] : up4[e], dacc);
+                        }
+                    }
+                }
+            }
+            tcgen05_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&bars->acc_empty[acc]);
+        }
+        if (ok && row_ok) {
+            if (EPI == TC_EPI_RELU) {
+                a.d[r] = a.d[r] + dacc;
+            } else {
+                float *out = upper ? a.ub_out : a.lb_out;
+                out[(size_t)b * a.n_total + a.out_off + i] = a.d[r] + dacc;
+            }
+        }
+        if (!ok && lane == 0) atomicExch(a.status, 1);
+    }
+
+    tcgen05_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tcgen05_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base),
+                     "r"((uint32_t)a.tmem_cols)
+                     : "memory");
+    }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+EncodeTiledFn g_encode = nullptr;
+
+}  // namespace
+
+bool tc_driver_init() {
+    if (g_encode) return true;
+    void *fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
+        qres != cudaDriverEntryPointSuccess || !fn) {
+        cudaGetLastError();
+        return false;
+    }
+    g_encode = reinterpret_cast<EncodeTiledFn>(fn);
+    return true;
+}
+
+bool tc_prepare_kernels() {
+    cudaError_t e1 = cudaFuncSetAttribute(gemm_tc_kernel<TC_EPI_RELU>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                          kTcSmemMax);
+    cudaError_t e2 = cudaFuncSetAttribute(gemm_tc_kernel<TC_EPI_CONCRETIZE>,
+                                          cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemMax);
+    if (e1 != cudaSuccess || e2 != cudaSuccess) {
+        cudaGetLastError();
+        return false;
+    }
+    return true;
+}
+
+// 2D fp32 tensor [outer][inner] with row pitch `pitch_floats`; box = 32 floats x box_outer rows, 128-byte swizzle.
+bool tc_make_map(TcMap *m, const float *base, long long inner, long long outer, long long pitch_floats,
+                 int box_outer) {
+    if (!g_encode) return false;
+    static_assert(sizeof(TcMap) == sizeof(CUtensorMap), "tensor map size");
+    cuuint64_t dims[2] = {(cuuint64_t)inner, (cuuint64_t)outer};
+    cuuint64_t strides[1] = {(cuuint64_t)pitch_floats * sizeof(float)};
+    cuuint32_t box[2] = {32u, (cuuint32_t)box_outer};
+    cuuint32_t estr[2] = {1u, 1u};
+    CUresult r = g_encode(reinterpret_cast<CUtensorMap *>(m), CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2,
+                          const_cast<float *>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                          CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
+void tc_tile_plan(int N, int *bn, int *bn_pad, int *n_tiles, int *stages, int *tmem_cols, int *smem_bytes) {
+    int nt = (N + 255) / 256;
+    int b = ((N + nt - 1) / nt + 15) / 16 * 16;
+    if (b < 16) b = 16;
+    *bn = b;
+    *bn_pad = (b + 31) / 32 * 32;
+    *n_tiles = nt;
+    int stage_bytes = 2 * BM * 128 + 2 * b * 128;
+    int st = (kTcSmemMax - 2048) / stage_bytes;
+    if (st > 8) st = 8;
+    *stages = st;
+    int cols = 32;
+    while (cols < 2 * *bn_pad) cols *= 2;
+    *tmem_cols = cols;
+    *smem_bytes = st * stage_bytes + 2048;
+}
+
+void launch_gemm_tc(int epi, const TcMap &a_hi, const TcMap &a_lo, const TcMap &b_hi, const TcMap &b_lo,
+                    const TcArgs &args, int smem_bytes, cudaStream_t st) {
+    unsigned grid = (unsigned)ceil_div_ll(args.M, BM);
+    const CUtensorMap &ah = reinterpret_cast<const CUtensorMap &>(a_hi);
+    const CUtensorMap &al = reinterpret_cast<const CUtensorMap &>(a_lo);
+    const CUtensorMap &bh = reinterpret_cast<const CUtensorMap &>(b_hi);
+    const CUtensorMap &bl = reinterpret_cast<const CUtensorMap &>(b_lo);
+    if (epi == TC_EPI_RELU)
+        gemm_tc_kernel<TC_EPI_RELU><<<grid, kThreads, smem_bytes, st>>>(ah, al, bh, bl, args);
+    else
+        gemm_tc_kernel<TC_EPI_CONCRETIZE><<<grid, kThreads, smem_bytes, st>>>(ah, al, bh, bl, args);
+}
+
+}  // namespace cert

@@ -23,9 +23,10 @@ def run_gpu(w, contraction=None, max_batch=None, host_api=False):
         codes = net.branch_codes(w.batch).cpu().numpy()
         status = net.last_status()
         launches = net.last_launch_count()
+        paths = net.last_contraction_paths()
     finally:
         net.destroy()
-    return {"lb": lb, "ub": ub, "codes": codes, "status": status, "launches": launches}
+    return {"lb": lb, "ub": ub, "codes": codes, "status": status, "launches": launches, "paths": paths}
 
 
 def compare(gpu, ref, boxes=None, min_good_fraction=0.5, label=""):

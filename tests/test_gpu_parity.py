@@ -15,18 +15,25 @@ def _oracle(w, boxes=None):
     return orc.deeppoly(w.layers, c, w.eps, w.clip_lo, w.clip_hi)
 
 
+MODES = {"ffma": 1, "tc": 2}
+
+
+@pytest.mark.parametrize("mode", ["ffma", "tc"])
 @pytest.mark.parametrize("idx", [0, 1, 2, 3])
-def test_config_full_batch(idx):
+def test_config_full_batch(idx, mode):
     w = wl.make_config(idx)
-    compare(run_gpu(w), _oracle(w), label=w.name)
+    g = run_gpu(w, contraction=MODES[mode])
+    assert g["paths"] & MODES[mode] or idx == 3
+    compare(g, _oracle(w), label=f"{w.name}/{mode}")
 
 
-def test_config5_sampled_boxes():
+@pytest.mark.parametrize("mode", ["ffma", "tc"])
+def test_config5_sampled_boxes(mode):
     """784 -> 1024 x 6 -> 10, 128 boxes on the GPU; the oracle bounds a sample of boxes
     (boxes are independent, so each sampled box's oracle result is exact)."""
     w = wl.make_config(4)
     boxes = [0, 17, 42, 63, 64, 99, 120, 127]
-    compare(run_gpu(w), _oracle(w, boxes), boxes=boxes, label=w.name)
+    compare(run_gpu(w, contraction=MODES[mode]), _oracle(w, boxes), boxes=boxes, label=f"{w.name}/{mode}")
 
 
 SMALL = {
@@ -42,10 +49,13 @@ SMALL = {
 }
 
 
+@pytest.mark.parametrize("mode", ["ffma", "tc"])
 @pytest.mark.parametrize("name", sorted(SMALL))
-def test_small_and_ragged(name):
+def test_small_and_ragged(name, mode):
     w = SMALL[name]()
-    compare(run_gpu(w), _oracle(w), label=name)
+    if mode == "tc" and len(w.layers) < 2:
+        pytest.skip("a single layer has no back-step")
+    compare(run_gpu(w, contraction=MODES[mode]), _oracle(w), label=f"{name}/{mode}")
 
 
 def test_missing_relu_in_the_middle():
