@@ -155,6 +155,41 @@ int cert_net_last_launch_count(const cert_net_t *net);
  * maps), as the benchmark's roofline numerator. */
 double cert_net_backstep_flops(const cert_net_t *net, int batch);
 
+/*
+ * (No counterpart in the paper: an addition for embedders.)
+ *
+ * Interval bounds of a single FC layer over `batch` L-infinity boxes, the
+ * same numbers cert_deeppoly_bounds returns for a one-layer net, without any
+ * allocation.  It is meant for callers that are not allowed to obtain device
+ * memory themselves: code that runs under another framework's memory pool and
+ * must not go around it, services whose memory budget is fixed at start-up,
+ * and latency-sensitive loops where the implicit synchronisation of
+ * cudaMalloc / cudaFree is not acceptable.  Neither this call nor anything it
+ * uses calls cudaMalloc, cudaFree or an allocating library routine.
+ *
+ *   weight   DEVICE float32 [out_features][in_features] row-major (unpadded)
+ *   bias     DEVICE float32 [out_features]
+ *   centers  DEVICE float32 [batch][in_features]
+ *   lb_out, ub_out  DEVICE float32 [batch][out_features]
+ * The caller owns all five.  The box endpoints, which the regular path keeps
+ * in the net's workspace, are held in a fixed 8 MiB array that is part of the
+ * library image (every GPU that loads the library carries it until the
+ * process ends).  Limit: batch * round_up(in_features, 32) <= 1048576;
+ * beyond it the call returns CERT_ERR_BATCH_TOO_LARGE and does nothing.
+ *
+ * The first call on each device looks up the array's device address (a
+ * synchronous runtime query made with that device current); make that first
+ * call before starting any stream capture.  All calls on a device share the
+ * one array: a call overwrites every element it later reads, so nothing
+ * needs clearing between calls, but two calls whose kernels overlap on the
+ * GPU (different streams, no ordering between them) race on it.  Work is
+ * enqueued on `stream`; the call does not wait for it.
+ */
+cert_status_t cert_first_layer_bounds_noalloc(const float *weight, const float *bias, int out_features,
+                                              int in_features, const float *centers, float eps,
+                                              float clip_lo, float clip_hi, int batch, float *lb_out,
+                                              float *ub_out, void *stream);
+
 const char *cert_status_string(cert_status_t s);
 
 #ifdef __cplusplus

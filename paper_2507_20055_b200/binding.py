@@ -30,7 +30,7 @@ EXPORTS = [
     "cert_net_num_neurons", "cert_net_num_relu_neurons", "cert_net_branch_codes",
     "cert_net_last_status", "cert_net_set_contraction", "cert_net_last_launch_count",
     "cert_net_backstep_flops", "cert_status_string", "cert_net_set_profiling", "cert_net_profile",
-    "cert_net_last_contraction_paths",
+    "cert_net_last_contraction_paths", "cert_first_layer_bounds_noalloc",
 ]
 CLASS_NAMES = ["input", "relax", "relu_step", "affine", "conv", "concretize"]
 
@@ -71,6 +71,8 @@ _lib.cert_net_set_profiling.argtypes = [_vp, _i]
 _lib.cert_net_set_profiling.restype = _i
 _lib.cert_net_profile.argtypes = [_vp, _vp, _vp]
 _lib.cert_net_profile.restype = _i
+_lib.cert_first_layer_bounds_noalloc.argtypes = [_vp, _vp, _i, _i, _vp, _f, _f, _f, _i, _vp, _vp, _vp]
+_lib.cert_first_layer_bounds_noalloc.restype = _i
 _lib.cert_status_string.argtypes = [_i]
 _lib.cert_status_string.restype = ctypes.c_char_p
 
@@ -203,6 +205,23 @@ class CertNet:
             self.destroy()
         except Exception:
             pass
+
+
+def first_layer_bounds_noalloc(weight, bias, centers, eps, clip_lo, clip_hi, lb_out, ub_out, stream=None):
+    """Interval bounds of one FC layer without any allocation inside the library.
+
+    All tensors are the caller's torch CUDA tensors (float32, contiguous): weight [out, in],
+    bias [out], centers [batch, in], lb_out / ub_out [batch, out].  For embedders that may not
+    allocate device memory; see cert_first_layer_bounds_noalloc in cert.h for the limit and the
+    rules on sharing.  Raises CertError on a bad argument or a batch beyond the built-in limit.
+    """
+    import torch
+    st = stream if stream is not None else torch.cuda.current_stream()
+    out_features, in_features = weight.shape
+    _check(_lib.cert_first_layer_bounds_noalloc(weight.data_ptr(), bias.data_ptr(), out_features, in_features,
+                                                centers.data_ptr(), float(eps), float(clip_lo), float(clip_hi),
+                                                centers.shape[0], lb_out.data_ptr(), ub_out.data_ptr(),
+                                                st.cuda_stream), "cert_first_layer_bounds_noalloc")
 
 
 # C-ABI names, as plain functions
