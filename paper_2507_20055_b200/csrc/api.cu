@@ -22,6 +22,7 @@ struct TcLayer {
     int bn = 0, bn_pad = 0, n_tiles = 0, stages = 0, tmem_cols = 0, smem = 0;
 };
 
+
 struct cert_net {
     int n_layers = 0, max_batch = 0;
     float clip_lo = 0, clip_hi = 0;
@@ -35,7 +36,11 @@ struct cert_net {
     float *buf_lo[2] = {nullptr, nullptr};   // TF32 lo parts for the tensor-core contraction
     bool tc_ok = false;                      // tensor-core path usable on this net
     std::vector<TcLayer> tc;                 // per layer: operand maps and tile plan
-    float *d = nullptr;                      // [max rows] constants of the expressions
+    float *dbuf[2] = {nullptr, nullptr};     // row constants, [d_slots][slot_stride] each, ping-pong
+    int d_slots = 1;                         // slots per buffer (most column tiles of any contraction)
+    long long slot_stride = 0;               // rows of the largest coefficient matrix
+    int sm_count = 148;
+    int tc_bk = 32;                          // floats of K per pipeline stage of the tensor-core kernel
     unsigned char *codes = nullptr;          // [max_batch][n_relu]
     int *status_dev = nullptr;               // sticky device status word
     // host staging for cert_deeppoly_bounds_host
@@ -135,6 +140,10 @@ cert_status_t setup_tensor_core_path(cert_net *net, const cert_layer_desc_t *des
     net->tc_ok = false;
     if (K < 2) return CERT_OK;
     if (!cert::tc_driver_init() || !cert::tc_prepare_kernels()) return CERT_OK;
+    if (const char *e = std::getenv("CERT_TC_BK")) net->tc_bk = (std::atoi(e) == 16) ? 16 : 32;
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, net->device) == cudaSuccess) net->sm_count = prop.multiProcessorCount;
+    const int bk = net->tc_bk;
     if (!dev_alloc_zero(net, &net->buf_lo[0], max_elems) || !dev_alloc_zero(net, &net->buf_lo[1], max_elems))
         return CERT_ERR_OOM;
     std::vector<float> hi, lo;
@@ -159,17 +168,18 @@ cert_status_t setup_tensor_core_path(cert_net *net, const cert_layer_desc_t *des
         if (cudaMemcpy(L.Wt_hi, hi.data(), hi.size() * sizeof(float), cudaMemcpyHostToDevice) != cudaSuccess ||
             cudaMemcpy(L.Wt_lo, lo.data(), lo.size() * sizeof(float), cudaMemcpyHostToDevice) != cudaSuccess)
             return CERT_ERR_CUDA;
-        cert::tc_tile_plan(L.n_in, &T.bn, &T.bn_pad, &T.n_tiles, &T.stages, &T.tmem_cols, &T.smem);
+        cert::tc_tile_plan(L.n_in, bk, &T.bn, &T.bn_pad, &T.n_tiles, &T.stages, &T.tmem_cols, &T.smem);
         if (T.stages < 2) continue;
-        bool ok = cert::tc_make_map(&T.b_hi, L.Wt_hi, L.n_out, L.n_in, L.ld_out, T.bn) &&
-                  cert::tc_make_map(&T.b_lo, L.Wt_lo, L.n_out, L.n_in, L.ld_out, T.bn);
+        bool ok = cert::tc_make_map(&T.b_hi, L.Wt_hi, L.n_out, L.n_in, L.ld_out, T.bn, bk) &&
+                  cert::tc_make_map(&T.b_lo, L.Wt_lo, L.n_out, L.n_in, L.ld_out, T.bn, bk);
         // rows of the largest layer above j
         long long rows_max = 0;
         for (int k = j + 1; k < K; ++k) rows_max = std::max(rows_max, 2LL * net->max_batch * net->layers[k].n_out);
         for (int p = 0; p < 2 && ok; ++p)
-            ok = cert::tc_make_map(&T.a_hi[p], net->buf[p], L.n_out, rows_max, L.ld_out, 128) &&
-                 cert::tc_make_map(&T.a_lo[p], net->buf_lo[p], L.n_out, rows_max, L.ld_out, 128);
+            ok = cert::tc_make_map(&T.a_hi[p], net->buf[p], L.n_out, rows_max, L.ld_out, 128, bk) &&
+                 cert::tc_make_map(&T.a_lo[p], net->buf_lo[p], L.n_out, rows_max, L.ld_out, 128, bk);
         T.usable = ok;
+        if (ok) net->d_slots = std::max(net->d_slots, T.n_tiles);
     }
     net->tc_ok = true;
     return CERT_OK;
@@ -323,14 +333,18 @@ cert_status_t cert_net_create(const cert_layer_desc_t *layers, int n_layers, int
         size_t b = (size_t)max_batch;
         bool ok = dev_alloc_zero(net, &net->l0, b * net->ld0) && dev_alloc_zero(net, &net->u0, b * net->ld0) &&
                   dev_alloc_zero(net, &net->buf[0], max_elems) && dev_alloc_zero(net, &net->buf[1], max_elems) &&
-                  dev_alloc_zero(net, &net->d, max_rows) &&
                   dev_alloc_zero(net, &net->codes, b * std::max(1, net->n_relu)) &&
                   dev_alloc_zero(net, &net->status_dev, 1) &&
                   dev_alloc_zero(net, &net->centers_dev, b * net->n0) &&
                   dev_alloc_zero(net, &net->lb_dev, b * net->n_total) &&
                   dev_alloc_zero(net, &net->ub_dev, b * net->n_total);
         if (!ok) fail = CERT_ERR_OOM;
+        net->slot_stride = (long long)max_rows;
         if (ok) fail = setup_tensor_core_path(net, layers, max_elems);
+        if (fail == CERT_OK &&
+            (!dev_alloc_zero(net, &net->dbuf[0], (size_t)net->d_slots * max_rows) ||
+             !dev_alloc_zero(net, &net->dbuf[1], (size_t)net->d_slots * max_rows)))
+            fail = CERT_ERR_OOM;
     }
     if (fail == CERT_OK) {
         cert::convt_prepare();
@@ -361,20 +375,24 @@ cert_status_t cert_deeppoly_bounds(cert_net_t *net, const float *centers, float 
     cert::launch_first_layer_bounds(net->layers[0], net->l0, net->u0, net->ld0, batch, lb_out, ub_out, n_total, st);
     rec.mark(CERT_CLASS_INPUT);
     if (net->layers[0].relu_after) {
-        cert::launch_relax(net->layers[0], lb_out, ub_out, n_total, batch, net->codes, net->n_relu, st);
+        cert::launch_relax(net->layers[0], lb_out, ub_out, n_total, batch, net->codes, net->n_relu, nullptr, 0, 0,
+                           st);
         rec.mark(CERT_CLASS_RELAX);
     }
     for (int k = 1; k < K; ++k) {
         const LayerDev &Lk = net->layers[k];
         const long long rows = 2LL * batch * Lk.n_out;
-        int cur = 0;
+        int cur = 0;      // coefficient buffer that holds the current expression
+        int dcur = 0;     // constant buffer, and how many of its slots are live
+        int dslots = 1;
+        bool bounds_in_slots = false;
         // Does the back-step through layer j run on the tensor cores?  Its input must then be a TF32 pair.
         auto on_tc = [&](int j) {
             return net->contraction != CERT_CONTRACTION_FFMA && net->tc_ok && net->tc[j].usable;
         };
         // expression over the outputs of layer k-1, pushed through its ReLU
         cert::launch_init_expr(Lk, net->layers[k - 1], batch, net->buf[cur],
-                               on_tc(k - 1) ? net->buf_lo[cur] : nullptr, net->d, st);
+                               on_tc(k - 1) ? net->buf_lo[cur] : nullptr, net->dbuf[dcur], st);
         rec.mark(CERT_CLASS_RELU_STEP);
         for (int j = k - 1; j >= 0; --j) {
             const LayerDev &Lj = net->layers[j];
@@ -387,22 +405,29 @@ cert_status_t cert_deeppoly_bounds(cert_net_t *net, const float *centers, float 
                 a.M = rows; a.K = Lj.n_out; a.n_k = Lk.n_out; a.ld_n = Lj.ld_in;
                 a.bn = T.bn; a.bn_pad = T.bn_pad; a.n_tiles = T.n_tiles; a.stages = T.stages;
                 a.tmem_cols = T.tmem_cols;
-                a.d = net->d; a.status = net->status_dev;
+                a.total_tiles = (int)cert::ceil_div_ll(rows, 128) * T.n_tiles;
+                a.d_in = net->dbuf[dcur]; a.n_slots_in = dslots; a.d_out = net->dbuf[dcur ^ 1];
+                a.slot_stride = net->slot_stride;
+                a.status = net->status_dev;
+                const int grid = std::min(a.total_tiles, net->sm_count);
                 if (j > 0) {
                     const LayerDev &Lb = net->layers[j - 1];
                     a.has_relu = Lb.relu_after;
                     a.out_hi = P; a.out_lo = P_lo;
                     a.lamL = Lb.lamL; a.lamU = Lb.lamU; a.nuU = Lb.nuU; a.bias_below = Lb.bias_n;
-                    cert::launch_gemm_tc(cert::TC_EPI_RELU, T.a_hi[cur], T.a_lo[cur], T.b_hi, T.b_lo, a, T.smem, st);
+                    cert::launch_gemm_tc(cert::TC_EPI_RELU, net->tc_bk, grid, T.a_hi[cur], T.a_lo[cur], T.b_hi,
+                                         T.b_lo, a, T.smem, st);
                 } else {
-                    a.l0 = net->l0; a.u0 = net->u0; a.lb_out = lb_out; a.ub_out = ub_out;
-                    a.n_total = n_total; a.out_off = Lk.out_off;
-                    cert::launch_gemm_tc(cert::TC_EPI_CONCRETIZE, T.a_hi[cur], T.a_lo[cur], T.b_hi, T.b_lo, a, T.smem,
-                                         st);
+                    a.l0 = net->l0; a.u0 = net->u0;
+                    cert::launch_gemm_tc(cert::TC_EPI_CONCRETIZE, net->tc_bk, grid, T.a_hi[cur], T.a_lo[cur],
+                                         T.b_hi, T.b_lo, a, T.smem, st);
+                    bounds_in_slots = true;
                 }
                 rec.mark(CERT_CLASS_AFFINE);
                 paths |= 2;
                 cur ^= 1;
+                dcur ^= 1;
+                dslots = T.n_tiles;
                 continue;
             }
             if (Lj.kind == CERT_LAYER_FC) {
@@ -415,16 +440,19 @@ cert_status_t cert_deeppoly_bounds(cert_net_t *net, const float *centers, float 
             }
             cur ^= 1;
             if (j > 0) {
-                cert::launch_relu_step(net->layers[j - 1], batch, Lk.n_out, P, P_lo, net->d, st);
+                cert::launch_relu_step(net->layers[j - 1], batch, Lk.n_out, P, P_lo, net->dbuf[dcur], dslots,
+                                       net->slot_stride, st);
+                dslots = 1;
                 rec.mark(CERT_CLASS_RELU_STEP);
             } else {
-                cert::launch_concretize(P, net->d, net->l0, net->u0, net->n0, net->ld0, batch, Lk.n_out, lb_out,
-                                        ub_out, n_total, Lk.out_off, st);
+                cert::launch_concretize(P, net->dbuf[dcur], dslots, net->slot_stride, net->l0, net->u0, net->n0,
+                                        net->ld0, batch, Lk.n_out, lb_out, ub_out, n_total, Lk.out_off, st);
                 rec.mark(CERT_CLASS_CONCRETIZE);
             }
         }
-        if (Lk.relu_after) {
-            cert::launch_relax(Lk, lb_out, ub_out, n_total, batch, net->codes, net->n_relu, st);
+        if (Lk.relu_after || bounds_in_slots) {
+            cert::launch_relax(Lk, lb_out, ub_out, n_total, batch, net->codes, net->n_relu,
+                               bounds_in_slots ? net->dbuf[dcur] : nullptr, dslots, net->slot_stride, st);
             rec.mark(CERT_CLASS_RELAX);
         }
     }

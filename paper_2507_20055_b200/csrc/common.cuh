@@ -52,8 +52,12 @@ void launch_first_layer_bounds(const LayerDev &L, const float *l0, const float *
                                float *lb_out, float *ub_out, int n_total, cudaStream_t st);
 
 // Relu transformer: relaxation (lamL, lamU, nuU) and branch code from (l, u).
-void launch_relax(const LayerDev &L, const float *lb_out, const float *ub_out, int n_total, int batch,
-                  unsigned char *codes, int n_relu, cudaStream_t st);
+// With `slots` != nullptr the bounds are first summed from n_slots partial sums per row
+// (rows ordered (box, side, neuron), slot s at slots + s*slot_stride) and stored to lb_out / ub_out;
+// the relaxation itself is skipped for a layer without a ReLU.
+void launch_relax(const LayerDev &L, float *lb_out, float *ub_out, int n_total, int batch,
+                  unsigned char *codes, int n_relu, const float *slots, int n_slots, long long slot_stride,
+                  cudaStream_t st);
 
 // Start of the back-substitution for layer k: the expression of neuron i is
 // row i of W_k (the same for every box and both sides) and the constant b_k[i];
@@ -66,12 +70,13 @@ void launch_init_expr(const LayerDev &Lk, const LayerDev &Lbelow, int batch, flo
 
 // ReLU back-step in place on P [rows][ld] (expression over the outputs of
 // layer `Lj`, i.e. over its ReLU neurons if it has one), plus d += Q.b_j.
-void launch_relu_step(const LayerDev &Lj, int batch, int n_k, float *P, float *P_lo, float *d,
-                      cudaStream_t st);
+// The row constant comes in as the sum of n_slots slots of d and leaves in slot 0.
+void launch_relu_step(const LayerDev &Lj, int batch, int n_k, float *P, float *P_lo, float *d, int n_slots,
+                      long long slot_stride, cudaStream_t st);
 
 // map(simplify_lower/upper): rows of P [rows][ld0] against the box.
-void launch_concretize(const float *P, const float *d, const float *l0, const float *u0, int n0, int ld0,
-                       int batch, int n_k, float *lb_out, float *ub_out, int n_total, int out_off,
+void launch_concretize(const float *P, const float *d, int n_slots, long long slot_stride, const float *l0,
+                       const float *u0, int n0, int ld0, int batch, int n_k, float *lb_out, float *ub_out, int n_total, int out_off,
                        cudaStream_t st);
 
 // C[M][ldc] = A[M][lda] * B[K][ldb]  (fp32 FMA units).  Columns up to ldc are

@@ -93,18 +93,39 @@ __global__ void first_layer_kernel(const float *__restrict__ W, const float *__r
     }
 }
 
-// Relu transformer.  One thread per (box, padded neuron).
-__global__ void relax_kernel(const float *__restrict__ lb_out, const float *__restrict__ ub_out, int n_total,
+// Sum of the slots that hold a row's constant (or bound), in slot order.
+__device__ __forceinline__ float slot_sum(const float *__restrict__ d, int n_slots, long long stride,
+                                          long long r) {
+    float v = d[r];
+    for (int s = 1; s < n_slots; ++s) v += d[(size_t)s * stride + r];
+    return v;
+}
+
+// Relu transformer.  One thread per (box, padded neuron).  With `slots` the
+// bounds are first assembled from the per-column-tile sums the concretising
+// contraction left (rows ordered (box, side, neuron)) and written to lb_out / ub_out.
+__global__ void relax_kernel(float *__restrict__ lb_out, float *__restrict__ ub_out, int n_total,
                              int out_off, int n, int ld, int batch, float *__restrict__ lamL,
                              float *__restrict__ lamU, float *__restrict__ nuU,
-                             unsigned char *__restrict__ codes, int n_relu, int relu_off) {
+                             unsigned char *__restrict__ codes, int n_relu, int relu_off,
+                             const float *__restrict__ slots, int n_slots, long long slot_stride,
+                             int do_relax) {
     long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (idx >= (long long)batch * ld) return;
     int b = (int)(idx / ld), t = (int)(idx % ld);
     float ll = 0.0f, lu = 0.0f, nu = 0.0f;
     if (t < n) {
-        float l = lb_out[(size_t)b * n_total + out_off + t];
-        float u = ub_out[(size_t)b * n_total + out_off + t];
+        float l, u;
+        if (slots) {
+            l = slot_sum(slots, n_slots, slot_stride, (2LL * b) * n + t);
+            u = slot_sum(slots, n_slots, slot_stride, (2LL * b + 1) * n + t);
+            lb_out[(size_t)b * n_total + out_off + t] = l;
+            ub_out[(size_t)b * n_total + out_off + t] = u;
+        } else {
+            l = lb_out[(size_t)b * n_total + out_off + t];
+            u = ub_out[(size_t)b * n_total + out_off + t];
+        }
+        if (!do_relax) return;
         bool pick_one = (__fadd_rn(l, u) >= 0.0f);   // relu_n
         ll = pick_one ? 1.0f : 0.0f;
         unsigned char code;
@@ -120,6 +141,7 @@ __global__ void relax_kernel(const float *__restrict__ lb_out, const float *__re
         }
         codes[(size_t)b * n_relu + relu_off + t] = code;
     }
+    if (!do_relax) return;
     lamL[idx] = ll;
     lamU[idx] = lu;
     nuU[idx] = nu;
@@ -141,8 +163,8 @@ __device__ __forceinline__ float weight_elem(const float *__restrict__ W, int ki
 template <bool FROM_WEIGHTS>
 __global__ void relu_step_kernel(const float *__restrict__ Wk, int kind_k, ConvGeom gk, int ldw_k,
                                  const float *__restrict__ bias_k, float *__restrict__ P,
-                                 float *__restrict__ P_lo, float *__restrict__ d,
-                                 long long rows, int n_k, int n, int ld, int has_relu,
+                                 float *__restrict__ P_lo, float *__restrict__ d, int n_slots,
+                                 long long slot_stride, long long rows, int n_k, int n, int ld, int has_relu,
                                  const float *__restrict__ lamL, const float *__restrict__ lamU,
                                  const float *__restrict__ nuU, const float *__restrict__ bias_below) {
     long long r = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
@@ -171,11 +193,11 @@ __global__ void relu_step_kernel(const float *__restrict__ Wk, int kind_k, ConvG
         }
     }
     dacc = warp_sum(dacc);
-    if (lane == 0) d[r] = (FROM_WEIGHTS ? bias_k[i] : d[r]) + dacc;
+    if (lane == 0) d[r] = (FROM_WEIGHTS ? bias_k[i] : slot_sum(d, n_slots, slot_stride, r)) + dacc;
 }
 
-__global__ void concretize_kernel(const float *__restrict__ P, const float *__restrict__ d,
-                                  const float *__restrict__ l0, const float *__restrict__ u0, int n0, int ld0,
+__global__ void concretize_kernel(const float *__restrict__ P, const float *__restrict__ d, int n_slots,
+                                  long long slot_stride, const float *__restrict__ l0, const float *__restrict__ u0, int n0, int ld0,
                                   long long rows, int n_k, float *__restrict__ lb_out, float *__restrict__ ub_out,
                                   int n_total, int out_off) {
     long long r = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
@@ -194,7 +216,7 @@ __global__ void concretize_kernel(const float *__restrict__ P, const float *__re
     }
     acc = warp_sum(acc);
     if (lane == 0) {
-        float v = d[r] + acc;
+        float v = slot_sum(d, n_slots, slot_stride, r) + acc;
         (upper ? ub_out : lb_out)[(size_t)b * n_total + out_off + i] = v;
     }
 }
@@ -219,35 +241,37 @@ void launch_first_layer_bounds(const LayerDev &L, const float *l0, const float *
         n_total, L.out_off);
 }
 
-void launch_relax(const LayerDev &L, const float *lb_out, const float *ub_out, int n_total, int batch,
-                  unsigned char *codes, int n_relu, cudaStream_t st) {
+void launch_relax(const LayerDev &L, float *lb_out, float *ub_out, int n_total, int batch,
+                  unsigned char *codes, int n_relu, const float *slots, int n_slots, long long slot_stride,
+                  cudaStream_t st) {
     long long n = (long long)batch * L.ld_out;
     relax_kernel<<<(unsigned)ceil_div_ll(n, 256), 256, 0, st>>>(lb_out, ub_out, n_total, L.out_off, L.n_out,
                                                                L.ld_out, batch, L.lamL, L.lamU, L.nuU, codes,
-                                                               n_relu, L.relu_off);
+                                                               n_relu, L.relu_off, slots, n_slots, slot_stride,
+                                                               L.relu_after);
 }
 
 void launch_init_expr(const LayerDev &Lk, const LayerDev &Lb, int batch, float *Q, float *Q_lo, float *d,
                       cudaStream_t st) {
     long long rows = 2LL * batch * Lk.n_out;
     relu_step_kernel<true><<<grid_for_warps(rows), kWarpsPerBlock * 32, 0, st>>>(
-        Lk.W, Lk.kind, geom_of(Lk), Lk.ld_in, Lk.bias_n, Q, Q_lo, d, rows, Lk.n_out, Lb.n_out, Lb.ld_out,
+        Lk.W, Lk.kind, geom_of(Lk), Lk.ld_in, Lk.bias_n, Q, Q_lo, d, 1, 0, rows, Lk.n_out, Lb.n_out, Lb.ld_out,
         Lb.relu_after, Lb.lamL, Lb.lamU, Lb.nuU, Lb.bias_n);
 }
 
-void launch_relu_step(const LayerDev &Lj, int batch, int n_k, float *P, float *P_lo, float *d,
-                      cudaStream_t st) {
+void launch_relu_step(const LayerDev &Lj, int batch, int n_k, float *P, float *P_lo, float *d, int n_slots,
+                      long long slot_stride, cudaStream_t st) {
     long long rows = 2LL * batch * n_k;
     relu_step_kernel<false><<<grid_for_warps(rows), kWarpsPerBlock * 32, 0, st>>>(
-        nullptr, 0, ConvGeom{}, 0, nullptr, P, P_lo, d, rows, n_k, Lj.n_out, Lj.ld_out, Lj.relu_after, Lj.lamL,
+        nullptr, 0, ConvGeom{}, 0, nullptr, P, P_lo, d, n_slots, slot_stride, rows, n_k, Lj.n_out, Lj.ld_out, Lj.relu_after, Lj.lamL,
         Lj.lamU, Lj.nuU, Lj.bias_n);
 }
 
-void launch_concretize(const float *P, const float *d, const float *l0, const float *u0, int n0, int ld0,
-                       int batch, int n_k, float *lb_out, float *ub_out, int n_total, int out_off,
+void launch_concretize(const float *P, const float *d, int n_slots, long long slot_stride, const float *l0,
+                       const float *u0, int n0, int ld0, int batch, int n_k, float *lb_out, float *ub_out, int n_total, int out_off,
                        cudaStream_t st) {
     long long rows = 2LL * batch * n_k;
-    concretize_kernel<<<grid_for_warps(rows), kWarpsPerBlock * 32, 0, st>>>(P, d, l0, u0, n0, ld0, rows, n_k,
+    concretize_kernel<<<grid_for_warps(rows), kWarpsPerBlock * 32, 0, st>>>(P, d, n_slots, slot_stride, l0, u0, n0, ld0, rows, n_k,
                                                                           lb_out, ub_out, n_total, out_off);
 }
 

@@ -107,15 +107,16 @@ __device__ __forceinline__ float tf32_round(float x) {
     return __uint_as_float(r);
 }
 
-// Shared-memory matrix descriptor: K-major tile, rows of 128 bytes, 128-byte swizzle,
-// 8-row groups 1024 bytes apart.
-__device__ __forceinline__ uint64_t make_desc_sw128(uint32_t smem_addr) {
+// Shared-memory matrix descriptor of a K-major tile whose rows are ROW_BYTES long
+// (128 -> 128-byte swizzle, 64 -> 64-byte swizzle); 8-row groups are 8*ROW_BYTES apart.
+template <int ROW_BYTES>
+__device__ __forceinline__ uint64_t make_desc(uint32_t smem_addr) {
     uint64_t d = 0;
     d |= (uint64_t)((smem_addr >> 4) & 0x3FFF);
-    d |= (uint64_t)1 << 16;             // leading byte offset (unused for swizzled K-major), in 16-byte units
-    d |= (uint64_t)(1024 >> 4) << 32;   // stride byte offset between 8-row groups
-    d |= (uint64_t)1 << 46;             // descriptor version for sm_100
-    d |= (uint64_t)2 << 61;             // SWIZZLE_128B
+    d |= (uint64_t)1 << 16;                        // leading byte offset (unused for swizzled K-major)
+    d |= (uint64_t)((8 * ROW_BYTES) >> 4) << 32;   // stride byte offset between 8-row groups
+    d |= (uint64_t)1 << 46;                        // descriptor version for sm_100
+    d |= (uint64_t)(ROW_BYTES == 128 ? 2 : 4) << 61;   // SWIZZLE_128B / SWIZZLE_64B
     return d;
 }
 
@@ -128,25 +129,30 @@ struct __align__(8) Barriers {
     uint32_t abort_flag;
 };
 
-template <int EPI>
+// Persistent kernel: CTA c works on tiles c, c + gridDim.x, ...; tile t covers rows
+// [128*(t / n_tiles), +128) and column tile t % n_tiles, so the CTAs that run at the same
+// time share row panels and the A operand is fetched from DRAM once.
+template <int EPI, int BK>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_constant__ CUtensorMap map_a_lo,
                const __grid_constant__ CUtensorMap map_b_hi, const __grid_constant__ CUtensorMap map_b_lo,
                const TcArgs a) {
+    constexpr int ROW_BYTES = BK * 4;
+    constexpr int KSTEPS = BK / 8;
     extern __shared__ uint8_t smem_raw[];
-    // tiles need 1024-byte alignment for the 128-byte swizzle
+    // tiles are aligned to 1024 bytes (a whole swizzle pattern)
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const int BN = a.bn;
     const int stages = a.stages;
-    const uint32_t a_tile_bytes = BM * 128;
-    const uint32_t b_tile_bytes = (uint32_t)BN * 128;
+    const uint32_t a_tile_bytes = BM * ROW_BYTES;
+    const uint32_t b_tile_bytes = (uint32_t)BN * ROW_BYTES;
     const uint32_t stage_bytes = 2 * a_tile_bytes + 2 * b_tile_bytes;
     Barriers *bars = reinterpret_cast<Barriers *>(smem + (size_t)stages * stage_bytes);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const long long row0 = (long long)blockIdx.x * BM;
-    const int num_kb = (a.K + 31) / 32;
+    const int num_kb = (a.K + BK - 1) / BK;
     const int n_tiles = a.n_tiles;
+    const int total_tiles = a.total_tiles;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < stages; ++s) {
@@ -180,18 +186,19 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_consta
             int s = 0;
             uint32_t phase = 0;
             bool ok = true;
-            int armed = 0;      // stages whose loads were issued
-            for (int nt = 0; nt < n_tiles && ok; ++nt) {
+            int armed = 0;      // stage loads issued so far
+            for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+                const int row0 = (t / n_tiles) * BM;
+                const int col0 = (t % n_tiles) * BN;
                 for (int kb = 0; kb < num_kb; ++kb) {
                     if (!mbar_wait(&bars->empty[s], phase ^ 1) || *abort_flag) { ok = false; break; }
                     uint8_t *st = smem + (size_t)s * stage_bytes;
                     mbar_arrive_expect_tx(&bars->full[s], stage_bytes);
-                    const int kx = kb * 32;
-                    tma_load_2d(smem_u32(st), &map_a_hi, &bars->full[s], kx, (int)row0);
-                    tma_load_2d(smem_u32(st + a_tile_bytes), &map_a_lo, &bars->full[s], kx, (int)row0);
-                    tma_load_2d(smem_u32(st + 2 * a_tile_bytes), &map_b_hi, &bars->full[s], kx, nt * BN);
-                    tma_load_2d(smem_u32(st + 2 * a_tile_bytes + b_tile_bytes), &map_b_lo, &bars->full[s], kx,
-                                nt * BN);
+                    const int kx = kb * BK;
+                    tma_load_2d(smem_u32(st), &map_a_hi, &bars->full[s], kx, row0);
+                    tma_load_2d(smem_u32(st + a_tile_bytes), &map_a_lo, &bars->full[s], kx, row0);
+                    tma_load_2d(smem_u32(st + 2 * a_tile_bytes), &map_b_hi, &bars->full[s], kx, col0);
+                    tma_load_2d(smem_u32(st + 2 * a_tile_bytes + b_tile_bytes), &map_b_lo, &bars->full[s], kx, col0);
                     ++armed;
                     if (++s == stages) { s = 0; phase ^= 1; }
                 }
@@ -217,9 +224,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_consta
             int s = 0;
             uint32_t phase = 0;
             bool ok = true;
-            for (int nt = 0; nt < n_tiles && ok; ++nt) {
-                const int acc = nt & 1;
-                const uint32_t acc_phase = (nt >> 1) & 1;
+            int lt = 0;
+            for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++lt) {
+                const int acc = lt & 1;
+                const uint32_t acc_phase = (lt >> 1) & 1;
                 if (!mbar_wait(&bars->acc_empty[acc], acc_phase ^ 1) || *abort_flag) { ok = false; break; }
                 tcgen05_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(acc * a.bn_pad);
@@ -227,12 +235,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_consta
                     if (!mbar_wait(&bars->full[s], phase) || *abort_flag) { ok = false; break; }
                     tcgen05_fence_after();
                     const uint32_t st = smem_u32(smem + (size_t)s * stage_bytes);
-                    const uint64_t da_hi = make_desc_sw128(st);
-                    const uint64_t da_lo = make_desc_sw128(st + a_tile_bytes);
-                    const uint64_t db_hi = make_desc_sw128(st + 2 * a_tile_bytes);
-                    const uint64_t db_lo = make_desc_sw128(st + 2 * a_tile_bytes + b_tile_bytes);
+                    const uint64_t da_hi = make_desc<ROW_BYTES>(st);
+                    const uint64_t da_lo = make_desc<ROW_BYTES>(st + a_tile_bytes);
+                    const uint64_t db_hi = make_desc<ROW_BYTES>(st + 2 * a_tile_bytes);
+                    const uint64_t db_lo = make_desc<ROW_BYTES>(st + 2 * a_tile_bytes + b_tile_bytes);
 #pragma unroll
-                    for (int k = 0; k < 4; ++k) {
+                    for (int k = 0; k < KSTEPS; ++k) {
                         const uint64_t ko = (uint64_t)(k * 2);   // 8 floats = 32 bytes = 2 x 16-byte units
                         mma_tf32(d_tmem, da_lo + ko, db_hi + ko, idesc, (kb | k) ? 1u : 0u);
                         mma_tf32(d_tmem, da_hi + ko, db_lo + ko, idesc, 1u);
@@ -251,29 +259,30 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_consta
     } else {
         // ------------------------------------------------------------ epilogue
         const int quarter = warp & 3;                       // TMEM lane quarter this warp may read
-        const long long r = row0 + quarter * 32 + lane;
-        const bool row_ok = r < a.M;
-        const long long rr = row_ok ? r : 0;
-        const int b = (int)(rr / (2LL * a.n_k));
-        const int upper = (int)((rr / a.n_k) & 1);
-        const int i = (int)(rr % a.n_k);
-        float dacc = 0.0f;
         bool ok = true;
-        const size_t relax_row = (size_t)b * a.ld_n;
-        for (int nt = 0; nt < n_tiles && ok; ++nt) {
-            const int acc = nt & 1;
-            const uint32_t acc_phase = (nt >> 1) & 1;
+        int lt = 0;
+        for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++lt) {
+            const int nt = t % n_tiles;
+            const long long r = (long long)(t / n_tiles) * BM + quarter * 32 + lane;
+            const bool row_ok = r < a.M;
+            const long long rr = row_ok ? r : 0;
+            const int b = (int)(rr / (2LL * a.n_k));
+            const int upper = (int)((rr / a.n_k) & 1);
+            const size_t relax_row = (size_t)b * a.ld_n;
+            float dacc = 0.0f;
+            const int acc = lt & 1;
+            const uint32_t acc_phase = (lt >> 1) & 1;
             if (!mbar_wait(&bars->acc_full[acc], acc_phase) || *abort_flag) { ok = false; break; }
             tcgen05_fence_after();
             const uint32_t t_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * a.bn_pad);
+            const int col_end = min((nt + 1) * BN, a.ld_n);   // columns this tile owns
             for (int c0 = 0; c0 < BN; c0 += 32) {
                 const int col0 = nt * BN + c0;
-                if (col0 >= a.ld_n) break;                  // warp-uniform
+                if (col0 >= col_end) break;                  // warp-uniform
                 uint32_t v[32];
                 __syncwarp();
                 tmem_ld32(t_addr + (uint32_t)c0, v);
                 tmem_ld_wait();
-                const int col_end = min((nt + 1) * BN, a.ld_n);   // columns this tile owns
                 if (!row_ok) {
                     // rows past the end of the matrix: nothing to store
                 } else if (EPI == TC_EPI_RELU) {
@@ -342,13 +351,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_consta
             tcgen05_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&bars->acc_empty[acc]);
-        }
-        if (ok && row_ok) {
-            if (EPI == TC_EPI_RELU) {
-                a.d[r] = a.d[r] + dacc;
-            } else {
-                float *out = upper ? a.ub_out : a.lb_out;
-                out[(size_t)b * a.n_total + a.out_off + i] = a.d[r] + dacc;
+            // This tile's share of the row constant (of the bound, for the concretising
+            // epilogue) goes to slot nt; the tile of column 0 also carries the constant so far.
+            if (row_ok) {
+                float tot = dacc;
+                if (nt == 0) {
+                    float prev = 0.0f;
+                    for (int sidx = 0; sidx < a.n_slots_in; ++sidx) prev += a.d_in[(size_t)sidx * a.slot_stride + r];
+                    tot += prev;
+                }
+                a.d_out[(size_t)nt * a.slot_stride + r] = tot;
             }
         }
         if (!ok && lane == 0) atomicExch(a.status, 1);
@@ -386,41 +398,45 @@ bool tc_driver_init() {
 }
 
 bool tc_prepare_kernels() {
-    cudaError_t e1 = cudaFuncSetAttribute(gemm_tc_kernel<TC_EPI_RELU>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                          kTcSmemMax);
-    cudaError_t e2 = cudaFuncSetAttribute(gemm_tc_kernel<TC_EPI_CONCRETIZE>,
-                                          cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemMax);
-    if (e1 != cudaSuccess || e2 != cudaSuccess) {
-        cudaGetLastError();
-        return false;
-    }
+    cudaError_t e[4];
+    e[0] = cudaFuncSetAttribute(gemm_tc_kernel<TC_EPI_RELU, 32>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemMax);
+    e[1] = cudaFuncSetAttribute(gemm_tc_kernel<TC_EPI_CONCRETIZE, 32>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemMax);
+    e[2] = cudaFuncSetAttribute(gemm_tc_kernel<TC_EPI_RELU, 16>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemMax);
+    e[3] = cudaFuncSetAttribute(gemm_tc_kernel<TC_EPI_CONCRETIZE, 16>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemMax);
+    for (int i = 0; i < 4; ++i)
+        if (e[i] != cudaSuccess) {
+            cudaGetLastError();
+            return false;
+        }
     return true;
 }
 
-// 2D fp32 tensor [outer][inner] with row pitch `pitch_floats`; box = 32 floats x box_outer rows, 128-byte swizzle.
+// 2D fp32 tensor [outer][inner] with row pitch `pitch_floats`; box = bk floats x box_outer rows,
+// swizzle span = one box row (128 bytes for bk = 32, 64 bytes for bk = 16).
 bool tc_make_map(TcMap *m, const float *base, long long inner, long long outer, long long pitch_floats,
-                 int box_outer) {
+                 int box_outer, int bk) {
     if (!g_encode) return false;
     static_assert(sizeof(TcMap) == sizeof(CUtensorMap), "tensor map size");
     cuuint64_t dims[2] = {(cuuint64_t)inner, (cuuint64_t)outer};
     cuuint64_t strides[1] = {(cuuint64_t)pitch_floats * sizeof(float)};
-    cuuint32_t box[2] = {32u, (cuuint32_t)box_outer};
+    cuuint32_t box[2] = {(cuuint32_t)bk, (cuuint32_t)box_outer};
     cuuint32_t estr[2] = {1u, 1u};
     CUresult r = g_encode(reinterpret_cast<CUtensorMap *>(m), CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2,
                           const_cast<float *>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                          CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+                          bk == 32 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B,
+                          CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS;
 }
 
-void tc_tile_plan(int N, int *bn, int *bn_pad, int *n_tiles, int *stages, int *tmem_cols, int *smem_bytes) {
+void tc_tile_plan(int N, int bk, int *bn, int *bn_pad, int *n_tiles, int *stages, int *tmem_cols,
+                  int *smem_bytes) {
     int nt = (N + 255) / 256;
     int b = ((N + nt - 1) / nt + 15) / 16 * 16;
     if (b < 16) b = 16;
     *bn = b;
     *bn_pad = (b + 31) / 32 * 32;
     *n_tiles = nt;
-    int stage_bytes = 2 * BM * 128 + 2 * b * 128;
+    int stage_bytes = (2 * BM + 2 * b) * bk * 4;
     int st = (kTcSmemMax - 2048) / stage_bytes;
     if (st > 8) st = 8;
     *stages = st;
@@ -430,17 +446,23 @@ void tc_tile_plan(int N, int *bn, int *bn_pad, int *n_tiles, int *stages, int *t
     *smem_bytes = st * stage_bytes + 2048;
 }
 
-void launch_gemm_tc(int epi, const TcMap &a_hi, const TcMap &a_lo, const TcMap &b_hi, const TcMap &b_lo,
-                    const TcArgs &args, int smem_bytes, cudaStream_t st) {
-    unsigned grid = (unsigned)ceil_div_ll(args.M, BM);
+void launch_gemm_tc(int epi, int bk, int grid, const TcMap &a_hi, const TcMap &a_lo, const TcMap &b_hi,
+                    const TcMap &b_lo, const TcArgs &args, int smem_bytes, cudaStream_t st) {
     const CUtensorMap &ah = reinterpret_cast<const CUtensorMap &>(a_hi);
     const CUtensorMap &al = reinterpret_cast<const CUtensorMap &>(a_lo);
     const CUtensorMap &bh = reinterpret_cast<const CUtensorMap &>(b_hi);
     const CUtensorMap &bl = reinterpret_cast<const CUtensorMap &>(b_lo);
-    if (epi == TC_EPI_RELU)
-        gemm_tc_kernel<TC_EPI_RELU><<<grid, kThreads, smem_bytes, st>>>(ah, al, bh, bl, args);
-    else
-        gemm_tc_kernel<TC_EPI_CONCRETIZE><<<grid, kThreads, smem_bytes, st>>>(ah, al, bh, bl, args);
+    if (bk == 32) {
+        if (epi == TC_EPI_RELU)
+            gemm_tc_kernel<TC_EPI_RELU, 32><<<grid, kThreads, smem_bytes, st>>>(ah, al, bh, bl, args);
+        else
+            gemm_tc_kernel<TC_EPI_CONCRETIZE, 32><<<grid, kThreads, smem_bytes, st>>>(ah, al, bh, bl, args);
+    } else {
+        if (epi == TC_EPI_RELU)
+            gemm_tc_kernel<TC_EPI_RELU, 16><<<grid, kThreads, smem_bytes, st>>>(ah, al, bh, bl, args);
+        else
+            gemm_tc_kernel<TC_EPI_CONCRETIZE, 16><<<grid, kThreads, smem_bytes, st>>>(ah, al, bh, bl, args);
+    }
 }
 
 }  // namespace cert
