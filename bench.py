@@ -163,11 +163,14 @@ def main():
         dist.barrier()
     from paper_2507_20055_b200 import binding
 
-    # Boxes are independent: each rank bounds its own batch of the same shape (weak scaling),
-    # with its own seed; the weights are replicated.  No collective on the data path.
+    # Boxes are independent: the job's boxes (per-GPU batch x ranks: weak scaling) are split with
+    # box_shard, the weights are replicated, and there is no collective on the data path.
     if world > 1:
-        w = wl.make_config(args.config, batch=args.batch)
-        w.centers = wl.centers_uniform(w.batch, w.centers.shape[1], seed=0, stream=1000 + rank)
+        from paper_2507_20055_b200 import sharding
+        per_gpu = w.batch
+        everything = wl.centers_uniform(per_gpu * world, w.centers.shape[1], seed=0)
+        w.centers = sharding.shard_centers(everything, rank, world)
+        assert w.batch == per_gpu
     B = w.batch
     net = binding.CertNet(w.layers, B, w.clip_lo, w.clip_hi)
     mode = {"auto": binding.CONTRACTION_AUTO, "ffma": binding.CONTRACTION_FFMA, "tc": binding.CONTRACTION_TC3XTF32}

@@ -176,20 +176,44 @@ __global__ void relu_step_kernel(const float *__restrict__ Wk, int kind_k, ConvG
     float *prow = P + (size_t)r * ld;
     const float *ll = lamL + (size_t)b * ld, *lu = lamU + (size_t)b * ld, *nu = nuU + (size_t)b * ld;
     float dacc = 0.0f;
-    for (int t = lane; t < ld; t += 32) {
-        float q = 0.0f;
-        if (t < n) {
-            float c = FROM_WEIGHTS ? weight_elem(Wk, kind_k, gk, ldw_k, i, t) : prow[t];
-            q = has_relu ? relu_backstep(c, upper, ll[t], lu[t], nu[t], dacc) : c;
-            dacc = fmaf(q, bias_below[t], dacc);
+    // four consecutive columns per lane: 16-byte accesses (every row pitch is a multiple of 32 floats)
+    for (int t = lane * 4; t < ld; t += 128) {
+        float c[4], q[4];
+        if (FROM_WEIGHTS && kind_k != CERT_LAYER_FC) {
+#pragma unroll
+            for (int e = 0; e < 4; ++e) c[e] = (t + e < n) ? weight_elem(Wk, kind_k, gk, ldw_k, i, t + e) : 0.0f;
+        } else {
+            const float4 c4 = *reinterpret_cast<const float4 *>(FROM_WEIGHTS ? Wk + (size_t)i * ldw_k + t : prow + t);
+            c[0] = c4.x; c[1] = c4.y; c[2] = c4.z; c[3] = c4.w;
         }
+        const float4 bz4 = *reinterpret_cast<const float4 *>(bias_below + t);
+        const float bz[4] = {bz4.x, bz4.y, bz4.z, bz4.w};
+        if (has_relu) {
+            const float4 l4 = *reinterpret_cast<const float4 *>(ll + t);
+            const float4 u4 = *reinterpret_cast<const float4 *>(lu + t);
+            const float4 n4 = *reinterpret_cast<const float4 *>(nu + t);
+            const float la[4] = {l4.x, l4.y, l4.z, l4.w}, ua[4] = {u4.x, u4.y, u4.z, u4.w},
+                        na[4] = {n4.x, n4.y, n4.z, n4.w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) q[e] = (t + e < n) ? relu_backstep(c[e], upper, la[e], ua[e], na[e], dacc) : 0.0f;
+        } else {
+#pragma unroll
+            for (int e = 0; e < 4; ++e) q[e] = (t + e < n) ? c[e] : 0.0f;
+        }
+#pragma unroll
+        for (int e = 0; e < 4; ++e) dacc = fmaf(q[e], bz[e], dacc);
         if (P_lo) {
             // operand form of the tensor-core contraction: q = hi + lo, both TF32
-            float h = tf32_round(q);
-            prow[t] = h;
-            P_lo[(size_t)r * ld + t] = tf32_round(q - h);
+            float h[4], l[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                h[e] = tf32_round(q[e]);
+                l[e] = tf32_round(q[e] - h[e]);
+            }
+            *reinterpret_cast<float4 *>(prow + t) = make_float4(h[0], h[1], h[2], h[3]);
+            *reinterpret_cast<float4 *>(P_lo + (size_t)r * ld + t) = make_float4(l[0], l[1], l[2], l[3]);
         } else {
-            prow[t] = q;
+            *reinterpret_cast<float4 *>(prow + t) = make_float4(q[0], q[1], q[2], q[3]);
         }
     }
     dacc = warp_sum(dacc);
