@@ -98,6 +98,22 @@ def oracle_sample(w, n_boxes, threads=None):
             "sample": f"first {n_boxes} of {w.batch} boxes of {w.name}, one box per thread, {dt:.1f} s wall"}, dt
 
 
+def backstep_flops_by_class(layers, batch):
+    """Algorithmic flops of one call's back-steps: for every layer k, 2*batch*n_k rows go through every
+    earlier layer j; an FC step costs 2*n_j*n_{j-1} per row, a conv step 2*n_j*c_in*kh*kw (dense maps)."""
+    out = {"affine": 0.0, "conv": 0.0}
+    for k in range(1, len(layers)):
+        rows = 2.0 * batch * layers[k].n_out
+        for j in range(k):
+            L = layers[j]
+            if L.kind == "fc":
+                out["affine"] += rows * 2.0 * L.n_out * L.n_in
+            else:
+                _, c_in, kh, kw = L.weight.shape
+                out["conv"] += rows * 2.0 * L.n_out * c_in * kh * kw
+    return out
+
+
 def run_reference(args, w):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
@@ -255,23 +271,26 @@ def main():
     if rank == 0:
         peaks = load_peaks()
         flops_call = net.backstep_flops(B)
-        con_ms = cls_ms.get("affine", 0.0) + cls_ms.get("conv", 0.0)
-        con_n = cls_n.get("affine", 0) + cls_n.get("conv", 0)
+        fl = backstep_flops_by_class(w.layers, B)
+        assert abs(fl["affine"] + fl["conv"] - flops_call) <= 1e-6 * flops_call
+        # the dominant kernel class: FC back-steps (tensor cores unless --contraction ffma) or conv back-steps (FMA units)
         dom = "affine" if cls_ms.get("affine", 0.0) >= cls_ms.get("conv", 0.0) else "conv"
-        achieved = flops_call * args.steps / (con_ms / 1000.0) / 1e12 if con_ms > 0 else None
+        dom_ms, dom_n = cls_ms.get(dom, 0.0), cls_n.get(dom, 0)
+        achieved = fl[dom] * args.steps / (dom_ms / 1000.0) / 1e12 if dom_ms > 0 else None
         sm_max = (clocks or {}).get("sm_max_mhz") or 1965.0
         ffma_peak = 148 * 128 * 2 * sm_max * 1e6 / 1e12
         # fp32-accurate work on the tensor cores costs three TF32 products per multiply-add;
         # TF32 dense peak = measured bf16 (sustained: the kernel runs inside a long step) x 1/2 (nominal ratio)
         tc_peak = peaks["bf16_tflops_sustained"] * 0.5 / 3.0
-        used_tc = bool(net.last_contraction_paths() & 2)
+        used_tc = dom == "affine" and bool(net.last_contraction_paths() & 2)
         roof = {"bound": "tensor" if used_tc else "alu",
                 "achieved": achieved, "peak": tc_peak if used_tc else ffma_peak, "unit": "TFLOP/s",
                 "frac": (achieved / (tc_peak if used_tc else ffma_peak)) if achieved else None,
                 "traffic": None,
-                "kernel": dom + " back-step", "launches_per_step": con_n // max(1, args.steps),
-                "avg_launch_ms": con_ms / con_n if con_n else None,
-                "flops_per_step": flops_call, "peak_source": peaks["source"],
+                "kernel": dom + " back-step", "launches_per_step": dom_n // max(1, args.steps),
+                "avg_launch_ms": dom_ms / dom_n if dom_n else None,
+                "flops_per_step": fl[dom], "flops_per_step_all_backsteps": flops_call,
+                "peak_source": peaks["source"],
                 "peak_note": ("bf16_tflops_sustained/2/3 (3xTF32)" if used_tc else "148 SM x 128 FMA x 2 x sm_max_mhz"),
                 "class_ms_per_step": {k: v / args.steps for k, v in cls_ms.items()}}
         out = {

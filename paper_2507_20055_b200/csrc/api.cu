@@ -56,7 +56,7 @@ struct cert_net {
 };
 
 namespace cert {
-size_t convt_smem_bytes(const LayerDev &L);
+bool convt_supported(const LayerDev &L);
 void convt_prepare();
 }  // namespace cert
 
@@ -141,8 +141,6 @@ cert_status_t setup_tensor_core_path(cert_net *net, const cert_layer_desc_t *des
     if (K < 2) return CERT_OK;
     if (!cert::tc_driver_init() || !cert::tc_prepare_kernels()) return CERT_OK;
     if (const char *e = std::getenv("CERT_TC_BK")) net->tc_bk = (std::atoi(e) == 16) ? 16 : 32;
-    cudaDeviceProp prop;
-    if (cudaGetDeviceProperties(&prop, net->device) == cudaSuccess) net->sm_count = prop.multiProcessorCount;
     const int bk = net->tc_bk;
     if (!dev_alloc_zero(net, &net->buf_lo[0], max_elems) || !dev_alloc_zero(net, &net->buf_lo[1], max_elems))
         return CERT_ERR_OOM;
@@ -233,6 +231,11 @@ cert_status_t cert_net_create(const cert_layer_desc_t *layers, int n_layers, int
     cert_net *net = new (std::nothrow) cert_net;
     if (!net) return CERT_ERR_OOM;
     net->device = dev;
+    {
+        cudaDeviceProp prop;
+        if (cudaGetDeviceProperties(&prop, dev) == cudaSuccess) net->sm_count = prop.multiProcessorCount;
+        else cudaGetLastError();
+    }
     net->n_layers = n_layers;
     net->max_batch = max_batch;
     net->clip_lo = clip_lo;
@@ -305,7 +308,7 @@ cert_status_t cert_net_create(const cert_layer_desc_t *layers, int n_layers, int
             if (cudaMemcpy(L.Wct, host.data(), nw * sizeof(float), cudaMemcpyHostToDevice) != cudaSuccess) {
                 fail = CERT_ERR_CUDA; break;
             }
-            if (cert::convt_smem_bytes(L) > 200 * 1024) { fail = CERT_ERR_UNSUPPORTED; break; }
+            if (!cert::convt_supported(L)) { fail = CERT_ERR_UNSUPPORTED; break; }
         }
         if (L.relu_after) {
             size_t n = (size_t)max_batch * L.ld_out;
@@ -435,7 +438,7 @@ cert_status_t cert_deeppoly_bounds(cert_net_t *net, const float *centers, float 
                 rec.mark(CERT_CLASS_AFFINE);
                 paths |= 1;
             } else {
-                cert::launch_convt_ffma(Lj, Q, P, rows, st);
+                cert::launch_convt_ffma(Lj, Q, P, rows, net->sm_count, st);
                 rec.mark(CERT_CLASS_CONV);
             }
             cur ^= 1;

@@ -86,6 +86,7 @@ void launch_gemm_ffma(const float *A, int lda, const float *B, int ldb, float *C
 
 // P[r][(ci,iy,ix)] = sum over (co,ky,kx) of Q[r][(co,oy,ox)] * W[co][ci][ky][kx]: the exact
 // transpose of the conv layer applied to every row's coefficient map.
-void launch_convt_ffma(const LayerDev &L, const float *Q, float *P, long long rows, cudaStream_t st);
+// `sms`: number of multiprocessors (the kernel is persistent, one block per multiprocessor).
+void launch_convt_ffma(const LayerDev &L, const float *Q, float *P, long long rows, int sms, cudaStream_t st);
 
 }  // namespace cert
