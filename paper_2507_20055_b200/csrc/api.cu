@@ -433,14 +433,33 @@ cert_status_t cert_deeppoly_bounds(cert_net_t *net, const float *centers, float 
                 dslots = T.n_tiles;
                 continue;
             }
-            if (Lj.kind == CERT_LAYER_FC) {
-                cert::launch_gemm_ffma(Q, Lj.ld_out, Lj.W, Lj.ld_in, P, Lj.ld_in, rows, Lj.n_in, Lj.n_out, st);
-                rec.mark(CERT_CLASS_AFFINE);
-                paths |= 1;
-            } else {
-                cert::launch_convt_ffma(Lj, Q, P, rows, net->sm_count, st);
+            if (Lj.kind == CERT_LAYER_CONV2D) {
+                // conv back-step with what follows it fused: the ReLU back-step below, or the concretisation
+                cert::ConvtEpilogue ep;
+                std::memset(&ep, 0, sizeof(ep));
+                ep.n_k = Lk.n_out;
+                ep.d_in = net->dbuf[dcur]; ep.n_slots_in = dslots; ep.slot_stride = net->slot_stride;
+                ep.d_out = net->dbuf[dcur];
+                if (j > 0) {
+                    const LayerDev &Lb = net->layers[j - 1];
+                    ep.mode = cert::CONVT_EPI_RELU;
+                    ep.has_relu = Lb.relu_after;
+                    ep.lamL = Lb.lamL; ep.lamU = Lb.lamU; ep.nuU = Lb.nuU; ep.bias_below = Lb.bias_n;
+                    ep.P = P; ep.P_lo = P_lo;
+                } else {
+                    ep.mode = cert::CONVT_EPI_CONCRETIZE;
+                    ep.l0 = net->l0; ep.u0 = net->u0;
+                    ep.lb_out = lb_out; ep.ub_out = ub_out; ep.n_total = n_total; ep.out_off = Lk.out_off;
+                }
+                cert::launch_convt_ffma(Lj, Q, rows, net->sm_count, ep, st);
                 rec.mark(CERT_CLASS_CONV);
+                cur ^= 1;
+                dslots = 1;
+                continue;
             }
+            cert::launch_gemm_ffma(Q, Lj.ld_out, Lj.W, Lj.ld_in, P, Lj.ld_in, rows, Lj.n_in, Lj.n_out, st);
+            rec.mark(CERT_CLASS_AFFINE);
+            paths |= 1;
             cur ^= 1;
             if (j > 0) {
                 cert::launch_relu_step(net->layers[j - 1], batch, Lk.n_out, P, P_lo, net->dbuf[dcur], dslots,

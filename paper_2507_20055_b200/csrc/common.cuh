@@ -84,9 +84,32 @@ void launch_concretize(const float *P, const float *d, int n_slots, long long sl
 void launch_gemm_ffma(const float *A, int lda, const float *B, int ldb, float *C, int ldc, long long M,
                       int N, int K, cudaStream_t st);
 
+// What the conv back-step kernel applies to its result while it is still in registers.
+enum { CONVT_EPI_RELU = 0, CONVT_EPI_CONCRETIZE = 1 };
+struct ConvtEpilogue {
+    int mode;                 // CONVT_EPI_RELU: ReLU back-step through the layer below + constant's share of the
+                              // next affine step, result stored; CONVT_EPI_CONCRETIZE: bounds against the box
+    int n_k;                  // neurons of the layer being bounded (decodes a row into box, side, neuron)
+    // row constants: sum over n_slots_in slots of d_in in, slot 0 of d_out out (may be the same buffer)
+    const float *d_in;
+    int n_slots_in;
+    long long slot_stride;
+    float *d_out;
+    // CONVT_EPI_RELU
+    int has_relu;
+    const float *lamL, *lamU, *nuU;   // [batch][ld_in] relaxation of the ReLU below
+    const float *bias_below;          // [ld_in]
+    float *P, *P_lo;                  // result [rows][ld_in]; P_lo != nullptr: stored as a TF32 pair
+    // CONVT_EPI_CONCRETIZE
+    const float *l0, *u0;             // [batch][ld_in]
+    float *lb_out, *ub_out;
+    int n_total, out_off;
+};
+
 // P[r][(ci,iy,ix)] = sum over (co,ky,kx) of Q[r][(co,oy,ox)] * W[co][ci][ky][kx]: the exact
-// transpose of the conv layer applied to every row's coefficient map.
-// `sms`: number of multiprocessors (the kernel is persistent, one block per multiprocessor).
-void launch_convt_ffma(const LayerDev &L, const float *Q, float *P, long long rows, int sms, cudaStream_t st);
+// transpose of the conv layer applied to every row's coefficient map, followed by `ep`.
+// `sms`: number of multiprocessors (the kernel is persistent).
+void launch_convt_ffma(const LayerDev &L, const float *Q, long long rows, int sms, const ConvtEpilogue &ep,
+                       cudaStream_t st);
 
 }  // namespace cert

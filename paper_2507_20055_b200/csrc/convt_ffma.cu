@@ -5,15 +5,22 @@
 //   P[r][ci][iy][ix] = sum over (co, ky, kx) with (iy + pad - ky) = stride * oy and
 //                      (ix + pad - kx) = stride * ox of  Q[r][co][oy][ox] * W[co][ci][ky][kx]
 //
+// and what follows the step on the path is applied to P while it is still in
+// registers: either the ReLU back-step through the layer below
+// (replace_lower/upper, clamp form of Section 4.3) plus the constant's share
+// P'.b of the next affine step, or the concretisation against the input box
+// (map(simplify_lower/upper)), in which case P is never stored.
+//
 // Implicit GEMM on the fp32 FMA units (the channel count below a conv layer is
 // 3..16: too narrow an N for the tensor cores).  Input pixels fall into
 // stride x stride classes by ((iy + pad) mod stride, (ix + pad) mod stride);
 // every pixel of a class uses the same kernel taps, so a warp that works on one
 // class reads its weights as warp-uniform 16-byte shared-memory loads.  A block
-// stages the maps of a group of rows in shared memory inside a zero halo (no
-// bounds tests in the inner loop); a thread accumulates PXT pixels x CT
-// channels in registers, so a coefficient read from shared memory feeds CT
-// FMAs and a weight PXT FMAs.
+// stages the maps of RB rows in shared memory inside a zero halo (no bounds
+// tests in the inner loop); a thread accumulates PXT pixels x CT channels in
+// registers.  A lane always works for the same row of the group (lane / (32/RB)),
+// so a row's constant is summed in registers, then across the lanes of its
+// group by shuffles and across warps in a fixed order: no atomics.
 #include "common.cuh"
 
 namespace cert {
@@ -22,9 +29,9 @@ namespace {
 
 constexpr int kThreads = 256;
 constexpr int kWarps = kThreads / 32;
-constexpr int PXT = 4;                       // pixels per thread
 constexpr int kMaxStride = 4;
-constexpr size_t kSmemBudget = 200 * 1024;
+constexpr int kMaxRowsPerGroup = 8;
+constexpr size_t kSmemBudget = 100 * 1024;   // two blocks per multiprocessor: one stages while the other computes
 
 // Shared-memory plan of one conv layer's back-step, derived on the host.
 struct ConvtPlan {
@@ -32,7 +39,7 @@ struct ConvtPlan {
     int HP, WP;              // padded map height / width
     int map_stride;          // floats between consecutive rows' staged maps
     int cpad;                // c_in rounded up to 4 (weights are staged as [co][ky][kx][cpad])
-    int rows_per_group;      // rows staged per pass
+    int rows_per_group;      // rows staged per pass: a power of two <= 8
     size_t smem_bytes;
 };
 
@@ -62,37 +69,58 @@ ConvtPlan make_plan(const LayerDev &L) {
     p.halo_x = rx.lo < 0 ? -rx.lo : 0;
     p.HP = p.halo_y + std::max(L.h_out, ry.hi + 1);
     p.WP = p.halo_x + std::max(L.w_out, rx.hi + 1);
-    // Pixels per class row; consecutive lanes walk them and then move to the next staged row, so a map
-    // stride congruent to that count modulo 32 keeps a warp's loads on distinct banks.
-    int wc = (L.w_in + L.stride - 1) / L.stride;
-    int ms = L.c_out * p.HP * p.WP;
-    while (ms % 32 != wc % 32) ++ms;
-    p.map_stride = ms;
     p.cpad = round_up(L.c_in, 4);
-    size_t w_bytes = sizeof(float) * (size_t)L.c_out * L.kh * L.kw * p.cpad;
-    size_t per_row = sizeof(float) * (size_t)ms;
-    long long fit = w_bytes < kSmemBudget ? (long long)((kSmemBudget - w_bytes) / per_row) : 0;
-    p.rows_per_group = (int)std::min<long long>(fit, 16);
-    p.smem_bytes = w_bytes + per_row * (size_t)std::max(p.rows_per_group, 1);
+    const size_t w_bytes = sizeof(float) * (size_t)L.c_out * L.kh * L.kw * p.cpad;
+    const size_t fixed = w_bytes + sizeof(float) * kWarps * kMaxRowsPerGroup;
+    const int map = L.c_out * p.HP * p.WP;
+    p.rows_per_group = 0;
+    for (int rb = kMaxRowsPerGroup; rb >= 1; rb /= 2) {
+        // The 32/rb lanes that work for one row read consecutive pixels; a map stride congruent to
+        // 32/rb modulo 32 puts the rows' lane groups on distinct banks.
+        int ms = map;
+        while (ms % 32 != (32 / rb) % 32) ++ms;
+        size_t bytes = fixed + sizeof(float) * (size_t)ms * rb;
+        if (bytes <= kSmemBudget) {
+            p.rows_per_group = rb;
+            p.map_stride = ms;
+            p.smem_bytes = bytes;
+            break;
+        }
+    }
     return p;
 }
 
-// Q [rows][ld_out] maps (c_out, h_out, w_out); P [rows][ld_in] maps (c_in, h_in, w_in).
+__device__ __forceinline__ float tf32_round(float x) {
+    uint32_t r;
+    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(x));
+    return __uint_as_float(r);
+}
+
+__device__ __forceinline__ void cp_async4(float *smem_dst, const float *gsrc, bool live) {
+    const uint32_t dst = static_cast<uint32_t>(__cvta_generic_to_shared(smem_dst));
+    const int src_bytes = live ? 4 : 0;     // 0: nothing is read, the word is zero-filled
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(dst), "l"(gsrc), "r"(src_bytes) : "memory");
+}
+
+// Q [rows][ld_out] maps (c_out, h_out, w_out); the result maps (c_in, h_in, w_in) with pitch ld_in.
 // Wct: weights laid out [c_out][kh][kw][c_in].
-template <int CT>
-__global__ void __launch_bounds__(kThreads, 1)
-convt_kernel(const float *__restrict__ Q, int ld_out, float *__restrict__ P, int ld_in,
-             const float *__restrict__ Wct, ConvGeom g, ConvtPlan pl, long long rows) {
+template <int CT, int PXT, int EPI>
+__global__ void __launch_bounds__(kThreads, 2)
+convt_kernel(const float *__restrict__ Q, int ld_out, int ld_in, const float *__restrict__ Wct, ConvGeom g,
+             ConvtPlan pl, long long rows, ConvtEpilogue ep) {
     extern __shared__ __align__(16) float smem[];
     const int n_out = g.c_out * g.h_out * g.w_out;
     const int n_in = g.c_in * g.h_in * g.w_in;
     const int hw_in = g.h_in * g.w_in, hw_out = g.h_out * g.w_out;
     const int n_w = g.c_out * g.kh * g.kw * pl.cpad;
     const int RB = pl.rows_per_group;
+    const int G = 32 / RB;             // lanes per row of the group
     const int plane = pl.HP * pl.WP;
     float *Ws = smem;                  // [c_out][kh][kw][cpad]
-    float *Qs = smem + n_w;            // [RB][map_stride], each map [c_out][HP][WP] inside its halo
+    float *red = smem + n_w;           // [kWarps][kMaxRowsPerGroup] partial row constants
+    float *Qs = red + kWarps * kMaxRowsPerGroup;   // [RB][map_stride], each map [c_out][HP][WP] inside its halo
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int rl = lane / G, gl = lane % G;
 
     for (int i = threadIdx.x; i < n_w; i += kThreads) {
         int ci = i % pl.cpad, tap = i / pl.cpad;
@@ -102,61 +130,67 @@ convt_kernel(const float *__restrict__ Q, int ld_out, float *__restrict__ P, int
 
     const int s = g.stride;
     const int n_classes = s * s;
+    const int d_ox = kThreads % g.w_out, d_oy = (kThreads / g.w_out) % g.h_out, d_co = kThreads / hw_out;
 
     for (long long r0 = (long long)blockIdx.x * RB; r0 < rows; r0 += (long long)gridDim.x * RB) {
         __syncthreads();
-        // stage the maps of rows r0 .. r0+RB-1 (rows past the end read as zero); the element index
-        // advances by the block size, its (co, oy, ox) decomposition with it
-        {
-            const int d_ox = kThreads % g.w_out, d_oy = (kThreads / g.w_out) % g.h_out, d_co = kThreads / hw_out;
-            for (int rl = 0; rl < RB; ++rl) {
-                const bool live = r0 + rl < rows;
-                const float *qrow = Q + (size_t)(r0 + rl) * ld_out;
-                float *qs = Qs + rl * pl.map_stride + pl.halo_y * pl.WP + pl.halo_x;
-                int e = threadIdx.x;
-                int co = e / hw_out, oy = (e % hw_out) / g.w_out, ox = e % g.w_out;
-                for (; e < n_out; e += kThreads) {
-                    qs[co * plane + oy * pl.WP + ox] = live ? qrow[e] : 0.0f;
-                    ox += d_ox;
-                    if (ox >= g.w_out) { ox -= g.w_out; ++oy; }
-                    oy += d_oy;
-                    if (oy >= g.h_out) { oy -= g.h_out; ++co; }
-                    co += d_co;
-                }
+        // Stage the maps of rows r0 .. r0+RB-1 with asynchronous 4-byte copies (rows past the end are
+        // zero-filled).  The element index advances by the block size, its (co, oy, ox) split with it.
+        for (int q = 0; q < RB; ++q) {
+            const bool live = r0 + q < rows;
+            const float *qrow = Q + (size_t)(live ? r0 + q : r0) * ld_out;
+            float *qs = Qs + q * pl.map_stride + pl.halo_y * pl.WP + pl.halo_x;
+            int e = threadIdx.x;
+            int co = e / hw_out, oy = (e % hw_out) / g.w_out, ox = e % g.w_out;
+            for (; e < n_out; e += kThreads) {
+                cp_async4(qs + co * plane + oy * pl.WP + ox, qrow + e, live);
+                ox += d_ox;
+                if (ox >= g.w_out) { ox -= g.w_out; ++oy; }
+                oy += d_oy;
+                if (oy >= g.h_out) { oy -= g.h_out; ++co; }
+                co += d_co;
             }
         }
+        asm volatile("cp.async.commit_group;" ::: "memory");
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
         __syncthreads();
 
-        // Work units: (class, chunk of 32*PXT items); an item is (row of the group, pixel of the class).
+        // This lane's row, and where its relaxation / box vectors start.
+        const long long r = r0 + rl;
+        const bool row_ok = r < rows;
+        const long long rr = row_ok ? r : 0;
+        const int box = (int)(rr / (2LL * ep.n_k));
+        const int upper = (int)((rr / ep.n_k) & 1);
+        const size_t vec = (size_t)box * ld_in;
+        float dacc = 0.0f;
+
+        // Work units: (class, chunk of G*PXT pixels); every lane group of the warp does the chunk for its row.
         int unit_base = 0;
         for (int cls = 0; cls < n_classes; ++cls) {
             const int cy = cls / s, cx = cls % s;
             // pixels of the class: iy = cy - pad + s*uy, 0 <= iy < h_in; then oy = uy - my for ky = cy + s*my
-            const int uy0 = (g.pad - cy + s - 1 >= 0) ? (g.pad - cy + s - 1) / s : 0;
-            const int ux0 = (g.pad - cx + s - 1 >= 0) ? (g.pad - cx + s - 1) / s : 0;
+            const int uy0 = (g.pad - cy + s - 1) / s, ux0 = (g.pad - cx + s - 1) / s;   // numerators are >= 0
             const int uy1 = (g.h_in - 1 + g.pad - cy >= 0) ? (g.h_in - 1 + g.pad - cy) / s : -1;
             const int ux1 = (g.w_in - 1 + g.pad - cx >= 0) ? (g.w_in - 1 + g.pad - cx) / s : -1;
             const int Hc = uy1 - uy0 + 1, Wc = ux1 - ux0 + 1;
             const int n_my = cy < g.kh ? (g.kh - cy + s - 1) / s : 0;
             const int n_mx = cx < g.kw ? (g.kw - cx + s - 1) / s : 0;
             if (Hc <= 0 || Wc <= 0) continue;
-            const int items = Hc * RB * Wc;
-            const int units = (items + 32 * PXT - 1) / (32 * PXT);
-            // warps take units round-robin across classes
-            int first = ((warp - unit_base) % kWarps + kWarps) % kWarps;
+            const int pixels = Hc * Wc;
+            const int units = (pixels + G * PXT - 1) / (G * PXT);
+            const int first = ((warp - unit_base) % kWarps + kWarps) % kWarps;   // units go round the warps
             for (int u = first; u < units; u += kWarps) {
                 int q_off[PXT], p_off[PXT];
-                long long p_row[PXT];
+                bool ok[PXT];
 #pragma unroll
                 for (int i = 0; i < PXT; ++i) {
-                    int it = u * (32 * PXT) + i * 32 + lane;
-                    bool ok = it < items;
-                    int itc = ok ? it : 0;
-                    int ux = itc % Wc, t2 = itc / Wc, rl = t2 % RB, uy = t2 / RB;
+                    const int p = u * (G * PXT) + i * G + gl;
+                    ok[i] = p < pixels;
+                    const int pc = ok[i] ? p : 0;
+                    const int uy = pc / Wc, ux = pc % Wc;
                     q_off[i] = rl * pl.map_stride + (uy0 + uy + pl.halo_y) * pl.WP + (ux0 + ux + pl.halo_x);
-                    int iy = cy - g.pad + s * (uy0 + uy), ix = cx - g.pad + s * (ux0 + ux);
-                    p_off[i] = iy * g.w_in + ix;
-                    p_row[i] = (ok && r0 + rl < rows) ? r0 + rl : -1;
+                    p_off[i] = (cy - g.pad + s * (uy0 + uy)) * g.w_in + (cx - g.pad + s * (ux0 + ux));
+                    ok[i] = ok[i] && row_ok;
                 }
                 for (int c0 = 0; c0 < g.c_in; c0 += CT) {
                     float acc[PXT][CT];
@@ -164,6 +198,7 @@ convt_kernel(const float *__restrict__ Q, int ld_out, float *__restrict__ P, int
                     for (int i = 0; i < PXT; ++i)
 #pragma unroll
                         for (int c = 0; c < CT; ++c) acc[i][c] = 0.0f;
+#pragma unroll 2
                     for (int co = 0; co < g.c_out; ++co) {
                         for (int my = 0; my < n_my; ++my) {
                             const int ky = cy + s * my;
@@ -173,7 +208,7 @@ convt_kernel(const float *__restrict__ Q, int ld_out, float *__restrict__ P, int
                                 float w[CT];
 #pragma unroll
                                 for (int c4 = 0; c4 < CT; c4 += 4) {
-                                    // cpad is a multiple of 4; channels past cpad (CT > remaining) are skipped
+                                    // cpad is a multiple of 4; channels past it read as zero
                                     float4 w4 = (c0 + c4 < pl.cpad) ? *reinterpret_cast<const float4 *>(wp + c4)
                                                                      : make_float4(0.f, 0.f, 0.f, 0.f);
                                     w[c4] = w4.x; w[c4 + 1] = w4.y; w[c4 + 2] = w4.z; w[c4 + 3] = w4.w;
@@ -188,33 +223,97 @@ convt_kernel(const float *__restrict__ Q, int ld_out, float *__restrict__ P, int
                             }
                         }
                     }
+                    // ---- what follows the step on the path, per element ----
 #pragma unroll
                     for (int i = 0; i < PXT; ++i) {
-                        if (p_row[i] < 0) continue;
-                        float *prow = P + (size_t)p_row[i] * ld_in + p_off[i];
+                        if (!ok[i]) continue;
 #pragma unroll
-                        for (int c = 0; c < CT; ++c)
-                            if (c0 + c < g.c_in) prow[(size_t)(c0 + c) * hw_in] = acc[i][c];
+                        for (int c = 0; c < CT; ++c) {
+                            if (c0 + c >= g.c_in) continue;
+                            const int t = (c0 + c) * hw_in + p_off[i];
+                            const float v = acc[i][c];
+                            const bool nonneg = (v >= 0.0f);
+                            if (EPI == CONVT_EPI_CONCRETIZE) {
+                                // lower rows: c >= 0 ? c*l : c*u; upper rows: c >= 0 ? c*u : c*l
+                                const float bnd = (nonneg != (upper != 0)) ? ep.l0[vec + t] : ep.u0[vec + t];
+                                dacc = fmaf(v, bnd, dacc);
+                            } else {
+                                float qv = v;
+                                if (ep.has_relu) {
+                                    const bool use_lower = upper ? !nonneg : nonneg;
+                                    if (use_lower) {
+                                        qv = v * ep.lamL[vec + t];
+                                    } else {
+                                        dacc = fmaf(v, ep.nuU[vec + t], dacc);
+                                        qv = v * ep.lamU[vec + t];
+                                    }
+                                }
+                                dacc = fmaf(qv, ep.bias_below[t], dacc);
+                                const size_t o = (size_t)r * ld_in + t;
+                                if (ep.P_lo) {
+                                    const float h = tf32_round(qv);
+                                    ep.P[o] = h;
+                                    ep.P_lo[o] = tf32_round(qv - h);
+                                } else {
+                                    ep.P[o] = qv;
+                                }
+                            }
+                        }
                     }
                 }
             }
             unit_base += units;
         }
-        // keep the padded tail of the rows at zero
-        for (int rl = 0; rl < RB; ++rl) {
-            if (r0 + rl >= rows) break;
-            float *prow = P + (size_t)(r0 + rl) * ld_in;
-            for (int t = n_in + threadIdx.x; t < ld_in; t += kThreads) prow[t] = 0.0f;
+
+        // Row constants: lanes of a group by shuffles, warps in warp order.
+        for (int o = 1; o < G; o <<= 1) dacc += __shfl_xor_sync(0xffffffffu, dacc, o);
+        if (gl == 0) red[warp * kMaxRowsPerGroup + rl] = dacc;
+        __syncthreads();
+        if (threadIdx.x < RB && r0 + threadIdx.x < rows) {
+            const long long row = r0 + threadIdx.x;
+            float tot = ep.d_in[row];
+            for (int sl = 1; sl < ep.n_slots_in; ++sl) tot += ep.d_in[(size_t)sl * ep.slot_stride + row];
+            for (int w2 = 0; w2 < kWarps; ++w2) tot += red[w2 * kMaxRowsPerGroup + threadIdx.x];
+            if (EPI == CONVT_EPI_CONCRETIZE) {
+                const int b2 = (int)(row / (2LL * ep.n_k)), up2 = (int)((row / ep.n_k) & 1), i2 = (int)(row % ep.n_k);
+                (up2 ? ep.ub_out : ep.lb_out)[(size_t)b2 * ep.n_total + ep.out_off + i2] = tot;
+            } else {
+                ep.d_out[row] = tot;
+            }
+        }
+        if (EPI == CONVT_EPI_RELU) {
+            // keep the padded tail of the rows at zero
+            for (int q = 0; q < RB; ++q) {
+                if (r0 + q >= rows) break;
+                const size_t o = (size_t)(r0 + q) * ld_in;
+                for (int t = n_in + threadIdx.x; t < ld_in; t += kThreads) {
+                    ep.P[o + t] = 0.0f;
+                    if (ep.P_lo) ep.P_lo[o + t] = 0.0f;
+                }
+            }
         }
     }
 }
 
-template <int CT>
-void launch_ct(const LayerDev &L, const ConvtPlan &pl, const float *Q, float *P, long long rows, int sms,
-               cudaStream_t st) {
+template <int CT, int PXT>
+void launch_ct(const LayerDev &L, const ConvtPlan &pl, const float *Q, long long rows, int sms,
+               const ConvtEpilogue &ep, cudaStream_t st) {
     long long groups = ceil_div_ll(rows, pl.rows_per_group);
-    int grid = (int)std::min<long long>(groups, sms);
-    convt_kernel<CT><<<grid, kThreads, pl.smem_bytes, st>>>(Q, L.ld_out, P, L.ld_in, L.Wct, geom_of(L), pl, rows);
+    int grid = (int)std::min<long long>(groups, 2LL * sms);
+    if (ep.mode == CONVT_EPI_CONCRETIZE)
+        convt_kernel<CT, PXT, CONVT_EPI_CONCRETIZE><<<grid, kThreads, pl.smem_bytes, st>>>(
+            Q, L.ld_out, L.ld_in, L.Wct, geom_of(L), pl, rows, ep);
+    else
+        convt_kernel<CT, PXT, CONVT_EPI_RELU><<<grid, kThreads, pl.smem_bytes, st>>>(
+            Q, L.ld_out, L.ld_in, L.Wct, geom_of(L), pl, rows, ep);
+}
+
+template <int CT, int PXT>
+void prepare_ct() {
+    cudaFuncSetAttribute(convt_kernel<CT, PXT, CONVT_EPI_RELU>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                         (int)kSmemBudget);
+    cudaFuncSetAttribute(convt_kernel<CT, PXT, CONVT_EPI_CONCRETIZE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                         (int)kSmemBudget);
 }
 
 }  // namespace
@@ -226,16 +325,17 @@ bool convt_supported(const LayerDev &L) {
 }
 
 void convt_prepare() {
-    cudaFuncSetAttribute(convt_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget);
-    cudaFuncSetAttribute(convt_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget);
-    cudaFuncSetAttribute(convt_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget);
+    prepare_ct<4, 4>();
+    prepare_ct<8, 4>();
+    prepare_ct<16, 2>();
 }
 
-void launch_convt_ffma(const LayerDev &L, const float *Q, float *P, long long rows, int sms, cudaStream_t st) {
+void launch_convt_ffma(const LayerDev &L, const float *Q, long long rows, int sms, const ConvtEpilogue &ep,
+                       cudaStream_t st) {
     const ConvtPlan pl = make_plan(L);
-    if (L.c_in <= 4) launch_ct<4>(L, pl, Q, P, rows, sms, st);
-    else if (L.c_in <= 8) launch_ct<8>(L, pl, Q, P, rows, sms, st);
-    else launch_ct<16>(L, pl, Q, P, rows, sms, st);
+    if (L.c_in <= 4) launch_ct<4, 4>(L, pl, Q, rows, sms, ep, st);
+    else if (L.c_in <= 8) launch_ct<8, 4>(L, pl, Q, rows, sms, ep, st);
+    else launch_ct<16, 2>(L, pl, Q, rows, sms, ep, st);
 }
 
 }  // namespace cert

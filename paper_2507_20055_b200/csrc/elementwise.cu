@@ -147,18 +147,6 @@ __global__ void relax_kernel(float *__restrict__ lb_out, float *__restrict__ ub_
     nuU[idx] = nu;
 }
 
-// Coefficient of prev-neuron t in the expression of neuron i of layer L.
-__device__ __forceinline__ float weight_elem(const float *__restrict__ W, int kind, const ConvGeom &g,
-                                             int ld_in, int i, int t) {
-    if (kind == CERT_LAYER_FC) return W[(size_t)i * ld_in + t];
-    int hw = g.h_out * g.w_out;
-    int co = i / hw, oy = (i / g.w_out) % g.h_out, ox = i % g.w_out;
-    int ci = t / (g.h_in * g.w_in), iy = (t / g.w_in) % g.h_in, ix = t % g.w_in;
-    int ky = iy - (oy * g.stride - g.pad), kx = ix - (ox * g.stride - g.pad);
-    if (ky < 0 || ky >= g.kh || kx < 0 || kx >= g.kw) return 0.0f;
-    return W[(((size_t)co * g.c_in + ci) * g.kh + ky) * g.kw + kx];
-}
-
 // FROM_WEIGHTS: source is row i of W_k (start of a back-substitution), else P in place.
 template <bool FROM_WEIGHTS>
 __global__ void relu_step_kernel(const float *__restrict__ Wk, int kind_k, ConvGeom gk, int ldw_k,
@@ -176,12 +164,35 @@ __global__ void relu_step_kernel(const float *__restrict__ Wk, int kind_k, ConvG
     float *prow = P + (size_t)r * ld;
     const float *ll = lamL + (size_t)b * ld, *lu = lamU + (size_t)b * ld, *nu = nuU + (size_t)b * ld;
     float dacc = 0.0f;
+    // Conv layer k: neuron i = (co, oy, ox) sees the window [y0, y0+kh) x [x0, x0+kw) of every input
+    // channel; column t = (ci, iy, ix) is tracked incrementally (the column index advances by 128).
+    int co = 0, y0 = 0, x0 = 0, ci = 0, iy = 0, ix = 0, d_ci = 0, d_iy = 0, d_ix = 0;
+    if (FROM_WEIGHTS && kind_k != CERT_LAYER_FC) {
+        const int hw_o = gk.h_out * gk.w_out, hw_i = gk.h_in * gk.w_in;
+        co = i / hw_o;
+        y0 = ((i / gk.w_out) % gk.h_out) * gk.stride - gk.pad;
+        x0 = (i % gk.w_out) * gk.stride - gk.pad;
+        const int t0 = lane * 4;
+        ci = t0 / hw_i; iy = (t0 / gk.w_in) % gk.h_in; ix = t0 % gk.w_in;
+        d_ci = 128 / hw_i; d_iy = (128 / gk.w_in) % gk.h_in; d_ix = 128 % gk.w_in;
+    }
     // four consecutive columns per lane: 16-byte accesses (every row pitch is a multiple of 32 floats)
     for (int t = lane * 4; t < ld; t += 128) {
         float c[4], q[4];
         if (FROM_WEIGHTS && kind_k != CERT_LAYER_FC) {
+            int cie = ci, iye = iy, ixe = ix;
 #pragma unroll
-            for (int e = 0; e < 4; ++e) c[e] = (t + e < n) ? weight_elem(Wk, kind_k, gk, ldw_k, i, t + e) : 0.0f;
+            for (int e = 0; e < 4; ++e) {
+                const int ky = iye - y0, kx = ixe - x0;
+                const bool in = (t + e < n) && ky >= 0 && ky < gk.kh && kx >= 0 && kx < gk.kw;
+                c[e] = in ? Wk[(((size_t)co * gk.c_in + cie) * gk.kh + ky) * gk.kw + kx] : 0.0f;
+                if (++ixe >= gk.w_in) { ixe = 0; if (++iye >= gk.h_in) { iye = 0; ++cie; } }
+            }
+            ix += d_ix;
+            if (ix >= gk.w_in) { ix -= gk.w_in; ++iy; }
+            iy += d_iy;
+            if (iy >= gk.h_in) { iy -= gk.h_in; ++ci; }
+            ci += d_ci;
         } else {
             const float4 c4 = *reinterpret_cast<const float4 *>(FROM_WEIGHTS ? Wk + (size_t)i * ldw_k + t : prow + t);
             c[0] = c4.x; c[1] = c4.y; c[2] = c4.z; c[3] = c4.w;
