@@ -17,9 +17,10 @@
 // in either ping-pong buffer.
 struct TcLayer {
     bool usable = false;
-    cert::TcMap b_hi, b_lo;
+    cert::TcMap b_hi, b_lo;          // box = this CTA's share of the column tile
     cert::TcMap a_hi[2], a_lo[2];
-    int bn = 0, bn_pad = 0, n_tiles = 0, stages = 0, tmem_cols = 0, smem = 0;
+    cert::TcMap o_hi[2], o_lo[2];    // store maps of the result (width = neurons below, padded); j >= 1 only
+    cert::TcPlan plan;
 };
 
 
@@ -40,7 +41,7 @@ struct cert_net {
     int d_slots = 1;                         // slots per buffer (most column tiles of any contraction)
     long long slot_stride = 0;               // rows of the largest coefficient matrix
     int sm_count = 148;
-    int tc_bk = 32;                          // floats of K per pipeline stage of the tensor-core kernel
+    int tc_ctas = 1;                         // CTAs per row panel of the tensor-core kernel (2: cta_group::2)
     unsigned char *codes = nullptr;          // [max_batch][n_relu]
     int *status_dev = nullptr;               // sticky device status word
     // host staging for cert_deeppoly_bounds_host
@@ -139,9 +140,13 @@ cert_status_t setup_tensor_core_path(cert_net *net, const cert_layer_desc_t *des
     net->tc.assign(K, TcLayer());
     net->tc_ok = false;
     if (K < 2) return CERT_OK;
-    if (!cert::tc_driver_init() || !cert::tc_prepare_kernels()) return CERT_OK;
-    if (const char *e = std::getenv("CERT_TC_BK")) net->tc_bk = (std::atoi(e) == 16) ? 16 : 32;
-    const int bk = net->tc_bk;
+    bool pair_ok = false;
+    if (!cert::tc_driver_init() || !cert::tc_prepare_kernels(&pair_ok)) return CERT_OK;
+    net->tc_ctas = (pair_ok && net->sm_count >= 2) ? 2 : 1;
+    if (const char *e = std::getenv("CERT_TC_CTAS")) {
+        if (std::atoi(e) == 1) net->tc_ctas = 1;
+    }
+    const int ctas = net->tc_ctas;
     if (!dev_alloc_zero(net, &net->buf_lo[0], max_elems) || !dev_alloc_zero(net, &net->buf_lo[1], max_elems))
         return CERT_ERR_OOM;
     std::vector<float> hi, lo;
@@ -166,18 +171,22 @@ cert_status_t setup_tensor_core_path(cert_net *net, const cert_layer_desc_t *des
         if (cudaMemcpy(L.Wt_hi, hi.data(), hi.size() * sizeof(float), cudaMemcpyHostToDevice) != cudaSuccess ||
             cudaMemcpy(L.Wt_lo, lo.data(), lo.size() * sizeof(float), cudaMemcpyHostToDevice) != cudaSuccess)
             return CERT_ERR_CUDA;
-        cert::tc_tile_plan(L.n_in, bk, &T.bn, &T.bn_pad, &T.n_tiles, &T.stages, &T.tmem_cols, &T.smem);
-        if (T.stages < 2) continue;
-        bool ok = cert::tc_make_map(&T.b_hi, L.Wt_hi, L.n_out, L.n_in, L.ld_out, T.bn, bk) &&
-                  cert::tc_make_map(&T.b_lo, L.Wt_lo, L.n_out, L.n_in, L.ld_out, T.bn, bk);
+        T.plan = cert::tc_tile_plan(L.n_in, ctas);
+        if (T.plan.stages < 2) continue;
+        bool ok = cert::tc_make_map(&T.b_hi, L.Wt_hi, L.n_out, L.n_in, L.ld_out, T.plan.bn / ctas) &&
+                  cert::tc_make_map(&T.b_lo, L.Wt_lo, L.n_out, L.n_in, L.ld_out, T.plan.bn / ctas);
         // rows of the largest layer above j
         long long rows_max = 0;
         for (int k = j + 1; k < K; ++k) rows_max = std::max(rows_max, 2LL * net->max_batch * net->layers[k].n_out);
-        for (int p = 0; p < 2 && ok; ++p)
-            ok = cert::tc_make_map(&T.a_hi[p], net->buf[p], L.n_out, rows_max, L.ld_out, 128, bk) &&
-                 cert::tc_make_map(&T.a_lo[p], net->buf_lo[p], L.n_out, rows_max, L.ld_out, 128, bk);
+        for (int p = 0; p < 2 && ok; ++p) {
+            ok = cert::tc_make_map(&T.a_hi[p], net->buf[p], L.n_out, rows_max, L.ld_out, 128) &&
+                 cert::tc_make_map(&T.a_lo[p], net->buf_lo[p], L.n_out, rows_max, L.ld_out, 128);
+            if (ok && j > 0)
+                ok = cert::tc_make_map(&T.o_hi[p], net->buf[p], L.ld_in, rows_max, L.ld_in, 32) &&
+                     cert::tc_make_map(&T.o_lo[p], net->buf_lo[p], L.ld_in, rows_max, L.ld_in, 32);
+        }
         T.usable = ok;
-        if (ok) net->d_slots = std::max(net->d_slots, T.n_tiles);
+        if (ok) net->d_slots = std::max(net->d_slots, T.plan.n_tiles);
     }
     net->tc_ok = true;
     return CERT_OK;
@@ -406,31 +415,32 @@ cert_status_t cert_deeppoly_bounds(cert_net_t *net, const float *centers, float 
                 cert::TcArgs a;
                 std::memset(&a, 0, sizeof(a));
                 a.M = rows; a.K = Lj.n_out; a.n_k = Lk.n_out; a.ld_n = Lj.ld_in;
-                a.bn = T.bn; a.bn_pad = T.bn_pad; a.n_tiles = T.n_tiles; a.stages = T.stages;
-                a.tmem_cols = T.tmem_cols;
-                a.total_tiles = (int)cert::ceil_div_ll(rows, 128) * T.n_tiles;
+                a.bn = T.plan.bn; a.n_tiles = T.plan.n_tiles; a.stages = T.plan.stages;
+                a.tmem_cols = T.plan.tmem_cols;
+                const int ctas = net->tc_ctas;
+                a.total_tiles = (int)cert::ceil_div_ll(rows, 128 * ctas) * T.plan.n_tiles;
                 a.d_in = net->dbuf[dcur]; a.n_slots_in = dslots; a.d_out = net->dbuf[dcur ^ 1];
                 a.slot_stride = net->slot_stride;
                 a.status = net->status_dev;
-                const int grid = std::min(a.total_tiles, net->sm_count);
+                const int groups = std::min(a.total_tiles, net->sm_count / ctas);
                 if (j > 0) {
                     const LayerDev &Lb = net->layers[j - 1];
                     a.has_relu = Lb.relu_after;
-                    a.out_hi = P; a.out_lo = P_lo;
+                    a.split_out = P_lo != nullptr;
                     a.lamL = Lb.lamL; a.lamU = Lb.lamU; a.nuU = Lb.nuU; a.bias_below = Lb.bias_n;
-                    cert::launch_gemm_tc(cert::TC_EPI_RELU, net->tc_bk, grid, T.a_hi[cur], T.a_lo[cur], T.b_hi,
-                                         T.b_lo, a, T.smem, st);
+                    cert::launch_gemm_tc(cert::TC_EPI_RELU, ctas, groups, T.a_hi[cur], T.a_lo[cur], T.b_hi, T.b_lo,
+                                         T.o_hi[cur ^ 1], T.o_lo[cur ^ 1], a, T.plan.smem_bytes, st);
                 } else {
                     a.l0 = net->l0; a.u0 = net->u0;
-                    cert::launch_gemm_tc(cert::TC_EPI_CONCRETIZE, net->tc_bk, grid, T.a_hi[cur], T.a_lo[cur],
-                                         T.b_hi, T.b_lo, a, T.smem, st);
+                    cert::launch_gemm_tc(cert::TC_EPI_CONCRETIZE, ctas, groups, T.a_hi[cur], T.a_lo[cur], T.b_hi,
+                                         T.b_lo, T.a_hi[cur], T.a_lo[cur], a, T.plan.smem_bytes, st);
                     bounds_in_slots = true;
                 }
                 rec.mark(CERT_CLASS_AFFINE);
                 paths |= 2;
                 cur ^= 1;
                 dcur ^= 1;
-                dslots = T.n_tiles;
+                dslots = T.plan.n_tiles;
                 continue;
             }
             if (Lj.kind == CERT_LAYER_CONV2D) {

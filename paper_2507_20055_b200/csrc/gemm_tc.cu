@@ -10,11 +10,18 @@
 // Every fp32 operand x is held as hi = tf32(x) and lo = tf32(x - hi); the
 // product is hi*hi + lo*hi + hi*lo accumulated in fp32 in tensor memory.
 //
-// One CTA owns a panel of 128 rows and walks the column tiles of W_j, so the
-// thread that owns a row (its TMEM lane) carries that row's constant across
-// all columns in a register: no atomics, fixed summation order.
+// Persistent kernel.  A work tile is a row panel (128 rows per CTA) times a
+// column tile of W_j; the thread that owns a row (its TMEM lane) adds that
+// tile's share of the row constant in a register and writes it to the tile's
+// slot: no atomics, fixed summation order.
+// CTAS = 2: two CTAs of a cluster share a 256-row panel.  Each stages its own
+// 128 rows of Q and its own half of the W_j tile, the leader issues
+// tcgen05.mma.cta_group::2 over both halves (every B byte is staged and read
+// once per pair, not once per CTA), and each CTA runs the epilogue of its own
+// 128 accumulator rows.
 // Warp roles: warp 0 = TMA producer, warp 1 = MMA issuer and TMEM owner,
-// warps 2..5 = epilogue (one TMEM lane quarter each).
+// warps 2..5 = epilogue (one TMEM lane quarter each); results leave through a
+// swizzled shared-memory slab and TMA stores.
 #include <cuda.h>
 
 #include "common.cuh"
@@ -24,13 +31,41 @@ namespace cert {
 
 namespace {
 
-constexpr int BM = 128;
+constexpr int BM = 128;                  // rows per CTA
+constexpr int BK = 32;                   // floats of K per stage: one 128-byte swizzle row
 constexpr int kThreads = 192;
+constexpr int kATileBytes = BM * BK * 4;
+constexpr int kSlabBytes = 32 * 128;     // 32 rows x 32 floats per epilogue warp and output array
+constexpr int kEpiBytes = 4 * 2 * kSlabBytes;
 constexpr unsigned long long kWaitCycles = 2000000000ull;   // about a second
 
 // ---------------------------------------------------------------- PTX wrappers
 __device__ __forceinline__ uint32_t smem_u32(const void *p) {
     return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ uint32_t cluster_id_x() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%clusterid.x;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ uint32_t num_clusters_x() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%nclusterid.x;" : "=r"(r));
+    return r;
+}
+// Address of the same shared-memory location in CTA `rank` of the cluster.
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
 __device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
@@ -39,8 +74,9 @@ __device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t *bar, uint32_t by
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes)
                  : "memory");
 }
-__device__ __forceinline__ void mbar_arrive(uint64_t *bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+// Arrive on a barrier given by its cluster address (this CTA's or the peer's).
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
 __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
     uint32_t ok;
@@ -62,30 +98,71 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity) {
     }
     return true;
 }
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, uint64_t *bar, int x, int y) {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-        ::"r"(dst), "l"(map), "r"(smem_u32(bar)), "r"(x), "r"(y)
-        : "memory");
+// TMA tile load into this CTA's shared memory; `bar_addr` is the cluster address of the barrier
+// that counts the bytes (for a CTA pair: the leader's barrier, for both CTAs' loads).
+template <int CTAS>
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, uint32_t bar_addr, int x, int y) {
+    if (CTAS == 2) {
+        asm volatile(
+            "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes "
+            "[%0], [%1, {%3, %4}], [%2];"
+            ::"r"(dst), "l"(map), "r"(bar_addr), "r"(x), "r"(y)
+            : "memory");
+    } else {
+        asm volatile(
+            "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+            ::"r"(dst), "l"(map), "r"(bar_addr), "r"(x), "r"(y)
+            : "memory");
+    }
 }
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap *map, uint32_t src, int x, int y) {
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+                 ::"l"(map), "r"(src), "r"(x), "r"(y)
+                 : "memory");
+}
+__device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void tcgen05_fence_before() {
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
 }
 __device__ __forceinline__ void tcgen05_fence_after() {
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 }
+// Arrive on `bar` (same offset in every CTA of the group) when the MMAs issued so far retire.
+template <int CTAS>
 __device__ __forceinline__ void tcgen05_commit(uint64_t *bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
-                 : "memory");
+    if (CTAS == 2) {
+        const uint16_t mask = 3;
+        asm volatile(
+            "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+            ::"r"(smem_u32(bar)), "h"(mask)
+            : "memory");
+    } else {
+        asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];"
+                     ::"r"(smem_u32(bar))
+                     : "memory");
+    }
 }
+template <int CTAS>
 __device__ __forceinline__ void mma_tf32(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
                                          uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
-        : "memory");
+    if (CTAS == 2) {
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "setp.ne.b32 p, %4, 0;\n\t"
+            "tcgen05.mma.cta_group::2.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
+            ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+            : "memory");
+    } else {
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "setp.ne.b32 p, %4, 0;\n\t"
+            "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
+            ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+            : "memory");
+    }
 }
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
     asm volatile(
@@ -107,16 +184,15 @@ __device__ __forceinline__ float tf32_round(float x) {
     return __uint_as_float(r);
 }
 
-// Shared-memory matrix descriptor of a K-major tile whose rows are ROW_BYTES long
-// (128 -> 128-byte swizzle, 64 -> 64-byte swizzle); 8-row groups are 8*ROW_BYTES apart.
-template <int ROW_BYTES>
+// Shared-memory matrix descriptor of a K-major tile with 128-byte rows (128-byte swizzle);
+// 8-row groups are 1024 bytes apart.
 __device__ __forceinline__ uint64_t make_desc(uint32_t smem_addr) {
     uint64_t d = 0;
     d |= (uint64_t)((smem_addr >> 4) & 0x3FFF);
     d |= (uint64_t)1 << 16;                        // leading byte offset (unused for swizzled K-major)
-    d |= (uint64_t)((8 * ROW_BYTES) >> 4) << 32;   // stride byte offset between 8-row groups
+    d |= (uint64_t)(1024 >> 4) << 32;              // stride byte offset between 8-row groups
     d |= (uint64_t)1 << 46;                        // descriptor version for sm_100
-    d |= (uint64_t)(ROW_BYTES == 128 ? 2 : 4) << 61;   // SWIZZLE_128B / SWIZZLE_64B
+    d |= (uint64_t)2 << 61;                        // SWIZZLE_128B
     return d;
 }
 
@@ -129,30 +205,33 @@ struct __align__(8) Barriers {
     uint32_t abort_flag;
 };
 
-// Persistent kernel: CTA c works on tiles c, c + gridDim.x, ...; tile t covers rows
-// [128*(t / n_tiles), +128) and column tile t % n_tiles, so the CTAs that run at the same
-// time share row panels and the A operand is fetched from DRAM once.
-template <int EPI, int BK>
+// Group g (a CTA, or a CTA pair) works on tiles g, g + n_groups, ...; tile t covers row panel
+// t / n_tiles and column tile t % n_tiles, so the groups that run at the same time share row
+// panels and the A operand is fetched from DRAM once.
+template <int EPI, int CTAS>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_constant__ CUtensorMap map_a_lo,
                const __grid_constant__ CUtensorMap map_b_hi, const __grid_constant__ CUtensorMap map_b_lo,
+               const __grid_constant__ CUtensorMap map_o_hi, const __grid_constant__ CUtensorMap map_o_lo,
                const TcArgs a) {
-    constexpr int ROW_BYTES = BK * 4;
-    constexpr int KSTEPS = BK / 8;
     extern __shared__ uint8_t smem_raw[];
     // tiles are aligned to 1024 bytes (a whole swizzle pattern)
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const int BN = a.bn;
+    const int BNL = BN / CTAS;                 // rows of the W_j tile this CTA stages
     const int stages = a.stages;
-    const uint32_t a_tile_bytes = BM * ROW_BYTES;
-    const uint32_t b_tile_bytes = (uint32_t)BN * ROW_BYTES;
-    const uint32_t stage_bytes = 2 * a_tile_bytes + 2 * b_tile_bytes;
-    Barriers *bars = reinterpret_cast<Barriers *>(smem + (size_t)stages * stage_bytes);
+    const uint32_t b_tile_bytes = (uint32_t)BNL * BK * 4;
+    const uint32_t stage_bytes = 2 * kATileBytes + 2 * b_tile_bytes;
+    uint8_t *epi_smem = smem + (size_t)stages * stage_bytes;
+    Barriers *bars = reinterpret_cast<Barriers *>(epi_smem + kEpiBytes);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int num_kb = (a.K + BK - 1) / BK;
     const int n_tiles = a.n_tiles;
     const int total_tiles = a.total_tiles;
+    const uint32_t rank = CTAS == 2 ? cluster_ctarank() : 0u;
+    const int group = CTAS == 2 ? (int)cluster_id_x() : (int)blockIdx.x;
+    const int n_groups = CTAS == 2 ? (int)num_clusters_x() : (int)gridDim.x;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < stages; ++s) {
@@ -161,21 +240,30 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_consta
         }
         for (int i = 0; i < 2; ++i) {
             mbar_init(&bars->acc_full[i], 1);
-            mbar_init(&bars->acc_empty[i], 4);
+            mbar_init(&bars->acc_empty[i], 4 * CTAS);
         }
         bars->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
     if (warp == 1) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
-                         smem_u32(&bars->tmem_base)),
-                     "r"((uint32_t)a.tmem_cols)
-                     : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        if (CTAS == 2) {
+            asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
+                             smem_u32(&bars->tmem_base)),
+                         "r"((uint32_t)a.tmem_cols)
+                         : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+        } else {
+            asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
+                             smem_u32(&bars->tmem_base)),
+                         "r"((uint32_t)a.tmem_cols)
+                         : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        }
     }
     tcgen05_fence_before();
     __syncthreads();
+    if (CTAS == 2) cluster_sync_all();      // the peer's barriers exist before anything arrives on them
     tcgen05_fence_after();
     const uint32_t tmem_base = bars->tmem_base;
     volatile uint32_t *abort_flag = &bars->abort_flag;
@@ -187,18 +275,20 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_consta
             uint32_t phase = 0;
             bool ok = true;
             int armed = 0;      // stage loads issued so far
-            for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
-                const int row0 = (t / n_tiles) * BM;
-                const int col0 = (t % n_tiles) * BN;
+            for (int t = group; t < total_tiles && ok; t += n_groups) {
+                const int row0 = (t / n_tiles) * (BM * CTAS) + (int)rank * BM;
+                const int col0 = (t % n_tiles) * BN + (int)rank * BNL;
                 for (int kb = 0; kb < num_kb; ++kb) {
                     if (!mbar_wait(&bars->empty[s], phase ^ 1) || *abort_flag) { ok = false; break; }
                     uint8_t *st = smem + (size_t)s * stage_bytes;
-                    mbar_arrive_expect_tx(&bars->full[s], stage_bytes);
+                    // the leader's barrier counts the bytes of every CTA of the group
+                    if (rank == 0) mbar_arrive_expect_tx(&bars->full[s], stage_bytes * CTAS);
+                    const uint32_t bar = CTAS == 2 ? map_to_cta(smem_u32(&bars->full[s]), 0) : smem_u32(&bars->full[s]);
                     const int kx = kb * BK;
-                    tma_load_2d(smem_u32(st), &map_a_hi, &bars->full[s], kx, row0);
-                    tma_load_2d(smem_u32(st + a_tile_bytes), &map_a_lo, &bars->full[s], kx, row0);
-                    tma_load_2d(smem_u32(st + 2 * a_tile_bytes), &map_b_hi, &bars->full[s], kx, col0);
-                    tma_load_2d(smem_u32(st + 2 * a_tile_bytes + b_tile_bytes), &map_b_lo, &bars->full[s], kx, col0);
+                    tma_load_2d<CTAS>(smem_u32(st), &map_a_hi, bar, kx, row0);
+                    tma_load_2d<CTAS>(smem_u32(st + kATileBytes), &map_a_lo, bar, kx, row0);
+                    tma_load_2d<CTAS>(smem_u32(st + 2 * kATileBytes), &map_b_hi, bar, kx, col0);
+                    tma_load_2d<CTAS>(smem_u32(st + 2 * kATileBytes + b_tile_bytes), &map_b_lo, bar, kx, col0);
                     ++armed;
                     if (++s == stages) { s = 0; phase ^= 1; }
                 }
@@ -206,50 +296,52 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_consta
             if (!ok) {
                 *abort_flag = 1;
                 atomicExch(a.status, 1);
-                // let the copies already in flight land before the CTA gives its shared memory back
-                int back = armed < stages ? armed : stages;
-                int ss = s;
-                uint32_t ph = phase;
-                for (int i = 0; i < back; ++i) {
-                    if (--ss < 0) { ss = stages - 1; ph ^= 1; }
-                    mbar_wait(&bars->full[ss], ph);
+                if (rank == 0) {
+                    // let the copies already in flight land before the CTA gives its shared memory back
+                    int back = armed < stages ? armed : stages;
+                    int ss = s;
+                    uint32_t ph = phase;
+                    for (int i = 0; i < back; ++i) {
+                        if (--ss < 0) { ss = stages - 1; ph ^= 1; }
+                        mbar_wait(&bars->full[ss], ph);
+                    }
                 }
             }
         }
     } else if (warp == 1) {
-        // ------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
+        // ------------------------------------------------------------ MMA issuer (the leader CTA of a pair)
+        if (lane == 0 && rank == 0) {
             const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(BN >> 3) << 17) |
-                                   ((uint32_t)(BM >> 4) << 24);
+                                   ((uint32_t)((BM * CTAS) >> 4) << 24);
             int s = 0;
             uint32_t phase = 0;
             bool ok = true;
             int lt = 0;
-            for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++lt) {
+            for (int t = group; t < total_tiles && ok; t += n_groups, ++lt) {
                 const int acc = lt & 1;
                 const uint32_t acc_phase = (lt >> 1) & 1;
                 if (!mbar_wait(&bars->acc_empty[acc], acc_phase ^ 1) || *abort_flag) { ok = false; break; }
                 tcgen05_fence_after();
-                const uint32_t d_tmem = tmem_base + (uint32_t)(acc * a.bn_pad);
+                const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
                 for (int kb = 0; kb < num_kb; ++kb) {
                     if (!mbar_wait(&bars->full[s], phase) || *abort_flag) { ok = false; break; }
                     tcgen05_fence_after();
                     const uint32_t st = smem_u32(smem + (size_t)s * stage_bytes);
-                    const uint64_t da_hi = make_desc<ROW_BYTES>(st);
-                    const uint64_t da_lo = make_desc<ROW_BYTES>(st + a_tile_bytes);
-                    const uint64_t db_hi = make_desc<ROW_BYTES>(st + 2 * a_tile_bytes);
-                    const uint64_t db_lo = make_desc<ROW_BYTES>(st + 2 * a_tile_bytes + b_tile_bytes);
+                    const uint64_t da_hi = make_desc(st);
+                    const uint64_t da_lo = make_desc(st + kATileBytes);
+                    const uint64_t db_hi = make_desc(st + 2 * kATileBytes);
+                    const uint64_t db_lo = make_desc(st + 2 * kATileBytes + b_tile_bytes);
 #pragma unroll
-                    for (int k = 0; k < KSTEPS; ++k) {
+                    for (int k = 0; k < BK / 8; ++k) {
                         const uint64_t ko = (uint64_t)(k * 2);   // 8 floats = 32 bytes = 2 x 16-byte units
-                        mma_tf32(d_tmem, da_lo + ko, db_hi + ko, idesc, (kb | k) ? 1u : 0u);
-                        mma_tf32(d_tmem, da_hi + ko, db_lo + ko, idesc, 1u);
-                        mma_tf32(d_tmem, da_hi + ko, db_hi + ko, idesc, 1u);
+                        mma_tf32<CTAS>(d_tmem, da_lo + ko, db_hi + ko, idesc, (kb | k) ? 1u : 0u);
+                        mma_tf32<CTAS>(d_tmem, da_hi + ko, db_lo + ko, idesc, 1u);
+                        mma_tf32<CTAS>(d_tmem, da_hi + ko, db_hi + ko, idesc, 1u);
                     }
-                    tcgen05_commit(&bars->empty[s]);     // frees the stage when these MMAs retire
+                    tcgen05_commit<CTAS>(&bars->empty[s]);     // frees the stage (in every CTA) when these MMAs retire
                     if (++s == stages) { s = 0; phase ^= 1; }
                 }
-                if (ok) tcgen05_commit(&bars->acc_full[acc]);
+                if (ok) tcgen05_commit<CTAS>(&bars->acc_full[acc]);
             }
             if (!ok) {
                 *abort_flag = 1;
@@ -259,11 +351,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_consta
     } else {
         // ------------------------------------------------------------ epilogue
         const int quarter = warp & 3;                       // TMEM lane quarter this warp may read
+        uint8_t *slab_hi = epi_smem + (size_t)(warp - 2) * 2 * kSlabBytes;
+        uint8_t *slab_lo = slab_hi + kSlabBytes;
+        const uint32_t acc_empty_addr0 = CTAS == 2 ? map_to_cta(smem_u32(&bars->acc_empty[0]), 0)
+                                                   : smem_u32(&bars->acc_empty[0]);
         bool ok = true;
         int lt = 0;
-        for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++lt) {
+        for (int t = group; t < total_tiles && ok; t += n_groups, ++lt) {
             const int nt = t % n_tiles;
-            const long long r = (long long)(t / n_tiles) * BM + quarter * 32 + lane;
+            const long long warp_row0 = (long long)(t / n_tiles) * (BM * CTAS) + (int)rank * BM + quarter * 32;
+            const long long r = warp_row0 + lane;
             const bool row_ok = r < a.M;
             const long long rr = row_ok ? r : 0;
             const int b = (int)(rr / (2LL * a.n_k));
@@ -274,24 +371,23 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_consta
             const uint32_t acc_phase = (lt >> 1) & 1;
             if (!mbar_wait(&bars->acc_full[acc], acc_phase) || *abort_flag) { ok = false; break; }
             tcgen05_fence_after();
-            const uint32_t t_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * a.bn_pad);
-            const int col_end = min((nt + 1) * BN, a.ld_n);   // columns this tile owns
+            const uint32_t t_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN);
             for (int c0 = 0; c0 < BN; c0 += 32) {
                 const int col0 = nt * BN + c0;
-                if (col0 >= col_end) break;                  // warp-uniform
+                if (col0 >= a.ld_n) break;                   // warp-uniform; ld_n is a multiple of 32
                 uint32_t v[32];
                 __syncwarp();
                 tmem_ld32(t_addr + (uint32_t)c0, v);
                 tmem_ld_wait();
-                if (!row_ok) {
-                    // rows past the end of the matrix: nothing to store
-                } else if (EPI == TC_EPI_RELU) {
-                    float *qh = a.out_hi + (size_t)r * a.ld_n + col0;
-                    float *ql = a.out_lo ? a.out_lo + (size_t)r * a.ld_n + col0 : nullptr;
+                if (EPI == TC_EPI_RELU) {
+                    // the slab is free again once the previous chunk's stores have read it
+                    if (lane == 0) tma_store_wait_read();
+                    __syncwarp();
+                    const uint32_t row_hi = smem_u32(slab_hi) + (uint32_t)lane * 128u;
+                    const uint32_t row_lo = smem_u32(slab_lo) + (uint32_t)lane * 128u;
 #pragma unroll
                     for (int g = 0; g < 8; ++g) {
                         const int col = col0 + g * 4;
-                        if (col >= col_end) break;
                         float q[4];
                         const float4 bz = *reinterpret_cast<const float4 *>(a.bias_below + col);
                         if (a.has_relu) {
@@ -316,26 +412,37 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_consta
                         dacc = fmaf(q[1], bz.y, dacc);
                         dacc = fmaf(q[2], bz.z, dacc);
                         dacc = fmaf(q[3], bz.w, dacc);
-                        if (ql) {
+                        // 16-byte chunk g of this lane's slab row, at its 128-byte-swizzle position
+                        const uint32_t sw = (uint32_t)((g ^ (lane & 7)) << 4);
+                        if (a.split_out) {
                             float h[4], l[4];
 #pragma unroll
                             for (int e = 0; e < 4; ++e) {
                                 h[e] = tf32_round(q[e]);
                                 l[e] = tf32_round(q[e] - h[e]);
                             }
-                            *reinterpret_cast<float4 *>(qh + g * 4) = make_float4(h[0], h[1], h[2], h[3]);
-                            *reinterpret_cast<float4 *>(ql + g * 4) = make_float4(l[0], l[1], l[2], l[3]);
+                            asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(row_hi + sw), "f"(h[0]),
+                                         "f"(h[1]), "f"(h[2]), "f"(h[3]) : "memory");
+                            asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(row_lo + sw), "f"(l[0]),
+                                         "f"(l[1]), "f"(l[2]), "f"(l[3]) : "memory");
                         } else {
-                            *reinterpret_cast<float4 *>(qh + g * 4) = make_float4(q[0], q[1], q[2], q[3]);
+                            asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(row_hi + sw), "f"(q[0]),
+                                         "f"(q[1]), "f"(q[2]), "f"(q[3]) : "memory");
                         }
                     }
-                } else {
+                    fence_async_smem();
+                    __syncwarp();
+                    // rows past the end of the matrix land in scratch rows of the workspace or are clipped
+                    if (lane == 0) {
+                        tma_store_2d(&map_o_hi, smem_u32(slab_hi), col0, (int)warp_row0);
+                        if (a.split_out) tma_store_2d(&map_o_lo, smem_u32(slab_lo), col0, (int)warp_row0);
+                        tma_store_commit();
+                    }
+                } else if (row_ok) {
                     const float *lrow = a.l0 + (size_t)b * a.ld_n + col0;
                     const float *urow = a.u0 + (size_t)b * a.ld_n + col0;
 #pragma unroll
                     for (int g = 0; g < 8; ++g) {
-                        const int col = col0 + g * 4;
-                        if (col >= col_end) break;
                         const float4 l4 = *reinterpret_cast<const float4 *>(lrow + g * 4);
                         const float4 u4 = *reinterpret_cast<const float4 *>(urow + g * 4);
                         const float lo4[4] = {l4.x, l4.y, l4.z, l4.w}, up4[4] = {u4.x, u4.y, u4.z, u4.w};
@@ -350,7 +457,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_consta
             }
             tcgen05_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(&bars->acc_empty[acc]);
+            if (lane == 0) mbar_arrive_cluster(acc_empty_addr0 + (uint32_t)(acc * sizeof(uint64_t)));
             // This tile's share of the row constant (of the bound, for the concretising
             // epilogue) goes to slot nt; the tile of column 0 also carries the constant so far.
             if (row_ok) {
@@ -363,16 +470,23 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_consta
                 a.d_out[(size_t)nt * a.slot_stride + r] = tot;
             }
         }
+        if (EPI == TC_EPI_RELU && lane == 0) tma_store_wait_all();
         if (!ok && lane == 0) atomicExch(a.status, 1);
     }
 
     tcgen05_fence_before();
     __syncthreads();
+    if (CTAS == 2) cluster_sync_all();      // no CTA leaves while its peer may still reach into it
     if (warp == 1) {
         tcgen05_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base),
-                     "r"((uint32_t)a.tmem_cols)
-                     : "memory");
+        if (CTAS == 2)
+            asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base),
+                         "r"((uint32_t)a.tmem_cols)
+                         : "memory");
+        else
+            asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base),
+                         "r"((uint32_t)a.tmem_cols)
+                         : "memory");
     }
 }
 
@@ -381,6 +495,25 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t
                                   CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
                                   CUtensorMapFloatOOBfill);
 EncodeTiledFn g_encode = nullptr;
+
+template <int EPI, int CTAS>
+void launch_one(int groups, const CUtensorMap &ah, const CUtensorMap &al, const CUtensorMap &bh,
+                const CUtensorMap &bl, const CUtensorMap &oh, const CUtensorMap &ol, const TcArgs &args,
+                int smem_bytes, cudaStream_t st) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(groups * CTAS), 1, 1);
+    cfg.blockDim = dim3(kThreads, 1, 1);
+    cfg.dynamicSmemBytes = (size_t)smem_bytes;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = CTAS;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaLaunchKernelEx(&cfg, gemm_tc_kernel<EPI, CTAS>, ah, al, bh, bl, oh, ol, args);
+}
 
 }  // namespace
 
@@ -397,71 +530,84 @@ bool tc_driver_init() {
     return true;
 }
 
-bool tc_prepare_kernels() {
+bool tc_prepare_kernels(bool *pair_ok) {
     cudaError_t e[4];
-    e[0] = cudaFuncSetAttribute(gemm_tc_kernel<TC_EPI_RELU, 32>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemMax);
-    e[1] = cudaFuncSetAttribute(gemm_tc_kernel<TC_EPI_CONCRETIZE, 32>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemMax);
-    e[2] = cudaFuncSetAttribute(gemm_tc_kernel<TC_EPI_RELU, 16>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemMax);
-    e[3] = cudaFuncSetAttribute(gemm_tc_kernel<TC_EPI_CONCRETIZE, 16>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemMax);
+    e[0] = cudaFuncSetAttribute(gemm_tc_kernel<TC_EPI_RELU, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemMax);
+    e[1] = cudaFuncSetAttribute(gemm_tc_kernel<TC_EPI_CONCRETIZE, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemMax);
+    e[2] = cudaFuncSetAttribute(gemm_tc_kernel<TC_EPI_RELU, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemMax);
+    e[3] = cudaFuncSetAttribute(gemm_tc_kernel<TC_EPI_CONCRETIZE, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemMax);
     for (int i = 0; i < 4; ++i)
         if (e[i] != cudaSuccess) {
             cudaGetLastError();
             return false;
         }
+    // can a cluster of two such CTAs be resident?
+    *pair_ok = false;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(2, 1, 1);
+    cfg.blockDim = dim3(kThreads, 1, 1);
+    cfg.dynamicSmemBytes = kTcSmemMax;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    int n_clusters = 0;
+    if (cudaOccupancyMaxActiveClusters(&n_clusters, gemm_tc_kernel<TC_EPI_RELU, 2>, &cfg) == cudaSuccess)
+        *pair_ok = n_clusters >= 1;
+    else
+        cudaGetLastError();
     return true;
 }
 
-// 2D fp32 tensor [outer][inner] with row pitch `pitch_floats`; box = bk floats x box_outer rows,
-// swizzle span = one box row (128 bytes for bk = 32, 64 bytes for bk = 16).
 bool tc_make_map(TcMap *m, const float *base, long long inner, long long outer, long long pitch_floats,
-                 int box_outer, int bk) {
+                 int box_outer) {
     if (!g_encode) return false;
     static_assert(sizeof(TcMap) == sizeof(CUtensorMap), "tensor map size");
     cuuint64_t dims[2] = {(cuuint64_t)inner, (cuuint64_t)outer};
     cuuint64_t strides[1] = {(cuuint64_t)pitch_floats * sizeof(float)};
-    cuuint32_t box[2] = {(cuuint32_t)bk, (cuuint32_t)box_outer};
+    cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)box_outer};
     cuuint32_t estr[2] = {1u, 1u};
     CUresult r = g_encode(reinterpret_cast<CUtensorMap *>(m), CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2,
                           const_cast<float *>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                          bk == 32 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B,
-                          CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+                          CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS;
 }
 
-void tc_tile_plan(int N, int bk, int *bn, int *bn_pad, int *n_tiles, int *stages, int *tmem_cols,
-                  int *smem_bytes) {
-    int nt = (N + 255) / 256;
-    int b = ((N + nt - 1) / nt + 15) / 16 * 16;
-    if (b < 16) b = 16;
-    *bn = b;
-    *bn_pad = (b + 31) / 32 * 32;
-    *n_tiles = nt;
-    int stage_bytes = (2 * BM + 2 * b) * bk * 4;
-    int st = (kTcSmemMax - 2048) / stage_bytes;
-    if (st > 8) st = 8;
-    *stages = st;
+TcPlan tc_tile_plan(int N, int ctas) {
+    TcPlan p;
+    p.n_tiles = (N + 255) / 256;
+    int b = ((N + p.n_tiles - 1) / p.n_tiles + 31) / 32 * 32;
+    p.bn = b;
+    const int stage_bytes = 2 * kATileBytes + 2 * (b / ctas) * BK * 4;
+    const int fixed = kEpiBytes + (int)sizeof(Barriers) + 1024;   // epilogue slabs, barriers, alignment slack
+    int st = (kTcSmemMax - fixed) / stage_bytes;
+    p.stages = st > 8 ? 8 : st;
     int cols = 32;
-    while (cols < 2 * *bn_pad) cols *= 2;
-    *tmem_cols = cols;
-    *smem_bytes = st * stage_bytes + 2048;
+    while (cols < 2 * b) cols *= 2;
+    p.tmem_cols = cols;
+    p.smem_bytes = p.stages * stage_bytes + fixed;
+    return p;
 }
 
-void launch_gemm_tc(int epi, int bk, int grid, const TcMap &a_hi, const TcMap &a_lo, const TcMap &b_hi,
-                    const TcMap &b_lo, const TcArgs &args, int smem_bytes, cudaStream_t st) {
+void launch_gemm_tc(int epi, int ctas, int groups, const TcMap &a_hi, const TcMap &a_lo, const TcMap &b_hi,
+                    const TcMap &b_lo, const TcMap &o_hi, const TcMap &o_lo, const TcArgs &args, int smem_bytes,
+                    cudaStream_t st) {
     const CUtensorMap &ah = reinterpret_cast<const CUtensorMap &>(a_hi);
     const CUtensorMap &al = reinterpret_cast<const CUtensorMap &>(a_lo);
     const CUtensorMap &bh = reinterpret_cast<const CUtensorMap &>(b_hi);
     const CUtensorMap &bl = reinterpret_cast<const CUtensorMap &>(b_lo);
-    if (bk == 32) {
-        if (epi == TC_EPI_RELU)
-            gemm_tc_kernel<TC_EPI_RELU, 32><<<grid, kThreads, smem_bytes, st>>>(ah, al, bh, bl, args);
-        else
-            gemm_tc_kernel<TC_EPI_CONCRETIZE, 32><<<grid, kThreads, smem_bytes, st>>>(ah, al, bh, bl, args);
+    const CUtensorMap &oh = reinterpret_cast<const CUtensorMap &>(o_hi);
+    const CUtensorMap &ol = reinterpret_cast<const CUtensorMap &>(o_lo);
+    if (ctas == 2) {
+        if (epi == TC_EPI_RELU) launch_one<TC_EPI_RELU, 2>(groups, ah, al, bh, bl, oh, ol, args, smem_bytes, st);
+        else launch_one<TC_EPI_CONCRETIZE, 2>(groups, ah, al, bh, bl, oh, ol, args, smem_bytes, st);
     } else {
-        if (epi == TC_EPI_RELU)
-            gemm_tc_kernel<TC_EPI_RELU, 16><<<grid, kThreads, smem_bytes, st>>>(ah, al, bh, bl, args);
-        else
-            gemm_tc_kernel<TC_EPI_CONCRETIZE, 16><<<grid, kThreads, smem_bytes, st>>>(ah, al, bh, bl, args);
+        if (epi == TC_EPI_RELU) launch_one<TC_EPI_RELU, 1>(groups, ah, al, bh, bl, oh, ol, args, smem_bytes, st);
+        else launch_one<TC_EPI_CONCRETIZE, 1>(groups, ah, al, bh, bl, oh, ol, args, smem_bytes, st);
     }
 }
 

@@ -15,16 +15,24 @@ struct alignas(64) TcMap {
     unsigned char bytes[128];
 };
 
+// Tile plan of the back-step through one layer (N = neurons below the layer).
+struct TcPlan {
+    int bn;          // columns per tile: a multiple of 32, at most 256
+    int n_tiles;     // column tiles
+    int stages;      // pipeline stages of K
+    int tmem_cols;   // tensor-memory columns (two accumulators)
+    int smem_bytes;
+};
+
 struct TcArgs {
     long long M;     // rows of the coefficient matrix = batch * 2 * n_k
     int K;           // neurons of layer j (columns of Q, rows of W_j)
     int n_k;         // neurons of the layer being bounded (decodes a row into box, side, neuron)
     int ld_n;        // padded width of the output (neurons below layer j)
-    int bn, bn_pad, n_tiles, stages, tmem_cols;
-    int total_tiles; // row panels x column tiles
+    int bn, n_tiles, stages, tmem_cols;
+    int total_tiles; // row panels x column tiles (a row panel is 128 rows per CTA of the group)
     int has_relu;    // a ReLU sits on the neurons below layer j
-    // ReLU back-step epilogue
-    float *out_hi, *out_lo;                      // Q' [M][ld_n]; out_lo == nullptr: unsplit fp32 in out_hi
+    int split_out;   // ReLU epilogue: store the result as a TF32 pair (a tensor-core step follows)
     const float *lamL, *lamU, *nuU;              // [batch][ld_n]
     const float *bias_below;                     // [ld_n] bias of the affine layer below (next step)
     // concretisation epilogue
@@ -41,12 +49,16 @@ struct TcArgs {
 };
 
 bool tc_driver_init();
-bool tc_prepare_kernels();
+// Sets the kernels' shared-memory limits; *pair_ok tells whether the two-CTA form can be launched.
+bool tc_prepare_kernels(bool *pair_ok);
+// 2D fp32 tensor [outer][inner] with row pitch `pitch_floats`; box = 32 floats x box_outer rows, 128-byte swizzle.
 bool tc_make_map(TcMap *m, const float *base, long long inner, long long outer, long long pitch_floats,
-                 int box_outer, int bk);
-void tc_tile_plan(int N, int bk, int *bn, int *bn_pad, int *n_tiles, int *stages, int *tmem_cols,
-                  int *smem_bytes);
-void launch_gemm_tc(int epi, int bk, int grid, const TcMap &a_hi, const TcMap &a_lo, const TcMap &b_hi,
-                    const TcMap &b_lo, const TcArgs &args, int smem_bytes, cudaStream_t st);
+                 int box_outer);
+TcPlan tc_tile_plan(int N, int ctas);
+// ctas = 1: one CTA per 128-row panel; ctas = 2: a CTA pair shares a 256-row panel (cta_group::2).
+// `groups` = CTAs (ctas = 1) or CTA pairs (ctas = 2) to launch.
+void launch_gemm_tc(int epi, int ctas, int groups, const TcMap &a_hi, const TcMap &a_lo, const TcMap &b_hi,
+                    const TcMap &b_lo, const TcMap &o_hi, const TcMap &o_lo, const TcArgs &args, int smem_bytes,
+                    cudaStream_t st);
 
 }  // namespace cert
