@@ -25,6 +25,15 @@ import numpy as np
 
 from paper_2507_20055_b200 import workloads as wl
 
+# DRAM traffic of the dominant kernel, from the ncu capture summarised under profiles/ (read + written bytes
+# of one launch of the ReLU-epilogue contraction, 16-box case, per row of the coefficient matrix; traffic
+# grows in proportion to the rows, so a full launch is rows x this figure).  None for workloads not captured.
+NCU_TRAFFIC_BYTES_PER_ROW = {
+    "fc6x1024_b128": {"bytes_per_row": (313.425152e6 + 215.404800e6) / 32768.0,
+                      "kernel": "gemm_tc_kernel<TC_EPI_RELU, 2>",
+                      "source": "profiles/gemm_tc_kernel_fc6x1024.md (16 boxes, scaled by rows)"},
+}
+
 METRIC = "input boxes/sec fully bounded (DeepPoly)"
 UNIT = "boxes/s"
 
@@ -283,10 +292,16 @@ def main():
         # TF32 dense peak = measured bf16 (sustained: the kernel runs inside a long step) x 1/2 (nominal ratio)
         tc_peak = peaks["bf16_tflops_sustained"] * 0.5 / 3.0
         used_tc = dom == "affine" and bool(net.last_contraction_paths() & 2)
+        traffic, traffic_note = None, "no ncu capture for this workload / contraction mode"
+        cap = NCU_TRAFFIC_BYTES_PER_ROW.get(w.name)
+        if cap and used_tc and (net.last_contraction_paths() & 4):
+            rows_per_launch = 2.0 * B * max(l.n_out for l in w.layers[1:-1] or w.layers[1:])
+            traffic = cap["bytes_per_row"] * rows_per_launch
+            traffic_note = f"{cap['kernel']}: {cap['source']}"
         roof = {"bound": "tensor" if used_tc else "alu",
                 "achieved": achieved, "peak": tc_peak if used_tc else ffma_peak, "unit": "TFLOP/s",
                 "frac": (achieved / (tc_peak if used_tc else ffma_peak)) if achieved else None,
-                "traffic": None,
+                "traffic": traffic, "traffic_note": traffic_note,
                 "kernel": dom + " back-step", "launches_per_step": dom_n // max(1, args.steps),
                 "avg_launch_ms": dom_ms / dom_n if dom_n else None,
                 "flops_per_step": fl[dom], "flops_per_step_all_backsteps": flops_call,

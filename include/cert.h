@@ -124,10 +124,14 @@ cert_status_t cert_net_last_status(cert_net_t *net, void *stream);
  *   FFMA:    fp32 FMA units, unfused ReLU step and concretisation kernels.
  *   TC3XTF32: tcgen05 tensor cores with a 3-term TF32 split (fp32-accurate),
  *            ReLU back-step and concretisation fused into the epilogue.
+ * Conv back-steps always run on the FMA units, with the same fusions.
+ * (The environment variable CERT_TC_CTAS=1, read at create, keeps the
+ * tensor-core kernel to one CTA per row panel instead of CTA pairs.)
  */
 enum { CERT_CONTRACTION_AUTO = 0, CERT_CONTRACTION_FFMA = 1, CERT_CONTRACTION_TC3XTF32 = 2 };
 cert_status_t cert_net_set_contraction(cert_net_t *net, int mode);
-/* Which contraction kernels the most recent call ran: bit 0 = FFMA, bit 1 = TC3XTF32. */
+/* Which contraction kernels the most recent call ran: bit 0 = FFMA, bit 1 = TC3XTF32,
+ * bit 2 = the TC3XTF32 kernel ran in its CTA-pair form (tcgen05 cta_group::2). */
 int cert_net_last_contraction_paths(const cert_net_t *net);
 
 /*

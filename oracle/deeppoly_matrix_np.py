@@ -59,8 +59,13 @@ def box(centers, eps, clip_lo, clip_hi):
     return l0, u0
 
 
-def deeppoly_matrix(layers, centers, eps, clip_lo=0.0, clip_hi=1.0, decision_fp32=True):
-    """Returns lb, ub [batch, n_total] float64 and codes [batch, n_relu] uint8."""
+def deeppoly_matrix(layers, centers, eps, clip_lo=0.0, clip_hi=1.0, decision_fp32=True, backsteps=None):
+    """Returns lb, ub [batch, n_total] float64 and codes [batch, n_relu] uint8.
+
+    backsteps: optional list with one traversal-step count per affine layer (negative: to the
+    input).  A traversal that stops early is simplified against the concrete bounds of the
+    neurons it reached (Section 6.2, DeepPoly_p; 0 everywhere is the IBP listing, 0 except at
+    the last layer the CROWN-IBP listing of Appendix C)."""
     A = [dense_matrix(l) for l in layers]
     bias = [dense_bias(l) for l in layers]
     L0, U0 = box(centers, eps, clip_lo, clip_hi)
@@ -73,11 +78,14 @@ def deeppoly_matrix(layers, centers, eps, clip_lo=0.0, clip_hi=1.0, decision_fp3
     for b in range(batch):
         l0, u0 = L0[b], U0[b]
         lam_l, lam_u, nu_u = [], [], []
+        act_l, act_u = [], []       # concrete bounds of each layer's outputs (after its ReLU, if any)
         off, coff = 0, 0
         for k, layer in enumerate(layers):
             Cl, Cu = A[k].copy(), A[k].copy()
             dl, du = bias[k].copy(), bias[k].copy()
-            for j in range(k - 1, -1, -1):
+            limit = -1 if backsteps is None else int(backsteps[k])
+            stop_at = -1 if limit < 0 else max(k - 1 - limit, -1)   # layer whose outputs the expression ends on
+            for j in range(k - 1, stop_at, -1):
                 if layers[j].relu_after:
                     Clp, Clm = np.clip(Cl, 0.0, None), np.clip(Cl, None, 0.0)
                     Cup, Cum = np.clip(Cu, 0.0, None), np.clip(Cu, None, 0.0)
@@ -89,9 +97,14 @@ def deeppoly_matrix(layers, centers, eps, clip_lo=0.0, clip_hi=1.0, decision_fp3
                 du = du + Cu @ bias[j]
                 Cl = Cl @ A[j]
                 Cu = Cu @ A[j]
-            lb = np.clip(Cl, 0.0, None) @ l0 + np.clip(Cl, None, 0.0) @ u0 + dl
-            ub = np.clip(Cu, 0.0, None) @ u0 + np.clip(Cu, None, 0.0) @ l0 + du
+            lo_in, up_in = (l0, u0) if stop_at < 0 else (act_l[stop_at], act_u[stop_at])
+            lb = np.clip(Cl, 0.0, None) @ lo_in + np.clip(Cl, None, 0.0) @ up_in + dl
+            ub = np.clip(Cu, 0.0, None) @ up_in + np.clip(Cu, None, 0.0) @ lo_in + du
             n_k = lb.shape[0]
+            if layer.relu_after:
+                act_l.append(np.maximum(lb, 0.0)); act_u.append(np.maximum(ub, 0.0))
+            else:
+                act_l.append(lb); act_u.append(ub)
             lb_all[b, off:off + n_k], ub_all[b, off:off + n_k] = lb, ub
             off += n_k
             if layer.relu_after:

@@ -207,7 +207,8 @@ static void relu_relaxation(double l, double u, int decision_fp32, double *lamL,
 /* One box: bounds of every affine neuron, layer after layer
  * (flow(forward, priority = layer)). */
 static int one_box(const oracle_layer_t *layers, int n_layers, const float *center, float eps,
-                   float clip_lo, float clip_hi, int decision_fp32, int max_backsteps,
+                   float clip_lo, float clip_hi, int decision_fp32, int max_backsteps_all,
+                   const int *backsteps_per_layer,
                    double *lb, double *ub, unsigned char *codes, double *margins)
 {
     int n0 = layer_n_in(&layers[0]);
@@ -238,6 +239,8 @@ static int one_box(const oracle_layer_t *layers, int n_layers, const float *cent
     int code_off = 0;
     for (int k = 0; k < n_layers; ++k) {
         int n_k = layer_n_out(&layers[k]);
+        /* how many traversal steps the expressions of this layer take: all of them, or p */
+        int max_backsteps = backsteps_per_layer ? backsteps_per_layer[k] : max_backsteps_all;
         for (int i = 0; i < n_k; ++i) {
             for (int upper = 0; upper < 2; ++upper) {
                 double d;
@@ -308,13 +311,23 @@ int oracle_num_relu_neurons(const oracle_layer_t *layers, int n_layers)
 /*
  * lb, ub: [batch][n_total] float64, affine layers concatenated in order.
  * codes, margins (optional, may be NULL): [batch][n_relu].
- * max_backsteps < 0: full DeepPoly.  max_backsteps = p >= 0: DeepPoly_p.
+ * max_backsteps < 0: full DeepPoly.  max_backsteps = p >= 0: DeepPoly_p
+ * (Section 6.2: the traversal runs for p iterations at every affine layer; one
+ * iteration here is one affine layer of the network together with the Relu
+ * layer on top of it, so that p = number of affine layers is full DeepPoly).
+ * backsteps_per_layer (optional, [n_layers]): a step count per affine layer,
+ * overriding max_backsteps; this covers the other certifiers of Appendix C
+ * that differ from DeepPoly only in where they traverse:
+ *   IBP listing:       Affine -> map(simplify_*) of prev.dot(w)+b, no traversal: 0 everywhere;
+ *   CROWN-IBP listing: the same, except curr[last_layer] == 1 -> backsubs_*: 0, ..., 0, -1,
+ * with the Relu transformer (relu(l), relu(u), relu_n, compute_upper) unchanged.
  * n_threads: boxes are independent and are the only parallel axis.
  * Returns 0, or 1 on allocation failure, 2 on a malformed network.
  */
-int oracle_deeppoly(const oracle_layer_t *layers, int n_layers, const float *centers, float eps,
-                    int batch, float clip_lo, float clip_hi, int decision_fp32, int max_backsteps,
-                    int n_threads, double *lb, double *ub, unsigned char *codes, double *margins)
+int oracle_backsub(const oracle_layer_t *layers, int n_layers, const float *centers, float eps,
+                   int batch, float clip_lo, float clip_hi, int decision_fp32, int max_backsteps,
+                   const int *backsteps_per_layer,
+                   int n_threads, double *lb, double *ub, unsigned char *codes, double *margins)
 {
     if (n_layers < 1 || batch < 0) return 2;
     for (int k = 1; k < n_layers; ++k)
@@ -331,7 +344,7 @@ int oracle_deeppoly(const oracle_layer_t *layers, int n_layers, const float *cen
 #pragma omp parallel for schedule(dynamic, 1)
     for (int b = 0; b < batch; ++b) {
         int e = one_box(layers, n_layers, centers + (size_t)b * n0, eps, clip_lo, clip_hi,
-                        decision_fp32, max_backsteps, lb + (size_t)b * n_total,
+                        decision_fp32, max_backsteps, backsteps_per_layer, lb + (size_t)b * n_total,
                         ub + (size_t)b * n_total, codes ? codes + (size_t)b * n_relu : NULL,
                         margins ? margins + (size_t)b * n_relu : NULL);
         if (e) {
@@ -340,6 +353,14 @@ int oracle_deeppoly(const oracle_layer_t *layers, int n_layers, const float *cen
         }
     }
     return err;
+}
+
+int oracle_deeppoly(const oracle_layer_t *layers, int n_layers, const float *centers, float eps,
+                    int batch, float clip_lo, float clip_hi, int decision_fp32, int max_backsteps,
+                    int n_threads, double *lb, double *ub, unsigned char *codes, double *margins)
+{
+    return oracle_backsub(layers, n_layers, centers, eps, batch, clip_lo, clip_hi, decision_fp32,
+                          max_backsteps, NULL, n_threads, lb, ub, codes, margins);
 }
 
 int oracle_max_threads(void)

@@ -41,6 +41,7 @@ def _load():
     if _lib is None:
         _lib = ctypes.CDLL(build())
         _lib.oracle_deeppoly.restype = ctypes.c_int
+        _lib.oracle_backsub.restype = ctypes.c_int
         _lib.oracle_num_neurons.restype = ctypes.c_int
         _lib.oracle_num_relu_neurons.restype = ctypes.c_int
         _lib.oracle_max_threads.restype = ctypes.c_int
@@ -76,9 +77,11 @@ def _marshal(layers):
 
 
 def deeppoly(layers, centers, eps, clip_lo=0.0, clip_hi=1.0, decision_fp32=True,
-             max_backsteps: int = -1, n_threads: Optional[int] = None):
+             max_backsteps: int = -1, n_threads: Optional[int] = None, backsteps_per_layer=None):
     """Bounds of every affine neuron for every box.
 
+    max_backsteps = p >= 0 is DeepPoly_p; backsteps_per_layer (one count per affine layer,
+    negative = traverse to the input) overrides it.
     Returns dict(lb, ub: float64 [batch, n_total]; codes: uint8 [batch, n_relu];
     margins: float64 [batch, n_relu]).  Layers are concatenated in order.
     """
@@ -92,13 +95,30 @@ def deeppoly(layers, centers, eps, clip_lo=0.0, clip_hi=1.0, decision_fp32=True,
     ub = np.empty((batch, n_total), dtype=np.float64)
     codes = np.empty((batch, n_relu), dtype=np.uint8)
     margins = np.empty((batch, n_relu), dtype=np.float64)
-    rc = lib.oracle_deeppoly(arr, ctypes.c_int(len(layers)), ctypes.c_void_p(centers.ctypes.data),
-                             ctypes.c_float(eps), ctypes.c_int(batch), ctypes.c_float(clip_lo),
-                             ctypes.c_float(clip_hi), ctypes.c_int(int(decision_fp32)),
-                             ctypes.c_int(max_backsteps), ctypes.c_int(n_threads or 0),
-                             ctypes.c_void_p(lb.ctypes.data), ctypes.c_void_p(ub.ctypes.data),
-                             ctypes.c_void_p(codes.ctypes.data), ctypes.c_void_p(margins.ctypes.data))
+    steps = None
+    if backsteps_per_layer is not None:
+        steps = np.ascontiguousarray(backsteps_per_layer, dtype=np.int32)
+        assert steps.shape == (len(layers),)
+    rc = lib.oracle_backsub(arr, ctypes.c_int(len(layers)), ctypes.c_void_p(centers.ctypes.data),
+                            ctypes.c_float(eps), ctypes.c_int(batch), ctypes.c_float(clip_lo),
+                            ctypes.c_float(clip_hi), ctypes.c_int(int(decision_fp32)),
+                            ctypes.c_int(max_backsteps),
+                            ctypes.c_void_p(steps.ctypes.data if steps is not None else None),
+                            ctypes.c_int(n_threads or 0),
+                            ctypes.c_void_p(lb.ctypes.data), ctypes.c_void_p(ub.ctypes.data),
+                            ctypes.c_void_p(codes.ctypes.data), ctypes.c_void_p(margins.ctypes.data))
     if rc != 0:
-        raise RuntimeError(f"oracle_deeppoly failed with code {rc}")
+        raise RuntimeError(f"oracle_backsub failed with code {rc}")
     del keep
     return {"lb": lb, "ub": ub, "codes": codes, "margins": margins}
+
+
+def ibp(layers, centers, eps, clip_lo=0.0, clip_hi=1.0, **kw):
+    """IBP listing of Appendix C: no traversal at any layer."""
+    return deeppoly(layers, centers, eps, clip_lo, clip_hi, backsteps_per_layer=[0] * len(layers), **kw)
+
+
+def crown_ibp(layers, centers, eps, clip_lo=0.0, clip_hi=1.0, **kw):
+    """CROWN-IBP listing of Appendix C: intervals everywhere, back-substitution at the last layer."""
+    return deeppoly(layers, centers, eps, clip_lo, clip_hi,
+                    backsteps_per_layer=[0] * (len(layers) - 1) + [-1], **kw)

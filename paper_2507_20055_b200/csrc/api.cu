@@ -48,7 +48,7 @@ struct cert_net {
     float *centers_dev = nullptr, *lb_dev = nullptr, *ub_dev = nullptr;
     int last_batch = 0;
     int last_launches = 0;
-    int last_paths = 0;              // bit 0: an FFMA contraction ran, bit 1: a tensor-core one
+    int last_paths = 0;              // bit 0: an FFMA contraction ran, bit 1: a tensor-core one, bit 2: in CTA pairs
     // optional per-launch event timing (events are created when profiling is switched on)
     bool profiling = false;
     std::vector<cudaEvent_t> prof_events;
@@ -437,7 +437,7 @@ cert_status_t cert_deeppoly_bounds(cert_net_t *net, const float *centers, float 
                     bounds_in_slots = true;
                 }
                 rec.mark(CERT_CLASS_AFFINE);
-                paths |= 2;
+                paths |= 2 | (net->tc_ctas == 2 ? 4 : 0);
                 cur ^= 1;
                 dcur ^= 1;
                 dslots = T.plan.n_tiles;
