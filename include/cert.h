@@ -85,6 +85,26 @@ cert_status_t cert_net_create(const cert_layer_desc_t *layers, int n_layers, int
 cert_status_t cert_deeppoly_bounds(cert_net_t *net, const float *centers, float eps, int batch,
                                    float *lb_out, float *ub_out, void *stream);
 
+/*
+ * The same flow with a bounded traversal (Section 6.2, DeepPoly_p: "at each
+ * Affine layer, the backsubstitution is performed for p iterations"; one
+ * iteration = one affine layer together with the Relu layer on top of it).
+ *   backsteps  HOST int [n_layers] or NULL.  backsteps[k] >= 0: the expressions
+ *            of affine layer k (0-based) are back-substituted through at most
+ *            that many layers and then simplified (map(simplify_lower/upper))
+ *            against the concrete bounds of the neurons reached: relu(l),
+ *            relu(u) of that layer's neurons under a ReLU, else l, u, or the
+ *            input box.  Negative, or NULL: to the input (DeepPoly).
+ * Certifiers of Appendix C that differ from DeepPoly only in this respect:
+ *   IBP listing        backsteps = {0, 0, ..., 0}
+ *   CROWN-IBP listing  backsteps = {0, ..., 0, -1}   (curr[last_layer] == 1 -> backsubs_*)
+ * The Relu transformer (relaxation from the resulting bounds) is the same in
+ * all of them.  Everything else is as for cert_deeppoly_bounds, which is this
+ * call with backsteps = NULL.  The array is read before the call returns.
+ */
+cert_status_t cert_backsub_bounds(cert_net_t *net, const float *centers, float eps, int batch,
+                                  const int *backsteps, float *lb_out, float *ub_out, void *stream);
+
 /* Same, with HOST buffers (pageable or pinned): copies centers to the device,
  * runs cert_deeppoly_bounds, copies the bounds back and waits for the stream. */
 cert_status_t cert_deeppoly_bounds_host(cert_net_t *net, const float *centers_host, float eps,

@@ -26,7 +26,8 @@ CERT_OK = 0
 CONTRACTION_AUTO, CONTRACTION_FFMA, CONTRACTION_TC3XTF32 = 0, 1, 2
 
 EXPORTS = [
-    "cert_net_create", "cert_deeppoly_bounds", "cert_deeppoly_bounds_host", "cert_net_destroy",
+    "cert_net_create", "cert_deeppoly_bounds", "cert_backsub_bounds", "cert_deeppoly_bounds_host",
+    "cert_net_destroy",
     "cert_net_num_neurons", "cert_net_num_relu_neurons", "cert_net_branch_codes",
     "cert_net_last_status", "cert_net_set_contraction", "cert_net_last_launch_count",
     "cert_net_backstep_flops", "cert_status_string", "cert_net_set_profiling", "cert_net_profile",
@@ -47,6 +48,8 @@ _lib.cert_net_create.argtypes = [ctypes.POINTER(cert_layer_desc_t), _i, _i, _f, 
 _lib.cert_net_create.restype = _i
 _lib.cert_deeppoly_bounds.argtypes = [_vp, _vp, _f, _i, _vp, _vp, _vp]
 _lib.cert_deeppoly_bounds.restype = _i
+_lib.cert_backsub_bounds.argtypes = [_vp, _vp, _f, _i, _vp, _vp, _vp, _vp]
+_lib.cert_backsub_bounds.restype = _i
 _lib.cert_deeppoly_bounds_host.argtypes = [_vp, _vp, _f, _i, _vp, _vp, _vp]
 _lib.cert_deeppoly_bounds_host.restype = _i
 _lib.cert_net_destroy.argtypes = [_vp]
@@ -125,6 +128,7 @@ class CertNet:
         self.n0 = int(layers[0].n_in)
         self.n_total = int(_lib.cert_net_num_neurons(h))
         self.n_relu = int(_lib.cert_net_num_relu_neurons(h))
+        self.n_layers = len(layers)
 
     # -- raw-pointer form (what the C ABI takes) --
     def deeppoly_bounds_ptr(self, centers_ptr: int, eps: float, batch: int, lb_ptr: int, ub_ptr: int,
@@ -146,6 +150,35 @@ class CertNet:
         self.deeppoly_bounds_ptr(centers.data_ptr(), eps, batch, lb_out.data_ptr(), ub_out.data_ptr(),
                                  st.cuda_stream)
         return lb_out, ub_out
+
+    def backsub_bounds(self, centers, eps: float, backsteps=None, lb_out=None, ub_out=None, stream=None):
+        """cert_backsub_bounds: backsteps = one traversal depth per affine layer (negative: to the input)."""
+        import torch
+        assert centers.is_cuda and centers.dtype == torch.float32 and centers.is_contiguous()
+        batch = centers.shape[0]
+        assert centers.shape[1] == self.n0
+        if lb_out is None:
+            lb_out = torch.empty((batch, self.n_total), dtype=torch.float32, device=centers.device)
+        if ub_out is None:
+            ub_out = torch.empty((batch, self.n_total), dtype=torch.float32, device=centers.device)
+        st = stream if stream is not None else torch.cuda.current_stream(centers.device)
+        steps = None
+        if backsteps is not None:
+            assert len(backsteps) == self.n_layers
+            steps = (ctypes.c_int * self.n_layers)(*[int(x) for x in backsteps])
+        _check(_lib.cert_backsub_bounds(self._h, centers.data_ptr(), float(eps), int(batch),
+                                        ctypes.addressof(steps) if steps is not None else None,
+                                        lb_out.data_ptr(), ub_out.data_ptr(), st.cuda_stream), "cert_backsub_bounds")
+        return lb_out, ub_out
+
+    def deeppoly_p_bounds(self, centers, eps: float, p: int, **kw):
+        return self.backsub_bounds(centers, eps, [int(p)] * self.n_layers, **kw)
+
+    def ibp_bounds(self, centers, eps: float, **kw):
+        return self.backsub_bounds(centers, eps, [0] * self.n_layers, **kw)
+
+    def crown_ibp_bounds(self, centers, eps: float, **kw):
+        return self.backsub_bounds(centers, eps, [0] * (self.n_layers - 1) + [-1], **kw)
 
     # -- host numpy arrays (copies inside the library) --
     def deeppoly_bounds_host(self, centers: np.ndarray, eps: float, lb: Optional[np.ndarray] = None,
@@ -227,6 +260,7 @@ def first_layer_bounds_noalloc(weight, bias, centers, eps, clip_lo, clip_hi, lb_
 # C-ABI names, as plain functions
 cert_net_create = _lib.cert_net_create
 cert_deeppoly_bounds = _lib.cert_deeppoly_bounds
+cert_backsub_bounds = _lib.cert_backsub_bounds
 cert_deeppoly_bounds_host = _lib.cert_deeppoly_bounds_host
 cert_net_destroy = _lib.cert_net_destroy
 lib = _lib

@@ -324,6 +324,10 @@ cert_status_t cert_net_create(const cert_layer_desc_t *layers, int n_layers, int
             if (!dev_alloc_zero(net, &L.lamL, n) || !dev_alloc_zero(net, &L.lamU, n) ||
                 !dev_alloc_zero(net, &L.nuU, n)) { fail = CERT_ERR_OOM; break; }
         }
+        if (k + 1 < n_layers) {
+            size_t n = (size_t)max_batch * L.ld_out;
+            if (!dev_alloc_zero(net, &L.actL, n) || !dev_alloc_zero(net, &L.actU, n)) { fail = CERT_ERR_OOM; break; }
+        }
     }
     if (fail == CERT_OK) {
         net->n0 = net->layers[0].n_in;
@@ -373,6 +377,11 @@ cert_status_t cert_net_create(const cert_layer_desc_t *layers, int n_layers, int
 
 cert_status_t cert_deeppoly_bounds(cert_net_t *net, const float *centers, float eps, int batch, float *lb_out,
                                    float *ub_out, void *stream) {
+    return cert_backsub_bounds(net, centers, eps, batch, nullptr, lb_out, ub_out, stream);
+}
+
+cert_status_t cert_backsub_bounds(cert_net_t *net, const float *centers, float eps, int batch,
+                                  const int *backsteps, float *lb_out, float *ub_out, void *stream) {
     if (!net || !centers || !lb_out || !ub_out) return CERT_ERR_INVALID_ARG;
     if (batch < 1 || !(eps >= 0.0f) || std::isinf(eps)) return CERT_ERR_INVALID_ARG;
     if (batch > net->max_batch) return CERT_ERR_BATCH_TOO_LARGE;
@@ -386,7 +395,7 @@ cert_status_t cert_deeppoly_bounds(cert_net_t *net, const float *centers, float 
     rec.mark(CERT_CLASS_INPUT);
     cert::launch_first_layer_bounds(net->layers[0], net->l0, net->u0, net->ld0, batch, lb_out, ub_out, n_total, st);
     rec.mark(CERT_CLASS_INPUT);
-    if (net->layers[0].relu_after) {
+    if (net->layers[0].relu_after || K > 1) {
         cert::launch_relax(net->layers[0], lb_out, ub_out, n_total, batch, net->codes, net->n_relu, nullptr, 0, 0,
                            st);
         rec.mark(CERT_CLASS_RELAX);
@@ -394,6 +403,23 @@ cert_status_t cert_deeppoly_bounds(cert_net_t *net, const float *centers, float 
     for (int k = 1; k < K; ++k) {
         const LayerDev &Lk = net->layers[k];
         const long long rows = 2LL * batch * Lk.n_out;
+        // The traversal of layer k's expressions goes through layers k-1 .. j_end and is then simplified
+        // against the concrete bounds of what it has reached: the box (j_end = 0), or the outputs of
+        // layer j_end-1.  With no step at all the bounds are the interval step of W_k.
+        const int steps = (backsteps && backsteps[k] >= 0) ? std::min(backsteps[k], k) : k;
+        const int j_end = k - steps;
+        if (steps == 0) {
+            const LayerDev &Lb = net->layers[k - 1];
+            cert::launch_first_layer_bounds(Lk, Lb.actL, Lb.actU, Lb.ld_out, batch, lb_out, ub_out, n_total, st);
+            rec.mark(CERT_CLASS_CONCRETIZE);
+            if (Lk.relu_after || k + 1 < K) {
+                cert::launch_relax(Lk, lb_out, ub_out, n_total, batch, net->codes, net->n_relu, nullptr, 0, 0, st);
+                rec.mark(CERT_CLASS_RELAX);
+            }
+            continue;
+        }
+        const float *box_l = j_end == 0 ? net->l0 : net->layers[j_end - 1].actL;
+        const float *box_u = j_end == 0 ? net->u0 : net->layers[j_end - 1].actU;
         int cur = 0;      // coefficient buffer that holds the current expression
         int dcur = 0;     // constant buffer, and how many of its slots are live
         int dslots = 1;
@@ -406,10 +432,10 @@ cert_status_t cert_deeppoly_bounds(cert_net_t *net, const float *centers, float 
         cert::launch_init_expr(Lk, net->layers[k - 1], batch, net->buf[cur],
                                on_tc(k - 1) ? net->buf_lo[cur] : nullptr, net->dbuf[dcur], st);
         rec.mark(CERT_CLASS_RELU_STEP);
-        for (int j = k - 1; j >= 0; --j) {
+        for (int j = k - 1; j >= j_end; --j) {
             const LayerDev &Lj = net->layers[j];
             float *Q = net->buf[cur], *P = net->buf[cur ^ 1];
-            float *P_lo = (j > 0 && on_tc(j - 1)) ? net->buf_lo[cur ^ 1] : nullptr;
+            float *P_lo = (j > j_end && on_tc(j - 1)) ? net->buf_lo[cur ^ 1] : nullptr;
             if (on_tc(j)) {
                 const TcLayer &T = net->tc[j];
                 cert::TcArgs a;
@@ -423,7 +449,7 @@ cert_status_t cert_deeppoly_bounds(cert_net_t *net, const float *centers, float 
                 a.slot_stride = net->slot_stride;
                 a.status = net->status_dev;
                 const int groups = std::min(a.total_tiles, net->sm_count / ctas);
-                if (j > 0) {
+                if (j > j_end) {
                     const LayerDev &Lb = net->layers[j - 1];
                     a.has_relu = Lb.relu_after;
                     a.split_out = P_lo != nullptr;
@@ -431,7 +457,7 @@ cert_status_t cert_deeppoly_bounds(cert_net_t *net, const float *centers, float 
                     cert::launch_gemm_tc(cert::TC_EPI_RELU, ctas, groups, T.a_hi[cur], T.a_lo[cur], T.b_hi, T.b_lo,
                                          T.o_hi[cur ^ 1], T.o_lo[cur ^ 1], a, T.plan.smem_bytes, st);
                 } else {
-                    a.l0 = net->l0; a.u0 = net->u0;
+                    a.l0 = box_l; a.u0 = box_u;
                     cert::launch_gemm_tc(cert::TC_EPI_CONCRETIZE, ctas, groups, T.a_hi[cur], T.a_lo[cur], T.b_hi,
                                          T.b_lo, T.a_hi[cur], T.a_lo[cur], a, T.plan.smem_bytes, st);
                     bounds_in_slots = true;
@@ -450,7 +476,7 @@ cert_status_t cert_deeppoly_bounds(cert_net_t *net, const float *centers, float 
                 ep.n_k = Lk.n_out;
                 ep.d_in = net->dbuf[dcur]; ep.n_slots_in = dslots; ep.slot_stride = net->slot_stride;
                 ep.d_out = net->dbuf[dcur];
-                if (j > 0) {
+                if (j > j_end) {
                     const LayerDev &Lb = net->layers[j - 1];
                     ep.mode = cert::CONVT_EPI_RELU;
                     ep.has_relu = Lb.relu_after;
@@ -458,7 +484,7 @@ cert_status_t cert_deeppoly_bounds(cert_net_t *net, const float *centers, float 
                     ep.P = P; ep.P_lo = P_lo;
                 } else {
                     ep.mode = cert::CONVT_EPI_CONCRETIZE;
-                    ep.l0 = net->l0; ep.u0 = net->u0;
+                    ep.l0 = box_l; ep.u0 = box_u;
                     ep.lb_out = lb_out; ep.ub_out = ub_out; ep.n_total = n_total; ep.out_off = Lk.out_off;
                 }
                 cert::launch_convt_ffma(Lj, Q, rows, net->sm_count, ep, st);
@@ -471,18 +497,18 @@ cert_status_t cert_deeppoly_bounds(cert_net_t *net, const float *centers, float 
             rec.mark(CERT_CLASS_AFFINE);
             paths |= 1;
             cur ^= 1;
-            if (j > 0) {
+            if (j > j_end) {
                 cert::launch_relu_step(net->layers[j - 1], batch, Lk.n_out, P, P_lo, net->dbuf[dcur], dslots,
                                        net->slot_stride, st);
                 dslots = 1;
                 rec.mark(CERT_CLASS_RELU_STEP);
             } else {
-                cert::launch_concretize(P, net->dbuf[dcur], dslots, net->slot_stride, net->l0, net->u0, net->n0,
-                                        net->ld0, batch, Lk.n_out, lb_out, ub_out, n_total, Lk.out_off, st);
+                cert::launch_concretize(P, net->dbuf[dcur], dslots, net->slot_stride, box_l, box_u, Lj.n_in,
+                                        Lj.ld_in, batch, Lk.n_out, lb_out, ub_out, n_total, Lk.out_off, st);
                 rec.mark(CERT_CLASS_CONCRETIZE);
             }
         }
-        if (Lk.relu_after || bounds_in_slots) {
+        if (Lk.relu_after || bounds_in_slots || k + 1 < K) {
             cert::launch_relax(Lk, lb_out, ub_out, n_total, batch, net->codes, net->n_relu,
                                bounds_in_slots ? net->dbuf[dcur] : nullptr, dslots, net->slot_stride, st);
             rec.mark(CERT_CLASS_RELAX);

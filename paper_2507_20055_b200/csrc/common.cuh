@@ -29,6 +29,8 @@ struct LayerDev {
     int relu_off;            // offset in the branch-code rows (valid if relu_after)
     // relaxation of the ReLU on top (valid if relu_after): [max_batch][ld_out]
     float *lamL, *lamU, *nuU;
+    // concrete bounds of this layer's outputs (after its ReLU, if any): [max_batch][ld_out]; null for the last layer
+    float *actL, *actU;
 };
 
 // Conv geometry handed to kernels by value.
@@ -46,8 +48,9 @@ inline ConvGeom geom_of(const LayerDev &L) {
 void launch_box(const float *centers, float eps, float lo, float hi, int batch, int n0, int ld0,
                 float *l0, float *u0, cudaStream_t st);
 
-// Bounds of the first affine layer: the expression is already over the input
-// (empty traversal), so they are simplify_lower/upper of the layer's rows.
+// Bounds of an affine layer without traversal: simplify_lower/upper of the layer's rows against
+// the concrete bounds l0, u0 [batch][ld0] of its inputs (the box for the first layer, where the
+// expression is already over the input; the bounds of the layer below for an interval step).
 void launch_first_layer_bounds(const LayerDev &L, const float *l0, const float *u0, int ld0, int batch,
                                float *lb_out, float *ub_out, int n_total, cudaStream_t st);
 

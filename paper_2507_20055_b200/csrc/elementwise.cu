@@ -104,16 +104,20 @@ __device__ __forceinline__ float slot_sum(const float *__restrict__ d, int n_slo
 // Relu transformer.  One thread per (box, padded neuron).  With `slots` the
 // bounds are first assembled from the per-column-tile sums the concretising
 // contraction left (rows ordered (box, side, neuron)) and written to lb_out / ub_out.
+// actL / actU (optional) receive the concrete bounds of the layer's outputs, relu(l) and
+// relu(u) under a ReLU (Relu transformer, first two components), else l and u: what a
+// traversal that stops on this layer is simplified against.
 __global__ void relax_kernel(float *__restrict__ lb_out, float *__restrict__ ub_out, int n_total,
                              int out_off, int n, int ld, int batch, float *__restrict__ lamL,
                              float *__restrict__ lamU, float *__restrict__ nuU,
+                             float *__restrict__ actL, float *__restrict__ actU,
                              unsigned char *__restrict__ codes, int n_relu, int relu_off,
                              const float *__restrict__ slots, int n_slots, long long slot_stride,
                              int do_relax) {
     long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (idx >= (long long)batch * ld) return;
     int b = (int)(idx / ld), t = (int)(idx % ld);
-    float ll = 0.0f, lu = 0.0f, nu = 0.0f;
+    float ll = 0.0f, lu = 0.0f, nu = 0.0f, al = 0.0f, au = 0.0f;
     if (t < n) {
         float l, u;
         if (slots) {
@@ -125,21 +129,30 @@ __global__ void relax_kernel(float *__restrict__ lb_out, float *__restrict__ ub_
             l = lb_out[(size_t)b * n_total + out_off + t];
             u = ub_out[(size_t)b * n_total + out_off + t];
         }
-        if (!do_relax) return;
-        bool pick_one = (__fadd_rn(l, u) >= 0.0f);   // relu_n
-        ll = pick_one ? 1.0f : 0.0f;
-        unsigned char code;
-        if (l >= 0.0f) {                              // compute_upper, first test
-            lu = 1.0f; code = 1;
-        } else if (u <= 0.0f) {                       // second test
-            lu = 0.0f; code = 0;
-        } else {
-            float den = __fsub_rn(u, l);
-            lu = __fdiv_rn(u, den);
-            nu = -__fdiv_rn(__fmul_rn(u, l), den);
-            code = (unsigned char)(2 + (pick_one ? 1 : 0));
+        al = l;
+        au = u;
+        if (do_relax) {
+            al = l >= 0.0f ? l : 0.0f;
+            au = u >= 0.0f ? u : 0.0f;
+            bool pick_one = (__fadd_rn(l, u) >= 0.0f);   // relu_n
+            ll = pick_one ? 1.0f : 0.0f;
+            unsigned char code;
+            if (l >= 0.0f) {                              // compute_upper, first test
+                lu = 1.0f; code = 1;
+            } else if (u <= 0.0f) {                       // second test
+                lu = 0.0f; code = 0;
+            } else {
+                float den = __fsub_rn(u, l);
+                lu = __fdiv_rn(u, den);
+                nu = -__fdiv_rn(__fmul_rn(u, l), den);
+                code = (unsigned char)(2 + (pick_one ? 1 : 0));
+            }
+            codes[(size_t)b * n_relu + relu_off + t] = code;
         }
-        codes[(size_t)b * n_relu + relu_off + t] = code;
+    }
+    if (actL) {
+        actL[idx] = al;
+        actU[idx] = au;
     }
     if (!do_relax) return;
     lamL[idx] = ll;
@@ -281,9 +294,9 @@ void launch_relax(const LayerDev &L, float *lb_out, float *ub_out, int n_total, 
                   cudaStream_t st) {
     long long n = (long long)batch * L.ld_out;
     relax_kernel<<<(unsigned)ceil_div_ll(n, 256), 256, 0, st>>>(lb_out, ub_out, n_total, L.out_off, L.n_out,
-                                                               L.ld_out, batch, L.lamL, L.lamU, L.nuU, codes,
-                                                               n_relu, L.relu_off, slots, n_slots, slot_stride,
-                                                               L.relu_after);
+                                                               L.ld_out, batch, L.lamL, L.lamU, L.nuU, L.actL,
+                                                               L.actU, codes, n_relu, L.relu_off, slots, n_slots,
+                                                               slot_stride, L.relu_after);
 }
 
 void launch_init_expr(const LayerDev &Lk, const LayerDev &Lb, int batch, float *Q, float *Q_lo, float *d,

@@ -6,7 +6,7 @@ TOL = 1e-4            # |gpu - oracle| <= TOL * (1 + |oracle|)
 MARGIN_MIN = 1e-5     # boxes with a sign test closer to zero than this are ill-conditioned
 
 
-def run_gpu(w, contraction=None, max_batch=None, host_api=False):
+def run_gpu(w, contraction=None, max_batch=None, host_api=False, backsteps=None):
     import torch
     from paper_2507_20055_b200 import binding
     net = binding.CertNet(w.layers, max_batch or w.batch, w.clip_lo, w.clip_hi)
@@ -17,7 +17,10 @@ def run_gpu(w, contraction=None, max_batch=None, host_api=False):
             lb, ub = net.deeppoly_bounds_host(w.centers, w.eps)
         else:
             centers = torch.from_numpy(np.ascontiguousarray(w.centers)).cuda()
-            lb_t, ub_t = net.deeppoly_bounds(centers, w.eps)
+            if backsteps is None:
+                lb_t, ub_t = net.deeppoly_bounds(centers, w.eps)
+            else:
+                lb_t, ub_t = net.backsub_bounds(centers, w.eps, backsteps)
             torch.cuda.synchronize()
             lb, ub = lb_t.cpu().numpy(), ub_t.cpu().numpy()
         codes = net.branch_codes(w.batch).cpu().numpy()

@@ -138,3 +138,47 @@ def test_error_codes_on_device():
         assert L.cert_deeppoly_bounds(net._h, c.data_ptr(), 0.1, 0, out.data_ptr(), out.data_ptr(), None) == 1
     finally:
         net.destroy()
+
+
+# ---- bounded traversals: DeepPoly_p (Section 6.2), IBP and CROWN-IBP listings (Appendix C) ----
+
+VARIANT_NETS = {
+    "fc_ragged": lambda: wl.small_fc([37, 50, 33, 70, 40, 10], batch=5, eps=0.03, seed=81),
+    "fc_wide": lambda: wl.small_fc([64, 300, 130, 257, 3], batch=6, eps=0.02, seed=82),
+    "conv": lambda: wl.small_conv((3, 12, 12), [(8, 4, 2, 1), (12, 4, 2, 1)], [30, 5], batch=4, eps=0.01, seed=83),
+    "fc6x100": lambda: wl.make_config(1, batch=8),
+}
+
+
+def _variant_steps(K):
+    return {"ibp": [0] * K, "p1": [1] * K, "p2": [2] * K, "crown_ibp": [0] * (K - 1) + [-1],
+            "mixed": [(-1 if k % 2 else 1) for k in range(K)], "full_as_counts": list(range(K))}
+
+
+@pytest.mark.parametrize("mode", ["ffma", "tc"])
+@pytest.mark.parametrize("name", sorted(VARIANT_NETS))
+def test_bounded_traversals(name, mode):
+    w = VARIANT_NETS[name]()
+    for vname, steps in _variant_steps(len(w.layers)).items():
+        ref = orc.deeppoly(w.layers, w.centers, w.eps, w.clip_lo, w.clip_hi, backsteps_per_layer=steps)
+        g = run_gpu(w, contraction=MODES[mode], backsteps=steps)
+        compare(g, ref, label=f"{name}/{vname}/{mode}")
+
+
+def test_bounded_traversal_wrappers_and_null_array():
+    import torch
+    from paper_2507_20055_b200 import binding
+    w = wl.small_fc([20, 32, 32, 32, 6], batch=3, eps=0.05, seed=84)
+    net = binding.CertNet(w.layers, w.batch)
+    try:
+        c = torch.from_numpy(w.centers).cuda()
+        runs = {"ibp": (net.ibp_bounds(c, w.eps), orc.ibp(w.layers, w.centers, w.eps)),
+                "crown_ibp": (net.crown_ibp_bounds(c, w.eps), orc.crown_ibp(w.layers, w.centers, w.eps)),
+                "p1": (net.deeppoly_p_bounds(c, w.eps, 1), orc.deeppoly(w.layers, w.centers, w.eps, max_backsteps=1)),
+                "null": (net.backsub_bounds(c, w.eps, None), orc.deeppoly(w.layers, w.centers, w.eps))}
+        for name, ((lb, ub), ref) in runs.items():
+            torch.cuda.synchronize()
+            g = {"lb": lb.cpu().numpy(), "ub": ub.cpu().numpy(), "codes": ref["codes"], "status": net.last_status()}
+            compare(g, ref, label=name)
+    finally:
+        net.destroy()
