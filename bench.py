@@ -94,26 +94,41 @@ class ClockSampler:
                 "sm_max_mhz": max(mx) if mx else None, "samples": len(sm), "reasons": sorted(reasons)}
 
 
-def oracle_sample(w, n_boxes, threads=None):
+def oracle_sample(w, n_boxes, threads=None, backsteps=None):
     """Times the oracle, as it stands, on the first n_boxes boxes of the workload."""
     from oracle import deeppoly_oracle as orc
     orc.build()
     cores = threads or orc.max_threads()
     c = w.centers[:n_boxes]
     t0 = time.perf_counter()
-    orc.deeppoly(w.layers, c, w.eps, w.clip_lo, w.clip_hi, n_threads=cores)
+    orc.deeppoly(w.layers, c, w.eps, w.clip_lo, w.clip_hi, n_threads=cores, backsteps_per_layer=backsteps)
     dt = time.perf_counter() - t0
     return {"value": n_boxes / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
             "sample": f"first {n_boxes} of {w.batch} boxes of {w.name}, one box per thread, {dt:.1f} s wall"}, dt
 
 
-def backstep_flops_by_class(layers, batch):
-    """Algorithmic flops of one call's back-steps: for every layer k, 2*batch*n_k rows go through every
-    earlier layer j; an FC step costs 2*n_j*n_{j-1} per row, a conv step 2*n_j*c_in*kh*kw (dense maps)."""
+def certifier_steps(name, n_layers):
+    """Traversal depth per affine layer (None = to the input everywhere) for a certifier name."""
+    if name == "deeppoly":
+        return None
+    if name == "ibp":
+        return [0] * n_layers
+    if name == "crown_ibp":
+        return [0] * (n_layers - 1) + [-1]
+    if name.startswith("deeppoly_p"):
+        return [int(name[len("deeppoly_p"):])] * n_layers
+    raise SystemExit(f"unknown certifier {name!r}")
+
+
+def backstep_flops_by_class(layers, batch, steps=None):
+    """Algorithmic flops of one call's back-steps: for every layer k, 2*batch*n_k rows go through the
+    earlier layers its traversal reaches; an FC step costs 2*n_j*n_{j-1} per row, a conv step
+    2*n_j*c_in*kh*kw (dense maps)."""
     out = {"affine": 0.0, "conv": 0.0}
     for k in range(1, len(layers)):
         rows = 2.0 * batch * layers[k].n_out
-        for j in range(k):
+        depth = k if steps is None or steps[k] < 0 else min(steps[k], k)
+        for j in range(k - depth, k):
             L = layers[j]
             if L.kind == "fc":
                 out["affine"] += rows * 2.0 * L.n_out * L.n_in
@@ -136,7 +151,7 @@ def run_reference(args, w):
         n_boxes = max(1, min(cores, 16) // 2)     # about 11 s per box per core
     times = []
     for i in range(args.warmup + args.steps):
-        base, dt = oracle_sample(w, n_boxes)
+        base, dt = oracle_sample(w, n_boxes, backsteps=args.backsteps)
         if i >= args.warmup:
             times.append(dt)
     ms = 1000.0 * sum(times) / len(times)
@@ -146,7 +161,7 @@ def run_reference(args, w):
         "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": w.name, "boxes_per_step": n_boxes, "eps": w.eps,
+        "config": {"workload": w.name, "certifier": args.certifier, "boxes_per_step": n_boxes, "eps": w.eps,
                    "note": "each step bounds a sample of the workload's boxes on the host cores"},
         "cpu_baseline": base,
         "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -162,11 +177,14 @@ def main():
     ap.add_argument("--config", type=int, default=4, help="0..4: index into the benchmark configurations")
     ap.add_argument("--batch", type=int, default=None)
     ap.add_argument("--contraction", default="auto", choices=["auto", "ffma", "tc"])
+    ap.add_argument("--certifier", default="deeppoly",
+                    help="deeppoly | ibp | crown_ibp | deeppoly_pN (N back-substitution steps per layer)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--ref-boxes", type=int, default=None)
     args = ap.parse_args()
 
     w = wl.make_config(args.config, batch=args.batch)
+    args.backsteps = certifier_steps(args.certifier, len(w.layers))
     if args.impl == "reference":
         run_reference(args, w)
         return
@@ -213,7 +231,7 @@ def main():
         torch.cuda.synchronize()
 
     def step_device():
-        net.deeppoly_bounds(centers, w.eps, lb, ub, stream=stream)
+        net.backsub_bounds(centers, w.eps, args.backsteps, lb, ub, stream=stream)
 
     # ---- device-resident timing: K steps, each bracketed by events on the launching stream,
     #      L2 flushed between steps outside the bracket ----
@@ -260,12 +278,12 @@ def main():
     ub_pin = torch.empty((B, net.n_total), dtype=torch.float32).pin_memory()
     c_np, lb_np, ub_np = centers_pin.numpy(), lb_pin.numpy(), ub_pin.numpy()
     for _ in range(2):
-        net.deeppoly_bounds_host(c_np, w.eps, lb_np, ub_np, stream.cuda_stream)
+        net.deeppoly_bounds_host(c_np, w.eps, lb_np, ub_np, stream.cuda_stream, args.backsteps)
     barrier()
     e2e_steps = max(3, min(args.steps, 10))
     t0 = time.perf_counter()
     for _ in range(e2e_steps):
-        net.deeppoly_bounds_host(c_np, w.eps, lb_np, ub_np, stream.cuda_stream)   # returns after the D2H copy
+        net.deeppoly_bounds_host(c_np, w.eps, lb_np, ub_np, stream.cuda_stream, args.backsteps)   # returns after the D2H copy
     torch.cuda.synchronize()
     e2e_s = time.perf_counter() - t0
 
@@ -280,8 +298,11 @@ def main():
     if rank == 0:
         peaks = load_peaks()
         flops_call = net.backstep_flops(B)
-        fl = backstep_flops_by_class(w.layers, B)
-        assert abs(fl["affine"] + fl["conv"] - flops_call) <= 1e-6 * flops_call
+        fl = backstep_flops_by_class(w.layers, B, args.backsteps)
+        if args.backsteps is None:
+            assert abs(fl["affine"] + fl["conv"] - flops_call) <= 1e-6 * flops_call
+        else:
+            flops_call = fl["affine"] + fl["conv"]
         # the dominant kernel class: FC back-steps (tensor cores unless --contraction ffma) or conv back-steps (FMA units)
         dom = "affine" if cls_ms.get("affine", 0.0) >= cls_ms.get("conv", 0.0) else "conv"
         dom_ms, dom_n = cls_ms.get(dom, 0.0), cls_n.get(dom, 0)
@@ -312,7 +333,7 @@ def main():
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": total_ms_max / args.steps, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": {"workload": w.name, "boxes_per_gpu": B, "eps": w.eps,
+            "config": {"workload": w.name, "certifier": args.certifier, "boxes_per_gpu": B, "eps": w.eps,
                        "net": "->".join(str(x) for x in [w.layers[0].n_in] + [l.n_out for l in w.layers]),
                        "contraction": args.contraction, "parallelism": f"replicas over boxes x{world}",
                        "l2": "256 MiB flush write between timed steps; per-step coefficient traffic exceeds L2"},
@@ -325,7 +346,7 @@ def main():
             from oracle import deeppoly_oracle as orc
             orc.build()
             n_boxes = min(n_boxes, B) if args.config != 4 else min(B, orc.max_threads(), 16)
-            out["cpu_baseline"], _ = oracle_sample(w, n_boxes)
+            out["cpu_baseline"], _ = oracle_sample(w, n_boxes, backsteps=args.backsteps)
         print(json.dumps(out))
     net.destroy()
     if world > 1:

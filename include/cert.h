@@ -110,6 +110,10 @@ cert_status_t cert_backsub_bounds(cert_net_t *net, const float *centers, float e
 cert_status_t cert_deeppoly_bounds_host(cert_net_t *net, const float *centers_host, float eps,
                                         int batch, float *lb_host, float *ub_host, void *stream);
 
+/* cert_backsub_bounds with HOST buffers, in the same way. */
+cert_status_t cert_backsub_bounds_host(cert_net_t *net, const float *centers_host, float eps, int batch,
+                                       const int *backsteps, float *lb_host, float *ub_host, void *stream);
+
 /* Frees the device and host memory of the net.  Synchronises the device. */
 cert_status_t cert_net_destroy(cert_net_t *net);
 

@@ -27,6 +27,7 @@ CONTRACTION_AUTO, CONTRACTION_FFMA, CONTRACTION_TC3XTF32 = 0, 1, 2
 
 EXPORTS = [
     "cert_net_create", "cert_deeppoly_bounds", "cert_backsub_bounds", "cert_deeppoly_bounds_host",
+    "cert_backsub_bounds_host",
     "cert_net_destroy",
     "cert_net_num_neurons", "cert_net_num_relu_neurons", "cert_net_branch_codes",
     "cert_net_last_status", "cert_net_set_contraction", "cert_net_last_launch_count",
@@ -50,6 +51,8 @@ _lib.cert_deeppoly_bounds.argtypes = [_vp, _vp, _f, _i, _vp, _vp, _vp]
 _lib.cert_deeppoly_bounds.restype = _i
 _lib.cert_backsub_bounds.argtypes = [_vp, _vp, _f, _i, _vp, _vp, _vp, _vp]
 _lib.cert_backsub_bounds.restype = _i
+_lib.cert_backsub_bounds_host.argtypes = [_vp, _vp, _f, _i, _vp, _vp, _vp, _vp]
+_lib.cert_backsub_bounds_host.restype = _i
 _lib.cert_deeppoly_bounds_host.argtypes = [_vp, _vp, _f, _i, _vp, _vp, _vp]
 _lib.cert_deeppoly_bounds_host.restype = _i
 _lib.cert_net_destroy.argtypes = [_vp]
@@ -182,16 +185,21 @@ class CertNet:
 
     # -- host numpy arrays (copies inside the library) --
     def deeppoly_bounds_host(self, centers: np.ndarray, eps: float, lb: Optional[np.ndarray] = None,
-                             ub: Optional[np.ndarray] = None, stream_ptr: int = 0):
+                             ub: Optional[np.ndarray] = None, stream_ptr: int = 0, backsteps=None):
         centers = np.ascontiguousarray(centers, dtype=np.float32)
         batch = centers.shape[0]
         if lb is None:
             lb = np.empty((batch, self.n_total), dtype=np.float32)
         if ub is None:
             ub = np.empty((batch, self.n_total), dtype=np.float32)
-        _check(_lib.cert_deeppoly_bounds_host(self._h, centers.ctypes.data, float(eps), batch,
-                                              lb.ctypes.data, ub.ctypes.data, stream_ptr),
-               "cert_deeppoly_bounds_host")
+        steps = None
+        if backsteps is not None:
+            assert len(backsteps) == self.n_layers
+            steps = (ctypes.c_int * self.n_layers)(*[int(x) for x in backsteps])
+        _check(_lib.cert_backsub_bounds_host(self._h, centers.ctypes.data, float(eps), batch,
+                                             ctypes.addressof(steps) if steps is not None else None,
+                                             lb.ctypes.data, ub.ctypes.data, stream_ptr),
+               "cert_backsub_bounds_host")
         return lb, ub
 
     def set_profiling(self, on: bool):

@@ -527,6 +527,11 @@ cert_status_t cert_backsub_bounds(cert_net_t *net, const float *centers, float e
 
 cert_status_t cert_deeppoly_bounds_host(cert_net_t *net, const float *centers_host, float eps, int batch,
                                         float *lb_host, float *ub_host, void *stream) {
+    return cert_backsub_bounds_host(net, centers_host, eps, batch, nullptr, lb_host, ub_host, stream);
+}
+
+cert_status_t cert_backsub_bounds_host(cert_net_t *net, const float *centers_host, float eps, int batch,
+                                       const int *backsteps, float *lb_host, float *ub_host, void *stream) {
     if (!net || !centers_host || !lb_host || !ub_host) return CERT_ERR_INVALID_ARG;
     if (batch < 1) return CERT_ERR_INVALID_ARG;
     if (batch > net->max_batch) return CERT_ERR_BATCH_TOO_LARGE;
@@ -537,7 +542,7 @@ cert_status_t cert_deeppoly_bounds_host(cert_net_t *net, const float *centers_ho
         cudaGetLastError();
         return CERT_ERR_CUDA;
     }
-    cert_status_t s = cert_deeppoly_bounds(net, net->centers_dev, eps, batch, net->lb_dev, net->ub_dev, stream);
+    cert_status_t s = cert_backsub_bounds(net, net->centers_dev, eps, batch, backsteps, net->lb_dev, net->ub_dev, stream);
     if (s != CERT_OK) return s;
     if (cudaMemcpyAsync(lb_host, net->lb_dev, out_bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
         cudaMemcpyAsync(ub_host, net->ub_dev, out_bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
