@@ -102,6 +102,67 @@ __device__ __forceinline__ void cp_async4(float *smem_dst, const float *gsrc, bo
     asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(dst), "l"(gsrc), "r"(src_bytes) : "memory");
 }
 
+// acc[i][c] += sum over output channels and the class's taps of Q * W for PXT pixels x CT channels.
+// q[i]: this lane's pixels in the staged maps (tap (0,0), channel 0); w: the class's tap (0,0) of
+// output channel 0 at input channel c0.  TY, TX: taps per axis when known at compile time (the loops
+// then unroll and the tap offsets live in registers), 0 = take n_my, n_mx at run time.
+template <int CT, int PXT, int TY, int TX>
+__device__ __forceinline__ void accumulate_taps(float (&acc)[PXT][CT], const float *const (&q)[PXT],
+                                                const float *w, int c_out, int plane, int w_co_stride,
+                                                int w_my_stride, int w_mx_stride, int WP, int n_my, int n_mx) {
+    constexpr int CTL = (CT + 3) / 4 * 4;       // weights are read in 16-byte pieces
+    const int ty = TY > 0 ? TY : n_my, tx = TX > 0 ? TX : n_mx;
+#pragma unroll 2
+    for (int co = 0; co < c_out; ++co) {
+        const float *wc = w + co * w_co_stride;
+        const int qc = co * plane;
+#pragma unroll
+        for (int my = 0; my < ty; ++my) {
+#pragma unroll
+            for (int mx = 0; mx < tx; ++mx) {
+                float wv[CTL];
+#pragma unroll
+                for (int c4 = 0; c4 < CTL; c4 += 4) {
+                    const float4 w4 = *reinterpret_cast<const float4 *>(wc + my * w_my_stride + mx * w_mx_stride + c4);
+                    wv[c4] = w4.x; wv[c4 + 1] = w4.y; wv[c4 + 2] = w4.z; wv[c4 + 3] = w4.w;
+                }
+                const int shift = qc - my * WP - mx;
+#pragma unroll
+                for (int i = 0; i < PXT; ++i) {
+                    const float qv = q[i][shift];
+#pragma unroll
+                    for (int c = 0; c < CT; ++c) acc[i][c] = fmaf(qv, wv[c], acc[i][c]);
+                }
+            }
+        }
+    }
+}
+
+// The same for a channel chunk of which only `left` (< round_up(CT, 4)) channels exist in the staged rows.
+template <int CT, int PXT>
+__device__ __forceinline__ void accumulate_tail(float (&acc)[PXT][CT], const float *const (&q)[PXT],
+                                                const float *w, int c_out, int plane, int w_co_stride,
+                                                int w_my_stride, int w_mx_stride, int WP, int n_my, int n_mx,
+                                                int left) {
+    for (int co = 0; co < c_out; ++co) {
+        for (int my = 0; my < n_my; ++my) {
+            for (int mx = 0; mx < n_mx; ++mx) {
+                const float *wc = w + co * w_co_stride + my * w_my_stride + mx * w_mx_stride;
+                float wv[CT];
+#pragma unroll
+                for (int c = 0; c < CT; ++c) wv[c] = c < left ? wc[c] : 0.0f;
+                const int shift = co * plane - my * WP - mx;
+#pragma unroll
+                for (int i = 0; i < PXT; ++i) {
+                    const float qv = q[i][shift];
+#pragma unroll
+                    for (int c = 0; c < CT; ++c) acc[i][c] = fmaf(qv, wv[c], acc[i][c]);
+                }
+            }
+        }
+    }
+}
+
 // Q [rows][ld_out] maps (c_out, h_out, w_out); the result maps (c_in, h_in, w_in) with pitch ld_in.
 // Wct: weights laid out [c_out][kh][kw][c_in].
 template <int CT, int PXT, int EPI>
@@ -198,29 +259,27 @@ convt_kernel(const float *__restrict__ Q, int ld_out, int ld_in, const float *__
                     for (int i = 0; i < PXT; ++i)
 #pragma unroll
                         for (int c = 0; c < CT; ++c) acc[i][c] = 0.0f;
-#pragma unroll 2
-                    for (int co = 0; co < g.c_out; ++co) {
-                        for (int my = 0; my < n_my; ++my) {
-                            const int ky = cy + s * my;
-                            for (int mx = 0; mx < n_mx; ++mx) {
-                                const int kx = cx + s * mx;
-                                const float *wp = Ws + ((co * g.kh + ky) * g.kw + kx) * pl.cpad + c0;
-                                float w[CT];
+                    {
+                        const float *qp[PXT];
 #pragma unroll
-                                for (int c4 = 0; c4 < CT; c4 += 4) {
-                                    // cpad is a multiple of 4; channels past it read as zero
-                                    float4 w4 = (c0 + c4 < pl.cpad) ? *reinterpret_cast<const float4 *>(wp + c4)
-                                                                     : make_float4(0.f, 0.f, 0.f, 0.f);
-                                    w[c4] = w4.x; w[c4 + 1] = w4.y; w[c4 + 2] = w4.z; w[c4 + 3] = w4.w;
-                                }
-                                const int shift = co * plane - my * pl.WP - mx;
-#pragma unroll
-                                for (int i = 0; i < PXT; ++i) {
-                                    const float q = Qs[q_off[i] + shift];
-#pragma unroll
-                                    for (int c = 0; c < CT; ++c) acc[i][c] = fmaf(q, w[c], acc[i][c]);
-                                }
-                            }
+                        for (int i = 0; i < PXT; ++i) qp[i] = Qs + q_off[i];
+                        // weights of the class's first tap (ky, kx) = (cy, cx); further taps are s apart.
+                        // A channel chunk that starts past the padded channel count cannot occur (c0 < c_in <= cpad);
+                        // a chunk wider than what is left reads the zero padding up to a multiple of 4 only.
+                        const float *w0 = Ws + (cy * g.kw + cx) * pl.cpad + c0;
+                        const int w_co = g.kh * g.kw * pl.cpad, w_my = s * g.kw * pl.cpad, w_mx = s * pl.cpad;
+                        const bool whole = c0 + ((CT + 3) / 4 * 4) <= pl.cpad;   // the 16-byte reads stay inside the channel row
+                        if (!whole) {
+                            accumulate_tail<CT, PXT>(acc, qp, w0, g.c_out, plane, w_co, w_my, w_mx, pl.WP, n_my, n_mx,
+                                                     pl.cpad - c0);
+                        } else if (n_my == 2 && n_mx == 2) {
+                            accumulate_taps<CT, PXT, 2, 2>(acc, qp, w0, g.c_out, plane, w_co, w_my, w_mx, pl.WP, 2, 2);
+                        } else if (n_my == 1 && n_mx == 1) {
+                            accumulate_taps<CT, PXT, 1, 1>(acc, qp, w0, g.c_out, plane, w_co, w_my, w_mx, pl.WP, 1, 1);
+                        } else if (n_my == 3 && n_mx == 3) {
+                            accumulate_taps<CT, PXT, 3, 3>(acc, qp, w0, g.c_out, plane, w_co, w_my, w_mx, pl.WP, 3, 3);
+                        } else {
+                            accumulate_taps<CT, PXT, 0, 0>(acc, qp, w0, g.c_out, plane, w_co, w_my, w_mx, pl.WP, n_my, n_mx);
                         }
                     }
                     // ---- what follows the step on the path, per element ----
@@ -325,6 +384,7 @@ bool convt_supported(const LayerDev &L) {
 }
 
 void convt_prepare() {
+    prepare_ct<3, 8>();
     prepare_ct<4, 4>();
     prepare_ct<8, 4>();
     prepare_ct<16, 2>();
@@ -333,7 +393,8 @@ void convt_prepare() {
 void launch_convt_ffma(const LayerDev &L, const float *Q, long long rows, int sms, const ConvtEpilogue &ep,
                        cudaStream_t st) {
     const ConvtPlan pl = make_plan(L);
-    if (L.c_in <= 4) launch_ct<4, 4>(L, pl, Q, rows, sms, ep, st);
+    if (L.c_in == 3) launch_ct<3, 8>(L, pl, Q, rows, sms, ep, st);
+    else if (L.c_in <= 4) launch_ct<4, 4>(L, pl, Q, rows, sms, ep, st);
     else if (L.c_in <= 8) launch_ct<8, 4>(L, pl, Q, rows, sms, ep, st);
     else launch_ct<16, 2>(L, pl, Q, rows, sms, ep, st);
 }
