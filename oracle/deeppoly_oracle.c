@@ -159,6 +159,33 @@ static void replace_through_relu(int n, int upper, const double *lamL, const dou
     }
 }
 
+/* SkipPoly (Appendix C, SkipPoly listing): the shape of a ReLU neuron t on top of affine
+ * layer Lj is expressed two layers back,
+ *   L_t = relu_n(prev)       = (l + u >= 0) ? prev[L] : 0
+ *   U_t = compute_upper(prev) = l >= 0 ? prev[U] : u <= 0 ? 0 : u/(u-l) * prev[U] - u*l/(u-l)
+ * with prev[L] = prev[U] = w_t.a + b_t over the inputs a of the affine layer, so one traversal
+ * round replaces the ReLU neurons by expressions over a directly:
+ *   coefficient c  ->  c * (slope * w_t[s]) on every a_s,  constant += c * (slope * b_t + intercept).
+ * row: scratch of n_in doubles.                                                              */
+static void replace_through_relu_skip(const oracle_layer_t *Lj, int upper, const double *lamL,
+                                      const double *lamU, const double *nuU, const double *coef,
+                                      double *next, double *row, double *d)
+{
+    int n_in = layer_n_in(Lj), n_out = layer_n_out(Lj);
+    for (int s = 0; s < n_in; ++s) next[s] = 0.0;
+    for (int t = 0; t < n_out; ++t) {
+        double c = coef[t];
+        if (c == 0.0) continue;
+        int use_L = upper ? !(c >= 0.0) : (c >= 0.0);
+        double slope = use_L ? lamL[t] : lamU[t];
+        double intercept = use_L ? 0.0 : nuU[t];
+        double b;
+        affine_row(Lj, t, row, &b);
+        for (int s = 0; s < n_in; ++s) next[s] += c * (slope * row[s]);
+        *d += c * (slope * b + intercept);
+    }
+}
+
 /* simplify_lower / simplify_upper summed over the input neurons. */
 static double concretize(int n, int upper, const double *coef, double d,
                          const double *l0, const double *u0)
@@ -208,7 +235,7 @@ static void relu_relaxation(double l, double u, int decision_fp32, double *lamL,
  * (flow(forward, priority = layer)). */
 static int one_box(const oracle_layer_t *layers, int n_layers, const float *center, float eps,
                    float clip_lo, float clip_hi, int decision_fp32, int max_backsteps_all,
-                   const int *backsteps_per_layer,
+                   const int *backsteps_per_layer, int skip_form,
                    double *lb, double *ub, unsigned char *codes, double *margins)
 {
     int n0 = layer_n_in(&layers[0]);
@@ -222,8 +249,9 @@ static int one_box(const oracle_layer_t *layers, int n_layers, const float *cent
     double *coef = malloc(sizeof(double) * n_max), *next = malloc(sizeof(double) * n_max);
     double *lamL = malloc(sizeof(double) * n_total), *lamU = malloc(sizeof(double) * n_total);
     double *nuU = malloc(sizeof(double) * n_total);
+    double *row = malloc(sizeof(double) * n_max);
     int *off = malloc(sizeof(int) * (n_layers + 1));
-    if (!l0 || !u0 || !coef || !next || !lamL || !lamU || !nuU || !off) return 1;
+    if (!l0 || !u0 || !coef || !next || !lamL || !lamU || !nuU || !off || !row) return 1;
 
     /* The box endpoints are binary32 values: fl(c -/+ eps) clipped. */
     for (int s = 0; s < n0; ++s) {
@@ -249,10 +277,15 @@ static int one_box(const oracle_layer_t *layers, int n_layers, const float *cent
                 int j = k - 1;                 /* coef is over the outputs of layer j */
                 for (; j >= 0; --j) {
                     if (max_backsteps >= 0 && steps >= max_backsteps) break;
-                    if (layers[j].relu_after)
-                        replace_through_relu(layer_n_out(&layers[j]), upper, lamL + off[j],
-                                             lamU + off[j], nuU + off[j], coef, &d);
-                    replace_through_affine(&layers[j], coef, next, &d);
+                    if (skip_form && layers[j].relu_after) {
+                        replace_through_relu_skip(&layers[j], upper, lamL + off[j], lamU + off[j],
+                                                  nuU + off[j], coef, next, row, &d);
+                    } else {
+                        if (layers[j].relu_after)
+                            replace_through_relu(layer_n_out(&layers[j]), upper, lamL + off[j],
+                                                 lamU + off[j], nuU + off[j], coef, &d);
+                        replace_through_affine(&layers[j], coef, next, &d);
+                    }
                     double *tmp = coef; coef = next; next = tmp;
                     ++steps;
                 }
@@ -288,7 +321,7 @@ static int one_box(const oracle_layer_t *layers, int n_layers, const float *cent
             code_off += n_k;
         }
     }
-    free(l0); free(u0); free(coef); free(next); free(lamL); free(lamU); free(nuU); free(off);
+    free(l0); free(u0); free(coef); free(next); free(lamL); free(lamU); free(nuU); free(off); free(row);
     return 0;
 }
 
@@ -321,12 +354,14 @@ int oracle_num_relu_neurons(const oracle_layer_t *layers, int n_layers)
  *   IBP listing:       Affine -> map(simplify_*) of prev.dot(w)+b, no traversal: 0 everywhere;
  *   CROWN-IBP listing: the same, except curr[last_layer] == 1 -> backsubs_*: 0, ..., 0, -1,
  * with the Relu transformer (relu(l), relu(u), relu_n, compute_upper) unchanged.
+ * skip_form != 0: the SkipPoly listing (ReLU shapes expressed two layers back; one traversal
+ * round per ReLU layer).
  * n_threads: boxes are independent and are the only parallel axis.
  * Returns 0, or 1 on allocation failure, 2 on a malformed network.
  */
 int oracle_backsub(const oracle_layer_t *layers, int n_layers, const float *centers, float eps,
                    int batch, float clip_lo, float clip_hi, int decision_fp32, int max_backsteps,
-                   const int *backsteps_per_layer,
+                   const int *backsteps_per_layer, int skip_form,
                    int n_threads, double *lb, double *ub, unsigned char *codes, double *margins)
 {
     if (n_layers < 1 || batch < 0) return 2;
@@ -344,7 +379,8 @@ int oracle_backsub(const oracle_layer_t *layers, int n_layers, const float *cent
 #pragma omp parallel for schedule(dynamic, 1)
     for (int b = 0; b < batch; ++b) {
         int e = one_box(layers, n_layers, centers + (size_t)b * n0, eps, clip_lo, clip_hi,
-                        decision_fp32, max_backsteps, backsteps_per_layer, lb + (size_t)b * n_total,
+                        decision_fp32, max_backsteps, backsteps_per_layer, skip_form,
+                        lb + (size_t)b * n_total,
                         ub + (size_t)b * n_total, codes ? codes + (size_t)b * n_relu : NULL,
                         margins ? margins + (size_t)b * n_relu : NULL);
         if (e) {
@@ -360,7 +396,7 @@ int oracle_deeppoly(const oracle_layer_t *layers, int n_layers, const float *cen
                     int n_threads, double *lb, double *ub, unsigned char *codes, double *margins)
 {
     return oracle_backsub(layers, n_layers, centers, eps, batch, clip_lo, clip_hi, decision_fp32,
-                          max_backsteps, NULL, n_threads, lb, ub, codes, margins);
+                          max_backsteps, NULL, 0, n_threads, lb, ub, codes, margins);
 }
 
 int oracle_max_threads(void)

@@ -77,11 +77,13 @@ def _marshal(layers):
 
 
 def deeppoly(layers, centers, eps, clip_lo=0.0, clip_hi=1.0, decision_fp32=True,
-             max_backsteps: int = -1, n_threads: Optional[int] = None, backsteps_per_layer=None):
+             max_backsteps: int = -1, n_threads: Optional[int] = None, backsteps_per_layer=None,
+             skip_form: bool = False):
     """Bounds of every affine neuron for every box.
 
     max_backsteps = p >= 0 is DeepPoly_p; backsteps_per_layer (one count per affine layer,
-    negative = traverse to the input) overrides it.
+    negative = traverse to the input) overrides it.  skip_form: the SkipPoly listing (ReLU shapes
+    expressed over the neurons two layers back).
     Returns dict(lb, ub: float64 [batch, n_total]; codes: uint8 [batch, n_relu];
     margins: float64 [batch, n_relu]).  Layers are concatenated in order.
     """
@@ -104,7 +106,7 @@ def deeppoly(layers, centers, eps, clip_lo=0.0, clip_hi=1.0, decision_fp32=True,
                             ctypes.c_float(clip_hi), ctypes.c_int(int(decision_fp32)),
                             ctypes.c_int(max_backsteps),
                             ctypes.c_void_p(steps.ctypes.data if steps is not None else None),
-                            ctypes.c_int(n_threads or 0),
+                            ctypes.c_int(int(bool(skip_form))), ctypes.c_int(n_threads or 0),
                             ctypes.c_void_p(lb.ctypes.data), ctypes.c_void_p(ub.ctypes.data),
                             ctypes.c_void_p(codes.ctypes.data), ctypes.c_void_p(margins.ctypes.data))
     if rc != 0:
@@ -116,6 +118,11 @@ def deeppoly(layers, centers, eps, clip_lo=0.0, clip_hi=1.0, decision_fp32=True,
 def ibp(layers, centers, eps, clip_lo=0.0, clip_hi=1.0, **kw):
     """IBP listing of Appendix C: no traversal at any layer."""
     return deeppoly(layers, centers, eps, clip_lo, clip_hi, backsteps_per_layer=[0] * len(layers), **kw)
+
+
+def skippoly(layers, centers, eps, clip_lo=0.0, clip_hi=1.0, **kw):
+    """SkipPoly listing of Appendix C."""
+    return deeppoly(layers, centers, eps, clip_lo, clip_hi, skip_form=True, **kw)
 
 
 def crown_ibp(layers, centers, eps, clip_lo=0.0, clip_hi=1.0, **kw):

@@ -182,3 +182,12 @@ def test_bounded_traversal_wrappers_and_null_array():
             compare(g, ref, label=name)
     finally:
         net.destroy()
+
+
+@pytest.mark.parametrize("name", ["fc_ragged", "conv"])
+def test_fused_steps_against_the_skippoly_listing(name):
+    """The GPU path takes a ReLU layer and the affine layer below it in one kernel, which is the traversal
+    of the SkipPoly listing (Appendix C: ReLU shapes expressed two layers back, one round per ReLU layer)."""
+    w = VARIANT_NETS[name]()
+    ref = orc.skippoly(w.layers, w.centers, w.eps, w.clip_lo, w.clip_hi)
+    compare(run_gpu(w), ref, label=f"{name}/skippoly")

@@ -138,3 +138,41 @@ def test_ibp_never_beats_crown_ibp_at_the_last_layer_on_a_linear_tail():
     assert (c["codes"] <= 1).all()
     assert (c["lb"][:, -3:] >= a["lb"][:, -3:] - 1e-12).all()
     assert (c["ub"][:, -3:] <= a["ub"][:, -3:] + 1e-12).all()
+
+
+# ---- SkipPoly listing (Appendix C): ReLU shapes expressed two layers back ----
+
+def test_skippoly_w1_hand_values():
+    """On the 2-2-2-1 example every slope the upper shapes multiply into the weights is a dyadic or a
+    multiple of 1/19, and the hand evaluation of the SkipPoly listing gives DeepPoly's numbers: the shape of a
+    ReLU neuron over the layer two back is its DeepPoly shape with the affine neuron's expression substituted."""
+    g, layers = _w1()
+    r = orc.skippoly(layers, np.array([g["center"]], np.float32), g["eps"], *g["clip"])
+    np.testing.assert_allclose(r["lb"][0], _fr(g["lb"]), rtol=0, atol=1e-14)
+    np.testing.assert_allclose(r["ub"][0], _fr(g["ub"]), rtol=0, atol=1e-14)
+    assert r["codes"][0].tolist() == g["codes"]
+
+
+@pytest.mark.parametrize("make", NETS)
+def test_skippoly_has_deeppoly_precision(make):
+    """Section 6.1: expressing the ReLU bounds two layers back does not change the bounds ("without
+    sacrificing precision"); only the order of the floating-point products differs."""
+    w = make()
+    a = orc.deeppoly(w.layers, w.centers, w.eps, w.clip_lo, w.clip_hi)
+    b = orc.skippoly(w.layers, w.centers, w.eps, w.clip_lo, w.clip_hi)
+    np.testing.assert_allclose(b["lb"], a["lb"], rtol=1e-11, atol=1e-11)
+    np.testing.assert_allclose(b["ub"], a["ub"], rtol=1e-11, atol=1e-11)
+    assert np.array_equal(a["codes"], b["codes"])
+
+
+def test_skippoly_soundness_and_missing_relu():
+    w = wl.small_fc([8, 16, 16, 16, 4], batch=2, eps=0.1, seed=35)
+    w.layers[1].relu_after = False            # an affine layer directly on an affine layer
+    r = orc.skippoly(w.layers, w.centers, w.eps, w.clip_lo, w.clip_hi)
+    a = orc.deeppoly(w.layers, w.centers, w.eps, w.clip_lo, w.clip_hi)
+    np.testing.assert_allclose(r["lb"], a["lb"], rtol=1e-11, atol=1e-11)
+    L0, U0 = mat.box(w.centers, w.eps, w.clip_lo, w.clip_hi)
+    for b in range(w.batch):
+        z = mat.forward_preactivations(w.layers, _samples(L0[b], U0[b], 50_000, seed=b))
+        assert (z.min(axis=0) >= r["lb"][b] - 1e-9 * (1 + np.abs(r["lb"][b]))).all()
+        assert (z.max(axis=0) <= r["ub"][b] + 1e-9 * (1 + np.abs(r["ub"][b]))).all()
