@@ -21,6 +21,11 @@
 // registers.  A lane always works for the same row of the group (lane / (32/RB)),
 // so a row's constant is summed in registers, then across the lanes of its
 // group by shuffles and across warps in a fixed order: no atomics.
+//
+// Stride 2 with at most 4 channels below (an image layer): the four classes of the pixels
+// (2uy + cy - pad, 2ux + cx - pad) read the same coefficients Q[co][uy - dy][ux - dx], so a thread
+// takes all four classes of its positions (uy, ux) at once and every coefficient read from shared
+// memory feeds 4 x CT FMAs instead of CT (convt_s2_kernel).
 #include "common.cuh"
 
 namespace cert {
@@ -41,6 +46,9 @@ struct ConvtPlan {
     int cpad;                // c_in rounded up to 4 (weights are staged as [co][ky][kx][cpad])
     int rows_per_group;      // rows staged per pass: a power of two <= 8
     size_t smem_bytes;
+    // stride-2 form: taps per axis (ceil(k/2)), extent of the position grid; n_w = staged weight count
+    int s2;                  // 1: convt_s2_kernel applies
+    int ty, tx, hu, wu, n_w;
 };
 
 struct AxisRange { int lo, hi; };
@@ -70,7 +78,24 @@ ConvtPlan make_plan(const LayerDev &L) {
     p.HP = p.halo_y + std::max(L.h_out, ry.hi + 1);
     p.WP = p.halo_x + std::max(L.w_out, rx.hi + 1);
     p.cpad = round_up(L.c_in, 4);
-    const size_t w_bytes = sizeof(float) * (size_t)L.c_out * L.kh * L.kw * p.cpad;
+    p.n_w = L.c_out * L.kh * L.kw * p.cpad;
+    // Stride-2 form: positions u in [0, hu) x [0, wu) cover every class's pixels (u = (i + pad - c) / 2);
+    // taps dy < ty, dx < tx; weights staged with the kernel padded to 2*ty x 2*tx (zeros), and a halo of
+    // at least ty-1, tx-1 so that a position whose tap does not exist reads staged zeros or staged data,
+    // never anything else.
+    p.ty = (L.kh + 1) / 2;
+    p.tx = (L.kw + 1) / 2;
+    p.s2 = (L.stride == 2 && L.c_in <= 4 && p.ty == p.tx && p.ty >= 1 && p.ty <= 3) ? 1 : 0;
+    if (p.s2) {
+        p.hu = (L.h_in - 1 + L.pad) / 2 + 1;
+        p.wu = (L.w_in - 1 + L.pad) / 2 + 1;
+        p.halo_y = std::max(p.halo_y, p.ty - 1);
+        p.halo_x = std::max(p.halo_x, p.tx - 1);
+        p.HP = p.halo_y + std::max(std::max(L.h_out, ry.hi + 1), p.hu);
+        p.WP = p.halo_x + std::max(std::max(L.w_out, rx.hi + 1), p.wu);
+        p.n_w = L.c_out * (2 * p.ty) * (2 * p.tx) * p.cpad;
+    }
+    const size_t w_bytes = sizeof(float) * (size_t)p.n_w;
     const size_t fixed = w_bytes + sizeof(float) * kWarps * kMaxRowsPerGroup;
     const int map = L.c_out * p.HP * p.WP;
     p.rows_per_group = 0;
@@ -178,7 +203,7 @@ convt_kernel(const float *__restrict__ Q, int ld_out, int ld_in, const float *__
     const int G = 32 / RB;             // lanes per row of the group
     const int plane = pl.HP * pl.WP;
     float *Ws = smem;                  // [c_out][kh][kw][cpad]
-    float *red = smem + n_w;           // [kWarps][kMaxRowsPerGroup] partial row constants
+    float *red = smem + pl.n_w;        // [kWarps][kMaxRowsPerGroup] partial row constants
     float *Qs = red + kWarps * kMaxRowsPerGroup;   // [RB][map_stride], each map [c_out][HP][WP] inside its halo
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int rl = lane / G, gl = lane % G;
@@ -354,6 +379,204 @@ convt_kernel(const float *__restrict__ Q, int ld_out, int ld_in, const float *__
     }
 }
 
+// One element v = P[r][t] of the back-step's result: ReLU back-step through the layer below and the
+// constant's share of the next affine step (result stored), or its term of the concretisation.
+template <int EPI>
+__device__ __forceinline__ void finish_element(float v, int t, long long r, int upper, size_t vec, int ld_in,
+                                               const ConvtEpilogue &ep, float &dacc) {
+    const bool nonneg = (v >= 0.0f);
+    if (EPI == CONVT_EPI_CONCRETIZE) {
+        // lower rows: c >= 0 ? c*l : c*u; upper rows: c >= 0 ? c*u : c*l
+        const float bnd = (nonneg != (upper != 0)) ? ep.l0[vec + t] : ep.u0[vec + t];
+        dacc = fmaf(v, bnd, dacc);
+    } else {
+        float qv = v;
+        if (ep.has_relu) {
+            const bool use_lower = upper ? !nonneg : nonneg;
+            if (use_lower) {
+                qv = v * ep.lamL[vec + t];
+            } else {
+                dacc = fmaf(v, ep.nuU[vec + t], dacc);
+                qv = v * ep.lamU[vec + t];
+            }
+        }
+        dacc = fmaf(qv, ep.bias_below[t], dacc);
+        const size_t o = (size_t)r * ld_in + t;
+        if (ep.P_lo) {
+            const float h = tf32_round(qv);
+            ep.P[o] = h;
+            ep.P_lo[o] = tf32_round(qv - h);
+        } else {
+            ep.P[o] = qv;
+        }
+    }
+}
+
+// Stride 2, c_in <= 4.  A thread takes PXT positions (uy, ux) of its row and, for each, the four
+// pixels (2uy + cy - pad, 2ux + cx - pad), cy, cx in {0, 1}; tap (dy, dx) of class (cy, cx) is kernel
+// element (cy + 2dy, cx + 2dx) and reads Q[co][uy - dy][ux - dx] for every class.  Weights are staged
+// as [c_out][2*T][2*T][cpad] with zeros where the kernel has no such element.
+template <int CT, int PXT, int T, int EPI>
+__global__ void __launch_bounds__(kThreads, 2)
+convt_s2_kernel(const float *__restrict__ Q, int ld_out, int ld_in, const float *__restrict__ Wct, ConvGeom g,
+                ConvtPlan pl, long long rows, ConvtEpilogue ep) {
+    extern __shared__ __align__(16) float smem[];
+    const int n_out = g.c_out * g.h_out * g.w_out;
+    const int n_in = g.c_in * g.h_in * g.w_in;
+    const int hw_in = g.h_in * g.w_in, hw_out = g.h_out * g.w_out;
+    const int RB = pl.rows_per_group;
+    const int G = 32 / RB;             // lanes per row of the group
+    const int plane = pl.HP * pl.WP;
+    float *Ws = smem;                  // [c_out][2T][2T][cpad]
+    float *red = smem + pl.n_w;        // [kWarps][kMaxRowsPerGroup] partial row constants
+    float *Qs = red + kWarps * kMaxRowsPerGroup;   // [RB][map_stride], each map [c_out][HP][WP] inside its halo
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int rl = lane / G, gl = lane % G;
+
+    for (int i = threadIdx.x; i < pl.n_w; i += kThreads) {
+        const int ci = i % pl.cpad;
+        int rest = i / pl.cpad;
+        const int kx = rest % (2 * T); rest /= 2 * T;
+        const int ky = rest % (2 * T);
+        const int co = rest / (2 * T);
+        const bool real = ci < g.c_in && ky < g.kh && kx < g.kw;
+        Ws[i] = real ? Wct[(((size_t)co * g.kh + ky) * g.kw + kx) * g.c_in + ci] : 0.0f;
+    }
+    for (int i = threadIdx.x; i < RB * pl.map_stride; i += kThreads) Qs[i] = 0.0f;   // halos stay zero
+
+    const int d_ox = kThreads % g.w_out, d_oy = (kThreads / g.w_out) % g.h_out, d_co = kThreads / hw_out;
+    const int positions = pl.hu * pl.wu;
+    const int units = (positions + G * PXT - 1) / (G * PXT);
+    const int w_co = 4 * T * T * pl.cpad, w_ky = 2 * T * pl.cpad;
+
+    for (long long r0 = (long long)blockIdx.x * RB; r0 < rows; r0 += (long long)gridDim.x * RB) {
+        __syncthreads();
+        for (int q = 0; q < RB; ++q) {
+            const bool live = r0 + q < rows;
+            const float *qrow = Q + (size_t)(live ? r0 + q : r0) * ld_out;
+            float *qs = Qs + q * pl.map_stride + pl.halo_y * pl.WP + pl.halo_x;
+            int e = threadIdx.x;
+            int co = e / hw_out, oy = (e % hw_out) / g.w_out, ox = e % g.w_out;
+            for (; e < n_out; e += kThreads) {
+                cp_async4(qs + co * plane + oy * pl.WP + ox, qrow + e, live);
+                ox += d_ox;
+                if (ox >= g.w_out) { ox -= g.w_out; ++oy; }
+                oy += d_oy;
+                if (oy >= g.h_out) { oy -= g.h_out; ++co; }
+                co += d_co;
+            }
+        }
+        asm volatile("cp.async.commit_group;" ::: "memory");
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
+        __syncthreads();
+
+        const long long r = r0 + rl;
+        const bool row_ok = r < rows;
+        const long long rr = row_ok ? r : 0;
+        const int box = (int)(rr / (2LL * ep.n_k));
+        const int upper = (int)((rr / ep.n_k) & 1);
+        const size_t vec = (size_t)box * ld_in;
+        float dacc = 0.0f;
+        for (int u = warp; u < units; u += kWarps) {
+            int q_off[PXT], uy[PXT], ux[PXT];
+            bool ok[PXT];
+#pragma unroll
+            for (int i = 0; i < PXT; ++i) {
+                const int p = u * (G * PXT) + i * G + gl;
+                ok[i] = p < positions && row_ok;
+                const int pc = p < positions ? p : 0;
+                uy[i] = pc / pl.wu;
+                ux[i] = pc % pl.wu;
+                q_off[i] = rl * pl.map_stride + (uy[i] + pl.halo_y) * pl.WP + (ux[i] + pl.halo_x);
+            }
+            float acc[PXT][4][CT];
+#pragma unroll
+            for (int i = 0; i < PXT; ++i)
+#pragma unroll
+                for (int cls = 0; cls < 4; ++cls)
+#pragma unroll
+                    for (int c = 0; c < CT; ++c) acc[i][cls][c] = 0.0f;
+#pragma unroll 2
+            for (int co = 0; co < g.c_out; ++co) {
+                const float *wc = Ws + co * w_co;
+                const float *qc = Qs + co * plane;
+#pragma unroll
+                for (int dy = 0; dy < T; ++dy) {
+#pragma unroll
+                    for (int dx = 0; dx < T; ++dx) {
+                        float qv[PXT];
+#pragma unroll
+                        for (int i = 0; i < PXT; ++i) qv[i] = qc[q_off[i] - dy * pl.WP - dx];
+#pragma unroll
+                        for (int cy = 0; cy < 2; ++cy) {
+#pragma unroll
+                            for (int cx = 0; cx < 2; ++cx) {
+                                // kernel element (cy + 2dy, cx + 2dx), channels 0..3 (cpad = 4 here)
+                                const float4 w4 = *reinterpret_cast<const float4 *>(
+                                    wc + (cy + 2 * dy) * w_ky + (cx + 2 * dx) * pl.cpad);
+                                const float wv[4] = {w4.x, w4.y, w4.z, w4.w};
+#pragma unroll
+                                for (int i = 0; i < PXT; ++i)
+#pragma unroll
+                                    for (int c = 0; c < CT; ++c)
+                                        acc[i][cy * 2 + cx][c] = fmaf(qv[i], wv[c], acc[i][cy * 2 + cx][c]);
+                            }
+                        }
+                    }
+                }
+            }
+            // ---- what follows the step on the path, per element ----
+#pragma unroll
+            for (int i = 0; i < PXT; ++i) {
+                if (!ok[i]) continue;
+#pragma unroll
+                for (int cy = 0; cy < 2; ++cy) {
+                    const int iy = 2 * uy[i] + cy - g.pad;
+                    if (iy < 0 || iy >= g.h_in) continue;
+#pragma unroll
+                    for (int cx = 0; cx < 2; ++cx) {
+                        const int ix = 2 * ux[i] + cx - g.pad;
+                        if (ix < 0 || ix >= g.w_in) continue;
+#pragma unroll
+                        for (int c = 0; c < CT; ++c) {
+                            if (c >= g.c_in) continue;
+                            finish_element<EPI>(acc[i][cy * 2 + cx][c], c * hw_in + iy * g.w_in + ix, r, upper, vec,
+                                                ld_in, ep, dacc);
+                        }
+                    }
+                }
+            }
+        }
+        // Row constants: lanes of a group by shuffles, warps in warp order.
+        for (int o = 1; o < G; o <<= 1) dacc += __shfl_xor_sync(0xffffffffu, dacc, o);
+        if (gl == 0) red[warp * kMaxRowsPerGroup + rl] = dacc;
+        __syncthreads();
+        if (threadIdx.x < RB && r0 + threadIdx.x < rows) {
+            const long long row = r0 + threadIdx.x;
+            float tot = ep.d_in[row];
+            for (int sl = 1; sl < ep.n_slots_in; ++sl) tot += ep.d_in[(size_t)sl * ep.slot_stride + row];
+            for (int w2 = 0; w2 < kWarps; ++w2) tot += red[w2 * kMaxRowsPerGroup + threadIdx.x];
+            if (EPI == CONVT_EPI_CONCRETIZE) {
+                const int b2 = (int)(row / (2LL * ep.n_k)), up2 = (int)((row / ep.n_k) & 1), i2 = (int)(row % ep.n_k);
+                (up2 ? ep.ub_out : ep.lb_out)[(size_t)b2 * ep.n_total + ep.out_off + i2] = tot;
+            } else {
+                ep.d_out[row] = tot;
+            }
+        }
+        if (EPI == CONVT_EPI_RELU) {
+            // keep the padded tail of the rows at zero
+            for (int q = 0; q < RB; ++q) {
+                if (r0 + q >= rows) break;
+                const size_t o = (size_t)(r0 + q) * ld_in;
+                for (int t = n_in + threadIdx.x; t < ld_in; t += kThreads) {
+                    ep.P[o + t] = 0.0f;
+                    if (ep.P_lo) ep.P_lo[o + t] = 0.0f;
+                }
+            }
+        }
+    }
+}
+
 template <int CT, int PXT>
 void launch_ct(const LayerDev &L, const ConvtPlan &pl, const float *Q, long long rows, int sms,
                const ConvtEpilogue &ep, cudaStream_t st) {
@@ -375,6 +598,35 @@ void prepare_ct() {
                          (int)kSmemBudget);
 }
 
+template <int CT, int PXT, int T>
+void launch_s2(const LayerDev &L, const ConvtPlan &pl, const float *Q, long long rows, int sms,
+               const ConvtEpilogue &ep, cudaStream_t st) {
+    long long groups = ceil_div_ll(rows, pl.rows_per_group);
+    int grid = (int)std::min<long long>(groups, 2LL * sms);
+    if (ep.mode == CONVT_EPI_CONCRETIZE)
+        convt_s2_kernel<CT, PXT, T, CONVT_EPI_CONCRETIZE><<<grid, kThreads, pl.smem_bytes, st>>>(
+            Q, L.ld_out, L.ld_in, L.Wct, geom_of(L), pl, rows, ep);
+    else
+        convt_s2_kernel<CT, PXT, T, CONVT_EPI_RELU><<<grid, kThreads, pl.smem_bytes, st>>>(
+            Q, L.ld_out, L.ld_in, L.Wct, geom_of(L), pl, rows, ep);
+}
+
+template <int CT, int PXT>
+void launch_s2_taps(const LayerDev &L, const ConvtPlan &pl, const float *Q, long long rows, int sms,
+                    const ConvtEpilogue &ep, cudaStream_t st) {
+    if (pl.ty == 1) launch_s2<CT, PXT, 1>(L, pl, Q, rows, sms, ep, st);
+    else if (pl.ty == 2) launch_s2<CT, PXT, 2>(L, pl, Q, rows, sms, ep, st);
+    else launch_s2<CT, PXT, 3>(L, pl, Q, rows, sms, ep, st);
+}
+
+template <int CT, int PXT, int T>
+void prepare_s2() {
+    cudaFuncSetAttribute(convt_s2_kernel<CT, PXT, T, CONVT_EPI_RELU>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                         (int)kSmemBudget);
+    cudaFuncSetAttribute(convt_s2_kernel<CT, PXT, T, CONVT_EPI_CONCRETIZE>,
+                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget);
+}
+
 }  // namespace
 
 // Whether the back-step through this conv layer fits the kernel's shared-memory plan.
@@ -384,6 +636,8 @@ bool convt_supported(const LayerDev &L) {
 }
 
 void convt_prepare() {
+    prepare_s2<3, 5, 1>(); prepare_s2<3, 5, 2>(); prepare_s2<3, 5, 3>();
+    prepare_s2<4, 4, 1>(); prepare_s2<4, 4, 2>(); prepare_s2<4, 4, 3>();
     prepare_ct<3, 8>();
     prepare_ct<4, 4>();
     prepare_ct<8, 4>();
@@ -393,6 +647,11 @@ void convt_prepare() {
 void launch_convt_ffma(const LayerDev &L, const float *Q, long long rows, int sms, const ConvtEpilogue &ep,
                        cudaStream_t st) {
     const ConvtPlan pl = make_plan(L);
+    if (pl.s2) {
+        if (L.c_in == 3) launch_s2_taps<3, 5>(L, pl, Q, rows, sms, ep, st);
+        else launch_s2_taps<4, 4>(L, pl, Q, rows, sms, ep, st);
+        return;
+    }
     if (L.c_in == 3) launch_ct<3, 8>(L, pl, Q, rows, sms, ep, st);
     else if (L.c_in <= 4) launch_ct<4, 4>(L, pl, Q, rows, sms, ep, st);
     else if (L.c_in <= 8) launch_ct<8, 4>(L, pl, Q, rows, sms, ep, st);
