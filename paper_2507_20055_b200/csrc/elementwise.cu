@@ -160,7 +160,57 @@ __global__ void relax_kernel(float *__restrict__ lb_out, float *__restrict__ ub_
     nuU[idx] = nu;
 }
 
-// FROM_WEIGHTS: source is row i of W_k (start of a back-substitution), else P in place.
+// Start of a back-substitution at a conv layer k: the expression of neuron i = (co, oy, ox) is zero except
+// on the window [y0, y0+kh) x [x0, x0+kw) of every input channel, so a warp clears its row with 16-byte
+// stores and then places the c_in*kh*kw window coefficients, pushed through the ReLU below as in
+// relu_step_kernel (a zero coefficient contributes nothing to the row or to the constant).
+__global__ void conv_expr_start_kernel(const float *__restrict__ Wk, ConvGeom gk, const float *__restrict__ bias_k,
+                                       float *__restrict__ P, float *__restrict__ P_lo, float *__restrict__ d,
+                                       long long rows, int n_k, int ld, int has_relu,
+                                       const float *__restrict__ lamL, const float *__restrict__ lamU,
+                                       const float *__restrict__ nuU, const float *__restrict__ bias_below) {
+    long long r = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    int lane = threadIdx.x & 31;
+    if (r >= rows) return;
+    int b = (int)(r / (2LL * n_k));
+    int upper = (int)((r / n_k) & 1);
+    int i = (int)(r % n_k);
+    float *prow = P + (size_t)r * ld;
+    float *lrow = P_lo ? P_lo + (size_t)r * ld : nullptr;
+    const float4 zero = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int t = lane * 4; t < ld; t += 128) {
+        *reinterpret_cast<float4 *>(prow + t) = zero;
+        if (lrow) *reinterpret_cast<float4 *>(lrow + t) = zero;
+    }
+    __syncwarp();      // orders the clearing stores before the window stores of other lanes
+    const float *ll = lamL + (size_t)b * ld, *lu = lamU + (size_t)b * ld, *nu = nuU + (size_t)b * ld;
+    const int hw_o = gk.h_out * gk.w_out;
+    const int co = i / hw_o;
+    const int y0 = ((i / gk.w_out) % gk.h_out) * gk.stride - gk.pad;
+    const int x0 = (i % gk.w_out) * gk.stride - gk.pad;
+    const int khw = gk.kh * gk.kw, taps = gk.c_in * khw;
+    float dacc = 0.0f;
+    for (int q = lane; q < taps; q += 32) {
+        const int ci = q / khw, ky = (q / gk.kw) % gk.kh, kx = q % gk.kw;
+        const int iy = y0 + ky, ix = x0 + kx;
+        if (iy < 0 || iy >= gk.h_in || ix < 0 || ix >= gk.w_in) continue;
+        const int t = (ci * gk.h_in + iy) * gk.w_in + ix;
+        const float c = Wk[(size_t)co * taps + q];
+        const float qv = has_relu ? relu_backstep(c, upper, ll[t], lu[t], nu[t], dacc) : c;
+        dacc = fmaf(qv, bias_below[t], dacc);
+        if (lrow) {
+            const float h = tf32_round(qv);
+            prow[t] = h;
+            lrow[t] = tf32_round(qv - h);
+        } else {
+            prow[t] = qv;
+        }
+    }
+    dacc = warp_sum(dacc);
+    if (lane == 0) d[r] = bias_k[i] + dacc;
+}
+
+// FROM_WEIGHTS: source is row i of the FC layer W_k (start of a back-substitution), else P in place.
 template <bool FROM_WEIGHTS>
 __global__ void relu_step_kernel(const float *__restrict__ Wk, int kind_k, ConvGeom gk, int ldw_k,
                                  const float *__restrict__ bias_k, float *__restrict__ P,
@@ -177,36 +227,10 @@ __global__ void relu_step_kernel(const float *__restrict__ Wk, int kind_k, ConvG
     float *prow = P + (size_t)r * ld;
     const float *ll = lamL + (size_t)b * ld, *lu = lamU + (size_t)b * ld, *nu = nuU + (size_t)b * ld;
     float dacc = 0.0f;
-    // Conv layer k: neuron i = (co, oy, ox) sees the window [y0, y0+kh) x [x0, x0+kw) of every input
-    // channel; column t = (ci, iy, ix) is tracked incrementally (the column index advances by 128).
-    int co = 0, y0 = 0, x0 = 0, ci = 0, iy = 0, ix = 0, d_ci = 0, d_iy = 0, d_ix = 0;
-    if (FROM_WEIGHTS && kind_k != CERT_LAYER_FC) {
-        const int hw_o = gk.h_out * gk.w_out, hw_i = gk.h_in * gk.w_in;
-        co = i / hw_o;
-        y0 = ((i / gk.w_out) % gk.h_out) * gk.stride - gk.pad;
-        x0 = (i % gk.w_out) * gk.stride - gk.pad;
-        const int t0 = lane * 4;
-        ci = t0 / hw_i; iy = (t0 / gk.w_in) % gk.h_in; ix = t0 % gk.w_in;
-        d_ci = 128 / hw_i; d_iy = (128 / gk.w_in) % gk.h_in; d_ix = 128 % gk.w_in;
-    }
     // four consecutive columns per lane: 16-byte accesses (every row pitch is a multiple of 32 floats)
     for (int t = lane * 4; t < ld; t += 128) {
         float c[4], q[4];
-        if (FROM_WEIGHTS && kind_k != CERT_LAYER_FC) {
-            int cie = ci, iye = iy, ixe = ix;
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                const int ky = iye - y0, kx = ixe - x0;
-                const bool in = (t + e < n) && ky >= 0 && ky < gk.kh && kx >= 0 && kx < gk.kw;
-                c[e] = in ? Wk[(((size_t)co * gk.c_in + cie) * gk.kh + ky) * gk.kw + kx] : 0.0f;
-                if (++ixe >= gk.w_in) { ixe = 0; if (++iye >= gk.h_in) { iye = 0; ++cie; } }
-            }
-            ix += d_ix;
-            if (ix >= gk.w_in) { ix -= gk.w_in; ++iy; }
-            iy += d_iy;
-            if (iy >= gk.h_in) { iy -= gk.h_in; ++ci; }
-            ci += d_ci;
-        } else {
+        {
             const float4 c4 = *reinterpret_cast<const float4 *>(FROM_WEIGHTS ? Wk + (size_t)i * ldw_k + t : prow + t);
             c[0] = c4.x; c[1] = c4.y; c[2] = c4.z; c[3] = c4.w;
         }
@@ -302,6 +326,12 @@ void launch_relax(const LayerDev &L, float *lb_out, float *ub_out, int n_total, 
 void launch_init_expr(const LayerDev &Lk, const LayerDev &Lb, int batch, float *Q, float *Q_lo, float *d,
                       cudaStream_t st) {
     long long rows = 2LL * batch * Lk.n_out;
+    if (Lk.kind != CERT_LAYER_FC) {
+        conv_expr_start_kernel<<<grid_for_warps(rows), kWarpsPerBlock * 32, 0, st>>>(
+            Lk.W, geom_of(Lk), Lk.bias_n, Q, Q_lo, d, rows, Lk.n_out, Lb.ld_out, Lb.relu_after, Lb.lamL, Lb.lamU,
+            Lb.nuU, Lb.bias_n);
+        return;
+    }
     relu_step_kernel<true><<<grid_for_warps(rows), kWarpsPerBlock * 32, 0, st>>>(
         Lk.W, Lk.kind, geom_of(Lk), Lk.ld_in, Lk.bias_n, Q, Q_lo, d, 1, 0, rows, Lk.n_out, Lb.n_out, Lb.ld_out,
         Lb.relu_after, Lb.lamL, Lb.lamU, Lb.nuU, Lb.bias_n);
