@@ -159,6 +159,16 @@ cert_status_t cert_net_set_contraction(cert_net_t *net, int mode);
 int cert_net_last_contraction_paths(const cert_net_t *net);
 
 /*
+ * Conv-sourced rows as patches (on by default).  The expressions of a conv layer's neurons over conv
+ * layers below are zero outside a receptive-field window (Section 5 keeps such rows as convolution /
+ * patches blocks); while the traversal stays in conv layers and the window is at most half the map,
+ * the rows travel as [channels][window] patches instead of dense coefficient maps.  Off: every
+ * back-step works on dense maps.  The bounds are the same up to summation order.
+ * cert_net_last_contraction_paths sets bit 3 when a traversal of the last call ran on patches.
+ */
+cert_status_t cert_net_set_conv_patches(cert_net_t *net, int on);
+
+/*
  * Per-kernel-class device times.  With profiling on, cert_deeppoly_bounds
  * records a CUDA event on `stream` after every launch (the events are created
  * by cert_net_set_profiling, not in the hot call).  cert_net_profile waits for

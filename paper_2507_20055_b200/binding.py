@@ -32,7 +32,7 @@ EXPORTS = [
     "cert_net_num_neurons", "cert_net_num_relu_neurons", "cert_net_branch_codes",
     "cert_net_last_status", "cert_net_set_contraction", "cert_net_last_launch_count",
     "cert_net_backstep_flops", "cert_status_string", "cert_net_set_profiling", "cert_net_profile",
-    "cert_net_last_contraction_paths", "cert_first_layer_bounds_noalloc",
+    "cert_net_last_contraction_paths", "cert_first_layer_bounds_noalloc", "cert_net_set_conv_patches",
 ]
 CLASS_NAMES = ["input", "relax", "relu_step", "affine", "conv", "concretize"]
 
@@ -73,6 +73,8 @@ _lib.cert_net_backstep_flops.argtypes = [_vp, _i]
 _lib.cert_net_backstep_flops.restype = ctypes.c_double
 _lib.cert_net_last_contraction_paths.argtypes = [_vp]
 _lib.cert_net_last_contraction_paths.restype = _i
+_lib.cert_net_set_conv_patches.argtypes = [_vp, _i]
+_lib.cert_net_set_conv_patches.restype = _i
 _lib.cert_net_set_profiling.argtypes = [_vp, _i]
 _lib.cert_net_set_profiling.restype = _i
 _lib.cert_net_profile.argtypes = [_vp, _vp, _vp]
@@ -226,6 +228,9 @@ class CertNet:
 
     def set_contraction(self, mode: int):
         _check(_lib.cert_net_set_contraction(self._h, int(mode)), "cert_net_set_contraction")
+
+    def set_conv_patches(self, on: bool):
+        _check(_lib.cert_net_set_conv_patches(self._h, int(bool(on))), "cert_net_set_conv_patches")
 
     def last_contraction_paths(self) -> int:
         return int(_lib.cert_net_last_contraction_paths(self._h))

@@ -42,19 +42,22 @@ struct cert_net {
     long long slot_stride = 0;               // rows of the largest coefficient matrix
     int sm_count = 148;
     int tc_ctas = 1;                         // CTAs per row panel of the tensor-core kernel (2: cta_group::2)
+    bool conv_patches = true;                // conv-sourced rows travel as receptive-field patches where they can
     unsigned char *codes = nullptr;          // [max_batch][n_relu]
     int *status_dev = nullptr;               // sticky device status word
     // host staging for cert_deeppoly_bounds_host
     float *centers_dev = nullptr, *lb_dev = nullptr, *ub_dev = nullptr;
     int last_batch = 0;
     int last_launches = 0;
-    int last_paths = 0;              // bit 0: an FFMA contraction ran, bit 1: a tensor-core one, bit 2: in CTA pairs
+    int last_paths = 0;              // bit 0: an FFMA contraction ran, bit 1: a tensor-core one, bit 2: in CTA pairs, bit 3: a traversal ran on patches
     // optional per-launch event timing (events are created when profiling is switched on)
     bool profiling = false;
     std::vector<cudaEvent_t> prof_events;
     std::vector<int> prof_class;   // class of the launch between event i and i+1
     int prof_marks = 0;
 };
+
+constexpr int kMaxPatchLevels = 16;
 
 namespace cert {
 bool convt_supported(const LayerDev &L);
@@ -364,6 +367,7 @@ cert_status_t cert_net_create(const cert_layer_desc_t *layers, int n_layers, int
     }
     if (fail == CERT_OK) {
         cert::convt_prepare();
+        cert::conv_patch_prepare();
         if (cudaDeviceSynchronize() != cudaSuccess) fail = CERT_ERR_CUDA;
     }
     if (fail != CERT_OK) {
@@ -428,6 +432,40 @@ cert_status_t cert_backsub_bounds(cert_net_t *net, const float *centers, float e
         auto on_tc = [&](int j) {
             return net->contraction != CERT_CONTRACTION_FFMA && net->tc_ok && net->tc[j].usable;
         };
+        // A conv layer over conv layers: rows as receptive-field patches instead of dense maps.
+        cert::PatchLevel lv[kMaxPatchLevels];
+        if (net->conv_patches && cert::conv_patch_plan(net->layers.data(), k, j_end, lv, kMaxPatchLevels)) {
+            cert::launch_patch_start(Lk, net->layers[k - 1], lv[0], batch, net->buf[cur], net->dbuf[dcur], st);
+            rec.mark(CERT_CLASS_RELU_STEP);
+            for (int j = k - 1, m = 0; j >= j_end; --j, ++m) {
+                const LayerDev &Lj = net->layers[j];
+                cert::ConvtEpilogue ep;
+                std::memset(&ep, 0, sizeof(ep));
+                ep.n_k = Lk.n_out;
+                ep.d_in = net->dbuf[dcur]; ep.n_slots_in = 1; ep.slot_stride = net->slot_stride;
+                ep.d_out = net->dbuf[dcur];
+                if (j > j_end) {
+                    const LayerDev &Lb = net->layers[j - 1];
+                    ep.mode = cert::CONVT_EPI_RELU;
+                    ep.has_relu = Lb.relu_after;
+                    ep.lamL = Lb.lamL; ep.lamU = Lb.lamU; ep.nuU = Lb.nuU; ep.bias_below = Lb.bias_n;
+                    ep.P = net->buf[cur ^ 1];
+                } else {
+                    ep.mode = cert::CONVT_EPI_CONCRETIZE;
+                    ep.l0 = box_l; ep.u0 = box_u;
+                    ep.lb_out = lb_out; ep.ub_out = ub_out; ep.n_total = n_total; ep.out_off = Lk.out_off;
+                }
+                cert::launch_patch_step(Lk, Lj, lv[m], lv[m + 1], net->buf[cur], rows, net->sm_count, ep, st);
+                rec.mark(CERT_CLASS_CONV);
+                cur ^= 1;
+            }
+            if (Lk.relu_after || k + 1 < K) {
+                cert::launch_relax(Lk, lb_out, ub_out, n_total, batch, net->codes, net->n_relu, nullptr, 0, 0, st);
+                rec.mark(CERT_CLASS_RELAX);
+            }
+            paths |= 8;
+            continue;
+        }
         // expression over the outputs of layer k-1, pushed through its ReLU
         cert::launch_init_expr(Lk, net->layers[k - 1], batch, net->buf[cur],
                                on_tc(k - 1) ? net->buf_lo[cur] : nullptr, net->dbuf[dcur], st);
@@ -649,6 +687,12 @@ cert_status_t cert_net_profile(cert_net_t *net, float *ms_out, int *launches_out
 }
 
 int cert_net_last_contraction_paths(const cert_net_t *net) { return net ? net->last_paths : -1; }
+
+cert_status_t cert_net_set_conv_patches(cert_net_t *net, int on) {
+    if (!net) return CERT_ERR_INVALID_ARG;
+    net->conv_patches = on != 0;
+    return CERT_OK;
+}
 
 int cert_net_last_launch_count(const cert_net_t *net) { return net ? net->last_launches : -1; }
 

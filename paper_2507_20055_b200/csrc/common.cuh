@@ -115,4 +115,22 @@ struct ConvtEpilogue {
 void launch_convt_ffma(const LayerDev &L, const float *Q, long long rows, int sms, const ConvtEpilogue &ep,
                        cudaStream_t st);
 
+// ---- conv back-steps on receptive-field patches (conv_patch.cu) ----
+// One level of a conv neuron's expression held as a window [c][ph][pw] whose origin in the map is
+// (oy, ox) * a - b for the neuron's output position (oy, ox).
+struct PatchLevel {
+    int c, ph, pw, a, b, elems, pitch;
+};
+// Plans the traversal of conv layer k's expressions through layers k-1 .. j_end on patches:
+// levels[0] is over the outputs of layer k-1, levels[m] over the inputs of layer k-m.  False when a
+// layer on the way is not a conv layer or a window is not much smaller than its map.
+bool conv_patch_plan(const LayerDev *layers, int k, int j_end, PatchLevel *levels, int max_levels);
+void conv_patch_prepare();
+// Start: the kernel of layer k as a patch over the outputs of the layer below, through that layer's ReLU.
+void launch_patch_start(const LayerDev &Lk, const LayerDev &Lb, const PatchLevel &lv, int batch, float *patch,
+                        float *d, cudaStream_t st);
+// Back-step of the patches through conv layer j, followed by `ep` (ep.P = output patches, pitch out.pitch).
+void launch_patch_step(const LayerDev &Lk, const LayerDev &Lj, const PatchLevel &in, const PatchLevel &out,
+                       const float *in_patch, long long rows, int sms, const ConvtEpilogue &ep, cudaStream_t st);
+
 }  // namespace cert

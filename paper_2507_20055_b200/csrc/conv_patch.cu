@@ -1,0 +1,241 @@
+// Conv back-steps on receptive-field patches.
+//
+// The expression of a conv neuron (co, oy, ox) of layer k over the outputs of a conv layer below is
+// zero outside a window: the kernel's footprint, grown by (ph - 1) * stride + kernel at every further
+// conv layer it is pushed through (the paper keeps such rows as convolution / patches blocks instead of
+// dense ones, Section 5 and Appendix B).  While every layer between k and the end of the traversal is a
+// conv layer and the window is smaller than the map, a row is held as the patch [C][ph][pw] plus the
+// window's origin, which is a function of (oy, ox) alone:
+//
+//   level j (expression over the outputs of layer j):  origin_j = (oy, ox) * a_j - b_j
+//   start (j = k-1):            ph = kh_k,                a = stride_k,      b = pad_k
+//   through conv layer j:       ph' = (ph-1)*s_j + kh_j,  a' = a * s_j,      b' = b * s_j + pad_j
+//
+// In patch coordinates the back-step is a transposed convolution without padding,
+//   out[ci][s*py + ky][s*px + kx] += in[co][py][px] * W[co][ci][ky][kx],
+// and window positions that fall outside the image belong to no neuron: they carry no coefficient.
+// The ReLU back-step below (replace_lower/upper) or the concretisation (map(simplify_*)) is applied
+// to each element at its position in the image, exactly as in the dense kernels.
+// One warp per row; row constants are warp-shuffle sums (fixed order).
+#include "common.cuh"
+
+namespace cert {
+
+namespace {
+
+constexpr int kWarpsPerBlock = 8;
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+// replace_lower / replace_upper through a ReLU neuron with L = lamL*z, U = lamU*z + nuU.
+__device__ __forceinline__ float relu_backstep(float c, int upper, float lamL, float lamU, float nuU,
+                                               float &dacc) {
+    const bool nonneg = (c >= 0.0f);
+    const bool use_lower = upper ? !nonneg : nonneg;
+    if (use_lower) return c * lamL;
+    dacc = fmaf(c, nuU, dacc);
+    return c * lamU;
+}
+
+// Start at conv layer k: patch over the layer's inputs = its kernel [c_in][kh][kw] at origin
+// (oy*stride - pad, ox*stride - pad), pushed through the ReLU below; constant = bias + the nu terms +
+// Q.b of the layer below.  Out-of-image window positions get 0.
+__global__ void patch_start_kernel(const float *__restrict__ Wk, ConvGeom gk, const float *__restrict__ bias_k,
+                                   float *__restrict__ patch, int pitch, float *__restrict__ d, long long rows,
+                                   int n_k, int ld, int has_relu, const float *__restrict__ lamL,
+                                   const float *__restrict__ lamU, const float *__restrict__ nuU,
+                                   const float *__restrict__ bias_below) {
+    const long long r = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int lane = threadIdx.x & 31;
+    if (r >= rows) return;
+    const int b = (int)(r / (2LL * n_k));
+    const int upper = (int)((r / n_k) & 1);
+    const int i = (int)(r % n_k);
+    const int hw_o = gk.h_out * gk.w_out;
+    const int co = i / hw_o;
+    const int y0 = ((i / gk.w_out) % gk.h_out) * gk.stride - gk.pad;
+    const int x0 = (i % gk.w_out) * gk.stride - gk.pad;
+    const int khw = gk.kh * gk.kw, taps = gk.c_in * khw;
+    const size_t vec = (size_t)b * ld;
+    float *prow = patch + (size_t)r * pitch;
+    float dacc = 0.0f;
+    for (int q = lane; q < pitch; q += 32) {
+        float qv = 0.0f;
+        if (q < taps) {
+            const int ci = q / khw, ky = (q / gk.kw) % gk.kh, kx = q % gk.kw;
+            const int iy = y0 + ky, ix = x0 + kx;
+            if (iy >= 0 && iy < gk.h_in && ix >= 0 && ix < gk.w_in) {
+                const int t = (ci * gk.h_in + iy) * gk.w_in + ix;
+                const float c = Wk[(size_t)co * taps + q];
+                qv = has_relu ? relu_backstep(c, upper, lamL[vec + t], lamU[vec + t], nuU[vec + t], dacc) : c;
+                dacc = fmaf(qv, bias_below[t], dacc);
+            }
+        }
+        prow[q] = qv;
+    }
+    dacc = warp_sum(dacc);
+    if (lane == 0) d[r] = bias_k[i] + dacc;
+}
+
+// Geometry of one patch back-step through conv layer j for the rows of conv layer k.
+struct PatchStep {
+    int ph, pw;              // input patch (over the outputs of layer j): [c_out][ph][pw]
+    int qh, qw;              // output patch (over the inputs of layer j): [c_in][qh][qw], qh = (ph-1)*s + kh
+    int pitch_in, pitch_out; // floats per row of the patch buffers
+    int a, b;                // origin of the output patch = (oy, ox) * a - b
+    int hw_k, w_k;           // layer k's output map h*w and w (decode neuron -> (oy, ox))
+};
+
+// Shared memory: weights [c_out][c_in][kh][kw], then one input patch per warp.
+template <int EPI>
+__global__ void __launch_bounds__(kWarpsPerBlock * 32)
+patch_step_kernel(const float *__restrict__ in, const float *__restrict__ W, ConvGeom g, PatchStep ps,
+                  long long rows, int ld_in, ConvtEpilogue ep) {
+    extern __shared__ __align__(16) float smem[];
+    const int n_w = g.c_out * g.c_in * g.kh * g.kw;
+    const int n_inp = g.c_out * ps.ph * ps.pw;
+    float *Ws = smem;
+    float *my_patch = smem + n_w + (threadIdx.x >> 5) * n_inp;
+    for (int i = threadIdx.x; i < n_w; i += blockDim.x) Ws[i] = W[i];
+    __syncthreads();
+
+    const int lane = threadIdx.x & 31;
+    const int warps_total = gridDim.x * kWarpsPerBlock;
+    const int s = g.stride;
+    const int khw = g.kh * g.kw, w_co = g.c_in * khw;
+    const int phw = ps.ph * ps.pw, qhw = ps.qh * ps.qw;
+    const int n_outp = g.c_in * qhw;
+    const int hw_in = g.h_in * g.w_in;
+
+    for (long long r = (long long)blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5); r < rows; r += warps_total) {
+        __syncwarp();
+        const float *irow = in + (size_t)r * ps.pitch_in;
+        for (int e = lane; e < n_inp; e += 32) my_patch[e] = irow[e];
+        __syncwarp();
+
+        const int box = (int)(r / (2LL * ep.n_k));
+        const int upper = (int)((r / ep.n_k) & 1);
+        const int i = (int)(r % ep.n_k);
+        const int oy = (i / ps.w_k) % (ps.hw_k / ps.w_k), ox = i % ps.w_k;
+        const int gy0 = oy * ps.a - ps.b, gx0 = ox * ps.a - ps.b;      // origin of the output patch in the image
+        const size_t vec = (size_t)box * ld_in;
+        float dacc = 0.0f;
+        for (int e = lane; e < n_outp; e += 32) {
+            const int ci = e / qhw, y = (e % qhw) / ps.qw, x = e % ps.qw;
+            const int gy = gy0 + y, gx = gx0 + x;
+            const bool inside = gy >= 0 && gy < g.h_in && gx >= 0 && gx < g.w_in;
+            float acc = 0.0f;
+            if (inside) {
+                for (int ky = y % s; ky < g.kh && ky <= y; ky += s) {
+                    const int py = (y - ky) / s;
+                    if (py >= ps.ph) continue;
+                    for (int kx = x % s; kx < g.kw && kx <= x; kx += s) {
+                        const int px = (x - kx) / s;
+                        if (px >= ps.pw) continue;
+                        const float *ip = my_patch + py * ps.pw + px;
+                        const float *wp = Ws + (ci * g.kh + ky) * g.kw + kx;
+#pragma unroll 4
+                        for (int co = 0; co < g.c_out; ++co) acc = fmaf(ip[co * phw], wp[co * w_co], acc);
+                    }
+                }
+                const int t = ci * hw_in + gy * g.w_in + gx;
+                if (EPI == CONVT_EPI_CONCRETIZE) {
+                    const bool nonneg = (acc >= 0.0f);
+                    dacc = fmaf(acc, (nonneg != (upper != 0)) ? ep.l0[vec + t] : ep.u0[vec + t], dacc);
+                } else {
+                    if (ep.has_relu) acc = relu_backstep(acc, upper, ep.lamL[vec + t], ep.lamU[vec + t], ep.nuU[vec + t], dacc);
+                    dacc = fmaf(acc, ep.bias_below[t], dacc);
+                }
+            }
+            if (EPI == CONVT_EPI_RELU) ep.P[(size_t)r * ps.pitch_out + e] = acc;
+        }
+        if (EPI == CONVT_EPI_RELU) {
+            for (int e = n_outp + lane; e < ps.pitch_out; e += 32) ep.P[(size_t)r * ps.pitch_out + e] = 0.0f;
+        }
+        dacc = warp_sum(dacc);
+        if (lane == 0) {
+            float tot = ep.d_in[r];
+            for (int sl = 1; sl < ep.n_slots_in; ++sl) tot += ep.d_in[(size_t)sl * ep.slot_stride + r];
+            tot += dacc;
+            if (EPI == CONVT_EPI_CONCRETIZE)
+                (upper ? ep.ub_out : ep.lb_out)[(size_t)box * ep.n_total + ep.out_off + i] = tot;
+            else
+                ep.d_out[r] = tot;
+        }
+    }
+}
+
+}  // namespace
+
+constexpr size_t kPatchSmemMax = 96 * 1024;
+
+static size_t patch_step_smem(const LayerDev &Lj, const PatchLevel &in) {
+    return sizeof(float) * ((size_t)Lj.c_out * Lj.c_in * Lj.kh * Lj.kw + (size_t)kWarpsPerBlock * in.elems);
+}
+
+bool conv_patch_plan(const LayerDev *layers, int k, int j_end, PatchLevel *levels, int max_levels) {
+    const LayerDev &Lk = layers[k];
+    if (Lk.kind != CERT_LAYER_CONV2D || k - j_end + 1 > max_levels) return false;
+    PatchLevel lv;
+    lv.c = Lk.c_in; lv.ph = Lk.kh; lv.pw = Lk.kw; lv.a = Lk.stride; lv.b = Lk.pad;
+    lv.elems = lv.c * lv.ph * lv.pw;
+    lv.pitch = round_up(lv.elems, 4);
+    if (2 * lv.elems > Lk.n_in) return false;            // the window is not much smaller than the map
+    levels[0] = lv;
+    for (int j = k - 1, m = 1; j >= j_end; --j, ++m) {
+        const LayerDev &Lj = layers[j];
+        if (Lj.kind != CERT_LAYER_CONV2D) return false;
+        if (patch_step_smem(Lj, levels[m - 1]) > kPatchSmemMax) return false;
+        PatchLevel nx;
+        nx.c = Lj.c_in;
+        nx.ph = (levels[m - 1].ph - 1) * Lj.stride + Lj.kh;
+        nx.pw = (levels[m - 1].pw - 1) * Lj.stride + Lj.kw;
+        nx.a = levels[m - 1].a * Lj.stride;
+        nx.b = levels[m - 1].b * Lj.stride + Lj.pad;
+        nx.elems = nx.c * nx.ph * nx.pw;
+        nx.pitch = round_up(nx.elems, 4);
+        if (2 * nx.elems > Lj.n_in) return false;
+        levels[m] = nx;
+    }
+    return true;
+}
+
+void conv_patch_prepare() {
+    cudaFuncSetAttribute(patch_step_kernel<CONVT_EPI_RELU>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                         (int)kPatchSmemMax);
+    cudaFuncSetAttribute(patch_step_kernel<CONVT_EPI_CONCRETIZE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                         (int)kPatchSmemMax);
+}
+
+void launch_patch_start(const LayerDev &Lk, const LayerDev &Lb, const PatchLevel &lv, int batch, float *patch,
+                        float *d, cudaStream_t st) {
+    const long long rows = 2LL * batch * Lk.n_out;
+    const unsigned grid = (unsigned)ceil_div_ll(rows, kWarpsPerBlock);
+    patch_start_kernel<<<grid, kWarpsPerBlock * 32, 0, st>>>(Lk.W, geom_of(Lk), Lk.bias_n, patch, lv.pitch, d, rows,
+                                                              Lk.n_out, Lb.ld_out, Lb.relu_after, Lb.lamL, Lb.lamU,
+                                                              Lb.nuU, Lb.bias_n);
+}
+
+void launch_patch_step(const LayerDev &Lk, const LayerDev &Lj, const PatchLevel &in, const PatchLevel &out,
+                       const float *in_patch, long long rows, int sms, const ConvtEpilogue &ep, cudaStream_t st) {
+    PatchStep ps;
+    ps.ph = in.ph; ps.pw = in.pw; ps.qh = out.ph; ps.qw = out.pw;
+    ps.pitch_in = in.pitch; ps.pitch_out = out.pitch;
+    ps.a = out.a; ps.b = out.b;
+    ps.hw_k = Lk.h_out * Lk.w_out; ps.w_k = Lk.w_out;
+    const size_t smem = patch_step_smem(Lj, in);
+    const long long blocks_needed = ceil_div_ll(rows, kWarpsPerBlock);
+    const int grid = (int)std::min<long long>(blocks_needed, 8LL * sms);
+    if (ep.mode == CONVT_EPI_CONCRETIZE)
+        patch_step_kernel<CONVT_EPI_CONCRETIZE><<<grid, kWarpsPerBlock * 32, smem, st>>>(in_patch, Lj.W, geom_of(Lj), ps,
+                                                                                      rows, Lj.ld_in, ep);
+    else
+        patch_step_kernel<CONVT_EPI_RELU><<<grid, kWarpsPerBlock * 32, smem, st>>>(in_patch, Lj.W, geom_of(Lj), ps, rows,
+                                                                                Lj.ld_in, ep);
+}
+
+}  // namespace cert

@@ -6,13 +6,15 @@ TOL = 1e-4            # |gpu - oracle| <= TOL * (1 + |oracle|)
 MARGIN_MIN = 1e-5     # boxes with a sign test closer to zero than this are ill-conditioned
 
 
-def run_gpu(w, contraction=None, max_batch=None, host_api=False, backsteps=None):
+def run_gpu(w, contraction=None, max_batch=None, host_api=False, backsteps=None, conv_patches=None):
     import torch
     from paper_2507_20055_b200 import binding
     net = binding.CertNet(w.layers, max_batch or w.batch, w.clip_lo, w.clip_hi)
     try:
         if contraction is not None:
             net.set_contraction(contraction)
+        if conv_patches is not None:
+            net.set_conv_patches(conv_patches)
         if host_api:
             lb, ub = net.deeppoly_bounds_host(w.centers, w.eps)
         else:

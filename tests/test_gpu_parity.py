@@ -191,3 +191,30 @@ def test_fused_steps_against_the_skippoly_listing(name):
     w = VARIANT_NETS[name]()
     ref = orc.skippoly(w.layers, w.centers, w.eps, w.clip_lo, w.clip_hi)
     compare(run_gpu(w), ref, label=f"{name}/skippoly")
+
+
+# ---- conv-sourced rows as dense maps and as receptive-field patches ----
+
+CONV_NETS = {
+    "convsmall": lambda: wl.make_config(3, batch=4),
+    "k3s2_k3s1": lambda: wl.small_conv((2, 9, 7), [(5, 3, 2, 1), (6, 3, 1, 1)], [20, 4], batch=3, eps=0.02, seed=66),
+    "k4s2_k4s2": lambda: wl.small_conv((3, 12, 12), [(8, 4, 2, 1), (12, 4, 2, 1)], [30, 5], batch=4, eps=0.01, seed=67),
+    "three_convs": lambda: wl.small_conv((2, 20, 18), [(4, 3, 1, 1), (6, 4, 2, 1), (8, 3, 2, 0)], [12, 3], batch=2,
+                                         eps=0.01, seed=85),
+    "k5s1p0_k2s2": lambda: wl.small_conv((1, 14, 14), [(6, 5, 1, 0), (4, 2, 2, 0)], [5], batch=2, eps=0.03, seed=86),
+}
+
+
+@pytest.mark.parametrize("patches", [False, True])
+@pytest.mark.parametrize("name", sorted(CONV_NETS))
+def test_conv_rows_dense_and_patches(name, patches):
+    w = CONV_NETS[name]()
+    ref = _oracle(w)
+    g = run_gpu(w, conv_patches=patches)
+    # the small nets' windows are not much smaller than their maps: those stay dense either way
+    expect_patches = patches and name in ("convsmall", "three_convs", "k5s1p0_k2s2")
+    assert bool(g["paths"] & 8) == expect_patches
+    compare(g, ref, label=f"{name}/patches={patches}")
+    steps = [0] + [1] * (len(w.layers) - 1)
+    ref1 = orc.deeppoly(w.layers, w.centers, w.eps, w.clip_lo, w.clip_hi, backsteps_per_layer=steps)
+    compare(run_gpu(w, conv_patches=patches, backsteps=steps), ref1, label=f"{name}/patches={patches}/p1")
