@@ -120,21 +120,46 @@ def certifier_steps(name, n_layers):
     raise SystemExit(f"unknown certifier {name!r}")
 
 
-def backstep_flops_by_class(layers, batch, steps=None):
+def patch_levels(layers, k, j_end):
+    """Window sizes [(channels, ph, pw), ...] of conv layer k's rows pushed through layers k-1 .. j_end, or None
+    where the library keeps dense maps (a non-conv layer on the way, or a window above half its map)."""
+    Lk = layers[k]
+    if Lk.kind != "conv":
+        return None
+    _, c_in, kh, kw = Lk.weight.shape
+    lv = [(c_in, kh, kw)]
+    if 2 * c_in * kh * kw > Lk.n_in:
+        return None
+    for j in range(k - 1, j_end - 1, -1):
+        Lj = layers[j]
+        if Lj.kind != "conv":
+            return None
+        _, cj, kjh, kjw = Lj.weight.shape
+        _, ph, pw = lv[-1]
+        nx = (cj, (ph - 1) * Lj.stride + kjh, (pw - 1) * Lj.stride + kjw)
+        if 2 * nx[0] * nx[1] * nx[2] > Lj.n_in:
+            return None
+        lv.append(nx)
+    return lv
+
+
+def backstep_flops_by_class(layers, batch, steps=None, patches=True):
     """Algorithmic flops of one call's back-steps: for every layer k, 2*batch*n_k rows go through the
-    earlier layers its traversal reaches; an FC step costs 2*n_j*n_{j-1} per row, a conv step
-    2*n_j*c_in*kh*kw (dense maps)."""
+    earlier layers its traversal reaches; an FC step costs 2*n_j*n_{j-1} per row, a conv step on dense
+    coefficient maps 2*n_j*c_in*kh*kw, a conv step on a receptive-field patch 2*(window elements)*c_in*kh*kw."""
     out = {"affine": 0.0, "conv": 0.0}
     for k in range(1, len(layers)):
         rows = 2.0 * batch * layers[k].n_out
         depth = k if steps is None or steps[k] < 0 else min(steps[k], k)
-        for j in range(k - depth, k):
+        lv = patch_levels(layers, k, k - depth) if (patches and depth > 0) else None
+        for m, j in enumerate(range(k - 1, k - depth - 1, -1)):
             L = layers[j]
             if L.kind == "fc":
                 out["affine"] += rows * 2.0 * L.n_out * L.n_in
             else:
                 _, c_in, kh, kw = L.weight.shape
-                out["conv"] += rows * 2.0 * L.n_out * c_in * kh * kw
+                elems = lv[m][0] * lv[m][1] * lv[m][2] if lv else L.n_out
+                out["conv"] += rows * 2.0 * elems * c_in * kh * kw
     return out
 
 
@@ -297,12 +322,13 @@ def main():
 
     if rank == 0:
         peaks = load_peaks()
-        flops_call = net.backstep_flops(B)
-        fl = backstep_flops_by_class(w.layers, B, args.backsteps)
-        if args.backsteps is None:
-            assert abs(fl["affine"] + fl["conv"] - flops_call) <= 1e-6 * flops_call
-        else:
-            flops_call = fl["affine"] + fl["conv"]
+        used_patches = bool(net.last_contraction_paths() & 8)
+        fl = backstep_flops_by_class(w.layers, B, args.backsteps, patches=used_patches)
+        flops_call = fl["affine"] + fl["conv"]
+        fl_dense = backstep_flops_by_class(w.layers, B, args.backsteps, patches=False)
+        if args.backsteps is None:      # the library's own count (dense maps) must agree
+            lib_count = net.backstep_flops(B)
+            assert abs(fl_dense["affine"] + fl_dense["conv"] - lib_count) <= 1e-6 * lib_count
         # the dominant kernel class: FC back-steps (tensor cores unless --contraction ffma) or conv back-steps (FMA units)
         dom = "affine" if cls_ms.get("affine", 0.0) >= cls_ms.get("conv", 0.0) else "conv"
         dom_ms, dom_n = cls_ms.get(dom, 0.0), cls_n.get(dom, 0)
@@ -326,6 +352,7 @@ def main():
                 "kernel": dom + " back-step", "launches_per_step": dom_n // max(1, args.steps),
                 "avg_launch_ms": dom_ms / dom_n if dom_n else None,
                 "flops_per_step": fl[dom], "flops_per_step_all_backsteps": flops_call,
+                "flops_per_step_if_dense_maps": fl_dense[dom], "conv_rows_as_patches": used_patches,
                 "peak_source": peaks["source"],
                 "peak_note": ("bf16_tflops_sustained/2/3 (3xTF32)" if used_tc else "148 SM x 128 FMA x 2 x sm_max_mhz"),
                 "class_ms_per_step": {k: v / args.steps for k, v in cls_ms.items()}}

@@ -90,7 +90,14 @@ struct PatchStep {
     int hw_k, w_k;           // layer k's output map h*w and w (decode neuron -> (oy, ox))
 };
 
-// Shared memory: weights [c_out][c_in][kh][kw], then one input patch per warp.
+// Shared memory: weights [c_out][c_in][kh][kw]; index tables (built once per block, so that the row loop has
+// no divisions): pix[p] = (y << 16) | x of output pixel p; for every output row y the taps (ky << 16) | py with
+// y = s*py + ky, 0 <= py < ph, ky < kh (count in ycnt[y]), the same for columns; then one input patch per warp.
+__host__ __device__ inline int patch_taps_max(int k, int s) { return (k + s - 1) / s; }
+__host__ __device__ inline int patch_table_ints(const ConvGeom &g, int qh, int qw) {
+    return qh * qw + qh * (patch_taps_max(g.kh, g.stride) + 1) + qw * (patch_taps_max(g.kw, g.stride) + 1);
+}
+
 template <int EPI>
 __global__ void __launch_bounds__(kWarpsPerBlock * 32)
 patch_step_kernel(const float *__restrict__ in, const float *__restrict__ W, ConvGeom g, PatchStep ps,
@@ -98,14 +105,31 @@ patch_step_kernel(const float *__restrict__ in, const float *__restrict__ W, Con
     extern __shared__ __align__(16) float smem[];
     const int n_w = g.c_out * g.c_in * g.kh * g.kw;
     const int n_inp = g.c_out * ps.ph * ps.pw;
+    const int s = g.stride;
+    const int tym = patch_taps_max(g.kh, s), txm = patch_taps_max(g.kw, s);
     float *Ws = smem;
-    float *my_patch = smem + n_w + (threadIdx.x >> 5) * n_inp;
+    int *pix = reinterpret_cast<int *>(smem + n_w);
+    int *ycnt = pix + ps.qh * ps.qw, *ytab = ycnt + ps.qh;
+    int *xcnt = ytab + ps.qh * tym, *xtab = xcnt + ps.qw;
+    float *my_patch = reinterpret_cast<float *>(xtab + ps.qw * txm) + (threadIdx.x >> 5) * n_inp;
     for (int i = threadIdx.x; i < n_w; i += blockDim.x) Ws[i] = W[i];
+    for (int p = threadIdx.x; p < ps.qh * ps.qw; p += blockDim.x) pix[p] = ((p / ps.qw) << 16) | (p % ps.qw);
+    for (int y = threadIdx.x; y < ps.qh; y += blockDim.x) {
+        int n = 0;
+        for (int ky = y % s; ky < g.kh && ky <= y; ky += s)
+            if ((y - ky) / s < ps.ph) ytab[y * tym + n++] = (ky << 16) | ((y - ky) / s);
+        ycnt[y] = n;
+    }
+    for (int x = threadIdx.x; x < ps.qw; x += blockDim.x) {
+        int n = 0;
+        for (int kx = x % s; kx < g.kw && kx <= x; kx += s)
+            if ((x - kx) / s < ps.pw) xtab[x * txm + n++] = (kx << 16) | ((x - kx) / s);
+        xcnt[x] = n;
+    }
     __syncthreads();
 
     const int lane = threadIdx.x & 31;
     const int warps_total = gridDim.x * kWarpsPerBlock;
-    const int s = g.stride;
     const int khw = g.kh * g.kw, w_co = g.c_in * khw;
     const int phw = ps.ph * ps.pw, qhw = ps.qh * ps.qw;
     const int n_outp = g.c_in * qhw;
@@ -125,17 +149,20 @@ patch_step_kernel(const float *__restrict__ in, const float *__restrict__ W, Con
         const size_t vec = (size_t)box * ld_in;
         float dacc = 0.0f;
         for (int e = lane; e < n_outp; e += 32) {
-            const int ci = e / qhw, y = (e % qhw) / ps.qw, x = e % ps.qw;
+            const int ci = e / qhw;
+            const int yx = pix[e - ci * qhw];
+            const int y = yx >> 16, x = yx & 0xffff;
             const int gy = gy0 + y, gx = gx0 + x;
             const bool inside = gy >= 0 && gy < g.h_in && gx >= 0 && gx < g.w_in;
             float acc = 0.0f;
             if (inside) {
-                for (int ky = y % s; ky < g.kh && ky <= y; ky += s) {
-                    const int py = (y - ky) / s;
-                    if (py >= ps.ph) continue;
-                    for (int kx = x % s; kx < g.kw && kx <= x; kx += s) {
-                        const int px = (x - kx) / s;
-                        if (px >= ps.pw) continue;
+                const int ny = ycnt[y], nx = xcnt[x];
+                for (int a = 0; a < ny; ++a) {
+                    const int yt = ytab[y * tym + a];
+                    const int ky = yt >> 16, py = yt & 0xffff;
+                    for (int b2 = 0; b2 < nx; ++b2) {
+                        const int xt = xtab[x * txm + b2];
+                        const int kx = xt >> 16, px = xt & 0xffff;
                         const float *ip = my_patch + py * ps.pw + px;
                         const float *wp = Ws + (ci * g.kh + ky) * g.kw + kx;
 #pragma unroll 4
@@ -174,7 +201,9 @@ patch_step_kernel(const float *__restrict__ in, const float *__restrict__ W, Con
 constexpr size_t kPatchSmemMax = 96 * 1024;
 
 static size_t patch_step_smem(const LayerDev &Lj, const PatchLevel &in) {
-    return sizeof(float) * ((size_t)Lj.c_out * Lj.c_in * Lj.kh * Lj.kw + (size_t)kWarpsPerBlock * in.elems);
+    const int qh = (in.ph - 1) * Lj.stride + Lj.kh, qw = (in.pw - 1) * Lj.stride + Lj.kw;
+    return sizeof(float) * ((size_t)Lj.c_out * Lj.c_in * Lj.kh * Lj.kw + (size_t)patch_table_ints(geom_of(Lj), qh, qw) +
+                            (size_t)kWarpsPerBlock * in.elems);
 }
 
 bool conv_patch_plan(const LayerDev *layers, int k, int j_end, PatchLevel *levels, int max_levels) {
