@@ -125,6 +125,58 @@ def deeppoly_matrix(layers, centers, eps, clip_lo=0.0, clip_hi=1.0, decision_fp3
     return lb_all, ub_all, codes_all
 
 
+def reusecert_matrix(layers, centers, eps, clip_lo=0.0, clip_hi=1.0, decision_fp32=True):
+    """ReuseCert (Appendix C listing) in layer-level form: the shapes of every layer's outputs are kept as
+    matrices over the input, [coefficients | constant], and an affine layer composes them with its sign-split
+    weights: L_k = W+ L_below + W- U_below + b, U_k = W+ U_below + W- L_below + b (clamp form of Section 4.3).
+    Returns lb, ub [batch, n_total] and codes [batch, n_relu]."""
+    A = [dense_matrix(l) for l in layers]
+    bias = [dense_bias(l) for l in layers]
+    L0, U0 = box(centers, eps, clip_lo, clip_hi)
+    batch, n0 = L0.shape
+    n_total = sum(a.shape[0] for a in A)
+    n_relu = sum(a.shape[0] for a, l in zip(A, layers) if l.relu_after)
+    lb_all, ub_all = np.empty((batch, n_total)), np.empty((batch, n_total))
+    codes_all = np.empty((batch, n_relu), dtype=np.uint8)
+    for b in range(batch):
+        l0, u0 = L0[b], U0[b]
+        off = coff = 0
+        Lb = Ub = None                       # [n, n0 + 1]: last column is the constant
+        for k, layer in enumerate(layers):
+            Wp, Wm = np.clip(A[k], 0.0, None), np.clip(A[k], None, 0.0)
+            if k == 0:
+                Lk = Uk = np.concatenate([A[0], bias[0][:, None]], axis=1)
+            else:
+                Lk = Wp @ Lb + Wm @ Ub
+                Uk = Wp @ Ub + Wm @ Lb
+                Lk[:, -1] += bias[k]
+                Uk[:, -1] += bias[k]
+            lb = np.clip(Lk[:, :n0], 0.0, None) @ l0 + np.clip(Lk[:, :n0], None, 0.0) @ u0 + Lk[:, -1]
+            ub = np.clip(Uk[:, :n0], 0.0, None) @ u0 + np.clip(Uk[:, :n0], None, 0.0) @ l0 + Uk[:, -1]
+            n_k = lb.shape[0]
+            lb_all[b, off:off + n_k], ub_all[b, off:off + n_k] = lb, ub
+            off += n_k
+            if layer.relu_after:
+                if decision_fp32:
+                    lf, uf = lb.astype(np.float32), ub.astype(np.float32)
+                    active, inactive, pick = lf >= 0, uf <= 0, (lf + uf) >= 0
+                else:
+                    active, inactive, pick = lb >= 0, ub <= 0, (lb + ub) >= 0
+                unstable = ~active & ~inactive
+                den = np.where(unstable, ub - lb, 1.0)
+                lam_u = np.where(active, 1.0, np.where(inactive, 0.0, ub / den))
+                nu_u = np.where(unstable, -(ub * lb) / den, 0.0)
+                lam_l = np.where(pick, 1.0, 0.0)
+                Lb = lam_l[:, None] * Lk
+                Ub = lam_u[:, None] * Uk
+                Ub[:, -1] += nu_u
+                codes_all[b, coff:coff + n_k] = np.where(active, 1, np.where(inactive, 0, 2 + pick))
+                coff += n_k
+            else:
+                Lb, Ub = Lk.copy(), Uk.copy()
+    return lb_all, ub_all, codes_all
+
+
 def forward_preactivations(layers, x):
     """Plain float64 forward pass; x [m, n0]; returns [m, n_total] pre-activations."""
     A = [dense_matrix(l) for l in layers]

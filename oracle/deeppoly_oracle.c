@@ -399,6 +399,131 @@ int oracle_deeppoly(const oracle_layer_t *layers, int n_layers, const float *cen
                           max_backsteps, NULL, 0, n_threads, lb, ub, codes, margins);
 }
 
+/*
+ * ReuseCert (Appendix C, ReuseCert listing; Section 6.1): every neuron keeps polyhedral bounds
+ * L, U expressed over the input layer (stop_traverse(n) = n[layer] <= 1), so an affine neuron's
+ * traversal is a single round: each ReLU neuron below is replaced by its stored L / U.
+ *   Affine, first layer:  L = U = prev.dot(w) + b (already over the input).
+ *   Affine, later layers: L = backsubs_lower_L(prev.dot(w)+b): coefficient c of ReLU neuron t is
+ *                         replaced by c*L_t if c >= 0 else c*U_t (upper: swapped); L_t, U_t are
+ *                         affine expressions over the input.
+ *   Relu:  l = prev[L].map(simplify_lower), u = prev[U].map(simplify_upper);
+ *          L = relu_n(l,u,prev) = (l+u >= 0) ? prev[L] : 0
+ *          U = compute_upper(l,u,prev) = l >= 0 ? prev[U] : u <= 0 ? 0 : u/(u-l)*prev[U] - u*l/(u-l).
+ * The listing stores concrete bounds only for the first and the last affine layer; here the
+ * l, u that the Relu transformer computes are reported for every affine layer (for the first and
+ * last layer they are the listing's own backsubs_lower/upper values).
+ * An affine layer directly on an affine layer uses the lower layer's L, U unchanged.
+ */
+static int reusecert_box(const oracle_layer_t *layers, int n_layers, const float *center, float eps,
+                         float clip_lo, float clip_hi, int decision_fp32,
+                         double *lb, double *ub, unsigned char *codes, double *margins)
+{
+    int n0 = layer_n_in(&layers[0]);
+    int n_max = n0;
+    for (int k = 0; k < n_layers; ++k) {
+        int n = layer_n_out(&layers[k]);
+        if (n > n_max) n_max = n;
+    }
+    size_t mat = (size_t)n_max * n0;
+    double *l0 = malloc(sizeof(double) * n0), *u0 = malloc(sizeof(double) * n0);
+    /* below: L, U (coefficients [neuron][input] and constants) of the outputs of the layer below */
+    double *CLb = malloc(sizeof(double) * mat), *CUb = malloc(sizeof(double) * mat);
+    double *dLb = malloc(sizeof(double) * n_max), *dUb = malloc(sizeof(double) * n_max);
+    double *CL = malloc(sizeof(double) * mat), *CU = malloc(sizeof(double) * mat);
+    double *dL = malloc(sizeof(double) * n_max), *dU = malloc(sizeof(double) * n_max);
+    double *row = malloc(sizeof(double) * n_max);
+    if (!l0 || !u0 || !CLb || !CUb || !dLb || !dUb || !CL || !CU || !dL || !dU || !row) return 1;
+    for (int s = 0; s < n0; ++s) {
+        volatile float lo = center[s] - eps, hi = center[s] + eps;
+        float lo_c = lo < clip_lo ? clip_lo : lo;
+        float hi_c = hi > clip_hi ? clip_hi : hi;
+        l0[s] = (double)lo_c;
+        u0[s] = (double)hi_c;
+    }
+    int off = 0, code_off = 0;
+    for (int k = 0; k < n_layers; ++k) {
+        int n_k = layer_n_out(&layers[k]);
+        int n_prev = layer_n_in(&layers[k]);
+        for (int i = 0; i < n_k; ++i) {
+            double b;
+            affine_row(&layers[k], i, row, &b);
+            double *cl = CL + (size_t)i * n0, *cu = CU + (size_t)i * n0;
+            if (k == 0) {
+                for (int s = 0; s < n0; ++s) cl[s] = cu[s] = row[s];
+                dL[i] = dU[i] = b;
+            } else {
+                for (int s = 0; s < n0; ++s) cl[s] = cu[s] = 0.0;
+                double a_l = b, a_u = b;
+                for (int t = 0; t < n_prev; ++t) {
+                    double c = row[t];
+                    if (c == 0.0) continue;
+                    /* replace_lower: c >= 0 ? c*n[L] : c*n[U];  replace_upper: c >= 0 ? c*n[U] : c*n[L] */
+                    const double *pl = (c >= 0.0 ? CLb : CUb) + (size_t)t * n0;
+                    const double *pu = (c >= 0.0 ? CUb : CLb) + (size_t)t * n0;
+                    for (int s = 0; s < n0; ++s) { cl[s] += c * pl[s]; cu[s] += c * pu[s]; }
+                    a_l += c * (c >= 0.0 ? dLb[t] : dUb[t]);
+                    a_u += c * (c >= 0.0 ? dUb[t] : dLb[t]);
+                }
+                dL[i] = a_l; dU[i] = a_u;
+            }
+            lb[off + i] = concretize(n0, 0, cl, dL[i], l0, u0);
+            ub[off + i] = concretize(n0, 1, cu, dU[i], l0, u0);
+        }
+        /* shapes of this layer's outputs, over the input, for the layer above */
+        for (int t = 0; t < n_k; ++t) {
+            double lamL = 1.0, lamU = 1.0, nuU = 0.0;
+            if (layers[k].relu_after) {
+                unsigned char code; double margin;
+                relu_relaxation(lb[off + t], ub[off + t], decision_fp32, &lamL, &lamU, &nuU, &code, &margin);
+                if (codes) codes[code_off + t] = code;
+                if (margins) margins[code_off + t] = margin;
+            }
+            const double *cl = CL + (size_t)t * n0, *cu = CU + (size_t)t * n0;
+            double *bl = CLb + (size_t)t * n0, *bu = CUb + (size_t)t * n0;
+            for (int s = 0; s < n0; ++s) { bl[s] = lamL * cl[s]; bu[s] = lamU * cu[s]; }
+            dLb[t] = lamL * dL[t];
+            dUb[t] = lamU * dU[t] + nuU;
+        }
+        if (layers[k].relu_after) code_off += n_k;
+        off += n_k;
+    }
+    free(l0); free(u0); free(CLb); free(CUb); free(dLb); free(dUb); free(CL); free(CU); free(dL); free(dU);
+    free(row);
+    return 0;
+}
+
+/* Same outputs as oracle_deeppoly, for the ReuseCert certifier. */
+int oracle_reusecert(const oracle_layer_t *layers, int n_layers, const float *centers, float eps,
+                     int batch, float clip_lo, float clip_hi, int decision_fp32, int n_threads,
+                     double *lb, double *ub, unsigned char *codes, double *margins)
+{
+    if (n_layers < 1 || batch < 0) return 2;
+    for (int k = 1; k < n_layers; ++k)
+        if (layer_n_in(&layers[k]) != layer_n_out(&layers[k - 1])) return 2;
+    int n0 = layer_n_in(&layers[0]);
+    int n_total = oracle_num_neurons(layers, n_layers);
+    int n_relu = oracle_num_relu_neurons(layers, n_layers);
+    int err = 0;
+#ifdef _OPENMP
+    if (n_threads > 0) omp_set_num_threads(n_threads);
+#else
+    (void)n_threads;
+#endif
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int b = 0; b < batch; ++b) {
+        int e = reusecert_box(layers, n_layers, centers + (size_t)b * n0, eps, clip_lo, clip_hi,
+                              decision_fp32, lb + (size_t)b * n_total, ub + (size_t)b * n_total,
+                              codes ? codes + (size_t)b * n_relu : NULL,
+                              margins ? margins + (size_t)b * n_relu : NULL);
+        if (e) {
+#pragma omp atomic write
+            err = e;
+        }
+    }
+    return err;
+}
+
 int oracle_max_threads(void)
 {
 #ifdef _OPENMP

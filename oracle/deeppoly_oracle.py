@@ -42,6 +42,7 @@ def _load():
         _lib = ctypes.CDLL(build())
         _lib.oracle_deeppoly.restype = ctypes.c_int
         _lib.oracle_backsub.restype = ctypes.c_int
+        _lib.oracle_reusecert.restype = ctypes.c_int
         _lib.oracle_num_neurons.restype = ctypes.c_int
         _lib.oracle_num_relu_neurons.restype = ctypes.c_int
         _lib.oracle_max_threads.restype = ctypes.c_int
@@ -118,6 +119,31 @@ def deeppoly(layers, centers, eps, clip_lo=0.0, clip_hi=1.0, decision_fp32=True,
 def ibp(layers, centers, eps, clip_lo=0.0, clip_hi=1.0, **kw):
     """IBP listing of Appendix C: no traversal at any layer."""
     return deeppoly(layers, centers, eps, clip_lo, clip_hi, backsteps_per_layer=[0] * len(layers), **kw)
+
+
+def reusecert(layers, centers, eps, clip_lo=0.0, clip_hi=1.0, decision_fp32=True,
+              n_threads: Optional[int] = None):
+    """ReuseCert listing of Appendix C (bounds kept over the input layer and reused); same outputs as deeppoly()."""
+    lib = _load()
+    arr, keep = _marshal(layers)
+    centers = np.ascontiguousarray(centers, dtype=np.float32)
+    batch = centers.shape[0]
+    n_total = lib.oracle_num_neurons(arr, len(layers))
+    n_relu = lib.oracle_num_relu_neurons(arr, len(layers))
+    lb = np.empty((batch, n_total), dtype=np.float64)
+    ub = np.empty((batch, n_total), dtype=np.float64)
+    codes = np.empty((batch, n_relu), dtype=np.uint8)
+    margins = np.empty((batch, n_relu), dtype=np.float64)
+    rc = lib.oracle_reusecert(arr, ctypes.c_int(len(layers)), ctypes.c_void_p(centers.ctypes.data),
+                              ctypes.c_float(eps), ctypes.c_int(batch), ctypes.c_float(clip_lo),
+                              ctypes.c_float(clip_hi), ctypes.c_int(int(decision_fp32)),
+                              ctypes.c_int(n_threads or 0),
+                              ctypes.c_void_p(lb.ctypes.data), ctypes.c_void_p(ub.ctypes.data),
+                              ctypes.c_void_p(codes.ctypes.data), ctypes.c_void_p(margins.ctypes.data))
+    if rc != 0:
+        raise RuntimeError(f"oracle_reusecert failed with code {rc}")
+    del keep
+    return {"lb": lb, "ub": ub, "codes": codes, "margins": margins}
 
 
 def skippoly(layers, centers, eps, clip_lo=0.0, clip_hi=1.0, **kw):

@@ -176,3 +176,53 @@ def test_skippoly_soundness_and_missing_relu():
         z = mat.forward_preactivations(w.layers, _samples(L0[b], U0[b], 50_000, seed=b))
         assert (z.min(axis=0) >= r["lb"][b] - 1e-9 * (1 + np.abs(r["lb"][b]))).all()
         assert (z.max(axis=0) <= r["ub"][b] + 1e-9 * (1 + np.abs(r["ub"][b]))).all()
+
+
+# ---- ReuseCert listing (Appendix C): shapes kept over the input layer and reused ----
+
+def test_reusecert_w1_hand_values():
+    g, layers = _w1()
+    v = g["variants"]["reusecert"]
+    r = orc.reusecert(layers, np.array([g["center"]], np.float32), g["eps"], *g["clip"])
+    np.testing.assert_allclose(r["lb"][0], _fr(v["lb"]), rtol=0, atol=1e-14)
+    np.testing.assert_allclose(r["ub"][0], _fr(v["ub"]), rtol=0, atol=1e-14)
+    assert r["codes"][0].tolist() == v["codes"]
+
+
+@pytest.mark.parametrize("make", NETS)
+def test_reusecert_matrix_form_agrees(make):
+    w = make()
+    r = orc.reusecert(w.layers, w.centers, w.eps, w.clip_lo, w.clip_hi)
+    lb, ub, codes = mat.reusecert_matrix(w.layers, w.centers, w.eps, w.clip_lo, w.clip_hi)
+    np.testing.assert_allclose(r["lb"], lb, rtol=1e-10, atol=1e-10)
+    np.testing.assert_allclose(r["ub"], ub, rtol=1e-10, atol=1e-10)
+    assert np.array_equal(r["codes"], codes)
+
+
+def test_reusecert_equals_deeppoly_up_to_the_second_affine_layer_and_when_stable():
+    """One traversal round is all DeepPoly does at the second affine layer, so the first two layers agree;
+    with every neuron stable both are the exact range of the linear map."""
+    w = wl.small_fc([10, 24, 24, 24, 5], batch=3, eps=0.05, seed=21)
+    a = orc.deeppoly(w.layers, w.centers, w.eps, w.clip_lo, w.clip_hi)
+    r = orc.reusecert(w.layers, w.centers, w.eps, w.clip_lo, w.clip_hi)
+    np.testing.assert_allclose(r["lb"][:, :48], a["lb"][:, :48], rtol=1e-12, atol=1e-12)
+    np.testing.assert_allclose(r["ub"][:, :48], a["ub"][:, :48], rtol=1e-12, atol=1e-12)
+    assert not np.allclose(r["lb"][:, 48:], a["lb"][:, 48:], rtol=1e-6, atol=1e-6)   # later layers differ
+    s = wl.small_fc([6, 10, 10, 10, 3], batch=2, eps=0.0005, seed=33, b_sigma=5.0)
+    a = orc.deeppoly(s.layers, s.centers, s.eps, s.clip_lo, s.clip_hi)
+    r = orc.reusecert(s.layers, s.centers, s.eps, s.clip_lo, s.clip_hi)
+    assert (a["codes"] <= 1).all()
+    np.testing.assert_allclose(r["lb"], a["lb"], rtol=1e-11, atol=1e-11)
+    np.testing.assert_allclose(r["ub"], a["ub"], rtol=1e-11, atol=1e-11)
+
+
+@pytest.mark.parametrize("make", NETS[:2])
+def test_reusecert_is_sound_on_samples(make):
+    w = make()
+    r = orc.reusecert(w.layers, w.centers, w.eps, w.clip_lo, w.clip_hi)
+    L0, U0 = mat.box(w.centers, w.eps, w.clip_lo, w.clip_hi)
+    assert (r["lb"] <= r["ub"] + 1e-12).all()
+    for b in range(w.batch):
+        z = mat.forward_preactivations(w.layers, _samples(L0[b], U0[b], 50_000, seed=b))
+        assert (z.min(axis=0) >= r["lb"][b] - 1e-9 * (1 + np.abs(r["lb"][b]))).all()
+        assert (z.max(axis=0) <= r["ub"][b] + 1e-9 * (1 + np.abs(r["ub"][b]))).all()
