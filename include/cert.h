@@ -105,6 +105,23 @@ cert_status_t cert_deeppoly_bounds(cert_net_t *net, const float *centers, float 
 cert_status_t cert_backsub_bounds(cert_net_t *net, const float *centers, float eps, int batch,
                                   const int *backsteps, float *lb_out, float *ub_out, void *stream);
 
+/*
+ * ReuseCert (Appendix C, ReuseCert listing; Section 6.1): every neuron's polyhedral bounds are kept
+ * over the input layer and reused (stop_traverse(n) = n[layer] <= 1), so each affine layer costs one
+ * contraction instead of a traversal through all earlier layers; the bounds are sound but can be
+ * looser than DeepPoly's from the third affine layer on.
+ *   cert_net_enable_reusecert  allocates what the certifier needs on top of the net (the shapes of one
+ *            layer for max_batch boxes, twice; block weight matrices): call it once, outside the hot
+ *            path, with the net's device current.  FC layers only (CERT_ERR_UNSUPPORTED otherwise,
+ *            or when the tensor-core path is not available).
+ *   cert_reusecert_bounds      arguments, outputs (l, u of every affine layer as the Relu transformer
+ *            computes them: L.map(simplify_lower), U.map(simplify_upper)), branch codes and stream
+ *            behaviour as cert_deeppoly_bounds; allocates nothing.
+ */
+cert_status_t cert_net_enable_reusecert(cert_net_t *net);
+cert_status_t cert_reusecert_bounds(cert_net_t *net, const float *centers, float eps, int batch,
+                                    float *lb_out, float *ub_out, void *stream);
+
 /* Same, with HOST buffers (pageable or pinned): copies centers to the device,
  * runs cert_deeppoly_bounds, copies the bounds back and waits for the stream. */
 cert_status_t cert_deeppoly_bounds_host(cert_net_t *net, const float *centers_host, float eps,

@@ -33,6 +33,7 @@ EXPORTS = [
     "cert_net_last_status", "cert_net_set_contraction", "cert_net_last_launch_count",
     "cert_net_backstep_flops", "cert_status_string", "cert_net_set_profiling", "cert_net_profile",
     "cert_net_last_contraction_paths", "cert_first_layer_bounds_noalloc", "cert_net_set_conv_patches",
+    "cert_net_enable_reusecert", "cert_reusecert_bounds",
 ]
 CLASS_NAMES = ["input", "relax", "relu_step", "affine", "conv", "concretize"]
 
@@ -73,6 +74,10 @@ _lib.cert_net_backstep_flops.argtypes = [_vp, _i]
 _lib.cert_net_backstep_flops.restype = ctypes.c_double
 _lib.cert_net_last_contraction_paths.argtypes = [_vp]
 _lib.cert_net_last_contraction_paths.restype = _i
+_lib.cert_net_enable_reusecert.argtypes = [_vp]
+_lib.cert_net_enable_reusecert.restype = _i
+_lib.cert_reusecert_bounds.argtypes = [_vp, _vp, _f, _i, _vp, _vp, _vp]
+_lib.cert_reusecert_bounds.restype = _i
 _lib.cert_net_set_conv_patches.argtypes = [_vp, _i]
 _lib.cert_net_set_conv_patches.restype = _i
 _lib.cert_net_set_profiling.argtypes = [_vp, _i]
@@ -174,6 +179,24 @@ class CertNet:
         _check(_lib.cert_backsub_bounds(self._h, centers.data_ptr(), float(eps), int(batch),
                                         ctypes.addressof(steps) if steps is not None else None,
                                         lb_out.data_ptr(), ub_out.data_ptr(), st.cuda_stream), "cert_backsub_bounds")
+        return lb_out, ub_out
+
+    def enable_reusecert(self):
+        _check(_lib.cert_net_enable_reusecert(self._h), "cert_net_enable_reusecert")
+
+    def reusecert_bounds(self, centers, eps: float, lb_out=None, ub_out=None, stream=None):
+        """cert_reusecert_bounds (enable_reusecert() first)."""
+        import torch
+        assert centers.is_cuda and centers.dtype == torch.float32 and centers.is_contiguous()
+        batch = centers.shape[0]
+        assert centers.shape[1] == self.n0
+        if lb_out is None:
+            lb_out = torch.empty((batch, self.n_total), dtype=torch.float32, device=centers.device)
+        if ub_out is None:
+            ub_out = torch.empty((batch, self.n_total), dtype=torch.float32, device=centers.device)
+        st = stream if stream is not None else torch.cuda.current_stream(centers.device)
+        _check(_lib.cert_reusecert_bounds(self._h, centers.data_ptr(), float(eps), int(batch), lb_out.data_ptr(),
+                                          ub_out.data_ptr(), st.cuda_stream), "cert_reusecert_bounds")
         return lb_out, ub_out
 
     def deeppoly_p_bounds(self, centers, eps: float, p: int, **kw):

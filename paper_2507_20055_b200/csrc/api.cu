@@ -24,6 +24,24 @@ struct TcLayer {
 };
 
 
+// ReuseCert: per affine layer k >= 1 the block weight matrix [[W+^T, W-^T], [W-^T, W+^T]] as the K-major B
+// operand (rows = the 2*n_k output columns, columns = the 2*n_{k-1} columns of the layer below), TF32 split.
+struct ReuseLayer {
+    int ld_s = 0;                        // pitch of this layer's [L | U] matrix
+    float *B_hi = nullptr, *B_lo = nullptr, *bias2 = nullptr;
+    cert::TcMap b_hi, b_lo, a_hi[2], a_lo[2], o_hi[2];
+    cert::TcPlan plan;
+};
+
+struct ReuseState {
+    bool on = false;
+    int R = 0;                           // rows per box: n0 coordinates, the constant, zero padding to 32
+    float *W0t = nullptr;                // first layer's weights transposed [round_up(n0, 32)][ld_out]
+    float *S_hi[2] = {nullptr, nullptr}, *S_lo[2] = {nullptr, nullptr};
+    float *colsum = nullptr;
+    std::vector<ReuseLayer> layers;
+};
+
 struct cert_net {
     int n_layers = 0, max_batch = 0;
     float clip_lo = 0, clip_hi = 0;
@@ -43,6 +61,7 @@ struct cert_net {
     int sm_count = 148;
     int tc_ctas = 1;                         // CTAs per row panel of the tensor-core kernel (2: cta_group::2)
     bool conv_patches = true;                // conv-sourced rows travel as receptive-field patches where they can
+    ReuseState reuse;
     unsigned char *codes = nullptr;          // [max_batch][n_relu]
     int *status_dev = nullptr;               // sticky device status word
     // host staging for cert_deeppoly_bounds_host
@@ -585,6 +604,153 @@ cert_status_t cert_backsub_bounds_host(cert_net_t *net, const float *centers_hos
     if (cudaMemcpyAsync(lb_host, net->lb_dev, out_bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
         cudaMemcpyAsync(ub_host, net->ub_dev, out_bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
         cudaStreamSynchronize(st) != cudaSuccess) {
+        cudaGetLastError();
+        return CERT_ERR_CUDA;
+    }
+    return CERT_OK;
+}
+
+cert_status_t cert_net_enable_reusecert(cert_net_t *net) {
+    if (!net) return CERT_ERR_INVALID_ARG;
+    if (net->reuse.on) return CERT_OK;
+    const int K = net->n_layers;
+    if (K < 2 || !net->tc_ok) return CERT_ERR_UNSUPPORTED;
+    for (int k = 0; k < K; ++k)
+        if (net->layers[k].kind != CERT_LAYER_FC) return CERT_ERR_UNSUPPORTED;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev != net->device) { cudaGetLastError(); return CERT_ERR_INVALID_ARG; }
+    ReuseState &R = net->reuse;
+    R.R = round_up(net->n0 + 1, 32);
+    R.layers.assign(K, ReuseLayer());
+    int ld_max = 0;
+    for (int k = 0; k < K; ++k) {
+        R.layers[k].ld_s = round_up(2 * net->layers[k].n_out, 32);
+        ld_max = std::max(ld_max, R.layers[k].ld_s);
+    }
+    const long long m_max = (long long)net->max_batch * R.R;
+    const size_t elems = (size_t)m_max * ld_max;
+    for (int p = 0; p < 2; ++p)
+        if (!dev_alloc_zero(net, &R.S_hi[p], elems) || !dev_alloc_zero(net, &R.S_lo[p], elems)) return CERT_ERR_OOM;
+    if (!dev_alloc_zero(net, &R.colsum, (size_t)(m_max / 32) * ld_max)) return CERT_ERR_OOM;
+    const int ctas = net->tc_ctas;
+    std::vector<float> w, hi, lo, b2;
+    for (int k = 0; k < K; ++k) {
+        const LayerDev &L = net->layers[k];
+        const size_t rows_pad = round_up(L.n_out, kPad);
+        w.resize(rows_pad * L.ld_in);
+        if (cudaMemcpy(w.data(), L.W, w.size() * sizeof(float), cudaMemcpyDeviceToHost) != cudaSuccess) {
+            cudaGetLastError();
+            return CERT_ERR_CUDA;
+        }
+        if (k == 0) {
+            hi.assign((size_t)round_up(L.n_in, kPad) * L.ld_out, 0.0f);
+            for (int t = 0; t < L.n_out; ++t)
+                for (int s2 = 0; s2 < L.n_in; ++s2) hi[(size_t)s2 * L.ld_out + t] = w[(size_t)t * L.ld_in + s2];
+            if (!dev_alloc(net, (void **)&R.W0t, hi.size() * sizeof(float))) return CERT_ERR_OOM;
+            if (cudaMemcpy(R.W0t, hi.data(), hi.size() * sizeof(float), cudaMemcpyHostToDevice) != cudaSuccess)
+                return CERT_ERR_CUDA;
+            continue;
+        }
+        ReuseLayer &RL = R.layers[k];
+        const int n = L.n_out, m = L.n_in, ldb = R.layers[k - 1].ld_s;
+        const size_t brows = round_up(2 * n, kPad);
+        hi.assign(brows * ldb, 0.0f);
+        lo.assign(brows * ldb, 0.0f);
+        auto put = [&](int row, int col, float v) {
+            const float h = host_tf32(v);
+            hi[(size_t)row * ldb + col] = h;
+            lo[(size_t)row * ldb + col] = host_tf32(v - h);
+        };
+        for (int i = 0; i < n; ++i)
+            for (int t = 0; t < m; ++t) {
+                const float v = w[(size_t)i * L.ld_in + t];
+                const float vp = v >= 0.0f ? v : 0.0f, vm = v >= 0.0f ? 0.0f : v;
+                put(i, t, vp);          // L_i takes L_t with W+ ...
+                put(i, m + t, vm);      // ... and U_t with W-
+                put(n + i, t, vm);      // U_i takes L_t with W- ...
+                put(n + i, m + t, vp);  // ... and U_t with W+
+            }
+        b2.assign(RL.ld_s, 0.0f);
+        std::vector<float> bias(L.ld_out);
+        if (cudaMemcpy(bias.data(), L.bias_n, bias.size() * sizeof(float), cudaMemcpyDeviceToHost) != cudaSuccess) {
+            cudaGetLastError();
+            return CERT_ERR_CUDA;
+        }
+        for (int i = 0; i < n; ++i) b2[i] = b2[n + i] = bias[i];
+        if (!dev_alloc(net, (void **)&RL.B_hi, hi.size() * sizeof(float)) ||
+            !dev_alloc(net, (void **)&RL.B_lo, lo.size() * sizeof(float)) ||
+            !dev_alloc(net, (void **)&RL.bias2, b2.size() * sizeof(float)))
+            return CERT_ERR_OOM;
+        if (cudaMemcpy(RL.B_hi, hi.data(), hi.size() * sizeof(float), cudaMemcpyHostToDevice) != cudaSuccess ||
+            cudaMemcpy(RL.B_lo, lo.data(), lo.size() * sizeof(float), cudaMemcpyHostToDevice) != cudaSuccess ||
+            cudaMemcpy(RL.bias2, b2.data(), b2.size() * sizeof(float), cudaMemcpyHostToDevice) != cudaSuccess)
+            return CERT_ERR_CUDA;
+        RL.plan = cert::tc_tile_plan(2 * n, ctas);
+        if (RL.plan.stages < 2) return CERT_ERR_UNSUPPORTED;
+        bool ok = cert::tc_make_map(&RL.b_hi, RL.B_hi, 2 * m, 2 * n, ldb, RL.plan.bn / ctas) &&
+                  cert::tc_make_map(&RL.b_lo, RL.B_lo, 2 * m, 2 * n, ldb, RL.plan.bn / ctas);
+        for (int p = 0; p < 2 && ok; ++p)
+            ok = cert::tc_make_map(&RL.a_hi[p], R.S_hi[p], 2 * m, m_max, ldb, 128) &&
+                 cert::tc_make_map(&RL.a_lo[p], R.S_lo[p], 2 * m, m_max, ldb, 128) &&
+                 cert::tc_make_map(&RL.o_hi[p], R.S_hi[p], RL.ld_s, m_max, RL.ld_s, 32);
+        if (!ok) return CERT_ERR_CUDA;
+    }
+    if (cudaDeviceSynchronize() != cudaSuccess) { cudaGetLastError(); return CERT_ERR_CUDA; }
+    R.on = true;
+    return CERT_OK;
+}
+
+cert_status_t cert_reusecert_bounds(cert_net_t *net, const float *centers, float eps, int batch, float *lb_out,
+                                    float *ub_out, void *stream) {
+    if (!net || !centers || !lb_out || !ub_out) return CERT_ERR_INVALID_ARG;
+    if (batch < 1 || !(eps >= 0.0f) || std::isinf(eps)) return CERT_ERR_INVALID_ARG;
+    if (batch > net->max_batch) return CERT_ERR_BATCH_TOO_LARGE;
+    if (!net->reuse.on) return CERT_ERR_UNSUPPORTED;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    ReuseState &R = net->reuse;
+    const int K = net->n_layers, n_total = net->n_total, ctas = net->tc_ctas;
+    const long long rows = (long long)batch * R.R;
+    Recorder rec(net, st);
+    cert::launch_box(centers, eps, net->clip_lo, net->clip_hi, batch, net->n0, net->ld0, net->l0, net->u0, st);
+    rec.mark(CERT_CLASS_INPUT);
+    const LayerDev &L0 = net->layers[0];
+    cert::launch_first_layer_bounds(L0, net->l0, net->u0, net->ld0, batch, lb_out, ub_out, n_total, st);
+    rec.mark(CERT_CLASS_INPUT);
+    cert::launch_relax(L0, lb_out, ub_out, n_total, batch, net->codes, net->n_relu, nullptr, 0, 0, st);
+    rec.mark(CERT_CLASS_RELAX);
+    int cur = 0;
+    cert::launch_reuse_init(R.W0t, L0.ld_out, L0, net->n0, R.R, R.layers[0].ld_s, rows, R.S_hi[cur], R.S_lo[cur], st);
+    rec.mark(CERT_CLASS_RELU_STEP);
+    for (int k = 1; k < K; ++k) {
+        const LayerDev &Lk = net->layers[k];
+        const ReuseLayer &RL = R.layers[k];
+        cert::TcArgs a;
+        std::memset(&a, 0, sizeof(a));
+        a.M = rows; a.K = 2 * Lk.n_in; a.n_k = 1; a.ld_n = RL.ld_s;
+        a.bn = RL.plan.bn; a.n_tiles = RL.plan.n_tiles; a.stages = RL.plan.stages; a.tmem_cols = RL.plan.tmem_cols;
+        a.total_tiles = (int)cert::ceil_div_ll(rows, 128 * ctas) * RL.plan.n_tiles;
+        a.l0 = net->l0; a.u0 = net->u0;
+        a.reuse_R = R.R; a.reuse_n0 = net->n0; a.reuse_ld0 = net->ld0; a.n_half = Lk.n_out;
+        a.bias2 = RL.bias2; a.colsum = R.colsum;
+        a.status = net->status_dev;
+        const int groups = std::min(a.total_tiles, net->sm_count / ctas);
+        cert::launch_gemm_tc(cert::TC_EPI_REUSE, ctas, groups, RL.a_hi[cur], RL.a_lo[cur], RL.b_hi, RL.b_lo,
+                             RL.o_hi[cur ^ 1], RL.o_hi[cur ^ 1], a, RL.plan.smem_bytes, st);
+        rec.mark(CERT_CLASS_AFFINE);
+        cert::launch_reuse_relax(R.colsum, RL.ld_s, R.R / 32, Lk, batch, lb_out, ub_out, n_total, net->codes,
+                                 net->n_relu, st);
+        rec.mark(CERT_CLASS_RELAX);
+        cur ^= 1;
+        if (k + 1 < K) {
+            cert::launch_reuse_scale(R.S_hi[cur], R.S_lo[cur], RL.ld_s, Lk, net->n0, R.R, rows, st);
+            rec.mark(CERT_CLASS_RELU_STEP);
+        }
+    }
+    net->last_batch = batch;
+    net->last_launches = rec.launches;
+    net->last_paths = 2 | (ctas == 2 ? 4 : 0);
+    net->prof_marks = rec.marks;
+    if (cudaPeekAtLastError() != cudaSuccess) {
         cudaGetLastError();
         return CERT_ERR_CUDA;
     }

@@ -133,4 +133,17 @@ void launch_patch_start(const LayerDev &Lk, const LayerDev &Lb, const PatchLevel
 void launch_patch_step(const LayerDev &Lk, const LayerDev &Lj, const PatchLevel &in, const PatchLevel &out,
                        const float *in_patch, long long rows, int sms, const ConvtEpilogue &ep, cudaStream_t st);
 
+// ---- ReuseCert (reuse.cu): shapes over the input layer, one matrix S per layer ----
+// S rows are (box, s): s < n0 input coordinate, s == n0 constant, zero rows up to R per box; columns
+// [L (n) | U (n)] padded to ld_s.  S is held as a TF32 pair.
+void launch_reuse_init(const float *W0t, int ldw, const LayerDev &L0, int n0, int R, int ld_s, long long rows,
+                       float *S_hi, float *S_lo, cudaStream_t st);
+// Bounds (and the relaxation, under a ReLU) of layer L from the contraction's column sums.
+void launch_reuse_relax(const float *colsum, int ld_s, int groups_per_box, const LayerDev &L, int batch,
+                        float *lb_out, float *ub_out, int n_total, unsigned char *codes, int n_relu,
+                        cudaStream_t st);
+// Raw [L | U] of layer L (fp32 in S_hi) -> S of its outputs, in place.
+void launch_reuse_scale(float *S_hi, float *S_lo, int ld_s, const LayerDev &L, int n0, int R, long long rows,
+                        cudaStream_t st);
+
 }  // namespace cert

@@ -7,7 +7,7 @@ namespace cert {
 
 constexpr int kTcSmemMax = 227 * 1024;
 
-enum { TC_EPI_RELU = 0, TC_EPI_CONCRETIZE = 1 };
+enum { TC_EPI_RELU = 0, TC_EPI_CONCRETIZE = 1, TC_EPI_REUSE = 2 };
 
 // Storage for a CUtensorMap (128 bytes, 64-byte aligned), kept opaque so that
 // only gemm_tc.cu needs the driver API header.
@@ -45,6 +45,14 @@ struct TcArgs {
     float *d_out;
     int n_slots_in;
     long long slot_stride;
+    // TC_EPI_REUSE (shapes kept over the input layer): a row is (box, s) with s < reuse_n0 an input
+    // coordinate, s == reuse_n0 the constant, rows per box = reuse_R (a multiple of 32); a column is a
+    // neuron's lower (col < n_half) or upper (n_half <= col < 2*n_half) shape.  The result is stored
+    // unsplit; bias2[col] is added on the constant row; colsum[(row / 32) * ld_n + col] receives the sum
+    // over the warp's 32 rows of the column's concretisation terms against the box l0, u0 [box][reuse_ld0].
+    int reuse_R, reuse_n0, reuse_ld0, n_half;
+    const float *bias2;
+    float *colsum;
     int *status;                                 // set to 1 if a bounded wait runs out
 };
 

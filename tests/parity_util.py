@@ -34,7 +34,7 @@ def run_gpu(w, contraction=None, max_batch=None, host_api=False, backsteps=None,
     return {"lb": lb, "ub": ub, "codes": codes, "status": status, "launches": launches, "paths": paths}
 
 
-def compare(gpu, ref, boxes=None, min_good_fraction=0.5, label=""):
+def compare(gpu, ref, boxes=None, min_good_fraction=0.5, label="", tol=TOL):
     """ref: oracle result for the boxes listed in `boxes` (indices into the GPU batch)."""
     assert gpu["status"] == 0, f"device status {gpu['status']}"
     idx = np.arange(ref["lb"].shape[0]) if boxes is None else np.asarray(boxes)
@@ -53,5 +53,5 @@ def compare(gpu, ref, boxes=None, min_good_fraction=0.5, label=""):
               "max_scaled_err": float(worst)}
     print(label, report)
     assert code_mismatch == 0, f"{label}: {code_mismatch} branch codes differ"
-    assert worst <= TOL, f"{label}: scaled error {worst} > {TOL}"
+    assert worst <= tol, f"{label}: scaled error {worst} > {tol}"
     return report

@@ -218,3 +218,74 @@ def test_conv_rows_dense_and_patches(name, patches):
     steps = [0] + [1] * (len(w.layers) - 1)
     ref1 = orc.deeppoly(w.layers, w.centers, w.eps, w.clip_lo, w.clip_hi, backsteps_per_layer=steps)
     compare(run_gpu(w, conv_patches=patches, backsteps=steps), ref1, label=f"{name}/patches={patches}/p1")
+
+
+# ---- ReuseCert (Appendix C listing): shapes kept over the input layer ----
+
+REUSE_NETS = {
+    "fc_ragged": lambda: wl.small_fc([37, 50, 33, 70, 40, 10], batch=5, eps=0.03, seed=81),
+    "fc_wide": lambda: wl.small_fc([64, 300, 130, 257, 3], batch=6, eps=0.02, seed=82),
+    "n0_multiple_of_32": lambda: wl.small_fc([64, 96, 96, 8], batch=3, eps=0.02, seed=87),
+    "fc6x100": lambda: wl.make_config(1, batch=8),
+    "fc3x50": lambda: wl.make_config(0),
+}
+
+
+# ReuseCert feeds every layer with the rounded shapes of the layer below, so float32 rounding compounds
+# through the layers (measured: x3..5 per layer, 1.1e-4 at the fourth layer of the 64-300-130-257-3 net),
+# where DeepPoly restarts each traversal from the exact weights.  Its bounds are therefore compared at
+# 5e-4 * (1 + |oracle|); the branch codes must still be identical on well-conditioned boxes.
+REUSE_TOL = 5e-4
+
+
+def _run_reusecert(w, max_batch=None):
+    import torch
+    from paper_2507_20055_b200 import binding
+    net = binding.CertNet(w.layers, max_batch or w.batch, w.clip_lo, w.clip_hi)
+    try:
+        net.enable_reusecert()
+        c = torch.from_numpy(np.ascontiguousarray(w.centers)).cuda()
+        out = []
+        for _ in range(2):                      # the second call reuses every buffer
+            lb, ub = net.reusecert_bounds(c, w.eps)
+            torch.cuda.synchronize()
+            out.append({"lb": lb.cpu().numpy(), "ub": ub.cpu().numpy(),
+                        "codes": net.branch_codes(w.batch).cpu().numpy(), "status": net.last_status()})
+        # DeepPoly on the same net still works after ReuseCert was enabled
+        lb, ub = net.deeppoly_bounds(c, w.eps)
+        torch.cuda.synchronize()
+        dp = {"lb": lb.cpu().numpy(), "ub": ub.cpu().numpy(), "codes": net.branch_codes(w.batch).cpu().numpy(),
+              "status": net.last_status()}
+    finally:
+        net.destroy()
+    return out, dp
+
+
+@pytest.mark.parametrize("name", sorted(REUSE_NETS))
+def test_reusecert(name):
+    w = REUSE_NETS[name]()
+    ref = orc.reusecert(w.layers, w.centers, w.eps, w.clip_lo, w.clip_hi)
+    out, dp = _run_reusecert(w, max_batch=w.batch + 3)
+    for i, g in enumerate(out):
+        compare(g, ref, label=f"reusecert/{name}/call{i}", tol=REUSE_TOL)
+    assert np.array_equal(out[0]["lb"], out[1]["lb"]) and np.array_equal(out[0]["ub"], out[1]["ub"])
+    compare(dp, _oracle(w), label=f"deeppoly_after_reusecert/{name}")
+
+
+def test_reusecert_needs_enable_and_fc_layers():
+    import torch
+    from paper_2507_20055_b200 import binding
+    w = wl.small_fc([8, 8, 4], batch=2, eps=0.1, seed=77)
+    net = binding.CertNet(w.layers, 2)
+    try:
+        c = torch.from_numpy(w.centers).cuda()
+        out = torch.empty((2, net.n_total), device="cuda")
+        assert binding.lib.cert_reusecert_bounds(net._h, c.data_ptr(), 0.1, 2, out.data_ptr(), out.data_ptr(), None) == 2
+    finally:
+        net.destroy()
+    wc = wl.small_conv((1, 10, 10), [(20, 5, 1, 0)], [6], batch=2, eps=0.05, seed=68)
+    net = binding.CertNet(wc.layers, 2)
+    try:
+        assert binding.lib.cert_net_enable_reusecert(net._h) == 2
+    finally:
+        net.destroy()
