@@ -94,14 +94,17 @@ class ClockSampler:
                 "sm_max_mhz": max(mx) if mx else None, "samples": len(sm), "reasons": sorted(reasons)}
 
 
-def oracle_sample(w, n_boxes, threads=None, backsteps=None):
+def oracle_sample(w, n_boxes, threads=None, backsteps=None, certifier="deeppoly"):
     """Times the oracle, as it stands, on the first n_boxes boxes of the workload."""
     from oracle import deeppoly_oracle as orc
     orc.build()
     cores = threads or orc.max_threads()
     c = w.centers[:n_boxes]
     t0 = time.perf_counter()
-    orc.deeppoly(w.layers, c, w.eps, w.clip_lo, w.clip_hi, n_threads=cores, backsteps_per_layer=backsteps)
+    if certifier == "reusecert":
+        orc.reusecert(w.layers, c, w.eps, w.clip_lo, w.clip_hi, n_threads=cores)
+    else:
+        orc.deeppoly(w.layers, c, w.eps, w.clip_lo, w.clip_hi, n_threads=cores, backsteps_per_layer=backsteps)
     dt = time.perf_counter() - t0
     return {"value": n_boxes / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
             "sample": f"first {n_boxes} of {w.batch} boxes of {w.name}, one box per thread, {dt:.1f} s wall"}, dt
@@ -109,7 +112,7 @@ def oracle_sample(w, n_boxes, threads=None, backsteps=None):
 
 def certifier_steps(name, n_layers):
     """Traversal depth per affine layer (None = to the input everywhere) for a certifier name."""
-    if name == "deeppoly":
+    if name in ("deeppoly", "reusecert"):
         return None
     if name == "ibp":
         return [0] * n_layers
@@ -176,7 +179,7 @@ def run_reference(args, w):
         n_boxes = max(1, min(cores, 16) // 2)     # about 11 s per box per core
     times = []
     for i in range(args.warmup + args.steps):
-        base, dt = oracle_sample(w, n_boxes, backsteps=args.backsteps)
+        base, dt = oracle_sample(w, n_boxes, backsteps=args.backsteps, certifier=args.certifier)
         if i >= args.warmup:
             times.append(dt)
     ms = 1000.0 * sum(times) / len(times)
@@ -203,7 +206,7 @@ def main():
     ap.add_argument("--batch", type=int, default=None)
     ap.add_argument("--contraction", default="auto", choices=["auto", "ffma", "tc"])
     ap.add_argument("--certifier", default="deeppoly",
-                    help="deeppoly | ibp | crown_ibp | deeppoly_pN (N back-substitution steps per layer)")
+                    help="deeppoly | ibp | crown_ibp | deeppoly_pN (N back-substitution steps per layer) | reusecert")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--ref-boxes", type=int, default=None)
     args = ap.parse_args()
@@ -255,8 +258,15 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
+    reuse = args.certifier == "reusecert"
+    if reuse:
+        net.enable_reusecert()
+
     def step_device():
-        net.backsub_bounds(centers, w.eps, args.backsteps, lb, ub, stream=stream)
+        if reuse:
+            net.reusecert_bounds(centers, w.eps, lb, ub, stream=stream)
+        else:
+            net.backsub_bounds(centers, w.eps, args.backsteps, lb, ub, stream=stream)
 
     # ---- device-resident timing: K steps, each bracketed by events on the launching stream,
     #      L2 flushed between steps outside the bracket ----
@@ -302,13 +312,20 @@ def main():
     lb_pin = torch.empty((B, net.n_total), dtype=torch.float32).pin_memory()
     ub_pin = torch.empty((B, net.n_total), dtype=torch.float32).pin_memory()
     c_np, lb_np, ub_np = centers_pin.numpy(), lb_pin.numpy(), ub_pin.numpy()
+
+    def step_host():
+        if reuse:
+            net.reusecert_bounds_host(c_np, w.eps, lb_np, ub_np, stream.cuda_stream)
+        else:
+            net.deeppoly_bounds_host(c_np, w.eps, lb_np, ub_np, stream.cuda_stream, args.backsteps)
+
     for _ in range(2):
-        net.deeppoly_bounds_host(c_np, w.eps, lb_np, ub_np, stream.cuda_stream, args.backsteps)
+        step_host()
     barrier()
     e2e_steps = max(3, min(args.steps, 10))
     t0 = time.perf_counter()
     for _ in range(e2e_steps):
-        net.deeppoly_bounds_host(c_np, w.eps, lb_np, ub_np, stream.cuda_stream, args.backsteps)   # returns after the D2H copy
+        step_host()   # returns after the D2H copy
     torch.cuda.synchronize()
     e2e_s = time.perf_counter() - t0
 
@@ -324,9 +341,15 @@ def main():
         peaks = load_peaks()
         used_patches = bool(net.last_contraction_paths() & 8)
         fl = backstep_flops_by_class(w.layers, B, args.backsteps, patches=used_patches)
-        flops_call = fl["affine"] + fl["conv"]
         fl_dense = backstep_flops_by_class(w.layers, B, args.backsteps, patches=False)
-        if args.backsteps is None:      # the library's own count (dense maps) must agree
+        if reuse:
+            # one contraction per affine layer k >= 1: (n0 + 1) rows per box (coefficients and the constant),
+            # 2 n_{k-1} columns of shapes below against the 2 n_k shapes of the layer
+            n0 = w.layers[0].n_in
+            fl = {"affine": sum(2.0 * B * (n0 + 1) * (2 * l.n_in) * (2 * l.n_out) for l in w.layers[1:]), "conv": 0.0}
+            fl_dense = fl
+        flops_call = fl["affine"] + fl["conv"]
+        if args.backsteps is None and not reuse:      # the library's own count (dense maps) must agree
             lib_count = net.backstep_flops(B)
             assert abs(fl_dense["affine"] + fl_dense["conv"] - lib_count) <= 1e-6 * lib_count
         # the dominant kernel class: FC back-steps (tensor cores unless --contraction ffma) or conv back-steps (FMA units)
@@ -373,7 +396,7 @@ def main():
             from oracle import deeppoly_oracle as orc
             orc.build()
             n_boxes = min(n_boxes, B) if args.config != 4 else min(B, orc.max_threads(), 16)
-            out["cpu_baseline"], _ = oracle_sample(w, n_boxes, backsteps=args.backsteps)
+            out["cpu_baseline"], _ = oracle_sample(w, n_boxes, backsteps=args.backsteps, certifier=args.certifier)
         print(json.dumps(out))
     net.destroy()
     if world > 1:

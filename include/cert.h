@@ -121,6 +121,9 @@ cert_status_t cert_backsub_bounds(cert_net_t *net, const float *centers, float e
 cert_status_t cert_net_enable_reusecert(cert_net_t *net);
 cert_status_t cert_reusecert_bounds(cert_net_t *net, const float *centers, float eps, int batch,
                                     float *lb_out, float *ub_out, void *stream);
+/* The same with HOST buffers, as cert_deeppoly_bounds_host. */
+cert_status_t cert_reusecert_bounds_host(cert_net_t *net, const float *centers_host, float eps, int batch,
+                                         float *lb_host, float *ub_host, void *stream);
 
 /* Same, with HOST buffers (pageable or pinned): copies centers to the device,
  * runs cert_deeppoly_bounds, copies the bounds back and waits for the stream. */

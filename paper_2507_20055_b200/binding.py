@@ -33,7 +33,7 @@ EXPORTS = [
     "cert_net_last_status", "cert_net_set_contraction", "cert_net_last_launch_count",
     "cert_net_backstep_flops", "cert_status_string", "cert_net_set_profiling", "cert_net_profile",
     "cert_net_last_contraction_paths", "cert_first_layer_bounds_noalloc", "cert_net_set_conv_patches",
-    "cert_net_enable_reusecert", "cert_reusecert_bounds",
+    "cert_net_enable_reusecert", "cert_reusecert_bounds", "cert_reusecert_bounds_host",
 ]
 CLASS_NAMES = ["input", "relax", "relu_step", "affine", "conv", "concretize"]
 
@@ -78,6 +78,8 @@ _lib.cert_net_enable_reusecert.argtypes = [_vp]
 _lib.cert_net_enable_reusecert.restype = _i
 _lib.cert_reusecert_bounds.argtypes = [_vp, _vp, _f, _i, _vp, _vp, _vp]
 _lib.cert_reusecert_bounds.restype = _i
+_lib.cert_reusecert_bounds_host.argtypes = [_vp, _vp, _f, _i, _vp, _vp, _vp]
+_lib.cert_reusecert_bounds_host.restype = _i
 _lib.cert_net_set_conv_patches.argtypes = [_vp, _i]
 _lib.cert_net_set_conv_patches.restype = _i
 _lib.cert_net_set_profiling.argtypes = [_vp, _i]
@@ -198,6 +200,14 @@ class CertNet:
         _check(_lib.cert_reusecert_bounds(self._h, centers.data_ptr(), float(eps), int(batch), lb_out.data_ptr(),
                                           ub_out.data_ptr(), st.cuda_stream), "cert_reusecert_bounds")
         return lb_out, ub_out
+
+    def reusecert_bounds_host(self, centers: np.ndarray, eps: float, lb: np.ndarray, ub: np.ndarray,
+                              stream_ptr: int = 0):
+        centers = np.ascontiguousarray(centers, dtype=np.float32)
+        _check(_lib.cert_reusecert_bounds_host(self._h, centers.ctypes.data, float(eps), centers.shape[0],
+                                               lb.ctypes.data, ub.ctypes.data, stream_ptr),
+               "cert_reusecert_bounds_host")
+        return lb, ub
 
     def deeppoly_p_bounds(self, centers, eps: float, p: int, **kw):
         return self.backsub_bounds(centers, eps, [int(p)] * self.n_layers, **kw)

@@ -757,6 +757,29 @@ cert_status_t cert_reusecert_bounds(cert_net_t *net, const float *centers, float
     return CERT_OK;
 }
 
+cert_status_t cert_reusecert_bounds_host(cert_net_t *net, const float *centers_host, float eps, int batch,
+                                         float *lb_host, float *ub_host, void *stream) {
+    if (!net || !centers_host || !lb_host || !ub_host) return CERT_ERR_INVALID_ARG;
+    if (batch < 1) return CERT_ERR_INVALID_ARG;
+    if (batch > net->max_batch) return CERT_ERR_BATCH_TOO_LARGE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    size_t in_bytes = (size_t)batch * net->n0 * sizeof(float);
+    size_t out_bytes = (size_t)batch * net->n_total * sizeof(float);
+    if (cudaMemcpyAsync(net->centers_dev, centers_host, in_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) {
+        cudaGetLastError();
+        return CERT_ERR_CUDA;
+    }
+    cert_status_t s = cert_reusecert_bounds(net, net->centers_dev, eps, batch, net->lb_dev, net->ub_dev, stream);
+    if (s != CERT_OK) return s;
+    if (cudaMemcpyAsync(lb_host, net->lb_dev, out_bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+        cudaMemcpyAsync(ub_host, net->ub_dev, out_bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+        cudaStreamSynchronize(st) != cudaSuccess) {
+        cudaGetLastError();
+        return CERT_ERR_CUDA;
+    }
+    return CERT_OK;
+}
+
 cert_status_t cert_net_destroy(cert_net_t *net) {
     if (!net) return CERT_ERR_INVALID_ARG;
     cudaError_t e = cudaDeviceSynchronize();

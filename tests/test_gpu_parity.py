@@ -289,3 +289,25 @@ def test_reusecert_needs_enable_and_fc_layers():
         assert binding.lib.cert_net_enable_reusecert(net._h) == 2
     finally:
         net.destroy()
+
+
+def test_reusecert_config5_sampled_boxes():
+    """784 -> 1024 x 6 -> 10, 128 boxes on the GPU (the benchmark's launch configuration); the oracle bounds
+    a sample of boxes.  With 6144 ReLU neurons per box and ReuseCert's wider bounds most boxes have some neuron
+    whose sign test is within float32 noise of zero; those boxes are skipped as everywhere else, so more
+    boxes are sampled and a smaller share of them has to remain."""
+    import torch
+    from paper_2507_20055_b200 import binding
+    w = wl.make_config(4)
+    boxes = list(range(0, 128, 8))
+    ref = orc.reusecert(w.layers, w.centers[np.asarray(boxes)], w.eps, w.clip_lo, w.clip_hi)
+    net = binding.CertNet(w.layers, w.batch, w.clip_lo, w.clip_hi)
+    try:
+        net.enable_reusecert()
+        lb, ub = net.reusecert_bounds(torch.from_numpy(w.centers).cuda(), w.eps)
+        torch.cuda.synchronize()
+        g = {"lb": lb.cpu().numpy(), "ub": ub.cpu().numpy(), "codes": net.branch_codes(w.batch).cpu().numpy(),
+             "status": net.last_status()}
+    finally:
+        net.destroy()
+    compare(g, ref, boxes=boxes, label="reusecert/fc6x1024", tol=REUSE_TOL, min_good_fraction=0.1)
