@@ -204,7 +204,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", type=int, default=4, help="0..4: index into the benchmark configurations")
     ap.add_argument("--batch", type=int, default=None)
-    ap.add_argument("--contraction", default="auto", choices=["auto", "ffma", "tc"])
+    ap.add_argument("--contraction", default="auto", choices=["auto", "ffma", "tc", "tc16"],
+                    help="tc = tcgen05 3xTF32, tc16 = tcgen05 fp16 split (FC nets), ffma = FMA units")
     ap.add_argument("--certifier", default="deeppoly",
                     help="deeppoly | ibp | crown_ibp | deeppoly_pN (N back-substitution steps per layer) | reusecert")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -244,7 +245,8 @@ def main():
         assert w.batch == per_gpu
     B = w.batch
     net = binding.CertNet(w.layers, B, w.clip_lo, w.clip_hi)
-    mode = {"auto": binding.CONTRACTION_AUTO, "ffma": binding.CONTRACTION_FFMA, "tc": binding.CONTRACTION_TC3XTF32}
+    mode = {"auto": binding.CONTRACTION_AUTO, "ffma": binding.CONTRACTION_FFMA, "tc": binding.CONTRACTION_TC3XTF32,
+            "tc16": binding.CONTRACTION_TC3XFP16}
     net.set_contraction(mode[args.contraction])
     stream = torch.cuda.Stream()
     centers = torch.from_numpy(w.centers).cuda()
@@ -360,11 +362,13 @@ def main():
         ffma_peak = 148 * 128 * 2 * sm_max * 1e6 / 1e12
         # fp32-accurate work on the tensor cores costs three TF32 products per multiply-add;
         # TF32 dense peak = measured bf16 (sustained: the kernel runs inside a long step) x 1/2 (nominal ratio)
-        tc_peak = peaks["bf16_tflops_sustained"] * 0.5 / 3.0
+        used_fp16 = bool(net.last_contraction_paths() & 16)
+        # fp16 split: three fp16 products (bf16 rate) per multiply-add; TF32 split: three TF32 products (half that rate)
+        tc_peak = peaks["bf16_tflops_sustained"] * (1.0 if used_fp16 else 0.5) / 3.0
         used_tc = dom == "affine" and bool(net.last_contraction_paths() & 2)
         traffic, traffic_note = None, "no ncu capture for this workload / contraction mode"
         cap = NCU_TRAFFIC_BYTES_PER_ROW.get(w.name)
-        if cap and used_tc and (net.last_contraction_paths() & 4):
+        if cap and used_tc and (net.last_contraction_paths() & 4) and not used_fp16 and not reuse:
             rows_per_launch = 2.0 * B * max(l.n_out for l in w.layers[1:-1] or w.layers[1:])
             traffic = cap["bytes_per_row"] * rows_per_launch
             traffic_note = f"{cap['kernel']}: {cap['source']}"
@@ -377,7 +381,8 @@ def main():
                 "flops_per_step": fl[dom], "flops_per_step_all_backsteps": flops_call,
                 "flops_per_step_if_dense_maps": fl_dense[dom], "conv_rows_as_patches": used_patches,
                 "peak_source": peaks["source"],
-                "peak_note": ("bf16_tflops_sustained/2/3 (3xTF32)" if used_tc else "148 SM x 128 FMA x 2 x sm_max_mhz"),
+                "peak_note": (("bf16_tflops_sustained/3 (3xFP16)" if used_fp16 else "bf16_tflops_sustained/2/3 (3xTF32)")
+                              if used_tc else "148 SM x 128 FMA x 2 x sm_max_mhz"),
                 "class_ms_per_step": {k: v / args.steps for k, v in cls_ms.items()}}
         out = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,

@@ -30,7 +30,8 @@ typedef enum {
     CERT_ERR_OOM = 3,             /* device or host allocation failed                            */
     CERT_ERR_BATCH_TOO_LARGE = 4, /* batch > max_batch given at create                           */
     CERT_ERR_CUDA = 5,            /* a CUDA runtime or driver call failed                        */
-    CERT_ERR_TIMEOUT = 6          /* a bounded device-side wait ran out (see cert_net_last_status) */
+    CERT_ERR_TIMEOUT = 6,         /* a bounded device-side wait ran out (see cert_net_last_status) */
+    CERT_ERR_RANGE = 7            /* a coefficient left the fp16 range of CERT_CONTRACTION_TC3XFP16  */
 } cert_status_t;
 
 enum { CERT_LAYER_FC = 0, CERT_LAYER_CONV2D = 1 };
@@ -156,9 +157,10 @@ cert_status_t cert_net_branch_codes(cert_net_t *net, unsigned char *codes_out, v
 
 /*
  * Sticky device-side status.  Waits `stream`, then returns CERT_ERR_TIMEOUT
- * if any kernel of an earlier call on this net gave up a bounded wait (its
- * results are then invalid), CERT_ERR_CUDA if the stream reports an error,
- * else CERT_OK.  Clears the flag.
+ * if any kernel of an earlier call on this net gave up a bounded wait,
+ * CERT_ERR_RANGE if a coefficient left the fp16 range in TC3XFP16 mode (the
+ * results are invalid in both cases), CERT_ERR_CUDA if the stream reports an
+ * error, else CERT_OK.  Clears the flag.
  */
 cert_status_t cert_net_last_status(cert_net_t *net, void *stream);
 
@@ -168,14 +170,22 @@ cert_status_t cert_net_last_status(cert_net_t *net, void *stream);
  *   FFMA:    fp32 FMA units, unfused ReLU step and concretisation kernels.
  *   TC3XTF32: tcgen05 tensor cores with a 3-term TF32 split (fp32-accurate),
  *            ReLU back-step and concretisation fused into the epilogue.
+ *   TC3XFP16: the same kernel structure with an fp16 split (x = hi + 2^-11 lo, three fp16
+ *            products per multiply-add, exact in the fp32 accumulators): the accuracy of TC3XTF32 at
+ *            twice the tensor-core rate and half the operand bytes, for nets of FC layers only and
+ *            coefficients below 65504 in magnitude (beyond that cert_net_last_status reports
+ *            CERT_ERR_RANGE and the results are invalid; values under 6.1e-5 are held to 1.5e-11
+ *            absolute instead of 2^-22 relative).  Never chosen by AUTO.
  * Conv back-steps always run on the FMA units, with the same fusions.
  * (The environment variable CERT_TC_CTAS=1, read at create, keeps the
  * tensor-core kernel to one CTA per row panel instead of CTA pairs.)
  */
-enum { CERT_CONTRACTION_AUTO = 0, CERT_CONTRACTION_FFMA = 1, CERT_CONTRACTION_TC3XTF32 = 2 };
+enum { CERT_CONTRACTION_AUTO = 0, CERT_CONTRACTION_FFMA = 1, CERT_CONTRACTION_TC3XTF32 = 2,
+       CERT_CONTRACTION_TC3XFP16 = 3 };
 cert_status_t cert_net_set_contraction(cert_net_t *net, int mode);
 /* Which contraction kernels the most recent call ran: bit 0 = FFMA, bit 1 = TC3XTF32,
- * bit 2 = the TC3XTF32 kernel ran in its CTA-pair form (tcgen05 cta_group::2). */
+ * bit 2 = the TC3XTF32 kernel ran in its CTA-pair form (tcgen05 cta_group::2), bit 3 = a traversal ran on
+ * receptive-field patches, bit 4 = TC3XFP16. */
 int cert_net_last_contraction_paths(const cert_net_t *net);
 
 /*

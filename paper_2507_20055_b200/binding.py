@@ -23,7 +23,7 @@ if not os.path.exists(LIB_PATH):
 _lib = ctypes.CDLL(LIB_PATH)
 
 CERT_OK = 0
-CONTRACTION_AUTO, CONTRACTION_FFMA, CONTRACTION_TC3XTF32 = 0, 1, 2
+CONTRACTION_AUTO, CONTRACTION_FFMA, CONTRACTION_TC3XTF32, CONTRACTION_TC3XFP16 = 0, 1, 2, 3
 
 EXPORTS = [
     "cert_net_create", "cert_deeppoly_bounds", "cert_backsub_bounds", "cert_deeppoly_bounds_host",

@@ -11,10 +11,19 @@
 
 #include "common.cuh"
 #include "gemm_tc.cuh"
+#include "gemm_tc16.cuh"
 
 // Tensor-core operands of the back-step through one FC layer j: B = W_j transposed
 // (rows = neurons below, K-major), A = the coefficient matrix over layer j's neurons
 // in either ping-pong buffer.
+// The same operands for the fp16-split kernel (CTA pairs only).
+struct Tc16Layer {
+    bool usable = false;
+    __half *W_hi = nullptr, *W_lo = nullptr;     // W_j transposed, [round_up(n_in, 32)][ld_out]
+    cert::TcMap b_hi, b_lo, a_hi[2], a_lo[2], o_hi[2], o_lo[2];
+    cert::Tc16Plan plan;
+};
+
 struct TcLayer {
     bool usable = false;
     cert::TcMap b_hi, b_lo;          // box = this CTA's share of the column tile
@@ -55,6 +64,8 @@ struct cert_net {
     float *buf_lo[2] = {nullptr, nullptr};   // TF32 lo parts for the tensor-core contraction
     bool tc_ok = false;                      // tensor-core path usable on this net
     std::vector<TcLayer> tc;                 // per layer: operand maps and tile plan
+    bool tc16_ok = false;                    // fp16-split path usable (FC layers only, CTA pairs available)
+    std::vector<Tc16Layer> tc16;
     float *dbuf[2] = {nullptr, nullptr};     // row constants, [d_slots][slot_stride] each, ping-pong
     int d_slots = 1;                         // slots per buffer (most column tiles of any contraction)
     long long slot_stride = 0;               // rows of the largest coefficient matrix
@@ -211,6 +222,55 @@ cert_status_t setup_tensor_core_path(cert_net *net, const cert_layer_desc_t *des
         if (ok) net->d_slots = std::max(net->d_slots, T.plan.n_tiles);
     }
     net->tc_ok = true;
+
+    // fp16-split operands: nets of FC layers, CTA pairs available
+    bool all_fc = true;
+    for (int j = 0; j < K; ++j) all_fc = all_fc && net->layers[j].kind == CERT_LAYER_FC;
+    net->tc16.assign(K, Tc16Layer());
+    if (all_fc && ctas == 2 && cert::tc16_prepare_kernels()) {
+        bool all_ok = true;
+        std::vector<__half> h16, l16;
+        for (int j = 0; j < K - 1 && all_ok; ++j) {
+            LayerDev &L = net->layers[j];
+            Tc16Layer &T = net->tc16[j];
+            size_t rows_pad = round_up(L.n_in, kPad);
+            h16.assign(rows_pad * L.ld_out, __float2half_rn(0.0f));
+            l16.assign(rows_pad * L.ld_out, __float2half_rn(0.0f));
+            for (int t = 0; t < L.n_out; ++t)
+                for (int s2 = 0; s2 < L.n_in; ++s2) {
+                    const float w = descs[j].weight[(size_t)t * L.n_in + s2];
+                    if (!(std::fabs(w) <= 60000.0f)) all_ok = false;
+                    const __half h = __float2half_rn(w);
+                    h16[(size_t)s2 * L.ld_out + t] = h;
+                    l16[(size_t)s2 * L.ld_out + t] = __float2half_rn((w - __half2float(h)) * cert::kLoScale);
+                }
+            if (!dev_alloc(net, (void **)&T.W_hi, h16.size() * sizeof(__half)) ||
+                !dev_alloc(net, (void **)&T.W_lo, l16.size() * sizeof(__half)))
+                return CERT_ERR_OOM;
+            if (cudaMemcpy(T.W_hi, h16.data(), h16.size() * sizeof(__half), cudaMemcpyHostToDevice) != cudaSuccess ||
+                cudaMemcpy(T.W_lo, l16.data(), l16.size() * sizeof(__half), cudaMemcpyHostToDevice) != cudaSuccess)
+                return CERT_ERR_CUDA;
+            T.plan = cert::tc16_tile_plan(L.n_in);
+            if (T.plan.stages < 2) { all_ok = false; break; }
+            bool ok = cert::tc16_make_map(&T.b_hi, T.W_hi, L.n_out, L.n_in, L.ld_out, 64, T.plan.bn / 2) &&
+                      cert::tc16_make_map(&T.b_lo, T.W_lo, L.n_out, L.n_in, L.ld_out, 64, T.plan.bn / 2);
+            long long rows_max = 0;
+            for (int k = j + 1; k < K; ++k) rows_max = std::max(rows_max, 2LL * net->max_batch * net->layers[k].n_out);
+            for (int p = 0; p < 2 && ok; ++p) {
+                const __half *bh = reinterpret_cast<const __half *>(net->buf[p]);
+                const __half *bl = reinterpret_cast<const __half *>(net->buf_lo[p]);
+                ok = cert::tc16_make_map(&T.a_hi[p], bh, L.n_out, rows_max, L.ld_out, 64, 128) &&
+                     cert::tc16_make_map(&T.a_lo[p], bl, L.n_out, rows_max, L.ld_out, 64, 128);
+                if (ok && j > 0)
+                    ok = cert::tc16_make_map(&T.o_hi[p], bh, L.ld_in, rows_max, L.ld_in, 32, 32) &&
+                         cert::tc16_make_map(&T.o_lo[p], bl, L.ld_in, rows_max, L.ld_in, 32, 32);
+            }
+            T.usable = ok;
+            all_ok = all_ok && ok;
+            if (ok) net->d_slots = std::max(net->d_slots, 2 * T.plan.n_tiles);
+        }
+        net->tc16_ok = all_ok;
+    }
     return CERT_OK;
 }
 
@@ -246,6 +306,7 @@ const char *cert_status_string(cert_status_t s) {
         case CERT_ERR_BATCH_TOO_LARGE: return "batch larger than max_batch";
         case CERT_ERR_CUDA: return "CUDA error";
         case CERT_ERR_TIMEOUT: return "device-side wait timed out";
+        case CERT_ERR_RANGE: return "coefficient outside the fp16 range of the TC3XFP16 contraction";
     }
     return "unknown";
 }
@@ -451,6 +512,48 @@ cert_status_t cert_backsub_bounds(cert_net_t *net, const float *centers, float e
         auto on_tc = [&](int j) {
             return net->contraction != CERT_CONTRACTION_FFMA && net->tc_ok && net->tc[j].usable;
         };
+        // fp16-split tensor-core chain (FC nets): start, then one kernel per layer with the ReLU step fused,
+        // the last one concretising.
+        if (net->contraction == CERT_CONTRACTION_TC3XFP16 && net->tc16_ok) {
+            __half *qh[2] = {reinterpret_cast<__half *>(net->buf[0]), reinterpret_cast<__half *>(net->buf[1])};
+            __half *ql[2] = {reinterpret_cast<__half *>(net->buf_lo[0]), reinterpret_cast<__half *>(net->buf_lo[1])};
+            cert::launch_init_expr16(Lk, net->layers[k - 1], batch, qh[cur], ql[cur], net->dbuf[dcur], net->status_dev, st);
+            rec.mark(CERT_CLASS_RELU_STEP);
+            for (int j = k - 1; j >= j_end; --j) {
+                const LayerDev &Lj = net->layers[j];
+                const Tc16Layer &T = net->tc16[j];
+                cert::TcArgs a;
+                std::memset(&a, 0, sizeof(a));
+                a.M = rows; a.K = Lj.n_out; a.n_k = Lk.n_out; a.ld_n = Lj.ld_in;
+                a.bn = T.plan.bn; a.n_tiles = T.plan.n_tiles; a.stages = T.plan.stages; a.tmem_cols = T.plan.tmem_cols;
+                a.total_tiles = (int)cert::ceil_div_ll(rows, 256) * T.plan.n_tiles;
+                a.d_in = net->dbuf[dcur]; a.n_slots_in = dslots; a.d_out = net->dbuf[dcur ^ 1];
+                a.slot_stride = net->slot_stride;
+                a.status = net->status_dev;
+                const int pairs = std::min(a.total_tiles, net->sm_count / 2);
+                if (j > j_end) {
+                    const LayerDev &Lb = net->layers[j - 1];
+                    a.has_relu = Lb.relu_after;
+                    a.split_out = 1;
+                    a.lamL = Lb.lamL; a.lamU = Lb.lamU; a.nuU = Lb.nuU; a.bias_below = Lb.bias_n;
+                    cert::launch_gemm_tc16(cert::TC_EPI_RELU, pairs, T.a_hi[cur], T.a_lo[cur], T.b_hi, T.b_lo,
+                                           T.o_hi[cur ^ 1], T.o_lo[cur ^ 1], a, T.plan.smem_bytes, st);
+                } else {
+                    a.l0 = box_l; a.u0 = box_u;
+                    cert::launch_gemm_tc16(cert::TC_EPI_CONCRETIZE, pairs, T.a_hi[cur], T.a_lo[cur], T.b_hi, T.b_lo,
+                                           T.a_hi[cur], T.a_lo[cur], a, T.plan.smem_bytes, st);
+                }
+                rec.mark(CERT_CLASS_AFFINE);
+                cur ^= 1;
+                dcur ^= 1;
+                dslots = 2 * T.plan.n_tiles;
+            }
+            cert::launch_relax(Lk, lb_out, ub_out, n_total, batch, net->codes, net->n_relu, net->dbuf[dcur], dslots,
+                               net->slot_stride, st);
+            rec.mark(CERT_CLASS_RELAX);
+            paths |= 2 | 4 | 16;
+            continue;
+        }
         // A conv layer over conv layers: rows as receptive-field patches instead of dense maps.
         cert::PatchLevel lv[kMaxPatchLevels];
         if (net->conv_patches && cert::conv_patch_plan(net->layers.data(), k, j_end, lv, kMaxPatchLevels)) {
@@ -820,15 +923,17 @@ cert_status_t cert_net_last_status(cert_net_t *net, void *stream) {
     if (flag != 0) {
         cudaMemsetAsync(net->status_dev, 0, sizeof(int), st);
         cudaStreamSynchronize(st);
-        return CERT_ERR_TIMEOUT;
+        return (flag & 1) ? CERT_ERR_TIMEOUT : CERT_ERR_RANGE;
     }
     return CERT_OK;
 }
 
 cert_status_t cert_net_set_contraction(cert_net_t *net, int mode) {
     if (!net) return CERT_ERR_INVALID_ARG;
-    if (mode != CERT_CONTRACTION_AUTO && mode != CERT_CONTRACTION_FFMA && mode != CERT_CONTRACTION_TC3XTF32)
+    if (mode != CERT_CONTRACTION_AUTO && mode != CERT_CONTRACTION_FFMA && mode != CERT_CONTRACTION_TC3XTF32 &&
+        mode != CERT_CONTRACTION_TC3XFP16)
         return CERT_ERR_INVALID_ARG;
+    if (mode == CERT_CONTRACTION_TC3XFP16 && !net->tc16_ok) return CERT_ERR_UNSUPPORTED;
     if (mode == CERT_CONTRACTION_TC3XTF32 && !net->tc_ok) return CERT_ERR_UNSUPPORTED;
     net->contraction = mode;
     return CERT_OK;

@@ -1,0 +1,486 @@
+// Affine back-step on the tensor cores with an fp16 split (three fp16 products per fp32-accurate
+// multiply-add), the ReLU back-step or the concretisation fused into the epilogue.
+//
+//   P = Q * W_j   (Section 4.3, Matmul rewrite of the traversal step), then as in gemm_tc.cu.
+//
+// x = hi + 2^-11 * lo with hi = fp16(x), lo = fp16(2^11 * (x - hi)).  Per 16-wide k-step:
+//   D2 += Q_lo * W_hi,  D2 += Q_hi * W_lo   (cross terms, in units of 2^-11)
+//   D1 += Q_hi * W_hi
+// in two fp32 accumulators in tensor memory; the epilogue reads D1 + 2^-11 * D2.  fp16 products are exact
+// in fp32, so the result has the accuracy of the 3xTF32 form at twice the MMA rate and half the operand
+// bytes.  A coefficient beyond the fp16 range raises bit 1 of the status word.
+//
+// CTA pairs (tcgen05 cta_group::2) on 256-row panels, persistent over (row panel, column tile) work tiles
+// as in gemm_tc.cu.  The two accumulators of a 256-column tile fill tensor memory, so the epilogue of a
+// tile is not overlapped with the next tile's MMAs; eight epilogue warps (two per TMEM lane quarter, taking
+// alternate 32-column chunks) keep it short.  A row's constant for this tile is written by both of its
+// owner threads: 2 * n_tiles slots per row, summed in slot order by the next kernel.
+#include <cuda.h>
+#include <cuda_fp16.h>
+
+#include "common.cuh"
+#include "gemm_tc16.cuh"
+#include "tc_ptx.cuh"
+
+namespace cert {
+
+namespace {
+
+constexpr int BM = 128;                  // rows per CTA
+constexpr int BKH = 64;                  // halves of K per stage: one 128-byte swizzle row
+constexpr int kEpiWarps = 8;
+constexpr int kThreads16 = 64 + kEpiWarps * 32;
+constexpr int kATileBytes = BM * BKH * 2;
+constexpr int kSlabBytes16 = 32 * 64;    // 32 rows x 32 halves per epilogue warp and output array
+constexpr int kEpiBytes16 = kEpiWarps * 2 * kSlabBytes16;
+
+struct __align__(8) Barriers16 {
+    uint64_t full[8];
+    uint64_t empty[8];
+    uint64_t acc_full;
+    uint64_t acc_empty;
+    uint32_t tmem_base;
+    uint32_t abort_flag;
+};
+
+template <int EPI>
+__global__ void __launch_bounds__(kThreads16, 1)
+gemm_tc16_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_constant__ CUtensorMap map_a_lo,
+                 const __grid_constant__ CUtensorMap map_b_hi, const __grid_constant__ CUtensorMap map_b_lo,
+                 const __grid_constant__ CUtensorMap map_o_hi, const __grid_constant__ CUtensorMap map_o_lo,
+                 const TcArgs a) {
+    constexpr int CTAS = 2;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    const int BN = a.bn;
+    const int BNL = BN / CTAS;                 // rows of the W_j tile this CTA stages
+    const int stages = a.stages;
+    const uint32_t b_tile_bytes = (uint32_t)BNL * BKH * 2;
+    const uint32_t stage_bytes = 2 * kATileBytes + 2 * b_tile_bytes;
+    uint8_t *epi_smem = smem + (size_t)stages * stage_bytes;
+    Barriers16 *bars = reinterpret_cast<Barriers16 *>(epi_smem + kEpiBytes16);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int num_kb = (a.K + BKH - 1) / BKH;
+    const int n_tiles = a.n_tiles;
+    const int total_tiles = a.total_tiles;
+    const uint32_t rank = cluster_ctarank();
+    const int group = (int)cluster_id_x();
+    const int n_groups = (int)num_clusters_x();
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < stages; ++s) {
+            mbar_init(&bars->full[s], 1);
+            mbar_init(&bars->empty[s], 1);
+        }
+        mbar_init(&bars->acc_full, 1);
+        mbar_init(&bars->acc_empty, kEpiWarps * CTAS);
+        bars->abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
+                         smem_u32(&bars->tmem_base)),
+                     "r"((uint32_t)a.tmem_cols)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    }
+    tcgen05_fence_before();
+    __syncthreads();
+    cluster_sync_all();      // the peer's barriers exist before anything arrives on them
+    tcgen05_fence_after();
+    const uint32_t tmem_base = bars->tmem_base;
+    volatile uint32_t *abort_flag = &bars->abort_flag;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            int s = 0;
+            uint32_t phase = 0;
+            bool ok = true;
+            int armed = 0;
+            for (int t = group; t < total_tiles && ok; t += n_groups) {
+                const int row0 = (t / n_tiles) * (BM * CTAS) + (int)rank * BM;
+                const int col0 = (t % n_tiles) * BN + (int)rank * BNL;
+                for (int kb = 0; kb < num_kb; ++kb) {
+                    if (!mbar_wait(&bars->empty[s], phase ^ 1) || *abort_flag) { ok = false; break; }
+                    uint8_t *st = smem + (size_t)s * stage_bytes;
+                    if (rank == 0) mbar_arrive_expect_tx(&bars->full[s], stage_bytes * CTAS);
+                    const uint32_t bar = map_to_cta(smem_u32(&bars->full[s]), 0);
+                    const int kx = kb * BKH;
+                    tma_load_2d<CTAS>(smem_u32(st), &map_a_hi, bar, kx, row0);
+                    tma_load_2d<CTAS>(smem_u32(st + kATileBytes), &map_a_lo, bar, kx, row0);
+                    tma_load_2d<CTAS>(smem_u32(st + 2 * kATileBytes), &map_b_hi, bar, kx, col0);
+                    tma_load_2d<CTAS>(smem_u32(st + 2 * kATileBytes + b_tile_bytes), &map_b_lo, bar, kx, col0);
+                    ++armed;
+                    if (++s == stages) { s = 0; phase ^= 1; }
+                }
+            }
+            if (!ok) {
+                *abort_flag = 1;
+                atomicOr(a.status, 1);
+                if (rank == 0) {
+                    // let the copies already in flight land before the CTA gives its shared memory back
+                    int back = armed < stages ? armed : stages;
+                    int ss = s;
+                    uint32_t ph = phase;
+                    for (int i = 0; i < back; ++i) {
+                        if (--ss < 0) { ss = stages - 1; ph ^= 1; }
+                        mbar_wait(&bars->full[ss], ph);
+                    }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------ MMA issuer (the leader CTA)
+        if (lane == 0 && rank == 0) {
+            // kind::f16: D = f32, A = B = f16 (format 0), both K-major
+            const uint32_t idesc = (1u << 4) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)((BM * CTAS) >> 4) << 24);
+            int s = 0;
+            uint32_t phase = 0;
+            bool ok = true;
+            int lt = 0;
+            const uint32_t d1 = tmem_base, d2 = tmem_base + (uint32_t)BN;
+            for (int t = group; t < total_tiles && ok; t += n_groups, ++lt) {
+                if (!mbar_wait(&bars->acc_empty, (lt & 1) ^ 1) || *abort_flag) { ok = false; break; }
+                tcgen05_fence_after();
+                for (int kb = 0; kb < num_kb; ++kb) {
+                    if (!mbar_wait(&bars->full[s], phase) || *abort_flag) { ok = false; break; }
+                    tcgen05_fence_after();
+                    const uint32_t st = smem_u32(smem + (size_t)s * stage_bytes);
+                    const uint64_t da_hi = make_desc(st);
+                    const uint64_t da_lo = make_desc(st + kATileBytes);
+                    const uint64_t db_hi = make_desc(st + 2 * kATileBytes);
+                    const uint64_t db_lo = make_desc(st + 2 * kATileBytes + b_tile_bytes);
+#pragma unroll
+                    for (int k = 0; k < BKH / 16; ++k) {
+                        const uint64_t ko = (uint64_t)(k * 2);   // 16 halves = 32 bytes = 2 x 16-byte units
+                        const uint32_t first = (kb | k) ? 1u : 0u;
+                        mma_f16<CTAS>(d2, da_lo + ko, db_hi + ko, idesc, first);
+                        mma_f16<CTAS>(d2, da_hi + ko, db_lo + ko, idesc, 1u);
+                        mma_f16<CTAS>(d1, da_hi + ko, db_hi + ko, idesc, first);
+                    }
+                    tcgen05_commit<CTAS>(&bars->empty[s]);
+                    if (++s == stages) { s = 0; phase ^= 1; }
+                }
+                if (ok) tcgen05_commit<CTAS>(&bars->acc_full);
+            }
+            if (!ok) {
+                *abort_flag = 1;
+                atomicOr(a.status, 1);
+            }
+        }
+    } else {
+        // ------------------------------------------------------------ epilogue (8 warps)
+        const int ew = warp - 2;
+        const int quarter = warp & 3;                       // TMEM lane quarter this warp may read
+        const int half_id = ew >> 2;                        // which of the two warps of the quarter
+        uint8_t *slab_hi = epi_smem + (size_t)ew * 2 * kSlabBytes16;
+        uint8_t *slab_lo = slab_hi + kSlabBytes16;
+        const uint32_t acc_empty_addr = map_to_cta(smem_u32(&bars->acc_empty), 0);
+        bool ok = true, out_of_range = false;
+        int lt = 0;
+        for (int t = group; t < total_tiles && ok; t += n_groups, ++lt) {
+            const int nt = t % n_tiles;
+            const long long warp_row0 = (long long)(t / n_tiles) * (BM * CTAS) + (int)rank * BM + quarter * 32;
+            const long long r = warp_row0 + lane;
+            const bool row_ok = r < a.M;
+            const long long rr = row_ok ? r : 0;
+            const int b = (int)(rr / (2LL * a.n_k));
+            const int upper = (int)((rr / a.n_k) & 1);
+            const size_t relax_row = (size_t)b * a.ld_n;
+            float dacc = 0.0f;
+            if (!mbar_wait(&bars->acc_full, lt & 1) || *abort_flag) { ok = false; break; }
+            tcgen05_fence_after();
+            const uint32_t t_addr = tmem_base + ((uint32_t)(quarter * 32) << 16);
+            for (int c0 = 32 * half_id; c0 < BN; c0 += 64) {
+                const int col0 = nt * BN + c0;
+                if (col0 >= a.ld_n) break;                   // warp-uniform; ld_n is a multiple of 32
+                uint32_t v1[32], v2[32];
+                __syncwarp();
+                tmem_ld32(t_addr + (uint32_t)c0, v1);
+                tmem_ld32(t_addr + (uint32_t)(BN + c0), v2);
+                tmem_ld_wait();
+                if (EPI == TC_EPI_RELU) {
+                    // the slab is free again once the previous chunk's stores have read it
+                    if (lane == 0) tma_store_wait_read();
+                    __syncwarp();
+                    const uint32_t row_hi = smem_u32(slab_hi) + (uint32_t)lane * 64u;
+                    const uint32_t row_lo = smem_u32(slab_lo) + (uint32_t)lane * 64u;
+#pragma unroll
+                    for (int c16 = 0; c16 < 4; ++c16) {
+                        uint32_t ph[4], pl[4];              // 8 halves of hi, 8 of lo
+#pragma unroll
+                        for (int g2 = 0; g2 < 2; ++g2) {
+                            const int g = c16 * 2 + g2;
+                            const int col = col0 + g * 4;
+                            float q[4];
+                            const float4 bz = *reinterpret_cast<const float4 *>(a.bias_below + col);
+                            if (a.has_relu) {
+                                const float4 ll = *reinterpret_cast<const float4 *>(a.lamL + relax_row + col);
+                                const float4 lu = *reinterpret_cast<const float4 *>(a.lamU + relax_row + col);
+                                const float4 nu = *reinterpret_cast<const float4 *>(a.nuU + relax_row + col);
+                                const float l4[4] = {ll.x, ll.y, ll.z, ll.w}, u4[4] = {lu.x, lu.y, lu.z, lu.w},
+                                            n4[4] = {nu.x, nu.y, nu.z, nu.w};
+#pragma unroll
+                                for (int e = 0; e < 4; ++e) {
+                                    const float c = fmaf(__uint_as_float(v2[g * 4 + e]), kLoUnscale,
+                                                         __uint_as_float(v1[g * 4 + e]));
+                                    const bool nonneg = (c >= 0.0f);
+                                    const bool use_lower = upper ? !nonneg : nonneg;
+                                    q[e] = c * (use_lower ? l4[e] : u4[e]);
+                                    dacc = fmaf(c, use_lower ? 0.0f : n4[e], dacc);
+                                }
+                            } else {
+#pragma unroll
+                                for (int e = 0; e < 4; ++e)
+                                    q[e] = fmaf(__uint_as_float(v2[g * 4 + e]), kLoUnscale, __uint_as_float(v1[g * 4 + e]));
+                            }
+                            dacc = fmaf(q[0], bz.x, dacc);
+                            dacc = fmaf(q[1], bz.y, dacc);
+                            dacc = fmaf(q[2], bz.z, dacc);
+                            dacc = fmaf(q[3], bz.w, dacc);
+                            __half h[4], l[4];
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                out_of_range |= row_ok && !(fabsf(q[e]) <= 60000.0f);
+                                h[e] = __float2half_rn(q[e]);
+                                l[e] = __float2half_rn((q[e] - __half2float(h[e])) * kLoScale);
+                            }
+                            ph[g2 * 2 + 0] = (uint32_t)__half_as_ushort(h[0]) | ((uint32_t)__half_as_ushort(h[1]) << 16);
+                            ph[g2 * 2 + 1] = (uint32_t)__half_as_ushort(h[2]) | ((uint32_t)__half_as_ushort(h[3]) << 16);
+                            pl[g2 * 2 + 0] = (uint32_t)__half_as_ushort(l[0]) | ((uint32_t)__half_as_ushort(l[1]) << 16);
+                            pl[g2 * 2 + 1] = (uint32_t)__half_as_ushort(l[2]) | ((uint32_t)__half_as_ushort(l[3]) << 16);
+                        }
+                        // 16-byte chunk c16 of this lane's 64-byte slab row, at its 64-byte-swizzle position
+                        const uint32_t sw = (uint32_t)((c16 ^ ((lane >> 1) & 3)) << 4);
+                        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(row_hi + sw), "r"(ph[0]), "r"(ph[1]),
+                                     "r"(ph[2]), "r"(ph[3]) : "memory");
+                        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(row_lo + sw), "r"(pl[0]), "r"(pl[1]),
+                                     "r"(pl[2]), "r"(pl[3]) : "memory");
+                    }
+                    fence_async_smem();
+                    __syncwarp();
+                    // rows past the end of the matrix land in scratch rows of the workspace or are clipped
+                    if (lane == 0) {
+                        tma_store_2d(&map_o_hi, smem_u32(slab_hi), col0, (int)warp_row0);
+                        tma_store_2d(&map_o_lo, smem_u32(slab_lo), col0, (int)warp_row0);
+                        tma_store_commit();
+                    }
+                } else if (row_ok) {
+                    const float *lrow = a.l0 + (size_t)b * a.ld_n + col0;
+                    const float *urow = a.u0 + (size_t)b * a.ld_n + col0;
+#pragma unroll
+                    for (int g = 0; g < 8; ++g) {
+                        const float4 l4 = *reinterpret_cast<const float4 *>(lrow + g * 4);
+                        const float4 u4 = *reinterpret_cast<const float4 *>(urow + g * 4);
+                        const float lo4[4] = {l4.x, l4.y, l4.z, l4.w}, up4[4] = {u4.x, u4.y, u4.z, u4.w};
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const float c = fmaf(__uint_as_float(v2[g * 4 + e]), kLoUnscale, __uint_as_float(v1[g * 4 + e]));
+                            const bool nonneg = (c >= 0.0f);
+                            dacc = fmaf(c, (nonneg != (upper != 0)) ? lo4[e] : up4[e], dacc);
+                        }
+                    }
+                }
+            }
+            tcgen05_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(acc_empty_addr);
+            // This warp's share of the row constant (of the bound) goes to slot 2*nt + half_id; the first
+            // slot also carries the constant so far.
+            if (row_ok) {
+                float tot = dacc;
+                if (nt == 0 && half_id == 0) {
+                    float prev = 0.0f;
+                    for (int sidx = 0; sidx < a.n_slots_in; ++sidx) prev += a.d_in[(size_t)sidx * a.slot_stride + r];
+                    tot += prev;
+                }
+                a.d_out[(size_t)(2 * nt + half_id) * a.slot_stride + r] = tot;
+            }
+        }
+        if (EPI == TC_EPI_RELU && lane == 0) tma_store_wait_all();
+        if (__any_sync(0xffffffffu, out_of_range) && lane == 0) atomicOr(a.status, 2);
+        if (!ok && lane == 0) atomicOr(a.status, 1);
+    }
+
+    tcgen05_fence_before();
+    __syncthreads();
+    cluster_sync_all();      // no CTA leaves while its peer may still reach into it
+    if (warp == 1) {
+        tcgen05_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)a.tmem_cols)
+                     : "memory");
+    }
+}
+
+__device__ __forceinline__ float warp_sum16(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+// Start of a back-substitution at FC layer k as an fp16 pair: row i of W_k pushed through the ReLU below,
+// constant = b_k[i] + the nu terms + Q.b of the layer below.  One warp per row, 4 columns per lane.
+__global__ void expr_start16_kernel(const float *__restrict__ Wk, int ldw_k, const float *__restrict__ bias_k,
+                                    __half *__restrict__ Q_hi, __half *__restrict__ Q_lo, float *__restrict__ d,
+                                    long long rows, int n_k, int n, int ld, int has_relu,
+                                    const float *__restrict__ lamL, const float *__restrict__ lamU,
+                                    const float *__restrict__ nuU, const float *__restrict__ bias_below,
+                                    int *__restrict__ status) {
+    const long long r = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int lane = threadIdx.x & 31;
+    if (r >= rows) return;
+    const int b = (int)(r / (2LL * n_k));
+    const int upper = (int)((r / n_k) & 1);
+    const int i = (int)(r % n_k);
+    const float *ll = lamL + (size_t)b * ld, *lu = lamU + (size_t)b * ld, *nu = nuU + (size_t)b * ld;
+    float dacc = 0.0f;
+    bool out_of_range = false;
+    for (int t = lane * 4; t < ld; t += 128) {
+        const float4 c4 = *reinterpret_cast<const float4 *>(Wk + (size_t)i * ldw_k + t);
+        const float c[4] = {c4.x, c4.y, c4.z, c4.w};
+        const float4 bz4 = *reinterpret_cast<const float4 *>(bias_below + t);
+        const float bz[4] = {bz4.x, bz4.y, bz4.z, bz4.w};
+        float q[4];
+        if (has_relu) {
+            const float4 l4 = *reinterpret_cast<const float4 *>(ll + t);
+            const float4 u4 = *reinterpret_cast<const float4 *>(lu + t);
+            const float4 n4 = *reinterpret_cast<const float4 *>(nu + t);
+            const float la[4] = {l4.x, l4.y, l4.z, l4.w}, ua[4] = {u4.x, u4.y, u4.z, u4.w},
+                        na[4] = {n4.x, n4.y, n4.z, n4.w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                q[e] = 0.0f;
+                if (t + e < n) {
+                    const bool nonneg = (c[e] >= 0.0f);
+                    const bool use_lower = upper ? !nonneg : nonneg;
+                    q[e] = c[e] * (use_lower ? la[e] : ua[e]);
+                    if (!use_lower) dacc = fmaf(c[e], na[e], dacc);
+                }
+            }
+        } else {
+#pragma unroll
+            for (int e = 0; e < 4; ++e) q[e] = (t + e < n) ? c[e] : 0.0f;
+        }
+        __half h[4], l[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            dacc = fmaf(q[e], bz[e], dacc);
+            out_of_range |= !(fabsf(q[e]) <= 60000.0f);
+            h[e] = __float2half_rn(q[e]);
+            l[e] = __float2half_rn((q[e] - __half2float(h[e])) * kLoScale);
+        }
+        uint2 ph, pl;
+        ph.x = (uint32_t)__half_as_ushort(h[0]) | ((uint32_t)__half_as_ushort(h[1]) << 16);
+        ph.y = (uint32_t)__half_as_ushort(h[2]) | ((uint32_t)__half_as_ushort(h[3]) << 16);
+        pl.x = (uint32_t)__half_as_ushort(l[0]) | ((uint32_t)__half_as_ushort(l[1]) << 16);
+        pl.y = (uint32_t)__half_as_ushort(l[2]) | ((uint32_t)__half_as_ushort(l[3]) << 16);
+        *reinterpret_cast<uint2 *>(Q_hi + (size_t)r * ld + t) = ph;
+        *reinterpret_cast<uint2 *>(Q_lo + (size_t)r * ld + t) = pl;
+    }
+    dacc = warp_sum16(dacc);
+    if (lane == 0) d[r] = bias_k[i] + dacc;
+    if (__any_sync(0xffffffffu, out_of_range) && lane == 0) atomicOr(status, 2);
+}
+
+typedef CUresult (*EncodeTiledFn16)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                    const cuuint64_t *, const cuuint32_t *, const cuuint32_t *,
+                                    CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                    CUtensorMapFloatOOBfill);
+EncodeTiledFn16 g_encode16 = nullptr;
+
+template <int EPI>
+void launch_one16(int pairs, const CUtensorMap &ah, const CUtensorMap &al, const CUtensorMap &bh,
+                  const CUtensorMap &bl, const CUtensorMap &oh, const CUtensorMap &ol, const TcArgs &args,
+                  int smem_bytes, cudaStream_t st) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(pairs * 2), 1, 1);
+    cfg.blockDim = dim3(kThreads16, 1, 1);
+    cfg.dynamicSmemBytes = (size_t)smem_bytes;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaLaunchKernelEx(&cfg, gemm_tc16_kernel<EPI>, ah, al, bh, bl, oh, ol, args);
+}
+
+}  // namespace
+
+bool tc16_prepare_kernels() {
+    if (!g_encode16) {
+        void *fn = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
+            qres != cudaDriverEntryPointSuccess || !fn) {
+            cudaGetLastError();
+            return false;
+        }
+        g_encode16 = reinterpret_cast<EncodeTiledFn16>(fn);
+    }
+    if (cudaFuncSetAttribute(gemm_tc16_kernel<TC_EPI_RELU>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemMax) !=
+            cudaSuccess ||
+        cudaFuncSetAttribute(gemm_tc16_kernel<TC_EPI_CONCRETIZE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             kTcSmemMax) != cudaSuccess) {
+        cudaGetLastError();
+        return false;
+    }
+    return true;
+}
+
+bool tc16_make_map(TcMap *m, const __half *base, long long inner, long long outer, long long pitch_elems,
+                   int box_inner, int box_outer) {
+    if (!g_encode16) return false;
+    cuuint64_t dims[2] = {(cuuint64_t)inner, (cuuint64_t)outer};
+    cuuint64_t strides[1] = {(cuuint64_t)pitch_elems * sizeof(__half)};
+    cuuint32_t box[2] = {(cuuint32_t)box_inner, (cuuint32_t)box_outer};
+    cuuint32_t estr[2] = {1u, 1u};
+    CUresult r = g_encode16(reinterpret_cast<CUtensorMap *>(m), CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2,
+                            const_cast<__half *>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                            box_inner == 64 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B,
+                            CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
+Tc16Plan tc16_tile_plan(int N) {
+    Tc16Plan p;
+    p.n_tiles = (N + 255) / 256;
+    int b = ((N + p.n_tiles - 1) / p.n_tiles + 31) / 32 * 32;
+    p.bn = b;
+    const int stage_bytes = 2 * kATileBytes + 2 * (b / 2) * BKH * 2;
+    const int fixed = kEpiBytes16 + (int)sizeof(Barriers16) + 1024;
+    int st = (kTcSmemMax - fixed) / stage_bytes;
+    p.stages = st > 8 ? 8 : st;
+    int cols = 32;
+    while (cols < 2 * b) cols *= 2;
+    p.tmem_cols = cols;
+    p.smem_bytes = p.stages * stage_bytes + fixed;
+    return p;
+}
+
+void launch_gemm_tc16(int epi, int pairs, const TcMap &a_hi, const TcMap &a_lo, const TcMap &b_hi, const TcMap &b_lo,
+                      const TcMap &o_hi, const TcMap &o_lo, const TcArgs &args, int smem_bytes, cudaStream_t st) {
+    const CUtensorMap &ah = reinterpret_cast<const CUtensorMap &>(a_hi);
+    const CUtensorMap &al = reinterpret_cast<const CUtensorMap &>(a_lo);
+    const CUtensorMap &bh = reinterpret_cast<const CUtensorMap &>(b_hi);
+    const CUtensorMap &bl = reinterpret_cast<const CUtensorMap &>(b_lo);
+    const CUtensorMap &oh = reinterpret_cast<const CUtensorMap &>(o_hi);
+    const CUtensorMap &ol = reinterpret_cast<const CUtensorMap &>(o_lo);
+    if (epi == TC_EPI_RELU) launch_one16<TC_EPI_RELU>(pairs, ah, al, bh, bl, oh, ol, args, smem_bytes, st);
+    else launch_one16<TC_EPI_CONCRETIZE>(pairs, ah, al, bh, bl, oh, ol, args, smem_bytes, st);
+}
+
+void launch_init_expr16(const LayerDev &Lk, const LayerDev &Lb, int batch, __half *Q_hi, __half *Q_lo, float *d,
+                        int *status, cudaStream_t st) {
+    const long long rows = 2LL * batch * Lk.n_out;
+    expr_start16_kernel<<<(unsigned)ceil_div_ll(rows, 8), 256, 0, st>>>(
+        Lk.W, Lk.ld_in, Lk.bias_n, Q_hi, Q_lo, d, rows, Lk.n_out, Lb.n_out, Lb.ld_out, Lb.relu_after, Lb.lamL,
+        Lb.lamU, Lb.nuU, Lb.bias_n, status);
+}
+
+}  // namespace cert

@@ -1,0 +1,37 @@
+// Interface of the fp16-split tensor-core affine back-step (CERT_CONTRACTION_TC3XFP16).
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_fp16.h>
+#include <cstdint>
+
+#include "gemm_tc.cuh"
+
+namespace cert {
+
+// An fp32 value x is held as hi = fp16(x) and lo = fp16(2^11 * (x - hi)): 22 bits of significand, as the
+// TF32 pair, at half the bytes and twice the tensor-core rate.  Products are exact in the fp32
+// accumulators; hi*hi goes to one accumulator, the cross terms (scaled by 2^11) to a second one, and the
+// epilogue adds them as D1 + 2^-11 * D2.  Range: |x| must stay below 65504 (a larger coefficient raises the
+// range flag, bit 1 of the status word); below 6.1e-5 the pair is exact to 1.5e-11 absolute.
+constexpr float kLoScale = 2048.0f;
+constexpr float kLoUnscale = 1.0f / 2048.0f;
+
+struct Tc16Plan {
+    int bn, n_tiles, stages, tmem_cols, smem_bytes;
+};
+
+bool tc16_prepare_kernels();
+// 2D fp16 tensor [outer][inner], row pitch in elements; box = box_inner x box_outer elements;
+// box_inner = 64 -> 128-byte swizzle (operand tiles), 32 -> 64-byte swizzle (epilogue slabs).
+bool tc16_make_map(TcMap *m, const __half *base, long long inner, long long outer, long long pitch_elems,
+                   int box_inner, int box_outer);
+Tc16Plan tc16_tile_plan(int N);
+// CTA pairs only.  TcArgs as for the TF32 kernel; d_out receives 2 * n_tiles slots per row.
+void launch_gemm_tc16(int epi, int pairs, const TcMap &a_hi, const TcMap &a_lo, const TcMap &b_hi, const TcMap &b_lo,
+                      const TcMap &o_hi, const TcMap &o_lo, const TcArgs &args, int smem_bytes, cudaStream_t st);
+// Start of a traversal at FC layer k as an fp16 pair (see launch_init_expr).
+struct LayerDev;
+void launch_init_expr16(const LayerDev &Lk, const LayerDev &Lbelow, int batch, __half *Q_hi, __half *Q_lo, float *d,
+                        int *status, cudaStream_t st);
+
+}  // namespace cert

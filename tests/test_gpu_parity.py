@@ -311,3 +311,68 @@ def test_reusecert_config5_sampled_boxes():
     finally:
         net.destroy()
     compare(g, ref, boxes=boxes, label="reusecert/fc6x1024", tol=REUSE_TOL, min_good_fraction=0.1)
+
+
+# ---- fp16-split tensor-core contraction (CERT_CONTRACTION_TC3XFP16), nets of FC layers ----
+
+TC16 = 3
+FC_NETS = {
+    "fc3x50": lambda: wl.make_config(0),
+    "fc6x100": lambda: wl.make_config(1),
+    "fc9x200": lambda: wl.make_config(2),
+    "ragged_widths": SMALL["ragged_widths"],
+    "one_hidden": SMALL["one_hidden"],
+    "wide_then_narrow": SMALL["wide_then_narrow"],
+    "relu_on_last": SMALL["relu_on_last"],
+    "fc_ragged5": VARIANT_NETS["fc_ragged"],
+}
+
+
+@pytest.mark.parametrize("name", sorted(FC_NETS))
+def test_fp16_split_contraction(name):
+    w = FC_NETS[name]()
+    g = run_gpu(w, contraction=TC16)
+    assert g["paths"] & 16
+    compare(g, _oracle(w), label=f"{name}/tc16")
+
+
+def test_fp16_split_config5_sampled_boxes():
+    w = wl.make_config(4)
+    boxes = [0, 17, 42, 63, 64, 99, 120, 127]
+    g = run_gpu(w, contraction=TC16)
+    assert g["paths"] & 16
+    compare(g, _oracle(w, boxes), boxes=boxes, label=f"{w.name}/tc16")
+
+
+def test_fp16_split_bounded_traversals_and_missing_relu():
+    w = VARIANT_NETS["fc_wide"]()
+    for vname, steps in _variant_steps(len(w.layers)).items():
+        ref = orc.deeppoly(w.layers, w.centers, w.eps, w.clip_lo, w.clip_hi, backsteps_per_layer=steps)
+        compare(run_gpu(w, contraction=TC16, backsteps=steps), ref, label=f"fc_wide/{vname}/tc16")
+    w = wl.small_fc([24, 40, 36, 40, 6], batch=3, eps=0.05, seed=71)
+    w.layers[1].relu_after = False
+    compare(run_gpu(w, contraction=TC16), _oracle(w), label="no_relu_mid/tc16")
+
+
+def test_fp16_split_is_refused_for_conv_nets_and_flags_its_range():
+    import torch
+    from paper_2507_20055_b200 import binding
+    wc = wl.small_conv((1, 10, 10), [(20, 5, 1, 0)], [6], batch=2, eps=0.05, seed=68)
+    net = binding.CertNet(wc.layers, 2)
+    try:
+        assert binding.lib.cert_net_set_contraction(net._h, TC16) == 2      # CERT_ERR_UNSUPPORTED
+    finally:
+        net.destroy()
+    # weights of 300 make second-layer coefficients of 9e4 > 65504: the range flag must come up
+    w = wl.small_fc([8, 16, 16, 4], batch=2, eps=0.01, seed=88)
+    for l in w.layers:
+        l.weight = (np.sign(l.weight) * 300.0).astype(np.float32)
+    net = binding.CertNet(w.layers, 2, -1e30, 1e30)
+    try:
+        net.set_contraction(TC16)
+        net.deeppoly_bounds(torch.from_numpy(w.centers).cuda(), w.eps)
+        torch.cuda.synchronize()
+        assert net.last_status() == 7                                          # CERT_ERR_RANGE
+        assert net.last_status() == 0                                          # the flag is cleared by the read
+    finally:
+        net.destroy()
