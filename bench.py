@@ -204,8 +204,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", type=int, default=4, help="0..4: index into the benchmark configurations")
     ap.add_argument("--batch", type=int, default=None)
-    ap.add_argument("--contraction", default="auto", choices=["auto", "ffma", "tc", "tc16"],
-                    help="tc = tcgen05 3xTF32, tc16 = tcgen05 fp16 split (FC nets), ffma = FMA units")
+    ap.add_argument("--contraction", default="fastest", choices=["fastest", "auto", "ffma", "tc", "tc16"],
+                    help="tc = tcgen05 3xTF32, tc16 = tcgen05 fp16 split (FC nets), ffma = FMA units, auto = the "
+                         "library's default (tc), fastest = tc16 for FC nets, else auto")
     ap.add_argument("--certifier", default="deeppoly",
                     help="deeppoly | ibp | crown_ibp | deeppoly_pN (N back-substitution steps per layer) | reusecert")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -247,6 +248,9 @@ def main():
     net = binding.CertNet(w.layers, B, w.clip_lo, w.clip_hi)
     mode = {"auto": binding.CONTRACTION_AUTO, "ffma": binding.CONTRACTION_FFMA, "tc": binding.CONTRACTION_TC3XTF32,
             "tc16": binding.CONTRACTION_TC3XFP16}
+    if args.contraction == "fastest":
+        all_fc = all(l.kind == "fc" for l in w.layers)
+        args.contraction = "tc16" if (all_fc and len(w.layers) > 1 and args.certifier != "reusecert") else "auto"
     net.set_contraction(mode[args.contraction])
     stream = torch.cuda.Stream()
     centers = torch.from_numpy(w.centers).cuda()
@@ -308,6 +312,27 @@ def main():
                 cls_n[name] = cls_n.get(name, 0) + n
     net.set_profiling(False)
     clocks = sampler.stop() if rank == 0 else None
+
+    # ---- the same steps with the 3xTF32 contraction, for reference, when the fp16 split was timed above ----
+    tf32_ref = None
+    if args.contraction == "tc16" and world == 1:
+        net.set_contraction(binding.CONTRACTION_TC3XTF32)
+        n_ref = max(3, min(args.steps, 5))
+        ev2 = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_ref)]
+        with torch.cuda.stream(stream):
+            for _ in range(3):
+                step_device()
+            for i in range(n_ref):
+                flush.fill_(i & 0xFF)
+                ev2[i][0].record(stream)
+                step_device()
+                ev2[i][1].record(stream)
+        stream.synchronize()
+        ms_ref = sum(a.elapsed_time(b) for a, b in ev2) / n_ref
+        tf32_ref = {"value": B / (ms_ref / 1000.0), "unit": UNIT, "ms_per_step": ms_ref, "steps": n_ref,
+                    "contraction": "tc (3xTF32)"}
+        assert net.last_status(stream.cuda_stream) == 0
+        net.set_contraction(binding.CONTRACTION_TC3XFP16)
 
     # ---- end to end through the host-buffer entry point (pinned buffers, copies timed) ----
     centers_pin = torch.from_numpy(w.centers).pin_memory()
@@ -396,6 +421,8 @@ def main():
                     "d2h_bytes_per_step": int(2 * B * net.n_total * 4), "steps": e2e_steps},
             "gpu_launches": launches, "wall_s_timed_region": t_wall, "roofline": roof, "clocks": clocks,
         }
+        if tf32_ref is not None:
+            out["tf32_split"] = tf32_ref
         if world == 1 and not args.no_cpu_baseline:
             n_boxes = {0: 1, 1: 64, 2: 32, 3: 16, 4: 16}[args.config]
             from oracle import deeppoly_oracle as orc

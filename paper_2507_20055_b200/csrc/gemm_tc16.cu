@@ -3,17 +3,19 @@
 //
 //   P = Q * W_j   (Section 4.3, Matmul rewrite of the traversal step), then as in gemm_tc.cu.
 //
-// x = hi + 2^-11 * lo with hi = fp16(x), lo = fp16(2^11 * (x - hi)).  Per 16-wide k-step:
-//   D2 += Q_lo * W_hi,  D2 += Q_hi * W_lo   (cross terms, in units of 2^-11)
-//   D1 += Q_hi * W_hi
-// in two fp32 accumulators in tensor memory; the epilogue reads D1 + 2^-11 * D2.  fp16 products are exact
-// in fp32, so the result has the accuracy of the 3xTF32 form at twice the MMA rate and half the operand
-// bytes.  A coefficient beyond the fp16 range raises bit 1 of the status word.
+// x = hi + 2^-11 * lo with hi = fp16(x), lo = fp16(2^11 * (x - hi)).  A tile takes two passes over K into
+// one fp32 accumulator in tensor memory:
+//   pass 1:  D  = sum over K of  Q_lo * W_hi + Q_hi * W_lo      (cross terms, in units of 2^-11)
+//   pass 2:  D  = Q_hi * W_hi + D * 2^-11  for the first k-step (the MMA scales its input accumulator),
+//            D += Q_hi * W_hi             for the rest.
+// fp16 products are exact in fp32, so the result has the accuracy of the 3xTF32 form at twice the MMA rate;
+// pass 2 stages only the hi tiles (two k-blocks per pipeline stage).  A coefficient beyond the fp16 range
+// raises bit 1 of the status word.
 //
-// CTA pairs (tcgen05 cta_group::2) on 256-row panels, persistent over (row panel, column tile) work tiles
-// as in gemm_tc.cu.  The two accumulators of a 256-column tile fill tensor memory, so the epilogue of a
-// tile is not overlapped with the next tile's MMAs; eight epilogue warps (two per TMEM lane quarter, taking
-// alternate 32-column chunks) keep it short.  A row's constant for this tile is written by both of its
+// CTA pairs (tcgen05 cta_group::2) on 256-row panels, persistent over (row panel, column tile) work tiles,
+// two accumulators so that the epilogue of a tile overlaps the MMAs of the next, as in gemm_tc.cu.  A tile's
+// MMAs take half the time they take there, so eight epilogue warps (two per TMEM lane quarter, taking
+// alternate 32-column chunks) run the epilogue.  A row's constant for this tile is written by both of its
 // owner threads: 2 * n_tiles slots per row, summed in slot order by the next kernel.
 #include <cuda.h>
 #include <cuda_fp16.h>
@@ -37,8 +39,8 @@ constexpr int kEpiBytes16 = kEpiWarps * 2 * kSlabBytes16;
 struct __align__(8) Barriers16 {
     uint64_t full[8];
     uint64_t empty[8];
-    uint64_t acc_full;
-    uint64_t acc_empty;
+    uint64_t acc_full[2];
+    uint64_t acc_empty[2];
     uint32_t tmem_base;
     uint32_t abort_flag;
 };
@@ -73,8 +75,10 @@ gemm_tc16_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_cons
             mbar_init(&bars->full[s], 1);
             mbar_init(&bars->empty[s], 1);
         }
-        mbar_init(&bars->acc_full, 1);
-        mbar_init(&bars->acc_empty, kEpiWarps * CTAS);
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(&bars->acc_full[i], 1);
+            mbar_init(&bars->acc_empty[i], kEpiWarps * CTAS);
+        }
         bars->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -103,7 +107,8 @@ gemm_tc16_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_cons
             for (int t = group; t < total_tiles && ok; t += n_groups) {
                 const int row0 = (t / n_tiles) * (BM * CTAS) + (int)rank * BM;
                 const int col0 = (t % n_tiles) * BN + (int)rank * BNL;
-                for (int kb = 0; kb < num_kb; ++kb) {
+                // pass 1: all four tiles of a k-block per stage
+                for (int kb = 0; kb < num_kb && ok; ++kb) {
                     if (!mbar_wait(&bars->empty[s], phase ^ 1) || *abort_flag) { ok = false; break; }
                     uint8_t *st = smem + (size_t)s * stage_bytes;
                     if (rank == 0) mbar_arrive_expect_tx(&bars->full[s], stage_bytes * CTAS);
@@ -113,6 +118,22 @@ gemm_tc16_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_cons
                     tma_load_2d<CTAS>(smem_u32(st + kATileBytes), &map_a_lo, bar, kx, row0);
                     tma_load_2d<CTAS>(smem_u32(st + 2 * kATileBytes), &map_b_hi, bar, kx, col0);
                     tma_load_2d<CTAS>(smem_u32(st + 2 * kATileBytes + b_tile_bytes), &map_b_lo, bar, kx, col0);
+                    ++armed;
+                    if (++s == stages) { s = 0; phase ^= 1; }
+                }
+                // pass 2: the hi tiles of two k-blocks per stage (the second in the slots of the lo tiles)
+                for (int kb = 0; kb < num_kb && ok; kb += 2) {
+                    if (!mbar_wait(&bars->empty[s], phase ^ 1) || *abort_flag) { ok = false; break; }
+                    uint8_t *st = smem + (size_t)s * stage_bytes;
+                    const bool two = kb + 1 < num_kb;
+                    if (rank == 0) mbar_arrive_expect_tx(&bars->full[s], (two ? stage_bytes : stage_bytes / 2) * CTAS);
+                    const uint32_t bar = map_to_cta(smem_u32(&bars->full[s]), 0);
+                    tma_load_2d<CTAS>(smem_u32(st), &map_a_hi, bar, kb * BKH, row0);
+                    tma_load_2d<CTAS>(smem_u32(st + 2 * kATileBytes), &map_b_hi, bar, kb * BKH, col0);
+                    if (two) {
+                        tma_load_2d<CTAS>(smem_u32(st + kATileBytes), &map_a_hi, bar, (kb + 1) * BKH, row0);
+                        tma_load_2d<CTAS>(smem_u32(st + 2 * kATileBytes + b_tile_bytes), &map_b_hi, bar, (kb + 1) * BKH, col0);
+                    }
                     ++armed;
                     if (++s == stages) { s = 0; phase ^= 1; }
                 }
@@ -141,11 +162,14 @@ gemm_tc16_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_cons
             uint32_t phase = 0;
             bool ok = true;
             int lt = 0;
-            const uint32_t d1 = tmem_base, d2 = tmem_base + (uint32_t)BN;
             for (int t = group; t < total_tiles && ok; t += n_groups, ++lt) {
-                if (!mbar_wait(&bars->acc_empty, (lt & 1) ^ 1) || *abort_flag) { ok = false; break; }
+                const int acc = lt & 1;
+                const uint32_t acc_phase = (lt >> 1) & 1;
+                if (!mbar_wait(&bars->acc_empty[acc], acc_phase ^ 1) || *abort_flag) { ok = false; break; }
                 tcgen05_fence_after();
-                for (int kb = 0; kb < num_kb; ++kb) {
+                const uint32_t d = tmem_base + (uint32_t)(acc * BN);
+                // pass 1: cross terms
+                for (int kb = 0; kb < num_kb && ok; ++kb) {
                     if (!mbar_wait(&bars->full[s], phase) || *abort_flag) { ok = false; break; }
                     tcgen05_fence_after();
                     const uint32_t st = smem_u32(smem + (size_t)s * stage_bytes);
@@ -156,15 +180,32 @@ gemm_tc16_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_cons
 #pragma unroll
                     for (int k = 0; k < BKH / 16; ++k) {
                         const uint64_t ko = (uint64_t)(k * 2);   // 16 halves = 32 bytes = 2 x 16-byte units
-                        const uint32_t first = (kb | k) ? 1u : 0u;
-                        mma_f16<CTAS>(d2, da_lo + ko, db_hi + ko, idesc, first);
-                        mma_f16<CTAS>(d2, da_hi + ko, db_lo + ko, idesc, 1u);
-                        mma_f16<CTAS>(d1, da_hi + ko, db_hi + ko, idesc, first);
+                        mma_f16<CTAS>(d, da_lo + ko, db_hi + ko, idesc, (kb | k) ? 1u : 0u);
+                        mma_f16<CTAS>(d, da_hi + ko, db_lo + ko, idesc, 1u);
                     }
                     tcgen05_commit<CTAS>(&bars->empty[s]);
                     if (++s == stages) { s = 0; phase ^= 1; }
                 }
-                if (ok) tcgen05_commit<CTAS>(&bars->acc_full);
+                // pass 2: hi * hi on top of the cross terms scaled by 2^-11
+                for (int kb = 0; kb < num_kb && ok; kb += 2) {
+                    if (!mbar_wait(&bars->full[s], phase) || *abort_flag) { ok = false; break; }
+                    tcgen05_fence_after();
+                    const uint32_t st = smem_u32(smem + (size_t)s * stage_bytes);
+                    const int blocks = kb + 1 < num_kb ? 2 : 1;
+                    for (int h = 0; h < blocks; ++h) {
+                        const uint64_t da = make_desc(st + (uint32_t)h * kATileBytes);
+                        const uint64_t db = make_desc(st + 2 * kATileBytes + (uint32_t)h * b_tile_bytes);
+#pragma unroll
+                        for (int k = 0; k < BKH / 16; ++k) {
+                            const uint64_t ko = (uint64_t)(k * 2);
+                            if (kb == 0 && h == 0 && k == 0) mma_f16_pair_scaled<11>(d, da + ko, db + ko, idesc);
+                            else mma_f16<CTAS>(d, da + ko, db + ko, idesc, 1u);
+                        }
+                    }
+                    tcgen05_commit<CTAS>(&bars->empty[s]);
+                    if (++s == stages) { s = 0; phase ^= 1; }
+                }
+                if (ok) tcgen05_commit<CTAS>(&bars->acc_full[acc]);
             }
             if (!ok) {
                 *abort_flag = 1;
@@ -178,7 +219,7 @@ gemm_tc16_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_cons
         const int half_id = ew >> 2;                        // which of the two warps of the quarter
         uint8_t *slab_hi = epi_smem + (size_t)ew * 2 * kSlabBytes16;
         uint8_t *slab_lo = slab_hi + kSlabBytes16;
-        const uint32_t acc_empty_addr = map_to_cta(smem_u32(&bars->acc_empty), 0);
+        const uint32_t acc_empty_addr0 = map_to_cta(smem_u32(&bars->acc_empty[0]), 0);
         bool ok = true, out_of_range = false;
         int lt = 0;
         for (int t = group; t < total_tiles && ok; t += n_groups, ++lt) {
@@ -191,16 +232,17 @@ gemm_tc16_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_cons
             const int upper = (int)((rr / a.n_k) & 1);
             const size_t relax_row = (size_t)b * a.ld_n;
             float dacc = 0.0f;
-            if (!mbar_wait(&bars->acc_full, lt & 1) || *abort_flag) { ok = false; break; }
+            const int acc = lt & 1;
+            const uint32_t acc_phase = (lt >> 1) & 1;
+            if (!mbar_wait(&bars->acc_full[acc], acc_phase) || *abort_flag) { ok = false; break; }
             tcgen05_fence_after();
-            const uint32_t t_addr = tmem_base + ((uint32_t)(quarter * 32) << 16);
+            const uint32_t t_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN);
             for (int c0 = 32 * half_id; c0 < BN; c0 += 64) {
                 const int col0 = nt * BN + c0;
                 if (col0 >= a.ld_n) break;                   // warp-uniform; ld_n is a multiple of 32
-                uint32_t v1[32], v2[32];
+                uint32_t v[32];
                 __syncwarp();
-                tmem_ld32(t_addr + (uint32_t)c0, v1);
-                tmem_ld32(t_addr + (uint32_t)(BN + c0), v2);
+                tmem_ld32(t_addr + (uint32_t)c0, v);
                 tmem_ld_wait();
                 if (EPI == TC_EPI_RELU) {
                     // the slab is free again once the previous chunk's stores have read it
@@ -225,8 +267,7 @@ gemm_tc16_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_cons
                                             n4[4] = {nu.x, nu.y, nu.z, nu.w};
 #pragma unroll
                                 for (int e = 0; e < 4; ++e) {
-                                    const float c = fmaf(__uint_as_float(v2[g * 4 + e]), kLoUnscale,
-                                                         __uint_as_float(v1[g * 4 + e]));
+                                    const float c = __uint_as_float(v[g * 4 + e]);
                                     const bool nonneg = (c >= 0.0f);
                                     const bool use_lower = upper ? !nonneg : nonneg;
                                     q[e] = c * (use_lower ? l4[e] : u4[e]);
@@ -235,7 +276,7 @@ gemm_tc16_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_cons
                             } else {
 #pragma unroll
                                 for (int e = 0; e < 4; ++e)
-                                    q[e] = fmaf(__uint_as_float(v2[g * 4 + e]), kLoUnscale, __uint_as_float(v1[g * 4 + e]));
+                                    q[e] = __uint_as_float(v[g * 4 + e]);
                             }
                             dacc = fmaf(q[0], bz.x, dacc);
                             dacc = fmaf(q[1], bz.y, dacc);
@@ -278,7 +319,7 @@ gemm_tc16_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_cons
                         const float lo4[4] = {l4.x, l4.y, l4.z, l4.w}, up4[4] = {u4.x, u4.y, u4.z, u4.w};
 #pragma unroll
                         for (int e = 0; e < 4; ++e) {
-                            const float c = fmaf(__uint_as_float(v2[g * 4 + e]), kLoUnscale, __uint_as_float(v1[g * 4 + e]));
+                            const float c = __uint_as_float(v[g * 4 + e]);
                             const bool nonneg = (c >= 0.0f);
                             dacc = fmaf(c, (nonneg != (upper != 0)) ? lo4[e] : up4[e], dacc);
                         }
@@ -287,7 +328,7 @@ gemm_tc16_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_cons
             }
             tcgen05_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive_cluster(acc_empty_addr);
+            if (lane == 0) mbar_arrive_cluster(acc_empty_addr0 + (uint32_t)(acc * sizeof(uint64_t)));
             // This warp's share of the row constant (of the bound) goes to slot 2*nt + half_id; the first
             // slot also carries the constant so far.
             if (row_ok) {

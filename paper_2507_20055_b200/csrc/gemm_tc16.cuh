@@ -10,11 +10,10 @@ namespace cert {
 
 // An fp32 value x is held as hi = fp16(x) and lo = fp16(2^11 * (x - hi)): 22 bits of significand, as the
 // TF32 pair, at half the bytes and twice the tensor-core rate.  Products are exact in the fp32
-// accumulators; hi*hi goes to one accumulator, the cross terms (scaled by 2^11) to a second one, and the
-// epilogue adds them as D1 + 2^-11 * D2.  Range: |x| must stay below 65504 (a larger coefficient raises the
-// range flag, bit 1 of the status word); below 6.1e-5 the pair is exact to 1.5e-11 absolute.
+// accumulator; the cross terms (in units of 2^-11) are accumulated first and scaled by 2^-11 on the way
+// into the hi*hi pass.  Range: |x| must stay below 65504 (a larger coefficient raises the range flag,
+// bit 1 of the status word); below 6.1e-5 the pair is exact to 1.5e-11 absolute.
 constexpr float kLoScale = 2048.0f;
-constexpr float kLoUnscale = 1.0f / 2048.0f;
 
 struct Tc16Plan {
     int bn, n_tiles, stages, tmem_cols, smem_bytes;
