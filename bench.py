@@ -29,9 +29,12 @@ from paper_2507_20055_b200 import workloads as wl
 # of one launch of the ReLU-epilogue contraction, 16-box case, per row of the coefficient matrix; traffic
 # grows in proportion to the rows, so a full launch is rows x this figure).  None for workloads not captured.
 NCU_TRAFFIC_BYTES_PER_ROW = {
-    "fc6x1024_b128": {"bytes_per_row": (313.425152e6 + 215.404800e6) / 32768.0,
-                      "kernel": "gemm_tc_kernel<TC_EPI_RELU, 2>",
-                      "source": "profiles/gemm_tc_kernel_fc6x1024.md (16 boxes, scaled by rows)"},
+    ("fc6x1024_b128", "tc"): {"bytes_per_row": (313.425152e6 + 215.404800e6) / 32768.0,
+                              "kernel": "gemm_tc_kernel<TC_EPI_RELU, 2>",
+                              "source": "profiles/gemm_tc_kernel_fc6x1024.md (16 boxes, scaled by rows)"},
+    ("fc6x1024_b128", "tc16"): {"bytes_per_row": (138.941696e6 + 96.020224e6) / 32768.0,
+                                "kernel": "gemm_tc16_kernel<TC_EPI_RELU>",
+                                "source": "profiles/gemm_tc16_kernel_fc6x1024.md (16 boxes, scaled by rows)"},
 }
 
 METRIC = "input boxes/sec fully bounded (DeepPoly)"
@@ -392,8 +395,8 @@ def main():
         tc_peak = peaks["bf16_tflops_sustained"] * (1.0 if used_fp16 else 0.5) / 3.0
         used_tc = dom == "affine" and bool(net.last_contraction_paths() & 2)
         traffic, traffic_note = None, "no ncu capture for this workload / contraction mode"
-        cap = NCU_TRAFFIC_BYTES_PER_ROW.get(w.name)
-        if cap and used_tc and (net.last_contraction_paths() & 4) and not used_fp16 and not reuse:
+        cap = NCU_TRAFFIC_BYTES_PER_ROW.get((w.name, "tc16" if used_fp16 else "tc"))
+        if cap and used_tc and (net.last_contraction_paths() & 4) and not reuse and args.backsteps is None:
             rows_per_launch = 2.0 * B * max(l.n_out for l in w.layers[1:-1] or w.layers[1:])
             traffic = cap["bytes_per_row"] * rows_per_launch
             traffic_note = f"{cap['kernel']}: {cap['source']}"

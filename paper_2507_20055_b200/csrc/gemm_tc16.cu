@@ -363,7 +363,7 @@ __device__ __forceinline__ float warp_sum16(float v) {
 }
 
 // Start of a back-substitution at FC layer k as an fp16 pair: row i of W_k pushed through the ReLU below,
-// constant = b_k[i] + the nu terms + Q.b of the layer below.  One warp per row, 4 columns per lane.
+// constant = b_k[i] + the nu terms + Q.b of the layer below.  One warp per row, 8 columns per lane.
 __global__ void expr_start16_kernel(const float *__restrict__ Wk, int ldw_k, const float *__restrict__ bias_k,
                                     __half *__restrict__ Q_hi, __half *__restrict__ Q_lo, float *__restrict__ d,
                                     long long rows, int n_k, int n, int ld, int has_relu,
@@ -379,20 +379,27 @@ __global__ void expr_start16_kernel(const float *__restrict__ Wk, int ldw_k, con
     const float *ll = lamL + (size_t)b * ld, *lu = lamU + (size_t)b * ld, *nu = nuU + (size_t)b * ld;
     float dacc = 0.0f;
     bool out_of_range = false;
-    for (int t = lane * 4; t < ld; t += 128) {
-        const float4 c4 = *reinterpret_cast<const float4 *>(Wk + (size_t)i * ldw_k + t);
-        const float c[4] = {c4.x, c4.y, c4.z, c4.w};
-        const float4 bz4 = *reinterpret_cast<const float4 *>(bias_below + t);
-        const float bz[4] = {bz4.x, bz4.y, bz4.z, bz4.w};
-        float q[4];
+    // eight consecutive columns per lane: 16-byte stores of halves (row pitches are multiples of 32 elements)
+    for (int t = lane * 8; t < ld; t += 256) {
+        float c[8], bz[8], q[8];
+        {
+            const float4 x0 = *reinterpret_cast<const float4 *>(Wk + (size_t)i * ldw_k + t);
+            const float4 x1 = *reinterpret_cast<const float4 *>(Wk + (size_t)i * ldw_k + t + 4);
+            c[0] = x0.x; c[1] = x0.y; c[2] = x0.z; c[3] = x0.w; c[4] = x1.x; c[5] = x1.y; c[6] = x1.z; c[7] = x1.w;
+            const float4 y0 = *reinterpret_cast<const float4 *>(bias_below + t);
+            const float4 y1 = *reinterpret_cast<const float4 *>(bias_below + t + 4);
+            bz[0] = y0.x; bz[1] = y0.y; bz[2] = y0.z; bz[3] = y0.w; bz[4] = y1.x; bz[5] = y1.y; bz[6] = y1.z; bz[7] = y1.w;
+        }
         if (has_relu) {
-            const float4 l4 = *reinterpret_cast<const float4 *>(ll + t);
-            const float4 u4 = *reinterpret_cast<const float4 *>(lu + t);
-            const float4 n4 = *reinterpret_cast<const float4 *>(nu + t);
-            const float la[4] = {l4.x, l4.y, l4.z, l4.w}, ua[4] = {u4.x, u4.y, u4.z, u4.w},
-                        na[4] = {n4.x, n4.y, n4.z, n4.w};
+            float la[8], ua[8], na[8];
+            const float4 l0 = *reinterpret_cast<const float4 *>(ll + t), l1 = *reinterpret_cast<const float4 *>(ll + t + 4);
+            const float4 u0 = *reinterpret_cast<const float4 *>(lu + t), u1 = *reinterpret_cast<const float4 *>(lu + t + 4);
+            const float4 n0 = *reinterpret_cast<const float4 *>(nu + t), n1 = *reinterpret_cast<const float4 *>(nu + t + 4);
+            la[0] = l0.x; la[1] = l0.y; la[2] = l0.z; la[3] = l0.w; la[4] = l1.x; la[5] = l1.y; la[6] = l1.z; la[7] = l1.w;
+            ua[0] = u0.x; ua[1] = u0.y; ua[2] = u0.z; ua[3] = u0.w; ua[4] = u1.x; ua[5] = u1.y; ua[6] = u1.z; ua[7] = u1.w;
+            na[0] = n0.x; na[1] = n0.y; na[2] = n0.z; na[3] = n0.w; na[4] = n1.x; na[5] = n1.y; na[6] = n1.z; na[7] = n1.w;
 #pragma unroll
-            for (int e = 0; e < 4; ++e) {
+            for (int e = 0; e < 8; ++e) {
                 q[e] = 0.0f;
                 if (t + e < n) {
                     const bool nonneg = (c[e] >= 0.0f);
@@ -403,23 +410,24 @@ __global__ void expr_start16_kernel(const float *__restrict__ Wk, int ldw_k, con
             }
         } else {
 #pragma unroll
-            for (int e = 0; e < 4; ++e) q[e] = (t + e < n) ? c[e] : 0.0f;
+            for (int e = 0; e < 8; ++e) q[e] = (t + e < n) ? c[e] : 0.0f;
         }
-        __half h[4], l[4];
+        uint32_t ph[4], pl[4];
 #pragma unroll
-        for (int e = 0; e < 4; ++e) {
-            dacc = fmaf(q[e], bz[e], dacc);
-            out_of_range |= !(fabsf(q[e]) <= 60000.0f);
-            h[e] = __float2half_rn(q[e]);
-            l[e] = __float2half_rn((q[e] - __half2float(h[e])) * kLoScale);
+        for (int e = 0; e < 8; e += 2) {
+            __half h[2], l[2];
+#pragma unroll
+            for (int z = 0; z < 2; ++z) {
+                dacc = fmaf(q[e + z], bz[e + z], dacc);
+                out_of_range |= !(fabsf(q[e + z]) <= 60000.0f);
+                h[z] = __float2half_rn(q[e + z]);
+                l[z] = __float2half_rn((q[e + z] - __half2float(h[z])) * kLoScale);
+            }
+            ph[e >> 1] = (uint32_t)__half_as_ushort(h[0]) | ((uint32_t)__half_as_ushort(h[1]) << 16);
+            pl[e >> 1] = (uint32_t)__half_as_ushort(l[0]) | ((uint32_t)__half_as_ushort(l[1]) << 16);
         }
-        uint2 ph, pl;
-        ph.x = (uint32_t)__half_as_ushort(h[0]) | ((uint32_t)__half_as_ushort(h[1]) << 16);
-        ph.y = (uint32_t)__half_as_ushort(h[2]) | ((uint32_t)__half_as_ushort(h[3]) << 16);
-        pl.x = (uint32_t)__half_as_ushort(l[0]) | ((uint32_t)__half_as_ushort(l[1]) << 16);
-        pl.y = (uint32_t)__half_as_ushort(l[2]) | ((uint32_t)__half_as_ushort(l[3]) << 16);
-        *reinterpret_cast<uint2 *>(Q_hi + (size_t)r * ld + t) = ph;
-        *reinterpret_cast<uint2 *>(Q_lo + (size_t)r * ld + t) = pl;
+        *reinterpret_cast<uint4 *>(Q_hi + (size_t)r * ld + t) = make_uint4(ph[0], ph[1], ph[2], ph[3]);
+        *reinterpret_cast<uint4 *>(Q_lo + (size_t)r * ld + t) = make_uint4(pl[0], pl[1], pl[2], pl[3]);
     }
     dacc = warp_sum16(dacc);
     if (lane == 0) d[r] = bias_k[i] + dacc;
