@@ -363,41 +363,57 @@ __device__ __forceinline__ float warp_sum16(float v) {
 }
 
 // Start of a back-substitution at FC layer k as an fp16 pair: row i of W_k pushed through the ReLU below,
-// constant = b_k[i] + the nu terms + Q.b of the layer below.  One warp per row, 8 columns per lane.
+// constant = b_k[i] + the nu terms + Q.b of the layer below.  A warp takes kRowsPerWarp consecutive neurons
+// of one (box, side), 8 columns per lane: the relaxation and bias vectors are read once for those rows.
+constexpr int kRowsPerWarp = 4;
+
 __global__ void expr_start16_kernel(const float *__restrict__ Wk, int ldw_k, const float *__restrict__ bias_k,
                                     __half *__restrict__ Q_hi, __half *__restrict__ Q_lo, float *__restrict__ d,
-                                    long long rows, int n_k, int n, int ld, int has_relu,
+                                    long long n_warps, int n_k, int n, int ld, int has_relu,
                                     const float *__restrict__ lamL, const float *__restrict__ lamU,
                                     const float *__restrict__ nuU, const float *__restrict__ bias_below,
                                     int *__restrict__ status) {
-    const long long r = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const long long w = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int lane = threadIdx.x & 31;
-    if (r >= rows) return;
-    const int b = (int)(r / (2LL * n_k));
-    const int upper = (int)((r / n_k) & 1);
-    const int i = (int)(r % n_k);
+    if (w >= n_warps) return;
+    const int chunks = (n_k + kRowsPerWarp - 1) / kRowsPerWarp;
+    const long long grp = w / chunks;                  // (box, side)
+    const int i0 = (int)(w % chunks) * kRowsPerWarp;
+    const int b = (int)(grp >> 1);
+    const int upper = (int)(grp & 1);
+    const long long r0 = grp * n_k + i0;               // row of neuron i0
     const float *ll = lamL + (size_t)b * ld, *lu = lamU + (size_t)b * ld, *nu = nuU + (size_t)b * ld;
-    float dacc = 0.0f;
+    float dacc[kRowsPerWarp];
+#pragma unroll
+    for (int rr = 0; rr < kRowsPerWarp; ++rr) dacc[rr] = 0.0f;
     bool out_of_range = false;
     // eight consecutive columns per lane: 16-byte stores of halves (row pitches are multiples of 32 elements)
     for (int t = lane * 8; t < ld; t += 256) {
-        float c[8], bz[8], q[8];
+        float bz[8], la[8], ua[8], na[8];
         {
-            const float4 x0 = *reinterpret_cast<const float4 *>(Wk + (size_t)i * ldw_k + t);
-            const float4 x1 = *reinterpret_cast<const float4 *>(Wk + (size_t)i * ldw_k + t + 4);
-            c[0] = x0.x; c[1] = x0.y; c[2] = x0.z; c[3] = x0.w; c[4] = x1.x; c[5] = x1.y; c[6] = x1.z; c[7] = x1.w;
             const float4 y0 = *reinterpret_cast<const float4 *>(bias_below + t);
             const float4 y1 = *reinterpret_cast<const float4 *>(bias_below + t + 4);
             bz[0] = y0.x; bz[1] = y0.y; bz[2] = y0.z; bz[3] = y0.w; bz[4] = y1.x; bz[5] = y1.y; bz[6] = y1.z; bz[7] = y1.w;
         }
         if (has_relu) {
-            float la[8], ua[8], na[8];
             const float4 l0 = *reinterpret_cast<const float4 *>(ll + t), l1 = *reinterpret_cast<const float4 *>(ll + t + 4);
             const float4 u0 = *reinterpret_cast<const float4 *>(lu + t), u1 = *reinterpret_cast<const float4 *>(lu + t + 4);
             const float4 n0 = *reinterpret_cast<const float4 *>(nu + t), n1 = *reinterpret_cast<const float4 *>(nu + t + 4);
             la[0] = l0.x; la[1] = l0.y; la[2] = l0.z; la[3] = l0.w; la[4] = l1.x; la[5] = l1.y; la[6] = l1.z; la[7] = l1.w;
             ua[0] = u0.x; ua[1] = u0.y; ua[2] = u0.z; ua[3] = u0.w; ua[4] = u1.x; ua[5] = u1.y; ua[6] = u1.z; ua[7] = u1.w;
             na[0] = n0.x; na[1] = n0.y; na[2] = n0.z; na[3] = n0.w; na[4] = n1.x; na[5] = n1.y; na[6] = n1.z; na[7] = n1.w;
+        } else {
+#pragma unroll
+            for (int e = 0; e < 8; ++e) { la[e] = ua[e] = 1.0f; na[e] = 0.0f; }
+        }
+#pragma unroll
+        for (int rr = 0; rr < kRowsPerWarp; ++rr) {
+            if (i0 + rr >= n_k) break;
+            float c[8], q[8];
+            const float *wrow = Wk + (size_t)(i0 + rr) * ldw_k + t;
+            const float4 x0 = *reinterpret_cast<const float4 *>(wrow);
+            const float4 x1 = *reinterpret_cast<const float4 *>(wrow + 4);
+            c[0] = x0.x; c[1] = x0.y; c[2] = x0.z; c[3] = x0.w; c[4] = x1.x; c[5] = x1.y; c[6] = x1.z; c[7] = x1.w;
 #pragma unroll
             for (int e = 0; e < 8; ++e) {
                 q[e] = 0.0f;
@@ -405,32 +421,32 @@ __global__ void expr_start16_kernel(const float *__restrict__ Wk, int ldw_k, con
                     const bool nonneg = (c[e] >= 0.0f);
                     const bool use_lower = upper ? !nonneg : nonneg;
                     q[e] = c[e] * (use_lower ? la[e] : ua[e]);
-                    if (!use_lower) dacc = fmaf(c[e], na[e], dacc);
+                    if (!use_lower) dacc[rr] = fmaf(c[e], na[e], dacc[rr]);
                 }
             }
-        } else {
+            uint32_t ph[4], pl[4];
 #pragma unroll
-            for (int e = 0; e < 8; ++e) q[e] = (t + e < n) ? c[e] : 0.0f;
-        }
-        uint32_t ph[4], pl[4];
+            for (int e = 0; e < 8; e += 2) {
+                __half h[2], l[2];
 #pragma unroll
-        for (int e = 0; e < 8; e += 2) {
-            __half h[2], l[2];
-#pragma unroll
-            for (int z = 0; z < 2; ++z) {
-                dacc = fmaf(q[e + z], bz[e + z], dacc);
-                out_of_range |= !(fabsf(q[e + z]) <= 60000.0f);
-                h[z] = __float2half_rn(q[e + z]);
-                l[z] = __float2half_rn((q[e + z] - __half2float(h[z])) * kLoScale);
+                for (int z = 0; z < 2; ++z) {
+                    dacc[rr] = fmaf(q[e + z], bz[e + z], dacc[rr]);
+                    out_of_range |= !(fabsf(q[e + z]) <= 60000.0f);
+                    h[z] = __float2half_rn(q[e + z]);
+                    l[z] = __float2half_rn((q[e + z] - __half2float(h[z])) * kLoScale);
+                }
+                ph[e >> 1] = (uint32_t)__half_as_ushort(h[0]) | ((uint32_t)__half_as_ushort(h[1]) << 16);
+                pl[e >> 1] = (uint32_t)__half_as_ushort(l[0]) | ((uint32_t)__half_as_ushort(l[1]) << 16);
             }
-            ph[e >> 1] = (uint32_t)__half_as_ushort(h[0]) | ((uint32_t)__half_as_ushort(h[1]) << 16);
-            pl[e >> 1] = (uint32_t)__half_as_ushort(l[0]) | ((uint32_t)__half_as_ushort(l[1]) << 16);
+            *reinterpret_cast<uint4 *>(Q_hi + (size_t)(r0 + rr) * ld + t) = make_uint4(ph[0], ph[1], ph[2], ph[3]);
+            *reinterpret_cast<uint4 *>(Q_lo + (size_t)(r0 + rr) * ld + t) = make_uint4(pl[0], pl[1], pl[2], pl[3]);
         }
-        *reinterpret_cast<uint4 *>(Q_hi + (size_t)r * ld + t) = make_uint4(ph[0], ph[1], ph[2], ph[3]);
-        *reinterpret_cast<uint4 *>(Q_lo + (size_t)r * ld + t) = make_uint4(pl[0], pl[1], pl[2], pl[3]);
     }
-    dacc = warp_sum16(dacc);
-    if (lane == 0) d[r] = bias_k[i] + dacc;
+#pragma unroll
+    for (int rr = 0; rr < kRowsPerWarp; ++rr) {
+        const float tot = warp_sum16(dacc[rr]);
+        if (lane == 0 && i0 + rr < n_k) d[r0 + rr] = bias_k[i0 + rr] + tot;
+    }
     if (__any_sync(0xffffffffu, out_of_range) && lane == 0) atomicOr(status, 2);
 }
 
@@ -526,9 +542,9 @@ void launch_gemm_tc16(int epi, int pairs, const TcMap &a_hi, const TcMap &a_lo, 
 
 void launch_init_expr16(const LayerDev &Lk, const LayerDev &Lb, int batch, __half *Q_hi, __half *Q_lo, float *d,
                         int *status, cudaStream_t st) {
-    const long long rows = 2LL * batch * Lk.n_out;
-    expr_start16_kernel<<<(unsigned)ceil_div_ll(rows, 8), 256, 0, st>>>(
-        Lk.W, Lk.ld_in, Lk.bias_n, Q_hi, Q_lo, d, rows, Lk.n_out, Lb.n_out, Lb.ld_out, Lb.relu_after, Lb.lamL,
+    const long long n_warps = 2LL * batch * ((Lk.n_out + kRowsPerWarp - 1) / kRowsPerWarp);
+    expr_start16_kernel<<<(unsigned)ceil_div_ll(n_warps, 8), 256, 0, st>>>(
+        Lk.W, Lk.ld_in, Lk.bias_n, Q_hi, Q_lo, d, n_warps, Lk.n_out, Lb.n_out, Lb.ld_out, Lb.relu_after, Lb.lamL,
         Lb.lamU, Lb.nuU, Lb.bias_n, status);
 }
 
