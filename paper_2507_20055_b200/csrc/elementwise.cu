@@ -210,10 +210,80 @@ __global__ void conv_expr_start_kernel(const float *__restrict__ Wk, ConvGeom gk
     if (lane == 0) d[r] = bias_k[i] + dacc;
 }
 
-// FROM_WEIGHTS: source is row i of the FC layer W_k (start of a back-substitution), else P in place.
-template <bool FROM_WEIGHTS>
-__global__ void relu_step_kernel(const float *__restrict__ Wk, int kind_k, ConvGeom gk, int ldw_k,
-                                 const float *__restrict__ bias_k, float *__restrict__ P,
+// Start of a back-substitution at FC layer k: row i of W_k pushed through the ReLU below, constant =
+// b_k[i] + the nu terms + Q.b of the layer below.  A warp takes kStartRows consecutive neurons of one
+// (box, side), 4 columns per lane, so the relaxation and bias vectors are read once for those rows.
+// Q_lo != nullptr: the row is written as a TF32 pair.
+constexpr int kStartRows = 4;
+
+__global__ void fc_expr_start_kernel(const float *__restrict__ Wk, int ldw_k, const float *__restrict__ bias_k,
+                                     float *__restrict__ Q, float *__restrict__ Q_lo, float *__restrict__ d,
+                                     long long n_warps, int n_k, int n, int ld, int has_relu,
+                                     const float *__restrict__ lamL, const float *__restrict__ lamU,
+                                     const float *__restrict__ nuU, const float *__restrict__ bias_below) {
+    const long long w = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int lane = threadIdx.x & 31;
+    if (w >= n_warps) return;
+    const int chunks = (n_k + kStartRows - 1) / kStartRows;
+    const long long grp = w / chunks;                  // (box, side)
+    const int i0 = (int)(w % chunks) * kStartRows;
+    const int b = (int)(grp >> 1);
+    const int upper = (int)(grp & 1);
+    const long long r0 = grp * n_k + i0;
+    const float *ll = lamL + (size_t)b * ld, *lu = lamU + (size_t)b * ld, *nu = nuU + (size_t)b * ld;
+    float dacc[kStartRows];
+#pragma unroll
+    for (int rr = 0; rr < kStartRows; ++rr) dacc[rr] = 0.0f;
+    for (int t = lane * 4; t < ld; t += 128) {
+        const float4 bz4 = *reinterpret_cast<const float4 *>(bias_below + t);
+        const float bz[4] = {bz4.x, bz4.y, bz4.z, bz4.w};
+        float la[4] = {1.f, 1.f, 1.f, 1.f}, ua[4] = {1.f, 1.f, 1.f, 1.f}, na[4] = {0.f, 0.f, 0.f, 0.f};
+        if (has_relu) {
+            const float4 l4 = *reinterpret_cast<const float4 *>(ll + t);
+            const float4 u4 = *reinterpret_cast<const float4 *>(lu + t);
+            const float4 n4 = *reinterpret_cast<const float4 *>(nu + t);
+            la[0] = l4.x; la[1] = l4.y; la[2] = l4.z; la[3] = l4.w;
+            ua[0] = u4.x; ua[1] = u4.y; ua[2] = u4.z; ua[3] = u4.w;
+            na[0] = n4.x; na[1] = n4.y; na[2] = n4.z; na[3] = n4.w;
+        }
+#pragma unroll
+        for (int rr = 0; rr < kStartRows; ++rr) {
+            if (i0 + rr >= n_k) break;
+            const float4 c4 = *reinterpret_cast<const float4 *>(Wk + (size_t)(i0 + rr) * ldw_k + t);
+            const float c[4] = {c4.x, c4.y, c4.z, c4.w};
+            float q[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                q[e] = 0.0f;
+                if (t + e < n) q[e] = has_relu ? relu_backstep(c[e], upper, la[e], ua[e], na[e], dacc[rr]) : c[e];
+                dacc[rr] = fmaf(q[e], bz[e], dacc[rr]);
+            }
+            float *qrow = Q + (size_t)(r0 + rr) * ld + t;
+            if (Q_lo) {
+                float h[4], l[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    h[e] = tf32_round(q[e]);
+                    l[e] = tf32_round(q[e] - h[e]);
+                }
+                *reinterpret_cast<float4 *>(qrow) = make_float4(h[0], h[1], h[2], h[3]);
+                *reinterpret_cast<float4 *>(Q_lo + (size_t)(r0 + rr) * ld + t) = make_float4(l[0], l[1], l[2], l[3]);
+            } else {
+                *reinterpret_cast<float4 *>(qrow) = make_float4(q[0], q[1], q[2], q[3]);
+            }
+        }
+    }
+#pragma unroll
+    for (int rr = 0; rr < kStartRows; ++rr) {
+        const float tot = warp_sum(dacc[rr]);
+        if (lane == 0 && i0 + rr < n_k) d[r0 + rr] = bias_k[i0 + rr] + tot;
+    }
+}
+
+// ReLU back-step in place on P (expression over a layer's outputs), plus the constant's share Q.b of the
+// affine step that follows; the constant comes in as a sum of slots and leaves in slot 0.
+
+__global__ void relu_step_kernel(float *__restrict__ P,
                                  float *__restrict__ P_lo, float *__restrict__ d, int n_slots,
                                  long long slot_stride, long long rows, int n_k, int n, int ld, int has_relu,
                                  const float *__restrict__ lamL, const float *__restrict__ lamU,
@@ -223,7 +293,6 @@ __global__ void relu_step_kernel(const float *__restrict__ Wk, int kind_k, ConvG
     if (r >= rows) return;
     int b = (int)(r / (2LL * n_k));
     int upper = (int)((r / n_k) & 1);
-    int i = (int)(r % n_k);
     float *prow = P + (size_t)r * ld;
     const float *ll = lamL + (size_t)b * ld, *lu = lamU + (size_t)b * ld, *nu = nuU + (size_t)b * ld;
     float dacc = 0.0f;
@@ -231,7 +300,7 @@ __global__ void relu_step_kernel(const float *__restrict__ Wk, int kind_k, ConvG
     for (int t = lane * 4; t < ld; t += 128) {
         float c[4], q[4];
         {
-            const float4 c4 = *reinterpret_cast<const float4 *>(FROM_WEIGHTS ? Wk + (size_t)i * ldw_k + t : prow + t);
+            const float4 c4 = *reinterpret_cast<const float4 *>(prow + t);
             c[0] = c4.x; c[1] = c4.y; c[2] = c4.z; c[3] = c4.w;
         }
         const float4 bz4 = *reinterpret_cast<const float4 *>(bias_below + t);
@@ -265,7 +334,7 @@ __global__ void relu_step_kernel(const float *__restrict__ Wk, int kind_k, ConvG
         }
     }
     dacc = warp_sum(dacc);
-    if (lane == 0) d[r] = (FROM_WEIGHTS ? bias_k[i] : slot_sum(d, n_slots, slot_stride, r)) + dacc;
+    if (lane == 0) d[r] = slot_sum(d, n_slots, slot_stride, r) + dacc;
 }
 
 __global__ void concretize_kernel(const float *__restrict__ P, const float *__restrict__ d, int n_slots,
@@ -332,16 +401,17 @@ void launch_init_expr(const LayerDev &Lk, const LayerDev &Lb, int batch, float *
             Lb.nuU, Lb.bias_n);
         return;
     }
-    relu_step_kernel<true><<<grid_for_warps(rows), kWarpsPerBlock * 32, 0, st>>>(
-        Lk.W, Lk.kind, geom_of(Lk), Lk.ld_in, Lk.bias_n, Q, Q_lo, d, 1, 0, rows, Lk.n_out, Lb.n_out, Lb.ld_out,
-        Lb.relu_after, Lb.lamL, Lb.lamU, Lb.nuU, Lb.bias_n);
+    const long long n_warps = 2LL * batch * ((Lk.n_out + kStartRows - 1) / kStartRows);
+    fc_expr_start_kernel<<<grid_for_warps(n_warps), kWarpsPerBlock * 32, 0, st>>>(
+        Lk.W, Lk.ld_in, Lk.bias_n, Q, Q_lo, d, n_warps, Lk.n_out, Lb.n_out, Lb.ld_out, Lb.relu_after, Lb.lamL,
+        Lb.lamU, Lb.nuU, Lb.bias_n);
 }
 
 void launch_relu_step(const LayerDev &Lj, int batch, int n_k, float *P, float *P_lo, float *d, int n_slots,
                       long long slot_stride, cudaStream_t st) {
     long long rows = 2LL * batch * n_k;
-    relu_step_kernel<false><<<grid_for_warps(rows), kWarpsPerBlock * 32, 0, st>>>(
-        nullptr, 0, ConvGeom{}, 0, nullptr, P, P_lo, d, n_slots, slot_stride, rows, n_k, Lj.n_out, Lj.ld_out, Lj.relu_after, Lj.lamL,
+    relu_step_kernel<<<grid_for_warps(rows), kWarpsPerBlock * 32, 0, st>>>(
+        P, P_lo, d, n_slots, slot_stride, rows, n_k, Lj.n_out, Lj.ld_out, Lj.relu_after, Lj.lamL,
         Lj.lamU, Lj.nuU, Lj.bias_n);
 }
 
