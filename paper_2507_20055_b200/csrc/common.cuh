@@ -6,6 +6,7 @@
 #include <cuda_runtime.h>
 #include <cstdint>
 #include <cstdio>
+#include <utility>
 #include "../../include/cert.h"
 
 namespace cert {
@@ -13,6 +14,32 @@ namespace cert {
 constexpr int kPad = 32;  // every row of a coefficient / weight / relaxation array is padded to 32 floats
 
 inline int round_up(int x, int m) { return (x + m - 1) / m * m; }
+
+// Programmatic dependent launch for the chain of small dependent kernels of a call: a kernel lets the next one
+// be scheduled as soon as all of its own blocks have started (pdl_trigger), and touches global memory only
+// after the kernel before it has completed and flushed (pdl_wait).  Launch latency and each kernel's
+// set-up (barriers, tensor memory) then overlap the tail of the kernel before.  Both are no-ops for a kernel
+// launched without the attribute.
+#ifdef __CUDACC__
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+#endif
+bool pdl_enabled();   // false when the environment variable CERT_PDL is 0
+
+template <typename Kernel, typename... Args>
+inline void launch_chained(Kernel kernel, dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args &&...args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = pdl_enabled() ? 1 : 0;
+    cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+}
 inline long long ceil_div_ll(long long a, long long b) { return (a + b - 1) / b; }
 
 // One affine layer on the device.

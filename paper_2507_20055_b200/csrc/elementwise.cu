@@ -3,6 +3,8 @@
 // ReLU back-step and the unfused concretisation.  One warp owns one row of a
 // coefficient matrix; row sums are warp-shuffle trees, so every result is
 // deterministic.
+#include <cstdlib>
+
 #include "common.cuh"
 
 namespace cert {
@@ -37,6 +39,8 @@ __device__ __forceinline__ float relu_backstep(float c, int upper, float lamL, f
 
 __global__ void box_kernel(const float *__restrict__ centers, float eps, float lo, float hi, int batch,
                            int n0, int ld0, float *__restrict__ l0, float *__restrict__ u0) {
+    pdl_trigger();
+    pdl_wait();
     long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (idx >= (long long)batch * ld0) return;
     int b = (int)(idx / ld0), s = (int)(idx % ld0);
@@ -55,6 +59,8 @@ __global__ void first_layer_kernel(const float *__restrict__ W, const float *__r
                                    ConvGeom g, int n_in, int ld_in, int n_out, const float *__restrict__ l0,
                                    const float *__restrict__ u0, int ld0, int batch, float *__restrict__ lb_out,
                                    float *__restrict__ ub_out, int n_total, int out_off) {
+    pdl_trigger();
+    pdl_wait();
     long long warp = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     int lane = threadIdx.x & 31;
     if (warp >= (long long)batch * n_out) return;
@@ -114,6 +120,8 @@ __global__ void relax_kernel(float *__restrict__ lb_out, float *__restrict__ ub_
                              unsigned char *__restrict__ codes, int n_relu, int relu_off,
                              const float *__restrict__ slots, int n_slots, long long slot_stride,
                              int do_relax) {
+    pdl_trigger();
+    pdl_wait();
     long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (idx >= (long long)batch * ld) return;
     int b = (int)(idx / ld), t = (int)(idx % ld);
@@ -221,6 +229,8 @@ __global__ void fc_expr_start_kernel(const float *__restrict__ Wk, int ldw_k, co
                                      long long n_warps, int n_k, int n, int ld, int has_relu,
                                      const float *__restrict__ lamL, const float *__restrict__ lamU,
                                      const float *__restrict__ nuU, const float *__restrict__ bias_below) {
+    pdl_trigger();
+    pdl_wait();
     const long long w = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int lane = threadIdx.x & 31;
     if (w >= n_warps) return;
@@ -368,28 +378,35 @@ inline unsigned grid_for_warps(long long warps) {
 
 }  // namespace
 
+bool pdl_enabled() {
+    static const bool on = [] {
+        const char *e = std::getenv("CERT_PDL");
+        return !(e && e[0] == '0');
+    }();
+    return on;
+}
+
 void launch_box(const float *centers, float eps, float lo, float hi, int batch, int n0, int ld0, float *l0,
                 float *u0, cudaStream_t st) {
     long long n = (long long)batch * ld0;
-    box_kernel<<<(unsigned)ceil_div_ll(n, 256), 256, 0, st>>>(centers, eps, lo, hi, batch, n0, ld0, l0, u0);
+    launch_chained(box_kernel, dim3((unsigned)ceil_div_ll(n, 256)), dim3(256), 0, st, centers, eps, lo, hi, batch, n0, ld0,
+                   l0, u0);
 }
 
 void launch_first_layer_bounds(const LayerDev &L, const float *l0, const float *u0, int ld0, int batch,
                                float *lb_out, float *ub_out, int n_total, cudaStream_t st) {
     long long warps = (long long)batch * L.n_out;
-    first_layer_kernel<<<grid_for_warps(warps), kWarpsPerBlock * 32, 0, st>>>(
-        L.W, L.bias_n, L.kind, geom_of(L), L.n_in, L.ld_in, L.n_out, l0, u0, ld0, batch, lb_out, ub_out,
-        n_total, L.out_off);
+    launch_chained(first_layer_kernel, dim3(grid_for_warps(warps)), dim3(kWarpsPerBlock * 32), 0, st, L.W, L.bias_n,
+                   L.kind, geom_of(L), L.n_in, L.ld_in, L.n_out, l0, u0, ld0, batch, lb_out, ub_out, n_total, L.out_off);
 }
 
 void launch_relax(const LayerDev &L, float *lb_out, float *ub_out, int n_total, int batch,
                   unsigned char *codes, int n_relu, const float *slots, int n_slots, long long slot_stride,
                   cudaStream_t st) {
     long long n = (long long)batch * L.ld_out;
-    relax_kernel<<<(unsigned)ceil_div_ll(n, 256), 256, 0, st>>>(lb_out, ub_out, n_total, L.out_off, L.n_out,
-                                                               L.ld_out, batch, L.lamL, L.lamU, L.nuU, L.actL,
-                                                               L.actU, codes, n_relu, L.relu_off, slots, n_slots,
-                                                               slot_stride, L.relu_after);
+    launch_chained(relax_kernel, dim3((unsigned)ceil_div_ll(n, 256)), dim3(256), 0, st, lb_out, ub_out, n_total,
+                   L.out_off, L.n_out, L.ld_out, batch, L.lamL, L.lamU, L.nuU, L.actL, L.actU, codes, n_relu, L.relu_off,
+                   slots, n_slots, slot_stride, L.relu_after);
 }
 
 void launch_init_expr(const LayerDev &Lk, const LayerDev &Lb, int batch, float *Q, float *Q_lo, float *d,
@@ -402,9 +419,9 @@ void launch_init_expr(const LayerDev &Lk, const LayerDev &Lb, int batch, float *
         return;
     }
     const long long n_warps = 2LL * batch * ((Lk.n_out + kStartRows - 1) / kStartRows);
-    fc_expr_start_kernel<<<grid_for_warps(n_warps), kWarpsPerBlock * 32, 0, st>>>(
-        Lk.W, Lk.ld_in, Lk.bias_n, Q, Q_lo, d, n_warps, Lk.n_out, Lb.n_out, Lb.ld_out, Lb.relu_after, Lb.lamL,
-        Lb.lamU, Lb.nuU, Lb.bias_n);
+    launch_chained(fc_expr_start_kernel, dim3(grid_for_warps(n_warps)), dim3(kWarpsPerBlock * 32), 0, st, Lk.W, Lk.ld_in,
+                   Lk.bias_n, Q, Q_lo, d, n_warps, Lk.n_out, Lb.n_out, Lb.ld_out, Lb.relu_after, Lb.lamL, Lb.lamU, Lb.nuU,
+                   Lb.bias_n);
 }
 
 void launch_relu_step(const LayerDev &Lj, int batch, int n_k, float *P, float *P_lo, float *d, int n_slots,

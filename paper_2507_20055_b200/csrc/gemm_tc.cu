@@ -57,6 +57,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_consta
                const __grid_constant__ CUtensorMap map_b_hi, const __grid_constant__ CUtensorMap map_b_lo,
                const __grid_constant__ CUtensorMap map_o_hi, const __grid_constant__ CUtensorMap map_o_lo,
                const TcArgs a) {
+    pdl_trigger();
     extern __shared__ uint8_t smem_raw[];
     // tiles are aligned to 1024 bytes (a whole swizzle pattern)
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -108,6 +109,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_consta
     __syncthreads();
     if (CTAS == 2) cluster_sync_all();      // the peer's barriers exist before anything arrives on them
     tcgen05_fence_after();
+    pdl_wait();                             // everything above needed nothing from the kernel before
     const uint32_t tmem_base = bars->tmem_base;
     volatile uint32_t *abort_flag = &bars->abort_flag;
 
@@ -400,13 +402,15 @@ void launch_one(int groups, const CUtensorMap &ah, const CUtensorMap &al, const 
     cfg.blockDim = dim3(kThreads, 1, 1);
     cfg.dynamicSmemBytes = (size_t)smem_bytes;
     cfg.stream = st;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = CTAS;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = pdl_enabled() ? 2 : 1;
     cudaLaunchKernelEx(&cfg, gemm_tc_kernel<EPI, CTAS>, ah, al, bh, bl, oh, ol, args);
 }
 

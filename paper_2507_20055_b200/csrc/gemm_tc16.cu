@@ -52,6 +52,7 @@ gemm_tc16_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_cons
                  const __grid_constant__ CUtensorMap map_o_hi, const __grid_constant__ CUtensorMap map_o_lo,
                  const TcArgs a) {
     constexpr int CTAS = 2;
+    pdl_trigger();
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const int BN = a.bn;
@@ -94,6 +95,7 @@ gemm_tc16_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_cons
     __syncthreads();
     cluster_sync_all();      // the peer's barriers exist before anything arrives on them
     tcgen05_fence_after();
+    pdl_wait();              // everything above needed nothing from the kernel before
     const uint32_t tmem_base = bars->tmem_base;
     volatile uint32_t *abort_flag = &bars->abort_flag;
 
@@ -373,6 +375,8 @@ __global__ void expr_start16_kernel(const float *__restrict__ Wk, int ldw_k, con
                                     const float *__restrict__ lamL, const float *__restrict__ lamU,
                                     const float *__restrict__ nuU, const float *__restrict__ bias_below,
                                     int *__restrict__ status) {
+    pdl_trigger();
+    pdl_wait();
     const long long w = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int lane = threadIdx.x & 31;
     if (w >= n_warps) return;
@@ -465,13 +469,15 @@ void launch_one16(int pairs, const CUtensorMap &ah, const CUtensorMap &al, const
     cfg.blockDim = dim3(kThreads16, 1, 1);
     cfg.dynamicSmemBytes = (size_t)smem_bytes;
     cfg.stream = st;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = 2;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = pdl_enabled() ? 2 : 1;
     cudaLaunchKernelEx(&cfg, gemm_tc16_kernel<EPI>, ah, al, bh, bl, oh, ol, args);
 }
 
@@ -543,9 +549,9 @@ void launch_gemm_tc16(int epi, int pairs, const TcMap &a_hi, const TcMap &a_lo, 
 void launch_init_expr16(const LayerDev &Lk, const LayerDev &Lb, int batch, __half *Q_hi, __half *Q_lo, float *d,
                         int *status, cudaStream_t st) {
     const long long n_warps = 2LL * batch * ((Lk.n_out + kRowsPerWarp - 1) / kRowsPerWarp);
-    expr_start16_kernel<<<(unsigned)ceil_div_ll(n_warps, 8), 256, 0, st>>>(
-        Lk.W, Lk.ld_in, Lk.bias_n, Q_hi, Q_lo, d, n_warps, Lk.n_out, Lb.n_out, Lb.ld_out, Lb.relu_after, Lb.lamL,
-        Lb.lamU, Lb.nuU, Lb.bias_n, status);
+    launch_chained(expr_start16_kernel, dim3((unsigned)ceil_div_ll(n_warps, 8)), dim3(256), 0, st, Lk.W, Lk.ld_in,
+                   Lk.bias_n, Q_hi, Q_lo, d, n_warps, Lk.n_out, Lb.n_out, Lb.ld_out, Lb.relu_after, Lb.lamL, Lb.lamU, Lb.nuU,
+                   Lb.bias_n, status);
 }
 
 }  // namespace cert
