@@ -253,7 +253,7 @@ def main():
             "tc16": binding.CONTRACTION_TC3XFP16}
     if args.contraction == "fastest":
         all_fc = all(l.kind == "fc" for l in w.layers)
-        args.contraction = "tc16" if (all_fc and len(w.layers) > 1 and args.certifier != "reusecert") else "auto"
+        args.contraction = "tc16" if (all_fc and len(w.layers) > 1) else "auto"
     net.set_contraction(mode[args.contraction])
     stream = torch.cuda.Stream()
     centers = torch.from_numpy(w.centers).cuda()
@@ -318,7 +318,7 @@ def main():
 
     # ---- the same steps with the 3xTF32 contraction, for reference, when the fp16 split was timed above ----
     tf32_ref = None
-    if args.contraction == "tc16" and world == 1:
+    if args.contraction == "tc16" and world == 1 and not reuse:
         net.set_contraction(binding.CONTRACTION_TC3XTF32)
         n_ref = max(3, min(args.steps, 5))
         ev2 = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_ref)]

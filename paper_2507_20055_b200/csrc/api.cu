@@ -40,10 +40,16 @@ struct ReuseLayer {
     float *B_hi = nullptr, *B_lo = nullptr, *bias2 = nullptr;
     cert::TcMap b_hi, b_lo, a_hi[2], a_lo[2], o_hi[2];
     cert::TcPlan plan;
+    // fp16-split form: the same block matrix as an fp16 pair; shapes rotate through three buffers
+    // (pair in, raw fp32 result, pair out)
+    __half *B16_hi = nullptr, *B16_lo = nullptr;
+    cert::TcMap b16_hi, b16_lo, a16_hi[3], a16_lo[3], o32[3];
+    cert::Tc16Plan plan16;
 };
 
 struct ReuseState {
     bool on = false;
+    bool fp16_ready = false;
     int R = 0;                           // rows per box: n0 coordinates, the constant, zero padding to 32
     float *W0t = nullptr;                // first layer's weights transposed [round_up(n0, 32)][ld_out]
     float *S_hi[2] = {nullptr, nullptr}, *S_lo[2] = {nullptr, nullptr};
@@ -798,6 +804,58 @@ cert_status_t cert_net_enable_reusecert(cert_net_t *net) {
                  cert::tc_make_map(&RL.o_hi[p], R.S_hi[p], RL.ld_s, m_max, RL.ld_s, 32);
         if (!ok) return CERT_ERR_CUDA;
     }
+    // fp16-split operands (used when the net's contraction mode is TC3XFP16)
+    if (net->tc16_ok) {
+        float *X[3] = {R.S_hi[0], R.S_hi[1], R.S_lo[0]};
+        const size_t lo_off = elems;                 // halves: the lo part of a pair sits in the buffer's second half
+        std::vector<__half> h16, l16;
+        bool ok16 = true;
+        for (int k = 1; k < K && ok16; ++k) {
+            const LayerDev &L = net->layers[k];
+            ReuseLayer &RL = R.layers[k];
+            const int n = L.n_out, m = L.n_in, ldb = R.layers[k - 1].ld_s;
+            const size_t rows_pad = round_up(L.n_out, kPad);
+            w.resize(rows_pad * L.ld_in);
+            if (cudaMemcpy(w.data(), L.W, w.size() * sizeof(float), cudaMemcpyDeviceToHost) != cudaSuccess) {
+                cudaGetLastError();
+                return CERT_ERR_CUDA;
+            }
+            const size_t brows = round_up(2 * n, kPad);
+            h16.assign(brows * ldb, __float2half_rn(0.0f));
+            l16.assign(brows * ldb, __float2half_rn(0.0f));
+            auto put16 = [&](int row, int col, float v) {
+                const __half h = __float2half_rn(v);
+                h16[(size_t)row * ldb + col] = h;
+                l16[(size_t)row * ldb + col] = __float2half_rn((v - __half2float(h)) * cert::kLoScale);
+            };
+            for (int i = 0; i < n; ++i)
+                for (int t = 0; t < m; ++t) {
+                    const float v = w[(size_t)i * L.ld_in + t];
+                    const float vp = v >= 0.0f ? v : 0.0f, vm = v >= 0.0f ? 0.0f : v;
+                    put16(i, t, vp);
+                    put16(i, m + t, vm);
+                    put16(n + i, t, vm);
+                    put16(n + i, m + t, vp);
+                }
+            if (!dev_alloc(net, (void **)&RL.B16_hi, h16.size() * sizeof(__half)) ||
+                !dev_alloc(net, (void **)&RL.B16_lo, l16.size() * sizeof(__half)))
+                return CERT_ERR_OOM;
+            if (cudaMemcpy(RL.B16_hi, h16.data(), h16.size() * sizeof(__half), cudaMemcpyHostToDevice) != cudaSuccess ||
+                cudaMemcpy(RL.B16_lo, l16.data(), l16.size() * sizeof(__half), cudaMemcpyHostToDevice) != cudaSuccess)
+                return CERT_ERR_CUDA;
+            RL.plan16 = cert::tc16_tile_plan(2 * n);
+            if (RL.plan16.stages < 2) { ok16 = false; break; }
+            ok16 = cert::tc16_make_map(&RL.b16_hi, RL.B16_hi, 2 * m, 2 * n, ldb, 64, RL.plan16.bn / 2) &&
+                   cert::tc16_make_map(&RL.b16_lo, RL.B16_lo, 2 * m, 2 * n, ldb, 64, RL.plan16.bn / 2);
+            for (int p = 0; p < 3 && ok16; ++p) {
+                const __half *xh = reinterpret_cast<const __half *>(X[p]);
+                ok16 = cert::tc16_make_map(&RL.a16_hi[p], xh, 2 * m, m_max, ldb, 64, 128) &&
+                       cert::tc16_make_map(&RL.a16_lo[p], xh + lo_off, 2 * m, m_max, ldb, 64, 128) &&
+                       cert::tc_make_map(&RL.o32[p], X[p], RL.ld_s, m_max, RL.ld_s, 32);
+            }
+        }
+        R.fp16_ready = ok16;
+    }
     if (cudaDeviceSynchronize() != cudaSuccess) { cudaGetLastError(); return CERT_ERR_CUDA; }
     R.on = true;
     return CERT_OK;
@@ -821,6 +879,55 @@ cert_status_t cert_reusecert_bounds(cert_net_t *net, const float *centers, float
     rec.mark(CERT_CLASS_INPUT);
     cert::launch_relax(L0, lb_out, ub_out, n_total, batch, net->codes, net->n_relu, nullptr, 0, 0, st);
     rec.mark(CERT_CLASS_RELAX);
+    if (net->contraction == CERT_CONTRACTION_TC3XFP16 && R.fp16_ready) {
+        // fp16-split chain: pair in X[xa], raw fp32 result in X[xb], scaled pair out in X[xc]
+        float *X[3] = {R.S_hi[0], R.S_hi[1], R.S_lo[0]};
+        int ld_max = 0;
+        for (int k = 0; k < K; ++k) ld_max = std::max(ld_max, R.layers[k].ld_s);
+        const size_t lo_off = (size_t)net->max_batch * R.R * ld_max;
+        auto hi_of = [&](int p) { return reinterpret_cast<__half *>(X[p]); };
+        auto lo_of = [&](int p) { return reinterpret_cast<__half *>(X[p]) + lo_off; };
+        int xa = 0, xb = 1, xc = 2;
+        cert::launch_reuse_init16(R.W0t, L0.ld_out, L0, net->n0, R.R, R.layers[0].ld_s, rows, hi_of(xa), lo_of(xa),
+                                  net->status_dev, st);
+        rec.mark(CERT_CLASS_RELU_STEP);
+        for (int k = 1; k < K; ++k) {
+            const LayerDev &Lk = net->layers[k];
+            const ReuseLayer &RL = R.layers[k];
+            cert::TcArgs a;
+            std::memset(&a, 0, sizeof(a));
+            a.M = rows; a.K = 2 * Lk.n_in; a.n_k = 1; a.ld_n = RL.ld_s;
+            a.bn = RL.plan16.bn; a.n_tiles = RL.plan16.n_tiles; a.stages = RL.plan16.stages;
+            a.tmem_cols = RL.plan16.tmem_cols;
+            a.total_tiles = (int)cert::ceil_div_ll(rows, 256) * RL.plan16.n_tiles;
+            a.l0 = net->l0; a.u0 = net->u0;
+            a.reuse_R = R.R; a.reuse_n0 = net->n0; a.reuse_ld0 = net->ld0; a.n_half = Lk.n_out;
+            a.bias2 = RL.bias2; a.colsum = R.colsum;
+            a.status = net->status_dev;
+            const int pairs = std::min(a.total_tiles, net->sm_count / 2);
+            cert::launch_gemm_tc16(cert::TC_EPI_REUSE, pairs, RL.a16_hi[xa], RL.a16_lo[xa], RL.b16_hi, RL.b16_lo,
+                                   RL.o32[xb], RL.o32[xb], a, RL.plan16.smem_bytes, st);
+            rec.mark(CERT_CLASS_AFFINE);
+            cert::launch_reuse_relax(R.colsum, RL.ld_s, R.R / 32, Lk, batch, lb_out, ub_out, n_total, net->codes,
+                                     net->n_relu, st);
+            rec.mark(CERT_CLASS_RELAX);
+            if (k + 1 < K) {
+                cert::launch_reuse_scale16(X[xb], hi_of(xc), lo_of(xc), RL.ld_s, Lk, net->n0, R.R, rows, net->status_dev,
+                                           st);
+                rec.mark(CERT_CLASS_RELU_STEP);
+            }
+            const int t = xa; xa = xc; xc = xb; xb = t;
+        }
+        net->last_batch = batch;
+        net->last_launches = rec.launches;
+        net->last_paths = 2 | 4 | 16;
+        net->prof_marks = rec.marks;
+        if (cudaPeekAtLastError() != cudaSuccess) {
+            cudaGetLastError();
+            return CERT_ERR_CUDA;
+        }
+        return CERT_OK;
+    }
     int cur = 0;
     cert::launch_reuse_init(R.W0t, L0.ld_out, L0, net->n0, R.R, R.layers[0].ld_s, rows, R.S_hi[cur], R.S_lo[cur], st);
     rec.mark(CERT_CLASS_RELU_STEP);

@@ -4,6 +4,7 @@
 // `prev` neurons its columns (Section 3.2).
 #pragma once
 #include <cuda_runtime.h>
+#include <cuda_fp16.h>
 #include <cstdint>
 #include <cstdio>
 #include <utility>
@@ -169,6 +170,12 @@ void launch_reuse_init(const float *W0t, int ldw, const LayerDev &L0, int n0, in
 void launch_reuse_relax(const float *colsum, int ld_s, int groups_per_box, const LayerDev &L, int batch,
                         float *lb_out, float *ub_out, int n_total, unsigned char *codes, int n_relu,
                         cudaStream_t st);
+// The fp16-split forms: S as an fp16 pair (x = hi + 2^-11 lo); `status` bit 1 is raised when a value leaves
+// the fp16 range.  The scale step reads the raw fp32 result from one buffer and writes the pair to others.
+void launch_reuse_init16(const float *W0t, int ldw, const LayerDev &L0, int n0, int R, int ld_s, long long rows,
+                         __half *S_hi, __half *S_lo, int *status, cudaStream_t st);
+void launch_reuse_scale16(const float *raw, __half *S_hi, __half *S_lo, int ld_s, const LayerDev &L, int n0, int R,
+                          long long rows, int *status, cudaStream_t st);
 // Raw [L | U] of layer L (fp32 in S_hi) -> S of its outputs, in place.
 void launch_reuse_scale(float *S_hi, float *S_lo, int ld_s, const LayerDev &L, int n0, int R, long long rows,
                         cudaStream_t st);

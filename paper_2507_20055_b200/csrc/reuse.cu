@@ -13,6 +13,8 @@
 // The kernels here start the chain, turn those sums into bounds and relaxations (Relu transformer:
 // relu_n, compute_upper on l = L.map(simplify_lower), u = U.map(simplify_upper)), and scale the raw
 // [L_k | U_k] into S_k.
+#include <cuda_fp16.h>
+
 #include "common.cuh"
 
 namespace cert {
@@ -139,7 +141,114 @@ __global__ void reuse_scale_kernel(float *__restrict__ S_hi, float *__restrict__
     *reinterpret_cast<float4 *>(S_lo + (size_t)r * ld_s + col0) = make_float4(l[0], l[1], l[2], l[3]);
 }
 
+// The fp16-split forms (x = hi + 2^-11 lo, see gemm_tc16.cuh): the same two steps writing halves.
+constexpr float kLoScale16 = 2048.0f;
+
+__device__ __forceinline__ void store_pair16(float v, __half &h, __half &l, bool &out_of_range) {
+    out_of_range |= !(fabsf(v) <= 60000.0f);
+    h = __float2half_rn(v);
+    l = __float2half_rn((v - __half2float(h)) * kLoScale16);
+}
+
+__global__ void reuse_init16_kernel(const float *__restrict__ W0t, int ldw, const float *__restrict__ bias,
+                                    int n, int n0, int R, int ld_s, int ld_relax, int has_relu,
+                                    const float *__restrict__ lamL, const float *__restrict__ lamU,
+                                    const float *__restrict__ nuU, long long rows, __half *__restrict__ S_hi,
+                                    __half *__restrict__ S_lo, int *__restrict__ status) {
+    const int quads = ld_s / 4;
+    const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    bool out_of_range = false;
+    if (idx < rows * quads) {
+        const long long r = idx / quads;
+        const int col0 = (int)(idx % quads) * 4;
+        const int box = (int)(r / R), s = (int)(r % R);
+        __half h[4], l[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const int col = col0 + e;
+            float v = 0.0f;
+            if (col < 2 * n && s <= n0) {
+                const bool upper = col >= n;
+                const int t = upper ? col - n : col;
+                const float base = s < n0 ? W0t[(size_t)s * ldw + t] : bias[t];
+                float lam = 1.0f, nu = 0.0f;
+                if (has_relu) {
+                    lam = upper ? lamU[(size_t)box * ld_relax + t] : lamL[(size_t)box * ld_relax + t];
+                    nu = (upper && s == n0) ? nuU[(size_t)box * ld_relax + t] : 0.0f;
+                }
+                v = fmaf(lam, base, nu);
+            }
+            store_pair16(v, h[e], l[e], out_of_range);
+        }
+        uint2 ph, pl;
+        ph.x = (uint32_t)__half_as_ushort(h[0]) | ((uint32_t)__half_as_ushort(h[1]) << 16);
+        ph.y = (uint32_t)__half_as_ushort(h[2]) | ((uint32_t)__half_as_ushort(h[3]) << 16);
+        pl.x = (uint32_t)__half_as_ushort(l[0]) | ((uint32_t)__half_as_ushort(l[1]) << 16);
+        pl.y = (uint32_t)__half_as_ushort(l[2]) | ((uint32_t)__half_as_ushort(l[3]) << 16);
+        *reinterpret_cast<uint2 *>(S_hi + (size_t)r * ld_s + col0) = ph;
+        *reinterpret_cast<uint2 *>(S_lo + (size_t)r * ld_s + col0) = pl;
+    }
+    if (__any_sync(0xffffffffu, out_of_range) && (threadIdx.x & 31) == 0) atomicOr(status, 2);
+}
+
+// raw: fp32 [L_k | U_k] of the contraction; S_hi / S_lo: the scaled shapes as an fp16 pair (other buffers).
+__global__ void reuse_scale16_kernel(const float *__restrict__ raw, __half *__restrict__ S_hi,
+                                     __half *__restrict__ S_lo, int ld_s, int n, int n0, int R, int ld_relax,
+                                     int has_relu, const float *__restrict__ lamL, const float *__restrict__ lamU,
+                                     const float *__restrict__ nuU, long long rows, int *__restrict__ status) {
+    const int quads = ld_s / 4;
+    const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    bool out_of_range = false;
+    if (idx < rows * quads) {
+        const long long r = idx / quads;
+        const int col0 = (int)(idx % quads) * 4;
+        const int box = (int)(r / R), s = (int)(r % R);
+        const float4 rv4 = *reinterpret_cast<const float4 *>(raw + (size_t)r * ld_s + col0);
+        const float rv[4] = {rv4.x, rv4.y, rv4.z, rv4.w};
+        __half h[4], l[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const int col = col0 + e;
+            float v = 0.0f;
+            if (col < 2 * n && s <= n0) {
+                v = rv[e];
+                if (has_relu) {
+                    const bool upper = col >= n;
+                    const int t = upper ? col - n : col;
+                    const float lam = upper ? lamU[(size_t)box * ld_relax + t] : lamL[(size_t)box * ld_relax + t];
+                    const float nu = (upper && s == n0) ? nuU[(size_t)box * ld_relax + t] : 0.0f;
+                    v = fmaf(lam, v, nu);
+                }
+            }
+            store_pair16(v, h[e], l[e], out_of_range);
+        }
+        uint2 ph, pl;
+        ph.x = (uint32_t)__half_as_ushort(h[0]) | ((uint32_t)__half_as_ushort(h[1]) << 16);
+        ph.y = (uint32_t)__half_as_ushort(h[2]) | ((uint32_t)__half_as_ushort(h[3]) << 16);
+        pl.x = (uint32_t)__half_as_ushort(l[0]) | ((uint32_t)__half_as_ushort(l[1]) << 16);
+        pl.y = (uint32_t)__half_as_ushort(l[2]) | ((uint32_t)__half_as_ushort(l[3]) << 16);
+        *reinterpret_cast<uint2 *>(S_hi + (size_t)r * ld_s + col0) = ph;
+        *reinterpret_cast<uint2 *>(S_lo + (size_t)r * ld_s + col0) = pl;
+    }
+    if (__any_sync(0xffffffffu, out_of_range) && (threadIdx.x & 31) == 0) atomicOr(status, 2);
+}
+
 }  // namespace
+
+void launch_reuse_init16(const float *W0t, int ldw, const LayerDev &L0, int n0, int R, int ld_s, long long rows,
+                         __half *S_hi, __half *S_lo, int *status, cudaStream_t st) {
+    const long long threads = rows * (ld_s / 4);
+    reuse_init16_kernel<<<(unsigned)ceil_div_ll(threads, 256), 256, 0, st>>>(
+        W0t, ldw, L0.bias_n, L0.n_out, n0, R, ld_s, L0.ld_out, L0.relu_after, L0.lamL, L0.lamU, L0.nuU, rows, S_hi, S_lo,
+        status);
+}
+
+void launch_reuse_scale16(const float *raw, __half *S_hi, __half *S_lo, int ld_s, const LayerDev &L, int n0, int R,
+                          long long rows, int *status, cudaStream_t st) {
+    const long long threads = rows * (ld_s / 4);
+    reuse_scale16_kernel<<<(unsigned)ceil_div_ll(threads, 256), 256, 0, st>>>(
+        raw, S_hi, S_lo, ld_s, L.n_out, n0, R, L.ld_out, L.relu_after, L.lamL, L.lamU, L.nuU, rows, status);
+}
 
 void launch_reuse_init(const float *W0t, int ldw, const LayerDev &L0, int n0, int R, int ld_s, long long rows,
                        float *S_hi, float *S_lo, cudaStream_t st) {

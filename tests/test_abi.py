@@ -90,3 +90,14 @@ def test_product_does_not_import_the_oracle():
         if f.endswith((".py", ".c")):
             text = open(os.path.join(ROOT, "oracle", f)).read()
             assert "paper_2507_20055_b200" not in text and "cert.h" not in text
+
+
+def test_null_handles_of_the_other_entry_points(lib):
+    L = lib.lib
+    assert L.cert_backsub_bounds(None, None, 0.1, 1, None, None, None, None) == 1
+    assert L.cert_backsub_bounds_host(None, None, 0.1, 1, None, None, None, None) == 1
+    assert L.cert_reusecert_bounds(None, None, 0.1, 1, None, None, None) == 1
+    assert L.cert_reusecert_bounds_host(None, None, 0.1, 1, None, None, None) == 1
+    assert L.cert_net_enable_reusecert(None) == 1
+    assert L.cert_net_set_conv_patches(None, 1) == 1
+    assert b"fp16" in L.cert_status_string(7)

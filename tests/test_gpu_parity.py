@@ -238,11 +238,13 @@ REUSE_NETS = {
 REUSE_TOL = 5e-4
 
 
-def _run_reusecert(w, max_batch=None):
+def _run_reusecert(w, max_batch=None, contraction=None):
     import torch
     from paper_2507_20055_b200 import binding
     net = binding.CertNet(w.layers, max_batch or w.batch, w.clip_lo, w.clip_hi)
     try:
+        if contraction is not None:
+            net.set_contraction(contraction)
         net.enable_reusecert()
         c = torch.from_numpy(np.ascontiguousarray(w.centers)).cuda()
         out = []
@@ -261,13 +263,14 @@ def _run_reusecert(w, max_batch=None):
     return out, dp
 
 
+@pytest.mark.parametrize("mode", ["tc", "tc16"])
 @pytest.mark.parametrize("name", sorted(REUSE_NETS))
-def test_reusecert(name):
+def test_reusecert(name, mode):
     w = REUSE_NETS[name]()
     ref = orc.reusecert(w.layers, w.centers, w.eps, w.clip_lo, w.clip_hi)
-    out, dp = _run_reusecert(w, max_batch=w.batch + 3)
+    out, dp = _run_reusecert(w, max_batch=w.batch + 3, contraction={"tc": 2, "tc16": 3}[mode])
     for i, g in enumerate(out):
-        compare(g, ref, label=f"reusecert/{name}/call{i}", tol=REUSE_TOL)
+        compare(g, ref, label=f"reusecert/{name}/{mode}/call{i}", tol=REUSE_TOL)
     assert np.array_equal(out[0]["lb"], out[1]["lb"]) and np.array_equal(out[0]["ub"], out[1]["ub"])
     compare(dp, _oracle(w), label=f"deeppoly_after_reusecert/{name}")
 
@@ -291,7 +294,8 @@ def test_reusecert_needs_enable_and_fc_layers():
         net.destroy()
 
 
-def test_reusecert_config5_sampled_boxes():
+@pytest.mark.parametrize("mode", ["tc", "tc16"])
+def test_reusecert_config5_sampled_boxes(mode):
     """784 -> 1024 x 6 -> 10, 128 boxes on the GPU (the benchmark's launch configuration); the oracle bounds
     a sample of boxes.  With 6144 ReLU neurons per box and ReuseCert's wider bounds most boxes have some neuron
     whose sign test is within float32 noise of zero; those boxes are skipped as everywhere else, so more
@@ -303,6 +307,7 @@ def test_reusecert_config5_sampled_boxes():
     ref = orc.reusecert(w.layers, w.centers[np.asarray(boxes)], w.eps, w.clip_lo, w.clip_hi)
     net = binding.CertNet(w.layers, w.batch, w.clip_lo, w.clip_hi)
     try:
+        net.set_contraction({"tc": 2, "tc16": 3}[mode])
         net.enable_reusecert()
         lb, ub = net.reusecert_bounds(torch.from_numpy(w.centers).cuda(), w.eps)
         torch.cuda.synchronize()
@@ -310,7 +315,7 @@ def test_reusecert_config5_sampled_boxes():
              "status": net.last_status()}
     finally:
         net.destroy()
-    compare(g, ref, boxes=boxes, label="reusecert/fc6x1024", tol=REUSE_TOL, min_good_fraction=0.1)
+    compare(g, ref, boxes=boxes, label=f"reusecert/fc6x1024/{mode}", tol=REUSE_TOL, min_good_fraction=0.1)
 
 
 # ---- fp16-split tensor-core contraction (CERT_CONTRACTION_TC3XFP16), nets of FC layers ----
