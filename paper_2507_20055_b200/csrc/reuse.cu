@@ -150,21 +150,32 @@ __device__ __forceinline__ void store_pair16(float v, __half &h, __half &l, bool
     l = __float2half_rn((v - __half2float(h)) * kLoScale16);
 }
 
+__device__ __forceinline__ uint4 pack8(const __half (&x)[8]) {
+    uint4 p;
+    p.x = (uint32_t)__half_as_ushort(x[0]) | ((uint32_t)__half_as_ushort(x[1]) << 16);
+    p.y = (uint32_t)__half_as_ushort(x[2]) | ((uint32_t)__half_as_ushort(x[3]) << 16);
+    p.z = (uint32_t)__half_as_ushort(x[4]) | ((uint32_t)__half_as_ushort(x[5]) << 16);
+    p.w = (uint32_t)__half_as_ushort(x[6]) | ((uint32_t)__half_as_ushort(x[7]) << 16);
+    return p;
+}
+
+// One warp per row, a lane per group of 8 columns (16-byte stores of halves; pitches are multiples of 32 elements).
 __global__ void reuse_init16_kernel(const float *__restrict__ W0t, int ldw, const float *__restrict__ bias,
                                     int n, int n0, int R, int ld_s, int ld_relax, int has_relu,
                                     const float *__restrict__ lamL, const float *__restrict__ lamU,
                                     const float *__restrict__ nuU, long long rows, __half *__restrict__ S_hi,
                                     __half *__restrict__ S_lo, int *__restrict__ status) {
-    const int quads = ld_s / 4;
-    const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    // one warp per row, lanes over groups of 8 columns
+    const int octs = ld_s / 8;
+    const long long r = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int lane = threadIdx.x & 31;
     bool out_of_range = false;
-    if (idx < rows * quads) {
-        const long long r = idx / quads;
-        const int col0 = (int)(idx % quads) * 4;
-        const int box = (int)(r / R), s = (int)(r % R);
-        __half h[4], l[4];
+    const int box = r < rows ? (int)(r / R) : 0, s = r < rows ? (int)(r % R) : 0;
+    for (int o = lane; r < rows && o < octs; o += 32) {
+        const int col0 = o * 8;
+        __half h[8], l[8];
 #pragma unroll
-        for (int e = 0; e < 4; ++e) {
+        for (int e = 0; e < 8; ++e) {
             const int col = col0 + e;
             float v = 0.0f;
             if (col < 2 * n && s <= n0) {
@@ -180,13 +191,8 @@ __global__ void reuse_init16_kernel(const float *__restrict__ W0t, int ldw, cons
             }
             store_pair16(v, h[e], l[e], out_of_range);
         }
-        uint2 ph, pl;
-        ph.x = (uint32_t)__half_as_ushort(h[0]) | ((uint32_t)__half_as_ushort(h[1]) << 16);
-        ph.y = (uint32_t)__half_as_ushort(h[2]) | ((uint32_t)__half_as_ushort(h[3]) << 16);
-        pl.x = (uint32_t)__half_as_ushort(l[0]) | ((uint32_t)__half_as_ushort(l[1]) << 16);
-        pl.y = (uint32_t)__half_as_ushort(l[2]) | ((uint32_t)__half_as_ushort(l[3]) << 16);
-        *reinterpret_cast<uint2 *>(S_hi + (size_t)r * ld_s + col0) = ph;
-        *reinterpret_cast<uint2 *>(S_lo + (size_t)r * ld_s + col0) = pl;
+        *reinterpret_cast<uint4 *>(S_hi + (size_t)r * ld_s + col0) = pack8(h);
+        *reinterpret_cast<uint4 *>(S_lo + (size_t)r * ld_s + col0) = pack8(l);
     }
     if (__any_sync(0xffffffffu, out_of_range) && (threadIdx.x & 31) == 0) atomicOr(status, 2);
 }
@@ -196,18 +202,20 @@ __global__ void reuse_scale16_kernel(const float *__restrict__ raw, __half *__re
                                      __half *__restrict__ S_lo, int ld_s, int n, int n0, int R, int ld_relax,
                                      int has_relu, const float *__restrict__ lamL, const float *__restrict__ lamU,
                                      const float *__restrict__ nuU, long long rows, int *__restrict__ status) {
-    const int quads = ld_s / 4;
-    const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    // one warp per row, lanes over groups of 8 columns
+    const int octs = ld_s / 8;
+    const long long r = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int lane = threadIdx.x & 31;
     bool out_of_range = false;
-    if (idx < rows * quads) {
-        const long long r = idx / quads;
-        const int col0 = (int)(idx % quads) * 4;
-        const int box = (int)(r / R), s = (int)(r % R);
-        const float4 rv4 = *reinterpret_cast<const float4 *>(raw + (size_t)r * ld_s + col0);
-        const float rv[4] = {rv4.x, rv4.y, rv4.z, rv4.w};
-        __half h[4], l[4];
+    const int box = r < rows ? (int)(r / R) : 0, s = r < rows ? (int)(r % R) : 0;
+    for (int o = lane; r < rows && o < octs; o += 32) {
+        const int col0 = o * 8;
+        const float4 r0 = *reinterpret_cast<const float4 *>(raw + (size_t)r * ld_s + col0);
+        const float4 r1 = *reinterpret_cast<const float4 *>(raw + (size_t)r * ld_s + col0 + 4);
+        const float rv[8] = {r0.x, r0.y, r0.z, r0.w, r1.x, r1.y, r1.z, r1.w};
+        __half h[8], l[8];
 #pragma unroll
-        for (int e = 0; e < 4; ++e) {
+        for (int e = 0; e < 8; ++e) {
             const int col = col0 + e;
             float v = 0.0f;
             if (col < 2 * n && s <= n0) {
@@ -222,13 +230,8 @@ __global__ void reuse_scale16_kernel(const float *__restrict__ raw, __half *__re
             }
             store_pair16(v, h[e], l[e], out_of_range);
         }
-        uint2 ph, pl;
-        ph.x = (uint32_t)__half_as_ushort(h[0]) | ((uint32_t)__half_as_ushort(h[1]) << 16);
-        ph.y = (uint32_t)__half_as_ushort(h[2]) | ((uint32_t)__half_as_ushort(h[3]) << 16);
-        pl.x = (uint32_t)__half_as_ushort(l[0]) | ((uint32_t)__half_as_ushort(l[1]) << 16);
-        pl.y = (uint32_t)__half_as_ushort(l[2]) | ((uint32_t)__half_as_ushort(l[3]) << 16);
-        *reinterpret_cast<uint2 *>(S_hi + (size_t)r * ld_s + col0) = ph;
-        *reinterpret_cast<uint2 *>(S_lo + (size_t)r * ld_s + col0) = pl;
+        *reinterpret_cast<uint4 *>(S_hi + (size_t)r * ld_s + col0) = pack8(h);
+        *reinterpret_cast<uint4 *>(S_lo + (size_t)r * ld_s + col0) = pack8(l);
     }
     if (__any_sync(0xffffffffu, out_of_range) && (threadIdx.x & 31) == 0) atomicOr(status, 2);
 }
@@ -237,16 +240,14 @@ __global__ void reuse_scale16_kernel(const float *__restrict__ raw, __half *__re
 
 void launch_reuse_init16(const float *W0t, int ldw, const LayerDev &L0, int n0, int R, int ld_s, long long rows,
                          __half *S_hi, __half *S_lo, int *status, cudaStream_t st) {
-    const long long threads = rows * (ld_s / 4);
-    reuse_init16_kernel<<<(unsigned)ceil_div_ll(threads, 256), 256, 0, st>>>(
+    reuse_init16_kernel<<<(unsigned)ceil_div_ll(rows, 8), 256, 0, st>>>(
         W0t, ldw, L0.bias_n, L0.n_out, n0, R, ld_s, L0.ld_out, L0.relu_after, L0.lamL, L0.lamU, L0.nuU, rows, S_hi, S_lo,
         status);
 }
 
 void launch_reuse_scale16(const float *raw, __half *S_hi, __half *S_lo, int ld_s, const LayerDev &L, int n0, int R,
                           long long rows, int *status, cudaStream_t st) {
-    const long long threads = rows * (ld_s / 4);
-    reuse_scale16_kernel<<<(unsigned)ceil_div_ll(threads, 256), 256, 0, st>>>(
+    reuse_scale16_kernel<<<(unsigned)ceil_div_ll(rows, 8), 256, 0, st>>>(
         raw, S_hi, S_lo, ld_s, L.n_out, n0, R, L.ld_out, L.relu_after, L.lamL, L.lamU, L.nuU, rows, status);
 }
 
