@@ -33,6 +33,20 @@ struct TcLayer {
 };
 
 
+// Tensor-core form of one patch back-step: the rows of conv layer k, held as windows over the outputs of
+// conv layer j (level m = k-1-j), go to windows over j's inputs.  Between windows the conv layer is one
+// dense matrix T [K = c_out*ph*pw][N = c_in*qh*qw], the same for every neuron position and box, so the
+// step is a plain contraction; what depends on the position (the relaxation or the box at the window's
+// place in the map, and which window positions lie outside the map) enters through per-(box, position)
+// vectors gathered before the launch.
+struct TcPatchStep {
+    int K = 0, Kp = 0, N = 0, ldN = 0;   // window elements in / out and their padded widths
+    float *T_hi = nullptr, *T_lo = nullptr;      // T transposed, [ldN][Kp], TF32 split
+    float *bias_e = nullptr;             // [ldN] bias of the affine layer below, per window element; null at j = 0
+    cert::TcMap b_hi, b_lo, a_hi[2], a_lo[2], o_hi[2], o_lo[2];
+    cert::TcPlan plan;
+};
+
 // ReuseCert: per affine layer k >= 1 the block weight matrix [[W+^T, W-^T], [W-^T, W+^T]] as the K-major B
 // operand (rows = the 2*n_k output columns, columns = the 2*n_{k-1} columns of the layer below), TF32 split.
 struct ReuseLayer {
@@ -78,6 +92,8 @@ struct cert_net {
     int sm_count = 148;
     int tc_ctas = 1;                         // CTAs per row panel of the tensor-core kernel (2: cta_group::2)
     bool conv_patches = true;                // conv-sourced rows travel as receptive-field patches where they can
+    std::vector<std::vector<TcPatchStep>> tcp;   // [k]: the leading patch steps of layer k's traversal that can run on the tensor cores
+    float *gat[3] = {nullptr, nullptr, nullptr}; // gathered windows, [max_batch * positions][ldN] each
     ReuseState reuse;
     unsigned char *codes = nullptr;          // [max_batch][n_relu]
     int *status_dev = nullptr;               // sticky device status word
@@ -280,6 +296,90 @@ cert_status_t setup_tensor_core_path(cert_net *net, const cert_layer_desc_t *des
     return CERT_OK;
 }
 
+// Patch back-steps on the tensor cores: builds, for every conv layer k over conv layers, the dense
+// window-to-window matrices of the leading steps of its traversal.  A step qualifies while the dense
+// form does at most kPatchDenseRatio times the multiply-adds of the transposed convolution itself
+// (the tensor cores are far more than that ahead of the FMA patch kernel) and the matrix stays small.
+constexpr int kPatchDenseRatio = 24;
+constexpr size_t kPatchMatrixMax = 16u << 20;   // floats
+
+cert_status_t setup_patch_tc(cert_net *net, const cert_layer_desc_t *descs) {
+    const int K = net->n_layers;
+    net->tcp.assign(K, std::vector<TcPatchStep>());
+    if (!net->tc_ok) return CERT_OK;
+    const int ctas = net->tc_ctas;
+    size_t gat_floats = 0;
+    std::vector<float> hi, lo, be;
+    for (int k = 1; k < K; ++k) {
+        const LayerDev &Lk = net->layers[k];
+        if (Lk.kind != CERT_LAYER_CONV2D) continue;
+        cert::PatchLevel lv[kMaxPatchLevels];
+        int j_end = 0;
+        while (j_end < k && !cert::conv_patch_plan(net->layers.data(), k, j_end, lv, kMaxPatchLevels)) ++j_end;
+        if (j_end >= k) continue;
+        const long long rows_max = 2LL * net->max_batch * Lk.n_out;
+        for (int j = k - 1, m = 0; j >= j_end; --j, ++m) {
+            const LayerDev &Lj = net->layers[j];
+            const cert::PatchLevel &in = lv[m], &out = lv[m + 1];
+            TcPatchStep S;
+            S.K = in.elems; S.Kp = round_up(in.elems, kPad);
+            S.N = out.elems; S.ldN = round_up(out.elems, kPad);
+            if (out.ph * out.pw > kPatchDenseRatio * Lj.kh * Lj.kw) break;
+            if ((size_t)S.ldN * S.Kp > kPatchMatrixMax) break;
+            S.plan = cert::tc_tile_plan(S.N, ctas);
+            if (S.plan.stages < 2) break;
+            hi.assign((size_t)S.ldN * S.Kp, 0.0f);
+            lo.assign((size_t)S.ldN * S.Kp, 0.0f);
+            const float *W = descs[j].weight;          // [c_out][c_in][kh][kw]
+            for (int co = 0; co < Lj.c_out; ++co)
+                for (int py = 0; py < in.ph; ++py)
+                    for (int px = 0; px < in.pw; ++px) {
+                        const size_t kk = ((size_t)co * in.ph + py) * in.pw + px;
+                        for (int ci = 0; ci < Lj.c_in; ++ci)
+                            for (int ky = 0; ky < Lj.kh; ++ky)
+                                for (int kx = 0; kx < Lj.kw; ++kx) {
+                                    const size_t n = ((size_t)ci * out.ph + Lj.stride * py + ky) * out.pw +
+                                                     Lj.stride * px + kx;
+                                    const float w = W[(((size_t)co * Lj.c_in + ci) * Lj.kh + ky) * Lj.kw + kx];
+                                    const float h = host_tf32(w);
+                                    hi[n * S.Kp + kk] = h;
+                                    lo[n * S.Kp + kk] = host_tf32(w - h);
+                                }
+                    }
+            if (!dev_alloc(net, (void **)&S.T_hi, hi.size() * sizeof(float)) ||
+                !dev_alloc(net, (void **)&S.T_lo, lo.size() * sizeof(float)))
+                return CERT_ERR_OOM;
+            if (cudaMemcpy(S.T_hi, hi.data(), hi.size() * sizeof(float), cudaMemcpyHostToDevice) != cudaSuccess ||
+                cudaMemcpy(S.T_lo, lo.data(), lo.size() * sizeof(float), cudaMemcpyHostToDevice) != cudaSuccess)
+                return CERT_ERR_CUDA;
+            if (j > 0 && net->layers[j - 1].kind == CERT_LAYER_CONV2D) {
+                // a window element of channel c meets the bias of channel c of the conv layer below
+                be.assign(S.ldN, 0.0f);
+                const int qhw = out.ph * out.pw;
+                for (int e = 0; e < S.N; ++e) be[e] = descs[j - 1].bias[e / qhw];
+                if (!dev_alloc(net, (void **)&S.bias_e, be.size() * sizeof(float))) return CERT_ERR_OOM;
+                if (cudaMemcpy(S.bias_e, be.data(), be.size() * sizeof(float), cudaMemcpyHostToDevice) != cudaSuccess)
+                    return CERT_ERR_CUDA;
+            }
+            bool ok = cert::tc_make_map(&S.b_hi, S.T_hi, S.Kp, S.ldN, S.Kp, S.plan.bn / ctas) &&
+                      cert::tc_make_map(&S.b_lo, S.T_lo, S.Kp, S.ldN, S.Kp, S.plan.bn / ctas);
+            for (int p = 0; p < 2 && ok; ++p)
+                ok = cert::tc_make_map(&S.a_hi[p], net->buf[p], S.Kp, rows_max, S.Kp, 128) &&
+                     cert::tc_make_map(&S.a_lo[p], net->buf_lo[p], S.Kp, rows_max, S.Kp, 128) &&
+                     cert::tc_make_map(&S.o_hi[p], net->buf[p], S.ldN, rows_max, S.ldN, 32) &&
+                     cert::tc_make_map(&S.o_lo[p], net->buf_lo[p], S.ldN, rows_max, S.ldN, 32);
+            if (!ok) break;
+            net->d_slots = std::max(net->d_slots, S.plan.n_tiles);
+            gat_floats = std::max(gat_floats, (size_t)net->max_batch * Lk.h_out * Lk.w_out * S.ldN);
+            net->tcp[k].push_back(S);
+        }
+    }
+    if (gat_floats)
+        for (int i = 0; i < 3; ++i)
+            if (!dev_alloc_zero(net, &net->gat[i], gat_floats)) return CERT_ERR_OOM;
+    return CERT_OK;
+}
+
 // Counts launches; with profiling on, drops an event after each so that the
 // time between consecutive events is that launch's device time.
 struct Recorder {
@@ -446,6 +546,7 @@ cert_status_t cert_net_create(const cert_layer_desc_t *layers, int n_layers, int
         if (!ok) fail = CERT_ERR_OOM;
         net->slot_stride = (long long)max_rows;
         if (ok) fail = setup_tensor_core_path(net, layers, max_elems);
+        if (ok && fail == CERT_OK) fail = setup_patch_tc(net, layers);
         if (fail == CERT_OK &&
             (!dev_alloc_zero(net, &net->dbuf[0], (size_t)net->d_slots * max_rows) ||
              !dev_alloc_zero(net, &net->dbuf[1], (size_t)net->d_slots * max_rows)))
@@ -562,8 +663,65 @@ cert_status_t cert_backsub_bounds(cert_net_t *net, const float *centers, float e
         }
         // A conv layer over conv layers: rows as receptive-field patches instead of dense maps.
         cert::PatchLevel lv[kMaxPatchLevels];
-        if (net->conv_patches && cert::conv_patch_plan(net->layers.data(), k, j_end, lv, kMaxPatchLevels)) {
-            cert::launch_patch_start(Lk, net->layers[k - 1], lv[0], batch, net->buf[cur], net->dbuf[dcur], st);
+        const bool patches = net->conv_patches && cert::conv_patch_plan(net->layers.data(), k, j_end, lv, kMaxPatchLevels);
+        if (patches && net->contraction != CERT_CONTRACTION_FFMA && (int)net->tcp[k].size() >= steps) {
+            // every step of the traversal as a contraction with the conv layer's window-to-window matrix
+            const std::vector<TcPatchStep> &SS = net->tcp[k];
+            const int ctas = net->tc_ctas;
+            cert::launch_patch_start(Lk, net->layers[k - 1], SS[0].Kp, batch, net->buf[cur], net->buf_lo[cur],
+                                     net->dbuf[dcur], st);
+            rec.mark(CERT_CLASS_RELU_STEP);
+            for (int j = k - 1, m = 0; j >= j_end; --j, ++m) {
+                const LayerDev &Lj = net->layers[j];
+                const TcPatchStep &S = SS[m];
+                const float *src[3] = {nullptr, nullptr, nullptr};
+                const float fill[3] = {1.0f, 1.0f, 0.0f};
+                int n_arr = 3;
+                if (j > j_end) {
+                    const LayerDev &Lb = net->layers[j - 1];
+                    if (Lb.relu_after) { src[0] = Lb.lamL; src[1] = Lb.lamU; src[2] = Lb.nuU; }
+                } else {
+                    src[0] = box_l; src[1] = box_u;
+                    n_arr = 2;
+                }
+                cert::launch_patch_gather(Lk, Lj, lv[m + 1], S.ldN, batch, n_arr, src, fill, net->gat, st);
+                rec.mark(CERT_CLASS_CONV);
+                cert::TcArgs a;
+                std::memset(&a, 0, sizeof(a));
+                a.M = rows; a.K = S.Kp; a.n_k = Lk.n_out; a.ld_n = S.ldN;
+                a.n_pos = Lk.h_out * Lk.w_out;
+                a.bn = S.plan.bn; a.n_tiles = S.plan.n_tiles; a.stages = S.plan.stages;
+                a.tmem_cols = S.plan.tmem_cols;
+                a.total_tiles = (int)cert::ceil_div_ll(rows, 128 * ctas) * S.plan.n_tiles;
+                a.d_in = net->dbuf[dcur]; a.n_slots_in = dslots; a.d_out = net->dbuf[dcur ^ 1];
+                a.slot_stride = net->slot_stride;
+                a.status = net->status_dev;
+                const int groups = std::min(a.total_tiles, net->sm_count / ctas);
+                if (j > j_end) {
+                    a.has_relu = 1;          // the gathered slopes also blank the window outside the map
+                    a.split_out = 1;
+                    a.lamL = net->gat[0]; a.lamU = net->gat[1]; a.nuU = net->gat[2]; a.bias_below = S.bias_e;
+                    cert::launch_gemm_tc(cert::TC_EPI_RELU, ctas, groups, S.a_hi[cur], S.a_lo[cur], S.b_hi, S.b_lo,
+                                         S.o_hi[cur ^ 1], S.o_lo[cur ^ 1], a, S.plan.smem_bytes, st);
+                } else {
+                    a.l0 = net->gat[0]; a.u0 = net->gat[1];
+                    cert::launch_gemm_tc(cert::TC_EPI_CONCRETIZE, ctas, groups, S.a_hi[cur], S.a_lo[cur], S.b_hi,
+                                         S.b_lo, S.a_hi[cur], S.a_lo[cur], a, S.plan.smem_bytes, st);
+                }
+                rec.mark(CERT_CLASS_CONV);
+                cur ^= 1;
+                dcur ^= 1;
+                dslots = S.plan.n_tiles;
+            }
+            cert::launch_relax(Lk, lb_out, ub_out, n_total, batch, net->codes, net->n_relu, net->dbuf[dcur], dslots,
+                               net->slot_stride, st);
+            rec.mark(CERT_CLASS_RELAX);
+            paths |= 8 | 2 | (ctas == 2 ? 4 : 0);
+            continue;
+        }
+        if (patches) {
+            cert::launch_patch_start(Lk, net->layers[k - 1], lv[0].pitch, batch, net->buf[cur], nullptr,
+                                     net->dbuf[dcur], st);
             rec.mark(CERT_CLASS_RELU_STEP);
             for (int j = k - 1, m = 0; j >= j_end; --j, ++m) {
                 const LayerDev &Lj = net->layers[j];

@@ -155,8 +155,16 @@ struct PatchLevel {
 bool conv_patch_plan(const LayerDev *layers, int k, int j_end, PatchLevel *levels, int max_levels);
 void conv_patch_prepare();
 // Start: the kernel of layer k as a patch over the outputs of the layer below, through that layer's ReLU.
-void launch_patch_start(const LayerDev &Lk, const LayerDev &Lb, const PatchLevel &lv, int batch, float *patch,
-                        float *d, cudaStream_t st);
+// `pitch` floats per row; patch_lo != nullptr: written as a TF32 pair for a tensor-core step.
+void launch_patch_start(const LayerDev &Lk, const LayerDev &Lb, int pitch, int batch, float *patch,
+                        float *patch_lo, float *d, cudaStream_t st);
+// For the tensor-core form of a patch back-step (the conv layer as a dense matrix between windows, the
+// same for every position): windows of n_arr <= 3 per-neuron arrays [batch][Lj.ld_in] of the layer below
+// conv layer j, one vector of ld_dst floats per (box, output position of layer k), zero outside the map;
+// a null src[i] stands for fill[i] inside the map.
+void launch_patch_gather(const LayerDev &Lk, const LayerDev &Lj, const PatchLevel &out, int ld_dst, int batch,
+                         int n_arr, const float *const *src, const float *fill, float *const *dst,
+                         cudaStream_t st);
 // Back-step of the patches through conv layer j, followed by `ep` (ep.P = output patches, pitch out.pitch).
 void launch_patch_step(const LayerDev &Lk, const LayerDev &Lj, const PatchLevel &in, const PatchLevel &out,
                        const float *in_patch, long long rows, int sms, const ConvtEpilogue &ep, cudaStream_t st);

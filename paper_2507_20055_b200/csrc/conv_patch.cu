@@ -43,9 +43,17 @@ __device__ __forceinline__ float relu_backstep(float c, int upper, float lamL, f
 
 // Start at conv layer k: patch over the layer's inputs = its kernel [c_in][kh][kw] at origin
 // (oy*stride - pad, ox*stride - pad), pushed through the ReLU below; constant = bias + the nu terms +
-// Q.b of the layer below.  Out-of-image window positions get 0.
+// Q.b of the layer below.  Out-of-image window positions get 0.  With patch_lo the patch is written as a
+// TF32 pair (hi in patch, lo in patch_lo) for a tensor-core step.
+__device__ __forceinline__ float tf32_rn(float x) {
+    uint32_t u;
+    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(u) : "f"(x));
+    return __uint_as_float(u);
+}
+
 __global__ void patch_start_kernel(const float *__restrict__ Wk, ConvGeom gk, const float *__restrict__ bias_k,
-                                   float *__restrict__ patch, int pitch, float *__restrict__ d, long long rows,
+                                   float *__restrict__ patch, float *__restrict__ patch_lo, int pitch,
+                                   float *__restrict__ d, long long rows,
                                    int n_k, int ld, int has_relu, const float *__restrict__ lamL,
                                    const float *__restrict__ lamU, const float *__restrict__ nuU,
                                    const float *__restrict__ bias_below) {
@@ -75,10 +83,52 @@ __global__ void patch_start_kernel(const float *__restrict__ Wk, ConvGeom gk, co
                 dacc = fmaf(qv, bias_below[t], dacc);
             }
         }
-        prow[q] = qv;
+        if (patch_lo) {
+            const float h = tf32_rn(qv);
+            prow[q] = h;
+            patch_lo[(size_t)r * pitch + q] = tf32_rn(qv - h);
+        } else {
+            prow[q] = qv;
+        }
     }
     dacc = warp_sum(dacc);
     if (lane == 0) d[r] = bias_k[i] + dacc;
+}
+
+// Per (box, output position of the conv neuron): the window of up to three per-neuron arrays of the
+// layer the window lies in, laid out like the patch ([c][qh][qw], zero padded to ld_dst); positions
+// outside the map get 0, so that they drop out of whatever the values multiply.  A null source
+// stands for the constant fill[i] inside the map (no ReLU below: slopes 1, intercept 0).
+struct PatchGather {
+    int c, qh, qw;         // window
+    int h, w;              // map of the layer the window lies in
+    int a, b;              // window origin = (oy, ox) * a - b
+    int w_k, n_pos;        // layer k's output map: width, positions
+    int ld_src, ld_dst;
+    int n_arr;
+    const float *src[3];
+    float fill[3];
+    float *dst[3];
+};
+
+__global__ void patch_gather_kernel(const PatchGather g) {
+    const int v = blockIdx.x;                    // box * n_pos + position
+    const int box = v / g.n_pos, pos = v - box * g.n_pos;
+    const int gy0 = (pos / g.w_k) * g.a - g.b, gx0 = (pos % g.w_k) * g.a - g.b;
+    const int qhw = g.qh * g.qw, elems = g.c * qhw;
+    for (int e = threadIdx.x; e < g.ld_dst; e += blockDim.x) {
+        int t = -1;
+        if (e < elems) {
+            const int ci = e / qhw, rem = e - ci * qhw;
+            const int gy = gy0 + rem / g.qw, gx = gx0 + rem % g.qw;
+            if (gy >= 0 && gy < g.h && gx >= 0 && gx < g.w) t = (ci * g.h + gy) * g.w + gx;
+        }
+        for (int i = 0; i < g.n_arr; ++i) {
+            float val = 0.0f;
+            if (t >= 0) val = g.src[i] ? g.src[i][(size_t)box * g.ld_src + t] : g.fill[i];
+            g.dst[i][(size_t)v * g.ld_dst + e] = val;
+        }
+    }
 }
 
 // Geometry of one patch back-step through conv layer j for the rows of conv layer k.
@@ -240,13 +290,31 @@ void conv_patch_prepare() {
                          (int)kPatchSmemMax);
 }
 
-void launch_patch_start(const LayerDev &Lk, const LayerDev &Lb, const PatchLevel &lv, int batch, float *patch,
-                        float *d, cudaStream_t st) {
+void launch_patch_start(const LayerDev &Lk, const LayerDev &Lb, int pitch, int batch, float *patch,
+                        float *patch_lo, float *d, cudaStream_t st) {
     const long long rows = 2LL * batch * Lk.n_out;
     const unsigned grid = (unsigned)ceil_div_ll(rows, kWarpsPerBlock);
-    patch_start_kernel<<<grid, kWarpsPerBlock * 32, 0, st>>>(Lk.W, geom_of(Lk), Lk.bias_n, patch, lv.pitch, d, rows,
-                                                              Lk.n_out, Lb.ld_out, Lb.relu_after, Lb.lamL, Lb.lamU,
-                                                              Lb.nuU, Lb.bias_n);
+    patch_start_kernel<<<grid, kWarpsPerBlock * 32, 0, st>>>(Lk.W, geom_of(Lk), Lk.bias_n, patch, patch_lo, pitch, d,
+                                                              rows, Lk.n_out, Lb.ld_out, Lb.relu_after, Lb.lamL,
+                                                              Lb.lamU, Lb.nuU, Lb.bias_n);
+}
+
+void launch_patch_gather(const LayerDev &Lk, const LayerDev &Lj, const PatchLevel &out, int ld_dst, int batch,
+                         int n_arr, const float *const *src, const float *fill, float *const *dst,
+                         cudaStream_t st) {
+    PatchGather g;
+    g.c = out.c; g.qh = out.ph; g.qw = out.pw;
+    g.h = Lj.h_in; g.w = Lj.w_in;
+    g.a = out.a; g.b = out.b;
+    g.w_k = Lk.w_out; g.n_pos = Lk.h_out * Lk.w_out;
+    g.ld_src = Lj.ld_in; g.ld_dst = ld_dst;
+    g.n_arr = n_arr;
+    for (int i = 0; i < 3; ++i) {
+        g.src[i] = i < n_arr ? src[i] : nullptr;
+        g.fill[i] = i < n_arr ? fill[i] : 0.0f;
+        g.dst[i] = i < n_arr ? dst[i] : nullptr;
+    }
+    patch_gather_kernel<<<(unsigned)(batch * g.n_pos), 128, 0, st>>>(g);
 }
 
 void launch_patch_step(const LayerDev &Lk, const LayerDev &Lj, const PatchLevel &in, const PatchLevel &out,

@@ -210,7 +210,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_consta
             const long long rr = row_ok ? r : 0;
             const int b = (int)(rr / (2LL * a.n_k));
             const int upper = (int)((rr / a.n_k) & 1);
-            const size_t relax_row = (size_t)b * a.ld_n;
+            // the row's vector of the relaxation / box arrays: one per box, or (rows that are patches of
+            // a conv neuron's window) one per box and output position of the neuron
+            const size_t vec = a.n_pos ? (size_t)b * a.n_pos + (size_t)((rr % a.n_k) % a.n_pos) : (size_t)b;
+            const size_t relax_row = vec * a.ld_n;
             float dacc = 0.0f;
             const int acc = lt & 1;
             const uint32_t acc_phase = (lt >> 1) & 1;
@@ -336,8 +339,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_consta
                     }
                     if (warp_row0 < a.M) a.colsum[(size_t)(warp_row0 >> 5) * a.ld_n + col0 + lane] = w[0];
                 } else if (row_ok) {
-                    const float *lrow = a.l0 + (size_t)b * a.ld_n + col0;
-                    const float *urow = a.u0 + (size_t)b * a.ld_n + col0;
+                    const float *lrow = a.l0 + relax_row + col0;
+                    const float *urow = a.u0 + relax_row + col0;
 #pragma unroll
                     for (int g = 0; g < 8; ++g) {
                         const float4 l4 = *reinterpret_cast<const float4 *>(lrow + g * 4);

@@ -205,19 +205,34 @@ CONV_NETS = {
 }
 
 
-@pytest.mark.parametrize("patches", [False, True])
+@pytest.mark.parametrize("form", ["dense", "patches_fma", "patches_tc"])
 @pytest.mark.parametrize("name", sorted(CONV_NETS))
-def test_conv_rows_dense_and_patches(name, patches):
+def test_conv_rows_dense_and_patches(name, form):
+    """Rows of a conv layer over conv layers: as dense maps, as receptive-field patches on the FMA units (one
+    warp per row), and as patches on the tensor cores (the conv layer as a dense window-to-window matrix)."""
     w = CONV_NETS[name]()
     ref = _oracle(w)
-    g = run_gpu(w, conv_patches=patches)
+    patches = form != "dense"
+    contraction = MODES["ffma"] if form == "patches_fma" else None
+    g = run_gpu(w, conv_patches=patches, contraction=contraction)
     # the small nets' windows are not much smaller than their maps: those stay dense either way
     expect_patches = patches and name in ("convsmall", "three_convs", "k5s1p0_k2s2")
     assert bool(g["paths"] & 8) == expect_patches
-    compare(g, ref, label=f"{name}/patches={patches}")
+    if expect_patches and form == "patches_tc":
+        assert g["paths"] & 2
+    compare(g, ref, label=f"{name}/{form}")
     steps = [0] + [1] * (len(w.layers) - 1)
     ref1 = orc.deeppoly(w.layers, w.centers, w.eps, w.clip_lo, w.clip_hi, backsteps_per_layer=steps)
-    compare(run_gpu(w, conv_patches=patches, backsteps=steps), ref1, label=f"{name}/patches={patches}/p1")
+    compare(run_gpu(w, conv_patches=patches, contraction=contraction, backsteps=steps), ref1, label=f"{name}/{form}/p1")
+
+
+def test_conv_patches_on_tensor_cores_ragged_batch():
+    """Fewer boxes than the net was made for, rows not a multiple of the 256-row panel."""
+    w = wl.small_conv((2, 20, 18), [(4, 3, 1, 1), (6, 4, 2, 1), (8, 3, 2, 0)], [12, 3], batch=3, eps=0.01, seed=87)
+    ref = _oracle(w)
+    g = run_gpu(w, max_batch=5, conv_patches=True)
+    assert g["paths"] & 8 and g["paths"] & 2
+    compare(g, ref, label="three_convs/ragged")
 
 
 # ---- ReuseCert (Appendix C listing): shapes kept over the input layer ----
