@@ -51,48 +51,74 @@ __device__ __forceinline__ float tf32_rn(float x) {
     return __uint_as_float(u);
 }
 
-__global__ void patch_start_kernel(const float *__restrict__ Wk, ConvGeom gk, const float *__restrict__ bias_k,
-                                   float *__restrict__ patch, float *__restrict__ patch_lo, int pitch,
-                                   float *__restrict__ d, long long rows,
-                                   int n_k, int ld, int has_relu, const float *__restrict__ lamL,
-                                   const float *__restrict__ lamU, const float *__restrict__ nuU,
-                                   const float *__restrict__ bias_below) {
-    const long long r = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-    const int lane = threadIdx.x & 31;
-    if (r >= rows) return;
-    const int b = (int)(r / (2LL * n_k));
-    const int upper = (int)((r / n_k) & 1);
-    const int i = (int)(r % n_k);
+__global__ void __launch_bounds__(kWarpsPerBlock * 32)
+patch_start_kernel(const float *__restrict__ Wk, ConvGeom gk, const float *__restrict__ bias_k,
+                   float *__restrict__ patch, float *__restrict__ patch_lo, int pitch, float *__restrict__ d,
+                   int n_k, int ld, int has_relu, const float *__restrict__ lamL, const float *__restrict__ lamU,
+                   const float *__restrict__ nuU, const float *__restrict__ bias_below) {
+    // One block per (box, output position): the window of the relaxation below is the same for the
+    // 2 * c_out rows of that position, so it is looked up once and kept in shared memory.
+    extern __shared__ __align__(16) float win[];
+    float *sL = win, *sU = win + pitch, *sN = win + 2 * pitch, *sB = win + 3 * pitch;
     const int hw_o = gk.h_out * gk.w_out;
-    const int co = i / hw_o;
-    const int y0 = ((i / gk.w_out) % gk.h_out) * gk.stride - gk.pad;
-    const int x0 = (i % gk.w_out) * gk.stride - gk.pad;
+    const int box = blockIdx.x / hw_o, pos = blockIdx.x - box * hw_o;
+    const int y0 = (pos / gk.w_out) * gk.stride - gk.pad, x0 = (pos % gk.w_out) * gk.stride - gk.pad;
     const int khw = gk.kh * gk.kw, taps = gk.c_in * khw;
-    const size_t vec = (size_t)b * ld;
-    float *prow = patch + (size_t)r * pitch;
-    float dacc = 0.0f;
-    for (int q = lane; q < pitch; q += 32) {
-        float qv = 0.0f;
+    const size_t vec = (size_t)box * ld;
+    for (int q = threadIdx.x; q < pitch; q += blockDim.x) {
+        float l = 0.0f, u = 0.0f, n = 0.0f, bz = 0.0f;
         if (q < taps) {
             const int ci = q / khw, ky = (q / gk.kw) % gk.kh, kx = q % gk.kw;
             const int iy = y0 + ky, ix = x0 + kx;
             if (iy >= 0 && iy < gk.h_in && ix >= 0 && ix < gk.w_in) {
                 const int t = (ci * gk.h_in + iy) * gk.w_in + ix;
-                const float c = Wk[(size_t)co * taps + q];
-                qv = has_relu ? relu_backstep(c, upper, lamL[vec + t], lamU[vec + t], nuU[vec + t], dacc) : c;
-                dacc = fmaf(qv, bias_below[t], dacc);
+                l = has_relu ? lamL[vec + t] : 1.0f;
+                u = has_relu ? lamU[vec + t] : 1.0f;
+                n = has_relu ? nuU[vec + t] : 0.0f;
+                bz = bias_below[t];
             }
         }
-        if (patch_lo) {
-            const float h = tf32_rn(qv);
-            prow[q] = h;
-            patch_lo[(size_t)r * pitch + q] = tf32_rn(qv - h);
-        } else {
-            prow[q] = qv;
-        }
+        sL[q] = l; sU[q] = u; sN[q] = n; sB[q] = bz;
     }
-    dacc = warp_sum(dacc);
-    if (lane == 0) d[r] = bias_k[i] + dacc;
+    __syncthreads();
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    for (int rr = warp; rr < 2 * gk.c_out; rr += kWarpsPerBlock) {
+        const int upper = rr / gk.c_out, co = rr - upper * gk.c_out;
+        const int i = co * hw_o + pos;
+        const long long r = ((long long)box * 2 + upper) * n_k + i;
+        const float *wrow = Wk + (size_t)co * taps;
+        float dacc = 0.0f;
+        for (int q0 = lane * 4; q0 < pitch; q0 += 128) {
+            const float4 l4 = *reinterpret_cast<const float4 *>(sL + q0);
+            const float4 u4 = *reinterpret_cast<const float4 *>(sU + q0);
+            const float4 n4 = *reinterpret_cast<const float4 *>(sN + q0);
+            const float4 b4 = *reinterpret_cast<const float4 *>(sB + q0);
+            const float la[4] = {l4.x, l4.y, l4.z, l4.w}, ua[4] = {u4.x, u4.y, u4.z, u4.w};
+            const float na[4] = {n4.x, n4.y, n4.z, n4.w}, ba[4] = {b4.x, b4.y, b4.z, b4.w};
+            float qv[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const float c = (q0 + e < taps) ? wrow[q0 + e] : 0.0f;
+                qv[e] = relu_backstep(c, upper, la[e], ua[e], na[e], dacc);   // zero outside the map
+                dacc = fmaf(qv[e], ba[e], dacc);
+            }
+            float *dst = patch + (size_t)r * pitch + q0;
+            if (patch_lo) {
+                float h[4], lo[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    h[e] = tf32_rn(qv[e]);
+                    lo[e] = tf32_rn(qv[e] - h[e]);
+                }
+                *reinterpret_cast<float4 *>(dst) = make_float4(h[0], h[1], h[2], h[3]);
+                *reinterpret_cast<float4 *>(patch_lo + (size_t)r * pitch + q0) = make_float4(lo[0], lo[1], lo[2], lo[3]);
+            } else {
+                *reinterpret_cast<float4 *>(dst) = make_float4(qv[0], qv[1], qv[2], qv[3]);
+            }
+        }
+        dacc = warp_sum(dacc);
+        if (lane == 0) d[r] = bias_k[i] + dacc;
+    }
 }
 
 // Per (box, output position of the conv neuron): the window of up to three per-neuron arrays of the
@@ -264,6 +290,7 @@ bool conv_patch_plan(const LayerDev *layers, int k, int j_end, PatchLevel *level
     lv.elems = lv.c * lv.ph * lv.pw;
     lv.pitch = round_up(lv.elems, 4);
     if (2 * lv.elems > Lk.n_in) return false;            // the window is not much smaller than the map
+    if (16 * (size_t)round_up(lv.elems, kPad) > 48 * 1024) return false;   // the start kernel's shared-memory window
     levels[0] = lv;
     for (int j = k - 1, m = 1; j >= j_end; --j, ++m) {
         const LayerDev &Lj = layers[j];
@@ -292,11 +319,10 @@ void conv_patch_prepare() {
 
 void launch_patch_start(const LayerDev &Lk, const LayerDev &Lb, int pitch, int batch, float *patch,
                         float *patch_lo, float *d, cudaStream_t st) {
-    const long long rows = 2LL * batch * Lk.n_out;
-    const unsigned grid = (unsigned)ceil_div_ll(rows, kWarpsPerBlock);
-    patch_start_kernel<<<grid, kWarpsPerBlock * 32, 0, st>>>(Lk.W, geom_of(Lk), Lk.bias_n, patch, patch_lo, pitch, d,
-                                                              rows, Lk.n_out, Lb.ld_out, Lb.relu_after, Lb.lamL,
-                                                              Lb.lamU, Lb.nuU, Lb.bias_n);
+    const unsigned grid = (unsigned)(batch * Lk.h_out * Lk.w_out);
+    patch_start_kernel<<<grid, kWarpsPerBlock * 32, 4 * (size_t)pitch * sizeof(float), st>>>(
+        Lk.W, geom_of(Lk), Lk.bias_n, patch, patch_lo, pitch, d, Lk.n_out, Lb.ld_out, Lb.relu_after, Lb.lamL, Lb.lamU,
+        Lb.nuU, Lb.bias_n);
 }
 
 void launch_patch_gather(const LayerDev &Lk, const LayerDev &Lj, const PatchLevel &out, int ld_dst, int batch,

@@ -99,6 +99,43 @@ __global__ void first_layer_kernel(const float *__restrict__ W, const float *__r
     }
 }
 
+// The same for a conv layer with one thread per (box, neuron): a neuron has only c_in*kh*kw taps, and
+// the threads of a warp are neighbouring positions of one channel, so the weights are warp-uniform loads.
+__global__ void first_layer_conv_kernel(const float *__restrict__ W, const float *__restrict__ bias_n, ConvGeom g,
+                                        int n_out, const float *__restrict__ l0, const float *__restrict__ u0,
+                                        int ld0, int batch, float *__restrict__ lb_out,
+                                        float *__restrict__ ub_out, int n_total, int out_off) {
+    pdl_trigger();
+    pdl_wait();
+    const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= (long long)batch * n_out) return;
+    const int b = (int)(idx / n_out), i = (int)(idx % n_out);
+    const float *lrow = l0 + (size_t)b * ld0, *urow = u0 + (size_t)b * ld0;
+    const int hw = g.h_out * g.w_out;
+    const int co = i / hw, oy = (i / g.w_out) % g.h_out, ox = i % g.w_out;
+    const int y0 = oy * g.stride - g.pad, x0 = ox * g.stride - g.pad;
+    const float *w = W + (size_t)co * g.c_in * g.kh * g.kw;
+    float lo = 0.0f, hi = 0.0f;
+    for (int ci = 0; ci < g.c_in; ++ci)
+        for (int ky = 0; ky < g.kh; ++ky) {
+            const int iy = y0 + ky;
+            if (iy < 0 || iy >= g.h_in) continue;
+            const int base = (ci * g.h_in + iy) * g.w_in;
+            const float *wr = w + (ci * g.kh + ky) * g.kw;
+            for (int kx = 0; kx < g.kw; ++kx) {
+                const int ix = x0 + kx;
+                if (ix < 0 || ix >= g.w_in) continue;
+                const float c = wr[kx], l = lrow[base + ix], u = urow[base + ix];
+                const bool nn = (c >= 0.0f);
+                lo = fmaf(c, nn ? l : u, lo);
+                hi = fmaf(c, nn ? u : l, hi);
+            }
+        }
+    const float bb = bias_n[i];
+    lb_out[(size_t)b * n_total + out_off + i] = lo + bb;
+    ub_out[(size_t)b * n_total + out_off + i] = hi + bb;
+}
+
 // Sum of the slots that hold a row's constant (or bound), in slot order.
 __device__ __forceinline__ float slot_sum(const float *__restrict__ d, int n_slots, long long stride,
                                           long long r) {
@@ -396,6 +433,11 @@ void launch_box(const float *centers, float eps, float lo, float hi, int batch, 
 void launch_first_layer_bounds(const LayerDev &L, const float *l0, const float *u0, int ld0, int batch,
                                float *lb_out, float *ub_out, int n_total, cudaStream_t st) {
     long long warps = (long long)batch * L.n_out;
+    if (L.kind == CERT_LAYER_CONV2D) {
+        launch_chained(first_layer_conv_kernel, dim3((unsigned)ceil_div_ll(warps, 128)), dim3(128), 0, st, L.W, L.bias_n,
+                       geom_of(L), L.n_out, l0, u0, ld0, batch, lb_out, ub_out, n_total, L.out_off);
+        return;
+    }
     launch_chained(first_layer_kernel, dim3(grid_for_warps(warps)), dim3(kWarpsPerBlock * 32), 0, st, L.W, L.bias_n,
                    L.kind, geom_of(L), L.n_in, L.ld_in, L.n_out, l0, u0, ld0, batch, lb_out, ub_out, n_total, L.out_off);
 }
