@@ -185,7 +185,10 @@ enum { CERT_CONTRACTION_AUTO = 0, CERT_CONTRACTION_FFMA = 1, CERT_CONTRACTION_TC
 cert_status_t cert_net_set_contraction(cert_net_t *net, int mode);
 /* Which contraction kernels the most recent call ran: bit 0 = FFMA, bit 1 = TC3XTF32,
  * bit 2 = the TC3XTF32 kernel ran in its CTA-pair form (tcgen05 cta_group::2), bit 3 = a traversal ran on
- * receptive-field patches, bit 4 = TC3XFP16. */
+ * receptive-field patches, bit 4 = TC3XFP16, bit 5 = TC3XFP16 with a whole traversal per launch (nets whose
+ * hidden layers are at most 256 neurons wide keep the coefficient panel in shared memory from the start of
+ * a traversal to its concretisation; the environment variable CERT_CHAIN=0, read at create, keeps such nets
+ * on one launch per back-step). */
 int cert_net_last_contraction_paths(const cert_net_t *net);
 
 /*

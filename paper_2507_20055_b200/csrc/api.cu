@@ -12,6 +12,7 @@
 #include "common.cuh"
 #include "gemm_tc.cuh"
 #include "gemm_tc16.cuh"
+#include "chain16.cuh"
 
 // Tensor-core operands of the back-step through one FC layer j: B = W_j transposed
 // (rows = neurons below, K-major), A = the coefficient matrix over layer j's neurons
@@ -86,6 +87,10 @@ struct cert_net {
     std::vector<TcLayer> tc;                 // per layer: operand maps and tile plan
     bool tc16_ok = false;                    // fp16-split path usable (FC layers only, CTA pairs available)
     std::vector<Tc16Layer> tc16;
+    // fp16-split path, narrow nets: a whole traversal per launch with the coefficient panel kept in shared memory
+    bool chain_ok = false;
+    cert::ChainParams chain;
+    int chain_a_blocks = 0, chain_stages = 0, chain_smem = 0;
     float *dbuf[2] = {nullptr, nullptr};     // row constants, [d_slots][slot_stride] each, ping-pong
     int d_slots = 1;                         // slots per buffer (most column tiles of any contraction)
     long long slot_stride = 0;               // rows of the largest coefficient matrix
@@ -292,6 +297,33 @@ cert_status_t setup_tensor_core_path(cert_net *net, const cert_layer_desc_t *des
             if (ok) net->d_slots = std::max(net->d_slots, 2 * T.plan.n_tiles);
         }
         net->tc16_ok = all_ok;
+        // The chain kernel: every layer a traversal passes through at most kChainMaxWidth neurons wide.
+        bool chain = all_ok && K <= cert::kChainMaxLayers && cert::chain16_prepare();
+        if (const char *e = std::getenv("CERT_CHAIN")) chain = chain && std::atoi(e) != 0;
+        int widest = 0;
+        for (int j = 0; j + 1 < K; ++j) widest = std::max(widest, net->layers[j].n_out);
+        if (chain && widest <= cert::kChainMaxWidth) {
+            net->chain_a_blocks = (widest + 63) / 64;
+            net->chain_smem = cert::chain16_smem_bytes(net->chain_a_blocks, &net->chain_stages);
+            std::memset(&net->chain, 0, sizeof(net->chain));
+            for (int j = 0; j < K; ++j) {
+                const LayerDev &L = net->layers[j];
+                cert::ChainLayer &C = net->chain.layer[j];
+                C.n_out = L.n_out; C.n_in = L.n_in; C.ld_in = L.ld_in;
+                if (j + 1 < K) {
+                    net->chain.b_hi[j] = net->tc16[j].b_hi;
+                    net->chain.b_lo[j] = net->tc16[j].b_lo;
+                    C.bn = net->tc16[j].plan.bn; C.n_tiles = net->tc16[j].plan.n_tiles;
+                }
+                if (j > 0) {
+                    const LayerDev &Lb = net->layers[j - 1];
+                    C.relu_below = Lb.relu_after;
+                    C.lamL = Lb.lamL; C.lamU = Lb.lamU; C.nuU = Lb.nuU; C.bias_below = Lb.bias_n;
+                }
+            }
+            net->chain_ok = net->chain_stages >= 2;
+            net->d_slots = std::max(net->d_slots, cert::kChainColGroups);
+        }
     }
     return CERT_OK;
 }
@@ -621,6 +653,24 @@ cert_status_t cert_backsub_bounds(cert_net_t *net, const float *centers, float e
         };
         // fp16-split tensor-core chain (FC nets): start, then one kernel per layer with the ReLU step fused,
         // the last one concretising.
+        if (net->contraction == CERT_CONTRACTION_TC3XFP16 && net->chain_ok) {
+            cert::ChainArgs a;
+            std::memset(&a, 0, sizeof(a));
+            a.M = rows; a.n_k = Lk.n_out; a.k = k; a.j_end = j_end;
+            a.Wk = Lk.W; a.ldw_k = Lk.ld_in; a.bias_k = Lk.bias_n;
+            a.box_l = box_l; a.box_u = box_u;
+            a.d_out = net->dbuf[0]; a.slot_stride = net->slot_stride;
+            a.status = net->status_dev;
+            a.stages = net->chain_stages; a.a_blocks = net->chain_a_blocks;
+            const int pairs = (int)std::min<long long>(cert::ceil_div_ll(rows, 256), net->sm_count / 2);
+            cert::launch_chain16(net->chain, a, pairs, net->chain_smem, st);
+            rec.mark(CERT_CLASS_AFFINE);
+            cert::launch_relax(Lk, lb_out, ub_out, n_total, batch, net->codes, net->n_relu, net->dbuf[0], cert::kChainColGroups,
+                               net->slot_stride, st);
+            rec.mark(CERT_CLASS_RELAX);
+            paths |= 2 | 4 | 16 | 32;
+            continue;
+        }
         if (net->contraction == CERT_CONTRACTION_TC3XFP16 && net->tc16_ok) {
             __half *qh[2] = {reinterpret_cast<__half *>(net->buf[0]), reinterpret_cast<__half *>(net->buf[1])};
             __half *ql[2] = {reinterpret_cast<__half *>(net->buf_lo[0]), reinterpret_cast<__half *>(net->buf_lo[1])};

@@ -348,12 +348,32 @@ FC_NETS = {
 }
 
 
+@pytest.mark.parametrize("chain", [True, False])
 @pytest.mark.parametrize("name", sorted(FC_NETS))
-def test_fp16_split_contraction(name):
+def test_fp16_split_contraction(name, chain, monkeypatch):
+    """Narrow nets: a whole traversal per launch (the coefficient panel stays in shared memory), and, with
+    CERT_CHAIN=0 at create, one launch per back-step as for wide nets."""
+    if not chain:
+        monkeypatch.setenv("CERT_CHAIN", "0")
     w = FC_NETS[name]()
     g = run_gpu(w, contraction=TC16)
     assert g["paths"] & 16
-    compare(g, _oracle(w), label=f"{name}/tc16")
+    narrow = max(l.weight.shape[0] for l in w.layers[:-1]) <= 256
+    assert bool(g["paths"] & 32) == (chain and narrow)
+    compare(g, _oracle(w), label=f"{name}/tc16/chain={chain}")
+
+
+def test_fp16_split_chain_bounded_traversals_ragged_batch_and_missing_relu():
+    w = VARIANT_NETS["fc_ragged"]()
+    for vname, steps in _variant_steps(len(w.layers)).items():
+        ref = orc.deeppoly(w.layers, w.centers, w.eps, w.clip_lo, w.clip_hi, backsteps_per_layer=steps)
+        g = run_gpu(w, contraction=TC16, backsteps=steps, max_batch=w.batch + 2)
+        compare(g, ref, label=f"fc_ragged/{vname}/tc16 chain")
+    w = wl.small_fc([24, 40, 36, 40, 6], batch=3, eps=0.05, seed=71)
+    w.layers[1].relu_after = False
+    g = run_gpu(w, contraction=TC16)
+    assert g["paths"] & 32
+    compare(g, _oracle(w), label="no_relu_mid/tc16 chain")
 
 
 def test_fp16_split_config5_sampled_boxes():
