@@ -216,6 +216,7 @@ chain16_kernel(const __grid_constant__ ChainParams P, const ChainArgs a) {
                 for (int j = a.k - 1; j >= a.j_end && ok; --j) {
                     const ChainLayer &L = P.layer[j];
                     const int num_kb = (L.n_out + BKH - 1) / BKH;
+                    const int ksteps = (L.n_out + 15) / 16;       // 16-column MMA steps that hold neurons; the rest of the last block is zero
                     // the panel over layer j's neurons is in shared memory, in both CTAs
                     if (!mbar_wait_cluster(&bars->a_ready, a_phase) || *abort_flag) { ok = false; break; }
                     a_phase ^= 1;
@@ -239,6 +240,7 @@ chain16_kernel(const __grid_constant__ ChainParams P, const ChainArgs a) {
                             const uint64_t db_lo = make_desc(st + kBChunkBytes);
 #pragma unroll
                             for (int k = 0; k < BKH / 16; ++k) {
+                                if (kb * (BKH / 16) + k >= ksteps) break;
                                 const uint64_t ko = (uint64_t)(k * 2);   // 16 halves = 32 bytes = 2 x 16-byte units
                                 mma_f16<CTAS>(d, da_lo + ko, db_hi + ko, idesc, (kb | k) ? 1u : 0u);
                                 mma_f16<CTAS>(d, da_hi + ko, db_lo + ko, idesc, 1u);
@@ -257,6 +259,7 @@ chain16_kernel(const __grid_constant__ ChainParams P, const ChainArgs a) {
                                 const uint64_t db = make_desc(st + (uint32_t)h * kBChunkBytes);
 #pragma unroll
                                 for (int k = 0; k < BKH / 16; ++k) {
+                                    if ((kb + h) * (BKH / 16) + k >= ksteps) break;
                                     const uint64_t ko = (uint64_t)(k * 2);
                                     if (kb == 0 && h == 0 && k == 0) mma_f16_pair_scaled<11>(d, da + ko, db + ko, idesc);
                                     else mma_f16<CTAS>(d, da + ko, db + ko, idesc, 1u);
