@@ -410,7 +410,10 @@ def main():
                 "flops_per_step_if_dense_maps": fl_dense[dom], "conv_rows_as_patches": used_patches,
                 "peak_source": peaks["source"],
                 "peak_note": (("bf16_tflops_sustained/3 (3xFP16)" if used_fp16 else "bf16_tflops_sustained/2/3 (3xTF32)")
-                              if used_tc else "148 SM x 128 FMA x 2 x sm_max_mhz"),
+                              if used_tc else "148 SM x 128 FMA x 2 x sm_max_mhz" +
+                              ("; the conv class also holds the patch back-step, which runs on the tensor cores "
+                               "(gather + 3xTF32 contraction with the window-to-window matrix), counted at its "
+                               "algorithmic flops" if used_patches and args.contraction != "ffma" else "")),
                 "class_ms_per_step": {k: v / args.steps for k, v in cls_ms.items()}}
         out = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
