@@ -59,13 +59,19 @@ def box(centers, eps, clip_lo, clip_hi):
     return l0, u0
 
 
-def deeppoly_matrix(layers, centers, eps, clip_lo=0.0, clip_hi=1.0, decision_fp32=True, backsteps=None):
+def deeppoly_matrix(layers, centers, eps, clip_lo=0.0, clip_hi=1.0, decision_fp32=True, backsteps=None,
+                    skip_from=None):
     """Returns lb, ub [batch, n_total] float64 and codes [batch, n_relu] uint8.
 
     backsteps: optional list with one traversal-step count per affine layer (negative: to the
     input).  A traversal that stops early is simplified against the concrete bounds of the
     neurons it reached (Section 6.2, DeepPoly_p; 0 everywhere is the IBP listing, 0 except at
-    the last layer the CROWN-IBP listing of Appendix C)."""
+    the last layer the CROWN-IBP listing of Appendix C).
+    skip_from: optional residual connections (layer k adds the outputs of layer skip_from[k]; full
+    traversals only): the coefficient matrix on those outputs is set aside and joins the expression
+    when the traversal, highest layer first, has come down to that layer."""
+    if skip_from is not None:
+        assert backsteps is None
     A = [dense_matrix(l) for l in layers]
     bias = [dense_bias(l) for l in layers]
     L0, U0 = box(centers, eps, clip_lo, clip_hi)
@@ -85,7 +91,14 @@ def deeppoly_matrix(layers, centers, eps, clip_lo=0.0, clip_hi=1.0, decision_fp3
             dl, du = bias[k].copy(), bias[k].copy()
             limit = -1 if backsteps is None else int(backsteps[k])
             stop_at = -1 if limit < 0 else max(k - 1 - limit, -1)   # layer whose outputs the expression ends on
+            waiting = {}
+            if skip_from is not None and skip_from[k] >= 0:
+                eye = np.eye(A[k].shape[0])
+                waiting[skip_from[k]] = (eye, eye.copy())
             for j in range(k - 1, stop_at, -1):
+                if j in waiting:
+                    Wl, Wu = waiting.pop(j)
+                    Cl, Cu = Cl + Wl, Cu + Wu
                 if layers[j].relu_after:
                     Clp, Clm = np.clip(Cl, 0.0, None), np.clip(Cl, None, 0.0)
                     Cup, Cum = np.clip(Cu, 0.0, None), np.clip(Cu, None, 0.0)
@@ -93,6 +106,9 @@ def deeppoly_matrix(layers, centers, eps, clip_lo=0.0, clip_hi=1.0, decision_fp3
                     du = du + Cup @ nu_u[j]
                     Cl = Clp * lam_l[j] + Clm * lam_u[j]
                     Cu = Cup * lam_u[j] + Cum * lam_l[j]
+                if skip_from is not None and skip_from[j] >= 0:
+                    Wl, Wu = waiting.get(skip_from[j], (0.0, 0.0))
+                    waiting[skip_from[j]] = (Wl + Cl, Wu + Cu)
                 dl = dl + Cl @ bias[j]
                 du = du + Cu @ bias[j]
                 Cl = Cl @ A[j]

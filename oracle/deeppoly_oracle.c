@@ -235,7 +235,7 @@ static void relu_relaxation(double l, double u, int decision_fp32, double *lamL,
  * (flow(forward, priority = layer)). */
 static int one_box(const oracle_layer_t *layers, int n_layers, const float *center, float eps,
                    float clip_lo, float clip_hi, int decision_fp32, int max_backsteps_all,
-                   const int *backsteps_per_layer, int skip_form,
+                   const int *backsteps_per_layer, int skip_form, const int *skip_from,
                    double *lb, double *ub, unsigned char *codes, double *margins)
 {
     int n0 = layer_n_in(&layers[0]);
@@ -251,7 +251,11 @@ static int one_box(const oracle_layer_t *layers, int n_layers, const float *cent
     double *nuU = malloc(sizeof(double) * n_total);
     double *row = malloc(sizeof(double) * n_max);
     int *off = malloc(sizeof(int) * (n_layers + 1));
-    if (!l0 || !u0 || !coef || !next || !lamL || !lamU || !nuU || !off || !row) return 1;
+    /* Residual connections: pend + off[t] holds coefficients over the outputs of layer t that
+     * wait for the traversal to come down to that layer (has[t] != 0). */
+    double *pend = calloc((size_t)n_total, sizeof(double));
+    int *has = calloc((size_t)n_layers, sizeof(int));
+    if (!l0 || !u0 || !coef || !next || !lamL || !lamU || !nuU || !off || !row || !pend || !has) return 1;
 
     /* The box endpoints are binary32 values: fl(c -/+ eps) clipped. */
     for (int s = 0; s < n0; ++s) {
@@ -273,10 +277,23 @@ static int one_box(const oracle_layer_t *layers, int n_layers, const float *cent
             for (int upper = 0; upper < 2; ++upper) {
                 double d;
                 affine_row(&layers[k], i, coef, &d);
+                /* A neuron of a layer with a residual connection is an affine neuron whose prev
+                 * also holds neuron i of layer skip_from[k], with weight 1. */
+                if (skip_from && skip_from[k] >= 0) {
+                    pend[off[skip_from[k]] + i] += 1.0;
+                    has[skip_from[k]] = 1;
+                }
                 int steps = 0;
                 int j = k - 1;                 /* coef is over the outputs of layer j */
                 for (; j >= 0; --j) {
                     if (max_backsteps >= 0 && steps >= max_backsteps) break;
+                    if (has[j]) {
+                        /* priority -layer: neurons of layer j are replaced only now, with all the
+                         * coefficient they have gathered */
+                        int n_j = layer_n_out(&layers[j]);
+                        for (int t = 0; t < n_j; ++t) { coef[t] += pend[off[j] + t]; pend[off[j] + t] = 0.0; }
+                        has[j] = 0;
+                    }
                     if (skip_form && layers[j].relu_after) {
                         replace_through_relu_skip(&layers[j], upper, lamL + off[j], lamU + off[j],
                                                   nuU + off[j], coef, next, row, &d);
@@ -284,6 +301,12 @@ static int one_box(const oracle_layer_t *layers, int n_layers, const float *cent
                         if (layers[j].relu_after)
                             replace_through_relu(layer_n_out(&layers[j]), upper, lamL + off[j],
                                                  lamU + off[j], nuU + off[j], coef, &d);
+                        if (skip_from && skip_from[j] >= 0) {
+                            /* coef is over the affine neurons of layer j = W_j a_{j-1} + b_j + a_s */
+                            int sfrom = skip_from[j], n_j = layer_n_out(&layers[j]);
+                            for (int t = 0; t < n_j; ++t) pend[off[sfrom] + t] += coef[t];
+                            has[sfrom] = 1;
+                        }
                         replace_through_affine(&layers[j], coef, next, &d);
                     }
                     double *tmp = coef; coef = next; next = tmp;
@@ -322,6 +345,7 @@ static int one_box(const oracle_layer_t *layers, int n_layers, const float *cent
         }
     }
     free(l0); free(u0); free(coef); free(next); free(lamL); free(lamU); free(nuU); free(off); free(row);
+    free(pend); free(has);
     return 0;
 }
 
@@ -356,17 +380,32 @@ int oracle_num_relu_neurons(const oracle_layer_t *layers, int n_layers)
  * with the Relu transformer (relu(l), relu(u), relu_n, compute_upper) unchanged.
  * skip_form != 0: the SkipPoly listing (ReLU shapes expressed two layers back; one traversal
  * round per ReLU layer).
+ * skip_from (optional, [n_layers]): residual connections.  skip_from[k] = s >= 0 (s <= k-2, equal widths)
+ * makes layer k compute W_k a_{k-1} + b_k + a_s with a_s the outputs of layer s (after its ReLU, if it
+ * has one); -1 = none.  Reading: such a neuron is the listing's Affine neuron whose prev holds neurons
+ * of two layers (its own row of W_k over layer k-1, weight 1 on neuron i of layer s); the traversal's
+ * priority -layer then replaces the neurons of the highest layer first, so the coefficient on a_s waits
+ * until the rest of the expression has come down to layer s.
  * n_threads: boxes are independent and are the only parallel axis.
  * Returns 0, or 1 on allocation failure, 2 on a malformed network.
  */
 int oracle_backsub(const oracle_layer_t *layers, int n_layers, const float *centers, float eps,
                    int batch, float clip_lo, float clip_hi, int decision_fp32, int max_backsteps,
-                   const int *backsteps_per_layer, int skip_form,
+                   const int *backsteps_per_layer, int skip_form, const int *skip_from,
                    int n_threads, double *lb, double *ub, unsigned char *codes, double *margins)
 {
     if (n_layers < 1 || batch < 0) return 2;
     for (int k = 1; k < n_layers; ++k)
         if (layer_n_in(&layers[k]) != layer_n_out(&layers[k - 1])) return 2;
+    if (skip_from) {
+        /* residual connections: full traversals of the DeepPoly listing only */
+        if (skip_form || backsteps_per_layer || max_backsteps >= 0) return 2;
+        for (int k = 0; k < n_layers; ++k) {
+            int sfrom = skip_from[k];
+            if (sfrom < 0) continue;
+            if (sfrom > k - 2 || layer_n_out(&layers[sfrom]) != layer_n_out(&layers[k])) return 2;
+        }
+    }
     int n0 = layer_n_in(&layers[0]);
     int n_total = oracle_num_neurons(layers, n_layers);
     int n_relu = oracle_num_relu_neurons(layers, n_layers);
@@ -379,7 +418,7 @@ int oracle_backsub(const oracle_layer_t *layers, int n_layers, const float *cent
 #pragma omp parallel for schedule(dynamic, 1)
     for (int b = 0; b < batch; ++b) {
         int e = one_box(layers, n_layers, centers + (size_t)b * n0, eps, clip_lo, clip_hi,
-                        decision_fp32, max_backsteps, backsteps_per_layer, skip_form,
+                        decision_fp32, max_backsteps, backsteps_per_layer, skip_form, skip_from,
                         lb + (size_t)b * n_total,
                         ub + (size_t)b * n_total, codes ? codes + (size_t)b * n_relu : NULL,
                         margins ? margins + (size_t)b * n_relu : NULL);
@@ -396,7 +435,7 @@ int oracle_deeppoly(const oracle_layer_t *layers, int n_layers, const float *cen
                     int n_threads, double *lb, double *ub, unsigned char *codes, double *margins)
 {
     return oracle_backsub(layers, n_layers, centers, eps, batch, clip_lo, clip_hi, decision_fp32,
-                          max_backsteps, NULL, 0, n_threads, lb, ub, codes, margins);
+                          max_backsteps, NULL, 0, NULL, n_threads, lb, ub, codes, margins);
 }
 
 /*

@@ -79,12 +79,13 @@ def _marshal(layers):
 
 def deeppoly(layers, centers, eps, clip_lo=0.0, clip_hi=1.0, decision_fp32=True,
              max_backsteps: int = -1, n_threads: Optional[int] = None, backsteps_per_layer=None,
-             skip_form: bool = False):
+             skip_form: bool = False, skip_from=None):
     """Bounds of every affine neuron for every box.
 
     max_backsteps = p >= 0 is DeepPoly_p; backsteps_per_layer (one count per affine layer,
     negative = traverse to the input) overrides it.  skip_form: the SkipPoly listing (ReLU shapes
-    expressed over the neurons two layers back).
+    expressed over the neurons two layers back).  skip_from (one entry per affine layer, -1 = none): residual
+    connections, layer k adds the outputs of layer skip_from[k] to its affine result (full traversals only).
     Returns dict(lb, ub: float64 [batch, n_total]; codes: uint8 [batch, n_relu];
     margins: float64 [batch, n_relu]).  Layers are concatenated in order.
     """
@@ -102,12 +103,18 @@ def deeppoly(layers, centers, eps, clip_lo=0.0, clip_hi=1.0, decision_fp32=True,
     if backsteps_per_layer is not None:
         steps = np.ascontiguousarray(backsteps_per_layer, dtype=np.int32)
         assert steps.shape == (len(layers),)
+    skips = None
+    if skip_from is not None:
+        skips = np.ascontiguousarray(skip_from, dtype=np.int32)
+        assert skips.shape == (len(layers),)
     rc = lib.oracle_backsub(arr, ctypes.c_int(len(layers)), ctypes.c_void_p(centers.ctypes.data),
                             ctypes.c_float(eps), ctypes.c_int(batch), ctypes.c_float(clip_lo),
                             ctypes.c_float(clip_hi), ctypes.c_int(int(decision_fp32)),
                             ctypes.c_int(max_backsteps),
                             ctypes.c_void_p(steps.ctypes.data if steps is not None else None),
-                            ctypes.c_int(int(bool(skip_form))), ctypes.c_int(n_threads or 0),
+                            ctypes.c_int(int(bool(skip_form))),
+                            ctypes.c_void_p(skips.ctypes.data if skips is not None else None),
+                            ctypes.c_int(n_threads or 0),
                             ctypes.c_void_p(lb.ctypes.data), ctypes.c_void_p(ub.ctypes.data),
                             ctypes.c_void_p(codes.ctypes.data), ctypes.c_void_p(margins.ctypes.data))
     if rc != 0:

@@ -96,6 +96,9 @@ class Workload:
     clip_lo: float = 0.0
     clip_hi: float = 1.0
     notes: dict = field(default_factory=dict)
+    # residual connections: skip_from[k] = s >= 0 adds the outputs of layer s to layer k's affine result
+    # (equal widths, s <= k-2); None or -1 = none
+    skip_from: Optional[List[int]] = None
 
     @property
     def batch(self) -> int:
@@ -194,3 +197,37 @@ def small_conv(in_shape, convs, fcs, batch, eps, seed=2) -> Workload:
         layers[-1].relu_after = False
     n0 = in_shape[0] * in_shape[1] * in_shape[2]
     return Workload("conv_small", layers, centers_uniform(batch, n0, seed), eps)
+
+
+def residual_fc(n0, width, blocks, n_out, batch, eps, seed=3) -> Workload:
+    """x -> FC(width)+ReLU -> blocks x [FC(width)+ReLU -> FC(width) (+ block input) + ReLU] -> FC(n_out):
+    a fully connected residual net in the shape of the paper's "Skip" network (Appendix, table of DNNs)."""
+    sizes = [n0, width] + [width] * (2 * blocks) + [n_out]
+    layers = fc_net(sizes, seed)
+    skip = [-1] * len(layers)
+    for b in range(blocks):
+        skip[2 + 2 * b] = 2 * b          # the block's second layer adds the block's input (outputs of layer 2b)
+    return Workload(f"resfc_{n0}_{width}x{blocks}", layers, centers_uniform(batch, n0, seed), eps, skip_from=skip)
+
+
+def residual_conv(in_shape, c, blocks, n_out, batch, eps, seed=4) -> Workload:
+    """conv(c, 3x3, s2, p1)+ReLU -> blocks x [conv(c,3x3,s1,p1)+ReLU -> conv(c,3x3,s1,p1) (+ block input) + ReLU]
+    -> FC(n_out)."""
+    layers, stream = [], 0
+    l = conv_layer(tuple(in_shape), c, 3, 2, 1, seed, stream)
+    layers.append(l)
+    shape, stream = l.out_shape, stream + 2
+    skip = [-1]
+    for b in range(blocks):
+        for half in range(2):
+            l = conv_layer(shape, c, 3, 1, 1, seed, stream)
+            layers.append(l)
+            shape, stream = l.out_shape, stream + 2
+            skip.append(2 * b if half == 1 else -1)
+    n = shape[0] * shape[1] * shape[2]
+    w = (normal(seed, stream, n_out * n) * (2.0 / n) ** 0.5).astype(np.float32).reshape(n_out, n)
+    bb = (normal(seed, stream + 1, n_out) * 0.1).astype(np.float32)
+    layers.append(Layer("fc", w, bb, relu_after=False))
+    skip.append(-1)
+    n0 = in_shape[0] * in_shape[1] * in_shape[2]
+    return Workload("resconv", layers, centers_uniform(batch, n0, seed), eps, skip_from=skip)
