@@ -69,6 +69,25 @@ cert_status_t cert_net_create(const cert_layer_desc_t *layers, int n_layers, int
                               float clip_lo, float clip_hi, cert_net_t **out);
 
 /*
+ * The same for a network with residual connections (the paper's benchmark table lists one, "Skip";
+ * Appendix, table of DNNs).  skip_from is a HOST array of n_layers ints (or NULL for none):
+ * skip_from[k] = s >= 0 makes layer k compute W_k a_{k-1} + b_k + a_s, a_s being the outputs of layer s
+ * (after its ReLU, if it has one); -1 = no connection into layer k.  Under the DeepPoly listing
+ * (Appendix C) such a neuron is an Affine neuron whose prev holds neurons of two layers, and the
+ * traversal, which replaces the neurons of the highest layer first (priority -layer), lets the
+ * coefficient on a_s wait until the rest of the expression has come down to layer s; that is what the
+ * library does: the waiting coefficient matrix stays in a third workspace buffer and is added in the
+ * epilogue of the step that reaches layer s, before the ReLU back-step.
+ * Requirements (else CERT_ERR_INVALID_ARG): s <= k-2; layers s and k have the same number of neurons;
+ * connections follow one another (none starts before the previous one has ended).
+ * Such a net is bounded by full traversals only (cert_deeppoly_bounds; cert_backsub_bounds with depths
+ * that stop early returns CERT_ERR_UNSUPPORTED), on the TF32 tensor-core and FMA kernels with dense
+ * coefficient maps (CERT_CONTRACTION_TC3XFP16, patches and cert_net_enable_reusecert are refused).
+ */
+cert_status_t cert_net_create_residual(const cert_layer_desc_t *layers, int n_layers, const int *skip_from,
+                                       int max_batch, float clip_lo, float clip_hi, cert_net_t **out);
+
+/*
  * DeepPoly bounds of every affine neuron for `batch` L-infinity boxes.
  *   centers  DEVICE float32 [batch][n0]; box b is
  *            [max(c - eps, clip_lo), min(c + eps, clip_hi)] per coordinate,

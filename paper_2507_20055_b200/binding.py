@@ -26,7 +26,7 @@ CERT_OK = 0
 CONTRACTION_AUTO, CONTRACTION_FFMA, CONTRACTION_TC3XTF32, CONTRACTION_TC3XFP16 = 0, 1, 2, 3
 
 EXPORTS = [
-    "cert_net_create", "cert_deeppoly_bounds", "cert_backsub_bounds", "cert_deeppoly_bounds_host",
+    "cert_net_create", "cert_net_create_residual", "cert_deeppoly_bounds", "cert_backsub_bounds", "cert_deeppoly_bounds_host",
     "cert_backsub_bounds_host",
     "cert_net_destroy",
     "cert_net_num_neurons", "cert_net_num_relu_neurons", "cert_net_branch_codes",
@@ -48,6 +48,8 @@ class cert_layer_desc_t(ctypes.Structure):
 _vp, _i, _f = ctypes.c_void_p, ctypes.c_int, ctypes.c_float
 _lib.cert_net_create.argtypes = [ctypes.POINTER(cert_layer_desc_t), _i, _i, _f, _f, ctypes.POINTER(_vp)]
 _lib.cert_net_create.restype = _i
+_lib.cert_net_create_residual.argtypes = [ctypes.POINTER(cert_layer_desc_t), _i, _vp, _i, _f, _f, ctypes.POINTER(_vp)]
+_lib.cert_net_create_residual.restype = _i
 _lib.cert_deeppoly_bounds.argtypes = [_vp, _vp, _f, _i, _vp, _vp, _vp]
 _lib.cert_deeppoly_bounds.restype = _i
 _lib.cert_backsub_bounds.argtypes = [_vp, _vp, _f, _i, _vp, _vp, _vp, _vp]
@@ -130,11 +132,20 @@ def marshal_layers(layers: Sequence):
 class CertNet:
     """Owns a cert_net_t handle; the three calls of the C ABI plus the helpers."""
 
-    def __init__(self, layers: Sequence, max_batch: int, clip_lo: float = 0.0, clip_hi: float = 1.0):
+    def __init__(self, layers: Sequence, max_batch: int, clip_lo: float = 0.0, clip_hi: float = 1.0,
+                 skip_from=None):
+        """skip_from: residual connections, one entry per layer (-1 = none): cert_net_create_residual."""
         arr, keep = marshal_layers(layers)
         h = _vp()
-        _check(_lib.cert_net_create(arr, len(layers), int(max_batch), float(clip_lo), float(clip_hi),
-                                    ctypes.byref(h)), "cert_net_create")
+        if skip_from is None:
+            _check(_lib.cert_net_create(arr, len(layers), int(max_batch), float(clip_lo), float(clip_hi),
+                                        ctypes.byref(h)), "cert_net_create")
+        else:
+            assert len(skip_from) == len(layers)
+            skips = (ctypes.c_int * len(layers))(*[int(x) for x in skip_from])
+            _check(_lib.cert_net_create_residual(arr, len(layers), ctypes.cast(skips, _vp), int(max_batch),
+                                                 float(clip_lo), float(clip_hi), ctypes.byref(h)),
+                   "cert_net_create_residual")
         self._h = h
         self.max_batch = int(max_batch)
         self.n0 = int(layers[0].n_in)

@@ -28,8 +28,8 @@ struct Tc16Layer {
 struct TcLayer {
     bool usable = false;
     cert::TcMap b_hi, b_lo;          // box = this CTA's share of the column tile
-    cert::TcMap a_hi[2], a_lo[2];
-    cert::TcMap o_hi[2], o_lo[2];    // store maps of the result (width = neurons below, padded); j >= 1 only
+    cert::TcMap a_hi[3], a_lo[3];    // one per coefficient buffer
+    cert::TcMap o_hi[3], o_lo[3];    // store maps of the result (width = neurons below, padded); j >= 1 only
     cert::TcPlan plan;
 };
 
@@ -81,8 +81,12 @@ struct cert_net {
     std::vector<cert::LayerDev> layers;
     std::vector<void *> allocs;   // every device allocation, for destroy
     float *l0 = nullptr, *u0 = nullptr;      // [max_batch][ld0]
-    float *buf[2] = {nullptr, nullptr};      // ping-pong coefficient matrices (fp32, or the TF32 hi parts)
-    float *buf_lo[2] = {nullptr, nullptr};   // TF32 lo parts for the tensor-core contraction
+    // coefficient matrices (fp32, or the TF32 hi parts): two that alternate, and for nets with residual
+    // connections a third, so that the matrix a connection sets aside stays put while the traversal goes on
+    float *buf[3] = {nullptr, nullptr, nullptr};
+    float *buf_lo[3] = {nullptr, nullptr, nullptr};   // TF32 lo parts for the tensor-core contraction
+    std::vector<int> skip_from;              // residual connections: layer k adds the outputs of layer skip_from[k] (-1: none); empty: none at all
+    int n_buf = 2;
     bool tc_ok = false;                      // tensor-core path usable on this net
     std::vector<TcLayer> tc;                 // per layer: operand maps and tile plan
     bool tc16_ok = false;                    // fp16-split path usable (FC layers only, CTA pairs available)
@@ -151,6 +155,12 @@ void free_net(cert_net *net) {
     delete net;
 }
 
+// Neurons of a (validated) conv layer descriptor.
+int desc_conv_out(const cert_layer_desc_t &L) {
+    const int ho = (L.h_in + 2 * L.pad - L.kh) / L.stride + 1, wo = (L.w_in + 2 * L.pad - L.kw) / L.stride + 1;
+    return L.c_out * ho * wo;
+}
+
 cert_status_t validate(const cert_layer_desc_t *layers, int n_layers, int max_batch, float clip_lo,
                        float clip_hi) {
     if (!layers || n_layers < 1 || max_batch < 1) return CERT_ERR_INVALID_ARG;
@@ -207,8 +217,8 @@ cert_status_t setup_tensor_core_path(cert_net *net, const cert_layer_desc_t *des
         if (std::atoi(e) == 1) net->tc_ctas = 1;
     }
     const int ctas = net->tc_ctas;
-    if (!dev_alloc_zero(net, &net->buf_lo[0], max_elems) || !dev_alloc_zero(net, &net->buf_lo[1], max_elems))
-        return CERT_ERR_OOM;
+    for (int p = 0; p < net->n_buf; ++p)
+        if (!dev_alloc_zero(net, &net->buf_lo[p], max_elems)) return CERT_ERR_OOM;
     std::vector<float> hi, lo;
     for (int j = 0; j < K - 1; ++j) {
         LayerDev &L = net->layers[j];
@@ -238,7 +248,7 @@ cert_status_t setup_tensor_core_path(cert_net *net, const cert_layer_desc_t *des
         // rows of the largest layer above j
         long long rows_max = 0;
         for (int k = j + 1; k < K; ++k) rows_max = std::max(rows_max, 2LL * net->max_batch * net->layers[k].n_out);
-        for (int p = 0; p < 2 && ok; ++p) {
+        for (int p = 0; p < net->n_buf && ok; ++p) {
             ok = cert::tc_make_map(&T.a_hi[p], net->buf[p], L.n_out, rows_max, L.ld_out, 128) &&
                  cert::tc_make_map(&T.a_lo[p], net->buf_lo[p], L.n_out, rows_max, L.ld_out, 128);
             if (ok && j > 0)
@@ -251,7 +261,7 @@ cert_status_t setup_tensor_core_path(cert_net *net, const cert_layer_desc_t *des
     net->tc_ok = true;
 
     // fp16-split operands: nets of FC layers, CTA pairs available
-    bool all_fc = true;
+    bool all_fc = net->skip_from.empty();      // (nets with residual connections stay on the TF32 / FMA kernels)
     for (int j = 0; j < K; ++j) all_fc = all_fc && net->layers[j].kind == CERT_LAYER_FC;
     net->tc16.assign(K, Tc16Layer());
     if (all_fc && ctas == 2 && cert::tc16_prepare_kernels()) {
@@ -338,7 +348,7 @@ constexpr size_t kPatchMatrixMax = 16u << 20;   // floats
 cert_status_t setup_patch_tc(cert_net *net, const cert_layer_desc_t *descs) {
     const int K = net->n_layers;
     net->tcp.assign(K, std::vector<TcPatchStep>());
-    if (!net->tc_ok) return CERT_OK;
+    if (!net->tc_ok || !net->skip_from.empty()) return CERT_OK;
     const int ctas = net->tc_ctas;
     size_t gat_floats = 0;
     std::vector<float> hi, lo, be;
@@ -451,10 +461,31 @@ const char *cert_status_string(cert_status_t s) {
 
 cert_status_t cert_net_create(const cert_layer_desc_t *layers, int n_layers, int max_batch, float clip_lo,
                               float clip_hi, cert_net_t **out) {
+    return cert_net_create_residual(layers, n_layers, nullptr, max_batch, clip_lo, clip_hi, out);
+}
+
+cert_status_t cert_net_create_residual(const cert_layer_desc_t *layers, int n_layers, const int *skip_from,
+                                       int max_batch, float clip_lo, float clip_hi, cert_net_t **out) {
     if (!out) return CERT_ERR_INVALID_ARG;
     *out = nullptr;
     cert_status_t v = validate(layers, n_layers, max_batch, clip_lo, clip_hi);
     if (v != CERT_OK) return v;
+    bool any_skip = false;
+    if (skip_from) {
+        // a connection spans at least one layer, joins equal widths, and connections follow one another
+        // (none starts inside another's span)
+        int last_end = 0;
+        for (int k = 0; k < n_layers; ++k) {
+            const int s = skip_from[k];
+            if (s < 0) continue;
+            if (s > k - 2 || s < last_end) return CERT_ERR_INVALID_ARG;
+            const int n_s = layers[s].kind == CERT_LAYER_FC ? layers[s].out_features : desc_conv_out(layers[s]);
+            const int n_k = layers[k].kind == CERT_LAYER_FC ? layers[k].out_features : desc_conv_out(layers[k]);
+            if (n_s != n_k) return CERT_ERR_INVALID_ARG;
+            last_end = k;
+            any_skip = true;
+        }
+    }
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return CERT_ERR_CUDA; }
 
@@ -467,6 +498,11 @@ cert_status_t cert_net_create(const cert_layer_desc_t *layers, int n_layers, int
         else cudaGetLastError();
     }
     net->n_layers = n_layers;
+    if (any_skip) {
+        net->skip_from.assign(skip_from, skip_from + n_layers);
+        net->n_buf = 3;
+        net->conv_patches = false;
+    }
     net->max_batch = max_batch;
     net->clip_lo = clip_lo;
     net->clip_hi = clip_hi;
@@ -570,6 +606,7 @@ cert_status_t cert_net_create(const cert_layer_desc_t *layers, int n_layers, int
         size_t b = (size_t)max_batch;
         bool ok = dev_alloc_zero(net, &net->l0, b * net->ld0) && dev_alloc_zero(net, &net->u0, b * net->ld0) &&
                   dev_alloc_zero(net, &net->buf[0], max_elems) && dev_alloc_zero(net, &net->buf[1], max_elems) &&
+                  (net->n_buf < 3 || dev_alloc_zero(net, &net->buf[2], max_elems)) &&
                   dev_alloc_zero(net, &net->codes, b * std::max(1, net->n_relu)) &&
                   dev_alloc_zero(net, &net->status_dev, 1) &&
                   dev_alloc_zero(net, &net->centers_dev, b * net->n0) &&
@@ -611,6 +648,10 @@ cert_status_t cert_backsub_bounds(cert_net_t *net, const float *centers, float e
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const int K = net->n_layers;
     const int n_total = net->n_total;
+    const bool residual = !net->skip_from.empty();
+    if (residual && backsteps)
+        for (int k = 1; k < K; ++k)
+            if (backsteps[k] >= 0 && backsteps[k] < k) return CERT_ERR_UNSUPPORTED;   // full traversals only
     Recorder rec(net, st);
     int paths = 0;
 
@@ -806,10 +847,34 @@ cert_status_t cert_backsub_bounds(cert_net_t *net, const float *centers, float e
         cert::launch_init_expr(Lk, net->layers[k - 1], batch, net->buf[cur],
                                on_tc(k - 1) ? net->buf_lo[cur] : nullptr, net->dbuf[dcur], st);
         rec.mark(CERT_CLASS_RELU_STEP);
+        // Residual connections: the coefficients on a connection's source wait (kept: the buffer that holds
+        // them, untouched meanwhile; identity: the unit coefficient of layer k's own connection) until the
+        // step whose result is over that source's outputs, where they join before the ReLU back-step.
+        int wait_for = residual ? net->skip_from[k] : -1;
+        bool wait_identity = wait_for >= 0;
+        int kept = -1;
+        bool kept_pair = false;
         for (int j = k - 1; j >= j_end; --j) {
             const LayerDev &Lj = net->layers[j];
-            float *Q = net->buf[cur], *P = net->buf[cur ^ 1];
-            float *P_lo = (j > j_end && on_tc(j - 1)) ? net->buf_lo[cur ^ 1] : nullptr;
+            if (residual && net->skip_from[j] >= 0) {
+                // the expression is over layer j's affine neurons = W_j a_{j-1} + b_j + a_s: its matrix stays
+                // where it is as the coefficients on a_s
+                wait_for = net->skip_from[j];
+                wait_identity = false;
+                kept = cur;
+                kept_pair = on_tc(j);
+            }
+            int nxt = cur ^ 1;
+            if (residual) {
+                nxt = 0;
+                while (nxt == cur || nxt == kept) ++nxt;
+            }
+            const bool join = j > j_end && wait_for == j - 1;
+            const float *add_hi = (join && kept >= 0) ? net->buf[kept] : nullptr;
+            const float *add_lo = (join && kept >= 0 && kept_pair) ? net->buf_lo[kept] : nullptr;
+            const int add_identity = (join && wait_identity) ? 1 : 0;
+            float *Q = net->buf[cur], *P = net->buf[nxt];
+            float *P_lo = (j > j_end && on_tc(j - 1)) ? net->buf_lo[nxt] : nullptr;
             if (on_tc(j)) {
                 const TcLayer &T = net->tc[j];
                 cert::TcArgs a;
@@ -828,8 +893,9 @@ cert_status_t cert_backsub_bounds(cert_net_t *net, const float *centers, float e
                     a.has_relu = Lb.relu_after;
                     a.split_out = P_lo != nullptr;
                     a.lamL = Lb.lamL; a.lamU = Lb.lamU; a.nuU = Lb.nuU; a.bias_below = Lb.bias_n;
+                    a.add_hi = add_hi; a.add_lo = add_lo; a.add_identity = add_identity;
                     cert::launch_gemm_tc(cert::TC_EPI_RELU, ctas, groups, T.a_hi[cur], T.a_lo[cur], T.b_hi, T.b_lo,
-                                         T.o_hi[cur ^ 1], T.o_lo[cur ^ 1], a, T.plan.smem_bytes, st);
+                                         T.o_hi[nxt], T.o_lo[nxt], a, T.plan.smem_bytes, st);
                 } else {
                     a.l0 = box_l; a.u0 = box_u;
                     cert::launch_gemm_tc(cert::TC_EPI_CONCRETIZE, ctas, groups, T.a_hi[cur], T.a_lo[cur], T.b_hi,
@@ -838,7 +904,8 @@ cert_status_t cert_backsub_bounds(cert_net_t *net, const float *centers, float e
                 }
                 rec.mark(CERT_CLASS_AFFINE);
                 paths |= 2 | (net->tc_ctas == 2 ? 4 : 0);
-                cur ^= 1;
+                if (join) { wait_for = -1; wait_identity = false; kept = -1; }
+                cur = nxt;
                 dcur ^= 1;
                 dslots = T.plan.n_tiles;
                 continue;
@@ -856,6 +923,7 @@ cert_status_t cert_backsub_bounds(cert_net_t *net, const float *centers, float e
                     ep.has_relu = Lb.relu_after;
                     ep.lamL = Lb.lamL; ep.lamU = Lb.lamU; ep.nuU = Lb.nuU; ep.bias_below = Lb.bias_n;
                     ep.P = P; ep.P_lo = P_lo;
+                    ep.add_hi = add_hi; ep.add_lo = add_lo; ep.add_identity = add_identity;
                 } else {
                     ep.mode = cert::CONVT_EPI_CONCRETIZE;
                     ep.l0 = box_l; ep.u0 = box_u;
@@ -863,14 +931,20 @@ cert_status_t cert_backsub_bounds(cert_net_t *net, const float *centers, float e
                 }
                 cert::launch_convt_ffma(Lj, Q, rows, net->sm_count, ep, st);
                 rec.mark(CERT_CLASS_CONV);
-                cur ^= 1;
+                if (join) { wait_for = -1; wait_identity = false; kept = -1; }
+                cur = nxt;
                 dslots = 1;
                 continue;
             }
             cert::launch_gemm_ffma(Q, Lj.ld_out, Lj.W, Lj.ld_in, P, Lj.ld_in, rows, Lj.n_in, Lj.n_out, st);
             rec.mark(CERT_CLASS_AFFINE);
             paths |= 1;
-            cur ^= 1;
+            cur = nxt;
+            if (join) {
+                cert::launch_add_skip(P, add_hi, add_lo, add_identity, rows, Lj.n_in, Lj.ld_in, Lk.n_out, st);
+                rec.mark(CERT_CLASS_RELU_STEP);
+                wait_for = -1; wait_identity = false; kept = -1;
+            }
             if (j > j_end) {
                 cert::launch_relu_step(net->layers[j - 1], batch, Lk.n_out, P, P_lo, net->dbuf[dcur], dslots,
                                        net->slot_stride, st);
@@ -931,7 +1005,7 @@ cert_status_t cert_net_enable_reusecert(cert_net_t *net) {
     if (!net) return CERT_ERR_INVALID_ARG;
     if (net->reuse.on) return CERT_OK;
     const int K = net->n_layers;
-    if (K < 2 || !net->tc_ok) return CERT_ERR_UNSUPPORTED;
+    if (K < 2 || !net->tc_ok || !net->skip_from.empty()) return CERT_ERR_UNSUPPORTED;
     for (int k = 0; k < K; ++k)
         if (net->layers[k].kind != CERT_LAYER_FC) return CERT_ERR_UNSUPPORTED;
     int dev = 0;
@@ -1259,7 +1333,7 @@ cert_status_t cert_net_set_profiling(cert_net_t *net, int on) {
     if (on && net->prof_events.empty()) {
         // one event per launch of the longest schedule, plus the opening one
         int K = net->n_layers;
-        int n = 4 + K + K * (K + 1) + 8;
+        int n = 4 + 2 * K + K * (K + 1) + 8;
         net->prof_events.resize(n);
         net->prof_class.assign(n, 0);
         for (int i = 0; i < n; ++i)
@@ -1299,6 +1373,7 @@ int cert_net_last_contraction_paths(const cert_net_t *net) { return net ? net->l
 
 cert_status_t cert_net_set_conv_patches(cert_net_t *net, int on) {
     if (!net) return CERT_ERR_INVALID_ARG;
+    if (on && !net->skip_from.empty()) return CERT_ERR_UNSUPPORTED;   // rows of such nets stay dense
     net->conv_patches = on != 0;
     return CERT_OK;
 }

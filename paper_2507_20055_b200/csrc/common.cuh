@@ -105,6 +105,11 @@ void launch_init_expr(const LayerDev &Lk, const LayerDev &Lbelow, int batch, flo
 void launch_relu_step(const LayerDev &Lj, int batch, int n_k, float *P, float *P_lo, float *d, int n_slots,
                       long long slot_stride, cudaStream_t st);
 
+// P [rows][ld] += the waiting coefficients of a residual connection (see ConvtEpilogue::add_hi): S_hi (+ S_lo),
+// or 1 at column (row mod n_k) when `identity`.
+void launch_add_skip(float *P, const float *S_hi, const float *S_lo, int identity, long long rows, int n, int ld,
+                     int n_k, cudaStream_t st);
+
 // map(simplify_lower/upper): rows of P [rows][ld0] against the box.
 void launch_concretize(const float *P, const float *d, int n_slots, long long slot_stride, const float *l0,
                        const float *u0, int n0, int ld0, int batch, int n_k, float *lb_out, float *ub_out, int n_total, int out_off,
@@ -131,6 +136,11 @@ struct ConvtEpilogue {
     const float *lamL, *lamU, *nuU;   // [batch][ld_in] relaxation of the ReLU below
     const float *bias_below;          // [ld_in]
     float *P, *P_lo;                  // result [rows][ld_in]; P_lo != nullptr: stored as a TF32 pair
+    // Residual connection ending on the neurons below: coefficients that waited for the traversal to reach
+    // them are added before the ReLU back-step: a matrix [rows][ld_in] (fp32, or a TF32 pair), or the unit
+    // coefficient of the row's own neuron (the layer being bounded has the connection itself).
+    const float *add_hi, *add_lo;
+    int add_identity;
     // CONVT_EPI_CONCRETIZE
     const float *l0, *u0;             // [batch][ld_in]
     float *lb_out, *ub_out;

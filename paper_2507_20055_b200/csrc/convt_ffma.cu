@@ -115,6 +115,18 @@ ConvtPlan make_plan(const LayerDev &L) {
     return p;
 }
 
+// Coefficient of a residual connection that ends on the neurons this step reaches (0 without one).
+__device__ __forceinline__ float skip_addend(const ConvtEpilogue &ep, long long r, int t, int ld_in) {
+    float s = 0.0f;
+    if (ep.add_hi) {
+        const size_t o = (size_t)r * ld_in + t;
+        s = ep.add_hi[o];
+        if (ep.add_lo) s += ep.add_lo[o];
+    }
+    if (ep.add_identity && t == (int)(r % ep.n_k)) s += 1.0f;
+    return s;
+}
+
 __device__ __forceinline__ float tf32_round(float x) {
     uint32_t r;
     asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(x));
@@ -315,7 +327,7 @@ convt_kernel(const float *__restrict__ Q, int ld_out, int ld_in, const float *__
                         for (int c = 0; c < CT; ++c) {
                             if (c0 + c >= g.c_in) continue;
                             const int t = (c0 + c) * hw_in + p_off[i];
-                            const float v = acc[i][c];
+                            const float v = acc[i][c] + (EPI == CONVT_EPI_RELU ? skip_addend(ep, r, t, ld_in) : 0.0f);
                             const bool nonneg = (v >= 0.0f);
                             if (EPI == CONVT_EPI_CONCRETIZE) {
                                 // lower rows: c >= 0 ? c*l : c*u; upper rows: c >= 0 ? c*u : c*l
@@ -384,6 +396,7 @@ convt_kernel(const float *__restrict__ Q, int ld_out, int ld_in, const float *__
 template <int EPI>
 __device__ __forceinline__ void finish_element(float v, int t, long long r, int upper, size_t vec, int ld_in,
                                                const ConvtEpilogue &ep, float &dacc) {
+    if (EPI == CONVT_EPI_RELU) v += skip_addend(ep, r, t, ld_in);
     const bool nonneg = (v >= 0.0f);
     if (EPI == CONVT_EPI_CONCRETIZE) {
         // lower rows: c >= 0 ? c*l : c*u; upper rows: c >= 0 ? c*u : c*l

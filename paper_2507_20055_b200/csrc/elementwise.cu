@@ -136,6 +136,21 @@ __global__ void first_layer_conv_kernel(const float *__restrict__ W, const float
     ub_out[(size_t)b * n_total + out_off + i] = hi + bb;
 }
 
+// Joins the waiting coefficients of a residual connection to the expression that has reached its source.
+__global__ void add_skip_kernel(float *__restrict__ P, const float *__restrict__ S_hi,
+                                const float *__restrict__ S_lo, int identity, long long total, int n, int ld,
+                                int n_k) {
+    const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= total) return;
+    const long long r = idx / ld;
+    const int t = (int)(idx - r * ld);
+    if (t >= n) return;
+    float s = 0.0f;
+    if (S_hi) s = S_hi[idx] + (S_lo ? S_lo[idx] : 0.0f);
+    if (identity && t == (int)(r % n_k)) s += 1.0f;
+    P[idx] += s;
+}
+
 // Sum of the slots that hold a row's constant (or bound), in slot order.
 __device__ __forceinline__ float slot_sum(const float *__restrict__ d, int n_slots, long long stride,
                                           long long r) {
@@ -472,6 +487,12 @@ void launch_relu_step(const LayerDev &Lj, int batch, int n_k, float *P, float *P
     relu_step_kernel<<<grid_for_warps(rows), kWarpsPerBlock * 32, 0, st>>>(
         P, P_lo, d, n_slots, slot_stride, rows, n_k, Lj.n_out, Lj.ld_out, Lj.relu_after, Lj.lamL,
         Lj.lamU, Lj.nuU, Lj.bias_n);
+}
+
+void launch_add_skip(float *P, const float *S_hi, const float *S_lo, int identity, long long rows, int n, int ld,
+                     int n_k, cudaStream_t st) {
+    const long long total = rows * (long long)ld;
+    add_skip_kernel<<<(unsigned)ceil_div_ll(total, 256), 256, 0, st>>>(P, S_hi, S_lo, identity, total, n, ld, n_k);
 }
 
 void launch_concretize(const float *P, const float *d, int n_slots, long long slot_stride, const float *l0,

@@ -238,6 +238,24 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_consta
                         const int col = col0 + g * 4;
                         float q[4];
                         const float4 bz = *reinterpret_cast<const float4 *>(a.bias_below + col);
+                        if (a.add_hi || a.add_identity) {
+                            // a residual connection ends on these neurons: its waiting coefficients join first
+                            float s4[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+                            if (a.add_hi) {
+                                const size_t o = (size_t)rr * a.ld_n + col;
+                                const float4 sh = *reinterpret_cast<const float4 *>(a.add_hi + o);
+                                s4[0] = sh.x; s4[1] = sh.y; s4[2] = sh.z; s4[3] = sh.w;
+                                if (a.add_lo) {
+                                    const float4 sl = *reinterpret_cast<const float4 *>(a.add_lo + o);
+                                    s4[0] += sl.x; s4[1] += sl.y; s4[2] += sl.z; s4[3] += sl.w;
+                                }
+                            }
+                            const int own = a.add_identity ? (int)(rr % a.n_k) : -1;
+#pragma unroll
+                            for (int e = 0; e < 4; ++e)
+                                v[g * 4 + e] = __float_as_uint(__uint_as_float(v[g * 4 + e]) + s4[e] +
+                                                               (col + e == own ? 1.0f : 0.0f));
+                        }
                         if (a.has_relu) {
                             const float4 ll = *reinterpret_cast<const float4 *>(a.lamL + relax_row + col);
                             const float4 lu = *reinterpret_cast<const float4 *>(a.lamU + relax_row + col);

@@ -38,6 +38,11 @@ struct TcArgs {
     int split_out;   // ReLU epilogue: store the result as a TF32 pair (a tensor-core step follows)
     const float *lamL, *lamU, *nuU;              // [batch (* n_pos)][ld_n]
     const float *bias_below;                     // [ld_n] bias of the affine layer below (next step)
+    // ReLU epilogue, residual connection ending on the neurons below layer j: coefficients added to the
+    // product before the ReLU back-step: a matrix [rows][ld_n] (fp32, or a TF32 pair), and / or the unit
+    // coefficient of the row's own neuron (column = row mod n_k)
+    const float *add_hi, *add_lo;
+    int add_identity;
     // concretisation epilogue
     const float *l0, *u0;                        // [batch (* n_pos)][ld_n]
     // Row constants travel in slots: the constant of row r so far is the sum over

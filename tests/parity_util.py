@@ -9,7 +9,7 @@ MARGIN_MIN = 1e-5     # boxes with a sign test closer to zero than this are ill-
 def run_gpu(w, contraction=None, max_batch=None, host_api=False, backsteps=None, conv_patches=None):
     import torch
     from paper_2507_20055_b200 import binding
-    net = binding.CertNet(w.layers, max_batch or w.batch, w.clip_lo, w.clip_hi)
+    net = binding.CertNet(w.layers, max_batch or w.batch, w.clip_lo, w.clip_hi, skip_from=getattr(w, "skip_from", None))
     try:
         if contraction is not None:
             net.set_contraction(contraction)

@@ -416,3 +416,57 @@ def test_fp16_split_is_refused_for_conv_nets_and_flags_its_range():
         assert net.last_status() == 0                                          # the flag is cleared by the read
     finally:
         net.destroy()
+
+
+# ---- residual connections (cert_net_create_residual) ----
+
+RES_NETS = {
+    "resfc_small": lambda: wl.residual_fc(20, 24, 2, 5, batch=3, eps=0.03, seed=21),
+    "resfc_ragged": lambda: wl.residual_fc(50, 70, 3, 7, batch=5, eps=0.02, seed=22),
+    "resfc_wide": lambda: wl.residual_fc(64, 300, 2, 10, batch=4, eps=0.01, seed=23),
+    "resconv": lambda: wl.residual_conv((2, 10, 8), 4, 2, 6, batch=3, eps=0.02, seed=24),
+    "resconv_wide": lambda: wl.residual_conv((3, 16, 16), 8, 1, 10, batch=2, eps=0.01, seed=25),
+}
+
+
+@pytest.mark.parametrize("mode", ["ffma", "tc"])
+@pytest.mark.parametrize("name", sorted(RES_NETS))
+def test_residual_nets(name, mode):
+    w = RES_NETS[name]()
+    ref = orc.deeppoly(w.layers, w.centers, w.eps, w.clip_lo, w.clip_hi, skip_from=w.skip_from)
+    g = run_gpu(w, contraction=MODES[mode], max_batch=w.batch + 1)
+    compare(g, ref, label=f"{name}/{mode}")
+    # the connections matter: the same layers without them give other bounds
+    plain = orc.deeppoly(w.layers, w.centers, w.eps, w.clip_lo, w.clip_hi)
+    assert np.abs(plain["lb"] - g["lb"]).max() > 1e-3
+
+
+@pytest.mark.parametrize("mode", ["ffma", "tc"])
+def test_residual_connection_into_the_output_layer_and_back_to_back_blocks(mode):
+    w = wl.small_fc([12, 16, 16, 16, 16, 16], batch=3, eps=0.04, seed=26)
+    w.skip_from = [-1, -1, 0, -1, 2]        # layer 2 adds layer 0's outputs; the output layer adds layer 2's
+    ref = orc.deeppoly(w.layers, w.centers, w.eps, w.clip_lo, w.clip_hi, skip_from=w.skip_from)
+    compare(run_gpu(w, contraction=MODES[mode]), ref, label=f"output_connection/{mode}")
+
+
+def test_residual_refusals():
+    import torch
+    from paper_2507_20055_b200 import binding
+    w = wl.residual_fc(10, 12, 1, 3, batch=2, eps=0.02, seed=27)
+    # not two layers back; widths differ; a connection that starts inside another's span
+    w5 = wl.small_fc([10, 12, 12, 12, 12, 3], batch=2, eps=0.02, seed=28)
+    for layers, bad in ((w.layers, [-1, 0, -1, -1]), (w.layers, [-1, -1, -1, 1]), (w5.layers, [-1, -1, -1, 0, 2])):
+        with pytest.raises(binding.CertError):
+            binding.CertNet(layers, 2, skip_from=bad)
+    net = binding.CertNet(w.layers, 2, skip_from=w.skip_from)
+    try:
+        assert binding.lib.cert_net_set_contraction(net._h, 3) == 2          # fp16 split: CERT_ERR_UNSUPPORTED
+        assert binding.lib.cert_net_set_conv_patches(net._h, 1) == 2
+        assert binding.lib.cert_net_enable_reusecert(net._h) == 2
+        c = torch.from_numpy(w.centers).cuda()
+        with pytest.raises(binding.CertError):
+            net.backsub_bounds(c, w.eps, [1] * len(w.layers))                  # a traversal that stops early
+        net.backsub_bounds(c, w.eps, [-1] * len(w.layers))                     # full traversals are fine
+        torch.cuda.synchronize()
+    finally:
+        net.destroy()
