@@ -107,7 +107,8 @@ def oracle_sample(w, n_boxes, threads=None, backsteps=None, certifier="deeppoly"
     if certifier == "reusecert":
         orc.reusecert(w.layers, c, w.eps, w.clip_lo, w.clip_hi, n_threads=cores)
     else:
-        orc.deeppoly(w.layers, c, w.eps, w.clip_lo, w.clip_hi, n_threads=cores, backsteps_per_layer=backsteps)
+        orc.deeppoly(w.layers, c, w.eps, w.clip_lo, w.clip_hi, n_threads=cores, backsteps_per_layer=backsteps,
+                     skip_from=w.skip_from)
     dt = time.perf_counter() - t0
     return {"value": n_boxes / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
             "sample": f"first {n_boxes} of {w.batch} boxes of {w.name}, one box per thread, {dt:.1f} s wall"}, dt
@@ -176,7 +177,7 @@ def run_reference(args, w):
     from oracle import deeppoly_oracle as orc
     orc.build()
     cores = orc.max_threads()
-    per = {0: 1, 1: 4 * cores, 2: 2 * cores, 3: cores, 4: cores}
+    per = {0: 1, 1: 4 * cores, 2: 2 * cores, 3: cores, 4: cores, 5: 2 * cores}
     n_boxes = min(w.batch, args.ref_boxes or per[args.config])
     if args.config == 4 and not args.ref_boxes:
         n_boxes = max(1, min(cores, 16) // 2)     # about 11 s per box per core
@@ -205,7 +206,9 @@ def main():
     ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--config", type=int, default=4, help="0..4: index into the benchmark configurations")
+    ap.add_argument("--config", type=int, default=4,
+                    help="0..4: index into the benchmark configurations; 5: a fully connected residual net in the "
+                         "shape of the paper's 'Skip' network (784 -> 512 x 5 -> 10, two blocks, 64 boxes)")
     ap.add_argument("--batch", type=int, default=None)
     ap.add_argument("--contraction", default="fastest", choices=["fastest", "auto", "ffma", "tc", "tc16"],
                     help="tc = tcgen05 3xTF32, tc16 = tcgen05 fp16 split (FC nets), ffma = FMA units, auto = the "
@@ -216,7 +219,10 @@ def main():
     ap.add_argument("--ref-boxes", type=int, default=None)
     args = ap.parse_args()
 
-    w = wl.make_config(args.config, batch=args.batch)
+    if args.config == 5:
+        w = wl.residual_fc(784, 512, 2, 10, batch=args.batch or 64, eps=0.01, seed=0)
+    else:
+        w = wl.make_config(args.config, batch=args.batch)
     args.backsteps = certifier_steps(args.certifier, len(w.layers))
     if args.impl == "reference":
         run_reference(args, w)
@@ -248,12 +254,12 @@ def main():
         w.centers = sharding.shard_centers(everything, rank, world)
         assert w.batch == per_gpu
     B = w.batch
-    net = binding.CertNet(w.layers, B, w.clip_lo, w.clip_hi)
+    net = binding.CertNet(w.layers, B, w.clip_lo, w.clip_hi, skip_from=w.skip_from)
     mode = {"auto": binding.CONTRACTION_AUTO, "ffma": binding.CONTRACTION_FFMA, "tc": binding.CONTRACTION_TC3XTF32,
             "tc16": binding.CONTRACTION_TC3XFP16}
     if args.contraction == "fastest":
         all_fc = all(l.kind == "fc" for l in w.layers)
-        args.contraction = "tc16" if (all_fc and len(w.layers) > 1) else "auto"
+        args.contraction = "tc16" if (all_fc and len(w.layers) > 1 and w.skip_from is None) else "auto"
     net.set_contraction(mode[args.contraction])
     stream = torch.cuda.Stream()
     centers = torch.from_numpy(w.centers).cuda()
@@ -430,7 +436,7 @@ def main():
         if tf32_ref is not None:
             out["tf32_split"] = tf32_ref
         if world == 1 and not args.no_cpu_baseline:
-            n_boxes = {0: 1, 1: 64, 2: 32, 3: 16, 4: 16}[args.config]
+            n_boxes = {0: 1, 1: 64, 2: 32, 3: 16, 4: 16, 5: 32}[args.config]
             from oracle import deeppoly_oracle as orc
             orc.build()
             n_boxes = min(n_boxes, B) if args.config != 4 else min(B, orc.max_threads(), 16)
