@@ -470,3 +470,61 @@ def test_residual_refusals():
         torch.cuda.synchronize()
     finally:
         net.destroy()
+
+
+# ---- seeded sweep over shapes: every kernel family against the oracle on nets nobody tuned for ----
+
+def _random_fc(seed):
+    rng = np.random.default_rng(1000 + seed)
+    depth = int(rng.integers(2, 7))
+    sizes = [int(rng.integers(3, 90))] + [int(rng.integers(2, 300)) for _ in range(depth)] + [int(rng.integers(1, 12))]
+    w = wl.small_fc(sizes, batch=int(rng.integers(1, 6)), eps=float(rng.uniform(0.005, 0.05)), seed=200 + seed)
+    if rng.random() < 0.3:
+        w.layers[int(rng.integers(0, len(w.layers) - 1))].relu_after = False
+    return w
+
+
+def _random_conv(seed):
+    rng = np.random.default_rng(2000 + seed)
+    shape = (int(rng.integers(1, 4)), int(rng.integers(8, 17)), int(rng.integers(8, 17)))
+    convs, h, wd = [], shape[1], shape[2]
+    for _ in range(int(rng.integers(1, 4))):
+        k, s = int(rng.integers(2, 5)), int(rng.integers(1, 3))
+        p = int(rng.integers(0, min(2, k - 1) + 1))
+        ho, wo = (h + 2 * p - k) // s + 1, (wd + 2 * p - k) // s + 1
+        if ho < 2 or wo < 2:
+            break
+        convs.append((int(rng.integers(2, 9)), k, s, p))
+        h, wd = ho, wo
+    fcs = [int(rng.integers(4, 24)) for _ in range(int(rng.integers(1, 3)))]
+    return wl.small_conv(shape, convs, fcs, batch=int(rng.integers(1, 4)), eps=float(rng.uniform(0.005, 0.03)),
+                         seed=300 + seed)
+
+
+def _well_conditioned(make, seed):
+    """The net of `seed`, or of seed + 100, + 200, ... if too few of its boxes have branch decisions that float32
+    can reproduce (the bump is printed: it is part of the test's record)."""
+    from parity_util import MARGIN_MIN
+    for bump in range(6):
+        w = make(seed + 100 * bump)
+        ref = _oracle(w)
+        good = ref["margins"].min(axis=1) >= MARGIN_MIN if ref["margins"].shape[1] else np.ones(w.batch, bool)
+        if good.mean() >= 0.5:
+            print(f"seed {seed}: bump {bump}")
+            return w, ref
+    raise AssertionError("no well-conditioned net found")
+
+
+@pytest.mark.parametrize("seed", range(10))
+def test_random_fc_shapes_all_contractions(seed):
+    w, ref = _well_conditioned(_random_fc, seed)
+    for mode, contraction in (("ffma", 1), ("tc", 2), ("tc16", TC16)):
+        compare(run_gpu(w, contraction=contraction, max_batch=w.batch + (seed % 3)), ref, min_good_fraction=0.5,
+                label=f"random_fc[{seed}]/{mode}")
+
+
+@pytest.mark.parametrize("seed", range(8))
+def test_random_conv_shapes(seed):
+    w, ref = _well_conditioned(_random_conv, seed)
+    for form, kw in (("auto", {}), ("dense", {"conv_patches": False}), ("ffma", {"contraction": 1})):
+        compare(run_gpu(w, **kw), ref, min_good_fraction=0.5, label=f"random_conv[{seed}]/{form}")
