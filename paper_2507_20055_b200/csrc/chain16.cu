@@ -13,10 +13,11 @@
 //   end:     the last step's epilogue is map(simplify_lower/upper) against the box (or the stored
 //            bounds of the layer reached); only the bounds leave the kernel.
 //
-// A row's constant lives in registers of its two owner threads (the two column halves) for the whole
-// traversal and leaves as two slots, summed by the next kernel: fixed order, no atomics.
+// A row's constant lives in registers of its owner threads (one per column group) for the whole
+// traversal and leaves as kChainColGroups slots, summed by the next kernel: fixed order, no atomics.
 // Warp roles: warp 0 = TMA producer of W_j tiles, warp 1 = MMA issuer (leader CTA) and TMEM owner,
-// warps 2..9 = epilogue (two per TMEM lane quarter, alternate 32-column chunks).
+// warps 2..17 = epilogue (kChainColGroups per TMEM lane quarter, each taking every kChainColGroups-th
+// 32-column chunk; a step's MMAs and its epilogue cannot overlap, so the epilogue is spread wide).
 #include <cuda.h>
 #include <cuda_fp16.h>
 
@@ -281,7 +282,7 @@ chain16_kernel(const __grid_constant__ ChainParams P, const ChainArgs a) {
         // ------------------------------------------------------------ epilogue (8 warps)
         const int ew = warp - 2;
         const int quarter = warp & 3;                       // TMEM lane quarter this warp may read
-        const int half_id = ew >> 2;                        // which of the quarter's warps: it takes every kChainColGroups-th 32-column chunk
+        const int col_group = ew >> 2;                        // which of the quarter's warps: it takes every kChainColGroups-th 32-column chunk
         const int prow = quarter * 32 + lane;               // this thread's row of the CTA's panel
         const uint32_t a_hi0 = smem_u32(A_hi), a_lo0 = smem_u32(A_lo);
         const uint32_t acc_empty_addr0 = map_to_cta(smem_u32(&bars->acc_empty[0]), 0);
@@ -295,7 +296,7 @@ chain16_kernel(const __grid_constant__ ChainParams P, const ChainArgs a) {
             const int b = (int)(rr / (2LL * a.n_k));
             const int upper = (int)((rr / a.n_k) & 1);
             const int i = (int)(rr % a.n_k);
-            float dacc = (half_id == 0) ? a.bias_k[i] : 0.0f;
+            float dacc = (col_group == 0) ? a.bias_k[i] : 0.0f;
             {
                 // start: row i of W_k through the ReLU of layer k-1; the constant takes the nu terms and Q.b
                 const ChainLayer &Lk = P.layer[a.k];
@@ -303,7 +304,7 @@ chain16_kernel(const __grid_constant__ ChainParams P, const ChainArgs a) {
                 const int kp = (n + BKH - 1) / BKH * BKH;
                 const size_t relax_row = (size_t)b * Lk.ld_in;
                 const float *wrow = a.Wk + (size_t)i * a.ldw_k;
-                for (int c0 = 32 * half_id; c0 < kp; c0 += 32 * kChainColGroups) {
+                for (int c0 = 32 * col_group; c0 < kp; c0 += 32 * kChainColGroups) {
                     float q[32];
                     if (c0 < Lk.ld_in && row_ok) {
 #pragma unroll
@@ -364,7 +365,7 @@ chain16_kernel(const __grid_constant__ ChainParams P, const ChainArgs a) {
                         // ReLU back-step through the neurons below layer j; the result is the next step's operand.
                         // (A step that is not the last has a single column tile: n_in <= 256.)
                         const int kp = (n_in + BKH - 1) / BKH * BKH;
-                        for (int c0 = 32 * half_id; c0 < kp; c0 += 32 * kChainColGroups) {
+                        for (int c0 = 32 * col_group; c0 < kp; c0 += 32 * kChainColGroups) {
                             float q[32];
                             if (c0 < ld_in) {
                                 uint32_t v[32];
@@ -412,7 +413,7 @@ chain16_kernel(const __grid_constant__ ChainParams P, const ChainArgs a) {
                         }
                     } else {
                         // map(simplify_lower/upper) against the concrete bounds of what the traversal reached
-                        for (int c0 = 32 * half_id; c0 < bn; c0 += 32 * kChainColGroups) {
+                        for (int c0 = 32 * col_group; c0 < bn; c0 += 32 * kChainColGroups) {
                             const int col0 = nt * bn + c0;
                             if (col0 >= ld_in) break;              // warp-uniform; ld_in is a multiple of 32
                             uint32_t v[32];
@@ -440,7 +441,7 @@ chain16_kernel(const __grid_constant__ ChainParams P, const ChainArgs a) {
                     }
                 }
             }
-            if (ok && row_ok) a.d_out[(size_t)half_id * a.slot_stride + r] = dacc;
+            if (ok && row_ok) a.d_out[(size_t)col_group * a.slot_stride + r] = dacc;
         }
         if (out_of_range) atomicOr(a.status, 2);
         if (!ok) {
