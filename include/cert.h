@@ -184,6 +184,16 @@ cert_status_t cert_net_branch_codes(cert_net_t *net, unsigned char *codes_out, v
 cert_status_t cert_net_last_status(cert_net_t *net, void *stream);
 
 /*
+ * Self-test of the bounded waits (no counterpart in the paper).  Every device-side wait of the tensor-core
+ * kernels (on an mbarrier a TMA copy, an MMA commit or another warp completes) gives up after about a second,
+ * raises the net's status word and lets the kernel end normally, so that a lost signal costs a result, not the
+ * context.  This call enqueues, on `stream`, one tiny kernel that runs the same wait with a limit of about
+ * 0.1 ms on a barrier nothing ever arrives on; afterwards cert_net_last_status returns CERT_ERR_TIMEOUT (and
+ * clears the flag), and the net works as before.  Nothing faults, traps or hangs.
+ */
+cert_status_t cert_net_selftest_bounded_wait(cert_net_t *net, void *stream);
+
+/*
  * Which kernel carries the affine back-step C' = C * W (Section 4.3, Matmul
  * rewrite).  AUTO picks the tensor-core path where the shape allows it.
  *   FFMA:    fp32 FMA units, unfused ReLU step and concretisation kernels.

@@ -30,7 +30,7 @@ EXPORTS = [
     "cert_backsub_bounds_host",
     "cert_net_destroy",
     "cert_net_num_neurons", "cert_net_num_relu_neurons", "cert_net_branch_codes",
-    "cert_net_last_status", "cert_net_set_contraction", "cert_net_last_launch_count",
+    "cert_net_last_status", "cert_net_selftest_bounded_wait", "cert_net_set_contraction", "cert_net_last_launch_count",
     "cert_net_backstep_flops", "cert_status_string", "cert_net_set_profiling", "cert_net_profile",
     "cert_net_last_contraction_paths", "cert_first_layer_bounds_noalloc", "cert_net_set_conv_patches",
     "cert_net_enable_reusecert", "cert_reusecert_bounds", "cert_reusecert_bounds_host",
@@ -68,6 +68,8 @@ _lib.cert_net_branch_codes.argtypes = [_vp, _vp, _vp]
 _lib.cert_net_branch_codes.restype = _i
 _lib.cert_net_last_status.argtypes = [_vp, _vp]
 _lib.cert_net_last_status.restype = _i
+_lib.cert_net_selftest_bounded_wait.argtypes = [_vp, _vp]
+_lib.cert_net_selftest_bounded_wait.restype = _i
 _lib.cert_net_set_contraction.argtypes = [_vp, _i]
 _lib.cert_net_set_contraction.restype = _i
 _lib.cert_net_last_launch_count.argtypes = [_vp]
@@ -269,6 +271,10 @@ class CertNet:
 
     def last_status(self, stream_ptr: int = 0) -> int:
         return int(_lib.cert_net_last_status(self._h, stream_ptr))
+
+    def selftest_bounded_wait(self, stream_ptr: int = 0):
+        """Enqueues a kernel whose (short) bounded wait runs out; last_status() then reports CERT_ERR_TIMEOUT."""
+        _check(_lib.cert_net_selftest_bounded_wait(self._h, stream_ptr), "cert_net_selftest_bounded_wait")
 
     def set_contraction(self, mode: int):
         _check(_lib.cert_net_set_contraction(self._h, int(mode)), "cert_net_set_contraction")

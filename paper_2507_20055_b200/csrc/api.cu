@@ -1328,6 +1328,16 @@ cert_status_t cert_net_set_contraction(cert_net_t *net, int mode) {
     return CERT_OK;
 }
 
+cert_status_t cert_net_selftest_bounded_wait(cert_net_t *net, void *stream) {
+    if (!net) return CERT_ERR_INVALID_ARG;
+    cert::launch_bounded_wait_selftest(net->status_dev, static_cast<cudaStream_t>(stream));
+    if (cudaPeekAtLastError() != cudaSuccess) {
+        cudaGetLastError();
+        return CERT_ERR_CUDA;
+    }
+    return CERT_OK;
+}
+
 cert_status_t cert_net_set_profiling(cert_net_t *net, int on) {
     if (!net) return CERT_ERR_INVALID_ARG;
     if (on && net->prof_events.empty()) {

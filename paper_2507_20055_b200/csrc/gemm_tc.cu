@@ -408,6 +408,18 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_consta
     }
 }
 
+// What every wait in the tensor-core kernels does when it runs out, on a barrier nothing arrives on: the wait
+// returns after `limit` cycles, the kernel raises the status word and ends normally.
+__global__ void bounded_wait_selftest_kernel(int *status, unsigned long long limit) {
+    __shared__ uint64_t bar;
+    if (threadIdx.x == 0) {
+        mbar_init(&bar, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    if (threadIdx.x == 0 && !mbar_wait_for(&bar, 0, limit)) atomicOr(status, 1);
+}
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *,
                                   CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
@@ -436,6 +448,10 @@ void launch_one(int groups, const CUtensorMap &ah, const CUtensorMap &al, const 
 }
 
 }  // namespace
+
+void launch_bounded_wait_selftest(int *status, cudaStream_t st) {
+    bounded_wait_selftest_kernel<<<1, 32, 0, st>>>(status, 200000ull);      // about 0.1 ms
+}
 
 bool tc_driver_init() {
     if (g_encode) return true;

@@ -64,6 +64,8 @@ struct TcArgs {
     int *status;                                 // set to 1 if a bounded wait runs out
 };
 
+// One block that waits, with a short limit, on a barrier nothing arrives on, and then raises bit 0 of *status.
+void launch_bounded_wait_selftest(int *status, cudaStream_t st);
 bool tc_driver_init();
 // Sets the kernels' shared-memory limits; *pair_ok tells whether the two-CTA form can be launched.
 bool tc_prepare_kernels(bool *pair_ok);

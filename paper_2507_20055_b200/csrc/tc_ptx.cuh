@@ -59,14 +59,17 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
         : "memory");
     return ok != 0;
 }
-// Bounded wait: gives up after kWaitCycles and reports false.
-__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity) {
+// Bounded wait: gives up after `limit` cycles and reports false.
+__device__ __forceinline__ bool mbar_wait_for(uint64_t *bar, uint32_t parity, unsigned long long limit) {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     while (!mbar_try_wait(bar, parity)) {
-        if ((unsigned long long)(clock64() - t0) > kWaitCycles) return false;
+        if ((unsigned long long)(clock64() - t0) > limit) return false;
     }
     return true;
+}
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity) {
+    return mbar_wait_for(bar, parity, kWaitCycles);
 }
 // TMA tile load into this CTA's shared memory; `bar_addr` is the cluster address of the barrier
 // that counts the bytes (for a CTA pair: the leader's barrier, for both CTAs' loads).

@@ -528,3 +528,26 @@ def test_random_conv_shapes(seed):
     w, ref = _well_conditioned(_random_conv, seed)
     for form, kw in (("auto", {}), ("dense", {"conv_patches": False}), ("ffma", {"contraction": 1})):
         compare(run_gpu(w, **kw), ref, min_good_fraction=0.5, label=f"random_conv[{seed}]/{form}")
+
+
+# ---- a bounded wait that runs out: status word, host mapping, and the net stays usable ----
+
+def test_bounded_wait_runs_out_and_the_net_stays_usable():
+    import torch
+    from paper_2507_20055_b200 import binding
+    w = wl.small_fc([16, 24, 24, 5], batch=2, eps=0.02, seed=91)
+    ref = _oracle(w)
+    net = binding.CertNet(w.layers, w.batch, w.clip_lo, w.clip_hi)
+    try:
+        assert net.last_status() == 0
+        net.selftest_bounded_wait()                  # waits about 0.1 ms on a barrier nothing arrives on
+        assert net.last_status() == 6                # CERT_ERR_TIMEOUT, read after the stream has drained
+        assert net.last_status() == 0                # the read cleared it
+        c = torch.from_numpy(w.centers).cuda()
+        lb, ub = net.deeppoly_bounds(c, w.eps)
+        torch.cuda.synchronize()
+        g = {"lb": lb.cpu().numpy(), "ub": ub.cpu().numpy(), "codes": net.branch_codes(w.batch).cpu().numpy(),
+             "status": net.last_status()}
+        compare(g, ref, label="after a timed-out wait")
+    finally:
+        net.destroy()
