@@ -551,3 +551,37 @@ def test_bounded_wait_runs_out_and_the_net_stays_usable():
         compare(g, ref, label="after a timed-out wait")
     finally:
         net.destroy()
+
+
+# ---- the call allocates nothing and synchronises nothing: it can be captured into a CUDA graph ----
+
+@pytest.mark.parametrize("mode", ["tc", "tc16"])
+def test_call_is_capturable_in_a_cuda_graph(mode):
+    import torch
+    from paper_2507_20055_b200 import binding
+    w = wl.make_config(1, batch=8)               # 784 -> 100 x 6 -> 10
+    ref = _oracle(w)
+    net = binding.CertNet(w.layers, w.batch, w.clip_lo, w.clip_hi)
+    try:
+        net.set_contraction({"tc": 2, "tc16": 3}[mode])
+        c = torch.from_numpy(w.centers).cuda()
+        lb = torch.zeros((w.batch, net.n_total), dtype=torch.float32, device="cuda")
+        ub = torch.zeros_like(lb)
+        s = torch.cuda.Stream()
+        with torch.cuda.stream(s):
+            net.deeppoly_bounds(c, w.eps, lb_out=lb, ub_out=ub, stream=s)      # warm-up outside the capture
+        s.synchronize()
+        lb.zero_(); ub.zero_()
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=s):
+            net.deeppoly_bounds(c, w.eps, lb_out=lb, ub_out=ub, stream=s)
+        assert float(lb.abs().max()) == 0.0      # capturing ran nothing
+        for _ in range(3):
+            graph.replay()
+        torch.cuda.synchronize()
+        g = {"lb": lb.cpu().numpy(), "ub": ub.cpu().numpy(), "codes": net.branch_codes(w.batch).cpu().numpy(),
+             "status": net.last_status()}
+        compare(g, ref, label=f"graph replay/{mode}")
+    finally:
+        net.destroy()
