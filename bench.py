@@ -259,7 +259,7 @@ def main():
             "tc16": binding.CONTRACTION_TC3XFP16}
     if args.contraction == "fastest":
         all_fc = all(l.kind == "fc" for l in w.layers)
-        args.contraction = "tc16" if (all_fc and len(w.layers) > 1 and w.skip_from is None) else "auto"
+        args.contraction = "tc16" if (all_fc and len(w.layers) > 1) else "auto"
     net.set_contraction(mode[args.contraction])
     stream = torch.cuda.Stream()
     centers = torch.from_numpy(w.centers).cuda()

@@ -81,8 +81,8 @@ cert_status_t cert_net_create(const cert_layer_desc_t *layers, int n_layers, int
  * Requirements (else CERT_ERR_INVALID_ARG): s <= k-2; layers s and k have the same number of neurons;
  * connections follow one another (none starts before the previous one has ended).
  * Such a net is bounded by full traversals only (cert_deeppoly_bounds; cert_backsub_bounds with depths
- * that stop early returns CERT_ERR_UNSUPPORTED), on the TF32 tensor-core and FMA kernels with dense
- * coefficient maps (CERT_CONTRACTION_TC3XFP16, patches and cert_net_enable_reusecert are refused).
+ * that stop early returns CERT_ERR_UNSUPPORTED), with one launch per back-step and dense coefficient maps
+ * (patches and cert_net_enable_reusecert are refused; CERT_CONTRACTION_TC3XFP16 is available for FC nets).
  */
 cert_status_t cert_net_create_residual(const cert_layer_desc_t *layers, int n_layers, const int *skip_from,
                                        int max_batch, float clip_lo, float clip_hi, cert_net_t **out);

@@ -21,7 +21,7 @@
 struct Tc16Layer {
     bool usable = false;
     __half *W_hi = nullptr, *W_lo = nullptr;     // W_j transposed, [round_up(n_in, 32)][ld_out]
-    cert::TcMap b_hi, b_lo, a_hi[2], a_lo[2], o_hi[2], o_lo[2];
+    cert::TcMap b_hi, b_lo, a_hi[3], a_lo[3], o_hi[3], o_lo[3];   // one per coefficient buffer
     cert::Tc16Plan plan;
 };
 
@@ -261,7 +261,7 @@ cert_status_t setup_tensor_core_path(cert_net *net, const cert_layer_desc_t *des
     net->tc_ok = true;
 
     // fp16-split operands: nets of FC layers, CTA pairs available
-    bool all_fc = net->skip_from.empty();      // (nets with residual connections stay on the TF32 / FMA kernels)
+    bool all_fc = true;
     for (int j = 0; j < K; ++j) all_fc = all_fc && net->layers[j].kind == CERT_LAYER_FC;
     net->tc16.assign(K, Tc16Layer());
     if (all_fc && ctas == 2 && cert::tc16_prepare_kernels()) {
@@ -293,7 +293,7 @@ cert_status_t setup_tensor_core_path(cert_net *net, const cert_layer_desc_t *des
                       cert::tc16_make_map(&T.b_lo, T.W_lo, L.n_out, L.n_in, L.ld_out, 64, T.plan.bn / 2);
             long long rows_max = 0;
             for (int k = j + 1; k < K; ++k) rows_max = std::max(rows_max, 2LL * net->max_batch * net->layers[k].n_out);
-            for (int p = 0; p < 2 && ok; ++p) {
+            for (int p = 0; p < net->n_buf && ok; ++p) {
                 const __half *bh = reinterpret_cast<const __half *>(net->buf[p]);
                 const __half *bl = reinterpret_cast<const __half *>(net->buf_lo[p]);
                 ok = cert::tc16_make_map(&T.a_hi[p], bh, L.n_out, rows_max, L.ld_out, 64, 128) &&
@@ -308,7 +308,7 @@ cert_status_t setup_tensor_core_path(cert_net *net, const cert_layer_desc_t *des
         }
         net->tc16_ok = all_ok;
         // The chain kernel: every layer a traversal passes through at most kChainMaxWidth neurons wide.
-        bool chain = all_ok && K <= cert::kChainMaxLayers && cert::chain16_prepare();
+        bool chain = all_ok && net->skip_from.empty() && K <= cert::kChainMaxLayers && cert::chain16_prepare();
         if (const char *e = std::getenv("CERT_CHAIN")) chain = chain && std::atoi(e) != 0;
         int widest = 0;
         for (int j = 0; j + 1 < K; ++j) widest = std::max(widest, net->layers[j].n_out);
@@ -713,13 +713,30 @@ cert_status_t cert_backsub_bounds(cert_net_t *net, const float *centers, float e
             continue;
         }
         if (net->contraction == CERT_CONTRACTION_TC3XFP16 && net->tc16_ok) {
-            __half *qh[2] = {reinterpret_cast<__half *>(net->buf[0]), reinterpret_cast<__half *>(net->buf[1])};
-            __half *ql[2] = {reinterpret_cast<__half *>(net->buf_lo[0]), reinterpret_cast<__half *>(net->buf_lo[1])};
+            __half *qh[3] = {reinterpret_cast<__half *>(net->buf[0]), reinterpret_cast<__half *>(net->buf[1]),
+                             reinterpret_cast<__half *>(net->buf[2])};
+            __half *ql[3] = {reinterpret_cast<__half *>(net->buf_lo[0]), reinterpret_cast<__half *>(net->buf_lo[1]),
+                             reinterpret_cast<__half *>(net->buf_lo[2])};
             cert::launch_init_expr16(Lk, net->layers[k - 1], batch, qh[cur], ql[cur], net->dbuf[dcur], net->status_dev, st);
             rec.mark(CERT_CLASS_RELU_STEP);
+            // residual connections as in the TF32 schedule below: the waiting matrix keeps its buffer
+            int wait_for = residual ? net->skip_from[k] : -1;
+            bool wait_identity = wait_for >= 0;
+            int kept = -1;
             for (int j = k - 1; j >= j_end; --j) {
                 const LayerDev &Lj = net->layers[j];
                 const Tc16Layer &T = net->tc16[j];
+                if (residual && net->skip_from[j] >= 0) {
+                    wait_for = net->skip_from[j];
+                    wait_identity = false;
+                    kept = cur;
+                }
+                int nxt = cur ^ 1;
+                if (residual) {
+                    nxt = 0;
+                    while (nxt == cur || nxt == kept) ++nxt;
+                }
+                const bool join = j > j_end && wait_for == j - 1;
                 cert::TcArgs a;
                 std::memset(&a, 0, sizeof(a));
                 a.M = rows; a.K = Lj.n_out; a.n_k = Lk.n_out; a.ld_n = Lj.ld_in;
@@ -734,15 +751,21 @@ cert_status_t cert_backsub_bounds(cert_net_t *net, const float *centers, float e
                     a.has_relu = Lb.relu_after;
                     a.split_out = 1;
                     a.lamL = Lb.lamL; a.lamU = Lb.lamU; a.nuU = Lb.nuU; a.bias_below = Lb.bias_n;
+                    if (join && kept >= 0) {
+                        a.add_hi = reinterpret_cast<const float *>(qh[kept]);
+                        a.add_lo = reinterpret_cast<const float *>(ql[kept]);
+                    }
+                    a.add_identity = (join && wait_identity) ? 1 : 0;
                     cert::launch_gemm_tc16(cert::TC_EPI_RELU, pairs, T.a_hi[cur], T.a_lo[cur], T.b_hi, T.b_lo,
-                                           T.o_hi[cur ^ 1], T.o_lo[cur ^ 1], a, T.plan.smem_bytes, st);
+                                           T.o_hi[nxt], T.o_lo[nxt], a, T.plan.smem_bytes, st);
+                    if (join) { wait_for = -1; wait_identity = false; kept = -1; }
                 } else {
                     a.l0 = box_l; a.u0 = box_u;
                     cert::launch_gemm_tc16(cert::TC_EPI_CONCRETIZE, pairs, T.a_hi[cur], T.a_lo[cur], T.b_hi, T.b_lo,
                                            T.a_hi[cur], T.a_lo[cur], a, T.plan.smem_bytes, st);
                 }
                 rec.mark(CERT_CLASS_AFFINE);
-                cur ^= 1;
+                cur = nxt;
                 dcur ^= 1;
                 dslots = 2 * T.plan.n_tiles;
             }

@@ -227,7 +227,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_consta
                 __syncwarp();
                 tmem_ld32(t_addr + (uint32_t)c0, v);
                 tmem_ld_wait();
-                if (EPI == TC_EPI_RELU) {
+                if (EPI == TC_EPI_RELU || EPI == TC_EPI_RELU_SKIP) {
                     // the slab is free again once the previous chunk's stores have read it
                     if (lane == 0) tma_store_wait_read();
                     __syncwarp();
@@ -238,7 +238,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_consta
                         const int col = col0 + g * 4;
                         float q[4];
                         const float4 bz = *reinterpret_cast<const float4 *>(a.bias_below + col);
-                        if (a.add_hi || a.add_identity) {
+                        if (EPI == TC_EPI_RELU_SKIP) {
                             // a residual connection ends on these neurons: its waiting coefficients join first
                             float s4[4] = {0.0f, 0.0f, 0.0f, 0.0f};
                             if (a.add_hi) {
@@ -467,14 +467,16 @@ bool tc_driver_init() {
 }
 
 bool tc_prepare_kernels(bool *pair_ok) {
-    cudaError_t e[6];
+    cudaError_t e[8];
+    e[6] = cudaFuncSetAttribute(gemm_tc_kernel<TC_EPI_RELU_SKIP, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemMax);
+    e[7] = cudaFuncSetAttribute(gemm_tc_kernel<TC_EPI_RELU_SKIP, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemMax);
     e[0] = cudaFuncSetAttribute(gemm_tc_kernel<TC_EPI_RELU, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemMax);
     e[1] = cudaFuncSetAttribute(gemm_tc_kernel<TC_EPI_CONCRETIZE, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemMax);
     e[2] = cudaFuncSetAttribute(gemm_tc_kernel<TC_EPI_RELU, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemMax);
     e[3] = cudaFuncSetAttribute(gemm_tc_kernel<TC_EPI_CONCRETIZE, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemMax);
     e[4] = cudaFuncSetAttribute(gemm_tc_kernel<TC_EPI_REUSE, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemMax);
     e[5] = cudaFuncSetAttribute(gemm_tc_kernel<TC_EPI_REUSE, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemMax);
-    for (int i = 0; i < 6; ++i)
+    for (int i = 0; i < 8; ++i)
         if (e[i] != cudaSuccess) {
             cudaGetLastError();
             return false;
@@ -540,6 +542,12 @@ void launch_gemm_tc(int epi, int ctas, int groups, const TcMap &a_hi, const TcMa
     const CUtensorMap &bl = reinterpret_cast<const CUtensorMap &>(b_lo);
     const CUtensorMap &oh = reinterpret_cast<const CUtensorMap &>(o_hi);
     const CUtensorMap &ol = reinterpret_cast<const CUtensorMap &>(o_lo);
+    const bool skip = args.add_hi || args.add_identity;
+    if (epi == TC_EPI_RELU && skip) {
+        if (ctas == 2) launch_one<TC_EPI_RELU_SKIP, 2>(groups, ah, al, bh, bl, oh, ol, args, smem_bytes, st);
+        else launch_one<TC_EPI_RELU_SKIP, 1>(groups, ah, al, bh, bl, oh, ol, args, smem_bytes, st);
+        return;
+    }
     if (ctas == 2) {
         if (epi == TC_EPI_RELU) launch_one<TC_EPI_RELU, 2>(groups, ah, al, bh, bl, oh, ol, args, smem_bytes, st);
         else if (epi == TC_EPI_REUSE) launch_one<TC_EPI_REUSE, 2>(groups, ah, al, bh, bl, oh, ol, args, smem_bytes, st);

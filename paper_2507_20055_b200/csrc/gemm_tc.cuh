@@ -7,7 +7,9 @@ namespace cert {
 
 constexpr int kTcSmemMax = 227 * 1024;
 
-enum { TC_EPI_RELU = 0, TC_EPI_CONCRETIZE = 1, TC_EPI_REUSE = 2 };
+// TC_EPI_RELU_SKIP: the ReLU epilogue with the waiting coefficients of a residual connection added first (a
+// variant of its own so that the common epilogue carries no code for it).
+enum { TC_EPI_RELU = 0, TC_EPI_CONCRETIZE = 1, TC_EPI_REUSE = 2, TC_EPI_RELU_SKIP = 3 };
 
 // Storage for a CUtensorMap (128 bytes, 64-byte aligned), kept opaque so that
 // only gemm_tc.cu needs the driver API header.
@@ -40,7 +42,8 @@ struct TcArgs {
     const float *bias_below;                     // [ld_n] bias of the affine layer below (next step)
     // ReLU epilogue, residual connection ending on the neurons below layer j: coefficients added to the
     // product before the ReLU back-step: a matrix [rows][ld_n] (fp32, or a TF32 pair), and / or the unit
-    // coefficient of the row's own neuron (column = row mod n_k)
+    // coefficient of the row's own neuron (column = row mod n_k).  (The fp16-split kernel reads the two
+    // pointers as the hi and lo halves of an fp16 pair; both are then set.)
     const float *add_hi, *add_lo;
     int add_identity;
     // concretisation epilogue

@@ -246,7 +246,7 @@ gemm_tc16_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_cons
                 __syncwarp();
                 tmem_ld32(t_addr + (uint32_t)c0, v);
                 tmem_ld_wait();
-                if (EPI == TC_EPI_RELU) {
+                if (EPI == TC_EPI_RELU || EPI == TC_EPI_RELU_SKIP) {
                     // the slab is free again once the previous chunk's stores have read it
                     if (lane == 0) tma_store_wait_read();
                     __syncwarp();
@@ -261,6 +261,28 @@ gemm_tc16_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_cons
                             const int col = col0 + g * 4;
                             float q[4];
                             const float4 bz = *reinterpret_cast<const float4 *>(a.bias_below + col);
+                            if (EPI == TC_EPI_RELU_SKIP) {
+                                // a residual connection ends on these neurons: its waiting coefficients (an fp16
+                                // pair here) join before the ReLU back-step
+                                float s4[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+                                if (a.add_hi) {
+                                    const size_t o = (size_t)rr * a.ld_n + col;
+                                    const uint2 sh = *reinterpret_cast<const uint2 *>(reinterpret_cast<const __half *>(a.add_hi) + o);
+                                    const uint2 sl = *reinterpret_cast<const uint2 *>(reinterpret_cast<const __half *>(a.add_lo) + o);
+                                    const __half2 h01 = *reinterpret_cast<const __half2 *>(&sh.x), h23 = *reinterpret_cast<const __half2 *>(&sh.y);
+                                    const __half2 l01 = *reinterpret_cast<const __half2 *>(&sl.x), l23 = *reinterpret_cast<const __half2 *>(&sl.y);
+                                    const float2 fh01 = __half22float2(h01), fh23 = __half22float2(h23);
+                                    const float2 fl01 = __half22float2(l01), fl23 = __half22float2(l23);
+                                    const float inv = 1.0f / kLoScale;
+                                    s4[0] = fmaf(fl01.x, inv, fh01.x); s4[1] = fmaf(fl01.y, inv, fh01.y);
+                                    s4[2] = fmaf(fl23.x, inv, fh23.x); s4[3] = fmaf(fl23.y, inv, fh23.y);
+                                }
+                                const int own = a.add_identity ? (int)(rr % a.n_k) : -1;
+#pragma unroll
+                                for (int e = 0; e < 4; ++e)
+                                    v[g * 4 + e] = __float_as_uint(__uint_as_float(v[g * 4 + e]) + s4[e] +
+                                                                   (col + e == own ? 1.0f : 0.0f));
+                            }
                             if (a.has_relu) {
                                 const float4 ll = *reinterpret_cast<const float4 *>(a.lamL + relax_row + col);
                                 const float4 lu = *reinterpret_cast<const float4 *>(a.lamU + relax_row + col);
@@ -546,7 +568,9 @@ bool tc16_prepare_kernels() {
         }
         g_encode16 = reinterpret_cast<EncodeTiledFn16>(fn);
     }
-    if (cudaFuncSetAttribute(gemm_tc16_kernel<TC_EPI_RELU>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemMax) !=
+    if (cudaFuncSetAttribute(gemm_tc16_kernel<TC_EPI_RELU_SKIP>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemMax) !=
+            cudaSuccess ||
+        cudaFuncSetAttribute(gemm_tc16_kernel<TC_EPI_RELU>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemMax) !=
             cudaSuccess ||
         cudaFuncSetAttribute(gemm_tc16_kernel<TC_EPI_REUSE>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemMax) !=
             cudaSuccess ||
@@ -596,7 +620,9 @@ void launch_gemm_tc16(int epi, int pairs, const TcMap &a_hi, const TcMap &a_lo, 
     const CUtensorMap &bl = reinterpret_cast<const CUtensorMap &>(b_lo);
     const CUtensorMap &oh = reinterpret_cast<const CUtensorMap &>(o_hi);
     const CUtensorMap &ol = reinterpret_cast<const CUtensorMap &>(o_lo);
-    if (epi == TC_EPI_RELU) launch_one16<TC_EPI_RELU>(pairs, ah, al, bh, bl, oh, ol, args, smem_bytes, st);
+    const bool skip = args.add_hi || args.add_identity;
+    if (epi == TC_EPI_RELU && skip) launch_one16<TC_EPI_RELU_SKIP>(pairs, ah, al, bh, bl, oh, ol, args, smem_bytes, st);
+    else if (epi == TC_EPI_RELU) launch_one16<TC_EPI_RELU>(pairs, ah, al, bh, bl, oh, ol, args, smem_bytes, st);
     else if (epi == TC_EPI_REUSE) launch_one16<TC_EPI_REUSE>(pairs, ah, al, bh, bl, oh, ol, args, smem_bytes, st);
     else launch_one16<TC_EPI_CONCRETIZE>(pairs, ah, al, bh, bl, oh, ol, args, smem_bytes, st);
 }

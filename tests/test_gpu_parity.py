@@ -429,24 +429,28 @@ RES_NETS = {
 }
 
 
-@pytest.mark.parametrize("mode", ["ffma", "tc"])
+@pytest.mark.parametrize("mode", ["ffma", "tc", "tc16"])
 @pytest.mark.parametrize("name", sorted(RES_NETS))
 def test_residual_nets(name, mode):
     w = RES_NETS[name]()
+    if mode == "tc16" and any(l.kind != "fc" for l in w.layers):
+        pytest.skip("the fp16 split covers FC nets")
     ref = orc.deeppoly(w.layers, w.centers, w.eps, w.clip_lo, w.clip_hi, skip_from=w.skip_from)
-    g = run_gpu(w, contraction=MODES[mode], max_batch=w.batch + 1)
+    g = run_gpu(w, contraction={"ffma": 1, "tc": 2, "tc16": 3}[mode], max_batch=w.batch + 1)
+    if mode == "tc16":
+        assert g["paths"] & 16 and not g["paths"] & 32      # one launch per back-step, not the chain kernel
     compare(g, ref, label=f"{name}/{mode}")
     # the connections matter: the same layers without them give other bounds
     plain = orc.deeppoly(w.layers, w.centers, w.eps, w.clip_lo, w.clip_hi)
     assert np.abs(plain["lb"] - g["lb"]).max() > 1e-3
 
 
-@pytest.mark.parametrize("mode", ["ffma", "tc"])
+@pytest.mark.parametrize("mode", ["ffma", "tc", "tc16"])
 def test_residual_connection_into_the_output_layer_and_back_to_back_blocks(mode):
     w = wl.small_fc([12, 16, 16, 16, 16, 16], batch=3, eps=0.04, seed=26)
     w.skip_from = [-1, -1, 0, -1, 2]        # layer 2 adds layer 0's outputs; the output layer adds layer 2's
     ref = orc.deeppoly(w.layers, w.centers, w.eps, w.clip_lo, w.clip_hi, skip_from=w.skip_from)
-    compare(run_gpu(w, contraction=MODES[mode]), ref, label=f"output_connection/{mode}")
+    compare(run_gpu(w, contraction={"ffma": 1, "tc": 2, "tc16": 3}[mode]), ref, label=f"output_connection/{mode}")
 
 
 def test_residual_refusals():
@@ -460,8 +464,7 @@ def test_residual_refusals():
             binding.CertNet(layers, 2, skip_from=bad)
     net = binding.CertNet(w.layers, 2, skip_from=w.skip_from)
     try:
-        assert binding.lib.cert_net_set_contraction(net._h, 3) == 2          # fp16 split: CERT_ERR_UNSUPPORTED
-        assert binding.lib.cert_net_set_conv_patches(net._h, 1) == 2
+        assert binding.lib.cert_net_set_conv_patches(net._h, 1) == 2          # CERT_ERR_UNSUPPORTED
         assert binding.lib.cert_net_enable_reusecert(net._h) == 2
         c = torch.from_numpy(w.centers).cuda()
         with pytest.raises(binding.CertError):
