@@ -363,6 +363,23 @@ def test_fp16_split_contraction(name, chain, monkeypatch):
     compare(g, _oracle(w), label=f"{name}/tc16/chain={chain}")
 
 
+def test_fp16_split_chain_wide_input_and_many_layers():
+    """A CIFAR-sized input (14 column tiles in the concretising step) and the deepest net the chain kernel's
+    parameter block takes (12 layers); one layer more goes back to one launch per back-step."""
+    w = wl.small_fc([3072, 100, 100, 100, 10], batch=3, eps=0.004, seed=92)
+    g = run_gpu(w, contraction=TC16)
+    assert g["paths"] & 32
+    compare(g, _oracle(w), label="cifar_input/tc16 chain")
+    w = wl.small_fc([30] + [40] * 11 + [5], batch=2, eps=0.002, seed=93)          # 12 affine layers
+    g = run_gpu(w, contraction=TC16)
+    assert g["paths"] & 32
+    compare(g, _oracle(w), min_good_fraction=0.4, label="12 layers/tc16 chain")
+    w = wl.small_fc([30] + [40] * 12 + [5], batch=2, eps=0.002, seed=94)          # 13 affine layers
+    g = run_gpu(w, contraction=TC16)
+    assert g["paths"] & 16 and not g["paths"] & 32
+    compare(g, _oracle(w), min_good_fraction=0.4, label="13 layers/tc16 per step")
+
+
 def test_fp16_split_chain_bounded_traversals_ragged_batch_and_missing_relu():
     w = VARIANT_NETS["fc_ragged"]()
     for vname, steps in _variant_steps(len(w.layers)).items():
