@@ -67,11 +67,10 @@ def deeppoly_matrix(layers, centers, eps, clip_lo=0.0, clip_hi=1.0, decision_fp3
     input).  A traversal that stops early is simplified against the concrete bounds of the
     neurons it reached (Section 6.2, DeepPoly_p; 0 everywhere is the IBP listing, 0 except at
     the last layer the CROWN-IBP listing of Appendix C).
-    skip_from: optional residual connections (layer k adds the outputs of layer skip_from[k]; full
-    traversals only): the coefficient matrix on those outputs is set aside and joins the expression
-    when the traversal, highest layer first, has come down to that layer."""
-    if skip_from is not None:
-        assert backsteps is None
+    skip_from: optional residual connections (layer k adds the outputs of layer skip_from[k]): the
+    coefficient matrix on those outputs is set aside and joins the expression when the traversal, highest
+    layer first, has come down to that layer; if the traversal stops before, it is simplified against
+    that layer's concrete bounds."""
     A = [dense_matrix(l) for l in layers]
     bias = [dense_bias(l) for l in layers]
     L0, U0 = box(centers, eps, clip_lo, clip_hi)
@@ -113,9 +112,15 @@ def deeppoly_matrix(layers, centers, eps, clip_lo=0.0, clip_hi=1.0, decision_fp3
                 du = du + Cu @ bias[j]
                 Cl = Cl @ A[j]
                 Cu = Cu @ A[j]
+            if stop_at >= 0 and stop_at in waiting:
+                Wl, Wu = waiting.pop(stop_at)
+                Cl, Cu = Cl + Wl, Cu + Wu
             lo_in, up_in = (l0, u0) if stop_at < 0 else (act_l[stop_at], act_u[stop_at])
             lb = np.clip(Cl, 0.0, None) @ lo_in + np.clip(Cl, None, 0.0) @ up_in + dl
             ub = np.clip(Cu, 0.0, None) @ up_in + np.clip(Cu, None, 0.0) @ lo_in + du
+            for t2, (Wl, Wu) in waiting.items():      # neurons of lower layers still in the expression
+                lb = lb + np.clip(Wl, 0.0, None) @ act_l[t2] + np.clip(Wl, None, 0.0) @ act_u[t2]
+                ub = ub + np.clip(Wu, 0.0, None) @ act_u[t2] + np.clip(Wu, None, 0.0) @ act_l[t2]
             n_k = lb.shape[0]
             if layer.relu_after:
                 act_l.append(np.maximum(lb, 0.0)); act_u.append(np.maximum(ub, 0.0))

@@ -318,17 +318,34 @@ static int one_box(const oracle_layer_t *layers, int n_layers, const float *cent
                 } else {
                     /* Stopped early (DeepPoly_p, Section 6.2): simplify against the
                      * concrete bounds of the neurons reached: relu(l), relu(u) of
-                     * layer j when a ReLU follows it, else its own l, u. */
-                    int n_j = layer_n_out(&layers[j]);
-                    double *lj = next, *uj = malloc(sizeof(double) * n_j);
-                    if (!uj) return 1;
-                    for (int t = 0; t < n_j; ++t) {
-                        double l = lb[off[j] + t], u = ub[off[j] + t];
-                        if (layers[j].relu_after) { l = l >= 0.0 ? l : 0.0; u = u >= 0.0 ? u : 0.0; }
-                        lj[t] = l; uj[t] = u;
+                     * layer j when a ReLU follows it, else its own l, u.  With residual
+                     * connections the expression may also hold neurons of lower layers
+                     * (coefficients that were still waiting): map(simplify_*) treats every
+                     * neuron of the expression alike, each with its total coefficient. */
+                    v = d;
+                    for (int t2 = j; t2 >= 0; --t2) {
+                        if (t2 < j && !has[t2]) continue;
+                        int n_t = layer_n_out(&layers[t2]);
+                        double *lt = next, *ut = malloc(sizeof(double) * n_t);
+                        if (!ut) return 1;
+                        for (int t = 0; t < n_t; ++t) {
+                            double l = lb[off[t2] + t], u = ub[off[t2] + t];
+                            if (layers[t2].relu_after) { l = l >= 0.0 ? l : 0.0; u = u >= 0.0 ? u : 0.0; }
+                            lt[t] = l; ut[t] = u;
+                        }
+                        if (t2 == j) {
+                            if (has[j]) {
+                                for (int t = 0; t < n_t; ++t) { coef[t] += pend[off[j] + t]; pend[off[j] + t] = 0.0; }
+                                has[j] = 0;
+                            }
+                            v += concretize(n_t, upper, coef, 0.0, lt, ut);
+                        } else {
+                            v += concretize(n_t, upper, pend + off[t2], 0.0, lt, ut);
+                            for (int t = 0; t < n_t; ++t) pend[off[t2] + t] = 0.0;
+                            has[t2] = 0;
+                        }
+                        free(ut);
                     }
-                    v = concretize(n_j, upper, coef, d, lj, uj);
-                    free(uj);
                 }
                 if (upper) ub[off[k] + i] = v; else lb[off[k] + i] = v;
             }
@@ -380,6 +397,8 @@ int oracle_num_relu_neurons(const oracle_layer_t *layers, int n_layers)
  * with the Relu transformer (relu(l), relu(u), relu_n, compute_upper) unchanged.
  * skip_form != 0: the SkipPoly listing (ReLU shapes expressed two layers back; one traversal
  * round per ReLU layer).
+ * (A traversal that stops early with such a connection still open simplifies the waiting coefficients
+ * against the concrete bounds of their own layer, like every other neuron left in the expression.)
  * skip_from (optional, [n_layers]): residual connections.  skip_from[k] = s >= 0 (s <= k-2, equal widths)
  * makes layer k compute W_k a_{k-1} + b_k + a_s with a_s the outputs of layer s (after its ReLU, if it
  * has one); -1 = none.  Reading: such a neuron is the listing's Affine neuron whose prev holds neurons
@@ -398,8 +417,8 @@ int oracle_backsub(const oracle_layer_t *layers, int n_layers, const float *cent
     for (int k = 1; k < n_layers; ++k)
         if (layer_n_in(&layers[k]) != layer_n_out(&layers[k - 1])) return 2;
     if (skip_from) {
-        /* residual connections: full traversals of the DeepPoly listing only */
-        if (skip_form || backsteps_per_layer || max_backsteps >= 0) return 2;
+        /* residual connections: not in the SkipPoly form */
+        if (skip_form) return 2;
         for (int k = 0; k < n_layers; ++k) {
             int sfrom = skip_from[k];
             if (sfrom < 0) continue;

@@ -85,7 +85,7 @@ def deeppoly(layers, centers, eps, clip_lo=0.0, clip_hi=1.0, decision_fp32=True,
     max_backsteps = p >= 0 is DeepPoly_p; backsteps_per_layer (one count per affine layer,
     negative = traverse to the input) overrides it.  skip_form: the SkipPoly listing (ReLU shapes
     expressed over the neurons two layers back).  skip_from (one entry per affine layer, -1 = none): residual
-    connections, layer k adds the outputs of layer skip_from[k] to its affine result (full traversals only).
+    connections, layer k adds the outputs of layer skip_from[k] to its affine result.
     Returns dict(lb, ub: float64 [batch, n_total]; codes: uint8 [batch, n_relu];
     margins: float64 [batch, n_relu]).  Layers are concatenated in order.
     """

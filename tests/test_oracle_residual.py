@@ -132,4 +132,70 @@ def test_malformed_connections_are_refused():
     with pytest.raises(RuntimeError):
         orc.deeppoly(w.layers, w.centers, w.eps, skip_from=[-1, -1, -1, 1])        # widths differ
     with pytest.raises(RuntimeError):
-        orc.deeppoly(w.layers, w.centers, w.eps, skip_from=w.skip_from, max_backsteps=1)
+        orc.deeppoly(w.layers, w.centers, w.eps, skip_from=w.skip_from, skip_form=True)
+
+
+# ---- traversals that stop early (DeepPoly_p, IBP, CROWN-IBP) with a connection still open ----
+
+def test_hand_worked_example_early_stops():
+    g = json.load(open(os.path.join(GOLD, "residual_example.json")))
+    layers = [wl.Layer("fc", np.array(l["weight"], np.float32), np.array(l["bias"], np.float32),
+                       relu_after=l["relu_after"]) for l in g["layers"]]
+    c = np.array([g["center"]], np.float32)
+    runs = {"ibp": dict(backsteps_per_layer=[0, 0, 0]), "deeppoly_p1": dict(max_backsteps=1)}
+    for name, kw in runs.items():
+        v = g["variants"][name]
+        r = orc.deeppoly(layers, c, g["eps"], *g["clip"], skip_from=g["skip_from"], **kw)
+        np.testing.assert_allclose(r["lb"][0], v["lb"], rtol=0, atol=1e-15, err_msg=name)
+        np.testing.assert_allclose(r["ub"][0], v["ub"], rtol=0, atol=1e-15, err_msg=name)
+        assert r["codes"][0].tolist() == v["codes"], name
+        steps = kw.get("backsteps_per_layer", [1, 1, 1])
+        lb, ub, _ = mat.deeppoly_matrix(layers, c, g["eps"], *g["clip"], skip_from=g["skip_from"], backsteps=steps)
+        np.testing.assert_allclose(lb[0], v["lb"], rtol=0, atol=1e-15, err_msg=name)
+        np.testing.assert_allclose(ub[0], v["ub"], rtol=0, atol=1e-15, err_msg=name)
+
+
+def test_ibp_is_interval_arithmetic_with_the_connections():
+    w = wl.residual_fc(7, 9, 2, 3, batch=3, eps=0.05, seed=31)
+    r = orc.ibp(w.layers, w.centers, w.eps, w.clip_lo, w.clip_hi, skip_from=w.skip_from)
+    l, u = mat.box(w.centers, w.eps, w.clip_lo, w.clip_hi)
+    acts, off = [], 0
+    for k, layer in enumerate(w.layers):
+        W, b = layer.weight.astype(np.float64), layer.bias.astype(np.float64)
+        lo = l @ np.clip(W, 0, None).T + u @ np.clip(W, None, 0).T + b
+        up = u @ np.clip(W, 0, None).T + l @ np.clip(W, None, 0).T + b
+        if w.skip_from[k] >= 0:
+            lo, up = lo + acts[w.skip_from[k]][0], up + acts[w.skip_from[k]][1]
+        n = W.shape[0]
+        np.testing.assert_allclose(r["lb"][:, off:off + n], lo, rtol=0, atol=1e-12)
+        np.testing.assert_allclose(r["ub"][:, off:off + n], up, rtol=0, atol=1e-12)
+        off += n
+        l, u = (np.maximum(lo, 0), np.maximum(up, 0)) if layer.relu_after else (lo, up)
+        acts.append((l, u))
+
+
+@pytest.mark.parametrize("kind", ["fc", "conv"])
+def test_early_stops_sound_and_agree_with_the_layer_level_form(kind):
+    w = wl.residual_fc(8, 12, 2, 4, batch=3, eps=0.05, seed=32) if kind == "fc" else \
+        wl.residual_conv((2, 6, 6), 3, 2, 4, batch=2, eps=0.03, seed=33)
+    K = len(w.layers)
+    l0, u0 = mat.box(w.centers, w.eps, w.clip_lo, w.clip_hi)
+    rng = np.random.default_rng(6)
+    full = orc.deeppoly(w.layers, w.centers, w.eps, w.clip_lo, w.clip_hi, skip_from=w.skip_from)
+    for name, steps in {"ibp": [0] * K, "crown_ibp": [0] * (K - 1) + [-1], "p1": [1] * K, "p2": [2] * K,
+                        "p3": [3] * K, "mixed": [(-1 if k % 2 else 1) for k in range(K)]}.items():
+        r = orc.deeppoly(w.layers, w.centers, w.eps, w.clip_lo, w.clip_hi, skip_from=w.skip_from,
+                         backsteps_per_layer=steps)
+        lb, ub, codes = mat.deeppoly_matrix(w.layers, w.centers, w.eps, w.clip_lo, w.clip_hi, skip_from=w.skip_from,
+                                            backsteps=steps)
+        np.testing.assert_allclose(r["lb"], lb, rtol=0, atol=1e-10, err_msg=name)
+        np.testing.assert_allclose(r["ub"], ub, rtol=0, atol=1e-10, err_msg=name)
+        for b in range(w.batch):
+            uu = rng.random((2000, l0.shape[1]))
+            uu[1000:] = (uu[1000:] > 0.5)
+            z = _forward(w, l0[b] + uu * (u0[b] - l0[b]))
+            tol = 1e-9 * (1 + np.abs(z))
+            assert (z >= r["lb"][b] - tol).all() and (z <= r["ub"][b] + tol).all(), name
+    # as many steps as there are layers is the full traversal
+    r = orc.deeppoly(w.layers, w.centers, w.eps, w.clip_lo, w.clip_hi, skip_from=w.skip_from, max_backsteps=K)
+    np.testing.assert_allclose(r["lb"], full["lb"], rtol=0, atol=1e-13)
