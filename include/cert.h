@@ -80,9 +80,12 @@ cert_status_t cert_net_create(const cert_layer_desc_t *layers, int n_layers, int
  * epilogue of the step that reaches layer s, before the ReLU back-step.
  * Requirements (else CERT_ERR_INVALID_ARG): s <= k-2; layers s and k have the same number of neurons;
  * connections follow one another (none starts before the previous one has ended).
- * Such a net is bounded by full traversals only (cert_deeppoly_bounds; cert_backsub_bounds with depths
- * that stop early returns CERT_ERR_UNSUPPORTED), with one launch per back-step and dense coefficient maps
- * (patches and cert_net_enable_reusecert are refused; CERT_CONTRACTION_TC3XFP16 is available for FC nets).
+ * Such a net is bounded with one launch per back-step and dense coefficient maps (patches and
+ * cert_net_enable_reusecert are refused).  cert_backsub_bounds works as for other nets: a traversal that
+ * stops on a connection's source joins the waiting coefficients before it is simplified, one that stops
+ * above it simplifies them against the source's own concrete bounds (map(simplify_*) treats every neuron left
+ * in the expression alike).  CERT_CONTRACTION_TC3XFP16 is available for FC nets, for full traversals only
+ * (depths that stop early return CERT_ERR_UNSUPPORTED in that mode).
  */
 cert_status_t cert_net_create_residual(const cert_layer_desc_t *layers, int n_layers, const int *skip_from,
                                        int max_batch, float clip_lo, float clip_hi, cert_net_t **out);

@@ -85,6 +85,7 @@ struct cert_net {
     // connections a third, so that the matrix a connection sets aside stays put while the traversal goes on
     float *buf[3] = {nullptr, nullptr, nullptr};
     float *buf_lo[3] = {nullptr, nullptr, nullptr};   // TF32 lo parts for the tensor-core contraction
+    float *zeros = nullptr;                  // [widest layer, padded] zeros (nets with residual connections)
     std::vector<int> skip_from;              // residual connections: layer k adds the outputs of layer skip_from[k] (-1: none); empty: none at all
     int n_buf = 2;
     bool tc_ok = false;                      // tensor-core path usable on this net
@@ -616,6 +617,13 @@ cert_status_t cert_net_create_residual(const cert_layer_desc_t *layers, int n_la
         net->slot_stride = (long long)max_rows;
         if (ok) fail = setup_tensor_core_path(net, layers, max_elems);
         if (ok && fail == CERT_OK) fail = setup_patch_tc(net, layers);
+        if (ok && fail == CERT_OK && !net->skip_from.empty()) {
+            // a traversal that stops early may leave one more partial bound per row (the waiting coefficients)
+            net->d_slots += 1;
+            int ld_max = net->ld0;
+            for (const LayerDev &L : net->layers) ld_max = std::max(ld_max, L.ld_out);
+            if (!dev_alloc_zero(net, &net->zeros, (size_t)ld_max)) fail = CERT_ERR_OOM;
+        }
         if (fail == CERT_OK &&
             (!dev_alloc_zero(net, &net->dbuf[0], (size_t)net->d_slots * max_rows) ||
              !dev_alloc_zero(net, &net->dbuf[1], (size_t)net->d_slots * max_rows)))
@@ -649,9 +657,9 @@ cert_status_t cert_backsub_bounds(cert_net_t *net, const float *centers, float e
     const int K = net->n_layers;
     const int n_total = net->n_total;
     const bool residual = !net->skip_from.empty();
-    if (residual && backsteps)
+    if (residual && backsteps && net->contraction == CERT_CONTRACTION_TC3XFP16)
         for (int k = 1; k < K; ++k)
-            if (backsteps[k] >= 0 && backsteps[k] < k) return CERT_ERR_UNSUPPORTED;   // full traversals only
+            if (backsteps[k] >= 0 && backsteps[k] < k) return CERT_ERR_UNSUPPORTED;   // fp16 split: full traversals only
     Recorder rec(net, st);
     int paths = 0;
 
@@ -676,6 +684,10 @@ cert_status_t cert_backsub_bounds(cert_net_t *net, const float *centers, float e
             const LayerDev &Lb = net->layers[k - 1];
             cert::launch_first_layer_bounds(Lk, Lb.actL, Lb.actU, Lb.ld_out, batch, lb_out, ub_out, n_total, st);
             rec.mark(CERT_CLASS_CONCRETIZE);
+            if (residual && net->skip_from[k] >= 0) {
+                cert::launch_add_act_bounds(Lk, net->layers[net->skip_from[k]], batch, lb_out, ub_out, n_total, st);
+                rec.mark(CERT_CLASS_CONCRETIZE);
+            }
             if (Lk.relu_after || k + 1 < K) {
                 cert::launch_relax(Lk, lb_out, ub_out, n_total, batch, net->codes, net->n_relu, nullptr, 0, 0, st);
                 rec.mark(CERT_CLASS_RELAX);
@@ -892,7 +904,12 @@ cert_status_t cert_backsub_bounds(cert_net_t *net, const float *centers, float e
                 nxt = 0;
                 while (nxt == cur || nxt == kept) ++nxt;
             }
-            const bool join = j > j_end && wait_for == j - 1;
+            // The last step of a traversal that stops on the very neurons a connection waits for: the
+            // coefficients join before the simplification, so the step stores its result and the unfused
+            // concretisation follows.
+            const bool join_end = residual && j == j_end && j_end > 0 && wait_for == j_end - 1;
+            const bool join = (j > j_end && wait_for == j - 1) || join_end;
+            const bool store_step = j > j_end || join_end;
             const float *add_hi = (join && kept >= 0) ? net->buf[kept] : nullptr;
             const float *add_lo = (join && kept >= 0 && kept_pair) ? net->buf_lo[kept] : nullptr;
             const int add_identity = (join && wait_identity) ? 1 : 0;
@@ -911,11 +928,12 @@ cert_status_t cert_backsub_bounds(cert_net_t *net, const float *centers, float e
                 a.slot_stride = net->slot_stride;
                 a.status = net->status_dev;
                 const int groups = std::min(a.total_tiles, net->sm_count / ctas);
-                if (j > j_end) {
+                if (store_step) {
                     const LayerDev &Lb = net->layers[j - 1];
-                    a.has_relu = Lb.relu_after;
+                    a.has_relu = join_end ? 0 : Lb.relu_after;
                     a.split_out = P_lo != nullptr;
-                    a.lamL = Lb.lamL; a.lamU = Lb.lamU; a.nuU = Lb.nuU; a.bias_below = Lb.bias_n;
+                    a.lamL = Lb.lamL; a.lamU = Lb.lamU; a.nuU = Lb.nuU;
+                    a.bias_below = join_end ? net->zeros : Lb.bias_n;
                     a.add_hi = add_hi; a.add_lo = add_lo; a.add_identity = add_identity;
                     cert::launch_gemm_tc(cert::TC_EPI_RELU, ctas, groups, T.a_hi[cur], T.a_lo[cur], T.b_hi, T.b_lo,
                                          T.o_hi[nxt], T.o_lo[nxt], a, T.plan.smem_bytes, st);
@@ -931,6 +949,11 @@ cert_status_t cert_backsub_bounds(cert_net_t *net, const float *centers, float e
                 cur = nxt;
                 dcur ^= 1;
                 dslots = T.plan.n_tiles;
+                if (join_end) {
+                    cert::launch_concretize(P, net->dbuf[dcur], dslots, net->slot_stride, box_l, box_u, Lj.n_in,
+                                            Lj.ld_in, batch, Lk.n_out, lb_out, ub_out, n_total, Lk.out_off, st);
+                    rec.mark(CERT_CLASS_CONCRETIZE);
+                }
                 continue;
             }
             if (Lj.kind == CERT_LAYER_CONV2D) {
@@ -940,11 +963,12 @@ cert_status_t cert_backsub_bounds(cert_net_t *net, const float *centers, float e
                 ep.n_k = Lk.n_out;
                 ep.d_in = net->dbuf[dcur]; ep.n_slots_in = dslots; ep.slot_stride = net->slot_stride;
                 ep.d_out = net->dbuf[dcur];
-                if (j > j_end) {
+                if (store_step) {
                     const LayerDev &Lb = net->layers[j - 1];
                     ep.mode = cert::CONVT_EPI_RELU;
-                    ep.has_relu = Lb.relu_after;
-                    ep.lamL = Lb.lamL; ep.lamU = Lb.lamU; ep.nuU = Lb.nuU; ep.bias_below = Lb.bias_n;
+                    ep.has_relu = join_end ? 0 : Lb.relu_after;
+                    ep.lamL = Lb.lamL; ep.lamU = Lb.lamU; ep.nuU = Lb.nuU;
+                    ep.bias_below = join_end ? net->zeros : Lb.bias_n;
                     ep.P = P; ep.P_lo = P_lo;
                     ep.add_hi = add_hi; ep.add_lo = add_lo; ep.add_identity = add_identity;
                 } else {
@@ -957,6 +981,11 @@ cert_status_t cert_backsub_bounds(cert_net_t *net, const float *centers, float e
                 if (join) { wait_for = -1; wait_identity = false; kept = -1; }
                 cur = nxt;
                 dslots = 1;
+                if (join_end) {
+                    cert::launch_concretize(P, net->dbuf[dcur], dslots, net->slot_stride, box_l, box_u, Lj.n_in,
+                                            Lj.ld_in, batch, Lk.n_out, lb_out, ub_out, n_total, Lk.out_off, st);
+                    rec.mark(CERT_CLASS_CONCRETIZE);
+                }
                 continue;
             }
             cert::launch_gemm_ffma(Q, Lj.ld_out, Lj.W, Lj.ld_in, P, Lj.ld_in, rows, Lj.n_in, Lj.n_out, st);
@@ -978,6 +1007,20 @@ cert_status_t cert_backsub_bounds(cert_net_t *net, const float *centers, float e
                                         Lj.ld_in, batch, Lk.n_out, lb_out, ub_out, n_total, Lk.out_off, st);
                 rec.mark(CERT_CLASS_CONCRETIZE);
             }
+        }
+        if (residual && wait_for >= 0) {
+            // the traversal stopped above the connection's source: the waiting neurons are simplified against
+            // their own concrete bounds
+            const float *S_hi = kept >= 0 ? net->buf[kept] : nullptr;
+            const float *S_lo = (kept >= 0 && kept_pair) ? net->buf_lo[kept] : nullptr;
+            float *slot = nullptr;
+            if (bounds_in_slots) {
+                slot = net->dbuf[dcur] + (size_t)dslots * net->slot_stride;
+                ++dslots;
+            }
+            cert::launch_skip_concretize(S_hi, S_lo, wait_identity ? 1 : 0, net->layers[wait_for], rows, Lk, slot,
+                                         lb_out, ub_out, n_total, st);
+            rec.mark(CERT_CLASS_CONCRETIZE);
         }
         if (Lk.relu_after || bounds_in_slots || k + 1 < K) {
             cert::launch_relax(Lk, lb_out, ub_out, n_total, batch, net->codes, net->n_relu,

@@ -110,6 +110,16 @@ void launch_relu_step(const LayerDev &Lj, int batch, int n_k, float *P, float *P
 void launch_add_skip(float *P, const float *S_hi, const float *S_lo, int identity, long long rows, int n, int ld,
                      int n_k, cudaStream_t st);
 
+// Interval step of layer Lk with a residual connection from layer Ls: lb += actL_s, ub += actU_s.
+void launch_add_act_bounds(const LayerDev &Lk, const LayerDev &Ls, int batch, float *lb_out, float *ub_out,
+                           int n_total, cudaStream_t st);
+// A traversal of layer Lk's rows stopped while coefficients (S_hi (+ S_lo) [rows][Ls.ld_out], and / or the unit
+// coefficient of the row's own neuron) still waited on layer Ls's outputs: their simplification against Ls's
+// concrete output bounds goes to `slot` [rows] if given, else is added to lb_out / ub_out.
+void launch_skip_concretize(const float *S_hi, const float *S_lo, int identity, const LayerDev &Ls, long long rows,
+                            const LayerDev &Lk, float *slot, float *lb_out, float *ub_out, int n_total,
+                            cudaStream_t st);
+
 // map(simplify_lower/upper): rows of P [rows][ld0] against the box.
 void launch_concretize(const float *P, const float *d, int n_slots, long long slot_stride, const float *l0,
                        const float *u0, int n0, int ld0, int batch, int n_k, float *lb_out, float *ub_out, int n_total, int out_off,

@@ -151,6 +151,49 @@ __global__ void add_skip_kernel(float *__restrict__ P, const float *__restrict__
     P[idx] += s;
 }
 
+// Interval step of a layer with a residual connection: the source's concrete output bounds are added.
+__global__ void add_act_bounds_kernel(float *__restrict__ lb_out, float *__restrict__ ub_out, int n_total,
+                                      int out_off, int n_k, int batch, const float *__restrict__ actL,
+                                      const float *__restrict__ actU, int ld_act) {
+    const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= (long long)batch * n_k) return;
+    const int b = (int)(idx / n_k), i = (int)(idx % n_k);
+    lb_out[(size_t)b * n_total + out_off + i] += actL[(size_t)b * ld_act + i];
+    ub_out[(size_t)b * n_total + out_off + i] += actU[(size_t)b * ld_act + i];
+}
+
+// A traversal stopped with coefficients still waiting on a residual connection's source: those neurons are
+// simplified against their own concrete bounds (map(simplify_lower/upper)); one warp per row.  The term goes
+// to a slot of the row constants (slot != nullptr) or is added to the bounds already written.
+__global__ void skip_concretize_kernel(const float *__restrict__ S_hi, const float *__restrict__ S_lo, int identity,
+                                       const float *__restrict__ actL, const float *__restrict__ actU, int ld_act,
+                                       long long rows, int n, int ld, int n_k, float *__restrict__ slot,
+                                       float *__restrict__ lb_out, float *__restrict__ ub_out, int n_total,
+                                       int out_off) {
+    const long long r = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int lane = threadIdx.x & 31;
+    if (r >= rows) return;
+    const int b = (int)(r / (2LL * n_k));
+    const int upper = (int)((r / n_k) & 1);
+    const int i = (int)(r % n_k);
+    const float *lrow = actL + (size_t)b * ld_act, *urow = actU + (size_t)b * ld_act;
+    float term = 0.0f;
+    if (S_hi) {
+        for (int t = lane; t < n; t += 32) {
+            float c = S_hi[(size_t)r * ld + t];
+            if (S_lo) c += S_lo[(size_t)r * ld + t];
+            const bool nonneg = (c >= 0.0f);
+            term = fmaf(c, (nonneg != (upper != 0)) ? lrow[t] : urow[t], term);
+        }
+        term = warp_sum(term);
+    }
+    if (lane == 0) {
+        if (identity) term += upper ? urow[i] : lrow[i];
+        if (slot) slot[r] = term;
+        else (upper ? ub_out : lb_out)[(size_t)b * n_total + out_off + i] += term;
+    }
+}
+
 // Sum of the slots that hold a row's constant (or bound), in slot order.
 __device__ __forceinline__ float slot_sum(const float *__restrict__ d, int n_slots, long long stride,
                                           long long r) {
@@ -493,6 +536,21 @@ void launch_add_skip(float *P, const float *S_hi, const float *S_lo, int identit
                      int n_k, cudaStream_t st) {
     const long long total = rows * (long long)ld;
     add_skip_kernel<<<(unsigned)ceil_div_ll(total, 256), 256, 0, st>>>(P, S_hi, S_lo, identity, total, n, ld, n_k);
+}
+
+void launch_add_act_bounds(const LayerDev &Lk, const LayerDev &Ls, int batch, float *lb_out, float *ub_out,
+                           int n_total, cudaStream_t st) {
+    const long long n = (long long)batch * Lk.n_out;
+    add_act_bounds_kernel<<<(unsigned)ceil_div_ll(n, 256), 256, 0, st>>>(lb_out, ub_out, n_total, Lk.out_off, Lk.n_out,
+                                                                       batch, Ls.actL, Ls.actU, Ls.ld_out);
+}
+
+void launch_skip_concretize(const float *S_hi, const float *S_lo, int identity, const LayerDev &Ls, long long rows,
+                            const LayerDev &Lk, float *slot, float *lb_out, float *ub_out, int n_total,
+                            cudaStream_t st) {
+    skip_concretize_kernel<<<grid_for_warps(rows), kWarpsPerBlock * 32, 0, st>>>(
+        S_hi, S_lo, identity, Ls.actL, Ls.actU, Ls.ld_out, rows, Ls.n_out, Ls.ld_out, Lk.n_out, slot, lb_out, ub_out,
+        n_total, Lk.out_off);
 }
 
 void launch_concretize(const float *P, const float *d, int n_slots, long long slot_stride, const float *l0,

@@ -470,6 +470,24 @@ def test_residual_connection_into_the_output_layer_and_back_to_back_blocks(mode)
     compare(run_gpu(w, contraction={"ffma": 1, "tc": 2, "tc16": 3}[mode]), ref, label=f"output_connection/{mode}")
 
 
+@pytest.mark.parametrize("mode", ["ffma", "tc"])
+@pytest.mark.parametrize("name", ["resfc_ragged", "resfc_wide", "resconv"])
+def test_residual_nets_traversals_that_stop_early(name, mode):
+    """IBP, CROWN-IBP, DeepPoly_p and mixed depths: a traversal may end on a connection's source (the waiting
+    coefficients join before the simplification), above it (they are simplified on their own), or below it."""
+    w = RES_NETS[name]()
+    for vname, steps in _variant_steps(len(w.layers)).items():
+        ref = orc.deeppoly(w.layers, w.centers, w.eps, w.clip_lo, w.clip_hi, skip_from=w.skip_from,
+                           backsteps_per_layer=steps)
+        g = run_gpu(w, contraction=MODES[mode], backsteps=steps)
+        compare(g, ref, label=f"{name}/{vname}/{mode}")
+    for p in (3, 4):
+        steps = [p] * len(w.layers)
+        ref = orc.deeppoly(w.layers, w.centers, w.eps, w.clip_lo, w.clip_hi, skip_from=w.skip_from,
+                           backsteps_per_layer=steps)
+        compare(run_gpu(w, contraction=MODES[mode], backsteps=steps), ref, label=f"{name}/p{p}/{mode}")
+
+
 def test_residual_refusals():
     import torch
     from paper_2507_20055_b200 import binding
@@ -484,9 +502,10 @@ def test_residual_refusals():
         assert binding.lib.cert_net_set_conv_patches(net._h, 1) == 2          # CERT_ERR_UNSUPPORTED
         assert binding.lib.cert_net_enable_reusecert(net._h) == 2
         c = torch.from_numpy(w.centers).cuda()
+        net.set_contraction(3)
         with pytest.raises(binding.CertError):
-            net.backsub_bounds(c, w.eps, [1] * len(w.layers))                  # a traversal that stops early
-        net.backsub_bounds(c, w.eps, [-1] * len(w.layers))                     # full traversals are fine
+            net.backsub_bounds(c, w.eps, [1] * len(w.layers))                  # fp16 split: full traversals only
+        net.backsub_bounds(c, w.eps, [-1] * len(w.layers))
         torch.cuda.synchronize()
     finally:
         net.destroy()
