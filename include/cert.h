@@ -220,7 +220,9 @@ cert_status_t cert_net_set_contraction(cert_net_t *net, int mode);
  * receptive-field patches, bit 4 = TC3XFP16, bit 5 = TC3XFP16 with a whole traversal per launch (nets whose
  * hidden layers are at most 256 neurons wide keep the coefficient panel in shared memory from the start of
  * a traversal to its concretisation; the environment variable CERT_CHAIN=0, read at create, keeps such nets
- * on one launch per back-step). */
+ * on one launch per back-step), bit 6 = a conv back-step on dense coefficient maps ran in its banded
+ * tensor-core form (the environment variable CERT_CONV_BANDS=0, read at create, keeps those steps on the
+ * FMA units). */
 int cert_net_last_contraction_paths(const cert_net_t *net);
 
 /*

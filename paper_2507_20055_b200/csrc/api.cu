@@ -48,6 +48,21 @@ struct TcPatchStep {
     cert::TcPlan plan;
 };
 
+// Banded tensor-core form of the back-step through conv layer j on dense coefficient maps (TcArgs::n_bands):
+// s consecutive rows of the map below depend on `rin` consecutive rows of layer j's output map only, and the
+// matrix between the two is the same for every band.  With the maps held y-major both windows are contiguous
+// pieces of a row, so the step is the ordinary contraction with a K window per tile.  Usable for layer j when it
+// is for every layer below too: a traversal, once its matrix is y-major, stays on this form to its end.
+struct BandStep {
+    bool usable = false;
+    int K = 0, N = 0;                    // rin * c_out * w_out; s * c_in * w_in (both multiples of 32)
+    int rin = 0, o_shift = 0, y_shift = 0, n_bands = 0;
+    float *T_hi = nullptr, *T_lo = nullptr;      // band matrix transposed, [N][K], TF32 split
+    float *bias_y = nullptr;             // [ld_in] bias of layer j-1 per neuron, y-major; null for j = 0
+    cert::TcMap b_hi, b_lo, a_hi[2], a_lo[2], o_hi[2], o_lo[2];
+    cert::TcPlan plan;
+};
+
 // ReuseCert: per affine layer k >= 1 the block weight matrix [[W+^T, W-^T], [W-^T, W+^T]] as the K-major B
 // operand (rows = the 2*n_k output columns, columns = the 2*n_{k-1} columns of the layer below), TF32 split.
 struct ReuseLayer {
@@ -103,7 +118,9 @@ struct cert_net {
     int tc_ctas = 1;                         // CTAs per row panel of the tensor-core kernel (2: cta_group::2)
     bool conv_patches = true;                // conv-sourced rows travel as receptive-field patches where they can
     std::vector<std::vector<TcPatchStep>> tcp;   // [k]: the leading patch steps of layer k's traversal that can run on the tensor cores
-    float *gat[3] = {nullptr, nullptr, nullptr}; // gathered windows, [max_batch * positions][ldN] each
+    float *gat[3] = {nullptr, nullptr, nullptr}; // gathered windows, [max_batch * positions][ldN] each (y-major vectors for the banded form)
+    size_t gat_floats = 0;
+    std::vector<BandStep> band;                  // [j]: banded tensor-core form of the step through conv layer j
     ReuseState reuse;
     unsigned char *codes = nullptr;          // [max_batch][n_relu]
     int *status_dev = nullptr;               // sticky device status word
@@ -417,9 +434,113 @@ cert_status_t setup_patch_tc(cert_net *net, const cert_layer_desc_t *descs) {
             net->tcp[k].push_back(S);
         }
     }
-    if (gat_floats)
-        for (int i = 0; i < 3; ++i)
-            if (!dev_alloc_zero(net, &net->gat[i], gat_floats)) return CERT_ERR_OOM;
+    net->gat_floats = std::max(net->gat_floats, gat_floats);
+    return CERT_OK;
+}
+
+// Banded form of the dense conv back-steps, from the first layer upward while map rows are whole k-blocks
+// (channels * width a multiple of 32 on both sides) and the dense band matrix does at most kBandDenseRatio
+// times the multiply-adds of the convolution itself.
+constexpr int kBandDenseRatio = 12;
+
+cert_status_t setup_band_tc(cert_net *net, const cert_layer_desc_t *descs) {
+    const int K = net->n_layers;
+    net->band.assign(K, BandStep());
+    if (!net->tc_ok || !net->skip_from.empty()) return CERT_OK;
+    if (const char *e = std::getenv("CERT_CONV_BANDS")) {
+        if (std::atoi(e) == 0) return CERT_OK;
+    }
+    const int ctas = net->tc_ctas;
+    std::vector<float> hi, lo, be;
+    for (int j = 0; j + 1 < K; ++j) {
+        const LayerDev &L = net->layers[j];
+        if (L.kind != CERT_LAYER_CONV2D) break;
+        BandStep S;
+        const int s = L.stride;
+        const int row_in = L.c_out * L.w_out, row_out = L.c_in * L.w_in;
+        if (row_in % 32 || row_out % 32) break;
+        // rows of the output map a band needs: oy' = o_shift + (dy + pad - y_shift - ky) / s over all (dy, ky)
+        int best_rin = 1 << 30;
+        for (int ys = 0; ys < s; ++ys) {
+            int qmin = 1 << 30, qmax = -(1 << 30);
+            for (int dy = 0; dy < s; ++dy)
+                for (int ky = 0; ky < L.kh; ++ky) {
+                    const int num = dy + L.pad - ys - ky;
+                    if (((num % s) + s) % s) continue;
+                    const int q = num >= 0 ? num / s : -((-num) / s);
+                    qmin = std::min(qmin, q); qmax = std::max(qmax, q);
+                }
+            if (qmax >= qmin && qmax - qmin + 1 < best_rin) {
+                best_rin = qmax - qmin + 1; S.rin = best_rin; S.o_shift = -qmin; S.y_shift = ys;
+            }
+        }
+        if (best_rin > 8) break;
+        S.K = S.rin * row_in;
+        S.N = s * row_out;
+        S.n_bands = (L.h_in + S.y_shift + s - 1) / s;
+        // every band must reach at least one row of the map (its accumulator is written by its first k-block)
+        bool reach = true;
+        for (int i = 0; i < S.n_bands; ++i)
+            reach = reach && (i - S.o_shift < L.h_out) && (i - S.o_shift + S.rin > 0);
+        if (!reach) break;
+        if ((long long)S.K * S.N * S.n_bands > (long long)kBandDenseRatio * L.n_out * L.c_in * L.kh * L.kw) break;
+        if ((size_t)S.K * S.N > (size_t)(16u << 20)) break;
+        S.plan = cert::tc_tile_plan(S.N, ctas);
+        if (S.plan.stages < 2) break;
+        hi.assign((size_t)S.N * S.K, 0.0f);
+        lo.assign((size_t)S.N * S.K, 0.0f);
+        const float *W = descs[j].weight;
+        for (int dy = 0; dy < s; ++dy)
+            for (int ci = 0; ci < L.c_in; ++ci)
+                for (int ix = 0; ix < L.w_in; ++ix) {
+                    const size_t n = ((size_t)dy * L.c_in + ci) * L.w_in + ix;
+                    for (int r = 0; r < S.rin; ++r) {
+                        const int ky = dy + L.pad - S.y_shift + s * (S.o_shift - r);
+                        if (ky < 0 || ky >= L.kh) continue;
+                        for (int co = 0; co < L.c_out; ++co)
+                            for (int ox = 0; ox < L.w_out; ++ox) {
+                                const int kx = ix + L.pad - s * ox;
+                                if (kx < 0 || kx >= L.kw) continue;
+                                const size_t kk = ((size_t)r * L.c_out + co) * L.w_out + ox;
+                                const float w = W[(((size_t)co * L.c_in + ci) * L.kh + ky) * L.kw + kx];
+                                const float h = host_tf32(w);
+                                hi[n * S.K + kk] = h;
+                                lo[n * S.K + kk] = host_tf32(w - h);
+                            }
+                    }
+                }
+        if (!dev_alloc(net, (void **)&S.T_hi, hi.size() * sizeof(float)) ||
+            !dev_alloc(net, (void **)&S.T_lo, lo.size() * sizeof(float)))
+            return CERT_ERR_OOM;
+        if (cudaMemcpy(S.T_hi, hi.data(), hi.size() * sizeof(float), cudaMemcpyHostToDevice) != cudaSuccess ||
+            cudaMemcpy(S.T_lo, lo.data(), lo.size() * sizeof(float), cudaMemcpyHostToDevice) != cudaSuccess)
+            return CERT_ERR_CUDA;
+        if (j > 0) {
+            be.assign(L.ld_in, 0.0f);
+            for (int y = 0; y < L.h_in; ++y)
+                for (int ci = 0; ci < L.c_in; ++ci)
+                    for (int x = 0; x < L.w_in; ++x) be[((size_t)y * L.c_in + ci) * L.w_in + x] = descs[j - 1].bias[ci];
+            if (!dev_alloc(net, (void **)&S.bias_y, be.size() * sizeof(float))) return CERT_ERR_OOM;
+            if (cudaMemcpy(S.bias_y, be.data(), be.size() * sizeof(float), cudaMemcpyHostToDevice) != cudaSuccess)
+                return CERT_ERR_CUDA;
+        }
+        long long rows_max = 0;
+        for (int k = j + 1; k < K; ++k) rows_max = std::max(rows_max, 2LL * net->max_batch * net->layers[k].n_out);
+        bool ok = cert::tc_make_map(&S.b_hi, S.T_hi, S.K, S.N, S.K, S.plan.bn / ctas) &&
+                  cert::tc_make_map(&S.b_lo, S.T_lo, S.K, S.N, S.K, S.plan.bn / ctas);
+        for (int p = 0; p < 2 && ok; ++p) {
+            ok = cert::tc_make_map(&S.a_hi[p], net->buf[p], L.n_out, rows_max, L.ld_out, 128) &&
+                 cert::tc_make_map(&S.a_lo[p], net->buf_lo[p], L.n_out, rows_max, L.ld_out, 128);
+            if (ok && j > 0)
+                ok = cert::tc_make_map(&S.o_hi[p], net->buf[p], L.ld_in, rows_max, L.ld_in, 32) &&
+                     cert::tc_make_map(&S.o_lo[p], net->buf_lo[p], L.ld_in, rows_max, L.ld_in, 32);
+        }
+        if (!ok) break;
+        S.usable = true;
+        net->d_slots = std::max(net->d_slots, S.n_bands * S.plan.n_tiles);
+        net->gat_floats = std::max(net->gat_floats, (size_t)net->max_batch * L.ld_in);
+        net->band[j] = S;
+    }
     return CERT_OK;
 }
 
@@ -617,6 +738,10 @@ cert_status_t cert_net_create_residual(const cert_layer_desc_t *layers, int n_la
         net->slot_stride = (long long)max_rows;
         if (ok) fail = setup_tensor_core_path(net, layers, max_elems);
         if (ok && fail == CERT_OK) fail = setup_patch_tc(net, layers);
+        if (ok && fail == CERT_OK) fail = setup_band_tc(net, layers);
+        if (ok && fail == CERT_OK && net->gat_floats)
+            for (int i = 0; i < 3 && fail == CERT_OK; ++i)
+                if (!dev_alloc_zero(net, &net->gat[i], net->gat_floats)) fail = CERT_ERR_OOM;
         if (ok && fail == CERT_OK && !net->skip_from.empty()) {
             // a traversal that stops early may leave one more partial bound per row (the waiting coefficients)
             net->d_slots += 1;
@@ -704,6 +829,11 @@ cert_status_t cert_backsub_bounds(cert_net_t *net, const float *centers, float e
         auto on_tc = [&](int j) {
             return net->contraction != CERT_CONTRACTION_FFMA && net->tc_ok && net->tc[j].usable;
         };
+        // ... or, for a conv layer on dense maps, in the banded tensor-core form?  Its input is a TF32 pair too.
+        auto on_band = [&](int j) {
+            return net->contraction != CERT_CONTRACTION_FFMA && net->tc_ok && net->band[j].usable;
+        };
+        auto wants_pair = [&](int j) { return on_tc(j) || on_band(j); };
         // fp16-split tensor-core chain (FC nets): start, then one kernel per layer with the ReLU step fused,
         // the last one concretising.
         if (net->contraction == CERT_CONTRACTION_TC3XFP16 && net->chain_ok) {
@@ -880,8 +1010,9 @@ cert_status_t cert_backsub_bounds(cert_net_t *net, const float *centers, float e
         }
         // expression over the outputs of layer k-1, pushed through its ReLU
         cert::launch_init_expr(Lk, net->layers[k - 1], batch, net->buf[cur],
-                               on_tc(k - 1) ? net->buf_lo[cur] : nullptr, net->dbuf[dcur], st);
+                               wants_pair(k - 1) ? net->buf_lo[cur] : nullptr, net->dbuf[dcur], st);
         rec.mark(CERT_CLASS_RELU_STEP);
+        bool y_major = false;     // the coefficient maps are held [y][channel][x] (banded conv steps)
         // Residual connections: the coefficients on a connection's source wait (kept: the buffer that holds
         // them, untouched meanwhile; identity: the unit coefficient of layer k's own connection) until the
         // step whose result is over that source's outputs, where they join before the ReLU back-step.
@@ -897,7 +1028,7 @@ cert_status_t cert_backsub_bounds(cert_net_t *net, const float *centers, float e
                 wait_for = net->skip_from[j];
                 wait_identity = false;
                 kept = cur;
-                kept_pair = on_tc(j);
+                kept_pair = wants_pair(j);
             }
             int nxt = cur ^ 1;
             if (residual) {
@@ -914,7 +1045,63 @@ cert_status_t cert_backsub_bounds(cert_net_t *net, const float *centers, float e
             const float *add_lo = (join && kept >= 0 && kept_pair) ? net->buf_lo[kept] : nullptr;
             const int add_identity = (join && wait_identity) ? 1 : 0;
             float *Q = net->buf[cur], *P = net->buf[nxt];
-            float *P_lo = (j > j_end && on_tc(j - 1)) ? net->buf_lo[nxt] : nullptr;
+            float *P_lo = (j > j_end && wants_pair(j - 1)) ? net->buf_lo[nxt] : nullptr;
+            if (Lj.kind == CERT_LAYER_CONV2D && on_band(j)) {
+                // dense coefficient maps through conv layer j on the tensor cores, band by band
+                const BandStep &S = net->band[j];
+                const int ctas = net->tc_ctas;
+                if (!y_major) {
+                    cert::launch_to_ymajor_pair(net->buf[cur], net->buf_lo[cur], net->buf[nxt], net->buf_lo[nxt], rows,
+                                                Lj.c_out, Lj.h_out, Lj.w_out, Lj.ld_out, st);
+                    rec.mark(CERT_CLASS_CONV);
+                    cur = nxt;
+                    nxt = cur ^ 1;
+                    y_major = true;
+                }
+                const float *src[3] = {nullptr, nullptr, nullptr};
+                const float fill[3] = {1.0f, 1.0f, 0.0f};
+                int n_arr = 3;
+                if (j > j_end) {
+                    const LayerDev &Lb = net->layers[j - 1];
+                    if (Lb.relu_after) { src[0] = Lb.lamL; src[1] = Lb.lamU; src[2] = Lb.nuU; }
+                } else {
+                    src[0] = box_l; src[1] = box_u;
+                    n_arr = 2;
+                }
+                cert::launch_to_ymajor_vectors(Lj.c_in, Lj.h_in, Lj.w_in, Lj.ld_in, batch, n_arr, src, fill, net->gat, st);
+                rec.mark(CERT_CLASS_CONV);
+                cert::TcArgs a;
+                std::memset(&a, 0, sizeof(a));
+                a.M = rows; a.K = S.K; a.n_k = Lk.n_out; a.ld_n = Lj.ld_in;
+                a.n_bands = S.n_bands; a.band_rin = S.rin; a.band_o_shift = S.o_shift; a.band_h_in = Lj.h_out;
+                a.band_row_in = Lj.c_out * Lj.w_out;
+                a.band_s = Lj.stride; a.band_y_shift = S.y_shift; a.band_row_out = Lj.c_in * Lj.w_in;
+                a.bn = S.plan.bn; a.n_tiles = S.plan.n_tiles; a.stages = S.plan.stages;
+                a.tmem_cols = S.plan.tmem_cols;
+                a.total_tiles = (int)cert::ceil_div_ll(rows, 128 * ctas) * S.n_bands * S.plan.n_tiles;
+                a.d_in = net->dbuf[dcur]; a.n_slots_in = dslots; a.d_out = net->dbuf[dcur ^ 1];
+                a.slot_stride = net->slot_stride;
+                a.status = net->status_dev;
+                const int groups = std::min(a.total_tiles, net->sm_count / ctas);
+                if (j > j_end) {
+                    a.has_relu = 1;
+                    a.split_out = 1;          // a banded step follows
+                    a.lamL = net->gat[0]; a.lamU = net->gat[1]; a.nuU = net->gat[2]; a.bias_below = S.bias_y;
+                    cert::launch_gemm_tc(cert::TC_EPI_RELU_BAND, ctas, groups, S.a_hi[cur], S.a_lo[cur], S.b_hi, S.b_lo,
+                                         S.o_hi[nxt], S.o_lo[nxt], a, S.plan.smem_bytes, st);
+                } else {
+                    a.l0 = net->gat[0]; a.u0 = net->gat[1];
+                    cert::launch_gemm_tc(cert::TC_EPI_CONCRETIZE_BAND, ctas, groups, S.a_hi[cur], S.a_lo[cur], S.b_hi,
+                                         S.b_lo, S.a_hi[cur], S.a_lo[cur], a, S.plan.smem_bytes, st);
+                    bounds_in_slots = true;
+                }
+                rec.mark(CERT_CLASS_CONV);
+                paths |= 2 | (ctas == 2 ? 4 : 0) | 64;
+                cur = nxt;
+                dcur ^= 1;
+                dslots = S.n_bands * S.plan.n_tiles;
+                continue;
+            }
             if (on_tc(j)) {
                 const TcLayer &T = net->tc[j];
                 cert::TcArgs a;

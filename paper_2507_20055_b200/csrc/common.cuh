@@ -189,6 +189,14 @@ void launch_patch_gather(const LayerDev &Lk, const LayerDev &Lj, const PatchLeve
 void launch_patch_step(const LayerDev &Lk, const LayerDev &Lj, const PatchLevel &in, const PatchLevel &out,
                        const float *in_patch, long long rows, int sms, const ConvtEpilogue &ep, cudaStream_t st);
 
+// ---- y-major copies for the banded tensor-core form of the dense conv back-steps (conv_patch.cu) ----
+// Maps [c][h][w] -> [h][c][w]: a coefficient matrix held as a TF32 pair, and up to three per-neuron arrays
+// [batch][ld] (a null src[i] stands for fill[i]).
+void launch_to_ymajor_pair(const float *src_hi, const float *src_lo, float *dst_hi, float *dst_lo, long long rows,
+                           int c, int h, int w, int ld, cudaStream_t st);
+void launch_to_ymajor_vectors(int c, int h, int w, int ld, int batch, int n_arr, const float *const *src,
+                              const float *fill, float *const *dst, cudaStream_t st);
+
 // ---- ReuseCert (reuse.cu): shapes over the input layer, one matrix S per layer ----
 // S rows are (box, s): s < n0 input coordinate, s == n0 constant, zero rows up to R per box; columns
 // [L (n) | U (n)] padded to ld_s.  S is held as a TF32 pair.

@@ -325,6 +325,65 @@ void launch_patch_start(const LayerDev &Lk, const LayerDev &Lb, int pitch, int b
         Lb.nuU, Lb.bias_n);
 }
 
+// ---- y-major copies for the banded tensor-core form of the dense conv back-steps ----
+// A map [c][h][w] (flattened channel-major, as everywhere else) reordered to [h][c][w], so that a band of map
+// rows is one contiguous piece of the row.
+
+// Coefficient matrix (TF32 pair) of `rows` rows: dst[r][(y*c + ch)*w + x] = src[r][(ch*h + y)*w + x].
+__global__ void to_ymajor_pair_kernel(const float *__restrict__ src_hi, const float *__restrict__ src_lo,
+                                      float *__restrict__ dst_hi, float *__restrict__ dst_lo, long long rows, int c,
+                                      int h, int w, int ld) {
+    const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    const int n = c * h * w;
+    if (idx >= rows * (long long)n) return;
+    const long long r = idx / n;
+    const int e = (int)(idx - r * n);
+    const int y = e / (c * w), rem = e - y * (c * w);
+    const int ch = rem / w, x = rem - ch * w;
+    const size_t s = (size_t)r * ld + (size_t)(ch * h + y) * w + x;
+    dst_hi[(size_t)r * ld + e] = src_hi[s];
+    dst_lo[(size_t)r * ld + e] = src_lo[s];
+}
+
+// Up to three per-neuron arrays [batch][ld]; a null source stands for fill[i].
+struct YMajorVectors {
+    int c, h, w, ld, n_arr;
+    const float *src[3];
+    float fill[3];
+    float *dst[3];
+};
+
+__global__ void to_ymajor_vectors_kernel(const YMajorVectors g, int batch) {
+    const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    const int n = g.c * g.h * g.w;
+    if (idx >= (long long)batch * n) return;
+    const int b = (int)(idx / n), e = (int)(idx - (long long)b * n);
+    const int y = e / (g.c * g.w), rem = e - y * (g.c * g.w);
+    const int ch = rem / g.w, x = rem - ch * g.w;
+    const size_t s = (size_t)b * g.ld + (size_t)(ch * g.h + y) * g.w + x;
+    for (int i = 0; i < g.n_arr; ++i) g.dst[i][(size_t)b * g.ld + e] = g.src[i] ? g.src[i][s] : g.fill[i];
+}
+
+void launch_to_ymajor_pair(const float *src_hi, const float *src_lo, float *dst_hi, float *dst_lo, long long rows,
+                           int c, int h, int w, int ld, cudaStream_t st) {
+    const long long total = rows * (long long)c * h * w;
+    to_ymajor_pair_kernel<<<(unsigned)ceil_div_ll(total, 256), 256, 0, st>>>(src_hi, src_lo, dst_hi, dst_lo, rows, c, h,
+                                                                           w, ld);
+}
+
+void launch_to_ymajor_vectors(int c, int h, int w, int ld, int batch, int n_arr, const float *const *src,
+                              const float *fill, float *const *dst, cudaStream_t st) {
+    YMajorVectors g;
+    g.c = c; g.h = h; g.w = w; g.ld = ld; g.n_arr = n_arr;
+    for (int i = 0; i < 3; ++i) {
+        g.src[i] = i < n_arr ? src[i] : nullptr;
+        g.fill[i] = i < n_arr ? fill[i] : 0.0f;
+        g.dst[i] = i < n_arr ? dst[i] : nullptr;
+    }
+    const long long total = (long long)batch * c * h * w;
+    to_ymajor_vectors_kernel<<<(unsigned)ceil_div_ll(total, 256), 256, 0, st>>>(g, batch);
+}
+
 void launch_patch_gather(const LayerDev &Lk, const LayerDev &Lj, const PatchLevel &out, int ld_dst, int batch,
                          int n_arr, const float *const *src, const float *fill, float *const *dst,
                          cudaStream_t st) {

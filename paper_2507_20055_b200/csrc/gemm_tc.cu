@@ -57,6 +57,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_consta
                const __grid_constant__ CUtensorMap map_b_hi, const __grid_constant__ CUtensorMap map_b_lo,
                const __grid_constant__ CUtensorMap map_o_hi, const __grid_constant__ CUtensorMap map_o_lo,
                const TcArgs a) {
+    constexpr bool kBand = (EPI == TC_EPI_RELU_BAND || EPI == TC_EPI_CONCRETIZE_BAND);
+    constexpr bool kRelu = (EPI == TC_EPI_RELU || EPI == TC_EPI_RELU_SKIP || EPI == TC_EPI_RELU_BAND);
+    constexpr bool kStores = kRelu || EPI == TC_EPI_REUSE;
     pdl_trigger();
     extern __shared__ uint8_t smem_raw[];
     // tiles are aligned to 1024 bytes (a whole swizzle pattern)
@@ -120,18 +123,29 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_consta
             uint32_t phase = 0;
             bool ok = true;
             int armed = 0;      // stage loads issued so far
+            const int bands = kBand ? a.n_bands : 1;
             for (int t = group; t < total_tiles && ok; t += n_groups) {
-                const int row0 = (t / n_tiles) * (BM * CTAS) + (int)rank * BM;
+                const int row0 = (t / (n_tiles * bands)) * (BM * CTAS) + (int)rank * BM;
                 const int col0 = (t % n_tiles) * BN + (int)rank * BNL;
-                for (int kb = 0; kb < num_kb; ++kb) {
+                // banded form: the K window of this tile's band, clipped to the map (whole map rows = whole k-blocks)
+                int kb_lo = 0, kb_hi = num_kb, a_k0 = 0;
+                if (kBand) {
+                    const int first = (t / n_tiles) % bands - a.band_o_shift;      // first map row of the window
+                    const int per_row = a.band_row_in / BK;
+                    kb_lo = (first < 0 ? -first : 0) * per_row;
+                    const int rows_in = a.band_h_in - first < a.band_rin ? a.band_h_in - first : a.band_rin;
+                    kb_hi = rows_in * per_row;
+                    a_k0 = first * a.band_row_in;
+                }
+                for (int kb = kb_lo; kb < kb_hi; ++kb) {
                     if (!mbar_wait(&bars->empty[s], phase ^ 1) || *abort_flag) { ok = false; break; }
                     uint8_t *st = smem + (size_t)s * stage_bytes;
                     // the leader's barrier counts the bytes of every CTA of the group
                     if (rank == 0) mbar_arrive_expect_tx(&bars->full[s], stage_bytes * CTAS);
                     const uint32_t bar = CTAS == 2 ? map_to_cta(smem_u32(&bars->full[s]), 0) : smem_u32(&bars->full[s]);
                     const int kx = kb * BK;
-                    tma_load_2d<CTAS>(smem_u32(st), &map_a_hi, bar, kx, row0);
-                    tma_load_2d<CTAS>(smem_u32(st + kATileBytes), &map_a_lo, bar, kx, row0);
+                    tma_load_2d<CTAS>(smem_u32(st), &map_a_hi, bar, a_k0 + kx, row0);
+                    tma_load_2d<CTAS>(smem_u32(st + kATileBytes), &map_a_lo, bar, a_k0 + kx, row0);
                     tma_load_2d<CTAS>(smem_u32(st + 2 * kATileBytes), &map_b_hi, bar, kx, col0);
                     tma_load_2d<CTAS>(smem_u32(st + 2 * kATileBytes + b_tile_bytes), &map_b_lo, bar, kx, col0);
                     ++armed;
@@ -168,7 +182,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_consta
                 if (!mbar_wait(&bars->acc_empty[acc], acc_phase ^ 1) || *abort_flag) { ok = false; break; }
                 tcgen05_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
-                for (int kb = 0; kb < num_kb; ++kb) {
+                int kb_lo = 0, kb_hi = num_kb;
+                if (kBand) {
+                    const int first = (t / n_tiles) % a.n_bands - a.band_o_shift;
+                    const int per_row = a.band_row_in / BK;
+                    kb_lo = (first < 0 ? -first : 0) * per_row;
+                    kb_hi = (a.band_h_in - first < a.band_rin ? a.band_h_in - first : a.band_rin) * per_row;
+                }
+                for (int kb = kb_lo; kb < kb_hi; ++kb) {
                     if (!mbar_wait(&bars->full[s], phase) || *abort_flag) { ok = false; break; }
                     tcgen05_fence_after();
                     const uint32_t st = smem_u32(smem + (size_t)s * stage_bytes);
@@ -179,7 +200,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_consta
 #pragma unroll
                     for (int k = 0; k < BK / 8; ++k) {
                         const uint64_t ko = (uint64_t)(k * 2);   // 8 floats = 32 bytes = 2 x 16-byte units
-                        mma_tf32<CTAS>(d_tmem, da_lo + ko, db_hi + ko, idesc, (kb | k) ? 1u : 0u);
+                        mma_tf32<CTAS>(d_tmem, da_lo + ko, db_hi + ko, idesc, ((kb - kb_lo) | k) ? 1u : 0u);
                         mma_tf32<CTAS>(d_tmem, da_hi + ko, db_lo + ko, idesc, 1u);
                         mma_tf32<CTAS>(d_tmem, da_hi + ko, db_hi + ko, idesc, 1u);
                     }
@@ -202,9 +223,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_consta
                                                    : smem_u32(&bars->acc_empty[0]);
         bool ok = true;
         int lt = 0;
+        const int bands = kBand ? a.n_bands : 1;
         for (int t = group; t < total_tiles && ok; t += n_groups, ++lt) {
             const int nt = t % n_tiles;
-            const long long warp_row0 = (long long)(t / n_tiles) * (BM * CTAS) + (int)rank * BM + quarter * 32;
+            const int band = kBand ? (t / n_tiles) % bands : 0;
+            // first column of the band's window in the (y-major) output row; may be negative at the top of the map
+            const int band_col0 = kBand ? (band * a.band_s - a.band_y_shift) * a.band_row_out : 0;
+            const long long warp_row0 = (long long)(t / (n_tiles * bands)) * (BM * CTAS) + (int)rank * BM + quarter * 32;
             const long long r = warp_row0 + lane;
             const bool row_ok = r < a.M;
             const long long rr = row_ok ? r : 0;
@@ -221,13 +246,19 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_consta
             tcgen05_fence_after();
             const uint32_t t_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN);
             for (int c0 = 0; c0 < BN; c0 += 32) {
-                const int col0 = nt * BN + c0;
-                if (col0 >= a.ld_n) break;                   // warp-uniform; ld_n is a multiple of 32
+                int col0 = nt * BN + c0;
+                if (kBand) {
+                    if (col0 >= a.band_s * a.band_row_out) break;
+                    col0 += band_col0;
+                    if (col0 < 0 || col0 >= a.ld_n) continue;    // a map row above or below the map: no such neurons
+                } else if (col0 >= a.ld_n) {
+                    break;                                   // warp-uniform; ld_n is a multiple of 32
+                }
                 uint32_t v[32];
                 __syncwarp();
                 tmem_ld32(t_addr + (uint32_t)c0, v);
                 tmem_ld_wait();
-                if (EPI == TC_EPI_RELU || EPI == TC_EPI_RELU_SKIP) {
+                if (kRelu) {
                     // the slab is free again once the previous chunk's stores have read it
                     if (lane == 0) tma_store_wait_read();
                     __syncwarp();
@@ -380,15 +411,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_consta
             // epilogue) goes to slot nt; the tile of column 0 also carries the constant so far.
             if (EPI != TC_EPI_REUSE && row_ok) {
                 float tot = dacc;
-                if (nt == 0) {
+                const int slot = band * n_tiles + nt;
+                if (slot == 0) {
                     float prev = 0.0f;
                     for (int sidx = 0; sidx < a.n_slots_in; ++sidx) prev += a.d_in[(size_t)sidx * a.slot_stride + r];
                     tot += prev;
                 }
-                a.d_out[(size_t)nt * a.slot_stride + r] = tot;
+                a.d_out[(size_t)slot * a.slot_stride + r] = tot;
             }
         }
-        if (EPI != TC_EPI_CONCRETIZE && lane == 0) tma_store_wait_all();
+        if (kStores && lane == 0) tma_store_wait_all();
         if (!ok && lane == 0) atomicExch(a.status, 1);
     }
 
@@ -467,7 +499,11 @@ bool tc_driver_init() {
 }
 
 bool tc_prepare_kernels(bool *pair_ok) {
-    cudaError_t e[8];
+    cudaError_t e[12];
+    e[8] = cudaFuncSetAttribute(gemm_tc_kernel<TC_EPI_RELU_BAND, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemMax);
+    e[9] = cudaFuncSetAttribute(gemm_tc_kernel<TC_EPI_RELU_BAND, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemMax);
+    e[10] = cudaFuncSetAttribute(gemm_tc_kernel<TC_EPI_CONCRETIZE_BAND, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemMax);
+    e[11] = cudaFuncSetAttribute(gemm_tc_kernel<TC_EPI_CONCRETIZE_BAND, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemMax);
     e[6] = cudaFuncSetAttribute(gemm_tc_kernel<TC_EPI_RELU_SKIP, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemMax);
     e[7] = cudaFuncSetAttribute(gemm_tc_kernel<TC_EPI_RELU_SKIP, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemMax);
     e[0] = cudaFuncSetAttribute(gemm_tc_kernel<TC_EPI_RELU, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemMax);
@@ -476,7 +512,7 @@ bool tc_prepare_kernels(bool *pair_ok) {
     e[3] = cudaFuncSetAttribute(gemm_tc_kernel<TC_EPI_CONCRETIZE, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemMax);
     e[4] = cudaFuncSetAttribute(gemm_tc_kernel<TC_EPI_REUSE, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemMax);
     e[5] = cudaFuncSetAttribute(gemm_tc_kernel<TC_EPI_REUSE, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemMax);
-    for (int i = 0; i < 8; ++i)
+    for (int i = 0; i < 12; ++i)
         if (e[i] != cudaSuccess) {
             cudaGetLastError();
             return false;
@@ -542,6 +578,16 @@ void launch_gemm_tc(int epi, int ctas, int groups, const TcMap &a_hi, const TcMa
     const CUtensorMap &bl = reinterpret_cast<const CUtensorMap &>(b_lo);
     const CUtensorMap &oh = reinterpret_cast<const CUtensorMap &>(o_hi);
     const CUtensorMap &ol = reinterpret_cast<const CUtensorMap &>(o_lo);
+    if (epi == TC_EPI_RELU_BAND || epi == TC_EPI_CONCRETIZE_BAND) {
+        if (epi == TC_EPI_RELU_BAND) {
+            if (ctas == 2) launch_one<TC_EPI_RELU_BAND, 2>(groups, ah, al, bh, bl, oh, ol, args, smem_bytes, st);
+            else launch_one<TC_EPI_RELU_BAND, 1>(groups, ah, al, bh, bl, oh, ol, args, smem_bytes, st);
+        } else {
+            if (ctas == 2) launch_one<TC_EPI_CONCRETIZE_BAND, 2>(groups, ah, al, bh, bl, oh, ol, args, smem_bytes, st);
+            else launch_one<TC_EPI_CONCRETIZE_BAND, 1>(groups, ah, al, bh, bl, oh, ol, args, smem_bytes, st);
+        }
+        return;
+    }
     const bool skip = args.add_hi || args.add_identity;
     if (epi == TC_EPI_RELU && skip) {
         if (ctas == 2) launch_one<TC_EPI_RELU_SKIP, 2>(groups, ah, al, bh, bl, oh, ol, args, smem_bytes, st);

@@ -9,7 +9,10 @@ constexpr int kTcSmemMax = 227 * 1024;
 
 // TC_EPI_RELU_SKIP: the ReLU epilogue with the waiting coefficients of a residual connection added first (a
 // variant of its own so that the common epilogue carries no code for it).
-enum { TC_EPI_RELU = 0, TC_EPI_CONCRETIZE = 1, TC_EPI_REUSE = 2, TC_EPI_RELU_SKIP = 3 };
+// TC_EPI_RELU_BAND / TC_EPI_CONCRETIZE_BAND: the two path epilogues for the banded form of a conv back-step
+// (TcArgs::n_bands), again as variants of their own.
+enum { TC_EPI_RELU = 0, TC_EPI_CONCRETIZE = 1, TC_EPI_REUSE = 2, TC_EPI_RELU_SKIP = 3, TC_EPI_RELU_BAND = 4,
+       TC_EPI_CONCRETIZE_BAND = 5 };
 
 // Storage for a CUtensorMap (128 bytes, 64-byte aligned), kept opaque so that
 // only gemm_tc.cu needs the driver API header.
@@ -36,6 +39,17 @@ struct TcArgs {
     int n_pos;       // 0: the arrays below hold one vector per box.  > 0: the rows are receptive-field patches of
                      // conv neurons with n_pos output positions; the arrays hold one vector per (box, position),
                      // already gathered to the patch's window (zero outside the map)
+    // Banded form of a conv back-step on dense coefficient maps (n_bands > 0).  Maps are held row-major by map
+    // row ("y-major": [y][channel][x]), so the coefficients of `band_rin` consecutive rows of layer j's output map
+    // are one contiguous K window of a row of A, and the `s` rows of the map below that depend on them are one
+    // contiguous window of the output row.  A work tile is (row panel, band, column tile of the band); the B
+    // operand is the band matrix [s * band_row_out][band_rin * band_row_in], the same for every band.
+    //   A window of band i:  rows i - band_o_shift .. + band_rin - 1 of the map, clipped to [0, band_h_in)
+    //   output window:       columns (i * band_s - band_y_shift) * band_row_out .. + band_s * band_row_out - 1,
+    //                        32-column chunks outside [0, ld_n) are dropped
+    // The relaxation / box arrays are y-major copies, indexed by the output column.
+    int n_bands, band_rin, band_o_shift, band_h_in, band_row_in;   // band_row_in = channels * width of layer j's output map
+    int band_s, band_y_shift, band_row_out;                        // band_row_out = channels * width of the map below
     int has_relu;    // a ReLU sits on the neurons below layer j
     int split_out;   // ReLU epilogue: store the result as a TF32 pair (a tensor-core step follows)
     const float *lamL, *lamU, *nuU;              // [batch (* n_pos)][ld_n]

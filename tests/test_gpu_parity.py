@@ -202,6 +202,10 @@ CONV_NETS = {
     "three_convs": lambda: wl.small_conv((2, 20, 18), [(4, 3, 1, 1), (6, 4, 2, 1), (8, 3, 2, 0)], [12, 3], batch=2,
                                          eps=0.01, seed=85),
     "k5s1p0_k2s2": lambda: wl.small_conv((1, 14, 14), [(6, 5, 1, 0), (4, 2, 2, 0)], [5], batch=2, eps=0.03, seed=86),
+    # map rows (channels x width) that are multiples of 32 floats: the dense steps take the banded tensor-core form
+    "pow2_two_convs": lambda: wl.small_conv((2, 32, 32), [(4, 4, 2, 1), (8, 4, 2, 1)], [12, 4], batch=2, eps=0.01, seed=89),
+    "pow2_first_only": lambda: wl.small_conv((2, 16, 16), [(8, 4, 2, 1), (6, 4, 2, 1)], [20, 5], batch=3, eps=0.01, seed=90),
+    "pow2_k3s1": lambda: wl.small_conv((4, 8, 8), [(8, 3, 1, 1), (8, 3, 1, 1)], [10, 3], batch=2, eps=0.01, seed=95),
 }
 
 
@@ -217,9 +221,12 @@ def test_conv_rows_dense_and_patches(name, form):
     g = run_gpu(w, conv_patches=patches, contraction=contraction)
     # the small nets' windows are not much smaller than their maps: those stay dense either way
     expect_patches = patches and name in ("convsmall", "three_convs", "k5s1p0_k2s2")
-    assert bool(g["paths"] & 8) == expect_patches
+    if not name.startswith("pow2"):
+        assert bool(g["paths"] & 8) == expect_patches
     if expect_patches and form == "patches_tc":
         assert g["paths"] & 2
+    banded = form != "patches_fma" and name in ("convsmall", "pow2_two_convs", "pow2_first_only", "pow2_k3s1")
+    assert bool(g["paths"] & 64) == banded
     compare(g, ref, label=f"{name}/{form}")
     steps = [0] + [1] * (len(w.layers) - 1)
     ref1 = orc.deeppoly(w.layers, w.centers, w.eps, w.clip_lo, w.clip_hi, backsteps_per_layer=steps)
