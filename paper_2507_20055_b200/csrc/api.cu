@@ -59,6 +59,9 @@ struct BandStep {
     int rin = 0, o_shift = 0, y_shift = 0, n_bands = 0;
     float *T_hi = nullptr, *T_lo = nullptr;      // band matrix transposed, [N][K], TF32 split
     float *bias_y = nullptr;             // [ld_in] bias of layer j-1 per neuron, y-major; null for j = 0
+    float *bias_out_y = nullptr;         // [ld_out] this layer's bias per output neuron, y-major
+    float *W_above_y = nullptr;          // the FC layer j+1's weights with their columns in y-major order, [pad(n)][ld_out]
+                                         // (a traversal that starts there writes its first matrix y-major at once)
     cert::TcMap b_hi, b_lo, a_hi[2], a_lo[2], o_hi[2], o_lo[2];
     cert::TcPlan plan;
 };
@@ -536,9 +539,33 @@ cert_status_t setup_band_tc(cert_net *net, const cert_layer_desc_t *descs) {
                      cert::tc_make_map(&S.o_lo[p], net->buf_lo[p], L.ld_in, rows_max, L.ld_in, 32);
         }
         if (!ok) break;
+        {
+            // y-major forms of what the start of a traversal at an FC layer right above needs
+            be.assign(L.ld_out, 0.0f);
+            for (int y = 0; y < L.h_out; ++y)
+                for (int co = 0; co < L.c_out; ++co)
+                    for (int x = 0; x < L.w_out; ++x) be[((size_t)y * L.c_out + co) * L.w_out + x] = descs[j].bias[co];
+            if (!dev_alloc(net, (void **)&S.bias_out_y, be.size() * sizeof(float))) return CERT_ERR_OOM;
+            if (cudaMemcpy(S.bias_out_y, be.data(), be.size() * sizeof(float), cudaMemcpyHostToDevice) != cudaSuccess)
+                return CERT_ERR_CUDA;
+            const LayerDev &La = net->layers[j + 1];
+            if (La.kind == CERT_LAYER_FC) {
+                const size_t rows_pad = round_up(La.n_out, kPad);
+                hi.assign(rows_pad * La.ld_in, 0.0f);
+                for (int i = 0; i < La.n_out; ++i)
+                    for (int y = 0; y < L.h_out; ++y)
+                        for (int co = 0; co < L.c_out; ++co)
+                            for (int x = 0; x < L.w_out; ++x)
+                                hi[(size_t)i * La.ld_in + ((size_t)y * L.c_out + co) * L.w_out + x] =
+                                    descs[j + 1].weight[(size_t)i * La.n_in + ((size_t)co * L.h_out + y) * L.w_out + x];
+                if (!dev_alloc(net, (void **)&S.W_above_y, hi.size() * sizeof(float))) return CERT_ERR_OOM;
+                if (cudaMemcpy(S.W_above_y, hi.data(), hi.size() * sizeof(float), cudaMemcpyHostToDevice) != cudaSuccess)
+                    return CERT_ERR_CUDA;
+            }
+        }
         S.usable = true;
         net->d_slots = std::max(net->d_slots, S.n_bands * S.plan.n_tiles);
-        net->gat_floats = std::max(net->gat_floats, (size_t)net->max_batch * L.ld_in);
+        net->gat_floats = std::max(net->gat_floats, (size_t)net->max_batch * std::max(L.ld_in, L.ld_out));
         net->band[j] = S;
     }
     return CERT_OK;
@@ -1009,10 +1036,29 @@ cert_status_t cert_backsub_bounds(cert_net_t *net, const float *centers, float e
             continue;
         }
         // expression over the outputs of layer k-1, pushed through its ReLU
-        cert::launch_init_expr(Lk, net->layers[k - 1], batch, net->buf[cur],
-                               wants_pair(k - 1) ? net->buf_lo[cur] : nullptr, net->dbuf[dcur], st);
-        rec.mark(CERT_CLASS_RELU_STEP);
         bool y_major = false;     // the coefficient maps are held [y][channel][x] (banded conv steps)
+        if (Lk.kind == CERT_LAYER_FC && on_band(k - 1) && net->band[k - 1].W_above_y) {
+            // an FC layer right above a banded conv layer: the same start with the columns of W_k, the relaxation
+            // and the bias below in y-major order writes the first matrix in the layout the banded steps read
+            const LayerDev &Lb = net->layers[k - 1];
+            const BandStep &S = net->band[k - 1];
+            const float *src[3] = {nullptr, nullptr, nullptr};
+            const float fill[3] = {1.0f, 1.0f, 0.0f};
+            if (Lb.relu_after) { src[0] = Lb.lamL; src[1] = Lb.lamU; src[2] = Lb.nuU; }
+            cert::launch_to_ymajor_vectors(Lb.c_out, Lb.h_out, Lb.w_out, Lb.ld_out, batch, 3, src, fill, net->gat, st);
+            rec.mark(CERT_CLASS_RELU_STEP);
+            LayerDev Lk_y = Lk, Lb_y = Lb;
+            Lk_y.W = S.W_above_y;
+            Lb_y.lamL = net->gat[0]; Lb_y.lamU = net->gat[1]; Lb_y.nuU = net->gat[2];
+            Lb_y.bias_n = S.bias_out_y;
+            Lb_y.relu_after = 1;
+            cert::launch_init_expr(Lk_y, Lb_y, batch, net->buf[cur], net->buf_lo[cur], net->dbuf[dcur], st);
+            y_major = true;
+        } else {
+            cert::launch_init_expr(Lk, net->layers[k - 1], batch, net->buf[cur],
+                                   wants_pair(k - 1) ? net->buf_lo[cur] : nullptr, net->dbuf[dcur], st);
+        }
+        rec.mark(CERT_CLASS_RELU_STEP);
         // Residual connections: the coefficients on a connection's source wait (kept: the buffer that holds
         // them, untouched meanwhile; identity: the unit coefficient of layer k's own connection) until the
         // step whose result is over that source's outputs, where they join before the ReLU back-step.
