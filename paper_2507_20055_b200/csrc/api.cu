@@ -971,8 +971,9 @@ cert_status_t cert_backsub_bounds(cert_net_t *net, const float *centers, float e
                 rec.mark(CERT_CLASS_CONV);
                 cert::TcArgs a;
                 std::memset(&a, 0, sizeof(a));
-                a.M = rows; a.K = S.Kp; a.n_k = Lk.n_out; a.ld_n = S.ldN;
-                a.n_pos = Lk.h_out * Lk.w_out;
+                // rows are ordered (box, position, side, channel): with "box" = (box, position) and c_out neurons
+                // per box this is the usual row order, and the gathered vectors are per such box
+                a.M = rows; a.K = S.Kp; a.n_k = Lk.c_out; a.ld_n = S.ldN;
                 a.bn = S.plan.bn; a.n_tiles = S.plan.n_tiles; a.stages = S.plan.stages;
                 a.tmem_cols = S.plan.tmem_cols;
                 a.total_tiles = (int)cert::ceil_div_ll(rows, 128 * ctas) * S.plan.n_tiles;
@@ -997,7 +998,7 @@ cert_status_t cert_backsub_bounds(cert_net_t *net, const float *centers, float e
                 dslots = S.plan.n_tiles;
             }
             cert::launch_relax(Lk, lb_out, ub_out, n_total, batch, net->codes, net->n_relu, net->dbuf[dcur], dslots,
-                               net->slot_stride, st);
+                               net->slot_stride, st, Lk.h_out * Lk.w_out);
             rec.mark(CERT_CLASS_RELAX);
             paths |= 8 | 2 | (ctas == 2 ? 4 : 0);
             continue;

@@ -86,9 +86,11 @@ void launch_first_layer_bounds(const LayerDev &L, const float *l0, const float *
 // With `slots` != nullptr the bounds are first summed from n_slots partial sums per row
 // (rows ordered (box, side, neuron), slot s at slots + s*slot_stride) and stored to lb_out / ub_out;
 // the relaxation itself is skipped for a layer without a ReLU.
+// slot_npos > 0: the slot rows are ordered (box, position, side, channel) for a conv layer with slot_npos
+// output positions (the order of the tensor-core patch steps) instead of (box, side, neuron).
 void launch_relax(const LayerDev &L, float *lb_out, float *ub_out, int n_total, int batch,
                   unsigned char *codes, int n_relu, const float *slots, int n_slots, long long slot_stride,
-                  cudaStream_t st);
+                  cudaStream_t st, int slot_npos = 0);
 
 // Start of the back-substitution for layer k: the expression of neuron i is
 // row i of W_k (the same for every box and both sides) and the constant b_k[i];
@@ -175,7 +177,8 @@ struct PatchLevel {
 bool conv_patch_plan(const LayerDev *layers, int k, int j_end, PatchLevel *levels, int max_levels);
 void conv_patch_prepare();
 // Start: the kernel of layer k as a patch over the outputs of the layer below, through that layer's ReLU.
-// `pitch` floats per row; patch_lo != nullptr: written as a TF32 pair for a tensor-core step.
+// `pitch` floats per row; patch_lo != nullptr: written as a TF32 pair for a tensor-core step, with the rows
+// ordered (box, position, side, channel) so that the rows of a tile share their position-dependent vectors.
 void launch_patch_start(const LayerDev &Lk, const LayerDev &Lb, int pitch, int batch, float *patch,
                         float *patch_lo, float *d, cudaStream_t st);
 // For the tensor-core form of a patch back-step (the conv layer as a dense matrix between windows, the

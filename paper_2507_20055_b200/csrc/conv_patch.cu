@@ -85,7 +85,9 @@ patch_start_kernel(const float *__restrict__ Wk, ConvGeom gk, const float *__res
     for (int rr = warp; rr < 2 * gk.c_out; rr += kWarpsPerBlock) {
         const int upper = rr / gk.c_out, co = rr - upper * gk.c_out;
         const int i = co * hw_o + pos;
-        const long long r = ((long long)box * 2 + upper) * n_k + i;
+        // tensor-core steps follow (patch_lo): rows ordered (box, position, side, channel); else (box, side, neuron)
+        const long long r = patch_lo ? (long long)blockIdx.x * 2 * gk.c_out + rr
+                                     : ((long long)box * 2 + upper) * n_k + i;
         const float *wrow = Wk + (size_t)co * taps;
         float dacc = 0.0f;
         for (int q0 = lane * 4; q0 < pitch; q0 += 128) {

@@ -214,7 +214,7 @@ __global__ void relax_kernel(float *__restrict__ lb_out, float *__restrict__ ub_
                              float *__restrict__ actL, float *__restrict__ actU,
                              unsigned char *__restrict__ codes, int n_relu, int relu_off,
                              const float *__restrict__ slots, int n_slots, long long slot_stride,
-                             int do_relax) {
+                             int slot_npos, int do_relax) {
     pdl_trigger();
     pdl_wait();
     long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
@@ -224,8 +224,15 @@ __global__ void relax_kernel(float *__restrict__ lb_out, float *__restrict__ ub_
     if (t < n) {
         float l, u;
         if (slots) {
-            l = slot_sum(slots, n_slots, slot_stride, (2LL * b) * n + t);
-            u = slot_sum(slots, n_slots, slot_stride, (2LL * b + 1) * n + t);
+            long long rl = (2LL * b) * n + t, ru = (2LL * b + 1) * n + t;
+            if (slot_npos > 0) {
+                // rows ordered (box, position, side, channel): the tensor-core patch steps of a conv layer
+                const int c = n / slot_npos, ch = t / slot_npos, pos = t - ch * slot_npos;
+                rl = (((long long)b * slot_npos + pos) * 2) * c + ch;
+                ru = rl + c;
+            }
+            l = slot_sum(slots, n_slots, slot_stride, rl);
+            u = slot_sum(slots, n_slots, slot_stride, ru);
             lb_out[(size_t)b * n_total + out_off + t] = l;
             ub_out[(size_t)b * n_total + out_off + t] = u;
         } else {
@@ -502,11 +509,11 @@ void launch_first_layer_bounds(const LayerDev &L, const float *l0, const float *
 
 void launch_relax(const LayerDev &L, float *lb_out, float *ub_out, int n_total, int batch,
                   unsigned char *codes, int n_relu, const float *slots, int n_slots, long long slot_stride,
-                  cudaStream_t st) {
+                  cudaStream_t st, int slot_npos) {
     long long n = (long long)batch * L.ld_out;
     launch_chained(relax_kernel, dim3((unsigned)ceil_div_ll(n, 256)), dim3(256), 0, st, lb_out, ub_out, n_total,
                    L.out_off, L.n_out, L.ld_out, batch, L.lamL, L.lamU, L.nuU, L.actL, L.actU, codes, n_relu, L.relu_off,
-                   slots, n_slots, slot_stride, L.relu_after);
+                   slots, n_slots, slot_stride, slot_npos, L.relu_after);
 }
 
 void launch_init_expr(const LayerDev &Lk, const LayerDev &Lb, int batch, float *Q, float *Q_lo, float *d,

@@ -235,10 +235,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_consta
             const long long rr = row_ok ? r : 0;
             const int b = (int)(rr / (2LL * a.n_k));
             const int upper = (int)((rr / a.n_k) & 1);
-            // the row's vector of the relaxation / box arrays: one per box, or (rows that are patches of
-            // a conv neuron's window) one per box and output position of the neuron
-            const size_t vec = a.n_pos ? (size_t)b * a.n_pos + (size_t)((rr % a.n_k) % a.n_pos) : (size_t)b;
-            const size_t relax_row = vec * a.ld_n;
+            const size_t relax_row = (size_t)b * a.ld_n;
             float dacc = 0.0f;
             const int acc = lt & 1;
             const uint32_t acc_phase = (lt >> 1) & 1;

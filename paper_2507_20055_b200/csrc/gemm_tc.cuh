@@ -36,9 +36,6 @@ struct TcArgs {
     int ld_n;        // padded width of the output (neurons below layer j)
     int bn, n_tiles, stages, tmem_cols;
     int total_tiles; // row panels x column tiles (a row panel is 128 rows per CTA of the group)
-    int n_pos;       // 0: the arrays below hold one vector per box.  > 0: the rows are receptive-field patches of
-                     // conv neurons with n_pos output positions; the arrays hold one vector per (box, position),
-                     // already gathered to the patch's window (zero outside the map)
     // Banded form of a conv back-step on dense coefficient maps (n_bands > 0).  Maps are held row-major by map
     // row ("y-major": [y][channel][x]), so the coefficients of `band_rin` consecutive rows of layer j's output map
     // are one contiguous K window of a row of A, and the `s` rows of the map below that depend on them are one
@@ -52,7 +49,7 @@ struct TcArgs {
     int band_s, band_y_shift, band_row_out;                        // band_row_out = channels * width of the map below
     int has_relu;    // a ReLU sits on the neurons below layer j
     int split_out;   // ReLU epilogue: store the result as a TF32 pair (a tensor-core step follows)
-    const float *lamL, *lamU, *nuU;              // [batch (* n_pos)][ld_n]
+    const float *lamL, *lamU, *nuU;              // [batch][ld_n] ("box" = whatever a group of 2 * n_k rows shares)
     const float *bias_below;                     // [ld_n] bias of the affine layer below (next step)
     // ReLU epilogue, residual connection ending on the neurons below layer j: coefficients added to the
     // product before the ReLU back-step: a matrix [rows][ld_n] (fp32, or a TF32 pair), and / or the unit
@@ -61,7 +58,7 @@ struct TcArgs {
     const float *add_hi, *add_lo;
     int add_identity;
     // concretisation epilogue
-    const float *l0, *u0;                        // [batch (* n_pos)][ld_n]
+    const float *l0, *u0;                        // [batch][ld_n]
     // Row constants travel in slots: the constant of row r so far is the sum over
     // s < n_slots_in of d_in[s*slot_stride + r]; this launch writes n_tiles slots to d_out
     // (slot 0 includes the sum of the input slots).  For the concretising epilogue the
