@@ -399,7 +399,8 @@ def main():
         used_fp16 = bool(net.last_contraction_paths() & 16)
         # fp16 split: three fp16 products (bf16 rate) per multiply-add; TF32 split: three TF32 products (half that rate)
         tc_peak = peaks["bf16_tflops_sustained"] * (1.0 if used_fp16 else 0.5) / 3.0
-        used_tc = dom == "affine" and bool(net.last_contraction_paths() & 2)
+        # conv back-steps: on the tensor cores when the dense steps ran in banded form (bit 6) beside the patch steps
+        used_tc = bool(net.last_contraction_paths() & 2) and (dom == "affine" or bool(net.last_contraction_paths() & 64))
         traffic, traffic_note = None, "no ncu capture for this workload / contraction mode"
         cap = NCU_TRAFFIC_BYTES_PER_ROW.get((w.name, "tc16" if used_fp16 else "tc"))
         if cap and used_tc and (net.last_contraction_paths() & 4) and not reuse and args.backsteps is None:
@@ -416,6 +417,8 @@ def main():
                 "flops_per_step_if_dense_maps": fl_dense[dom], "conv_rows_as_patches": used_patches,
                 "peak_source": peaks["source"],
                 "peak_note": (("bf16_tflops_sustained/3 (3xFP16)" if used_fp16 else "bf16_tflops_sustained/2/3 (3xTF32)")
+                              + ("; conv back-steps run as dense window / band contractions, counted here at their "
+                                 "algorithmic flops (the executed count is several times higher)" if dom == "conv" else "")
                               if used_tc else "148 SM x 128 FMA x 2 x sm_max_mhz" +
                               ("; the conv class also holds the patch back-step, which runs on the tensor cores "
                                "(gather + 3xTF32 contraction with the window-to-window matrix), counted at its "
