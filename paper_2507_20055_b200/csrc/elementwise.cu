@@ -323,9 +323,9 @@ __global__ void conv_expr_start_kernel(const float *__restrict__ Wk, ConvGeom gk
 // Start of a back-substitution at FC layer k: row i of W_k pushed through the ReLU below, constant =
 // b_k[i] + the nu terms + Q.b of the layer below.  A warp takes kStartRows consecutive neurons of one
 // (box, side), 4 columns per lane, so the relaxation and bias vectors are read once for those rows.
-// Q_lo != nullptr: the row is written as a TF32 pair.
-constexpr int kStartRows = 4;
-
+// Q_lo != nullptr: the row is written as a TF32 pair.  With few rows (a narrow layer over a wide one) a warp
+// takes one row, so that enough warps are in flight.
+template <int kStartRows>
 __global__ void fc_expr_start_kernel(const float *__restrict__ Wk, int ldw_k, const float *__restrict__ bias_k,
                                      float *__restrict__ Q, float *__restrict__ Q_lo, float *__restrict__ d,
                                      long long n_warps, int n_k, int n, int ld, int has_relu,
@@ -525,10 +525,16 @@ void launch_init_expr(const LayerDev &Lk, const LayerDev &Lb, int batch, float *
             Lb.nuU, Lb.bias_n);
         return;
     }
-    const long long n_warps = 2LL * batch * ((Lk.n_out + kStartRows - 1) / kStartRows);
-    launch_chained(fc_expr_start_kernel, dim3(grid_for_warps(n_warps)), dim3(kWarpsPerBlock * 32), 0, st, Lk.W, Lk.ld_in,
-                   Lk.bias_n, Q, Q_lo, d, n_warps, Lk.n_out, Lb.n_out, Lb.ld_out, Lb.relu_after, Lb.lamL, Lb.lamU, Lb.nuU,
-                   Lb.bias_n);
+    const long long warps4 = 2LL * batch * ((Lk.n_out + 3) / 4);
+    if (warps4 >= 148LL * 32) {
+        launch_chained(fc_expr_start_kernel<4>, dim3(grid_for_warps(warps4)), dim3(kWarpsPerBlock * 32), 0, st, Lk.W,
+                       Lk.ld_in, Lk.bias_n, Q, Q_lo, d, warps4, Lk.n_out, Lb.n_out, Lb.ld_out, Lb.relu_after, Lb.lamL,
+                       Lb.lamU, Lb.nuU, Lb.bias_n);
+    } else {
+        launch_chained(fc_expr_start_kernel<1>, dim3(grid_for_warps(rows)), dim3(kWarpsPerBlock * 32), 0, st, Lk.W,
+                       Lk.ld_in, Lk.bias_n, Q, Q_lo, d, rows, Lk.n_out, Lb.n_out, Lb.ld_out, Lb.relu_after, Lb.lamL,
+                       Lb.lamU, Lb.nuU, Lb.bias_n);
+    }
 }
 
 void launch_relu_step(const LayerDev &Lj, int batch, int n_k, float *P, float *P_lo, float *d, int n_slots,
