@@ -29,10 +29,10 @@ from paper_2507_20055_b200 import workloads as wl
 # of one launch of the ReLU-epilogue contraction, 16-box case, per row of the coefficient matrix; traffic
 # grows in proportion to the rows, so a full launch is rows x this figure).  None for workloads not captured.
 NCU_TRAFFIC_BYTES_PER_ROW = {
-    ("fc6x1024_b128", "tc"): {"bytes_per_row": (316.103168e6 + 217.877248e6) / 32768.0,
+    ("fc6x1024_b128", "tc"): {"bytes_per_row": (318.128896e6 + 218.081792e6) / 32768.0,
                               "kernel": "gemm_tc_kernel<TC_EPI_RELU, 2>",
                               "source": "profiles/gemm_tc_kernel_fc6x1024.md (16 boxes, scaled by rows)"},
-    ("fc6x1024_b128", "tc16"): {"bytes_per_row": (138.939392e6 + 96.243712e6) / 32768.0,
+    ("fc6x1024_b128", "tc16"): {"bytes_per_row": (139.057152e6 + 95.979264e6) / 32768.0,
                                 "kernel": "gemm_tc16_kernel<TC_EPI_RELU>",
                                 "source": "profiles/gemm_tc16_kernel_fc6x1024.md (16 boxes, scaled by rows)"},
 }
