@@ -233,6 +233,22 @@ def test_conv_rows_dense_and_patches(name, form):
     compare(run_gpu(w, conv_patches=patches, contraction=contraction, backsteps=steps), ref1, label=f"{name}/{form}/p1")
 
 
+def test_banded_conv_steps_ragged_batch_and_traversal_depths():
+    """Dense maps band by band on the tensor cores: fewer boxes than the net was made for, rows that do not fill the
+    last 256-row panel, traversals that stop on a conv layer's input map, and the FMA kernels as cross-check."""
+    w = wl.small_conv((2, 32, 32), [(4, 4, 2, 1), (8, 4, 2, 1)], [12, 4], batch=3, eps=0.01, seed=96)
+    K = len(w.layers)
+    for vname, steps in {"full": None, "p1": [1] * K, "p2": [2] * K, "crown_ibp": [0] * (K - 1) + [-1],
+                         "mixed": [0, 1, -1, 2]}.items():
+        ref = orc.deeppoly(w.layers, w.centers, w.eps, w.clip_lo, w.clip_hi, backsteps_per_layer=steps)
+        g = run_gpu(w, max_batch=w.batch + 2, backsteps=steps, conv_patches=False)
+        if vname in ("full", "p2", "crown_ibp"):
+            assert g["paths"] & 64, vname
+        compare(g, ref, label=f"banded/{vname}")
+        compare(run_gpu(w, max_batch=w.batch + 2, backsteps=steps, conv_patches=False, contraction=MODES["ffma"]), ref,
+                label=f"banded/{vname}/ffma cross-check")
+
+
 def test_conv_patches_on_tensor_cores_ragged_batch():
     """Fewer boxes than the net was made for, rows not a multiple of the 256-row panel."""
     w = wl.small_conv((2, 20, 18), [(4, 3, 1, 1), (6, 4, 2, 1), (8, 3, 2, 0)], [12, 3], batch=3, eps=0.01, seed=87)
