@@ -647,3 +647,33 @@ def test_call_is_capturable_in_a_cuda_graph(mode):
         compare(g, ref, label=f"graph replay/{mode}")
     finally:
         net.destroy()
+
+
+# ---- fixed summation order: two runs give the same bits ----
+
+@pytest.mark.parametrize("case", ["fc_tc", "fc_tc16", "fc_chain", "conv", "residual"])
+def test_results_are_bit_reproducible(case):
+    import torch
+    from paper_2507_20055_b200 import binding
+    if case == "conv":
+        w = wl.make_config(3, batch=6)
+    elif case == "residual":
+        w = wl.residual_fc(64, 300, 2, 10, batch=5, eps=0.01, seed=97)
+    elif case == "fc_chain":
+        w = wl.make_config(1, batch=16)
+    else:
+        w = wl.small_fc([200, 700, 700, 700, 10], batch=12, eps=0.01, seed=98)
+    net = binding.CertNet(w.layers, w.batch, w.clip_lo, w.clip_hi, skip_from=w.skip_from)
+    try:
+        net.set_contraction({"fc_tc": 2, "fc_tc16": 3, "fc_chain": 3, "conv": 0, "residual": 2}[case])
+        c = torch.from_numpy(w.centers).cuda()
+        runs = []
+        for _ in range(3):
+            lb, ub = net.deeppoly_bounds(c, w.eps)
+            torch.cuda.synchronize()
+            runs.append((lb.clone(), ub.clone()))
+        assert net.last_status() == 0
+        for lb, ub in runs[1:]:
+            assert torch.equal(lb, runs[0][0]) and torch.equal(ub, runs[0][1])
+    finally:
+        net.destroy()
