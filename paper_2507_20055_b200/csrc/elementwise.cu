@@ -480,6 +480,21 @@ inline unsigned grid_for_warps(long long warps) {
 
 }  // namespace
 
+// Multiprocessors of the current device (looked up once).
+static int sm_count() {
+    static int n = 0;
+    if (n == 0) {
+        int dev = 0, v = 0;
+        if (cudaGetDevice(&dev) == cudaSuccess &&
+            cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0)
+            n = v;
+        else
+            n = 148;
+        cudaGetLastError();
+    }
+    return n;
+}
+
 bool pdl_enabled() {
     static const bool on = [] {
         const char *e = std::getenv("CERT_PDL");
@@ -526,7 +541,7 @@ void launch_init_expr(const LayerDev &Lk, const LayerDev &Lb, int batch, float *
         return;
     }
     const long long warps4 = 2LL * batch * ((Lk.n_out + 3) / 4);
-    if (warps4 >= 148LL * 32) {
+    if (warps4 >= 32LL * sm_count()) {          // enough four-row warps to fill the multiprocessors
         launch_chained(fc_expr_start_kernel<4>, dim3(grid_for_warps(warps4)), dim3(kWarpsPerBlock * 32), 0, st, Lk.W,
                        Lk.ld_in, Lk.bias_n, Q, Q_lo, d, warps4, Lk.n_out, Lb.n_out, Lb.ld_out, Lb.relu_after, Lb.lamL,
                        Lb.lamU, Lb.nuU, Lb.bias_n);
