@@ -232,6 +232,11 @@ int cert_net_last_contraction_paths(const cert_net_t *net);
  * the rows travel as [channels][window] patches instead of dense coefficient maps.  Off: every
  * back-step works on dense maps.  The bounds are the same up to summation order.
  * cert_net_last_contraction_paths sets bit 3 when a traversal of the last call ran on patches.
+ * Unless the contraction mode is CERT_CONTRACTION_FFMA, both kinds of conv back-step run on the tensor
+ * cores where their geometry allows: a patch step as a contraction with the conv layer's dense
+ * window-to-window matrix (bit 1 beside bit 3), a step on dense maps band by band with the maps held
+ * [row][channel][column] (bit 6; needs channels x width a multiple of 32 floats on both sides of the layer
+ * and of every conv layer below it).  Other geometries use the FMA kernels.
  */
 cert_status_t cert_net_set_conv_patches(cert_net_t *net, int on);
 
