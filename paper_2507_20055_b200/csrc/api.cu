@@ -113,7 +113,7 @@ struct cert_net {
     // fp16-split path, narrow nets: a whole traversal per launch with the coefficient panel kept in shared memory
     bool chain_ok = false;
     cert::ChainParams chain;
-    int chain_a_blocks = 0, chain_stages = 0, chain_smem = 0;
+    int chain_a_blocks = 0, chain_stages = 0, chain_smem = 0, chain_chunk = 0, chain_vec_ld = 0;
     float *dbuf[2] = {nullptr, nullptr};     // row constants, [d_slots][slot_stride] each, ping-pong
     int d_slots = 1;                         // slots per buffer (most column tiles of any contraction)
     long long slot_stride = 0;               // rows of the largest coefficient matrix
@@ -335,7 +335,10 @@ cert_status_t setup_tensor_core_path(cert_net *net, const cert_layer_desc_t *des
         for (int j = 0; j + 1 < K; ++j) widest = std::max(widest, net->layers[j].n_out);
         if (chain && widest <= cert::kChainMaxWidth) {
             net->chain_a_blocks = (widest + 63) / 64;
-            net->chain_smem = cert::chain16_smem_bytes(net->chain_a_blocks, &net->chain_stages);
+            int max_bnl = 0;
+            for (int j = 0; j + 1 < K; ++j) max_bnl = std::max(max_bnl, net->tc16[j].plan.bn / 2);
+            net->chain_smem = cert::chain16_smem_bytes(net->chain_a_blocks, max_bnl, round_up(widest, kPad),
+                                                       &net->chain_stages, &net->chain_chunk, &net->chain_vec_ld);
             std::memset(&net->chain, 0, sizeof(net->chain));
             for (int j = 0; j < K; ++j) {
                 const LayerDev &L = net->layers[j];
@@ -872,6 +875,7 @@ cert_status_t cert_backsub_bounds(cert_net_t *net, const float *centers, float e
             a.d_out = net->dbuf[0]; a.slot_stride = net->slot_stride;
             a.status = net->status_dev;
             a.stages = net->chain_stages; a.a_blocks = net->chain_a_blocks;
+            a.b_chunk_bytes = net->chain_chunk; a.vec_ld = net->chain_vec_ld;
             const int pairs = (int)std::min<long long>(cert::ceil_div_ll(rows, 256), net->sm_count / 2);
             cert::launch_chain16(net->chain, a, pairs, net->chain_smem, st);
             rec.mark(CERT_CLASS_AFFINE);

@@ -35,8 +35,6 @@ constexpr int BKH = 64;                          // halves of K per block: one 1
 constexpr int kEpiWarps = 4 * kChainColGroups;   // kChainColGroups warps per TMEM lane quarter
 constexpr int kThreadsChain = 64 + kEpiWarps * 32;
 constexpr int kABlockBytes = BM * BKH * 2;       // one 64-column block of the panel (hi or lo): 16 KiB
-constexpr int kBChunkBytes = 128 * BKH * 2;      // this CTA's share of a W_j tile for one k-block (at most 128 rows)
-constexpr int kStageBytes = 2 * kBChunkBytes;
 constexpr int kAccCols = 256;                    // tensor-memory columns per accumulator
 constexpr int CTAS = 2;
 
@@ -46,6 +44,8 @@ struct __align__(8) BarriersChain {
     uint64_t acc_full[2];
     uint64_t acc_empty[2];
     uint64_t a_ready;           // the panel in shared memory is complete (both CTAs' epilogue warps arrive)
+    uint64_t vec_full[2];       // a step's relaxation / bias vectors have landed in staging buffer 0 / 1
+    uint64_t vec_empty[2];      // ... and every epilogue warp is done reading them
     uint32_t tmem_base;
     uint32_t abort_flag;
 };
@@ -69,6 +69,13 @@ __device__ __forceinline__ bool mbar_wait_cluster(uint64_t *bar, uint32_t parity
         if ((unsigned long long)(clock64() - t0) > kWaitCycles) return false;
     }
     return true;
+}
+
+// Plain (untiled) bulk copy global -> this CTA's shared memory; both addresses 16-byte aligned, size a multiple of 16.
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
+                 : "memory");
 }
 
 // Writes 32 consecutive columns [c0, c0+32) of panel row `row` as an fp16 pair into the K-major,
@@ -110,7 +117,11 @@ chain16_kernel(const __grid_constant__ ChainParams P, const ChainArgs a) {
     uint8_t *A_lo = smem + (size_t)a.a_blocks * kABlockBytes;
     uint8_t *Bst = smem + 2 * (size_t)a.a_blocks * kABlockBytes;
     const int stages = a.stages;
-    BarriersChain *bars = reinterpret_cast<BarriersChain *>(Bst + (size_t)stages * kStageBytes);
+    const int kBChunkBytes = a.b_chunk_bytes, kStageBytes = 2 * a.b_chunk_bytes;
+    float *vec_stage = reinterpret_cast<float *>(Bst + (size_t)stages * kStageBytes);
+    const int vec_floats = 7 * a.vec_ld;
+    BarriersChain *bars = reinterpret_cast<BarriersChain *>(reinterpret_cast<uint8_t *>(vec_stage) +
+                                                            2 * (size_t)vec_floats * sizeof(float));
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = cluster_ctarank();
@@ -128,6 +139,10 @@ chain16_kernel(const __grid_constant__ ChainParams P, const ChainArgs a) {
             mbar_init(&bars->acc_empty[i], kEpiWarps * CTAS);
         }
         mbar_init(&bars->a_ready, kEpiWarps * CTAS);
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(&bars->vec_full[i], 1);
+            mbar_init(&bars->vec_empty[i], kEpiWarps);
+        }
         bars->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -154,9 +169,37 @@ chain16_kernel(const __grid_constant__ ChainParams P, const ChainArgs a) {
             uint32_t phase = 0;
             bool ok = true;
             int armed = 0;
+            int vstep = 0;      // steps whose vectors were staged so far (buffer = vstep & 1)
             for (long long p = group; p < n_panels && ok; p += n_groups) {
+                // boxes of this CTA's 128 rows: the first two are staged
+                const long long row0 = p * (BM * CTAS) + (long long)rank * BM;
+                const long long last_row = (row0 + BM - 1 < a.M ? row0 + BM - 1 : a.M - 1);
+                const int b_last = (int)(last_row / (2LL * a.n_k));
+                int b_first = (int)(row0 / (2LL * a.n_k));
+                if (b_first > b_last) b_first = b_last;
+                const int nb = b_last - b_first + 1 < 2 ? b_last - b_first + 1 : 2;
                 for (int j = a.k - 1; j >= a.j_end && ok; --j) {
                     const ChainLayer &L = P.layer[j];
+                    if (a.vec_ld > 0 && j > a.j_end) {
+                        // the vectors the epilogue of this step reads: bias of the layer below, then per box lamL, lamU, nuU
+                        const int buf = vstep & 1;
+                        if (!mbar_wait(&bars->vec_empty[buf], ((vstep >> 1) & 1) ^ 1) || *abort_flag) { ok = false; break; }
+                        float *dst = vec_stage + (size_t)buf * vec_floats;
+                        const uint32_t bytes = (uint32_t)L.ld_in * sizeof(float);
+                        const uint32_t n_copies = 1u + (L.relu_below ? 3u * (uint32_t)nb : 0u);
+                        mbar_arrive_expect_tx(&bars->vec_full[buf], n_copies * bytes);
+                        const uint32_t vbar = smem_u32(&bars->vec_full[buf]);
+                        bulk_load(smem_u32(dst), L.bias_below, bytes, vbar);
+                        if (L.relu_below)
+                            for (int q = 0; q < nb; ++q) {
+                                const size_t off = (size_t)(b_first + q) * L.ld_in;
+                                float *d3 = dst + a.vec_ld + (size_t)q * 3 * a.vec_ld;
+                                bulk_load(smem_u32(d3), L.lamL + off, bytes, vbar);
+                                bulk_load(smem_u32(d3 + a.vec_ld), L.lamU + off, bytes, vbar);
+                                bulk_load(smem_u32(d3 + 2 * a.vec_ld), L.nuU + off, bytes, vbar);
+                            }
+                        ++vstep;
+                    }
                     const CUtensorMap *mh = reinterpret_cast<const CUtensorMap *>(&P.b_hi[j]);
                     const CUtensorMap *ml = reinterpret_cast<const CUtensorMap *>(&P.b_lo[j]);
                     const int num_kb = (L.n_out + BKH - 1) / BKH;
@@ -288,7 +331,7 @@ chain16_kernel(const __grid_constant__ ChainParams P, const ChainArgs a) {
         const uint32_t acc_empty_addr0 = map_to_cta(smem_u32(&bars->acc_empty[0]), 0);
         const uint32_t a_ready_addr = map_to_cta(smem_u32(&bars->a_ready), 0);
         bool ok = true, out_of_range = false;
-        int lt = 0;
+        int lt = 0, vstep = 0;
         for (long long p = group; p < n_panels && ok; p += n_groups) {
             const long long r = p * (BM * CTAS) + (long long)rank * BM + prow;
             const bool row_ok = r < a.M;
@@ -347,6 +390,13 @@ chain16_kernel(const __grid_constant__ ChainParams P, const ChainArgs a) {
                 __syncwarp();
                 if (lane == 0) mbar_arrive_cluster(a_ready_addr);
             }
+            // boxes of this CTA's 128 rows (the producer stages the vectors of the first two)
+            const long long cta_row0 = p * (BM * CTAS) + (long long)rank * BM;
+            const long long cta_last = (cta_row0 + BM - 1 < a.M ? cta_row0 + BM - 1 : a.M - 1);
+            const int b_last = (int)(cta_last / (2LL * a.n_k));
+            int b_first = (int)(cta_row0 / (2LL * a.n_k));
+            if (b_first > b_last) b_first = b_last;
+            const int nb = b_last - b_first + 1 < 2 ? b_last - b_first + 1 : 2;
             for (int j = a.k - 1; j >= a.j_end && ok; --j) {
                 const ChainLayer &L = P.layer[j];
                 const bool last = (j == a.j_end);
@@ -355,10 +405,24 @@ chain16_kernel(const __grid_constant__ ChainParams P, const ChainArgs a) {
                 const int ld_in = L.ld_in, n_in = L.n_in, bn = L.bn, n_tiles = L.n_tiles, relu_below = L.relu_below;
                 const float *lamL = L.lamL + relax_row, *lamU = L.lamU + relax_row, *nuU = L.nuU + relax_row;
                 const float *bias_below = L.bias_below;
+                // staged copies of these vectors (the producer fetched them while the MMAs ran): the bias always,
+                // the relaxation for rows of the CTA's first two boxes
+                const int vbuf = (a.vec_ld > 0 && !last) ? (vstep & 1) : -1;
+                if (vbuf >= 0) {
+                    const float *vs = vec_stage + (size_t)vbuf * vec_floats;
+                    bias_below = vs;
+                    const int sb = b - b_first;
+                    if (sb >= 0 && sb < nb) {
+                        lamL = vs + a.vec_ld + (size_t)sb * 3 * a.vec_ld;
+                        lamU = lamL + a.vec_ld;
+                        nuU = lamU + a.vec_ld;
+                    }
+                }
                 for (int nt = 0; nt < n_tiles && ok; ++nt, ++lt) {
                     const int acc = lt & 1;
                     const uint32_t acc_phase = (lt >> 1) & 1;
                     if (!mbar_wait(&bars->acc_full[acc], acc_phase) || *abort_flag) { ok = false; break; }
+                    if (vbuf >= 0 && (!mbar_wait(&bars->vec_full[vbuf], (vstep >> 1) & 1) || *abort_flag)) { ok = false; break; }
                     tcgen05_fence_after();
                     const uint32_t t_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * kAccCols);
                     if (!last) {
@@ -410,6 +474,7 @@ chain16_kernel(const __grid_constant__ ChainParams P, const ChainArgs a) {
                         if (lane == 0) {
                             mbar_arrive_cluster(acc_empty_addr0 + (uint32_t)(acc * sizeof(uint64_t)));
                             mbar_arrive_cluster(a_ready_addr);
+                            if (vbuf >= 0) mbar_arrive_cluster(map_to_cta(smem_u32(&bars->vec_empty[vbuf]), rank));
                         }
                     } else {
                         // map(simplify_lower/upper) against the concrete bounds of what the traversal reached
@@ -440,6 +505,7 @@ chain16_kernel(const __grid_constant__ ChainParams P, const ChainArgs a) {
                         if (lane == 0) mbar_arrive_cluster(acc_empty_addr0 + (uint32_t)(acc * sizeof(uint64_t)));
                     }
                 }
+                if (vbuf >= 0) ++vstep;
             }
             if (ok && row_ok) a.d_out[(size_t)col_group * a.slot_stride + r] = dacc;
         }
@@ -463,12 +529,22 @@ chain16_kernel(const __grid_constant__ ChainParams P, const ChainArgs a) {
 
 }  // namespace
 
-int chain16_smem_bytes(int a_blocks, int *stages) {
+int chain16_smem_bytes(int a_blocks, int max_bnl, int ld_max, int *stages, int *b_chunk_bytes, int *vec_ld) {
+    const int chunk = (max_bnl * BKH * 2 + 1023) / 1024 * 1024;
+    const int stage = 2 * chunk;
     const int fixed = 2 * a_blocks * kABlockBytes + (int)sizeof(BarriersChain) + 1024;
-    int st = (kTcSmemMax - fixed) / kStageBytes;
+    const int vec_bytes = 2 * 7 * ld_max * (int)sizeof(float);
+    *b_chunk_bytes = chunk;
+    // the staging buffers are taken if three pipeline stages still fit beside them
+    int st = (kTcSmemMax - fixed - vec_bytes) / stage;
+    *vec_ld = ld_max;
+    if (st < 3) {
+        st = (kTcSmemMax - fixed) / stage;
+        *vec_ld = 0;
+    }
     if (st > 8) st = 8;
     *stages = st;
-    return fixed + (st > 0 ? st : 0) * kStageBytes;
+    return fixed + (*vec_ld ? vec_bytes : 0) + (st > 0 ? st : 0) * stage;
 }
 
 bool chain16_prepare() {

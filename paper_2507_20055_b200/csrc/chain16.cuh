@@ -40,11 +40,16 @@ struct ChainArgs {
     int *status;                        // bit 0: a bounded wait ran out, bit 1: a coefficient left the fp16 range
     int stages;                         // pipeline stages of W_j tiles
     int a_blocks;                       // 64-column blocks of the coefficient panel held in shared memory
+    int b_chunk_bytes;                  // room for one CTA's share of a W_j tile k-block (a multiple of 1024)
+    int vec_ld;                         // > 0: the relaxation and bias vectors of a step are staged in shared memory
+                                        // (two buffers of 7 * vec_ld floats: bias, then lamL, lamU, nuU of two boxes)
 };
 
 bool chain16_prepare();
 // Shared memory the kernel needs for `a_blocks`; *stages receives the pipeline depth (< 2: does not fit).
-int chain16_smem_bytes(int a_blocks, int *stages);
+// `max_bnl` = most rows of a W_j tile a CTA stages, `ld_max` = widest padded hidden layer; *vec_ld receives ld_max
+// if the staging buffers fit beside three pipeline stages, else 0.
+int chain16_smem_bytes(int a_blocks, int max_bnl, int ld_max, int *stages, int *b_chunk_bytes, int *vec_ld);
 void launch_chain16(const ChainParams &P, const ChainArgs &a, int pairs, int smem_bytes, cudaStream_t st);
 
 }  // namespace cert
