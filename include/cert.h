@@ -209,6 +209,9 @@ cert_status_t cert_net_selftest_bounded_wait(cert_net_t *net, void *stream);
  *            CERT_ERR_RANGE and the results are invalid; values under 6.1e-5 are held to 1.5e-11
  *            absolute instead of 2^-22 relative).  Never chosen by AUTO.
  * Conv back-steps always run on the FMA units, with the same fusions.
+ * (The kernels of a call are chained with programmatic dependent launch, so that a kernel's launch and set-up
+ * overlap the tail of the one before; the environment variable CERT_PDL=0, read once per process, turns
+ * that off.)
  * (The environment variable CERT_TC_CTAS=1, read at create, keeps the
  * tensor-core kernel to one CTA per row panel instead of CTA pairs.)
  */
