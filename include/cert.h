@@ -208,7 +208,8 @@ cert_status_t cert_net_selftest_bounded_wait(cert_net_t *net, void *stream);
  *            coefficients below 65504 in magnitude (beyond that cert_net_last_status reports
  *            CERT_ERR_RANGE and the results are invalid; values under 6.1e-5 are held to 1.5e-11
  *            absolute instead of 2^-22 relative).  Never chosen by AUTO.
- * Conv back-steps always run on the FMA units, with the same fusions.
+ * Conv back-steps have the same fusions; under FFMA they run on the FMA units, otherwise on the TF32 tensor-core
+ * kernel where their geometry allows (see cert_net_set_conv_patches).
  * (The kernels of a call are chained with programmatic dependent launch, so that a kernel's launch and set-up
  * overlap the tail of the one before; the environment variable CERT_PDL=0, read once per process, turns
  * that off.)
