@@ -424,6 +424,11 @@ def main():
                                "(gather + 3xTF32 contraction with the window-to-window matrix), counted at its "
                                "algorithmic flops" if used_patches and args.contraction != "ffma" else "")),
                 "class_ms_per_step": {k: v / args.steps for k, v in cls_ms.items()}}
+        # branch statistics of the last call (Relu transformer): the share of ReLU neurons relaxed as unstable
+        torch.cuda.synchronize()
+        codes = net.branch_codes(B)
+        torch.cuda.synchronize()
+        unstable = float((codes >= 2).float().mean().item()) if codes.numel() else 0.0
         out = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": total_ms_max / args.steps, "higher_is_better": True,
@@ -435,6 +440,7 @@ def main():
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(B * net.n0 * 4),
                     "d2h_bytes_per_step": int(2 * B * net.n_total * 4), "steps": e2e_steps},
             "gpu_launches": launches, "wall_s_timed_region": t_wall, "roofline": roof, "clocks": clocks,
+            "unstable_fraction": unstable,
         }
         if tf32_ref is not None:
             out["tf32_split"] = tf32_ref
