@@ -677,3 +677,29 @@ def test_results_are_bit_reproducible(case):
             assert torch.equal(lb, runs[0][0]) and torch.equal(ub, runs[0][1])
     finally:
         net.destroy()
+
+
+@pytest.mark.parametrize("block", range(4))
+def test_random_nets_with_random_traversal_depths(block):
+    """Five FC, three conv and three residual nets per block, every contraction mode that takes them, one random
+    traversal depth per affine layer."""
+    rng = np.random.default_rng(4000 + block)
+    cases = [("fc", _random_fc(30 + 5 * block + i)) for i in range(5)] + \
+            [("conv", _random_conv(30 + 3 * block + i)) for i in range(3)]
+    for i in range(3):
+        r = np.random.default_rng(700 + 3 * block + i)
+        cases.append(("res", wl.residual_fc(int(r.integers(5, 60)), int(r.integers(8, 300)), int(r.integers(1, 4)),
+                                            int(r.integers(1, 9)), batch=int(r.integers(1, 5)), eps=0.02,
+                                            seed=800 + 3 * block + i)))
+    for kind, w in cases:
+        K = len(w.layers)
+        steps = [int(x) for x in rng.integers(-1, K, size=K)]
+        ref = orc.deeppoly(w.layers, w.centers, w.eps, w.clip_lo, w.clip_hi, skip_from=w.skip_from,
+                           backsteps_per_layer=steps)
+        good = ref["margins"].min(axis=1) >= 1e-5 if ref["margins"].shape[1] else np.ones(w.batch, bool)
+        if good.mean() < 0.5:
+            continue                      # ill-conditioned branch decisions: not a parity case
+        modes = {"fc": (1, 2, 3), "conv": (1, None), "res": (1, 2)}[kind]
+        for c in modes:
+            g = run_gpu(w, contraction=c, backsteps=steps, max_batch=w.batch + block % 2)
+            compare(g, ref, label=f"{kind}/{w.name}/mode {c}/depths {steps}")
