@@ -177,7 +177,7 @@ def run_reference(args, w):
     from oracle import deeppoly_oracle as orc
     orc.build()
     cores = orc.max_threads()
-    per = {0: 1, 1: 4 * cores, 2: 2 * cores, 3: cores, 4: cores, 5: 2 * cores}
+    per = {0: 1, 1: 4 * cores, 2: 2 * cores, 3: cores, 4: cores, 5: 2 * cores, 6: cores}
     n_boxes = min(w.batch, args.ref_boxes or per[args.config])
     if args.config == 4 and not args.ref_boxes:
         n_boxes = max(1, min(cores, 16) // 2)     # about 11 s per box per core
@@ -208,7 +208,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", type=int, default=4,
                     help="0..4: index into the benchmark configurations; 5: a fully connected residual net in the "
-                         "shape of the paper's 'Skip' network (784 -> 512 x 5 -> 10, two blocks, 64 boxes)")
+                         "shape of the paper's 'Skip' network (784 -> 512 x 5 -> 10, two blocks, 64 boxes); 6: a residual "
+                         "conv net (3x32x32 -> conv16 s2 -> two blocks of two 3x3 convs -> 10, 16 boxes)")
     ap.add_argument("--batch", type=int, default=None)
     ap.add_argument("--contraction", default="fastest", choices=["fastest", "auto", "ffma", "tc", "tc16"],
                     help="tc = tcgen05 3xTF32, tc16 = tcgen05 fp16 split (FC nets), ffma = FMA units, auto = the "
@@ -221,6 +222,8 @@ def main():
 
     if args.config == 5:
         w = wl.residual_fc(784, 512, 2, 10, batch=args.batch or 64, eps=0.01, seed=0)
+    elif args.config == 6:
+        w = wl.residual_conv((3, 32, 32), 16, 2, 10, batch=args.batch or 16, eps=2.0 / 255.0, seed=0)
     else:
         w = wl.make_config(args.config, batch=args.batch)
     args.backsteps = certifier_steps(args.certifier, len(w.layers))
@@ -445,7 +448,7 @@ def main():
         if tf32_ref is not None:
             out["tf32_split"] = tf32_ref
         if world == 1 and not args.no_cpu_baseline:
-            n_boxes = {0: 1, 1: 64, 2: 32, 3: 16, 4: 16, 5: 32}[args.config]
+            n_boxes = {0: 1, 1: 64, 2: 32, 3: 16, 4: 16, 5: 32, 6: 16}[args.config]
             from oracle import deeppoly_oracle as orc
             orc.build()
             n_boxes = min(n_boxes, B) if args.config != 4 else min(B, orc.max_threads(), 16)
