@@ -81,7 +81,9 @@ cert_status_t cert_net_create(const cert_layer_desc_t *layers, int n_layers, int
  * Requirements (else CERT_ERR_INVALID_ARG): s <= k-2; layers s and k have the same number of neurons;
  * connections follow one another (none starts before the previous one has ended).
  * Such a net is bounded with one launch per back-step and dense coefficient maps (patches and
- * cert_net_enable_reusecert are refused).  cert_backsub_bounds works as for other nets: a traversal that
+ * cert_net_enable_reusecert are refused; the banded tensor-core form of conv steps is used on full
+ * traversals when every connection ends on a conv layer that takes it and whose map has the shape of its
+ * source's).  cert_backsub_bounds works as for other nets: a traversal that
  * stops on a connection's source joins the waiting coefficients before it is simplified, one that stops
  * above it simplifies them against the source's own concrete bounds (map(simplify_*) treats every neuron left
  * in the expression alike).  CERT_CONTRACTION_TC3XFP16 is available for FC nets, for full traversals only

@@ -62,7 +62,7 @@ struct BandStep {
     float *bias_out_y = nullptr;         // [ld_out] this layer's bias per output neuron, y-major
     float *W_above_y = nullptr;          // the FC layer j+1's weights with their columns in y-major order, [pad(n)][ld_out]
                                          // (a traversal that starts there writes its first matrix y-major at once)
-    cert::TcMap b_hi, b_lo, a_hi[2], a_lo[2], o_hi[2], o_lo[2];
+    cert::TcMap b_hi, b_lo, a_hi[3], a_lo[3], o_hi[3], o_lo[3];   // one per coefficient buffer
     cert::TcPlan plan;
 };
 
@@ -124,6 +124,7 @@ struct cert_net {
     float *gat[3] = {nullptr, nullptr, nullptr}; // gathered windows, [max_batch * positions][ldN] each (y-major vectors for the banded form)
     size_t gat_floats = 0;
     std::vector<BandStep> band;                  // [j]: banded tensor-core form of the step through conv layer j
+    bool band_residual_ok = true;                // every layer a residual connection ends on takes the banded form
     ReuseState reuse;
     unsigned char *codes = nullptr;          // [max_batch][n_relu]
     int *status_dev = nullptr;               // sticky device status word
@@ -446,13 +447,14 @@ cert_status_t setup_patch_tc(cert_net *net, const cert_layer_desc_t *descs) {
 
 // Banded form of the dense conv back-steps, from the first layer upward while map rows are whole k-blocks
 // (channels * width a multiple of 32 on both sides) and the dense band matrix does at most kBandDenseRatio
-// times the multiply-adds of the convolution itself.
-constexpr int kBandDenseRatio = 12;
+// times the multiply-adds of the convolution itself (the split contraction runs about twenty times the rate the
+// FMA kernels reach on these steps; 3 x 3 stride-2 first layers on 3-channel inputs come to 15).
+constexpr int kBandDenseRatio = 16;
 
 cert_status_t setup_band_tc(cert_net *net, const cert_layer_desc_t *descs) {
     const int K = net->n_layers;
     net->band.assign(K, BandStep());
-    if (!net->tc_ok || !net->skip_from.empty()) return CERT_OK;
+    if (!net->tc_ok) return CERT_OK;
     if (const char *e = std::getenv("CERT_CONV_BANDS")) {
         if (std::atoi(e) == 0) return CERT_OK;
     }
@@ -534,7 +536,7 @@ cert_status_t setup_band_tc(cert_net *net, const cert_layer_desc_t *descs) {
         for (int k = j + 1; k < K; ++k) rows_max = std::max(rows_max, 2LL * net->max_batch * net->layers[k].n_out);
         bool ok = cert::tc_make_map(&S.b_hi, S.T_hi, S.K, S.N, S.K, S.plan.bn / ctas) &&
                   cert::tc_make_map(&S.b_lo, S.T_lo, S.K, S.N, S.K, S.plan.bn / ctas);
-        for (int p = 0; p < 2 && ok; ++p) {
+        for (int p = 0; p < net->n_buf && ok; ++p) {
             ok = cert::tc_make_map(&S.a_hi[p], net->buf[p], L.n_out, rows_max, L.ld_out, 128) &&
                  cert::tc_make_map(&S.a_lo[p], net->buf_lo[p], L.n_out, rows_max, L.ld_out, 128);
             if (ok && j > 0)
@@ -570,6 +572,15 @@ cert_status_t setup_band_tc(cert_net *net, const cert_layer_desc_t *descs) {
         net->d_slots = std::max(net->d_slots, S.n_bands * S.plan.n_tiles);
         net->gat_floats = std::max(net->gat_floats, (size_t)net->max_batch * std::max(L.ld_in, L.ld_out));
         net->band[j] = S;
+    }
+    // Nets with residual connections: a waiting matrix must be in the layout of the step it joins, which holds
+    // when every layer a connection ends on is itself banded (its matrix is then y-major when it is set aside).
+    for (int k = 0; k < K && !net->skip_from.empty(); ++k) {
+        if (net->skip_from[k] < 0) continue;
+        const LayerDev &D = net->layers[k], &S = net->layers[net->skip_from[k]];
+        if (!net->band[k].usable || S.kind != CERT_LAYER_CONV2D || S.c_out != D.c_out || S.h_out != D.h_out ||
+            S.w_out != D.w_out)
+            net->band_residual_ok = false;            // (the two maps must share one y-major order)
     }
     return CERT_OK;
 }
@@ -861,7 +872,8 @@ cert_status_t cert_backsub_bounds(cert_net_t *net, const float *centers, float e
         };
         // ... or, for a conv layer on dense maps, in the banded tensor-core form?  Its input is a TF32 pair too.
         auto on_band = [&](int j) {
-            return net->contraction != CERT_CONTRACTION_FFMA && net->tc_ok && net->band[j].usable;
+            return net->contraction != CERT_CONTRACTION_FFMA && net->tc_ok && net->band[j].usable &&
+                   (!residual || (net->band_residual_ok && steps == k));      // (residual nets: full traversals)
         };
         auto wants_pair = [&](int j) { return on_tc(j) || on_band(j); };
         // fp16-split tensor-core chain (FC nets): start, then one kernel per layer with the ReLU step fused,
@@ -1105,8 +1117,13 @@ cert_status_t cert_backsub_bounds(cert_net_t *net, const float *centers, float e
                     cert::launch_to_ymajor_pair(net->buf[cur], net->buf_lo[cur], net->buf[nxt], net->buf_lo[nxt], rows,
                                                 Lj.c_out, Lj.h_out, Lj.w_out, Lj.ld_out, st);
                     rec.mark(CERT_CLASS_CONV);
+                    if (kept == cur) kept = nxt;      // a matrix set aside at this very layer: its y-major copy waits
                     cur = nxt;
                     nxt = cur ^ 1;
+                    if (residual) {
+                        nxt = 0;
+                        while (nxt == cur || nxt == kept) ++nxt;
+                    }
                     y_major = true;
                 }
                 const float *src[3] = {nullptr, nullptr, nullptr};
@@ -1138,8 +1155,12 @@ cert_status_t cert_backsub_bounds(cert_net_t *net, const float *centers, float e
                     a.has_relu = 1;
                     a.split_out = 1;          // a banded step follows
                     a.lamL = net->gat[0]; a.lamU = net->gat[1]; a.nuU = net->gat[2]; a.bias_below = S.bias_y;
+                    if (join && kept >= 0) { a.add_hi = net->buf[kept]; a.add_lo = net->buf_lo[kept]; }
+                    a.add_identity = add_identity;
+                    a.band_c_out = Lj.c_in; a.band_h_out = Lj.h_in; a.band_w_out = Lj.w_in;
                     cert::launch_gemm_tc(cert::TC_EPI_RELU_BAND, ctas, groups, S.a_hi[cur], S.a_lo[cur], S.b_hi, S.b_lo,
                                          S.o_hi[nxt], S.o_lo[nxt], a, S.plan.smem_bytes, st);
+                    if (join) { wait_for = -1; wait_identity = false; kept = -1; }
                 } else {
                     a.l0 = net->gat[0]; a.u0 = net->gat[1];
                     cert::launch_gemm_tc(cert::TC_EPI_CONCRETIZE_BAND, ctas, groups, S.a_hi[cur], S.a_lo[cur], S.b_hi,

@@ -57,8 +57,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_consta
                const __grid_constant__ CUtensorMap map_b_hi, const __grid_constant__ CUtensorMap map_b_lo,
                const __grid_constant__ CUtensorMap map_o_hi, const __grid_constant__ CUtensorMap map_o_lo,
                const TcArgs a) {
-    constexpr bool kBand = (EPI == TC_EPI_RELU_BAND || EPI == TC_EPI_CONCRETIZE_BAND);
-    constexpr bool kRelu = (EPI == TC_EPI_RELU || EPI == TC_EPI_RELU_SKIP || EPI == TC_EPI_RELU_BAND);
+    constexpr bool kBand = (EPI == TC_EPI_RELU_BAND || EPI == TC_EPI_CONCRETIZE_BAND || EPI == TC_EPI_RELU_BAND_SKIP);
+    constexpr bool kRelu = (EPI == TC_EPI_RELU || EPI == TC_EPI_RELU_SKIP || EPI == TC_EPI_RELU_BAND ||
+                            EPI == TC_EPI_RELU_BAND_SKIP);
+    constexpr bool kSkip = (EPI == TC_EPI_RELU_SKIP || EPI == TC_EPI_RELU_BAND_SKIP);
     constexpr bool kStores = kRelu || EPI == TC_EPI_REUSE;
     pdl_trigger();
     extern __shared__ uint8_t smem_raw[];
@@ -266,7 +268,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_consta
                         const int col = col0 + g * 4;
                         float q[4];
                         const float4 bz = *reinterpret_cast<const float4 *>(a.bias_below + col);
-                        if (EPI == TC_EPI_RELU_SKIP) {
+                        if (kSkip) {
                             // a residual connection ends on these neurons: its waiting coefficients join first
                             float s4[4] = {0.0f, 0.0f, 0.0f, 0.0f};
                             if (a.add_hi) {
@@ -278,7 +280,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_consta
                                     s4[0] += sl.x; s4[1] += sl.y; s4[2] += sl.z; s4[3] += sl.w;
                                 }
                             }
-                            const int own = a.add_identity ? (int)(rr % a.n_k) : -1;
+                            int own = a.add_identity ? (int)(rr % a.n_k) : -1;
+                            if (kBand && own >= 0) {
+                                // channel-major neuron index -> its column in the y-major row
+                                const int hw = a.band_h_out * a.band_w_out;
+                                const int ch = own / hw, y = (own - ch * hw) / a.band_w_out, x = own % a.band_w_out;
+                                own = (y * a.band_c_out + ch) * a.band_w_out + x;
+                            }
 #pragma unroll
                             for (int e = 0; e < 4; ++e)
                                 v[g * 4 + e] = __float_as_uint(__uint_as_float(v[g * 4 + e]) + s4[e] +
@@ -496,7 +504,9 @@ bool tc_driver_init() {
 }
 
 bool tc_prepare_kernels(bool *pair_ok) {
-    cudaError_t e[12];
+    cudaError_t e[14];
+    e[12] = cudaFuncSetAttribute(gemm_tc_kernel<TC_EPI_RELU_BAND_SKIP, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemMax);
+    e[13] = cudaFuncSetAttribute(gemm_tc_kernel<TC_EPI_RELU_BAND_SKIP, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemMax);
     e[8] = cudaFuncSetAttribute(gemm_tc_kernel<TC_EPI_RELU_BAND, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemMax);
     e[9] = cudaFuncSetAttribute(gemm_tc_kernel<TC_EPI_RELU_BAND, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemMax);
     e[10] = cudaFuncSetAttribute(gemm_tc_kernel<TC_EPI_CONCRETIZE_BAND, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemMax);
@@ -509,7 +519,7 @@ bool tc_prepare_kernels(bool *pair_ok) {
     e[3] = cudaFuncSetAttribute(gemm_tc_kernel<TC_EPI_CONCRETIZE, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemMax);
     e[4] = cudaFuncSetAttribute(gemm_tc_kernel<TC_EPI_REUSE, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemMax);
     e[5] = cudaFuncSetAttribute(gemm_tc_kernel<TC_EPI_REUSE, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemMax);
-    for (int i = 0; i < 12; ++i)
+    for (int i = 0; i < 14; ++i)
         if (e[i] != cudaSuccess) {
             cudaGetLastError();
             return false;
@@ -575,6 +585,11 @@ void launch_gemm_tc(int epi, int ctas, int groups, const TcMap &a_hi, const TcMa
     const CUtensorMap &bl = reinterpret_cast<const CUtensorMap &>(b_lo);
     const CUtensorMap &oh = reinterpret_cast<const CUtensorMap &>(o_hi);
     const CUtensorMap &ol = reinterpret_cast<const CUtensorMap &>(o_lo);
+    if (epi == TC_EPI_RELU_BAND && (args.add_hi || args.add_identity)) {
+        if (ctas == 2) launch_one<TC_EPI_RELU_BAND_SKIP, 2>(groups, ah, al, bh, bl, oh, ol, args, smem_bytes, st);
+        else launch_one<TC_EPI_RELU_BAND_SKIP, 1>(groups, ah, al, bh, bl, oh, ol, args, smem_bytes, st);
+        return;
+    }
     if (epi == TC_EPI_RELU_BAND || epi == TC_EPI_CONCRETIZE_BAND) {
         if (epi == TC_EPI_RELU_BAND) {
             if (ctas == 2) launch_one<TC_EPI_RELU_BAND, 2>(groups, ah, al, bh, bl, oh, ol, args, smem_bytes, st);

@@ -12,7 +12,7 @@ constexpr int kTcSmemMax = 227 * 1024;
 // TC_EPI_RELU_BAND / TC_EPI_CONCRETIZE_BAND: the two path epilogues for the banded form of a conv back-step
 // (TcArgs::n_bands), again as variants of their own.
 enum { TC_EPI_RELU = 0, TC_EPI_CONCRETIZE = 1, TC_EPI_REUSE = 2, TC_EPI_RELU_SKIP = 3, TC_EPI_RELU_BAND = 4,
-       TC_EPI_CONCRETIZE_BAND = 5 };
+       TC_EPI_CONCRETIZE_BAND = 5, TC_EPI_RELU_BAND_SKIP = 6 };
 
 // Storage for a CUtensorMap (128 bytes, 64-byte aligned), kept opaque so that
 // only gemm_tc.cu needs the driver API header.
@@ -47,6 +47,8 @@ struct TcArgs {
     // The relaxation / box arrays are y-major copies, indexed by the output column.
     int n_bands, band_rin, band_o_shift, band_h_in, band_row_in;   // band_row_in = channels * width of layer j's output map
     int band_s, band_y_shift, band_row_out;                        // band_row_out = channels * width of the map below
+    int band_c_out, band_h_out, band_w_out;                        // the map below, for add_identity: the row's own neuron
+                                                                   // (channel-major index row mod n_k) sits at its y-major column
     int has_relu;    // a ReLU sits on the neurons below layer j
     int split_out;   // ReLU epilogue: store the result as a TF32 pair (a tensor-core step follows)
     const float *lamL, *lamU, *nuU;              // [batch][ld_n] ("box" = whatever a group of 2 * n_k rows shares)

@@ -466,6 +466,8 @@ RES_NETS = {
     "resfc_wide": lambda: wl.residual_fc(64, 300, 2, 10, batch=4, eps=0.01, seed=23),
     "resconv": lambda: wl.residual_conv((2, 10, 8), 4, 2, 6, batch=3, eps=0.02, seed=24),
     "resconv_wide": lambda: wl.residual_conv((3, 16, 16), 8, 1, 10, batch=2, eps=0.01, seed=25),
+    # map rows of 64 floats everywhere: the dense conv steps take the banded tensor-core form
+    "resconv_band": lambda: wl.residual_conv((4, 16, 16), 8, 2, 10, batch=3, eps=0.01, seed=29),
 }
 
 
@@ -479,6 +481,8 @@ def test_residual_nets(name, mode):
     g = run_gpu(w, contraction={"ffma": 1, "tc": 2, "tc16": 3}[mode], max_batch=w.batch + 1)
     if mode == "tc16":
         assert g["paths"] & 16 and not g["paths"] & 32      # one launch per back-step, not the chain kernel
+    if mode == "tc":
+        assert bool(g["paths"] & 64) == (name == "resconv_band")
     compare(g, ref, label=f"{name}/{mode}")
     # the connections matter: the same layers without them give other bounds
     plain = orc.deeppoly(w.layers, w.centers, w.eps, w.clip_lo, w.clip_hi)
@@ -494,7 +498,7 @@ def test_residual_connection_into_the_output_layer_and_back_to_back_blocks(mode)
 
 
 @pytest.mark.parametrize("mode", ["ffma", "tc"])
-@pytest.mark.parametrize("name", ["resfc_ragged", "resfc_wide", "resconv"])
+@pytest.mark.parametrize("name", ["resfc_ragged", "resfc_wide", "resconv", "resconv_band"])
 def test_residual_nets_traversals_that_stop_early(name, mode):
     """IBP, CROWN-IBP, DeepPoly_p and mixed depths: a traversal may end on a connection's source (the waiting
     coefficients join before the simplification), above it (they are simplified on their own), or below it."""
