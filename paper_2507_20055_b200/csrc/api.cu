@@ -1072,8 +1072,10 @@ cert_status_t cert_backsub_bounds(cert_net_t *net, const float *centers, float e
             cert::launch_init_expr(Lk_y, Lb_y, batch, net->buf[cur], net->buf_lo[cur], net->dbuf[dcur], st);
             y_major = true;
         } else {
+            // a conv layer right above a banded conv layer places its window coefficients at their y-major columns
+            y_major = Lk.kind == CERT_LAYER_CONV2D && on_band(k - 1);
             cert::launch_init_expr(Lk, net->layers[k - 1], batch, net->buf[cur],
-                                   wants_pair(k - 1) ? net->buf_lo[cur] : nullptr, net->dbuf[dcur], st);
+                                   wants_pair(k - 1) ? net->buf_lo[cur] : nullptr, net->dbuf[dcur], st, y_major);
         }
         rec.mark(CERT_CLASS_RELU_STEP);
         // Residual connections: the coefficients on a connection's source wait (kept: the buffer that holds

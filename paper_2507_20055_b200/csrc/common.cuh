@@ -99,7 +99,7 @@ void launch_relax(const LayerDev &L, float *lb_out, float *ub_out, int n_total, 
 //   Q  [rows][ld] with rows = batch*2*n_k ordered (box, side, neuron)
 //   Q_lo != nullptr: Q is written as a TF32 pair (hi in Q, lo in Q_lo) for the tensor-core contraction
 void launch_init_expr(const LayerDev &Lk, const LayerDev &Lbelow, int batch, float *Q, float *Q_lo, float *d,
-                      cudaStream_t st);
+                      cudaStream_t st, int y_major = 0);   // y_major (conv layer k): columns in [y][channel][x] order
 
 // ReLU back-step in place on P [rows][ld] (expression over the outputs of
 // layer `Lj`, i.e. over its ReLU neurons if it has one), plus d += Q.b_j.

@@ -278,7 +278,8 @@ __global__ void conv_expr_start_kernel(const float *__restrict__ Wk, ConvGeom gk
                                        float *__restrict__ P, float *__restrict__ P_lo, float *__restrict__ d,
                                        long long rows, int n_k, int ld, int has_relu,
                                        const float *__restrict__ lamL, const float *__restrict__ lamU,
-                                       const float *__restrict__ nuU, const float *__restrict__ bias_below) {
+                                       const float *__restrict__ nuU, const float *__restrict__ bias_below,
+                                       int y_major) {
     long long r = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     int lane = threadIdx.x & 31;
     if (r >= rows) return;
@@ -308,12 +309,14 @@ __global__ void conv_expr_start_kernel(const float *__restrict__ Wk, ConvGeom gk
         const float c = Wk[(size_t)co * taps + q];
         const float qv = has_relu ? relu_backstep(c, upper, ll[t], lu[t], nu[t], dacc) : c;
         dacc = fmaf(qv, bias_below[t], dacc);
+        // the column: channel-major, or [y][channel][x] for the banded steps
+        const int ts = y_major ? (iy * gk.c_in + ci) * gk.w_in + ix : t;
         if (lrow) {
             const float h = tf32_round(qv);
-            prow[t] = h;
-            lrow[t] = tf32_round(qv - h);
+            prow[ts] = h;
+            lrow[ts] = tf32_round(qv - h);
         } else {
-            prow[t] = qv;
+            prow[ts] = qv;
         }
     }
     dacc = warp_sum(dacc);
@@ -532,12 +535,12 @@ void launch_relax(const LayerDev &L, float *lb_out, float *ub_out, int n_total, 
 }
 
 void launch_init_expr(const LayerDev &Lk, const LayerDev &Lb, int batch, float *Q, float *Q_lo, float *d,
-                      cudaStream_t st) {
+                      cudaStream_t st, int y_major) {
     long long rows = 2LL * batch * Lk.n_out;
     if (Lk.kind != CERT_LAYER_FC) {
         conv_expr_start_kernel<<<grid_for_warps(rows), kWarpsPerBlock * 32, 0, st>>>(
             Lk.W, geom_of(Lk), Lk.bias_n, Q, Q_lo, d, rows, Lk.n_out, Lb.ld_out, Lb.relu_after, Lb.lamL, Lb.lamU,
-            Lb.nuU, Lb.bias_n);
+            Lb.nuU, Lb.bias_n, y_major);
         return;
     }
     const long long warps4 = 2LL * batch * ((Lk.n_out + 3) / 4);

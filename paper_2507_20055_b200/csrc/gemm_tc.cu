@@ -239,6 +239,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_consta
             const int upper = (int)((rr / a.n_k) & 1);
             const size_t relax_row = (size_t)b * a.ld_n;
             float dacc = 0.0f;
+            int own = -1;                  // kSkip: the column of the row's own neuron (unit coefficient), if it joins
+            if (kSkip && a.add_identity) {
+                own = (int)(rr % a.n_k);
+                if (kBand) {
+                    // channel-major neuron index -> its column in the y-major row
+                    const int hw = a.band_h_out * a.band_w_out;
+                    const int ch = own / hw, y = (own - ch * hw) / a.band_w_out, x = own % a.band_w_out;
+                    own = (y * a.band_c_out + ch) * a.band_w_out + x;
+                }
+            }
             const int acc = lt & 1;
             const uint32_t acc_phase = (lt >> 1) & 1;
             if (!mbar_wait(&bars->acc_full[acc], acc_phase) || *abort_flag) { ok = false; break; }
@@ -254,6 +264,18 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_consta
                     break;                                   // warp-uniform; ld_n is a multiple of 32
                 }
                 uint32_t v[32];
+                // a residual connection ends on these neurons: its waiting coefficients (this row's 32 columns,
+                // one 128-byte line per part) are requested before the accumulator is read
+                float4 sh[kSkip ? 8 : 1], sl[kSkip ? 8 : 1];
+                if (kSkip) {
+                    const float4 z4 = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+                    const size_t o = (size_t)rr * a.ld_n + col0;
+#pragma unroll
+                    for (int g = 0; g < 8; ++g) {
+                        sh[g] = a.add_hi ? __ldg(reinterpret_cast<const float4 *>(a.add_hi + o) + g) : z4;
+                        sl[g] = a.add_lo ? __ldg(reinterpret_cast<const float4 *>(a.add_lo + o) + g) : z4;
+                    }
+                }
                 __syncwarp();
                 tmem_ld32(t_addr + (uint32_t)c0, v);
                 tmem_ld_wait();
@@ -269,24 +291,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_consta
                         float q[4];
                         const float4 bz = *reinterpret_cast<const float4 *>(a.bias_below + col);
                         if (kSkip) {
-                            // a residual connection ends on these neurons: its waiting coefficients join first
-                            float s4[4] = {0.0f, 0.0f, 0.0f, 0.0f};
-                            if (a.add_hi) {
-                                const size_t o = (size_t)rr * a.ld_n + col;
-                                const float4 sh = *reinterpret_cast<const float4 *>(a.add_hi + o);
-                                s4[0] = sh.x; s4[1] = sh.y; s4[2] = sh.z; s4[3] = sh.w;
-                                if (a.add_lo) {
-                                    const float4 sl = *reinterpret_cast<const float4 *>(a.add_lo + o);
-                                    s4[0] += sl.x; s4[1] += sl.y; s4[2] += sl.z; s4[3] += sl.w;
-                                }
-                            }
-                            int own = a.add_identity ? (int)(rr % a.n_k) : -1;
-                            if (kBand && own >= 0) {
-                                // channel-major neuron index -> its column in the y-major row
-                                const int hw = a.band_h_out * a.band_w_out;
-                                const int ch = own / hw, y = (own - ch * hw) / a.band_w_out, x = own % a.band_w_out;
-                                own = (y * a.band_c_out + ch) * a.band_w_out + x;
-                            }
+                            // the waiting coefficients and the unit coefficient join before the ReLU back-step
+                            const float s4[4] = {sh[g].x + sl[g].x, sh[g].y + sl[g].y, sh[g].z + sl[g].z,
+                                                 sh[g].w + sl[g].w};
 #pragma unroll
                             for (int e = 0; e < 4; ++e)
                                 v[g * 4 + e] = __float_as_uint(__uint_as_float(v[g * 4 + e]) + s4[e] +
