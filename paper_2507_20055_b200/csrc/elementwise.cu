@@ -278,8 +278,7 @@ __global__ void conv_expr_start_kernel(const float *__restrict__ Wk, ConvGeom gk
                                        float *__restrict__ P, float *__restrict__ P_lo, float *__restrict__ d,
                                        long long rows, int n_k, int ld, int has_relu,
                                        const float *__restrict__ lamL, const float *__restrict__ lamU,
-                                       const float *__restrict__ nuU, const float *__restrict__ bias_below,
-                                       int y_major) {
+                                       const float *__restrict__ nuU, const float *__restrict__ bias_below) {
     long long r = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     int lane = threadIdx.x & 31;
     if (r >= rows) return;
@@ -309,15 +308,70 @@ __global__ void conv_expr_start_kernel(const float *__restrict__ Wk, ConvGeom gk
         const float c = Wk[(size_t)co * taps + q];
         const float qv = has_relu ? relu_backstep(c, upper, ll[t], lu[t], nu[t], dacc) : c;
         dacc = fmaf(qv, bias_below[t], dacc);
-        // the column: channel-major, or [y][channel][x] for the banded steps
-        const int ts = y_major ? (iy * gk.c_in + ci) * gk.w_in + ix : t;
         if (lrow) {
             const float h = tf32_round(qv);
-            prow[ts] = h;
-            lrow[ts] = tf32_round(qv - h);
+            prow[t] = h;
+            lrow[t] = tf32_round(qv - h);
         } else {
-            prow[ts] = qv;
+            prow[t] = qv;
         }
+    }
+    dacc = warp_sum(dacc);
+    if (lane == 0) d[r] = bias_k[i] + dacc;
+}
+
+// The same start with the columns in [y][channel][x] order (banded conv steps): the window's kh map rows are one
+// contiguous piece of the row, so a warp writes the row once, 16 bytes per lane, looking up the tap of each column
+// inside that piece and storing zeros elsewhere.
+__global__ void conv_expr_start_ymajor_kernel(const float *__restrict__ Wk, ConvGeom gk,
+                                              const float *__restrict__ bias_k, float *__restrict__ P,
+                                              float *__restrict__ P_lo, float *__restrict__ d, long long rows, int n_k,
+                                              int ld, int has_relu, const float *__restrict__ lamL,
+                                              const float *__restrict__ lamU, const float *__restrict__ nuU,
+                                              const float *__restrict__ bias_below) {
+    long long r = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    int lane = threadIdx.x & 31;
+    if (r >= rows) return;
+    int b = (int)(r / (2LL * n_k));
+    int upper = (int)((r / n_k) & 1);
+    int i = (int)(r % n_k);
+    float *prow = P + (size_t)r * ld;
+    float *lrow = P_lo ? P_lo + (size_t)r * ld : nullptr;
+    const float *ll = lamL + (size_t)b * ld, *lu = lamU + (size_t)b * ld, *nu = nuU + (size_t)b * ld;
+    const int hw_o = gk.h_out * gk.w_out;
+    const int co = i / hw_o;
+    const int y0 = ((i / gk.w_out) % gk.h_out) * gk.stride - gk.pad;
+    const int x0 = (i % gk.w_out) * gk.stride - gk.pad;
+    const int khw = gk.kh * gk.kw, taps = gk.c_in * khw;
+    const int row = gk.c_in * gk.w_in;
+    const int seg_lo = max(y0, 0) * row, seg_hi = min(y0 + gk.kh, gk.h_in) * row;
+    const float *wrow = Wk + (size_t)co * taps;
+    float dacc = 0.0f;
+    for (int t0 = lane * 4; t0 < ld; t0 += 128) {
+        float hi4[4] = {0.0f, 0.0f, 0.0f, 0.0f}, lo4[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+        if (t0 + 3 >= seg_lo && t0 < seg_hi) {
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const int t = t0 + e;
+                if (t < seg_lo || t >= seg_hi) continue;
+                const int iy = t / row, rem = t - iy * row;
+                const int ci = rem / gk.w_in, ix = rem - ci * gk.w_in;
+                const int kx = ix - x0;
+                if (kx < 0 || kx >= gk.kw) continue;
+                const float c = wrow[(ci * gk.kh + (iy - y0)) * gk.kw + kx];
+                const int ts = (ci * gk.h_in + iy) * gk.w_in + ix;      // channel-major: relaxation and bias below
+                const float qv = has_relu ? relu_backstep(c, upper, ll[ts], lu[ts], nu[ts], dacc) : c;
+                dacc = fmaf(qv, bias_below[ts], dacc);
+                if (lrow) {
+                    hi4[e] = tf32_round(qv);
+                    lo4[e] = tf32_round(qv - hi4[e]);
+                } else {
+                    hi4[e] = qv;
+                }
+            }
+        }
+        *reinterpret_cast<float4 *>(prow + t0) = make_float4(hi4[0], hi4[1], hi4[2], hi4[3]);
+        if (lrow) *reinterpret_cast<float4 *>(lrow + t0) = make_float4(lo4[0], lo4[1], lo4[2], lo4[3]);
     }
     dacc = warp_sum(dacc);
     if (lane == 0) d[r] = bias_k[i] + dacc;
@@ -537,10 +591,16 @@ void launch_relax(const LayerDev &L, float *lb_out, float *ub_out, int n_total, 
 void launch_init_expr(const LayerDev &Lk, const LayerDev &Lb, int batch, float *Q, float *Q_lo, float *d,
                       cudaStream_t st, int y_major) {
     long long rows = 2LL * batch * Lk.n_out;
+    if (Lk.kind != CERT_LAYER_FC && y_major) {
+        conv_expr_start_ymajor_kernel<<<grid_for_warps(rows), kWarpsPerBlock * 32, 0, st>>>(
+            Lk.W, geom_of(Lk), Lk.bias_n, Q, Q_lo, d, rows, Lk.n_out, Lb.ld_out, Lb.relu_after, Lb.lamL, Lb.lamU,
+            Lb.nuU, Lb.bias_n);
+        return;
+    }
     if (Lk.kind != CERT_LAYER_FC) {
         conv_expr_start_kernel<<<grid_for_warps(rows), kWarpsPerBlock * 32, 0, st>>>(
             Lk.W, geom_of(Lk), Lk.bias_n, Q, Q_lo, d, rows, Lk.n_out, Lb.ld_out, Lb.relu_after, Lb.lamL, Lb.lamU,
-            Lb.nuU, Lb.bias_n, y_major);
+            Lb.nuU, Lb.bias_n);
         return;
     }
     const long long warps4 = 2LL * batch * ((Lk.n_out + 3) / 4);
