@@ -264,16 +264,20 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_consta
                     break;                                   // warp-uniform; ld_n is a multiple of 32
                 }
                 uint32_t v[32];
-                // a residual connection ends on these neurons: its waiting coefficients (this row's 32 columns,
-                // one 128-byte line per part) are requested before the accumulator is read
-                float4 sh[kSkip ? 8 : 1], sl[kSkip ? 8 : 1];
-                if (kSkip) {
+                // a residual connection ends on these neurons: its waiting coefficients for the warp's 32 rows x 32
+                // columns are requested before the accumulator is read, four rows (128-byte lines) per instruction:
+                // load i brings 16-byte piece lane % 8 of row 4 i + lane / 8
+                float4 ch[kSkip ? 8 : 1], cl[kSkip ? 8 : 1];
+                const bool joins = kSkip && a.add_hi != nullptr;
+                if (kSkip && joins) {
                     const float4 z4 = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
-                    const size_t o = (size_t)rr * a.ld_n + col0;
 #pragma unroll
-                    for (int g = 0; g < 8; ++g) {
-                        sh[g] = a.add_hi ? __ldg(reinterpret_cast<const float4 *>(a.add_hi + o) + g) : z4;
-                        sl[g] = a.add_lo ? __ldg(reinterpret_cast<const float4 *>(a.add_lo + o) + g) : z4;
+                    for (int i = 0; i < 8; ++i) {
+                        long long rw = warp_row0 + 4 * i + (lane >> 3);
+                        if (rw >= a.M) rw = 0;
+                        const size_t o = (size_t)rw * a.ld_n + col0 + (lane & 7) * 4;
+                        ch[i] = __ldg(reinterpret_cast<const float4 *>(a.add_hi + o));
+                        cl[i] = a.add_lo ? __ldg(reinterpret_cast<const float4 *>(a.add_lo + o)) : z4;
                     }
                 }
                 __syncwarp();
@@ -285,6 +289,20 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_consta
                     __syncwarp();
                     const uint32_t row_hi = smem_u32(slab_hi) + (uint32_t)lane * 128u;
                     const uint32_t row_lo = smem_u32(slab_lo) + (uint32_t)lane * 128u;
+                    if (kSkip && joins) {
+                        // through the (free) slab to the lane that owns the row; a lane then reads and rewrites
+                        // only its own row
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) {
+                            const uint32_t rw = (uint32_t)(4 * i + (lane >> 3));
+                            const uint32_t off = rw * 128u + ((((uint32_t)lane & 7u) ^ (rw & 7u)) << 4);
+                            asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(smem_u32(slab_hi) + off),
+                                         "f"(ch[i].x), "f"(ch[i].y), "f"(ch[i].z), "f"(ch[i].w) : "memory");
+                            asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(smem_u32(slab_lo) + off),
+                                         "f"(cl[i].x), "f"(cl[i].y), "f"(cl[i].z), "f"(cl[i].w) : "memory");
+                        }
+                        __syncwarp();
+                    }
 #pragma unroll
                     for (int g = 0; g < 8; ++g) {
                         const int col = col0 + g * 4;
@@ -292,8 +310,17 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_consta
                         const float4 bz = *reinterpret_cast<const float4 *>(a.bias_below + col);
                         if (kSkip) {
                             // the waiting coefficients and the unit coefficient join before the ReLU back-step
-                            const float s4[4] = {sh[g].x + sl[g].x, sh[g].y + sl[g].y, sh[g].z + sl[g].z,
-                                                 sh[g].w + sl[g].w};
+                            float s4[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+                            if (joins) {
+                                const uint32_t swj = (uint32_t)((g ^ (lane & 7)) << 4);
+                                float h4[4], l4[4];
+                                asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(h4[0]), "=f"(h4[1]),
+                                             "=f"(h4[2]), "=f"(h4[3]) : "r"(row_hi + swj) : "memory");
+                                asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(l4[0]), "=f"(l4[1]),
+                                             "=f"(l4[2]), "=f"(l4[3]) : "r"(row_lo + swj) : "memory");
+#pragma unroll
+                                for (int e = 0; e < 4; ++e) s4[e] = h4[e] + l4[e];
+                            }
 #pragma unroll
                             for (int e = 0; e < 4; ++e)
                                 v[g * 4 + e] = __float_as_uint(__uint_as_float(v[g * 4 + e]) + s4[e] +
