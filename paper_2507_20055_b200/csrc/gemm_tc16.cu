@@ -243,6 +243,21 @@ gemm_tc16_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_cons
                 const int col0 = nt * BN + c0;
                 if (col0 >= a.ld_n) break;                   // warp-uniform; ld_n is a multiple of 32
                 uint32_t v[32];
+                // a residual connection ends on these neurons: its waiting coefficients (an fp16 pair here) for the
+                // warp's 32 rows x 32 columns are requested before the accumulator is read, eight rows (64-byte
+                // pieces of a row) per instruction: load i brings 16-byte piece lane % 4 of row 8 i + lane / 4
+                uint4 ch[EPI == TC_EPI_RELU_SKIP ? 4 : 1], cl[EPI == TC_EPI_RELU_SKIP ? 4 : 1];
+                const bool joins = EPI == TC_EPI_RELU_SKIP && a.add_hi != nullptr;
+                if (EPI == TC_EPI_RELU_SKIP && joins) {
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        long long rw = warp_row0 + 8 * i + (lane >> 2);
+                        if (rw >= a.M) rw = 0;
+                        const size_t o = (size_t)rw * a.ld_n + col0 + (lane & 3) * 8;
+                        ch[i] = __ldg(reinterpret_cast<const uint4 *>(reinterpret_cast<const __half *>(a.add_hi) + o));
+                        cl[i] = __ldg(reinterpret_cast<const uint4 *>(reinterpret_cast<const __half *>(a.add_lo) + o));
+                    }
+                }
                 __syncwarp();
                 tmem_ld32(t_addr + (uint32_t)c0, v);
                 tmem_ld_wait();
@@ -252,9 +267,31 @@ gemm_tc16_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_cons
                     __syncwarp();
                     const uint32_t row_hi = smem_u32(slab_hi) + (uint32_t)lane * 64u;
                     const uint32_t row_lo = smem_u32(slab_lo) + (uint32_t)lane * 64u;
+                    if (EPI == TC_EPI_RELU_SKIP && joins) {
+                        // through the (free) slab to the lane that owns the row; a lane then reads and rewrites
+                        // only its own row
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            const uint32_t rw = (uint32_t)(8 * i + (lane >> 2));
+                            const uint32_t off = rw * 64u + ((((uint32_t)lane & 3u) ^ ((rw >> 1) & 3u)) << 4);
+                            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(smem_u32(slab_hi) + off),
+                                         "r"(ch[i].x), "r"(ch[i].y), "r"(ch[i].z), "r"(ch[i].w) : "memory");
+                            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(smem_u32(slab_lo) + off),
+                                         "r"(cl[i].x), "r"(cl[i].y), "r"(cl[i].z), "r"(cl[i].w) : "memory");
+                        }
+                        __syncwarp();
+                    }
 #pragma unroll
                     for (int c16 = 0; c16 < 4; ++c16) {
                         uint32_t ph[4], pl[4];              // 8 halves of hi, 8 of lo
+                        uint32_t jh[4] = {0u, 0u, 0u, 0u}, jl[4] = {0u, 0u, 0u, 0u};     // the joining pair's 8 columns
+                        if (EPI == TC_EPI_RELU_SKIP && joins) {
+                            const uint32_t swj = (uint32_t)((c16 ^ ((lane >> 1) & 3)) << 4);
+                            asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(jh[0]), "=r"(jh[1]), "=r"(jh[2]),
+                                         "=r"(jh[3]) : "r"(row_hi + swj) : "memory");
+                            asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(jl[0]), "=r"(jl[1]), "=r"(jl[2]),
+                                         "=r"(jl[3]) : "r"(row_lo + swj) : "memory");
+                        }
 #pragma unroll
                         for (int g2 = 0; g2 < 2; ++g2) {
                             const int g = c16 * 2 + g2;
@@ -262,13 +299,11 @@ gemm_tc16_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_cons
                             float q[4];
                             const float4 bz = *reinterpret_cast<const float4 *>(a.bias_below + col);
                             if (EPI == TC_EPI_RELU_SKIP) {
-                                // a residual connection ends on these neurons: its waiting coefficients (an fp16
-                                // pair here) join before the ReLU back-step
+                                // the waiting coefficients and the unit coefficient join before the ReLU back-step
                                 float s4[4] = {0.0f, 0.0f, 0.0f, 0.0f};
-                                if (a.add_hi) {
-                                    const size_t o = (size_t)rr * a.ld_n + col;
-                                    const uint2 sh = *reinterpret_cast<const uint2 *>(reinterpret_cast<const __half *>(a.add_hi) + o);
-                                    const uint2 sl = *reinterpret_cast<const uint2 *>(reinterpret_cast<const __half *>(a.add_lo) + o);
+                                if (joins) {
+                                    const uint2 sh = make_uint2(jh[g2 * 2], jh[g2 * 2 + 1]);
+                                    const uint2 sl = make_uint2(jl[g2 * 2], jl[g2 * 2 + 1]);
                                     const __half2 h01 = *reinterpret_cast<const __half2 *>(&sh.x), h23 = *reinterpret_cast<const __half2 *>(&sh.y);
                                     const __half2 l01 = *reinterpret_cast<const __half2 *>(&sl.x), l23 = *reinterpret_cast<const __half2 *>(&sl.y);
                                     const float2 fh01 = __half22float2(h01), fh23 = __half22float2(h23);
