@@ -12,7 +12,7 @@ pytestmark = pytest.mark.gpu
 
 def _oracle(w, boxes=None):
     c = w.centers if boxes is None else w.centers[np.asarray(boxes)]
-    return orc.deeppoly(w.layers, c, w.eps, w.clip_lo, w.clip_hi)
+    return orc.deeppoly(w.layers, c, w.eps, w.clip_lo, w.clip_hi, skip_from=w.skip_from)
 
 
 MODES = {"ffma": 1, "tc": 2}
@@ -707,3 +707,35 @@ def test_random_nets_with_random_traversal_depths(block):
         for c in modes:
             g = run_gpu(w, contraction=c, backsteps=steps, max_batch=w.batch + block % 2)
             compare(g, ref, label=f"{kind}/{w.name}/mode {c}/depths {steps}")
+
+
+_BAND_GEOMETRIES = [((2, 16, 16), (4, 8, 12)), ((4, 16, 16), (4, 8)), ((1, 32, 32), (2, 4)), ((4, 8, 8), (8, 16)),
+                    ((3, 32, 32), (2, 4))]
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_random_residual_conv_nets_in_the_banded_form(seed):
+    """Residual conv nets whose map rows are multiples of 32 floats (the dense conv steps take the banded
+    tensor-core form, the joining step its own kernel variant): one to three blocks, some with the first block's
+    connection removed; full traversals and one random depth per layer; FMA and tensor-core modes."""
+    r = np.random.default_rng(900 + seed)
+    shape, channels = _BAND_GEOMETRIES[int(r.integers(len(_BAND_GEOMETRIES)))]
+
+    def make(s):
+        w = wl.residual_conv(shape, int(r.choice(channels)), int(r.integers(1, 4)), int(r.integers(2, 11)),
+                             batch=int(r.integers(1, 5)), eps=0.01, seed=1000 + s)
+        if seed % 3 == 0 and len(w.layers) > 4:
+            w.skip_from = [-1 if k == 2 else s_ for k, s_ in enumerate(w.skip_from)]
+        return w
+
+    w, ref = _well_conditioned(make, seed)
+    K = len(w.layers)
+    steps = [int(x) for x in r.integers(-1, K + 1, size=K)]
+    ref_steps = orc.deeppoly(w.layers, w.centers, w.eps, w.clip_lo, w.clip_hi, skip_from=w.skip_from,
+                             backsteps_per_layer=steps)
+    for mode, contraction in (("ffma", 1), ("tc", 2)):
+        g = run_gpu(w, contraction=contraction, max_batch=w.batch + seed % 2)
+        assert bool(g["paths"] & 64) == (mode == "tc")
+        compare(g, ref, min_good_fraction=0.5, label=f"residual_band[{seed}]/{mode}")
+        compare(run_gpu(w, contraction=contraction, backsteps=steps), ref_steps, min_good_fraction=0.5,
+                label=f"residual_band[{seed}]/{mode}/depths {steps}")
