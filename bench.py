@@ -105,13 +105,13 @@ def oracle_sample(w, n_boxes, threads=None, backsteps=None, certifier="deeppoly"
     c = w.centers[:n_boxes]
     t0 = time.perf_counter()
     if certifier == "reusecert":
-        orc.reusecert(w.layers, c, w.eps, w.clip_lo, w.clip_hi, n_threads=cores)
+        res = orc.reusecert(w.layers, c, w.eps, w.clip_lo, w.clip_hi, n_threads=cores)
     else:
-        orc.deeppoly(w.layers, c, w.eps, w.clip_lo, w.clip_hi, n_threads=cores, backsteps_per_layer=backsteps,
-                     skip_from=w.skip_from)
+        res = orc.deeppoly(w.layers, c, w.eps, w.clip_lo, w.clip_hi, n_threads=cores, backsteps_per_layer=backsteps,
+                           skip_from=w.skip_from)
     dt = time.perf_counter() - t0
-    return {"value": n_boxes / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
-            "sample": f"first {n_boxes} of {w.batch} boxes of {w.name}, one box per thread, {dt:.1f} s wall"}, dt
+    return {"value": n_boxes / dt, "unit": UNIT, "cores": min(cores, n_boxes), "kind": "oracle",
+            "sample": f"first {n_boxes} of {w.batch} boxes of {w.name}, one box per thread, {dt:.1f} s wall"}, dt, res
 
 
 def certifier_steps(name, n_layers):
@@ -183,7 +183,7 @@ def run_reference(args, w):
         n_boxes = max(1, min(cores, 16) // 2)     # about 11 s per box per core
     times = []
     for i in range(args.warmup + args.steps):
-        base, dt = oracle_sample(w, n_boxes, backsteps=args.backsteps, certifier=args.certifier)
+        base, dt, _ = oracle_sample(w, n_boxes, backsteps=args.backsteps, certifier=args.certifier)
         if i >= args.warmup:
             times.append(dt)
     ms = 1000.0 * sum(times) / len(times)
@@ -211,9 +211,9 @@ def main():
                          "shape of the paper's 'Skip' network (784 -> 512 x 5 -> 10, two blocks, 64 boxes); 6: a residual "
                          "conv net (3x32x32 -> conv16 s2 -> two blocks of two 3x3 convs -> 10, 16 boxes)")
     ap.add_argument("--batch", type=int, default=None)
-    ap.add_argument("--contraction", default="fastest", choices=["fastest", "auto", "ffma", "tc", "tc16"],
-                    help="tc = tcgen05 3xTF32, tc16 = tcgen05 fp16 split (FC nets), ffma = FMA units, auto = the "
-                         "library's default (tc), fastest = tc16 for FC nets, else auto")
+    ap.add_argument("--contraction", default="auto", choices=["auto", "ffma", "tc", "tc16"],
+                    help="auto = what the plain three-call ABI runs (the fp16 split where the net's weights prove its "
+                         "range, else 3xTF32); tc = tcgen05 3xTF32, tc16 = tcgen05 fp16 split (FC nets), ffma = FMA units")
     ap.add_argument("--certifier", default="deeppoly",
                     help="deeppoly | ibp | crown_ibp | deeppoly_pN (N back-substitution steps per layer) | reusecert")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -260,10 +260,10 @@ def main():
     net = binding.CertNet(w.layers, B, w.clip_lo, w.clip_hi, skip_from=w.skip_from)
     mode = {"auto": binding.CONTRACTION_AUTO, "ffma": binding.CONTRACTION_FFMA, "tc": binding.CONTRACTION_TC3XTF32,
             "tc16": binding.CONTRACTION_TC3XFP16}
-    if args.contraction == "fastest":
-        all_fc = all(l.kind == "fc" for l in w.layers)
-        args.contraction = "tc16" if (all_fc and len(w.layers) > 1) else "auto"
     net.set_contraction(mode[args.contraction])
+    resolved = args.contraction
+    if args.contraction == "auto":
+        resolved = {1: "ffma", 2: "tc", 3: "tc16"}[net.auto_contraction()]
     stream = torch.cuda.Stream()
     centers = torch.from_numpy(w.centers).cuda()
     lb = torch.empty((B, net.n_total), dtype=torch.float32, device="cuda")
@@ -327,7 +327,7 @@ def main():
 
     # ---- the same steps with the 3xTF32 contraction, for reference, when the fp16 split was timed above ----
     tf32_ref = None
-    if args.contraction == "tc16" and world == 1 and not reuse:
+    if resolved == "tc16" and world == 1 and not reuse:
         net.set_contraction(binding.CONTRACTION_TC3XTF32)
         n_ref = max(3, min(args.steps, 5))
         ev2 = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_ref)]
@@ -344,7 +344,7 @@ def main():
         tf32_ref = {"value": B / (ms_ref / 1000.0), "unit": UNIT, "ms_per_step": ms_ref, "steps": n_ref,
                     "contraction": "tc (3xTF32)"}
         assert net.last_status(stream.cuda_stream) == 0
-        net.set_contraction(binding.CONTRACTION_TC3XFP16)
+        net.set_contraction(mode[args.contraction])
 
     # ---- end to end through the host-buffer entry point (pinned buffers, copies timed) ----
     centers_pin = torch.from_numpy(w.centers).pin_memory()
@@ -438,7 +438,7 @@ def main():
             "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {"workload": w.name, "certifier": args.certifier, "boxes_per_gpu": B, "eps": w.eps,
                        "net": "->".join(str(x) for x in [w.layers[0].n_in] + [l.n_out for l in w.layers]),
-                       "contraction": args.contraction, "parallelism": f"replicas over boxes x{world}",
+                       "contraction": args.contraction, "contraction_resolved": resolved, "parallelism": f"replicas over boxes x{world}",
                        "l2": "256 MiB flush write between timed steps; per-step coefficient traffic exceeds L2"},
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(B * net.n0 * 4),
                     "d2h_bytes_per_step": int(2 * B * net.n_total * 4), "steps": e2e_steps},
@@ -452,7 +452,22 @@ def main():
             from oracle import deeppoly_oracle as orc
             orc.build()
             n_boxes = min(n_boxes, B) if args.config != 4 else min(B, orc.max_threads(), 16)
-            out["cpu_baseline"], _ = oracle_sample(w, n_boxes, backsteps=args.backsteps, certifier=args.certifier)
+            out["cpu_baseline"], _, ref = oracle_sample(w, n_boxes, backsteps=args.backsteps, certifier=args.certifier)
+            if args.config in (0, 1):
+                one, _, _ = oracle_sample(w, min(n_boxes, 4), threads=1, backsteps=args.backsteps,
+                                          certifier=args.certifier)
+                out["cpu_baseline"]["single_thread"] = {"value": one["value"], "unit": UNIT, "sample": one["sample"]}
+            # parity of the timed configuration: the bounds of the last timed device call against the oracle
+            # boxes just computed (same rule and tolerance as the tests: oracle/parity_rule.py)
+            from oracle import parity_rule
+            with torch.cuda.stream(stream):
+                step_device()
+            stream.synchronize()
+            rep = parity_rule.parity_report(lb[:n_boxes].cpu().numpy(), ub[:n_boxes].cpu().numpy(),
+                                            net.branch_codes(B)[:n_boxes].cpu().numpy(), ref, w.layers)
+            rep["tolerance"] = parity_rule.TOL
+            rep["ok"] = bool(rep["code_mismatches"] == 0 and rep["max_scaled_err"] <= parity_rule.TOL)
+            out["parity"] = rep
         print(json.dumps(out))
     net.destroy()
     if world > 1:

@@ -151,7 +151,12 @@ cert_status_t cert_reusecert_bounds_host(cert_net_t *net, const float *centers_h
                                          float *lb_host, float *ub_host, void *stream);
 
 /* Same, with HOST buffers (pageable or pinned): copies centers to the device,
- * runs cert_deeppoly_bounds, copies the bounds back and waits for the stream. */
+ * runs cert_deeppoly_bounds, copies the bounds back and waits for the stream.
+ * Because it waits anyway it also reads the device-side status word: it
+ * returns CERT_ERR_TIMEOUT / CERT_ERR_RANGE (and clears the word) instead of
+ * handing back bounds that a run-out wait or an fp16 overflow invalidated;
+ * under CERT_CONTRACTION_AUTO an overflow re-runs the call with the TF32 split
+ * first.  The three *_host calls all do this. */
 cert_status_t cert_deeppoly_bounds_host(cert_net_t *net, const float *centers_host, float eps,
                                         int batch, float *lb_host, float *ub_host, void *stream);
 
@@ -209,7 +214,14 @@ cert_status_t cert_net_selftest_bounded_wait(cert_net_t *net, void *stream);
  *            twice the tensor-core rate and half the operand bytes, for nets of FC layers only and
  *            coefficients below 65504 in magnitude (beyond that cert_net_last_status reports
  *            CERT_ERR_RANGE and the results are invalid; values under 6.1e-5 are held to 1.5e-11
- *            absolute instead of 2^-22 relative).  Never chosen by AUTO.
+ *            absolute instead of 2^-22 relative).
+ *   AUTO:    TC3XFP16 when the net's weights prove at create that no coefficient can leave that range on
+ *            any input: a ReLU back-step scales a coefficient by a slope in [0, 1], so every entry of a
+ *            traversal's matrix over layer j-1 is bounded by the matching entry of |W_k| |W_k-1| ... |W_j|,
+ *            and the largest entry of all those products (cert_net_fp16_coefficient_bound) must stay under
+ *            60000.  FC nets without residual connections only; otherwise, and whenever the proof fails,
+ *            TC3XTF32, or FFMA where the tensor-core path is unavailable.  cert_net_auto_contraction tells
+ *            which.  (The environment variable CERT_AUTO_FP16=0, read at create, keeps AUTO on TC3XTF32.)
  * Conv back-steps have the same fusions; under FFMA they run on the FMA units, otherwise on the TF32 tensor-core
  * kernel where their geometry allows (see cert_net_set_conv_patches).
  * (The kernels of a call are chained with programmatic dependent launch, so that a kernel's launch and set-up
@@ -221,6 +233,10 @@ cert_status_t cert_net_selftest_bounded_wait(cert_net_t *net, void *stream);
 enum { CERT_CONTRACTION_AUTO = 0, CERT_CONTRACTION_FFMA = 1, CERT_CONTRACTION_TC3XTF32 = 2,
        CERT_CONTRACTION_TC3XFP16 = 3 };
 cert_status_t cert_net_set_contraction(cert_net_t *net, int mode);
+/* The mode CERT_CONTRACTION_AUTO stands for on this net (one of the other three); -1 for a null net. */
+int cert_net_auto_contraction(const cert_net_t *net);
+/* Largest entry of the products |W_k| ... |W_j| (see AUTO above); INFINITY where no proof was attempted. */
+float cert_net_fp16_coefficient_bound(const cert_net_t *net);
 /* Which contraction kernels the most recent call ran: bit 0 = FFMA, bit 1 = TC3XTF32,
  * bit 2 = the TC3XTF32 kernel ran in its CTA-pair form (tcgen05 cta_group::2), bit 3 = a traversal ran on
  * receptive-field patches, bit 4 = TC3XFP16, bit 5 = TC3XFP16 with a whole traversal per launch (nets whose
@@ -263,6 +279,15 @@ cert_status_t cert_net_set_profiling(cert_net_t *net, int on);
 cert_status_t cert_net_profile(cert_net_t *net, float *ms_out /* HOST [CERT_N_CLASSES] */,
                                int *launches_out /* HOST [CERT_N_CLASSES] */);
 
+/*
+ * Guard words (no counterpart in the paper; memory-safety evidence).  Every device buffer the net owns
+ * (weights, coefficient matrices, row constants, relaxation and bound arrays, gathered windows, ...) is
+ * allocated with 256 guard bytes before and after it, filled with a fixed pattern at create.  This call
+ * waits for `stream` and reads all of them back: 0 = intact, i + 1 = the guard of the i-th allocation was
+ * overwritten (a kernel wrote outside its buffer), -1 = null net or a CUDA error.  Test and debugging aid.
+ */
+int cert_net_check_guards(cert_net_t *net, void *stream);
+
 /* Number of kernels the most recent cert_deeppoly_bounds call enqueued. */
 int cert_net_last_launch_count(const cert_net_t *net);
 
@@ -292,6 +317,8 @@ double cert_net_backstep_flops(const cert_net_t *net, int batch);
  * library image (every GPU that loads the library carries it until the
  * process ends).  Limit: batch * round_up(in_features, 32) <= 1048576;
  * beyond it the call returns CERT_ERR_BATCH_TOO_LARGE and does nothing.
+ * (batch * out_features beyond 8 * (2^31 - 1), more than one launch can
+ * cover, returns CERT_ERR_UNSUPPORTED.)
  *
  * The first call on each device looks up the array's device address (a
  * synchronous runtime query made with that device current); make that first

@@ -34,6 +34,7 @@ EXPORTS = [
     "cert_net_backstep_flops", "cert_status_string", "cert_net_set_profiling", "cert_net_profile",
     "cert_net_last_contraction_paths", "cert_first_layer_bounds_noalloc", "cert_net_set_conv_patches",
     "cert_net_enable_reusecert", "cert_reusecert_bounds", "cert_reusecert_bounds_host",
+    "cert_net_check_guards", "cert_net_auto_contraction", "cert_net_fp16_coefficient_bound",
 ]
 CLASS_NAMES = ["input", "relax", "relu_step", "affine", "conv", "concretize"]
 
@@ -92,6 +93,12 @@ _lib.cert_net_profile.argtypes = [_vp, _vp, _vp]
 _lib.cert_net_profile.restype = _i
 _lib.cert_first_layer_bounds_noalloc.argtypes = [_vp, _vp, _i, _i, _vp, _f, _f, _f, _i, _vp, _vp, _vp]
 _lib.cert_first_layer_bounds_noalloc.restype = _i
+_lib.cert_net_check_guards.argtypes = [_vp, _vp]
+_lib.cert_net_check_guards.restype = _i
+_lib.cert_net_auto_contraction.argtypes = [_vp]
+_lib.cert_net_auto_contraction.restype = _i
+_lib.cert_net_fp16_coefficient_bound.argtypes = [_vp]
+_lib.cert_net_fp16_coefficient_bound.restype = ctypes.c_float
 _lib.cert_status_string.argtypes = [_i]
 _lib.cert_status_string.restype = ctypes.c_char_p
 
@@ -131,6 +138,17 @@ def marshal_layers(layers: Sequence):
     return arr, keep
 
 
+def _check_tensor(name, t, shape, device=None):
+    """The kernels take raw pointers: a wrong dtype, layout, shape or device would be an out-of-bounds access."""
+    import torch
+    if not (t.is_cuda and t.dtype == torch.float32 and t.is_contiguous()):
+        raise ValueError(f"{name}: a contiguous float32 CUDA tensor is required")
+    if tuple(t.shape) != tuple(shape):
+        raise ValueError(f"{name}: shape {tuple(t.shape)}, expected {tuple(shape)}")
+    if device is not None and t.device != device:
+        raise ValueError(f"{name}: on {t.device}, expected {device}")
+
+
 class CertNet:
     """Owns a cert_net_t handle; the three calls of the C ABI plus the helpers."""
 
@@ -164,13 +182,14 @@ class CertNet:
     # -- torch tensors on the device --
     def deeppoly_bounds(self, centers, eps: float, lb_out=None, ub_out=None, stream=None):
         import torch
-        assert centers.is_cuda and centers.dtype == torch.float32 and centers.is_contiguous()
         batch = centers.shape[0]
-        assert centers.shape[1] == self.n0
+        _check_tensor("centers", centers, (batch, self.n0))
         if lb_out is None:
             lb_out = torch.empty((batch, self.n_total), dtype=torch.float32, device=centers.device)
         if ub_out is None:
             ub_out = torch.empty((batch, self.n_total), dtype=torch.float32, device=centers.device)
+        _check_tensor("lb_out", lb_out, (batch, self.n_total), centers.device)
+        _check_tensor("ub_out", ub_out, (batch, self.n_total), centers.device)
         st = stream if stream is not None else torch.cuda.current_stream(centers.device)
         self.deeppoly_bounds_ptr(centers.data_ptr(), eps, batch, lb_out.data_ptr(), ub_out.data_ptr(),
                                  st.cuda_stream)
@@ -179,13 +198,14 @@ class CertNet:
     def backsub_bounds(self, centers, eps: float, backsteps=None, lb_out=None, ub_out=None, stream=None):
         """cert_backsub_bounds: backsteps = one traversal depth per affine layer (negative: to the input)."""
         import torch
-        assert centers.is_cuda and centers.dtype == torch.float32 and centers.is_contiguous()
         batch = centers.shape[0]
-        assert centers.shape[1] == self.n0
+        _check_tensor("centers", centers, (batch, self.n0))
         if lb_out is None:
             lb_out = torch.empty((batch, self.n_total), dtype=torch.float32, device=centers.device)
         if ub_out is None:
             ub_out = torch.empty((batch, self.n_total), dtype=torch.float32, device=centers.device)
+        _check_tensor("lb_out", lb_out, (batch, self.n_total), centers.device)
+        _check_tensor("ub_out", ub_out, (batch, self.n_total), centers.device)
         st = stream if stream is not None else torch.cuda.current_stream(centers.device)
         steps = None
         if backsteps is not None:
@@ -202,13 +222,14 @@ class CertNet:
     def reusecert_bounds(self, centers, eps: float, lb_out=None, ub_out=None, stream=None):
         """cert_reusecert_bounds (enable_reusecert() first)."""
         import torch
-        assert centers.is_cuda and centers.dtype == torch.float32 and centers.is_contiguous()
         batch = centers.shape[0]
-        assert centers.shape[1] == self.n0
+        _check_tensor("centers", centers, (batch, self.n0))
         if lb_out is None:
             lb_out = torch.empty((batch, self.n_total), dtype=torch.float32, device=centers.device)
         if ub_out is None:
             ub_out = torch.empty((batch, self.n_total), dtype=torch.float32, device=centers.device)
+        _check_tensor("lb_out", lb_out, (batch, self.n_total), centers.device)
+        _check_tensor("ub_out", ub_out, (batch, self.n_total), centers.device)
         st = stream if stream is not None else torch.cuda.current_stream(centers.device)
         _check(_lib.cert_reusecert_bounds(self._h, centers.data_ptr(), float(eps), int(batch), lb_out.data_ptr(),
                                           ub_out.data_ptr(), st.cuda_stream), "cert_reusecert_bounds")
@@ -282,6 +303,16 @@ class CertNet:
     def set_conv_patches(self, on: bool):
         _check(_lib.cert_net_set_conv_patches(self._h, int(bool(on))), "cert_net_set_conv_patches")
 
+    def check_guards(self, stream_ptr: int = 0) -> int:
+        """0 = every guard word around the net's device buffers is intact, i + 1 = allocation i was overrun."""
+        return int(_lib.cert_net_check_guards(self._h, stream_ptr))
+
+    def auto_contraction(self) -> int:
+        return int(_lib.cert_net_auto_contraction(self._h))
+
+    def fp16_coefficient_bound(self) -> float:
+        return float(_lib.cert_net_fp16_coefficient_bound(self._h))
+
     def last_contraction_paths(self) -> int:
         return int(_lib.cert_net_last_contraction_paths(self._h))
 
@@ -312,8 +343,13 @@ def first_layer_bounds_noalloc(weight, bias, centers, eps, clip_lo, clip_hi, lb_
     rules on sharing.  Raises CertError on a bad argument or a batch beyond the built-in limit.
     """
     import torch
-    st = stream if stream is not None else torch.cuda.current_stream()
     out_features, in_features = weight.shape
+    batch = centers.shape[0]
+    for name, t, shape in (("weight", weight, (out_features, in_features)), ("bias", bias, (out_features,)),
+                           ("centers", centers, (batch, in_features)), ("lb_out", lb_out, (batch, out_features)),
+                           ("ub_out", ub_out, (batch, out_features))):
+        _check_tensor(name, t, shape, weight.device)
+    st = stream if stream is not None else torch.cuda.current_stream(weight.device)
     _check(_lib.cert_first_layer_bounds_noalloc(weight.data_ptr(), bias.data_ptr(), out_features, in_features,
                                                 centers.data_ptr(), float(eps), float(clip_lo), float(clip_hi),
                                                 centers.shape[0], lb_out.data_ptr(), ub_out.data_ptr(),

@@ -98,6 +98,10 @@ struct cert_net {
     int contraction = CERT_CONTRACTION_AUTO;
     std::vector<cert::LayerDev> layers;
     std::vector<void *> allocs;   // every device allocation, for destroy
+    // Guard words: every allocation is kGuardBytes longer at either end, filled with kGuardByte at create;
+    // cert_net_check_guards reads them back (a kernel that writes beyond a buffer lands there first).
+    struct Guarded { unsigned char *base; size_t bytes; };
+    std::vector<Guarded> guards;
     float *l0 = nullptr, *u0 = nullptr;      // [max_batch][ld0]
     // coefficient matrices (fp32, or the TF32 hi parts): two that alternate, and for nets with residual
     // connections a third, so that the matrix a connection sets aside stays put while the traversal goes on
@@ -109,6 +113,11 @@ struct cert_net {
     bool tc_ok = false;                      // tensor-core path usable on this net
     std::vector<TcLayer> tc;                 // per layer: operand maps and tile plan
     bool tc16_ok = false;                    // fp16-split path usable (FC layers only, CTA pairs available)
+    // AUTO takes the fp16 split: the net's weights prove that no coefficient of any traversal can leave the
+    // fp16 range (fp16_coef_bound = the largest entry of |W_k| |W_k-1| ... |W_j| over all k > j >= 1; slopes of a
+    // ReLU back-step lie in [0, 1], so every stored coefficient is below it in magnitude)
+    bool auto_fp16 = false;
+    float fp16_coef_bound = INFINITY;
     std::vector<Tc16Layer> tc16;
     // fp16-split path, narrow nets: a whole traversal per launch with the coefficient panel kept in shared memory
     bool chain_ok = false;
@@ -153,14 +162,26 @@ using cert::LayerDev;
 using cert::kPad;
 using cert::round_up;
 
+constexpr size_t kGuardBytes = 256;        // keeps the payload 256-byte aligned
+constexpr int kGuardByte = 0xA5;
+
 bool dev_alloc(cert_net *net, void **p, size_t bytes) {
     if (bytes == 0) bytes = 256;
-    if (cudaMalloc(p, bytes) != cudaSuccess) {
+    unsigned char *base = nullptr;
+    if (cudaMalloc(reinterpret_cast<void **>(&base), bytes + 2 * kGuardBytes) != cudaSuccess) {
         cudaGetLastError();
         *p = nullptr;
         return false;
     }
-    net->allocs.push_back(*p);
+    net->allocs.push_back(base);
+    if (cudaMemset(base, kGuardByte, kGuardBytes) != cudaSuccess ||
+        cudaMemset(base + kGuardBytes + bytes, kGuardByte, kGuardBytes) != cudaSuccess) {
+        cudaGetLastError();
+        *p = nullptr;
+        return false;
+    }
+    net->guards.push_back({base, bytes});
+    *p = base + kGuardBytes;
     return true;
 }
 
@@ -359,6 +380,80 @@ cert_status_t setup_tensor_core_path(cert_net *net, const cert_layer_desc_t *des
             net->chain_ok = net->chain_stages >= 2;
             net->d_slots = std::max(net->d_slots, cert::kChainColGroups);
         }
+    }
+    return CERT_OK;
+}
+
+// Range proof for the fp16 split (FC nets without residual connections).  A traversal of layer k holds, over the
+// outputs of layer j-1, the matrix W_k D W_{k-1} D ... W_j with diagonal ReLU slopes D in [0, 1] (sign-split
+// scaling never enlarges a coefficient), so each of its entries is at most the matching entry of
+// |W_k| |W_{k-1}| ... |W_j| in magnitude.  Those products are formed here, once, on the FMA units (the row
+// count is n_k, not batch * 2 * n_k); their largest entry goes to net->fp16_coef_bound.  Below kFp16Safe the
+// fp16 split cannot overflow on this net, whatever the input boxes, and AUTO takes it.
+constexpr float kFp16Safe = 60000.0f;       // fp16's largest finite value is 65504; the margin covers fp32 rounding here
+
+cert_status_t prove_fp16_range(cert_net *net) {
+    const int K = net->n_layers;
+    net->auto_fp16 = false;
+    net->fp16_coef_bound = INFINITY;
+    if (!net->tc16_ok || !net->skip_from.empty()) return CERT_OK;
+    std::vector<float *> absW(K, nullptr);
+    float *max_dev = nullptr;
+    cert_status_t rc = CERT_OK;
+    auto cleanup = [&]() {
+        for (float *p : absW) if (p) cudaFree(p);
+        if (max_dev) cudaFree(max_dev);
+    };
+    if (cudaMalloc(reinterpret_cast<void **>(&max_dev), sizeof(float)) != cudaSuccess ||
+        cudaMemset(max_dev, 0, sizeof(float)) != cudaSuccess) {
+        cudaGetLastError();
+        cleanup();
+        return CERT_ERR_OOM;
+    }
+    std::vector<float> host;
+    for (int j = 0; j < K && rc == CERT_OK; ++j) {
+        const LayerDev &L = net->layers[j];
+        const size_t n = (size_t)round_up(L.n_out, kPad) * L.ld_in;
+        host.resize(n);
+        if (cudaMemcpy(host.data(), L.W, n * sizeof(float), cudaMemcpyDeviceToHost) != cudaSuccess) { rc = CERT_ERR_CUDA; break; }
+        for (float &v : host) v = std::fabs(v);
+        if (cudaMalloc(reinterpret_cast<void **>(&absW[j]), n * sizeof(float)) != cudaSuccess) { rc = CERT_ERR_OOM; break; }
+        if (cudaMemcpy(absW[j], host.data(), n * sizeof(float), cudaMemcpyHostToDevice) != cudaSuccess) rc = CERT_ERR_CUDA;
+    }
+    for (int k = 1; k < K && rc == CERT_OK; ++k) {
+        const LayerDev &Lk = net->layers[k];
+        // the start of the traversal: |W_k| itself, rows padded like the coefficient matrices
+        const float *cur = absW[k];
+        cert::launch_absmax(cur, (long long)Lk.n_out * Lk.ld_in, max_dev, nullptr);
+        int p = 0;
+        for (int j = k - 1; j >= 1; --j) {
+            const LayerDev &Lj = net->layers[j];
+            cert::launch_gemm_ffma(cur, Lj.ld_out, absW[j], Lj.ld_in, net->buf[p], Lj.ld_in, Lk.n_out, Lj.n_in, Lj.n_out,
+                                   nullptr);
+            cert::launch_absmax(net->buf[p], (long long)Lk.n_out * Lj.ld_in, max_dev, nullptr);
+            cur = net->buf[p];
+            p ^= 1;
+        }
+    }
+    float bound = INFINITY;
+    if (rc == CERT_OK &&
+        (cudaDeviceSynchronize() != cudaSuccess ||
+         cudaMemcpy(&bound, max_dev, sizeof(float), cudaMemcpyDeviceToHost) != cudaSuccess))
+        rc = CERT_ERR_CUDA;
+    // the products went through the coefficient buffers: leave them as the kernels expect to find them (zero)
+    if (rc == CERT_OK && K > 2) {
+        size_t used = 0;
+        for (int k = 1; k < K; ++k)
+            for (int j = 1; j < k; ++j) used = std::max(used, (size_t)net->layers[k].n_out * net->layers[j].ld_in);
+        for (int p = 0; p < 2; ++p)
+            if (cudaMemset(net->buf[p], 0, used * sizeof(float)) != cudaSuccess) rc = CERT_ERR_CUDA;
+    }
+    cleanup();
+    if (rc != CERT_OK) { cudaGetLastError(); return rc; }
+    net->fp16_coef_bound = bound;
+    net->auto_fp16 = std::isfinite(bound) && bound <= kFp16Safe;
+    if (const char *e = std::getenv("CERT_AUTO_FP16")) {
+        if (std::atoi(e) == 0) net->auto_fp16 = false;
     }
     return CERT_OK;
 }
@@ -604,6 +699,542 @@ struct Recorder {
     }
 };
 
+// ---- the per-call schedule: one function per way a layer's traversal can run ----
+
+// What the schedules of one layer's traversal share.  The traversal of layer k's expressions goes through
+// layers k-1 .. j_end and is then simplified against the concrete bounds of what it has reached: the box
+// (j_end = 0), or the outputs of layer j_end-1.
+struct Traversal {
+    cert_net *net;
+    cudaStream_t st;
+    Recorder *rec;
+    int mode;                 // the contraction mode of this call (AUTO resolved)
+    int batch, k, j_end, steps;
+    long long rows;           // 2 * batch * n_k, ordered (box, side, neuron)
+    const float *box_l, *box_u;
+    float *lb_out, *ub_out;
+    int paths;                // bits of cert_net_last_contraction_paths this traversal sets
+
+    const LayerDev &layer(int j) const { return net->layers[j]; }
+    const LayerDev &Lk() const { return net->layers[k]; }
+    bool residual() const { return !net->skip_from.empty(); }
+    // Relu transformer of layer k; with `slots` its bounds are first summed from n_slots partial sums per row.
+    void relax(const float *slots, int n_slots, int slot_npos = 0) const {
+        cert::launch_relax(Lk(), lb_out, ub_out, net->n_total, batch, net->codes, net->n_relu, slots, n_slots,
+                           net->slot_stride, st, slot_npos);
+        rec->mark(CERT_CLASS_RELAX);
+    }
+};
+
+// The coefficient buffer a step writes to: the other one of two, or, in a net with residual connections, the one
+// of three that neither holds the current matrix nor the matrix a connection has set aside (`kept`, -1: none).
+int next_buffer(const Traversal &t, int cur, int kept) {
+    if (!t.residual()) return cur ^ 1;
+    int nxt = 0;
+    while (nxt == cur || nxt == kept) ++nxt;
+    return nxt;
+}
+
+// Coefficients that wait on a residual connection's source (layer `wait_for`): the matrix in buffer `kept`,
+// untouched meanwhile, or the unit coefficient of layer k's own connection (`identity`), until the step whose
+// result is over that source's outputs, where they join before the ReLU back-step.
+struct Waiting {
+    int wait_for = -1;
+    bool identity = false;
+    int kept = -1;
+    bool kept_pair = false;
+    void start(const Traversal &t) {
+        wait_for = t.residual() ? t.net->skip_from[t.k] : -1;
+        identity = wait_for >= 0;
+    }
+    // the expression is over layer j's affine neurons = W_j a_{j-1} + b_j + a_s: its matrix stays where it is
+    // as the coefficients on a_s
+    void set_aside(const Traversal &t, int j, int cur, bool pair) {
+        if (!t.residual() || t.net->skip_from[j] < 0) return;
+        wait_for = t.net->skip_from[j];
+        identity = false;
+        kept = cur;
+        kept_pair = pair;
+    }
+    void joined() { wait_for = -1; identity = false; kept = -1; }
+};
+
+// The fields every tensor-core launch of a traversal fills the same way: problem and tile sizes, the slots
+// the row constants travel in, the status word.  panel_rows = rows of a work tile's row panel.
+cert::TcArgs tc_args(const Traversal &t, int K, int n_k, int ld_n, int bn, int n_tiles, int stages, int tmem_cols,
+                     int panel_rows, int tiles_per_panel, int dcur, int dslots) {
+    cert::TcArgs a;
+    std::memset(&a, 0, sizeof(a));
+    a.M = t.rows; a.K = K; a.n_k = n_k; a.ld_n = ld_n;
+    a.bn = bn; a.n_tiles = n_tiles; a.stages = stages; a.tmem_cols = tmem_cols;
+    a.total_tiles = (int)cert::ceil_div_ll(t.rows, panel_rows) * tiles_per_panel;
+    a.d_in = t.net->dbuf[dcur]; a.n_slots_in = dslots; a.d_out = t.net->dbuf[dcur ^ 1];
+    a.slot_stride = t.net->slot_stride;
+    a.status = t.net->status_dev;
+    return a;
+}
+
+// The ReLU back-step through the neurons below layer j (relaxation of layer j-1) as a contraction's epilogue.
+void tc_relu_epilogue(cert::TcArgs &a, const LayerDev &Lb, bool split_out) {
+    a.has_relu = Lb.relu_after;
+    a.split_out = split_out ? 1 : 0;
+    a.lamL = Lb.lamL; a.lamU = Lb.lamU; a.nuU = Lb.nuU; a.bias_below = Lb.bias_n;
+}
+
+// No traversal at all: the interval step of W_k against the bounds of the layer below (IBP listing).
+void run_interval_step(Traversal &t) {
+    cert_net *net = t.net;
+    const LayerDev &Lk = t.Lk(), &Lb = t.layer(t.k - 1);
+    cert::launch_first_layer_bounds(Lk, Lb.actL, Lb.actU, Lb.ld_out, t.batch, t.lb_out, t.ub_out, net->n_total, t.st);
+    t.rec->mark(CERT_CLASS_CONCRETIZE);
+    if (t.residual() && net->skip_from[t.k] >= 0) {
+        cert::launch_add_act_bounds(Lk, t.layer(net->skip_from[t.k]), t.batch, t.lb_out, t.ub_out, net->n_total, t.st);
+        t.rec->mark(CERT_CLASS_CONCRETIZE);
+    }
+    if (Lk.relu_after || t.k + 1 < net->n_layers) t.relax(nullptr, 0);
+}
+
+// fp16 split, narrow FC nets: the whole traversal in one launch, the coefficient panel in shared memory.
+void run_chain16(Traversal &t) {
+    cert_net *net = t.net;
+    const LayerDev &Lk = t.Lk();
+    cert::ChainArgs a;
+    std::memset(&a, 0, sizeof(a));
+    a.M = t.rows; a.n_k = Lk.n_out; a.k = t.k; a.j_end = t.j_end;
+    a.Wk = Lk.W; a.ldw_k = Lk.ld_in; a.bias_k = Lk.bias_n;
+    a.box_l = t.box_l; a.box_u = t.box_u;
+    a.d_out = net->dbuf[0]; a.slot_stride = net->slot_stride;
+    a.status = net->status_dev;
+    a.stages = net->chain_stages; a.a_blocks = net->chain_a_blocks;
+    a.b_chunk_bytes = net->chain_chunk; a.vec_ld = net->chain_vec_ld;
+    const int pairs = (int)std::min<long long>(cert::ceil_div_ll(t.rows, 256), net->sm_count / 2);
+    cert::launch_chain16(net->chain, a, pairs, net->chain_smem, t.st);
+    t.rec->mark(CERT_CLASS_AFFINE);
+    t.relax(net->dbuf[0], cert::kChainColGroups);
+    t.paths |= 2 | 4 | 16 | 32;
+}
+
+// fp16 split, FC nets: the start, then one contraction per layer with the ReLU back-step fused, the last one
+// concretising.  Residual connections as in run_dense: the waiting matrix keeps its buffer.
+void run_tc16_steps(Traversal &t) {
+    cert_net *net = t.net;
+    const LayerDev &Lk = t.Lk();
+    __half *qh[3], *ql[3];
+    for (int p = 0; p < 3; ++p) {
+        qh[p] = reinterpret_cast<__half *>(net->buf[p]);
+        ql[p] = reinterpret_cast<__half *>(net->buf_lo[p]);
+    }
+    int cur = 0, dcur = 0, dslots = 1;
+    cert::launch_init_expr16(Lk, t.layer(t.k - 1), t.batch, qh[cur], ql[cur], net->dbuf[dcur], net->status_dev, t.st);
+    t.rec->mark(CERT_CLASS_RELU_STEP);
+    Waiting w;
+    w.start(t);
+    for (int j = t.k - 1; j >= t.j_end; --j) {
+        const LayerDev &Lj = t.layer(j);
+        const Tc16Layer &T = net->tc16[j];
+        w.set_aside(t, j, cur, true);
+        const int nxt = next_buffer(t, cur, w.kept);
+        const bool join = j > t.j_end && w.wait_for == j - 1;
+        cert::TcArgs a = tc_args(t, Lj.n_out, Lk.n_out, Lj.ld_in, T.plan.bn, T.plan.n_tiles, T.plan.stages,
+                                 T.plan.tmem_cols, 256, T.plan.n_tiles, dcur, dslots);
+        const int pairs = std::min(a.total_tiles, net->sm_count / 2);
+        if (j > t.j_end) {
+            tc_relu_epilogue(a, t.layer(j - 1), true);
+            if (join && w.kept >= 0) {
+                a.add_hi = reinterpret_cast<const float *>(qh[w.kept]);
+                a.add_lo = reinterpret_cast<const float *>(ql[w.kept]);
+            }
+            a.add_identity = (join && w.identity) ? 1 : 0;
+            cert::launch_gemm_tc16(cert::TC_EPI_RELU, pairs, T.a_hi[cur], T.a_lo[cur], T.b_hi, T.b_lo, T.o_hi[nxt],
+                                   T.o_lo[nxt], a, T.plan.smem_bytes, t.st);
+            if (join) w.joined();
+        } else {
+            a.l0 = t.box_l; a.u0 = t.box_u;
+            cert::launch_gemm_tc16(cert::TC_EPI_CONCRETIZE, pairs, T.a_hi[cur], T.a_lo[cur], T.b_hi, T.b_lo,
+                                   T.a_hi[cur], T.a_lo[cur], a, T.plan.smem_bytes, t.st);
+        }
+        t.rec->mark(CERT_CLASS_AFFINE);
+        cur = nxt;
+        dcur ^= 1;
+        dslots = 2 * T.plan.n_tiles;
+    }
+    t.relax(net->dbuf[dcur], dslots);
+    t.paths |= 2 | 4 | 16;
+}
+
+// A conv layer over conv layers, rows as receptive-field patches, every step as a contraction with the conv
+// layer's window-to-window matrix on the tensor cores.
+void run_patches_tc(Traversal &t, const cert::PatchLevel *lv) {
+    cert_net *net = t.net;
+    const LayerDev &Lk = t.Lk();
+    const std::vector<TcPatchStep> &SS = net->tcp[t.k];
+    const int ctas = net->tc_ctas;
+    int cur = 0, dcur = 0, dslots = 1;
+    cert::launch_patch_start(Lk, t.layer(t.k - 1), SS[0].Kp, t.batch, net->buf[cur], net->buf_lo[cur], net->dbuf[dcur],
+                             t.st);
+    t.rec->mark(CERT_CLASS_RELU_STEP);
+    for (int j = t.k - 1, m = 0; j >= t.j_end; --j, ++m) {
+        const LayerDev &Lj = t.layer(j);
+        const TcPatchStep &S = SS[m];
+        const float *src[3] = {nullptr, nullptr, nullptr};
+        const float fill[3] = {1.0f, 1.0f, 0.0f};
+        int n_arr = 3;
+        if (j > t.j_end) {
+            const LayerDev &Lb = t.layer(j - 1);
+            if (Lb.relu_after) { src[0] = Lb.lamL; src[1] = Lb.lamU; src[2] = Lb.nuU; }
+        } else {
+            src[0] = t.box_l; src[1] = t.box_u;
+            n_arr = 2;
+        }
+        cert::launch_patch_gather(Lk, Lj, lv[m + 1], S.ldN, t.batch, n_arr, src, fill, net->gat, t.st);
+        t.rec->mark(CERT_CLASS_CONV);
+        // rows are ordered (box, position, side, channel): with "box" = (box, position) and c_out neurons
+        // per box this is the usual row order, and the gathered vectors are per such box
+        cert::TcArgs a = tc_args(t, S.Kp, Lk.c_out, S.ldN, S.plan.bn, S.plan.n_tiles, S.plan.stages, S.plan.tmem_cols,
+                                 128 * ctas, S.plan.n_tiles, dcur, dslots);
+        const int groups = std::min(a.total_tiles, net->sm_count / ctas);
+        if (j > t.j_end) {
+            a.has_relu = 1;          // the gathered slopes also blank the window outside the map
+            a.split_out = 1;
+            a.lamL = net->gat[0]; a.lamU = net->gat[1]; a.nuU = net->gat[2]; a.bias_below = S.bias_e;
+            cert::launch_gemm_tc(cert::TC_EPI_RELU, ctas, groups, S.a_hi[cur], S.a_lo[cur], S.b_hi, S.b_lo,
+                                 S.o_hi[cur ^ 1], S.o_lo[cur ^ 1], a, S.plan.smem_bytes, t.st);
+        } else {
+            a.l0 = net->gat[0]; a.u0 = net->gat[1];
+            cert::launch_gemm_tc(cert::TC_EPI_CONCRETIZE, ctas, groups, S.a_hi[cur], S.a_lo[cur], S.b_hi, S.b_lo,
+                                 S.a_hi[cur], S.a_lo[cur], a, S.plan.smem_bytes, t.st);
+        }
+        t.rec->mark(CERT_CLASS_CONV);
+        cur ^= 1;
+        dcur ^= 1;
+        dslots = S.plan.n_tiles;
+    }
+    t.relax(net->dbuf[dcur], dslots, Lk.h_out * Lk.w_out);
+    t.paths |= 8 | 2 | (ctas == 2 ? 4 : 0);
+}
+
+// The same traversal with the patch steps on the FMA units (one warp per row).
+void run_patches_fma(Traversal &t, const cert::PatchLevel *lv) {
+    cert_net *net = t.net;
+    const LayerDev &Lk = t.Lk();
+    int cur = 0;
+    const int dcur = 0;
+    cert::launch_patch_start(Lk, t.layer(t.k - 1), lv[0].pitch, t.batch, net->buf[cur], nullptr, net->dbuf[dcur], t.st);
+    t.rec->mark(CERT_CLASS_RELU_STEP);
+    for (int j = t.k - 1, m = 0; j >= t.j_end; --j, ++m) {
+        cert::ConvtEpilogue ep;
+        std::memset(&ep, 0, sizeof(ep));
+        ep.n_k = Lk.n_out;
+        ep.d_in = net->dbuf[dcur]; ep.n_slots_in = 1; ep.slot_stride = net->slot_stride;
+        ep.d_out = net->dbuf[dcur];
+        if (j > t.j_end) {
+            const LayerDev &Lb = t.layer(j - 1);
+            ep.mode = cert::CONVT_EPI_RELU;
+            ep.has_relu = Lb.relu_after;
+            ep.lamL = Lb.lamL; ep.lamU = Lb.lamU; ep.nuU = Lb.nuU; ep.bias_below = Lb.bias_n;
+            ep.P = net->buf[cur ^ 1];
+        } else {
+            ep.mode = cert::CONVT_EPI_CONCRETIZE;
+            ep.l0 = t.box_l; ep.u0 = t.box_u;
+            ep.lb_out = t.lb_out; ep.ub_out = t.ub_out; ep.n_total = net->n_total; ep.out_off = Lk.out_off;
+        }
+        cert::launch_patch_step(Lk, t.layer(j), lv[m], lv[m + 1], net->buf[cur], t.rows, net->sm_count, ep, t.st);
+        t.rec->mark(CERT_CLASS_CONV);
+        cur ^= 1;
+    }
+    if (Lk.relu_after || t.k + 1 < net->n_layers) t.relax(nullptr, 0);
+    t.paths |= 8;
+}
+
+// Everything else: dense coefficient matrices, one launch per back-step (3xTF32 contraction, banded conv form,
+// FMA conv kernel, or the FMA chain of contraction + ReLU step), residual connections included.
+void run_dense(Traversal &t) {
+    cert_net *net = t.net;
+    const LayerDev &Lk = t.Lk();
+    const int K = net->n_layers, k = t.k, j_end = t.j_end, n_total = net->n_total;
+    const bool residual = t.residual();
+    cudaStream_t st = t.st;
+    Recorder &rec = *t.rec;
+    int cur = 0;      // coefficient buffer that holds the current expression
+    int dcur = 0;     // constant buffer, and how many of its slots are live
+    int dslots = 1;
+    bool bounds_in_slots = false;
+    // Does the back-step through layer j run on the tensor cores?  Its input must then be a TF32 pair.
+    auto on_tc = [&](int j) { return t.mode != CERT_CONTRACTION_FFMA && net->tc_ok && net->tc[j].usable; };
+    // ... or, for a conv layer on dense maps, in the banded tensor-core form?  Its input is a TF32 pair too.
+    auto on_band = [&](int j) {
+        return t.mode != CERT_CONTRACTION_FFMA && net->tc_ok && net->band[j].usable &&
+               (!residual || (net->band_residual_ok && t.steps == k));      // (residual nets: full traversals)
+    };
+    auto wants_pair = [&](int j) { return on_tc(j) || on_band(j); };
+
+    // expression over the outputs of layer k-1, pushed through its ReLU
+    bool y_major = false;     // the coefficient maps are held [y][channel][x] (banded conv steps)
+    if (Lk.kind == CERT_LAYER_FC && on_band(k - 1) && net->band[k - 1].W_above_y) {
+        // an FC layer right above a banded conv layer: the same start with the columns of W_k, the relaxation
+        // and the bias below in y-major order writes the first matrix in the layout the banded steps read
+        const LayerDev &Lb = t.layer(k - 1);
+        const BandStep &S = net->band[k - 1];
+        const float *src[3] = {nullptr, nullptr, nullptr};
+        const float fill[3] = {1.0f, 1.0f, 0.0f};
+        if (Lb.relu_after) { src[0] = Lb.lamL; src[1] = Lb.lamU; src[2] = Lb.nuU; }
+        cert::launch_to_ymajor_vectors(Lb.c_out, Lb.h_out, Lb.w_out, Lb.ld_out, t.batch, 3, src, fill, net->gat, st);
+        rec.mark(CERT_CLASS_RELU_STEP);
+        LayerDev Lk_y = Lk, Lb_y = Lb;
+        Lk_y.W = S.W_above_y;
+        Lb_y.lamL = net->gat[0]; Lb_y.lamU = net->gat[1]; Lb_y.nuU = net->gat[2];
+        Lb_y.bias_n = S.bias_out_y;
+        Lb_y.relu_after = 1;
+        cert::launch_init_expr(Lk_y, Lb_y, t.batch, net->buf[cur], net->buf_lo[cur], net->dbuf[dcur], st);
+        y_major = true;
+    } else {
+        // a conv layer right above a banded conv layer places its window coefficients at their y-major columns
+        y_major = Lk.kind == CERT_LAYER_CONV2D && on_band(k - 1);
+        cert::launch_init_expr(Lk, t.layer(k - 1), t.batch, net->buf[cur],
+                               wants_pair(k - 1) ? net->buf_lo[cur] : nullptr, net->dbuf[dcur], st, y_major);
+    }
+    rec.mark(CERT_CLASS_RELU_STEP);
+    Waiting w;
+    w.start(t);
+    for (int j = k - 1; j >= j_end; --j) {
+        const LayerDev &Lj = t.layer(j);
+        w.set_aside(t, j, cur, wants_pair(j));
+        int nxt = next_buffer(t, cur, w.kept);
+        // The last step of a traversal that stops on the very neurons a connection waits for: the
+        // coefficients join before the simplification, so the step stores its result and the unfused
+        // concretisation follows.
+        const bool join_end = residual && j == j_end && j_end > 0 && w.wait_for == j_end - 1;
+        const bool join = (j > j_end && w.wait_for == j - 1) || join_end;
+        const bool store_step = j > j_end || join_end;
+        const float *add_hi = (join && w.kept >= 0) ? net->buf[w.kept] : nullptr;
+        const float *add_lo = (join && w.kept >= 0 && w.kept_pair) ? net->buf_lo[w.kept] : nullptr;
+        const int add_identity = (join && w.identity) ? 1 : 0;
+        if (Lj.kind == CERT_LAYER_CONV2D && on_band(j)) {
+            // dense coefficient maps through conv layer j on the tensor cores, band by band
+            const BandStep &S = net->band[j];
+            const int ctas = net->tc_ctas;
+            if (!y_major) {
+                cert::launch_to_ymajor_pair(net->buf[cur], net->buf_lo[cur], net->buf[nxt], net->buf_lo[nxt], t.rows,
+                                            Lj.c_out, Lj.h_out, Lj.w_out, Lj.ld_out, st);
+                rec.mark(CERT_CLASS_CONV);
+                if (w.kept == cur) w.kept = nxt;      // a matrix set aside at this very layer: its y-major copy waits
+                cur = nxt;
+                nxt = next_buffer(t, cur, w.kept);
+                y_major = true;
+            }
+            const float *src[3] = {nullptr, nullptr, nullptr};
+            const float fill[3] = {1.0f, 1.0f, 0.0f};
+            int n_arr = 3;
+            if (j > j_end) {
+                const LayerDev &Lb = t.layer(j - 1);
+                if (Lb.relu_after) { src[0] = Lb.lamL; src[1] = Lb.lamU; src[2] = Lb.nuU; }
+            } else {
+                src[0] = t.box_l; src[1] = t.box_u;
+                n_arr = 2;
+            }
+            cert::launch_to_ymajor_vectors(Lj.c_in, Lj.h_in, Lj.w_in, Lj.ld_in, t.batch, n_arr, src, fill, net->gat, st);
+            rec.mark(CERT_CLASS_CONV);
+            cert::TcArgs a = tc_args(t, S.K, Lk.n_out, Lj.ld_in, S.plan.bn, S.plan.n_tiles, S.plan.stages,
+                                     S.plan.tmem_cols, 128 * ctas, S.n_bands * S.plan.n_tiles, dcur, dslots);
+            a.n_bands = S.n_bands; a.band_rin = S.rin; a.band_o_shift = S.o_shift; a.band_h_in = Lj.h_out;
+            a.band_row_in = Lj.c_out * Lj.w_out;
+            a.band_s = Lj.stride; a.band_y_shift = S.y_shift; a.band_row_out = Lj.c_in * Lj.w_in;
+            const int groups = std::min(a.total_tiles, net->sm_count / ctas);
+            if (j > j_end) {
+                a.has_relu = 1;
+                a.split_out = 1;          // a banded step follows
+                a.lamL = net->gat[0]; a.lamU = net->gat[1]; a.nuU = net->gat[2]; a.bias_below = S.bias_y;
+                if (join && w.kept >= 0) { a.add_hi = net->buf[w.kept]; a.add_lo = net->buf_lo[w.kept]; }
+                a.add_identity = add_identity;
+                a.band_c_out = Lj.c_in; a.band_h_out = Lj.h_in; a.band_w_out = Lj.w_in;
+                cert::launch_gemm_tc(cert::TC_EPI_RELU_BAND, ctas, groups, S.a_hi[cur], S.a_lo[cur], S.b_hi, S.b_lo,
+                                     S.o_hi[nxt], S.o_lo[nxt], a, S.plan.smem_bytes, st);
+                if (join) w.joined();
+            } else {
+                a.l0 = net->gat[0]; a.u0 = net->gat[1];
+                cert::launch_gemm_tc(cert::TC_EPI_CONCRETIZE_BAND, ctas, groups, S.a_hi[cur], S.a_lo[cur], S.b_hi,
+                                     S.b_lo, S.a_hi[cur], S.a_lo[cur], a, S.plan.smem_bytes, st);
+                bounds_in_slots = true;
+            }
+            rec.mark(CERT_CLASS_CONV);
+            t.paths |= 2 | (ctas == 2 ? 4 : 0) | 64;
+            cur = nxt;
+            dcur ^= 1;
+            dslots = S.n_bands * S.plan.n_tiles;
+            continue;
+        }
+        float *Q = net->buf[cur], *P = net->buf[nxt];
+        float *P_lo = (j > j_end && wants_pair(j - 1)) ? net->buf_lo[nxt] : nullptr;
+        if (on_tc(j)) {
+            const TcLayer &T = net->tc[j];
+            const int ctas = net->tc_ctas;
+            cert::TcArgs a = tc_args(t, Lj.n_out, Lk.n_out, Lj.ld_in, T.plan.bn, T.plan.n_tiles, T.plan.stages,
+                                     T.plan.tmem_cols, 128 * ctas, T.plan.n_tiles, dcur, dslots);
+            const int groups = std::min(a.total_tiles, net->sm_count / ctas);
+            if (store_step) {
+                tc_relu_epilogue(a, t.layer(j - 1), P_lo != nullptr);
+                if (join_end) { a.has_relu = 0; a.bias_below = net->zeros; }
+                a.add_hi = add_hi; a.add_lo = add_lo; a.add_identity = add_identity;
+                cert::launch_gemm_tc(cert::TC_EPI_RELU, ctas, groups, T.a_hi[cur], T.a_lo[cur], T.b_hi, T.b_lo,
+                                     T.o_hi[nxt], T.o_lo[nxt], a, T.plan.smem_bytes, st);
+            } else {
+                a.l0 = t.box_l; a.u0 = t.box_u;
+                cert::launch_gemm_tc(cert::TC_EPI_CONCRETIZE, ctas, groups, T.a_hi[cur], T.a_lo[cur], T.b_hi, T.b_lo,
+                                     T.a_hi[cur], T.a_lo[cur], a, T.plan.smem_bytes, st);
+                bounds_in_slots = true;
+            }
+            rec.mark(CERT_CLASS_AFFINE);
+            t.paths |= 2 | (ctas == 2 ? 4 : 0);
+            if (join) w.joined();
+            cur = nxt;
+            dcur ^= 1;
+            dslots = T.plan.n_tiles;
+            if (join_end) {
+                cert::launch_concretize(P, net->dbuf[dcur], dslots, net->slot_stride, t.box_l, t.box_u, Lj.n_in,
+                                        Lj.ld_in, t.batch, Lk.n_out, t.lb_out, t.ub_out, n_total, Lk.out_off, st);
+                rec.mark(CERT_CLASS_CONCRETIZE);
+            }
+            continue;
+        }
+        if (Lj.kind == CERT_LAYER_CONV2D) {
+            // conv back-step with what follows it fused: the ReLU back-step below, or the concretisation
+            cert::ConvtEpilogue ep;
+            std::memset(&ep, 0, sizeof(ep));
+            ep.n_k = Lk.n_out;
+            ep.d_in = net->dbuf[dcur]; ep.n_slots_in = dslots; ep.slot_stride = net->slot_stride;
+            ep.d_out = net->dbuf[dcur];
+            if (store_step) {
+                const LayerDev &Lb = t.layer(j - 1);
+                ep.mode = cert::CONVT_EPI_RELU;
+                ep.has_relu = join_end ? 0 : Lb.relu_after;
+                ep.lamL = Lb.lamL; ep.lamU = Lb.lamU; ep.nuU = Lb.nuU;
+                ep.bias_below = join_end ? net->zeros : Lb.bias_n;
+                ep.P = P; ep.P_lo = P_lo;
+                ep.add_hi = add_hi; ep.add_lo = add_lo; ep.add_identity = add_identity;
+            } else {
+                ep.mode = cert::CONVT_EPI_CONCRETIZE;
+                ep.l0 = t.box_l; ep.u0 = t.box_u;
+                ep.lb_out = t.lb_out; ep.ub_out = t.ub_out; ep.n_total = n_total; ep.out_off = Lk.out_off;
+            }
+            cert::launch_convt_ffma(Lj, Q, t.rows, net->sm_count, ep, st);
+            rec.mark(CERT_CLASS_CONV);
+            if (join) w.joined();
+            cur = nxt;
+            dslots = 1;
+            if (join_end) {
+                cert::launch_concretize(P, net->dbuf[dcur], dslots, net->slot_stride, t.box_l, t.box_u, Lj.n_in,
+                                        Lj.ld_in, t.batch, Lk.n_out, t.lb_out, t.ub_out, n_total, Lk.out_off, st);
+                rec.mark(CERT_CLASS_CONCRETIZE);
+            }
+            continue;
+        }
+        // FC layer on the FMA units: contraction, then the ReLU back-step or the concretisation as kernels of their own
+        cert::launch_gemm_ffma(Q, Lj.ld_out, Lj.W, Lj.ld_in, P, Lj.ld_in, t.rows, Lj.n_in, Lj.n_out, st);
+        rec.mark(CERT_CLASS_AFFINE);
+        t.paths |= 1;
+        cur = nxt;
+        if (join) {
+            cert::launch_add_skip(P, add_hi, add_lo, add_identity, t.rows, Lj.n_in, Lj.ld_in, Lk.n_out, st);
+            rec.mark(CERT_CLASS_RELU_STEP);
+            w.joined();
+        }
+        if (j > j_end) {
+            cert::launch_relu_step(t.layer(j - 1), t.batch, Lk.n_out, P, P_lo, net->dbuf[dcur], dslots,
+                                   net->slot_stride, st);
+            dslots = 1;
+            rec.mark(CERT_CLASS_RELU_STEP);
+        } else {
+            cert::launch_concretize(P, net->dbuf[dcur], dslots, net->slot_stride, t.box_l, t.box_u, Lj.n_in, Lj.ld_in,
+                                    t.batch, Lk.n_out, t.lb_out, t.ub_out, n_total, Lk.out_off, st);
+            rec.mark(CERT_CLASS_CONCRETIZE);
+        }
+    }
+    if (residual && w.wait_for >= 0) {
+        // the traversal stopped above the connection's source: the waiting neurons are simplified against
+        // their own concrete bounds
+        const float *S_hi = w.kept >= 0 ? net->buf[w.kept] : nullptr;
+        const float *S_lo = (w.kept >= 0 && w.kept_pair) ? net->buf_lo[w.kept] : nullptr;
+        float *slot = nullptr;
+        if (bounds_in_slots) {
+            slot = net->dbuf[dcur] + (size_t)dslots * net->slot_stride;
+            ++dslots;
+        }
+        cert::launch_skip_concretize(S_hi, S_lo, w.identity ? 1 : 0, t.layer(w.wait_for), t.rows, Lk, slot, t.lb_out,
+                                     t.ub_out, n_total, st);
+        rec.mark(CERT_CLASS_CONCRETIZE);
+    }
+    if (Lk.relu_after || bounds_in_slots || k + 1 < K) t.relax(bounds_in_slots ? net->dbuf[dcur] : nullptr, dslots);
+}
+
+// The contraction mode one call runs in.  AUTO: the fp16 split where the net's weights prove that no coefficient
+// can leave the fp16 range (cert_net::auto_fp16), else the TF32 split; `forced` >= 0 overrides the net's setting.
+int call_mode(const cert_net *net, int forced) {
+    int mode = forced >= 0 ? forced : net->contraction;
+    if (mode == CERT_CONTRACTION_AUTO && net->auto_fp16) mode = CERT_CONTRACTION_TC3XFP16;
+    return mode;
+}
+
+// flow(forward) over the layers: the bounds of the first layer against the box, then for every affine layer its
+// traversal in whichever schedule takes it, then the Relu transformer.
+cert_status_t backsub_impl(cert_net *net, const float *centers, float eps, int batch, const int *backsteps,
+                           float *lb_out, float *ub_out, cudaStream_t st, int forced_mode) {
+    if (!net || !centers || !lb_out || !ub_out) return CERT_ERR_INVALID_ARG;
+    if (batch < 1 || !(eps >= 0.0f) || std::isinf(eps)) return CERT_ERR_INVALID_ARG;
+    if (batch > net->max_batch) return CERT_ERR_BATCH_TOO_LARGE;
+    const int K = net->n_layers;
+    const int mode = call_mode(net, forced_mode);
+    const bool residual = !net->skip_from.empty();
+    if (residual && backsteps && mode == CERT_CONTRACTION_TC3XFP16)
+        for (int k = 1; k < K; ++k)
+            if (backsteps[k] >= 0 && backsteps[k] < k) return CERT_ERR_UNSUPPORTED;   // fp16 split: full traversals only
+    Recorder rec(net, st);
+    int paths = 0;
+
+    cert::launch_box(centers, eps, net->clip_lo, net->clip_hi, batch, net->n0, net->ld0, net->l0, net->u0, st);
+    rec.mark(CERT_CLASS_INPUT);
+    cert::launch_first_layer_bounds(net->layers[0], net->l0, net->u0, net->ld0, batch, lb_out, ub_out, net->n_total, st);
+    rec.mark(CERT_CLASS_INPUT);
+    if (net->layers[0].relu_after || K > 1) {
+        cert::launch_relax(net->layers[0], lb_out, ub_out, net->n_total, batch, net->codes, net->n_relu, nullptr, 0, 0,
+                           st);
+        rec.mark(CERT_CLASS_RELAX);
+    }
+    for (int k = 1; k < K; ++k) {
+        Traversal t;
+        t.net = net; t.st = st; t.rec = &rec; t.mode = mode; t.batch = batch; t.k = k;
+        t.steps = (backsteps && backsteps[k] >= 0) ? std::min(backsteps[k], k) : k;
+        t.j_end = k - t.steps;
+        t.rows = 2LL * batch * net->layers[k].n_out;
+        t.box_l = t.j_end == 0 ? net->l0 : net->layers[t.j_end - 1].actL;
+        t.box_u = t.j_end == 0 ? net->u0 : net->layers[t.j_end - 1].actU;
+        t.lb_out = lb_out; t.ub_out = ub_out;
+        t.paths = 0;
+        cert::PatchLevel lv[kMaxPatchLevels];
+        if (t.steps == 0) {
+            run_interval_step(t);
+        } else if (mode == CERT_CONTRACTION_TC3XFP16 && net->chain_ok) {
+            run_chain16(t);
+        } else if (mode == CERT_CONTRACTION_TC3XFP16 && net->tc16_ok) {
+            run_tc16_steps(t);
+        } else if (net->conv_patches && cert::conv_patch_plan(net->layers.data(), k, t.j_end, lv, kMaxPatchLevels)) {
+            if (mode != CERT_CONTRACTION_FFMA && (int)net->tcp[k].size() >= t.steps) run_patches_tc(t, lv);
+            else run_patches_fma(t, lv);
+        } else {
+            run_dense(t);
+        }
+        paths |= t.paths;
+    }
+    net->last_batch = batch;
+    net->last_launches = rec.launches;
+    net->last_paths = paths;
+    net->prof_marks = rec.marks;
+    if (cudaPeekAtLastError() != cudaSuccess) {
+        cudaGetLastError();
+        return CERT_ERR_CUDA;
+    }
+    return CERT_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -622,15 +1253,8 @@ const char *cert_status_string(cert_status_t s) {
     return "unknown";
 }
 
-cert_status_t cert_net_create(const cert_layer_desc_t *layers, int n_layers, int max_batch, float clip_lo,
-                              float clip_hi, cert_net_t **out) {
-    return cert_net_create_residual(layers, n_layers, nullptr, max_batch, clip_lo, clip_hi, out);
-}
-
-cert_status_t cert_net_create_residual(const cert_layer_desc_t *layers, int n_layers, const int *skip_from,
-                                       int max_batch, float clip_lo, float clip_hi, cert_net_t **out) {
-    if (!out) return CERT_ERR_INVALID_ARG;
-    *out = nullptr;
+static cert_status_t create_impl(const cert_layer_desc_t *layers, int n_layers, const int *skip_from, int max_batch,
+                                 float clip_lo, float clip_hi, cert_net_t **out, cert_net **partial) {
     cert_status_t v = validate(layers, n_layers, max_batch, clip_lo, clip_hi);
     if (v != CERT_OK) return v;
     bool any_skip = false;
@@ -654,6 +1278,7 @@ cert_status_t cert_net_create_residual(const cert_layer_desc_t *layers, int n_la
 
     cert_net *net = new (std::nothrow) cert_net;
     if (!net) return CERT_ERR_OOM;
+    *partial = net;                     // the caller frees it if anything below throws
     net->device = dev;
     {
         cudaDeviceProp prop;
@@ -778,6 +1403,7 @@ cert_status_t cert_net_create_residual(const cert_layer_desc_t *layers, int n_la
         if (!ok) fail = CERT_ERR_OOM;
         net->slot_stride = (long long)max_rows;
         if (ok) fail = setup_tensor_core_path(net, layers, max_elems);
+        if (ok && fail == CERT_OK) fail = prove_fp16_range(net);
         if (ok && fail == CERT_OK) fail = setup_patch_tc(net, layers);
         if (ok && fail == CERT_OK) fail = setup_band_tc(net, layers);
         if (ok && fail == CERT_OK && net->gat_floats)
@@ -800,6 +1426,7 @@ cert_status_t cert_net_create_residual(const cert_layer_desc_t *layers, int n_la
         cert::conv_patch_prepare();
         if (cudaDeviceSynchronize() != cudaSuccess) fail = CERT_ERR_CUDA;
     }
+    *partial = nullptr;
     if (fail != CERT_OK) {
         cudaGetLastError();
         free_net(net);
@@ -809,6 +1436,32 @@ cert_status_t cert_net_create_residual(const cert_layer_desc_t *layers, int n_la
     return CERT_OK;
 }
 
+cert_status_t cert_net_create(const cert_layer_desc_t *layers, int n_layers, int max_batch, float clip_lo,
+                              float clip_hi, cert_net_t **out) {
+    return cert_net_create_residual(layers, n_layers, nullptr, max_batch, clip_lo, clip_hi, out);
+}
+
+cert_status_t cert_net_create_residual(const cert_layer_desc_t *layers, int n_layers, const int *skip_from,
+                                       int max_batch, float clip_lo, float clip_hi, cert_net_t **out) {
+    if (!out) return CERT_ERR_INVALID_ARG;
+    *out = nullptr;
+    // the set-up code builds host vectors: a failed host allocation must come back as a status, not cross the C ABI
+    cert_net *partial = nullptr;
+    try {
+        return create_impl(layers, n_layers, skip_from, max_batch, clip_lo, clip_hi, out, &partial);
+    } catch (const std::bad_alloc &) {
+    } catch (...) {
+        cudaGetLastError();
+        if (partial) free_net(partial);
+        *out = nullptr;
+        return CERT_ERR_CUDA;
+    }
+    cudaGetLastError();
+    if (partial) free_net(partial);
+    *out = nullptr;
+    return CERT_ERR_OOM;
+}
+
 cert_status_t cert_deeppoly_bounds(cert_net_t *net, const float *centers, float eps, int batch, float *lb_out,
                                    float *ub_out, void *stream) {
     return cert_backsub_bounds(net, centers, eps, batch, nullptr, lb_out, ub_out, stream);
@@ -816,493 +1469,29 @@ cert_status_t cert_deeppoly_bounds(cert_net_t *net, const float *centers, float 
 
 cert_status_t cert_backsub_bounds(cert_net_t *net, const float *centers, float eps, int batch,
                                   const int *backsteps, float *lb_out, float *ub_out, void *stream) {
-    if (!net || !centers || !lb_out || !ub_out) return CERT_ERR_INVALID_ARG;
-    if (batch < 1 || !(eps >= 0.0f) || std::isinf(eps)) return CERT_ERR_INVALID_ARG;
-    if (batch > net->max_batch) return CERT_ERR_BATCH_TOO_LARGE;
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const int K = net->n_layers;
-    const int n_total = net->n_total;
-    const bool residual = !net->skip_from.empty();
-    if (residual && backsteps && net->contraction == CERT_CONTRACTION_TC3XFP16)
-        for (int k = 1; k < K; ++k)
-            if (backsteps[k] >= 0 && backsteps[k] < k) return CERT_ERR_UNSUPPORTED;   // fp16 split: full traversals only
-    Recorder rec(net, st);
-    int paths = 0;
-
-    cert::launch_box(centers, eps, net->clip_lo, net->clip_hi, batch, net->n0, net->ld0, net->l0, net->u0, st);
-    rec.mark(CERT_CLASS_INPUT);
-    cert::launch_first_layer_bounds(net->layers[0], net->l0, net->u0, net->ld0, batch, lb_out, ub_out, n_total, st);
-    rec.mark(CERT_CLASS_INPUT);
-    if (net->layers[0].relu_after || K > 1) {
-        cert::launch_relax(net->layers[0], lb_out, ub_out, n_total, batch, net->codes, net->n_relu, nullptr, 0, 0,
-                           st);
-        rec.mark(CERT_CLASS_RELAX);
-    }
-    for (int k = 1; k < K; ++k) {
-        const LayerDev &Lk = net->layers[k];
-        const long long rows = 2LL * batch * Lk.n_out;
-        // The traversal of layer k's expressions goes through layers k-1 .. j_end and is then simplified
-        // against the concrete bounds of what it has reached: the box (j_end = 0), or the outputs of
-        // layer j_end-1.  With no step at all the bounds are the interval step of W_k.
-        const int steps = (backsteps && backsteps[k] >= 0) ? std::min(backsteps[k], k) : k;
-        const int j_end = k - steps;
-        if (steps == 0) {
-            const LayerDev &Lb = net->layers[k - 1];
-            cert::launch_first_layer_bounds(Lk, Lb.actL, Lb.actU, Lb.ld_out, batch, lb_out, ub_out, n_total, st);
-            rec.mark(CERT_CLASS_CONCRETIZE);
-            if (residual && net->skip_from[k] >= 0) {
-                cert::launch_add_act_bounds(Lk, net->layers[net->skip_from[k]], batch, lb_out, ub_out, n_total, st);
-                rec.mark(CERT_CLASS_CONCRETIZE);
-            }
-            if (Lk.relu_after || k + 1 < K) {
-                cert::launch_relax(Lk, lb_out, ub_out, n_total, batch, net->codes, net->n_relu, nullptr, 0, 0, st);
-                rec.mark(CERT_CLASS_RELAX);
-            }
-            continue;
-        }
-        const float *box_l = j_end == 0 ? net->l0 : net->layers[j_end - 1].actL;
-        const float *box_u = j_end == 0 ? net->u0 : net->layers[j_end - 1].actU;
-        int cur = 0;      // coefficient buffer that holds the current expression
-        int dcur = 0;     // constant buffer, and how many of its slots are live
-        int dslots = 1;
-        bool bounds_in_slots = false;
-        // Does the back-step through layer j run on the tensor cores?  Its input must then be a TF32 pair.
-        auto on_tc = [&](int j) {
-            return net->contraction != CERT_CONTRACTION_FFMA && net->tc_ok && net->tc[j].usable;
-        };
-        // ... or, for a conv layer on dense maps, in the banded tensor-core form?  Its input is a TF32 pair too.
-        auto on_band = [&](int j) {
-            return net->contraction != CERT_CONTRACTION_FFMA && net->tc_ok && net->band[j].usable &&
-                   (!residual || (net->band_residual_ok && steps == k));      // (residual nets: full traversals)
-        };
-        auto wants_pair = [&](int j) { return on_tc(j) || on_band(j); };
-        // fp16-split tensor-core chain (FC nets): start, then one kernel per layer with the ReLU step fused,
-        // the last one concretising.
-        if (net->contraction == CERT_CONTRACTION_TC3XFP16 && net->chain_ok) {
-            cert::ChainArgs a;
-            std::memset(&a, 0, sizeof(a));
-            a.M = rows; a.n_k = Lk.n_out; a.k = k; a.j_end = j_end;
-            a.Wk = Lk.W; a.ldw_k = Lk.ld_in; a.bias_k = Lk.bias_n;
-            a.box_l = box_l; a.box_u = box_u;
-            a.d_out = net->dbuf[0]; a.slot_stride = net->slot_stride;
-            a.status = net->status_dev;
-            a.stages = net->chain_stages; a.a_blocks = net->chain_a_blocks;
-            a.b_chunk_bytes = net->chain_chunk; a.vec_ld = net->chain_vec_ld;
-            const int pairs = (int)std::min<long long>(cert::ceil_div_ll(rows, 256), net->sm_count / 2);
-            cert::launch_chain16(net->chain, a, pairs, net->chain_smem, st);
-            rec.mark(CERT_CLASS_AFFINE);
-            cert::launch_relax(Lk, lb_out, ub_out, n_total, batch, net->codes, net->n_relu, net->dbuf[0], cert::kChainColGroups,
-                               net->slot_stride, st);
-            rec.mark(CERT_CLASS_RELAX);
-            paths |= 2 | 4 | 16 | 32;
-            continue;
-        }
-        if (net->contraction == CERT_CONTRACTION_TC3XFP16 && net->tc16_ok) {
-            __half *qh[3] = {reinterpret_cast<__half *>(net->buf[0]), reinterpret_cast<__half *>(net->buf[1]),
-                             reinterpret_cast<__half *>(net->buf[2])};
-            __half *ql[3] = {reinterpret_cast<__half *>(net->buf_lo[0]), reinterpret_cast<__half *>(net->buf_lo[1]),
-                             reinterpret_cast<__half *>(net->buf_lo[2])};
-            cert::launch_init_expr16(Lk, net->layers[k - 1], batch, qh[cur], ql[cur], net->dbuf[dcur], net->status_dev, st);
-            rec.mark(CERT_CLASS_RELU_STEP);
-            // residual connections as in the TF32 schedule below: the waiting matrix keeps its buffer
-            int wait_for = residual ? net->skip_from[k] : -1;
-            bool wait_identity = wait_for >= 0;
-            int kept = -1;
-            for (int j = k - 1; j >= j_end; --j) {
-                const LayerDev &Lj = net->layers[j];
-                const Tc16Layer &T = net->tc16[j];
-                if (residual && net->skip_from[j] >= 0) {
-                    wait_for = net->skip_from[j];
-                    wait_identity = false;
-                    kept = cur;
-                }
-                int nxt = cur ^ 1;
-                if (residual) {
-                    nxt = 0;
-                    while (nxt == cur || nxt == kept) ++nxt;
-                }
-                const bool join = j > j_end && wait_for == j - 1;
-                cert::TcArgs a;
-                std::memset(&a, 0, sizeof(a));
-                a.M = rows; a.K = Lj.n_out; a.n_k = Lk.n_out; a.ld_n = Lj.ld_in;
-                a.bn = T.plan.bn; a.n_tiles = T.plan.n_tiles; a.stages = T.plan.stages; a.tmem_cols = T.plan.tmem_cols;
-                a.total_tiles = (int)cert::ceil_div_ll(rows, 256) * T.plan.n_tiles;
-                a.d_in = net->dbuf[dcur]; a.n_slots_in = dslots; a.d_out = net->dbuf[dcur ^ 1];
-                a.slot_stride = net->slot_stride;
-                a.status = net->status_dev;
-                const int pairs = std::min(a.total_tiles, net->sm_count / 2);
-                if (j > j_end) {
-                    const LayerDev &Lb = net->layers[j - 1];
-                    a.has_relu = Lb.relu_after;
-                    a.split_out = 1;
-                    a.lamL = Lb.lamL; a.lamU = Lb.lamU; a.nuU = Lb.nuU; a.bias_below = Lb.bias_n;
-                    if (join && kept >= 0) {
-                        a.add_hi = reinterpret_cast<const float *>(qh[kept]);
-                        a.add_lo = reinterpret_cast<const float *>(ql[kept]);
-                    }
-                    a.add_identity = (join && wait_identity) ? 1 : 0;
-                    cert::launch_gemm_tc16(cert::TC_EPI_RELU, pairs, T.a_hi[cur], T.a_lo[cur], T.b_hi, T.b_lo,
-                                           T.o_hi[nxt], T.o_lo[nxt], a, T.plan.smem_bytes, st);
-                    if (join) { wait_for = -1; wait_identity = false; kept = -1; }
-                } else {
-                    a.l0 = box_l; a.u0 = box_u;
-                    cert::launch_gemm_tc16(cert::TC_EPI_CONCRETIZE, pairs, T.a_hi[cur], T.a_lo[cur], T.b_hi, T.b_lo,
-                                           T.a_hi[cur], T.a_lo[cur], a, T.plan.smem_bytes, st);
-                }
-                rec.mark(CERT_CLASS_AFFINE);
-                cur = nxt;
-                dcur ^= 1;
-                dslots = 2 * T.plan.n_tiles;
-            }
-            cert::launch_relax(Lk, lb_out, ub_out, n_total, batch, net->codes, net->n_relu, net->dbuf[dcur], dslots,
-                               net->slot_stride, st);
-            rec.mark(CERT_CLASS_RELAX);
-            paths |= 2 | 4 | 16;
-            continue;
-        }
-        // A conv layer over conv layers: rows as receptive-field patches instead of dense maps.
-        cert::PatchLevel lv[kMaxPatchLevels];
-        const bool patches = net->conv_patches && cert::conv_patch_plan(net->layers.data(), k, j_end, lv, kMaxPatchLevels);
-        if (patches && net->contraction != CERT_CONTRACTION_FFMA && (int)net->tcp[k].size() >= steps) {
-            // every step of the traversal as a contraction with the conv layer's window-to-window matrix
-            const std::vector<TcPatchStep> &SS = net->tcp[k];
-            const int ctas = net->tc_ctas;
-            cert::launch_patch_start(Lk, net->layers[k - 1], SS[0].Kp, batch, net->buf[cur], net->buf_lo[cur],
-                                     net->dbuf[dcur], st);
-            rec.mark(CERT_CLASS_RELU_STEP);
-            for (int j = k - 1, m = 0; j >= j_end; --j, ++m) {
-                const LayerDev &Lj = net->layers[j];
-                const TcPatchStep &S = SS[m];
-                const float *src[3] = {nullptr, nullptr, nullptr};
-                const float fill[3] = {1.0f, 1.0f, 0.0f};
-                int n_arr = 3;
-                if (j > j_end) {
-                    const LayerDev &Lb = net->layers[j - 1];
-                    if (Lb.relu_after) { src[0] = Lb.lamL; src[1] = Lb.lamU; src[2] = Lb.nuU; }
-                } else {
-                    src[0] = box_l; src[1] = box_u;
-                    n_arr = 2;
-                }
-                cert::launch_patch_gather(Lk, Lj, lv[m + 1], S.ldN, batch, n_arr, src, fill, net->gat, st);
-                rec.mark(CERT_CLASS_CONV);
-                cert::TcArgs a;
-                std::memset(&a, 0, sizeof(a));
-                // rows are ordered (box, position, side, channel): with "box" = (box, position) and c_out neurons
-                // per box this is the usual row order, and the gathered vectors are per such box
-                a.M = rows; a.K = S.Kp; a.n_k = Lk.c_out; a.ld_n = S.ldN;
-                a.bn = S.plan.bn; a.n_tiles = S.plan.n_tiles; a.stages = S.plan.stages;
-                a.tmem_cols = S.plan.tmem_cols;
-                a.total_tiles = (int)cert::ceil_div_ll(rows, 128 * ctas) * S.plan.n_tiles;
-                a.d_in = net->dbuf[dcur]; a.n_slots_in = dslots; a.d_out = net->dbuf[dcur ^ 1];
-                a.slot_stride = net->slot_stride;
-                a.status = net->status_dev;
-                const int groups = std::min(a.total_tiles, net->sm_count / ctas);
-                if (j > j_end) {
-                    a.has_relu = 1;          // the gathered slopes also blank the window outside the map
-                    a.split_out = 1;
-                    a.lamL = net->gat[0]; a.lamU = net->gat[1]; a.nuU = net->gat[2]; a.bias_below = S.bias_e;
-                    cert::launch_gemm_tc(cert::TC_EPI_RELU, ctas, groups, S.a_hi[cur], S.a_lo[cur], S.b_hi, S.b_lo,
-                                         S.o_hi[cur ^ 1], S.o_lo[cur ^ 1], a, S.plan.smem_bytes, st);
-                } else {
-                    a.l0 = net->gat[0]; a.u0 = net->gat[1];
-                    cert::launch_gemm_tc(cert::TC_EPI_CONCRETIZE, ctas, groups, S.a_hi[cur], S.a_lo[cur], S.b_hi,
-                                         S.b_lo, S.a_hi[cur], S.a_lo[cur], a, S.plan.smem_bytes, st);
-                }
-                rec.mark(CERT_CLASS_CONV);
-                cur ^= 1;
-                dcur ^= 1;
-                dslots = S.plan.n_tiles;
-            }
-            cert::launch_relax(Lk, lb_out, ub_out, n_total, batch, net->codes, net->n_relu, net->dbuf[dcur], dslots,
-                               net->slot_stride, st, Lk.h_out * Lk.w_out);
-            rec.mark(CERT_CLASS_RELAX);
-            paths |= 8 | 2 | (ctas == 2 ? 4 : 0);
-            continue;
-        }
-        if (patches) {
-            cert::launch_patch_start(Lk, net->layers[k - 1], lv[0].pitch, batch, net->buf[cur], nullptr,
-                                     net->dbuf[dcur], st);
-            rec.mark(CERT_CLASS_RELU_STEP);
-            for (int j = k - 1, m = 0; j >= j_end; --j, ++m) {
-                const LayerDev &Lj = net->layers[j];
-                cert::ConvtEpilogue ep;
-                std::memset(&ep, 0, sizeof(ep));
-                ep.n_k = Lk.n_out;
-                ep.d_in = net->dbuf[dcur]; ep.n_slots_in = 1; ep.slot_stride = net->slot_stride;
-                ep.d_out = net->dbuf[dcur];
-                if (j > j_end) {
-                    const LayerDev &Lb = net->layers[j - 1];
-                    ep.mode = cert::CONVT_EPI_RELU;
-                    ep.has_relu = Lb.relu_after;
-                    ep.lamL = Lb.lamL; ep.lamU = Lb.lamU; ep.nuU = Lb.nuU; ep.bias_below = Lb.bias_n;
-                    ep.P = net->buf[cur ^ 1];
-                } else {
-                    ep.mode = cert::CONVT_EPI_CONCRETIZE;
-                    ep.l0 = box_l; ep.u0 = box_u;
-                    ep.lb_out = lb_out; ep.ub_out = ub_out; ep.n_total = n_total; ep.out_off = Lk.out_off;
-                }
-                cert::launch_patch_step(Lk, Lj, lv[m], lv[m + 1], net->buf[cur], rows, net->sm_count, ep, st);
-                rec.mark(CERT_CLASS_CONV);
-                cur ^= 1;
-            }
-            if (Lk.relu_after || k + 1 < K) {
-                cert::launch_relax(Lk, lb_out, ub_out, n_total, batch, net->codes, net->n_relu, nullptr, 0, 0, st);
-                rec.mark(CERT_CLASS_RELAX);
-            }
-            paths |= 8;
-            continue;
-        }
-        // expression over the outputs of layer k-1, pushed through its ReLU
-        bool y_major = false;     // the coefficient maps are held [y][channel][x] (banded conv steps)
-        if (Lk.kind == CERT_LAYER_FC && on_band(k - 1) && net->band[k - 1].W_above_y) {
-            // an FC layer right above a banded conv layer: the same start with the columns of W_k, the relaxation
-            // and the bias below in y-major order writes the first matrix in the layout the banded steps read
-            const LayerDev &Lb = net->layers[k - 1];
-            const BandStep &S = net->band[k - 1];
-            const float *src[3] = {nullptr, nullptr, nullptr};
-            const float fill[3] = {1.0f, 1.0f, 0.0f};
-            if (Lb.relu_after) { src[0] = Lb.lamL; src[1] = Lb.lamU; src[2] = Lb.nuU; }
-            cert::launch_to_ymajor_vectors(Lb.c_out, Lb.h_out, Lb.w_out, Lb.ld_out, batch, 3, src, fill, net->gat, st);
-            rec.mark(CERT_CLASS_RELU_STEP);
-            LayerDev Lk_y = Lk, Lb_y = Lb;
-            Lk_y.W = S.W_above_y;
-            Lb_y.lamL = net->gat[0]; Lb_y.lamU = net->gat[1]; Lb_y.nuU = net->gat[2];
-            Lb_y.bias_n = S.bias_out_y;
-            Lb_y.relu_after = 1;
-            cert::launch_init_expr(Lk_y, Lb_y, batch, net->buf[cur], net->buf_lo[cur], net->dbuf[dcur], st);
-            y_major = true;
-        } else {
-            // a conv layer right above a banded conv layer places its window coefficients at their y-major columns
-            y_major = Lk.kind == CERT_LAYER_CONV2D && on_band(k - 1);
-            cert::launch_init_expr(Lk, net->layers[k - 1], batch, net->buf[cur],
-                                   wants_pair(k - 1) ? net->buf_lo[cur] : nullptr, net->dbuf[dcur], st, y_major);
-        }
-        rec.mark(CERT_CLASS_RELU_STEP);
-        // Residual connections: the coefficients on a connection's source wait (kept: the buffer that holds
-        // them, untouched meanwhile; identity: the unit coefficient of layer k's own connection) until the
-        // step whose result is over that source's outputs, where they join before the ReLU back-step.
-        int wait_for = residual ? net->skip_from[k] : -1;
-        bool wait_identity = wait_for >= 0;
-        int kept = -1;
-        bool kept_pair = false;
-        for (int j = k - 1; j >= j_end; --j) {
-            const LayerDev &Lj = net->layers[j];
-            if (residual && net->skip_from[j] >= 0) {
-                // the expression is over layer j's affine neurons = W_j a_{j-1} + b_j + a_s: its matrix stays
-                // where it is as the coefficients on a_s
-                wait_for = net->skip_from[j];
-                wait_identity = false;
-                kept = cur;
-                kept_pair = wants_pair(j);
-            }
-            int nxt = cur ^ 1;
-            if (residual) {
-                nxt = 0;
-                while (nxt == cur || nxt == kept) ++nxt;
-            }
-            // The last step of a traversal that stops on the very neurons a connection waits for: the
-            // coefficients join before the simplification, so the step stores its result and the unfused
-            // concretisation follows.
-            const bool join_end = residual && j == j_end && j_end > 0 && wait_for == j_end - 1;
-            const bool join = (j > j_end && wait_for == j - 1) || join_end;
-            const bool store_step = j > j_end || join_end;
-            const float *add_hi = (join && kept >= 0) ? net->buf[kept] : nullptr;
-            const float *add_lo = (join && kept >= 0 && kept_pair) ? net->buf_lo[kept] : nullptr;
-            const int add_identity = (join && wait_identity) ? 1 : 0;
-            float *Q = net->buf[cur], *P = net->buf[nxt];
-            float *P_lo = (j > j_end && wants_pair(j - 1)) ? net->buf_lo[nxt] : nullptr;
-            if (Lj.kind == CERT_LAYER_CONV2D && on_band(j)) {
-                // dense coefficient maps through conv layer j on the tensor cores, band by band
-                const BandStep &S = net->band[j];
-                const int ctas = net->tc_ctas;
-                if (!y_major) {
-                    cert::launch_to_ymajor_pair(net->buf[cur], net->buf_lo[cur], net->buf[nxt], net->buf_lo[nxt], rows,
-                                                Lj.c_out, Lj.h_out, Lj.w_out, Lj.ld_out, st);
-                    rec.mark(CERT_CLASS_CONV);
-                    if (kept == cur) kept = nxt;      // a matrix set aside at this very layer: its y-major copy waits
-                    cur = nxt;
-                    nxt = cur ^ 1;
-                    if (residual) {
-                        nxt = 0;
-                        while (nxt == cur || nxt == kept) ++nxt;
-                    }
-                    y_major = true;
-                }
-                const float *src[3] = {nullptr, nullptr, nullptr};
-                const float fill[3] = {1.0f, 1.0f, 0.0f};
-                int n_arr = 3;
-                if (j > j_end) {
-                    const LayerDev &Lb = net->layers[j - 1];
-                    if (Lb.relu_after) { src[0] = Lb.lamL; src[1] = Lb.lamU; src[2] = Lb.nuU; }
-                } else {
-                    src[0] = box_l; src[1] = box_u;
-                    n_arr = 2;
-                }
-                cert::launch_to_ymajor_vectors(Lj.c_in, Lj.h_in, Lj.w_in, Lj.ld_in, batch, n_arr, src, fill, net->gat, st);
-                rec.mark(CERT_CLASS_CONV);
-                cert::TcArgs a;
-                std::memset(&a, 0, sizeof(a));
-                a.M = rows; a.K = S.K; a.n_k = Lk.n_out; a.ld_n = Lj.ld_in;
-                a.n_bands = S.n_bands; a.band_rin = S.rin; a.band_o_shift = S.o_shift; a.band_h_in = Lj.h_out;
-                a.band_row_in = Lj.c_out * Lj.w_out;
-                a.band_s = Lj.stride; a.band_y_shift = S.y_shift; a.band_row_out = Lj.c_in * Lj.w_in;
-                a.bn = S.plan.bn; a.n_tiles = S.plan.n_tiles; a.stages = S.plan.stages;
-                a.tmem_cols = S.plan.tmem_cols;
-                a.total_tiles = (int)cert::ceil_div_ll(rows, 128 * ctas) * S.n_bands * S.plan.n_tiles;
-                a.d_in = net->dbuf[dcur]; a.n_slots_in = dslots; a.d_out = net->dbuf[dcur ^ 1];
-                a.slot_stride = net->slot_stride;
-                a.status = net->status_dev;
-                const int groups = std::min(a.total_tiles, net->sm_count / ctas);
-                if (j > j_end) {
-                    a.has_relu = 1;
-                    a.split_out = 1;          // a banded step follows
-                    a.lamL = net->gat[0]; a.lamU = net->gat[1]; a.nuU = net->gat[2]; a.bias_below = S.bias_y;
-                    if (join && kept >= 0) { a.add_hi = net->buf[kept]; a.add_lo = net->buf_lo[kept]; }
-                    a.add_identity = add_identity;
-                    a.band_c_out = Lj.c_in; a.band_h_out = Lj.h_in; a.band_w_out = Lj.w_in;
-                    cert::launch_gemm_tc(cert::TC_EPI_RELU_BAND, ctas, groups, S.a_hi[cur], S.a_lo[cur], S.b_hi, S.b_lo,
-                                         S.o_hi[nxt], S.o_lo[nxt], a, S.plan.smem_bytes, st);
-                    if (join) { wait_for = -1; wait_identity = false; kept = -1; }
-                } else {
-                    a.l0 = net->gat[0]; a.u0 = net->gat[1];
-                    cert::launch_gemm_tc(cert::TC_EPI_CONCRETIZE_BAND, ctas, groups, S.a_hi[cur], S.a_lo[cur], S.b_hi,
-                                         S.b_lo, S.a_hi[cur], S.a_lo[cur], a, S.plan.smem_bytes, st);
-                    bounds_in_slots = true;
-                }
-                rec.mark(CERT_CLASS_CONV);
-                paths |= 2 | (ctas == 2 ? 4 : 0) | 64;
-                cur = nxt;
-                dcur ^= 1;
-                dslots = S.n_bands * S.plan.n_tiles;
-                continue;
-            }
-            if (on_tc(j)) {
-                const TcLayer &T = net->tc[j];
-                cert::TcArgs a;
-                std::memset(&a, 0, sizeof(a));
-                a.M = rows; a.K = Lj.n_out; a.n_k = Lk.n_out; a.ld_n = Lj.ld_in;
-                a.bn = T.plan.bn; a.n_tiles = T.plan.n_tiles; a.stages = T.plan.stages;
-                a.tmem_cols = T.plan.tmem_cols;
-                const int ctas = net->tc_ctas;
-                a.total_tiles = (int)cert::ceil_div_ll(rows, 128 * ctas) * T.plan.n_tiles;
-                a.d_in = net->dbuf[dcur]; a.n_slots_in = dslots; a.d_out = net->dbuf[dcur ^ 1];
-                a.slot_stride = net->slot_stride;
-                a.status = net->status_dev;
-                const int groups = std::min(a.total_tiles, net->sm_count / ctas);
-                if (store_step) {
-                    const LayerDev &Lb = net->layers[j - 1];
-                    a.has_relu = join_end ? 0 : Lb.relu_after;
-                    a.split_out = P_lo != nullptr;
-                    a.lamL = Lb.lamL; a.lamU = Lb.lamU; a.nuU = Lb.nuU;
-                    a.bias_below = join_end ? net->zeros : Lb.bias_n;
-                    a.add_hi = add_hi; a.add_lo = add_lo; a.add_identity = add_identity;
-                    cert::launch_gemm_tc(cert::TC_EPI_RELU, ctas, groups, T.a_hi[cur], T.a_lo[cur], T.b_hi, T.b_lo,
-                                         T.o_hi[nxt], T.o_lo[nxt], a, T.plan.smem_bytes, st);
-                } else {
-                    a.l0 = box_l; a.u0 = box_u;
-                    cert::launch_gemm_tc(cert::TC_EPI_CONCRETIZE, ctas, groups, T.a_hi[cur], T.a_lo[cur], T.b_hi,
-                                         T.b_lo, T.a_hi[cur], T.a_lo[cur], a, T.plan.smem_bytes, st);
-                    bounds_in_slots = true;
-                }
-                rec.mark(CERT_CLASS_AFFINE);
-                paths |= 2 | (net->tc_ctas == 2 ? 4 : 0);
-                if (join) { wait_for = -1; wait_identity = false; kept = -1; }
-                cur = nxt;
-                dcur ^= 1;
-                dslots = T.plan.n_tiles;
-                if (join_end) {
-                    cert::launch_concretize(P, net->dbuf[dcur], dslots, net->slot_stride, box_l, box_u, Lj.n_in,
-                                            Lj.ld_in, batch, Lk.n_out, lb_out, ub_out, n_total, Lk.out_off, st);
-                    rec.mark(CERT_CLASS_CONCRETIZE);
-                }
-                continue;
-            }
-            if (Lj.kind == CERT_LAYER_CONV2D) {
-                // conv back-step with what follows it fused: the ReLU back-step below, or the concretisation
-                cert::ConvtEpilogue ep;
-                std::memset(&ep, 0, sizeof(ep));
-                ep.n_k = Lk.n_out;
-                ep.d_in = net->dbuf[dcur]; ep.n_slots_in = dslots; ep.slot_stride = net->slot_stride;
-                ep.d_out = net->dbuf[dcur];
-                if (store_step) {
-                    const LayerDev &Lb = net->layers[j - 1];
-                    ep.mode = cert::CONVT_EPI_RELU;
-                    ep.has_relu = join_end ? 0 : Lb.relu_after;
-                    ep.lamL = Lb.lamL; ep.lamU = Lb.lamU; ep.nuU = Lb.nuU;
-                    ep.bias_below = join_end ? net->zeros : Lb.bias_n;
-                    ep.P = P; ep.P_lo = P_lo;
-                    ep.add_hi = add_hi; ep.add_lo = add_lo; ep.add_identity = add_identity;
-                } else {
-                    ep.mode = cert::CONVT_EPI_CONCRETIZE;
-                    ep.l0 = box_l; ep.u0 = box_u;
-                    ep.lb_out = lb_out; ep.ub_out = ub_out; ep.n_total = n_total; ep.out_off = Lk.out_off;
-                }
-                cert::launch_convt_ffma(Lj, Q, rows, net->sm_count, ep, st);
-                rec.mark(CERT_CLASS_CONV);
-                if (join) { wait_for = -1; wait_identity = false; kept = -1; }
-                cur = nxt;
-                dslots = 1;
-                if (join_end) {
-                    cert::launch_concretize(P, net->dbuf[dcur], dslots, net->slot_stride, box_l, box_u, Lj.n_in,
-                                            Lj.ld_in, batch, Lk.n_out, lb_out, ub_out, n_total, Lk.out_off, st);
-                    rec.mark(CERT_CLASS_CONCRETIZE);
-                }
-                continue;
-            }
-            cert::launch_gemm_ffma(Q, Lj.ld_out, Lj.W, Lj.ld_in, P, Lj.ld_in, rows, Lj.n_in, Lj.n_out, st);
-            rec.mark(CERT_CLASS_AFFINE);
-            paths |= 1;
-            cur = nxt;
-            if (join) {
-                cert::launch_add_skip(P, add_hi, add_lo, add_identity, rows, Lj.n_in, Lj.ld_in, Lk.n_out, st);
-                rec.mark(CERT_CLASS_RELU_STEP);
-                wait_for = -1; wait_identity = false; kept = -1;
-            }
-            if (j > j_end) {
-                cert::launch_relu_step(net->layers[j - 1], batch, Lk.n_out, P, P_lo, net->dbuf[dcur], dslots,
-                                       net->slot_stride, st);
-                dslots = 1;
-                rec.mark(CERT_CLASS_RELU_STEP);
-            } else {
-                cert::launch_concretize(P, net->dbuf[dcur], dslots, net->slot_stride, box_l, box_u, Lj.n_in,
-                                        Lj.ld_in, batch, Lk.n_out, lb_out, ub_out, n_total, Lk.out_off, st);
-                rec.mark(CERT_CLASS_CONCRETIZE);
-            }
-        }
-        if (residual && wait_for >= 0) {
-            // the traversal stopped above the connection's source: the waiting neurons are simplified against
-            // their own concrete bounds
-            const float *S_hi = kept >= 0 ? net->buf[kept] : nullptr;
-            const float *S_lo = (kept >= 0 && kept_pair) ? net->buf_lo[kept] : nullptr;
-            float *slot = nullptr;
-            if (bounds_in_slots) {
-                slot = net->dbuf[dcur] + (size_t)dslots * net->slot_stride;
-                ++dslots;
-            }
-            cert::launch_skip_concretize(S_hi, S_lo, wait_identity ? 1 : 0, net->layers[wait_for], rows, Lk, slot,
-                                         lb_out, ub_out, n_total, st);
-            rec.mark(CERT_CLASS_CONCRETIZE);
-        }
-        if (Lk.relu_after || bounds_in_slots || k + 1 < K) {
-            cert::launch_relax(Lk, lb_out, ub_out, n_total, batch, net->codes, net->n_relu,
-                               bounds_in_slots ? net->dbuf[dcur] : nullptr, dslots, net->slot_stride, st);
-            rec.mark(CERT_CLASS_RELAX);
-        }
-    }
-    net->last_batch = batch;
-    net->last_launches = rec.launches;
-    net->last_paths = paths;
-    net->prof_marks = rec.marks;
-    if (cudaPeekAtLastError() != cudaSuccess) {
-        cudaGetLastError();
-        return CERT_ERR_CUDA;
-    }
-    return CERT_OK;
+    return backsub_impl(net, centers, eps, batch, backsteps, lb_out, ub_out, static_cast<cudaStream_t>(stream), -1);
 }
 
 cert_status_t cert_deeppoly_bounds_host(cert_net_t *net, const float *centers_host, float eps, int batch,
                                         float *lb_host, float *ub_host, void *stream) {
     return cert_backsub_bounds_host(net, centers_host, eps, batch, nullptr, lb_host, ub_host, stream);
+}
+
+// Reads the sticky status word after the stream has drained; clears it when set.
+static cert_status_t read_status(cert_net *net, cudaStream_t st, int *flag_out) {
+    int flag = 0;
+    if (cudaMemcpyAsync(&flag, net->status_dev, sizeof(int), cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+        cudaStreamSynchronize(st) != cudaSuccess) {
+        cudaGetLastError();
+        return CERT_ERR_CUDA;
+    }
+    if (flag != 0 && (cudaMemsetAsync(net->status_dev, 0, sizeof(int), st) != cudaSuccess ||
+                      cudaStreamSynchronize(st) != cudaSuccess)) {
+        cudaGetLastError();
+        return CERT_ERR_CUDA;
+    }
+    *flag_out = flag;
+    return CERT_OK;
 }
 
 cert_status_t cert_backsub_bounds_host(cert_net_t *net, const float *centers_host, float eps, int batch,
@@ -1317,18 +1506,49 @@ cert_status_t cert_backsub_bounds_host(cert_net_t *net, const float *centers_hos
         cudaGetLastError();
         return CERT_ERR_CUDA;
     }
-    cert_status_t s = cert_backsub_bounds(net, net->centers_dev, eps, batch, backsteps, net->lb_dev, net->ub_dev, stream);
-    if (s != CERT_OK) return s;
-    if (cudaMemcpyAsync(lb_host, net->lb_dev, out_bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
-        cudaMemcpyAsync(ub_host, net->ub_dev, out_bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
-        cudaStreamSynchronize(st) != cudaSuccess) {
+    // This call waits for its results anyway, so it also reads the device's status word: bounds that a run-out
+    // wait or an fp16 overflow invalidated are never handed back as a success.  Under AUTO an overflow (which
+    // the create-time range proof rules out; this is the second line of defence) re-runs the call in the TF32 split.
+    int forced = -1;
+    for (int attempt = 0; attempt < 2; ++attempt) {
+        cert_status_t s = backsub_impl(net, net->centers_dev, eps, batch, backsteps, net->lb_dev, net->ub_dev, st, forced);
+        if (s != CERT_OK) return s;
+        if (cudaMemcpyAsync(lb_host, net->lb_dev, out_bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+            cudaMemcpyAsync(ub_host, net->ub_dev, out_bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) {
+            cudaGetLastError();
+            return CERT_ERR_CUDA;
+        }
+        int flag = 0;
+        s = read_status(net, st, &flag);
+        if (s != CERT_OK) return s;
+        if (flag & 1) return CERT_ERR_TIMEOUT;
+        if (flag & 2) {
+            if (net->contraction == CERT_CONTRACTION_AUTO && attempt == 0 && net->tc_ok) {
+                forced = CERT_CONTRACTION_TC3XTF32;
+                continue;
+            }
+            return CERT_ERR_RANGE;
+        }
+        return CERT_OK;
+    }
+    return CERT_ERR_RANGE;
+}
+
+static cert_status_t enable_reusecert_impl(cert_net_t *net);
+
+cert_status_t cert_net_enable_reusecert(cert_net_t *net) {
+    try {
+        return enable_reusecert_impl(net);
+    } catch (const std::bad_alloc &) {
+        cudaGetLastError();
+        return CERT_ERR_OOM;        // what was allocated so far belongs to the net and goes with it
+    } catch (...) {
         cudaGetLastError();
         return CERT_ERR_CUDA;
     }
-    return CERT_OK;
 }
 
-cert_status_t cert_net_enable_reusecert(cert_net_t *net) {
+static cert_status_t enable_reusecert_impl(cert_net_t *net) {
     if (!net) return CERT_ERR_INVALID_ARG;
     if (net->reuse.on) return CERT_OK;
     const int K = net->n_layers;
@@ -1591,11 +1811,15 @@ cert_status_t cert_reusecert_bounds_host(cert_net_t *net, const float *centers_h
     cert_status_t s = cert_reusecert_bounds(net, net->centers_dev, eps, batch, net->lb_dev, net->ub_dev, stream);
     if (s != CERT_OK) return s;
     if (cudaMemcpyAsync(lb_host, net->lb_dev, out_bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
-        cudaMemcpyAsync(ub_host, net->ub_dev, out_bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
-        cudaStreamSynchronize(st) != cudaSuccess) {
+        cudaMemcpyAsync(ub_host, net->ub_dev, out_bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) {
         cudaGetLastError();
         return CERT_ERR_CUDA;
     }
+    int flag = 0;
+    s = read_status(net, st, &flag);
+    if (s != CERT_OK) return s;
+    if (flag & 1) return CERT_ERR_TIMEOUT;
+    if (flag & 2) return CERT_ERR_RANGE;
     return CERT_OK;
 }
 
@@ -1629,20 +1853,38 @@ cert_status_t cert_net_branch_codes(cert_net_t *net, unsigned char *codes_out, v
 
 cert_status_t cert_net_last_status(cert_net_t *net, void *stream) {
     if (!net) return CERT_ERR_INVALID_ARG;
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
     int flag = 0;
-    if (cudaMemcpyAsync(&flag, net->status_dev, sizeof(int), cudaMemcpyDeviceToHost, st) != cudaSuccess ||
-        cudaStreamSynchronize(st) != cudaSuccess) {
-        cudaGetLastError();
-        return CERT_ERR_CUDA;
-    }
-    if (flag != 0) {
-        cudaMemsetAsync(net->status_dev, 0, sizeof(int), st);
-        cudaStreamSynchronize(st);
-        return (flag & 1) ? CERT_ERR_TIMEOUT : CERT_ERR_RANGE;
-    }
+    cert_status_t s = read_status(net, static_cast<cudaStream_t>(stream), &flag);
+    if (s != CERT_OK) return s;
+    if (flag != 0) return (flag & 1) ? CERT_ERR_TIMEOUT : CERT_ERR_RANGE;
     return CERT_OK;
 }
+
+int cert_net_check_guards(cert_net_t *net, void *stream) {
+    if (!net) return -1;
+    if (cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess) { cudaGetLastError(); return -1; }
+    unsigned char host[2 * kGuardBytes];
+    for (size_t i = 0; i < net->guards.size(); ++i) {
+        const cert_net::Guarded &g = net->guards[i];
+        if (cudaMemcpy(host, g.base, kGuardBytes, cudaMemcpyDeviceToHost) != cudaSuccess ||
+            cudaMemcpy(host + kGuardBytes, g.base + kGuardBytes + g.bytes, kGuardBytes, cudaMemcpyDeviceToHost) !=
+                cudaSuccess) {
+            cudaGetLastError();
+            return -1;
+        }
+        for (size_t b = 0; b < 2 * kGuardBytes; ++b)
+            if (host[b] != kGuardByte) return (int)i + 1;
+    }
+    return 0;
+}
+
+int cert_net_auto_contraction(const cert_net_t *net) {
+    if (!net) return -1;
+    if (net->auto_fp16) return CERT_CONTRACTION_TC3XFP16;
+    return net->tc_ok ? CERT_CONTRACTION_TC3XTF32 : CERT_CONTRACTION_FFMA;
+}
+
+float cert_net_fp16_coefficient_bound(const cert_net_t *net) { return net ? net->fp16_coef_bound : -1.0f; }
 
 cert_status_t cert_net_set_contraction(cert_net_t *net, int mode) {
     if (!net) return CERT_ERR_INVALID_ARG;

@@ -72,6 +72,9 @@ inline ConvGeom geom_of(const LayerDev &L) {
 
 // ---- launch wrappers (each enqueues exactly one kernel on `st`) ----
 
+// *out = max(*out, max |x[i]|) for *out >= 0 (set-up time: the range proof of the fp16 split).
+void launch_absmax(const float *x, long long n, float *out, cudaStream_t st);
+
 // l0 = max(c - eps, lo), u0 = min(c + eps, hi); rows padded with zeros.
 void launch_box(const float *centers, float eps, float lo, float hi, int batch, int n0, int ld0,
                 float *l0, float *u0, cudaStream_t st);

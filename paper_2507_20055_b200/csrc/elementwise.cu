@@ -3,6 +3,7 @@
 // ReLU back-step and the unfused concretisation.  One warp owns one row of a
 // coefficient matrix; row sums are warp-shuffle trees, so every result is
 // deterministic.
+#include <algorithm>
 #include <cstdlib>
 
 #include "common.cuh"
@@ -535,7 +536,23 @@ inline unsigned grid_for_warps(long long warps) {
     return (unsigned)ceil_div_ll(warps, kWarpsPerBlock);
 }
 
+// Largest |x| of an array, into *out (which the caller has set to zero or an earlier maximum): the bit pattern
+// of a non-negative float orders like the integer it is.
+__global__ void absmax_kernel(const float *__restrict__ x, long long n, float *__restrict__ out) {
+    float m = 0.0f;
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x)
+        m = fmaxf(m, fabsf(x[i]));
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+    if ((threadIdx.x & 31) == 0) atomicMax(reinterpret_cast<unsigned int *>(out), __float_as_uint(m));
+}
+
 }  // namespace
+
+void launch_absmax(const float *x, long long n, float *out, cudaStream_t st) {
+    const int blocks = (int)std::min<long long>(ceil_div_ll(n, 256), 1184);
+    absmax_kernel<<<blocks, 256, 0, st>>>(x, n, out);
+}
 
 // Multiprocessors of the current device (looked up once).
 static int sm_count() {

@@ -18,8 +18,10 @@ sgemm_nn_kernel(const float *__restrict__ A, int lda, const float *__restrict__ 
     __shared__ __align__(16) float As[2][BK][BM];
     __shared__ __align__(16) float Bs[2][BK][BN];
     const int tid = threadIdx.x;
-    const long long row0 = (long long)blockIdx.y * BM;
-    const int col0 = blockIdx.x * BN;
+    // one-dimensional grid (row tile major): the y extent of a grid stops at 65535 tiles, rows do not
+    const int col_tiles = (ldc + BN - 1) / BN;
+    const long long row0 = (long long)(blockIdx.x / col_tiles) * BM;
+    const int col0 = (int)(blockIdx.x % col_tiles) * BN;
     const int ty = tid / 16, tx = tid % 16;
 
     // global -> register staging
@@ -91,8 +93,18 @@ sgemm_nn_kernel(const float *__restrict__ A, int lda, const float *__restrict__ 
 void launch_gemm_ffma(const float *A, int lda, const float *B, int ldb, float *C, int ldc, long long M, int N,
                       int K, cudaStream_t st) {
     (void)N;
-    dim3 grid((unsigned)((ldc + BN - 1) / BN), (unsigned)ceil_div_ll(M, BM));
-    sgemm_nn_kernel<<<grid, 256, 0, st>>>(A, lda, B, ldb, C, ldc, M, K);
+    const long long col_tiles = (ldc + BN - 1) / BN;
+    long long row_tiles_left = ceil_div_ll(M, BM);
+    const long long max_row_tiles = 0x7FFFFFFFLL / col_tiles;      // blocks of one launch: at most 2^31 - 1
+    long long row0 = 0;
+    while (row_tiles_left > 0) {
+        const long long t = row_tiles_left < max_row_tiles ? row_tiles_left : max_row_tiles;
+        const long long rows = (M - row0) < t * BM ? (M - row0) : t * BM;
+        sgemm_nn_kernel<<<(unsigned)(t * col_tiles), 256, 0, st>>>(A + row0 * lda, lda, B, ldb, C + row0 * ldc, ldc,
+                                                                 rows, K);
+        row_tiles_left -= t;
+        row0 += t * BM;
+    }
 }
 
 }  // namespace cert

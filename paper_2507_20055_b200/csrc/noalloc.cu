@@ -55,6 +55,8 @@ extern "C" cert_status_t cert_first_layer_bounds_noalloc(const float *weight, co
     if (std::isnan(clip_lo) || std::isnan(clip_hi) || clip_lo > clip_hi) return CERT_ERR_INVALID_ARG;
     const int ld0 = cert::round_up(in_features, cert::kPad);
     if ((size_t)batch * (size_t)ld0 > kNoAllocMaxFloats) return CERT_ERR_BATCH_TOO_LARGE;
+    // one warp per (box, neuron), eight warps per block: the grid's x extent must hold them all
+    if ((long long)batch * out_features > 8LL * 0x7FFFFFFF) return CERT_ERR_UNSUPPORTED;
 
     float *scratch = nullptr;
     cert_status_t s = scratch_for_current_device(&scratch);
