@@ -217,6 +217,7 @@ def main():
     ap.add_argument("--certifier", default="deeppoly",
                     help="deeppoly | ibp | crown_ibp | deeppoly_pN (N back-substitution steps per layer) | reusecert")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-microbench", action="store_true", help="skip the peak micro-kernels (roofline against the bf16-derived peaks only)")
     ap.add_argument("--ref-boxes", type=int, default=None)
     args = ap.parse_args()
 
@@ -368,6 +369,19 @@ def main():
     torch.cuda.synchronize()
     e2e_s = time.perf_counter() - t0
 
+    # ---- the denominators, measured: micro-kernels that run nothing but the unit in question ----
+    micro = None
+    if rank == 0 and world == 1 and not args.no_microbench:
+        micro = {}
+        for name, kind in (("tcgen05_f16", 0), ("tcgen05_tf32", 1), ("ffma", 2)):
+            try:
+                bt, bmhz, bms = binding.peak_microbench(kind, 5.0, stream.cuda_stream)
+                st_, smhz, sms_ = binding.peak_microbench(kind, 250.0, stream.cuda_stream)
+                micro[name] = {"burst": {"tflops": bt, "sm_mhz": bmhz, "ms": bms},
+                               "sustained": {"tflops": st_, "sm_mhz": smhz, "ms": sms_}}
+            except binding.CertError as e:
+                micro[name] = {"error": str(e)}
+
     # ---- max over ranks ----
     t = torch.tensor([total_ms, e2e_s * 1000.0], dtype=torch.float64, device="cuda")
     if world > 1:
@@ -410,22 +424,48 @@ def main():
             rows_per_launch = 2.0 * B * max(l.n_out for l in w.layers[1:-1] or w.layers[1:])
             traffic = cap["bytes_per_row"] * rows_per_launch
             traffic_note = f"{cap['kernel']}: {cap['source']}"
+        derived_peak = tc_peak if used_tc else ffma_peak
+        peak, peak_source, frac_same_clock = derived_peak, peaks["source"], None
+        pipe = ("tcgen05_f16" if used_fp16 else "tcgen05_tf32") if used_tc else "ffma"
+        m = (micro or {}).get(pipe)
+        if m and "sustained" in m:
+            # the pipe's own measured rate, under the power limit like the timed step; a fp32-accurate
+            # multiply-add costs three products on the tensor cores
+            div = 3.0 if used_tc else 1.0
+            peak = m["sustained"]["tflops"] / div
+            peak_source = "microbench"
+            clk = (clocks or {}).get("sm_mhz")
+            if achieved and clk and m["sustained"]["sm_mhz"]:
+                frac_same_clock = (achieved / clk) / (peak / m["sustained"]["sm_mhz"])
+        if used_tc:
+            derived_note = "bf16_tflops_sustained/3 (3xFP16)" if used_fp16 else "bf16_tflops_sustained/2/3 (3xTF32)"
+            if dom == "conv":
+                derived_note += ("; conv back-steps run as dense window / band contractions, counted here at their "
+                                 "algorithmic flops (the executed count is several times higher)")
+        else:
+            derived_note = "148 SM x 128 FMA x 2 x sm_max_mhz"
+            if used_patches and args.contraction != "ffma":
+                derived_note += ("; the conv class also holds the patch back-step, which runs on the tensor cores "
+                                 "(gather + 3xTF32 contraction with the window-to-window matrix), counted at its "
+                                 "algorithmic flops")
+        peak_note = derived_note
+        if peak_source == "microbench":
+            peak_note = (f"microbench: {pipe} sustained" + (" / 3" if used_tc else "") +
+                         "; peak_bf16_derived = " + derived_note)
         roof = {"bound": "tensor" if used_tc else "alu",
-                "achieved": achieved, "peak": tc_peak if used_tc else ffma_peak, "unit": "TFLOP/s",
-                "frac": (achieved / (tc_peak if used_tc else ffma_peak)) if achieved else None,
+                "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
+                "frac": (achieved / peak) if achieved else None,
+                "frac_same_clock": frac_same_clock,
+                "peak_bf16_derived": derived_peak,
+                "frac_bf16_derived": (achieved / derived_peak) if achieved else None,
+                "peak_bf16_derived_source": peaks["source"],
                 "traffic": traffic, "traffic_note": traffic_note,
                 "kernel": dom + " back-step", "launches_per_step": dom_n // max(1, args.steps),
                 "avg_launch_ms": dom_ms / dom_n if dom_n else None,
                 "flops_per_step": fl[dom], "flops_per_step_all_backsteps": flops_call,
                 "flops_per_step_if_dense_maps": fl_dense[dom], "conv_rows_as_patches": used_patches,
-                "peak_source": peaks["source"],
-                "peak_note": (("bf16_tflops_sustained/3 (3xFP16)" if used_fp16 else "bf16_tflops_sustained/2/3 (3xTF32)")
-                              + ("; conv back-steps run as dense window / band contractions, counted here at their "
-                                 "algorithmic flops (the executed count is several times higher)" if dom == "conv" else "")
-                              if used_tc else "148 SM x 128 FMA x 2 x sm_max_mhz" +
-                              ("; the conv class also holds the patch back-step, which runs on the tensor cores "
-                               "(gather + 3xTF32 contraction with the window-to-window matrix), counted at its "
-                               "algorithmic flops" if used_patches and args.contraction != "ffma" else "")),
+                "peak_source": peak_source,
+                "peak_note": peak_note,
                 "class_ms_per_step": {k: v / args.steps for k, v in cls_ms.items()}}
         # branch statistics of the last call (Relu transformer): the share of ReLU neurons relaxed as unstable
         torch.cuda.synchronize()
@@ -445,6 +485,8 @@ def main():
             "gpu_launches": launches, "wall_s_timed_region": t_wall, "roofline": roof, "clocks": clocks,
             "unstable_fraction": unstable,
         }
+        if micro is not None:
+            out["peaks_microbench"] = micro
         if tf32_ref is not None:
             out["tf32_split"] = tf32_ref
         if world == 1 and not args.no_cpu_baseline:

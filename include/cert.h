@@ -136,12 +136,17 @@ cert_status_t cert_backsub_bounds(cert_net_t *net, const float *centers, float e
  * contraction instead of a traversal through all earlier layers; the bounds are sound but can be
  * looser than DeepPoly's from the third affine layer on.
  *   cert_net_enable_reusecert  allocates what the certifier needs on top of the net (the shapes of one
- *            layer for max_batch boxes, twice; block weight matrices): call it once, outside the hot
- *            path, with the net's device current.  FC layers only (CERT_ERR_UNSUPPORTED otherwise,
- *            or when the tensor-core path is not available).
+ *            layer for max_batch boxes, three times; block weight matrices): call it once, outside the
+ *            hot path, with the net's device current.  FC layers only, and only where the fp16-split
+ *            contraction is available (CERT_ERR_UNSUPPORTED otherwise): every layer's shapes are built
+ *            from the rounded shapes of the layer below, so rounding compounds with depth, and of the
+ *            two tensor-core forms only the fp16 split holds 1e-4 * (1 + |bound|) on the 6 x 1024 net.
  *   cert_reusecert_bounds      arguments, outputs (l, u of every affine layer as the Relu transformer
  *            computes them: L.map(simplify_lower), U.map(simplify_upper)), branch codes and stream
- *            behaviour as cert_deeppoly_bounds; allocates nothing.
+ *            behaviour as cert_deeppoly_bounds; allocates nothing.  Runs in the fp16 split whatever
+ *            CERT_CONTRACTION_AUTO resolves to; a net set to FFMA or TC3XTF32 is refused
+ *            (CERT_ERR_UNSUPPORTED).  A shape entry beyond the fp16 range raises CERT_ERR_RANGE in the
+ *            status word (cert_net_last_status; the *_host call returns it).
  */
 cert_status_t cert_net_enable_reusecert(cert_net_t *net);
 cert_status_t cert_reusecert_bounds(cert_net_t *net, const float *centers, float eps, int batch,
@@ -215,13 +220,15 @@ cert_status_t cert_net_selftest_bounded_wait(cert_net_t *net, void *stream);
  *            coefficients below 65504 in magnitude (beyond that cert_net_last_status reports
  *            CERT_ERR_RANGE and the results are invalid; values under 6.1e-5 are held to 1.5e-11
  *            absolute instead of 2^-22 relative).
- *   AUTO:    TC3XFP16 when the net's weights prove at create that no coefficient can leave that range on
- *            any input: a ReLU back-step scales a coefficient by a slope in [0, 1], so every entry of a
- *            traversal's matrix over layer j-1 is bounded by the matching entry of |W_k| |W_k-1| ... |W_j|,
- *            and the largest entry of all those products (cert_net_fp16_coefficient_bound) must stay under
- *            60000.  FC nets without residual connections only; otherwise, and whenever the proof fails,
- *            TC3XTF32, or FFMA where the tensor-core path is unavailable.  cert_net_auto_contraction tells
- *            which.  (The environment variable CERT_AUTO_FP16=0, read at create, keeps AUTO on TC3XTF32.)
+ *   AUTO:    decided per affine layer k at create.  TC3XFP16 for the traversal of layer k when the net's
+ *            weights prove that none of its coefficients can leave that range on any input: a ReLU
+ *            back-step scales a coefficient by a slope in [0, 1], so every entry of the traversal's matrix
+ *            over layer j-1 is bounded by the matching entry of |W_k| |W_k-1| ... |W_j|, and the largest
+ *            entry of those products over j (cert_net_fp16_coefficient_bound) must stay under 60000.  The
+ *            products grow with depth: on deep nets the last layers may stay on TC3XTF32 while the others
+ *            run in the fp16 split.  FC nets without residual connections only; otherwise, and for every
+ *            layer whose proof fails, TC3XTF32, or FFMA where the tensor-core path is unavailable.
+ *            (The environment variable CERT_AUTO_FP16=0, read at create, keeps AUTO on TC3XTF32.)
  * Conv back-steps have the same fusions; under FFMA they run on the FMA units, otherwise on the TF32 tensor-core
  * kernel where their geometry allows (see cert_net_set_conv_patches).
  * (The kernels of a call are chained with programmatic dependent launch, so that a kernel's launch and set-up
@@ -233,10 +240,12 @@ cert_status_t cert_net_selftest_bounded_wait(cert_net_t *net, void *stream);
 enum { CERT_CONTRACTION_AUTO = 0, CERT_CONTRACTION_FFMA = 1, CERT_CONTRACTION_TC3XTF32 = 2,
        CERT_CONTRACTION_TC3XFP16 = 3 };
 cert_status_t cert_net_set_contraction(cert_net_t *net, int mode);
-/* The mode CERT_CONTRACTION_AUTO stands for on this net (one of the other three); -1 for a null net. */
+/* What CERT_CONTRACTION_AUTO stands for on this net: CERT_CONTRACTION_TC3XFP16 if at least one layer's
+ * traversal passes the range proof, else CERT_CONTRACTION_TC3XTF32 or CERT_CONTRACTION_FFMA; -1 for a null net. */
 int cert_net_auto_contraction(const cert_net_t *net);
-/* Largest entry of the products |W_k| ... |W_j| (see AUTO above); INFINITY where no proof was attempted. */
-float cert_net_fp16_coefficient_bound(const cert_net_t *net);
+/* Largest entry of the products |W_k| ... |W_j|, j = k-1 .. 1, for affine layer k = `layer` (0-based; see AUTO
+ * above), or over all layers for layer < 0; INFINITY where no proof was attempted; -1 for bad arguments. */
+float cert_net_fp16_coefficient_bound(const cert_net_t *net, int layer);
 /* Which contraction kernels the most recent call ran: bit 0 = FFMA, bit 1 = TC3XTF32,
  * bit 2 = the TC3XTF32 kernel ran in its CTA-pair form (tcgen05 cta_group::2), bit 3 = a traversal ran on
  * receptive-field patches, bit 4 = TC3XFP16, bit 5 = TC3XFP16 with a whole traversal per launch (nets whose
@@ -332,6 +341,24 @@ cert_status_t cert_first_layer_bounds_noalloc(const float *weight, const float *
                                               int in_features, const float *centers, float eps,
                                               float clip_lo, float clip_hi, int batch, float *lb_out,
                                               float *ub_out, void *stream);
+
+/*
+ * (No counterpart in the paper: measurement support for the benchmark's roofline.)
+ *
+ * Measures, on the current device, the peak rate of the unit a contraction kernel of this library runs on, with
+ * a micro-kernel that does nothing else:
+ *   kind 0  tcgen05.mma kind::f16,  CTA pairs, 256 x 256 tiles, both operands resident in shared memory
+ *   kind 1  tcgen05.mma kind::tf32, the same shape
+ *   kind 2  fp32 fused multiply-adds in registers (one 1024-thread block per multiprocessor)
+ * The kernel is sized by a short calibration run to last about target_ms (0 < target_ms <= 2000); a few ms give
+ * a burst figure at boost clocks, a few hundred ms a figure under the power limit.  Outputs (HOST pointers):
+ * tflops_out = executed flops / CUDA-event time (2 per multiply-add), sm_mhz_out (may be NULL) = SM cycles per
+ * microsecond as the kernel itself saw them, ms_out (may be NULL) = the kernel's duration.  Allocates a few
+ * words of device memory and frees them; synchronises `stream`.  Every device-side wait is bounded
+ * (CERT_ERR_TIMEOUT if one runs out).
+ */
+cert_status_t cert_peak_microbench(int kind, double target_ms, double *tflops_out, double *sm_mhz_out,
+                                   double *ms_out, void *stream);
 
 const char *cert_status_string(cert_status_t s);
 

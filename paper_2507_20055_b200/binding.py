@@ -35,6 +35,7 @@ EXPORTS = [
     "cert_net_last_contraction_paths", "cert_first_layer_bounds_noalloc", "cert_net_set_conv_patches",
     "cert_net_enable_reusecert", "cert_reusecert_bounds", "cert_reusecert_bounds_host",
     "cert_net_check_guards", "cert_net_auto_contraction", "cert_net_fp16_coefficient_bound",
+    "cert_peak_microbench",
 ]
 CLASS_NAMES = ["input", "relax", "relu_step", "affine", "conv", "concretize"]
 
@@ -97,8 +98,10 @@ _lib.cert_net_check_guards.argtypes = [_vp, _vp]
 _lib.cert_net_check_guards.restype = _i
 _lib.cert_net_auto_contraction.argtypes = [_vp]
 _lib.cert_net_auto_contraction.restype = _i
-_lib.cert_net_fp16_coefficient_bound.argtypes = [_vp]
+_lib.cert_net_fp16_coefficient_bound.argtypes = [_vp, _i]
 _lib.cert_net_fp16_coefficient_bound.restype = ctypes.c_float
+_lib.cert_peak_microbench.argtypes = [_i, ctypes.c_double, _vp, _vp, _vp, _vp]
+_lib.cert_peak_microbench.restype = _i
 _lib.cert_status_string.argtypes = [_i]
 _lib.cert_status_string.restype = ctypes.c_char_p
 
@@ -310,8 +313,8 @@ class CertNet:
     def auto_contraction(self) -> int:
         return int(_lib.cert_net_auto_contraction(self._h))
 
-    def fp16_coefficient_bound(self) -> float:
-        return float(_lib.cert_net_fp16_coefficient_bound(self._h))
+    def fp16_coefficient_bound(self, layer: int = -1) -> float:
+        return float(_lib.cert_net_fp16_coefficient_bound(self._h, int(layer)))
 
     def last_contraction_paths(self) -> int:
         return int(_lib.cert_net_last_contraction_paths(self._h))
@@ -354,6 +357,16 @@ def first_layer_bounds_noalloc(weight, bias, centers, eps, clip_lo, clip_hi, lb_
                                                 centers.data_ptr(), float(eps), float(clip_lo), float(clip_hi),
                                                 centers.shape[0], lb_out.data_ptr(), ub_out.data_ptr(),
                                                 st.cuda_stream), "cert_first_layer_bounds_noalloc")
+
+
+def peak_microbench(kind: int, target_ms: float = 5.0, stream_ptr: int = 0):
+    """cert_peak_microbench: (TFLOP/s, SM MHz seen by the kernel, ms) for kind 0 = tcgen05 f16, 1 = tcgen05 tf32,
+    2 = fp32 FMA units."""
+    out = (ctypes.c_double * 3)()
+    base = ctypes.addressof(out)
+    _check(_lib.cert_peak_microbench(int(kind), float(target_ms), base, base + 8, base + 16, stream_ptr),
+           "cert_peak_microbench")
+    return float(out[0]), float(out[1]), float(out[2])
 
 
 # C-ABI names, as plain functions

@@ -66,15 +66,13 @@ struct BandStep {
     cert::TcPlan plan;
 };
 
-// ReuseCert: per affine layer k >= 1 the block weight matrix [[W+^T, W-^T], [W-^T, W+^T]] as the K-major B
-// operand (rows = the 2*n_k output columns, columns = the 2*n_{k-1} columns of the layer below), TF32 split.
+// ReuseCert (served in the fp16 split): per affine layer k >= 1 the block weight matrix
+// [[W+^T, W-^T], [W-^T, W+^T]] as the K-major B operand (rows = the 2*n_k output columns, columns = the 2*n_{k-1}
+// columns of the layer below) as an fp16 pair; the shapes rotate through three buffers (pair in, raw fp32
+// result, pair out).
 struct ReuseLayer {
     int ld_s = 0;                        // pitch of this layer's [L | U] matrix
-    float *B_hi = nullptr, *B_lo = nullptr, *bias2 = nullptr;
-    cert::TcMap b_hi, b_lo, a_hi[2], a_lo[2], o_hi[2];
-    cert::TcPlan plan;
-    // fp16-split form: the same block matrix as an fp16 pair; shapes rotate through three buffers
-    // (pair in, raw fp32 result, pair out)
+    float *bias2 = nullptr;
     __half *B16_hi = nullptr, *B16_lo = nullptr;
     cert::TcMap b16_hi, b16_lo, a16_hi[3], a16_lo[3], o32[3];
     cert::Tc16Plan plan16;
@@ -82,10 +80,10 @@ struct ReuseLayer {
 
 struct ReuseState {
     bool on = false;
-    bool fp16_ready = false;
     int R = 0;                           // rows per box: n0 coordinates, the constant, zero padding to 32
     float *W0t = nullptr;                // first layer's weights transposed [round_up(n0, 32)][ld_out]
-    float *S_hi[2] = {nullptr, nullptr}, *S_lo[2] = {nullptr, nullptr};
+    float *X[3] = {nullptr, nullptr, nullptr};   // shape buffers: an fp16 pair (hi, then lo at lo_off halves) or a raw fp32 result
+    size_t lo_off = 0;
     float *colsum = nullptr;
     std::vector<ReuseLayer> layers;
 };
@@ -116,8 +114,9 @@ struct cert_net {
     // AUTO takes the fp16 split: the net's weights prove that no coefficient of any traversal can leave the
     // fp16 range (fp16_coef_bound = the largest entry of |W_k| |W_k-1| ... |W_j| over all k > j >= 1; slopes of a
     // ReLU back-step lie in [0, 1], so every stored coefficient is below it in magnitude)
-    bool auto_fp16 = false;
-    float fp16_coef_bound = INFINITY;
+    bool auto_fp16 = false;                  // some layer's traversal passes the proof
+    float fp16_coef_bound = INFINITY;        // the largest bound over all layers
+    std::vector<float> fp16_layer_bound;     // [k]: the bound for the traversal of layer k (k >= 1)
     std::vector<Tc16Layer> tc16;
     // fp16-split path, narrow nets: a whole traversal per launch with the coefficient panel kept in shared memory
     bool chain_ok = false;
@@ -388,14 +387,17 @@ cert_status_t setup_tensor_core_path(cert_net *net, const cert_layer_desc_t *des
 // outputs of layer j-1, the matrix W_k D W_{k-1} D ... W_j with diagonal ReLU slopes D in [0, 1] (sign-split
 // scaling never enlarges a coefficient), so each of its entries is at most the matching entry of
 // |W_k| |W_{k-1}| ... |W_j| in magnitude.  Those products are formed here, once, on the FMA units (the row
-// count is n_k, not batch * 2 * n_k); their largest entry goes to net->fp16_coef_bound.  Below kFp16Safe the
-// fp16 split cannot overflow on this net, whatever the input boxes, and AUTO takes it.
+// count is n_k, not batch * 2 * n_k); their largest entry, per layer k, goes to net->fp16_layer_bound[k].  Below
+// kFp16Safe the fp16 split cannot overflow in that layer's traversal, whatever the input boxes, and AUTO takes
+// it for that layer (the products grow with the number of layers a traversal passes, so on deep nets the first
+// layers pass and the last ones stay on the TF32 split).
 constexpr float kFp16Safe = 60000.0f;       // fp16's largest finite value is 65504; the margin covers fp32 rounding here
 
 cert_status_t prove_fp16_range(cert_net *net) {
     const int K = net->n_layers;
     net->auto_fp16 = false;
     net->fp16_coef_bound = INFINITY;
+    net->fp16_layer_bound.assign(K, INFINITY);
     if (!net->tc16_ok || !net->skip_from.empty()) return CERT_OK;
     std::vector<float *> absW(K, nullptr);
     float *max_dev = nullptr;
@@ -404,8 +406,8 @@ cert_status_t prove_fp16_range(cert_net *net) {
         for (float *p : absW) if (p) cudaFree(p);
         if (max_dev) cudaFree(max_dev);
     };
-    if (cudaMalloc(reinterpret_cast<void **>(&max_dev), sizeof(float)) != cudaSuccess ||
-        cudaMemset(max_dev, 0, sizeof(float)) != cudaSuccess) {
+    if (cudaMalloc(reinterpret_cast<void **>(&max_dev), K * sizeof(float)) != cudaSuccess ||
+        cudaMemset(max_dev, 0, K * sizeof(float)) != cudaSuccess) {
         cudaGetLastError();
         cleanup();
         return CERT_ERR_OOM;
@@ -424,21 +426,21 @@ cert_status_t prove_fp16_range(cert_net *net) {
         const LayerDev &Lk = net->layers[k];
         // the start of the traversal: |W_k| itself, rows padded like the coefficient matrices
         const float *cur = absW[k];
-        cert::launch_absmax(cur, (long long)Lk.n_out * Lk.ld_in, max_dev, nullptr);
+        cert::launch_absmax(cur, (long long)Lk.n_out * Lk.ld_in, max_dev + k, nullptr);
         int p = 0;
         for (int j = k - 1; j >= 1; --j) {
             const LayerDev &Lj = net->layers[j];
             cert::launch_gemm_ffma(cur, Lj.ld_out, absW[j], Lj.ld_in, net->buf[p], Lj.ld_in, Lk.n_out, Lj.n_in, Lj.n_out,
                                    nullptr);
-            cert::launch_absmax(net->buf[p], (long long)Lk.n_out * Lj.ld_in, max_dev, nullptr);
+            cert::launch_absmax(net->buf[p], (long long)Lk.n_out * Lj.ld_in, max_dev + k, nullptr);
             cur = net->buf[p];
             p ^= 1;
         }
     }
-    float bound = INFINITY;
+    std::vector<float> bound(K, INFINITY);
     if (rc == CERT_OK &&
         (cudaDeviceSynchronize() != cudaSuccess ||
-         cudaMemcpy(&bound, max_dev, sizeof(float), cudaMemcpyDeviceToHost) != cudaSuccess))
+         cudaMemcpy(bound.data(), max_dev, K * sizeof(float), cudaMemcpyDeviceToHost) != cudaSuccess))
         rc = CERT_ERR_CUDA;
     // the products went through the coefficient buffers: leave them as the kernels expect to find them (zero)
     if (rc == CERT_OK && K > 2) {
@@ -450,11 +452,15 @@ cert_status_t prove_fp16_range(cert_net *net) {
     }
     cleanup();
     if (rc != CERT_OK) { cudaGetLastError(); return rc; }
-    net->fp16_coef_bound = bound;
-    net->auto_fp16 = std::isfinite(bound) && bound <= kFp16Safe;
-    if (const char *e = std::getenv("CERT_AUTO_FP16")) {
-        if (std::atoi(e) == 0) net->auto_fp16 = false;
+    bool off = false;
+    if (const char *e = std::getenv("CERT_AUTO_FP16")) off = std::atoi(e) == 0;
+    net->fp16_coef_bound = 0.0f;
+    for (int k = 1; k < K; ++k) {
+        net->fp16_layer_bound[k] = bound[k];
+        net->fp16_coef_bound = std::max(net->fp16_coef_bound, bound[k]);
+        if (!off && std::isfinite(bound[k]) && bound[k] <= kFp16Safe) net->auto_fp16 = true;
     }
+    if (off) net->fp16_layer_bound.assign(K, INFINITY);
     return CERT_OK;
 }
 
@@ -1166,11 +1172,14 @@ void run_dense(Traversal &t) {
     if (Lk.relu_after || bounds_in_slots || k + 1 < K) t.relax(bounds_in_slots ? net->dbuf[dcur] : nullptr, dslots);
 }
 
-// The contraction mode one call runs in.  AUTO: the fp16 split where the net's weights prove that no coefficient
-// can leave the fp16 range (cert_net::auto_fp16), else the TF32 split; `forced` >= 0 overrides the net's setting.
-int call_mode(const cert_net *net, int forced) {
-    int mode = forced >= 0 ? forced : net->contraction;
-    if (mode == CERT_CONTRACTION_AUTO && net->auto_fp16) mode = CERT_CONTRACTION_TC3XFP16;
+// The contraction mode the traversal of layer k runs in.  AUTO: the fp16 split where the net's weights prove that
+// no coefficient of that traversal can leave the fp16 range (cert_net::fp16_layer_bound), else the TF32 split;
+// `forced` >= 0 overrides the net's setting.
+int layer_mode(const cert_net *net, int forced, int k) {
+    const int mode = forced >= 0 ? forced : net->contraction;
+    if (mode == CERT_CONTRACTION_AUTO && net->tc16_ok && k < (int)net->fp16_layer_bound.size() &&
+        net->fp16_layer_bound[k] <= kFp16Safe)
+        return CERT_CONTRACTION_TC3XFP16;
     return mode;
 }
 
@@ -1182,9 +1191,8 @@ cert_status_t backsub_impl(cert_net *net, const float *centers, float eps, int b
     if (batch < 1 || !(eps >= 0.0f) || std::isinf(eps)) return CERT_ERR_INVALID_ARG;
     if (batch > net->max_batch) return CERT_ERR_BATCH_TOO_LARGE;
     const int K = net->n_layers;
-    const int mode = call_mode(net, forced_mode);
     const bool residual = !net->skip_from.empty();
-    if (residual && backsteps && mode == CERT_CONTRACTION_TC3XFP16)
+    if (residual && backsteps && (forced_mode >= 0 ? forced_mode : net->contraction) == CERT_CONTRACTION_TC3XFP16)
         for (int k = 1; k < K; ++k)
             if (backsteps[k] >= 0 && backsteps[k] < k) return CERT_ERR_UNSUPPORTED;   // fp16 split: full traversals only
     Recorder rec(net, st);
@@ -1200,6 +1208,7 @@ cert_status_t backsub_impl(cert_net *net, const float *centers, float eps, int b
         rec.mark(CERT_CLASS_RELAX);
     }
     for (int k = 1; k < K; ++k) {
+        const int mode = layer_mode(net, forced_mode, k);
         Traversal t;
         t.net = net; t.st = st; t.rec = &rec; t.mode = mode; t.batch = batch; t.k = k;
         t.steps = (backsteps && backsteps[k] >= 0) ? std::min(backsteps[k], k) : k;
@@ -1552,7 +1561,9 @@ static cert_status_t enable_reusecert_impl(cert_net_t *net) {
     if (!net) return CERT_ERR_INVALID_ARG;
     if (net->reuse.on) return CERT_OK;
     const int K = net->n_layers;
-    if (K < 2 || !net->tc_ok || !net->skip_from.empty()) return CERT_ERR_UNSUPPORTED;
+    // the fp16-split contraction only: it holds the stated tolerance on deep nets, where rounding compounds from
+    // layer to layer (each layer's shapes are built from the rounded shapes below), and the TF32 split does not
+    if (K < 2 || !net->tc16_ok || !net->skip_from.empty()) return CERT_ERR_UNSUPPORTED;
     for (int k = 0; k < K; ++k)
         if (net->layers[k].kind != CERT_LAYER_FC) return CERT_ERR_UNSUPPORTED;
     int dev = 0;
@@ -1566,12 +1577,13 @@ static cert_status_t enable_reusecert_impl(cert_net_t *net) {
         ld_max = std::max(ld_max, R.layers[k].ld_s);
     }
     const long long m_max = (long long)net->max_batch * R.R;
-    const size_t elems = (size_t)m_max * ld_max;
-    for (int p = 0; p < 2; ++p)
-        if (!dev_alloc_zero(net, &R.S_hi[p], elems) || !dev_alloc_zero(net, &R.S_lo[p], elems)) return CERT_ERR_OOM;
+    const size_t elems = (size_t)m_max * ld_max;       // floats per buffer: a raw result, or a pair of halves
+    R.lo_off = elems;                                  // in halves: the lo part of a pair is the buffer's second half
+    for (int p = 0; p < 3; ++p)
+        if (!dev_alloc_zero(net, &R.X[p], elems)) return CERT_ERR_OOM;
     if (!dev_alloc_zero(net, &R.colsum, (size_t)(m_max / 32) * ld_max)) return CERT_ERR_OOM;
-    const int ctas = net->tc_ctas;
-    std::vector<float> w, hi, lo, b2;
+    std::vector<float> w, t0, b2, bias;
+    std::vector<__half> h16, l16;
     for (int k = 0; k < K; ++k) {
         const LayerDev &L = net->layers[k];
         const size_t rows_pad = round_up(L.n_out, kPad);
@@ -1581,109 +1593,59 @@ static cert_status_t enable_reusecert_impl(cert_net_t *net) {
             return CERT_ERR_CUDA;
         }
         if (k == 0) {
-            hi.assign((size_t)round_up(L.n_in, kPad) * L.ld_out, 0.0f);
+            t0.assign((size_t)round_up(L.n_in, kPad) * L.ld_out, 0.0f);
             for (int t = 0; t < L.n_out; ++t)
-                for (int s2 = 0; s2 < L.n_in; ++s2) hi[(size_t)s2 * L.ld_out + t] = w[(size_t)t * L.ld_in + s2];
-            if (!dev_alloc(net, (void **)&R.W0t, hi.size() * sizeof(float))) return CERT_ERR_OOM;
-            if (cudaMemcpy(R.W0t, hi.data(), hi.size() * sizeof(float), cudaMemcpyHostToDevice) != cudaSuccess)
+                for (int s2 = 0; s2 < L.n_in; ++s2) t0[(size_t)s2 * L.ld_out + t] = w[(size_t)t * L.ld_in + s2];
+            if (!dev_alloc(net, (void **)&R.W0t, t0.size() * sizeof(float))) return CERT_ERR_OOM;
+            if (cudaMemcpy(R.W0t, t0.data(), t0.size() * sizeof(float), cudaMemcpyHostToDevice) != cudaSuccess)
                 return CERT_ERR_CUDA;
             continue;
         }
         ReuseLayer &RL = R.layers[k];
         const int n = L.n_out, m = L.n_in, ldb = R.layers[k - 1].ld_s;
         const size_t brows = round_up(2 * n, kPad);
-        hi.assign(brows * ldb, 0.0f);
-        lo.assign(brows * ldb, 0.0f);
-        auto put = [&](int row, int col, float v) {
-            const float h = host_tf32(v);
-            hi[(size_t)row * ldb + col] = h;
-            lo[(size_t)row * ldb + col] = host_tf32(v - h);
+        h16.assign(brows * ldb, __float2half_rn(0.0f));
+        l16.assign(brows * ldb, __float2half_rn(0.0f));
+        auto put16 = [&](int row, int col, float v) {
+            const __half h = __float2half_rn(v);
+            h16[(size_t)row * ldb + col] = h;
+            l16[(size_t)row * ldb + col] = __float2half_rn((v - __half2float(h)) * cert::kLoScale);
         };
         for (int i = 0; i < n; ++i)
             for (int t = 0; t < m; ++t) {
                 const float v = w[(size_t)i * L.ld_in + t];
                 const float vp = v >= 0.0f ? v : 0.0f, vm = v >= 0.0f ? 0.0f : v;
-                put(i, t, vp);          // L_i takes L_t with W+ ...
-                put(i, m + t, vm);      // ... and U_t with W-
-                put(n + i, t, vm);      // U_i takes L_t with W- ...
-                put(n + i, m + t, vp);  // ... and U_t with W+
+                put16(i, t, vp);          // L_i takes L_t with W+ ...
+                put16(i, m + t, vm);      // ... and U_t with W-
+                put16(n + i, t, vm);      // U_i takes L_t with W- ...
+                put16(n + i, m + t, vp);  // ... and U_t with W+
             }
         b2.assign(RL.ld_s, 0.0f);
-        std::vector<float> bias(L.ld_out);
+        bias.resize(L.ld_out);
         if (cudaMemcpy(bias.data(), L.bias_n, bias.size() * sizeof(float), cudaMemcpyDeviceToHost) != cudaSuccess) {
             cudaGetLastError();
             return CERT_ERR_CUDA;
         }
         for (int i = 0; i < n; ++i) b2[i] = b2[n + i] = bias[i];
-        if (!dev_alloc(net, (void **)&RL.B_hi, hi.size() * sizeof(float)) ||
-            !dev_alloc(net, (void **)&RL.B_lo, lo.size() * sizeof(float)) ||
+        if (!dev_alloc(net, (void **)&RL.B16_hi, h16.size() * sizeof(__half)) ||
+            !dev_alloc(net, (void **)&RL.B16_lo, l16.size() * sizeof(__half)) ||
             !dev_alloc(net, (void **)&RL.bias2, b2.size() * sizeof(float)))
             return CERT_ERR_OOM;
-        if (cudaMemcpy(RL.B_hi, hi.data(), hi.size() * sizeof(float), cudaMemcpyHostToDevice) != cudaSuccess ||
-            cudaMemcpy(RL.B_lo, lo.data(), lo.size() * sizeof(float), cudaMemcpyHostToDevice) != cudaSuccess ||
+        if (cudaMemcpy(RL.B16_hi, h16.data(), h16.size() * sizeof(__half), cudaMemcpyHostToDevice) != cudaSuccess ||
+            cudaMemcpy(RL.B16_lo, l16.data(), l16.size() * sizeof(__half), cudaMemcpyHostToDevice) != cudaSuccess ||
             cudaMemcpy(RL.bias2, b2.data(), b2.size() * sizeof(float), cudaMemcpyHostToDevice) != cudaSuccess)
             return CERT_ERR_CUDA;
-        RL.plan = cert::tc_tile_plan(2 * n, ctas);
-        if (RL.plan.stages < 2) return CERT_ERR_UNSUPPORTED;
-        bool ok = cert::tc_make_map(&RL.b_hi, RL.B_hi, 2 * m, 2 * n, ldb, RL.plan.bn / ctas) &&
-                  cert::tc_make_map(&RL.b_lo, RL.B_lo, 2 * m, 2 * n, ldb, RL.plan.bn / ctas);
-        for (int p = 0; p < 2 && ok; ++p)
-            ok = cert::tc_make_map(&RL.a_hi[p], R.S_hi[p], 2 * m, m_max, ldb, 128) &&
-                 cert::tc_make_map(&RL.a_lo[p], R.S_lo[p], 2 * m, m_max, ldb, 128) &&
-                 cert::tc_make_map(&RL.o_hi[p], R.S_hi[p], RL.ld_s, m_max, RL.ld_s, 32);
-        if (!ok) return CERT_ERR_CUDA;
-    }
-    // fp16-split operands (used when the net's contraction mode is TC3XFP16)
-    if (net->tc16_ok) {
-        float *X[3] = {R.S_hi[0], R.S_hi[1], R.S_lo[0]};
-        const size_t lo_off = elems;                 // halves: the lo part of a pair sits in the buffer's second half
-        std::vector<__half> h16, l16;
-        bool ok16 = true;
-        for (int k = 1; k < K && ok16; ++k) {
-            const LayerDev &L = net->layers[k];
-            ReuseLayer &RL = R.layers[k];
-            const int n = L.n_out, m = L.n_in, ldb = R.layers[k - 1].ld_s;
-            const size_t rows_pad = round_up(L.n_out, kPad);
-            w.resize(rows_pad * L.ld_in);
-            if (cudaMemcpy(w.data(), L.W, w.size() * sizeof(float), cudaMemcpyDeviceToHost) != cudaSuccess) {
-                cudaGetLastError();
-                return CERT_ERR_CUDA;
-            }
-            const size_t brows = round_up(2 * n, kPad);
-            h16.assign(brows * ldb, __float2half_rn(0.0f));
-            l16.assign(brows * ldb, __float2half_rn(0.0f));
-            auto put16 = [&](int row, int col, float v) {
-                const __half h = __float2half_rn(v);
-                h16[(size_t)row * ldb + col] = h;
-                l16[(size_t)row * ldb + col] = __float2half_rn((v - __half2float(h)) * cert::kLoScale);
-            };
-            for (int i = 0; i < n; ++i)
-                for (int t = 0; t < m; ++t) {
-                    const float v = w[(size_t)i * L.ld_in + t];
-                    const float vp = v >= 0.0f ? v : 0.0f, vm = v >= 0.0f ? 0.0f : v;
-                    put16(i, t, vp);
-                    put16(i, m + t, vm);
-                    put16(n + i, t, vm);
-                    put16(n + i, m + t, vp);
-                }
-            if (!dev_alloc(net, (void **)&RL.B16_hi, h16.size() * sizeof(__half)) ||
-                !dev_alloc(net, (void **)&RL.B16_lo, l16.size() * sizeof(__half)))
-                return CERT_ERR_OOM;
-            if (cudaMemcpy(RL.B16_hi, h16.data(), h16.size() * sizeof(__half), cudaMemcpyHostToDevice) != cudaSuccess ||
-                cudaMemcpy(RL.B16_lo, l16.data(), l16.size() * sizeof(__half), cudaMemcpyHostToDevice) != cudaSuccess)
-                return CERT_ERR_CUDA;
-            RL.plan16 = cert::tc16_tile_plan(2 * n);
-            if (RL.plan16.stages < 2) { ok16 = false; break; }
-            ok16 = cert::tc16_make_map(&RL.b16_hi, RL.B16_hi, 2 * m, 2 * n, ldb, 64, RL.plan16.bn / 2) &&
-                   cert::tc16_make_map(&RL.b16_lo, RL.B16_lo, 2 * m, 2 * n, ldb, 64, RL.plan16.bn / 2);
-            for (int p = 0; p < 3 && ok16; ++p) {
-                const __half *xh = reinterpret_cast<const __half *>(X[p]);
-                ok16 = cert::tc16_make_map(&RL.a16_hi[p], xh, 2 * m, m_max, ldb, 64, 128) &&
-                       cert::tc16_make_map(&RL.a16_lo[p], xh + lo_off, 2 * m, m_max, ldb, 64, 128) &&
-                       cert::tc_make_map(&RL.o32[p], X[p], RL.ld_s, m_max, RL.ld_s, 32);
-            }
+        RL.plan16 = cert::tc16_tile_plan(2 * n);
+        if (RL.plan16.stages < 2) return CERT_ERR_UNSUPPORTED;
+        bool ok = cert::tc16_make_map(&RL.b16_hi, RL.B16_hi, 2 * m, 2 * n, ldb, 64, RL.plan16.bn / 2) &&
+                  cert::tc16_make_map(&RL.b16_lo, RL.B16_lo, 2 * m, 2 * n, ldb, 64, RL.plan16.bn / 2);
+        for (int p = 0; p < 3 && ok; ++p) {
+            const __half *xh = reinterpret_cast<const __half *>(R.X[p]);
+            ok = cert::tc16_make_map(&RL.a16_hi[p], xh, 2 * m, m_max, ldb, 64, 128) &&
+                 cert::tc16_make_map(&RL.a16_lo[p], xh + R.lo_off, 2 * m, m_max, ldb, 64, 128) &&
+                 cert::tc_make_map(&RL.o32[p], R.X[p], RL.ld_s, m_max, RL.ld_s, 32);
         }
-        R.fp16_ready = ok16;
+        if (!ok) return CERT_ERR_CUDA;
     }
     if (cudaDeviceSynchronize() != cudaSuccess) { cudaGetLastError(); return CERT_ERR_CUDA; }
     R.on = true;
@@ -1696,9 +1658,12 @@ cert_status_t cert_reusecert_bounds(cert_net_t *net, const float *centers, float
     if (batch < 1 || !(eps >= 0.0f) || std::isinf(eps)) return CERT_ERR_INVALID_ARG;
     if (batch > net->max_batch) return CERT_ERR_BATCH_TOO_LARGE;
     if (!net->reuse.on) return CERT_ERR_UNSUPPORTED;
+    // served in the fp16 split only (see cert_net_enable_reusecert): a net set to another mode is refused
+    if (net->contraction != CERT_CONTRACTION_AUTO && net->contraction != CERT_CONTRACTION_TC3XFP16)
+        return CERT_ERR_UNSUPPORTED;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     ReuseState &R = net->reuse;
-    const int K = net->n_layers, n_total = net->n_total, ctas = net->tc_ctas;
+    const int K = net->n_layers, n_total = net->n_total;
     const long long rows = (long long)batch * R.R;
     Recorder rec(net, st);
     cert::launch_box(centers, eps, net->clip_lo, net->clip_hi, batch, net->n0, net->ld0, net->l0, net->u0, st);
@@ -1708,57 +1673,12 @@ cert_status_t cert_reusecert_bounds(cert_net_t *net, const float *centers, float
     rec.mark(CERT_CLASS_INPUT);
     cert::launch_relax(L0, lb_out, ub_out, n_total, batch, net->codes, net->n_relu, nullptr, 0, 0, st);
     rec.mark(CERT_CLASS_RELAX);
-    if (net->contraction == CERT_CONTRACTION_TC3XFP16 && R.fp16_ready) {
-        // fp16-split chain: pair in X[xa], raw fp32 result in X[xb], scaled pair out in X[xc]
-        float *X[3] = {R.S_hi[0], R.S_hi[1], R.S_lo[0]};
-        int ld_max = 0;
-        for (int k = 0; k < K; ++k) ld_max = std::max(ld_max, R.layers[k].ld_s);
-        const size_t lo_off = (size_t)net->max_batch * R.R * ld_max;
-        auto hi_of = [&](int p) { return reinterpret_cast<__half *>(X[p]); };
-        auto lo_of = [&](int p) { return reinterpret_cast<__half *>(X[p]) + lo_off; };
-        int xa = 0, xb = 1, xc = 2;
-        cert::launch_reuse_init16(R.W0t, L0.ld_out, L0, net->n0, R.R, R.layers[0].ld_s, rows, hi_of(xa), lo_of(xa),
-                                  net->status_dev, st);
-        rec.mark(CERT_CLASS_RELU_STEP);
-        for (int k = 1; k < K; ++k) {
-            const LayerDev &Lk = net->layers[k];
-            const ReuseLayer &RL = R.layers[k];
-            cert::TcArgs a;
-            std::memset(&a, 0, sizeof(a));
-            a.M = rows; a.K = 2 * Lk.n_in; a.n_k = 1; a.ld_n = RL.ld_s;
-            a.bn = RL.plan16.bn; a.n_tiles = RL.plan16.n_tiles; a.stages = RL.plan16.stages;
-            a.tmem_cols = RL.plan16.tmem_cols;
-            a.total_tiles = (int)cert::ceil_div_ll(rows, 256) * RL.plan16.n_tiles;
-            a.l0 = net->l0; a.u0 = net->u0;
-            a.reuse_R = R.R; a.reuse_n0 = net->n0; a.reuse_ld0 = net->ld0; a.n_half = Lk.n_out;
-            a.bias2 = RL.bias2; a.colsum = R.colsum;
-            a.status = net->status_dev;
-            const int pairs = std::min(a.total_tiles, net->sm_count / 2);
-            cert::launch_gemm_tc16(cert::TC_EPI_REUSE, pairs, RL.a16_hi[xa], RL.a16_lo[xa], RL.b16_hi, RL.b16_lo,
-                                   RL.o32[xb], RL.o32[xb], a, RL.plan16.smem_bytes, st);
-            rec.mark(CERT_CLASS_AFFINE);
-            cert::launch_reuse_relax(R.colsum, RL.ld_s, R.R / 32, Lk, batch, lb_out, ub_out, n_total, net->codes,
-                                     net->n_relu, st);
-            rec.mark(CERT_CLASS_RELAX);
-            if (k + 1 < K) {
-                cert::launch_reuse_scale16(X[xb], hi_of(xc), lo_of(xc), RL.ld_s, Lk, net->n0, R.R, rows, net->status_dev,
-                                           st);
-                rec.mark(CERT_CLASS_RELU_STEP);
-            }
-            const int t = xa; xa = xc; xc = xb; xb = t;
-        }
-        net->last_batch = batch;
-        net->last_launches = rec.launches;
-        net->last_paths = 2 | 4 | 16;
-        net->prof_marks = rec.marks;
-        if (cudaPeekAtLastError() != cudaSuccess) {
-            cudaGetLastError();
-            return CERT_ERR_CUDA;
-        }
-        return CERT_OK;
-    }
-    int cur = 0;
-    cert::launch_reuse_init(R.W0t, L0.ld_out, L0, net->n0, R.R, R.layers[0].ld_s, rows, R.S_hi[cur], R.S_lo[cur], st);
+    // pair in X[xa], raw fp32 result in X[xb], scaled pair out in X[xc]
+    auto hi_of = [&](int p) { return reinterpret_cast<__half *>(R.X[p]); };
+    auto lo_of = [&](int p) { return reinterpret_cast<__half *>(R.X[p]) + R.lo_off; };
+    int xa = 0, xb = 1, xc = 2;
+    cert::launch_reuse_init16(R.W0t, L0.ld_out, L0, net->n0, R.R, R.layers[0].ld_s, rows, hi_of(xa), lo_of(xa),
+                              net->status_dev, st);
     rec.mark(CERT_CLASS_RELU_STEP);
     for (int k = 1; k < K; ++k) {
         const LayerDev &Lk = net->layers[k];
@@ -1766,28 +1686,29 @@ cert_status_t cert_reusecert_bounds(cert_net_t *net, const float *centers, float
         cert::TcArgs a;
         std::memset(&a, 0, sizeof(a));
         a.M = rows; a.K = 2 * Lk.n_in; a.n_k = 1; a.ld_n = RL.ld_s;
-        a.bn = RL.plan.bn; a.n_tiles = RL.plan.n_tiles; a.stages = RL.plan.stages; a.tmem_cols = RL.plan.tmem_cols;
-        a.total_tiles = (int)cert::ceil_div_ll(rows, 128 * ctas) * RL.plan.n_tiles;
+        a.bn = RL.plan16.bn; a.n_tiles = RL.plan16.n_tiles; a.stages = RL.plan16.stages;
+        a.tmem_cols = RL.plan16.tmem_cols;
+        a.total_tiles = (int)cert::ceil_div_ll(rows, 256) * RL.plan16.n_tiles;
         a.l0 = net->l0; a.u0 = net->u0;
         a.reuse_R = R.R; a.reuse_n0 = net->n0; a.reuse_ld0 = net->ld0; a.n_half = Lk.n_out;
         a.bias2 = RL.bias2; a.colsum = R.colsum;
         a.status = net->status_dev;
-        const int groups = std::min(a.total_tiles, net->sm_count / ctas);
-        cert::launch_gemm_tc(cert::TC_EPI_REUSE, ctas, groups, RL.a_hi[cur], RL.a_lo[cur], RL.b_hi, RL.b_lo,
-                             RL.o_hi[cur ^ 1], RL.o_hi[cur ^ 1], a, RL.plan.smem_bytes, st);
+        const int pairs = std::min(a.total_tiles, net->sm_count / 2);
+        cert::launch_gemm_tc16(cert::TC_EPI_REUSE, pairs, RL.a16_hi[xa], RL.a16_lo[xa], RL.b16_hi, RL.b16_lo,
+                               RL.o32[xb], RL.o32[xb], a, RL.plan16.smem_bytes, st);
         rec.mark(CERT_CLASS_AFFINE);
         cert::launch_reuse_relax(R.colsum, RL.ld_s, R.R / 32, Lk, batch, lb_out, ub_out, n_total, net->codes,
                                  net->n_relu, st);
         rec.mark(CERT_CLASS_RELAX);
-        cur ^= 1;
         if (k + 1 < K) {
-            cert::launch_reuse_scale(R.S_hi[cur], R.S_lo[cur], RL.ld_s, Lk, net->n0, R.R, rows, st);
+            cert::launch_reuse_scale16(R.X[xb], hi_of(xc), lo_of(xc), RL.ld_s, Lk, net->n0, R.R, rows, net->status_dev, st);
             rec.mark(CERT_CLASS_RELU_STEP);
         }
+        const int t = xa; xa = xc; xc = xb; xb = t;
     }
     net->last_batch = batch;
     net->last_launches = rec.launches;
-    net->last_paths = 2 | (ctas == 2 ? 4 : 0);
+    net->last_paths = 2 | 4 | 16;
     net->prof_marks = rec.marks;
     if (cudaPeekAtLastError() != cudaSuccess) {
         cudaGetLastError();
@@ -1884,7 +1805,11 @@ int cert_net_auto_contraction(const cert_net_t *net) {
     return net->tc_ok ? CERT_CONTRACTION_TC3XTF32 : CERT_CONTRACTION_FFMA;
 }
 
-float cert_net_fp16_coefficient_bound(const cert_net_t *net) { return net ? net->fp16_coef_bound : -1.0f; }
+float cert_net_fp16_coefficient_bound(const cert_net_t *net, int layer) {
+    if (!net || layer >= net->n_layers) return -1.0f;
+    if (layer < 0) return net->fp16_coef_bound;
+    return layer < (int)net->fp16_layer_bound.size() ? net->fp16_layer_bound[layer] : INFINITY;
+}
 
 cert_status_t cert_net_set_contraction(cert_net_t *net, int mode) {
     if (!net) return CERT_ERR_INVALID_ARG;

@@ -205,21 +205,15 @@ void launch_to_ymajor_vectors(int c, int h, int w, int ld, int batch, int n_arr,
 
 // ---- ReuseCert (reuse.cu): shapes over the input layer, one matrix S per layer ----
 // S rows are (box, s): s < n0 input coordinate, s == n0 constant, zero rows up to R per box; columns
-// [L (n) | U (n)] padded to ld_s.  S is held as a TF32 pair.
-void launch_reuse_init(const float *W0t, int ldw, const LayerDev &L0, int n0, int R, int ld_s, long long rows,
-                       float *S_hi, float *S_lo, cudaStream_t st);
+// [L (n) | U (n)] padded to ld_s.  S is held as an fp16 pair (x = hi + 2^-11 lo); `status` bit 1 is raised when
+// a value leaves the fp16 range.
 // Bounds (and the relaxation, under a ReLU) of layer L from the contraction's column sums.
 void launch_reuse_relax(const float *colsum, int ld_s, int groups_per_box, const LayerDev &L, int batch,
                         float *lb_out, float *ub_out, int n_total, unsigned char *codes, int n_relu,
                         cudaStream_t st);
-// The fp16-split forms: S as an fp16 pair (x = hi + 2^-11 lo); `status` bit 1 is raised when a value leaves
-// the fp16 range.  The scale step reads the raw fp32 result from one buffer and writes the pair to others.
+// The first layer's S, and the scale step (reads the raw fp32 result from one buffer, writes the pair to others).
 void launch_reuse_init16(const float *W0t, int ldw, const LayerDev &L0, int n0, int R, int ld_s, long long rows,
                          __half *S_hi, __half *S_lo, int *status, cudaStream_t st);
 void launch_reuse_scale16(const float *raw, __half *S_hi, __half *S_lo, int ld_s, const LayerDev &L, int n0, int R,
                           long long rows, int *status, cudaStream_t st);
-// Raw [L | U] of layer L (fp32 in S_hi) -> S of its outputs, in place.
-void launch_reuse_scale(float *S_hi, float *S_lo, int ld_s, const LayerDev &L, int n0, int R, long long rows,
-                        cudaStream_t st);
-
 }  // namespace cert

@@ -61,7 +61,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_consta
     constexpr bool kRelu = (EPI == TC_EPI_RELU || EPI == TC_EPI_RELU_SKIP || EPI == TC_EPI_RELU_BAND ||
                             EPI == TC_EPI_RELU_BAND_SKIP);
     constexpr bool kSkip = (EPI == TC_EPI_RELU_SKIP || EPI == TC_EPI_RELU_BAND_SKIP);
-    constexpr bool kStores = kRelu || EPI == TC_EPI_REUSE;
+    constexpr bool kStores = kRelu;
     pdl_trigger();
     extern __shared__ uint8_t smem_raw[];
     // tiles are aligned to 1024 bytes (a whole swizzle pattern)
@@ -374,58 +374,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_consta
                         if (a.split_out) tma_store_2d(&map_o_lo, smem_u32(slab_lo), col0, (int)warp_row0);
                         tma_store_commit();
                     }
-                } else if (EPI == TC_EPI_REUSE) {
-                    if (lane == 0) tma_store_wait_read();
-                    __syncwarp();
-                    const int bx = (int)(rr / a.reuse_R), s_in = (int)(rr % a.reuse_R);
-                    const bool is_const = s_in == a.reuse_n0;
-                    const bool is_coord = s_in < a.reuse_n0;
-                    const float lo_s = is_coord ? a.l0[(size_t)bx * a.reuse_ld0 + s_in] : 0.0f;
-                    const float up_s = is_coord ? a.u0[(size_t)bx * a.reuse_ld0 + s_in] : 0.0f;
-                    const uint32_t row_hi = smem_u32(slab_hi) + (uint32_t)lane * 128u;
-                    float w[32];
-#pragma unroll
-                    for (int g = 0; g < 8; ++g) {
-                        float q[4];
-                        const float4 bz = *reinterpret_cast<const float4 *>(a.bias2 + col0 + g * 4);
-                        const float b4[4] = {bz.x, bz.y, bz.z, bz.w};
-#pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            const int col = col0 + g * 4 + e;
-                            float c = __uint_as_float(v[g * 4 + e]);
-                            if (is_const) c += b4[e];
-                            q[e] = c;
-                            // simplify_lower for a lower shape, simplify_upper for an upper one; the constant as it is
-                            const bool upper_col = col >= a.n_half;
-                            const bool nonneg = (c >= 0.0f);
-                            float term = c * ((nonneg != upper_col) ? lo_s : up_s);
-                            if (is_const) term = c;
-                            w[g * 4 + e] = (row_ok && col < 2 * a.n_half) ? term : 0.0f;
-                        }
-                        const uint32_t sw = (uint32_t)((g ^ (lane & 7)) << 4);
-                        asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(row_hi + sw), "f"(q[0]),
-                                     "f"(q[1]), "f"(q[2]), "f"(q[3]) : "memory");
-                    }
-                    fence_async_smem();
-                    __syncwarp();
-                    if (lane == 0) {
-                        tma_store_2d(&map_o_hi, smem_u32(slab_hi), col0, (int)warp_row0);
-                        tma_store_commit();
-                    }
-                    // Column sums over the warp's 32 rows by recursive halving: after the step with
-                    // distance d a lane keeps the columns whose index has the lane's bit d, so lane L
-                    // ends with column L.  Fixed order.
-#pragma unroll
-                    for (int d = 16; d >= 1; d >>= 1) {
-                        const bool hi_half = (lane & d) != 0;
-#pragma unroll
-                        for (int j = 0; j < d; ++j) {
-                            const float send = hi_half ? w[j] : w[j + d];
-                            const float keep = hi_half ? w[j + d] : w[j];
-                            w[j] = keep + __shfl_xor_sync(0xffffffffu, send, d);
-                        }
-                    }
-                    if (warp_row0 < a.M) a.colsum[(size_t)(warp_row0 >> 5) * a.ld_n + col0 + lane] = w[0];
                 } else if (row_ok) {
                     const float *lrow = a.l0 + relax_row + col0;
                     const float *urow = a.u0 + relax_row + col0;
@@ -448,7 +396,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_consta
             if (lane == 0) mbar_arrive_cluster(acc_empty_addr0 + (uint32_t)(acc * sizeof(uint64_t)));
             // This tile's share of the row constant (of the bound, for the concretising
             // epilogue) goes to slot nt; the tile of column 0 also carries the constant so far.
-            if (EPI != TC_EPI_REUSE && row_ok) {
+            if (row_ok) {
                 float tot = dacc;
                 const int slot = band * n_tiles + nt;
                 if (slot == 0) {
@@ -551,8 +499,7 @@ bool tc_prepare_kernels(bool *pair_ok) {
     e[1] = cudaFuncSetAttribute(gemm_tc_kernel<TC_EPI_CONCRETIZE, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemMax);
     e[2] = cudaFuncSetAttribute(gemm_tc_kernel<TC_EPI_RELU, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemMax);
     e[3] = cudaFuncSetAttribute(gemm_tc_kernel<TC_EPI_CONCRETIZE, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemMax);
-    e[4] = cudaFuncSetAttribute(gemm_tc_kernel<TC_EPI_REUSE, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemMax);
-    e[5] = cudaFuncSetAttribute(gemm_tc_kernel<TC_EPI_REUSE, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemMax);
+    e[4] = e[5] = cudaSuccess;      // (slots of a variant that no longer exists)
     for (int i = 0; i < 14; ++i)
         if (e[i] != cudaSuccess) {
             cudaGetLastError();
@@ -642,11 +589,9 @@ void launch_gemm_tc(int epi, int ctas, int groups, const TcMap &a_hi, const TcMa
     }
     if (ctas == 2) {
         if (epi == TC_EPI_RELU) launch_one<TC_EPI_RELU, 2>(groups, ah, al, bh, bl, oh, ol, args, smem_bytes, st);
-        else if (epi == TC_EPI_REUSE) launch_one<TC_EPI_REUSE, 2>(groups, ah, al, bh, bl, oh, ol, args, smem_bytes, st);
         else launch_one<TC_EPI_CONCRETIZE, 2>(groups, ah, al, bh, bl, oh, ol, args, smem_bytes, st);
     } else {
         if (epi == TC_EPI_RELU) launch_one<TC_EPI_RELU, 1>(groups, ah, al, bh, bl, oh, ol, args, smem_bytes, st);
-        else if (epi == TC_EPI_REUSE) launch_one<TC_EPI_REUSE, 1>(groups, ah, al, bh, bl, oh, ol, args, smem_bytes, st);
         else launch_one<TC_EPI_CONCRETIZE, 1>(groups, ah, al, bh, bl, oh, ol, args, smem_bytes, st);
     }
 }

@@ -69,7 +69,7 @@ struct TcArgs {
     float *d_out;
     int n_slots_in;
     long long slot_stride;
-    // TC_EPI_REUSE (shapes kept over the input layer): a row is (box, s) with s < reuse_n0 an input
+    // TC_EPI_REUSE (fp16-split kernel only; shapes kept over the input layer): a row is (box, s) with s < reuse_n0 an input
     // coordinate, s == reuse_n0 the constant, rows per box = reuse_R (a multiple of 32); a column is a
     // neuron's lower (col < n_half) or upper (n_half <= col < 2*n_half) shape.  The result is stored
     // unsplit; bias2[col] is added on the constant row; colsum[(row / 32) * ld_n + col] receives the sum

@@ -8,7 +8,7 @@
 //   column t < n:  lower shape L_t,  column n + t: upper shape U_t,  zero columns up to the pitch.
 // With that layout "replace every ReLU neuron below by its stored L / U" (replace_lower/upper) is
 //   [L_k | U_k] = S_{k-1} * [[W+^T, W-^T], [W-^T, W+^T]]   (+ the bias on the constant row),
-// one contraction per affine layer with rows = boxes x R, which the tensor-core kernel runs; its
+// one contraction per affine layer with rows = boxes x R, which the fp16-split tensor-core kernel runs; its
 // epilogue also leaves, per 32 rows, every column's concretisation terms (map(simplify_*)).
 // The kernels here start the chain, turn those sums into bounds and relaxations (Relu transformer:
 // relu_n, compute_upper on l = L.map(simplify_lower), u = U.map(simplify_upper)), and scale the raw
@@ -20,48 +20,6 @@
 namespace cert {
 
 namespace {
-
-__device__ __forceinline__ float tf32_round(float x) {
-    uint32_t r;
-    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(x));
-    return __uint_as_float(r);
-}
-
-// S of the first layer from its transposed weights W0t [>= n0 rows][ldw] and bias, scaled by the
-// relaxation of its ReLU (lamL = lamU = 1, nuU = 0 without one).  One thread per 4 columns.
-__global__ void reuse_init_kernel(const float *__restrict__ W0t, int ldw, const float *__restrict__ bias,
-                                  int n, int n0, int R, int ld_s, int ld_relax, int has_relu,
-                                  const float *__restrict__ lamL, const float *__restrict__ lamU,
-                                  const float *__restrict__ nuU, long long rows, float *__restrict__ S_hi,
-                                  float *__restrict__ S_lo) {
-    const int quads = ld_s / 4;
-    const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-    if (idx >= rows * quads) return;
-    const long long r = idx / quads;
-    const int col0 = (int)(idx % quads) * 4;
-    const int box = (int)(r / R), s = (int)(r % R);
-    float h[4], l[4];
-#pragma unroll
-    for (int e = 0; e < 4; ++e) {
-        const int col = col0 + e;
-        float v = 0.0f;
-        if (col < 2 * n && s <= n0) {
-            const bool upper = col >= n;
-            const int t = upper ? col - n : col;
-            const float base = s < n0 ? W0t[(size_t)s * ldw + t] : bias[t];
-            float lam = 1.0f, nu = 0.0f;
-            if (has_relu) {
-                lam = upper ? lamU[(size_t)box * ld_relax + t] : lamL[(size_t)box * ld_relax + t];
-                nu = (upper && s == n0) ? nuU[(size_t)box * ld_relax + t] : 0.0f;
-            }
-            v = fmaf(lam, base, nu);
-        }
-        h[e] = tf32_round(v);
-        l[e] = tf32_round(v - h[e]);
-    }
-    *reinterpret_cast<float4 *>(S_hi + (size_t)r * ld_s + col0) = make_float4(h[0], h[1], h[2], h[3]);
-    *reinterpret_cast<float4 *>(S_lo + (size_t)r * ld_s + col0) = make_float4(l[0], l[1], l[2], l[3]);
-}
 
 // Bounds of layer k from the column sums the contraction left (R/32 partial sums per box and column,
 // added in order), then the Relu transformer.  One thread per (box, padded neuron).
@@ -106,42 +64,9 @@ __global__ void reuse_relax_kernel(const float *__restrict__ colsum, int ld_s, i
     nuU[idx] = nu;
 }
 
-// S_k from the raw [L_k | U_k] (in place: hi overwrites the raw value): L_t *= lamL_t; U_t = lamU_t * U_t,
-// + nuU_t on the constant row.  Without a ReLU the shapes pass unchanged.  One thread per 4 columns.
-__global__ void reuse_scale_kernel(float *__restrict__ S_hi, float *__restrict__ S_lo, int ld_s, int n, int n0, int R,
-                                   int ld_relax, int has_relu, const float *__restrict__ lamL,
-                                   const float *__restrict__ lamU, const float *__restrict__ nuU, long long rows) {
-    const int quads = ld_s / 4;
-    const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-    if (idx >= rows * quads) return;
-    const long long r = idx / quads;
-    const int col0 = (int)(idx % quads) * 4;
-    const int box = (int)(r / R), s = (int)(r % R);
-    const float4 raw = *reinterpret_cast<const float4 *>(S_hi + (size_t)r * ld_s + col0);
-    const float rv[4] = {raw.x, raw.y, raw.z, raw.w};
-    float h[4], l[4];
-#pragma unroll
-    for (int e = 0; e < 4; ++e) {
-        const int col = col0 + e;
-        float v = 0.0f;
-        if (col < 2 * n && s <= n0) {
-            v = rv[e];
-            if (has_relu) {
-                const bool upper = col >= n;
-                const int t = upper ? col - n : col;
-                const float lam = upper ? lamU[(size_t)box * ld_relax + t] : lamL[(size_t)box * ld_relax + t];
-                const float nu = (upper && s == n0) ? nuU[(size_t)box * ld_relax + t] : 0.0f;
-                v = fmaf(lam, v, nu);
-            }
-        }
-        h[e] = tf32_round(v);
-        l[e] = tf32_round(v - h[e]);
-    }
-    *reinterpret_cast<float4 *>(S_hi + (size_t)r * ld_s + col0) = make_float4(h[0], h[1], h[2], h[3]);
-    *reinterpret_cast<float4 *>(S_lo + (size_t)r * ld_s + col0) = make_float4(l[0], l[1], l[2], l[3]);
-}
-
-// The fp16-split forms (x = hi + 2^-11 lo, see gemm_tc16.cuh): the same two steps writing halves.
+// S_k from the raw [L_k | U_k]: L_t *= lamL_t; U_t = lamU_t * U_t, + nuU_t on the constant row (without a ReLU
+// the shapes pass unchanged), and S of the first layer from its weights, both written as fp16 pairs
+// (x = hi + 2^-11 lo, see gemm_tc16.cuh).
 constexpr float kLoScale16 = 2048.0f;
 
 __device__ __forceinline__ void store_pair16(float v, __half &h, __half &l, bool &out_of_range) {
@@ -251,13 +176,6 @@ void launch_reuse_scale16(const float *raw, __half *S_hi, __half *S_lo, int ld_s
         raw, S_hi, S_lo, ld_s, L.n_out, n0, R, L.ld_out, L.relu_after, L.lamL, L.lamU, L.nuU, rows, status);
 }
 
-void launch_reuse_init(const float *W0t, int ldw, const LayerDev &L0, int n0, int R, int ld_s, long long rows,
-                       float *S_hi, float *S_lo, cudaStream_t st) {
-    const long long threads = rows * (ld_s / 4);
-    reuse_init_kernel<<<(unsigned)ceil_div_ll(threads, 256), 256, 0, st>>>(
-        W0t, ldw, L0.bias_n, L0.n_out, n0, R, ld_s, L0.ld_out, L0.relu_after, L0.lamL, L0.lamU, L0.nuU, rows, S_hi, S_lo);
-}
-
 void launch_reuse_relax(const float *colsum, int ld_s, int groups_per_box, const LayerDev &L, int batch,
                         float *lb_out, float *ub_out, int n_total, unsigned char *codes, int n_relu,
                         cudaStream_t st) {
@@ -265,13 +183,6 @@ void launch_reuse_relax(const float *colsum, int ld_s, int groups_per_box, const
     reuse_relax_kernel<<<(unsigned)ceil_div_ll(threads, 256), 256, 0, st>>>(
         colsum, ld_s, groups_per_box, L.n_out, L.ld_out, batch, lb_out, ub_out, n_total, L.out_off, L.relu_after,
         L.lamL, L.lamU, L.nuU, codes, n_relu, L.relu_off);
-}
-
-void launch_reuse_scale(float *S_hi, float *S_lo, int ld_s, const LayerDev &L, int n0, int R, long long rows,
-                        cudaStream_t st) {
-    const long long threads = rows * (ld_s / 4);
-    reuse_scale_kernel<<<(unsigned)ceil_div_ll(threads, 256), 256, 0, st>>>(
-        S_hi, S_lo, ld_s, L.n_out, n0, R, L.ld_out, L.relu_after, L.lamL, L.lamU, L.nuU, rows);
 }
 
 }  // namespace cert

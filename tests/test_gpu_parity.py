@@ -35,7 +35,7 @@ def test_config5_all_boxes(mode):
     w = wl.make_config(4)
     g = run_gpu(w, contraction={"ffma": 1, "tc": 2, "tc16": 3, "auto": 0}[mode])
     if mode in ("tc16", "auto"):
-        assert g["paths"] & 16            # AUTO proves the fp16 range at create and takes the fp16 split
+        assert g["paths"] & 16            # AUTO proves the fp16 range of the wide layers' traversals at create
     r = compare(g, cached_oracle(w), label=f"{w.name}/{mode}", min_compared=0.9)
     assert r["boxes"] == 128
 
@@ -273,11 +273,10 @@ REUSE_NETS = {
 }
 
 
-# ReuseCert feeds every layer with the rounded shapes of the layer below, so float32 rounding compounds
-# through the layers (measured: x3..5 per layer, 1.1e-4 at the fourth layer of the 64-300-130-257-3 net),
-# where DeepPoly restarts each traversal from the exact weights.  Its bounds are therefore compared at
-# 5e-4 * (1 + |oracle|); the branch codes must still be identical on well-conditioned boxes.
-REUSE_TOL = 5e-4
+# ReuseCert feeds every layer with the rounded shapes of the layer below, so float32 rounding compounds through
+# the layers where DeepPoly restarts each traversal from the exact weights.  The library serves it in the fp16
+# split only, which holds the common tolerance.
+REUSE_TOL = 1e-4
 
 
 def _run_reusecert(w, max_batch=None, contraction=None):
@@ -305,12 +304,12 @@ def _run_reusecert(w, max_batch=None, contraction=None):
     return out, dp
 
 
-@pytest.mark.parametrize("mode", ["tc", "tc16"])
+@pytest.mark.parametrize("mode", ["auto", "tc16"])
 @pytest.mark.parametrize("name", sorted(REUSE_NETS))
 def test_reusecert(name, mode):
     w = REUSE_NETS[name]()
     ref = orc.reusecert(w.layers, w.centers, w.eps, w.clip_lo, w.clip_hi)
-    out, dp = _run_reusecert(w, max_batch=w.batch + 3, contraction={"tc": 2, "tc16": 3}[mode])
+    out, dp = _run_reusecert(w, max_batch=w.batch + 3, contraction={"auto": 0, "tc16": 3}[mode])
     for i, g in enumerate(out):
         compare(g, ref, label=f"reusecert/{name}/{mode}/call{i}", tol=REUSE_TOL)
     assert np.array_equal(out[0]["lb"], out[1]["lb"]) and np.array_equal(out[0]["ub"], out[1]["ub"])
@@ -334,9 +333,20 @@ def test_reusecert_needs_enable_and_fc_layers():
         assert binding.lib.cert_net_enable_reusecert(net._h) == 2
     finally:
         net.destroy()
+    # a net pinned to the TF32 split or the FMA units is refused: ReuseCert runs in the fp16 split only
+    net = binding.CertNet(w.layers, 2)
+    try:
+        net.enable_reusecert()
+        c = torch.from_numpy(w.centers).cuda()
+        out = torch.empty((2, net.n_total), device="cuda")
+        for mode in (1, 2):
+            net.set_contraction(mode)
+            assert binding.lib.cert_reusecert_bounds(net._h, c.data_ptr(), 0.1, 2, out.data_ptr(), out.data_ptr(), None) == 2
+    finally:
+        net.destroy()
 
 
-@pytest.mark.parametrize("mode", ["tc", "tc16"])
+@pytest.mark.parametrize("mode", ["auto"])
 def test_reusecert_config5_all_boxes(mode):
     """784 -> 1024 x 6 -> 10, 128 boxes on the GPU (the benchmark's launch configuration), every box against the
     oracle.  With 6144 ReLU neurons per box and ReuseCert's wider bounds most boxes have some neuron whose sign
@@ -348,7 +358,7 @@ def test_reusecert_config5_all_boxes(mode):
     ref = cached_oracle(w, "reusecert")
     net = binding.CertNet(w.layers, w.batch, w.clip_lo, w.clip_hi)
     try:
-        net.set_contraction({"tc": 2, "tc16": 3}[mode])
+        net.set_contraction({"auto": 0, "tc16": 3}[mode])
         net.enable_reusecert()
         lb, ub = net.reusecert_bounds(torch.from_numpy(w.centers).cuda(), w.eps)
         torch.cuda.synchronize()
@@ -459,31 +469,37 @@ def _pm300_net():
 
 
 def test_auto_takes_the_fp16_split_only_where_the_weights_prove_its_range():
-    """CERT_CONTRACTION_AUTO: the largest entry of |W_k| ... |W_j| bounds every coefficient a traversal can hold.
-    Weights of +-300 give 16 * 300 * 300 > 65504: AUTO must stay on the TF32 split and return the oracle's bounds;
-    an ordinary net passes the proof and runs in the fp16 split."""
+    """CERT_CONTRACTION_AUTO, decided per layer: the largest entry of |W_k| ... |W_j| bounds every coefficient the
+    traversal of layer k can hold.  Weights of +-300 in a 8-16-16-4 net: the traversal of layer 1 holds |W_1| = 300
+    (fp16 split), that of layer 2 could reach 16 * 300 * 300 > 65504 and must run in the TF32 split; the bounds
+    are the oracle's.  An ordinary net passes the proof everywhere."""
     from paper_2507_20055_b200 import binding
     w = _pm300_net()
     net = binding.CertNet(w.layers, w.batch, w.clip_lo, w.clip_hi)
     try:
-        assert net.auto_contraction() == 2 and net.fp16_coefficient_bound() >= 16 * 300.0 * 300.0 * 0.999
+        assert net.fp16_coefficient_bound(1) == 300.0
+        assert net.fp16_coefficient_bound(2) >= 16 * 300.0 * 300.0 * 0.999
+        assert net.fp16_coefficient_bound() == net.fp16_coefficient_bound(2)
+        assert net.fp16_coefficient_bound(3) == -1.0            # no such layer
     finally:
         net.destroy()
     g = run_gpu(w)
-    assert g["paths"] & 2 and not g["paths"] & 16
+    assert g["paths"] & 2 and g["paths"] & 16         # both splits ran in the one call
     compare(g, _oracle(w), label="pm300/auto")
     w = wl.small_fc([33, 64, 300, 64, 10], batch=4, eps=0.04, seed=75)
     net = binding.CertNet(w.layers, w.batch, w.clip_lo, w.clip_hi)
     try:
         assert net.auto_contraction() == 3
-        # the bound really is the largest entry of the products of the absolute weights
+        # the bounds really are the largest entries of the products of the absolute weights
         a = [np.abs(l.weight.astype(np.float64)) for l in w.layers]
-        expect = max([m.max() for m in a[1:]] + [(a[2] @ a[1]).max(), (a[3] @ a[2]).max(), (a[3] @ a[2] @ a[1]).max()])
-        assert abs(net.fp16_coefficient_bound() - expect) <= 1e-5 * expect
+        expect = {1: a[1].max(), 2: max(a[2].max(), (a[2] @ a[1]).max()),
+                  3: max(a[3].max(), (a[3] @ a[2]).max(), (a[3] @ a[2] @ a[1]).max())}
+        for k, e in expect.items():
+            assert abs(net.fp16_coefficient_bound(k) - e) <= 1e-5 * e
     finally:
         net.destroy()
     g = run_gpu(w)
-    assert g["paths"] & 16
+    assert g["paths"] & 16 and not g["paths"] & 1
     compare(g, _oracle(w), label="ordinary/auto")
 
 
