@@ -31,7 +31,8 @@ typedef enum {
     CERT_ERR_BATCH_TOO_LARGE = 4, /* batch > max_batch given at create                           */
     CERT_ERR_CUDA = 5,            /* a CUDA runtime or driver call failed                        */
     CERT_ERR_TIMEOUT = 6,         /* a bounded device-side wait ran out (see cert_net_last_status) */
-    CERT_ERR_RANGE = 7            /* a coefficient left the fp16 range of CERT_CONTRACTION_TC3XFP16  */
+    CERT_ERR_RANGE = 7,           /* a coefficient left the fp16 range of CERT_CONTRACTION_TC3XFP16  */
+    CERT_ERR_BOUNDS = 8           /* checking build only: a kernel tried to store outside every buffer */
 } cert_status_t;
 
 enum { CERT_LAYER_FC = 0, CERT_LAYER_CONV2D = 1 };
@@ -193,8 +194,9 @@ cert_status_t cert_net_branch_codes(cert_net_t *net, unsigned char *codes_out, v
  * Sticky device-side status.  Waits `stream`, then returns CERT_ERR_TIMEOUT
  * if any kernel of an earlier call on this net gave up a bounded wait,
  * CERT_ERR_RANGE if a coefficient left the fp16 range in TC3XFP16 mode (the
- * results are invalid in both cases), CERT_ERR_CUDA if the stream reports an
- * error, else CERT_OK.  Clears the flag.
+ * results are invalid in both cases), CERT_ERR_BOUNDS if a checked store was
+ * refused (checking build, see cert_net_selftest_checked_store), CERT_ERR_CUDA
+ * if the stream reports an error, else CERT_OK.  Clears the flag.
  */
 cert_status_t cert_net_last_status(cert_net_t *net, void *stream);
 
@@ -296,6 +298,20 @@ cert_status_t cert_net_profile(cert_net_t *net, float *ms_out /* HOST [CERT_N_CL
  * overwritten (a kernel wrote outside its buffer), -1 = null net or a CUDA error.  Test and debugging aid.
  */
 int cert_net_check_guards(cert_net_t *net, void *stream);
+
+/*
+ * Checked stores (no counterpart in the paper; memory-safety evidence beside the guard words).  A library built
+ * with -DCERT_BOUNDS (paper_2507_20055_b200/build.py: build(defines=["CERT_BOUNDS"], lib=...)) looks up the
+ * address of every plain global store of its non-TMA kernels in a table of the buffers the call may write (the
+ * net's allocations, the caller's lb_out / ub_out); a store outside all of them is skipped and reported as
+ * CERT_ERR_BOUNDS by cert_net_last_status.  Slow; for tests on small shapes.
+ *   cert_built_with_checked_stores   1 in such a build, else 0.
+ *   cert_net_selftest_checked_store  enqueues one kernel that attempts a checked store one float past the end of
+ *            one of the net's buffers: the store is skipped (the guard words stay intact) and the next
+ *            cert_net_last_status returns CERT_ERR_BOUNDS.  CERT_ERR_UNSUPPORTED in an ordinary build.
+ */
+int cert_built_with_checked_stores(void);
+cert_status_t cert_net_selftest_checked_store(cert_net_t *net, void *stream);
 
 /* Number of kernels the most recent cert_deeppoly_bounds call enqueued. */
 int cert_net_last_launch_count(const cert_net_t *net);

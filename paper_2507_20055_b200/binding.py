@@ -13,7 +13,8 @@ from typing import Optional, Sequence
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libcert_b200.so")
+# CERT_LIB selects another build of the same library (the checking build of build.py), for tests
+LIB_PATH = os.environ.get("CERT_LIB") or os.path.join(_HERE, "libcert_b200.so")
 
 if not os.path.exists(LIB_PATH):
     raise ImportError(
@@ -35,7 +36,7 @@ EXPORTS = [
     "cert_net_last_contraction_paths", "cert_first_layer_bounds_noalloc", "cert_net_set_conv_patches",
     "cert_net_enable_reusecert", "cert_reusecert_bounds", "cert_reusecert_bounds_host",
     "cert_net_check_guards", "cert_net_auto_contraction", "cert_net_fp16_coefficient_bound",
-    "cert_peak_microbench",
+    "cert_peak_microbench", "cert_built_with_checked_stores", "cert_net_selftest_checked_store",
 ]
 CLASS_NAMES = ["input", "relax", "relu_step", "affine", "conv", "concretize"]
 
@@ -100,6 +101,10 @@ _lib.cert_net_auto_contraction.argtypes = [_vp]
 _lib.cert_net_auto_contraction.restype = _i
 _lib.cert_net_fp16_coefficient_bound.argtypes = [_vp, _i]
 _lib.cert_net_fp16_coefficient_bound.restype = ctypes.c_float
+_lib.cert_built_with_checked_stores.argtypes = []
+_lib.cert_built_with_checked_stores.restype = _i
+_lib.cert_net_selftest_checked_store.argtypes = [_vp, _vp]
+_lib.cert_net_selftest_checked_store.restype = _i
 _lib.cert_peak_microbench.argtypes = [_i, ctypes.c_double, _vp, _vp, _vp, _vp]
 _lib.cert_peak_microbench.restype = _i
 _lib.cert_status_string.argtypes = [_i]
@@ -305,6 +310,10 @@ class CertNet:
 
     def set_conv_patches(self, on: bool):
         _check(_lib.cert_net_set_conv_patches(self._h, int(bool(on))), "cert_net_set_conv_patches")
+
+    def selftest_checked_store(self, stream_ptr: int = 0):
+        """Checking build only: one store just past a buffer, which is refused; last_status() then reports 8."""
+        _check(_lib.cert_net_selftest_checked_store(self._h, stream_ptr), "cert_net_selftest_checked_store")
 
     def check_guards(self, stream_ptr: int = 0) -> int:
         """0 = every guard word around the net's device buffers is intact, i + 1 = allocation i was overrun."""

@@ -37,10 +37,21 @@ def needs_build() -> bool:
     return any(os.path.getmtime(d) > t for d in sources() + headers())
 
 
+CHECKED_LIB = os.path.join(HERE, "libcert_b200_checked.so")
+
+
+def build_checked(force: bool = False) -> str:
+    """The checking build (-DCERT_BOUNDS: every plain global store of the non-TMA kernels is looked up in a table
+    of the call's writable buffers first), as a library of its own beside the ordinary one."""
+    return build(force=force, defines=("CERT_BOUNDS",), lib=CHECKED_LIB)
+
+
 def build(force: bool = False, verbose: bool = False, defines=(), lib: str = LIB) -> str:
     """defines: extra -D macros (a checking build goes to a library of its own, see `lib`)."""
-    if not (force or lib != LIB or needs_build()) and os.path.exists(lib):
-        return lib
+    if not force and os.path.exists(lib):
+        t = os.path.getmtime(lib)
+        if not any(os.path.getmtime(d) > t for d in sources() + headers()):
+            return lib
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
     os.makedirs(OBJ, exist_ok=True)
     tag = "".join(sorted(d.replace("=", "_") + "." for d in defines))
@@ -62,4 +73,7 @@ def build(force: bool = False, verbose: bool = False, defines=(), lib: str = LIB
 
 if __name__ == "__main__":
     import sys
-    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    if "--checked" in sys.argv:
+        print(build_checked(force="--force" in sys.argv))
+    else:
+        print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))

@@ -150,6 +150,17 @@ struct cert_net {
 
 constexpr int kMaxPatchLevels = 16;
 
+#ifdef CERT_BOUNDS
+namespace { std::vector<void (*)(const cert::BoundsTable *)> &bounds_uploaders(); }
+namespace cert {
+void bounds_register_uploader(void (*upload)(const BoundsTable *)) { bounds_uploaders().push_back(upload); }
+void bounds_upload_all(const BoundsTable *t) {
+    cudaDeviceSynchronize();
+    for (auto fn : bounds_uploaders()) fn(t);
+}
+}  // namespace cert
+#endif
+
 namespace cert {
 bool convt_supported(const LayerDev &L);
 void convt_prepare();
@@ -391,6 +402,9 @@ cert_status_t setup_tensor_core_path(cert_net *net, const cert_layer_desc_t *des
 // kFp16Safe the fp16 split cannot overflow in that layer's traversal, whatever the input boxes, and AUTO takes
 // it for that layer (the products grow with the number of layers a traversal passes, so on deep nets the first
 // layers pass and the last ones stay on the TF32 split).
+#ifdef CERT_BOUNDS
+cert_status_t bounds_sync(cert_net *net, const void *const *extra, const size_t *extra_bytes, int n_extra);
+#endif
 constexpr float kFp16Safe = 60000.0f;       // fp16's largest finite value is 65504; the margin covers fp32 rounding here
 
 cert_status_t prove_fp16_range(cert_net *net) {
@@ -399,6 +413,12 @@ cert_status_t prove_fp16_range(cert_net *net) {
     net->fp16_coef_bound = INFINITY;
     net->fp16_layer_bound.assign(K, INFINITY);
     if (!net->tc16_ok || !net->skip_from.empty()) return CERT_OK;
+#ifdef CERT_BOUNDS
+    {
+        const cert_status_t bs = bounds_sync(net, nullptr, nullptr, 0);     // the products go through the checked FMA kernel
+        if (bs != CERT_OK) return bs;
+    }
+#endif
     std::vector<float *> absW(K, nullptr);
     float *max_dev = nullptr;
     cert_status_t rc = CERT_OK;
@@ -704,6 +724,36 @@ struct Recorder {
         cudaEventRecord(net->prof_events[marks], st);
     }
 };
+
+#ifdef CERT_BOUNDS
+// Checking build: the table of writable buffers (every allocation of the net plus the caller's arrays) goes to
+// every translation unit's device copy before a call's first launch.
+std::vector<void (*)(const cert::BoundsTable *)> &bounds_uploaders() {
+    static std::vector<void (*)(const cert::BoundsTable *)> v;
+    return v;
+}
+
+cert_status_t bounds_sync(cert_net *net, const void *const *extra, const size_t *extra_bytes, int n_extra) {
+    static cert::BoundsTable t;
+    t.n = 0;
+    t.status = net->status_dev;
+    for (const cert_net::Guarded &g : net->guards) {
+        if (t.n >= cert::kBoundsMax) return CERT_ERR_UNSUPPORTED;
+        t.lo[t.n] = (unsigned long long)(g.base + kGuardBytes);
+        t.hi[t.n] = t.lo[t.n] + g.bytes;
+        ++t.n;
+    }
+    for (int i = 0; i < n_extra; ++i) {
+        if (t.n >= cert::kBoundsMax) return CERT_ERR_UNSUPPORTED;
+        t.lo[t.n] = (unsigned long long)extra[i];
+        t.hi[t.n] = t.lo[t.n] + extra_bytes[i];
+        ++t.n;
+    }
+    cert::bounds_upload_all(&t);
+    if (cudaGetLastError() != cudaSuccess) return CERT_ERR_CUDA;
+    return CERT_OK;
+}
+#endif
 
 // ---- the per-call schedule: one function per way a layer's traversal can run ----
 
@@ -1195,6 +1245,14 @@ cert_status_t backsub_impl(cert_net *net, const float *centers, float eps, int b
     if (residual && backsteps && (forced_mode >= 0 ? forced_mode : net->contraction) == CERT_CONTRACTION_TC3XFP16)
         for (int k = 1; k < K; ++k)
             if (backsteps[k] >= 0 && backsteps[k] < k) return CERT_ERR_UNSUPPORTED;   // fp16 split: full traversals only
+#ifdef CERT_BOUNDS
+    {
+        const void *extra[2] = {lb_out, ub_out};
+        const size_t bytes[2] = {(size_t)batch * net->n_total * sizeof(float), (size_t)batch * net->n_total * sizeof(float)};
+        const cert_status_t bs = bounds_sync(net, extra, bytes, 2);
+        if (bs != CERT_OK) return bs;
+    }
+#endif
     Recorder rec(net, st);
     int paths = 0;
 
@@ -1258,6 +1316,7 @@ const char *cert_status_string(cert_status_t s) {
         case CERT_ERR_CUDA: return "CUDA error";
         case CERT_ERR_TIMEOUT: return "device-side wait timed out";
         case CERT_ERR_RANGE: return "coefficient outside the fp16 range of the TC3XFP16 contraction";
+        case CERT_ERR_BOUNDS: return "a checked store fell outside every buffer (checking build)";
     }
     return "unknown";
 }
@@ -1486,6 +1545,15 @@ cert_status_t cert_deeppoly_bounds_host(cert_net_t *net, const float *centers_ho
     return cert_backsub_bounds_host(net, centers_host, eps, batch, nullptr, lb_host, ub_host, stream);
 }
 
+// The status code a non-zero status word stands for: a run-out wait first, then a refused store of the checking
+// build, then an fp16 overflow.
+static cert_status_t status_of_flag(int flag) {
+    if (flag & 1) return CERT_ERR_TIMEOUT;
+    if (flag & 4) return CERT_ERR_BOUNDS;
+    if (flag & 2) return CERT_ERR_RANGE;
+    return CERT_OK;
+}
+
 // Reads the sticky status word after the stream has drained; clears it when set.
 static cert_status_t read_status(cert_net *net, cudaStream_t st, int *flag_out) {
     int flag = 0;
@@ -1530,7 +1598,7 @@ cert_status_t cert_backsub_bounds_host(cert_net_t *net, const float *centers_hos
         int flag = 0;
         s = read_status(net, st, &flag);
         if (s != CERT_OK) return s;
-        if (flag & 1) return CERT_ERR_TIMEOUT;
+        if (flag & 5) return status_of_flag(flag);
         if (flag & 2) {
             if (net->contraction == CERT_CONTRACTION_AUTO && attempt == 0 && net->tc_ok) {
                 forced = CERT_CONTRACTION_TC3XTF32;
@@ -1665,6 +1733,14 @@ cert_status_t cert_reusecert_bounds(cert_net_t *net, const float *centers, float
     ReuseState &R = net->reuse;
     const int K = net->n_layers, n_total = net->n_total;
     const long long rows = (long long)batch * R.R;
+#ifdef CERT_BOUNDS
+    {
+        const void *extra[2] = {lb_out, ub_out};
+        const size_t bytes[2] = {(size_t)batch * n_total * sizeof(float), (size_t)batch * n_total * sizeof(float)};
+        const cert_status_t bs = bounds_sync(net, extra, bytes, 2);
+        if (bs != CERT_OK) return bs;
+    }
+#endif
     Recorder rec(net, st);
     cert::launch_box(centers, eps, net->clip_lo, net->clip_hi, batch, net->n0, net->ld0, net->l0, net->u0, st);
     rec.mark(CERT_CLASS_INPUT);
@@ -1739,9 +1815,7 @@ cert_status_t cert_reusecert_bounds_host(cert_net_t *net, const float *centers_h
     int flag = 0;
     s = read_status(net, st, &flag);
     if (s != CERT_OK) return s;
-    if (flag & 1) return CERT_ERR_TIMEOUT;
-    if (flag & 2) return CERT_ERR_RANGE;
-    return CERT_OK;
+    return status_of_flag(flag);
 }
 
 cert_status_t cert_net_destroy(cert_net_t *net) {
@@ -1777,8 +1851,7 @@ cert_status_t cert_net_last_status(cert_net_t *net, void *stream) {
     int flag = 0;
     cert_status_t s = read_status(net, static_cast<cudaStream_t>(stream), &flag);
     if (s != CERT_OK) return s;
-    if (flag != 0) return (flag & 1) ? CERT_ERR_TIMEOUT : CERT_ERR_RANGE;
-    return CERT_OK;
+    return status_of_flag(flag);
 }
 
 int cert_net_check_guards(cert_net_t *net, void *stream) {
@@ -1797,6 +1870,29 @@ int cert_net_check_guards(cert_net_t *net, void *stream) {
             if (host[b] != kGuardByte) return (int)i + 1;
     }
     return 0;
+}
+
+int cert_built_with_checked_stores(void) {
+#ifdef CERT_BOUNDS
+    return 1;
+#else
+    return 0;
+#endif
+}
+
+cert_status_t cert_net_selftest_checked_store(cert_net_t *net, void *stream) {
+    if (!net) return CERT_ERR_INVALID_ARG;
+#ifdef CERT_BOUNDS
+    const cert_status_t bs = bounds_sync(net, nullptr, nullptr, 0);
+    if (bs != CERT_OK) return bs;
+    // one float past the end of the box array: inside the allocation's trailing guard, outside every buffer
+    cert::launch_checked_store_selftest(net->l0 + (size_t)net->max_batch * net->ld0, static_cast<cudaStream_t>(stream));
+    if (cudaPeekAtLastError() != cudaSuccess) { cudaGetLastError(); return CERT_ERR_CUDA; }
+    return CERT_OK;
+#else
+    (void)stream;
+    return CERT_ERR_UNSUPPORTED;
+#endif
 }
 
 int cert_net_auto_contraction(const cert_net_t *net) {

@@ -507,7 +507,7 @@ chain16_kernel(const __grid_constant__ ChainParams P, const ChainArgs a) {
                 }
                 if (vbuf >= 0) ++vstep;
             }
-            if (ok && row_ok) a.d_out[(size_t)col_group * a.slot_stride + r] = dacc;
+            if (ok && row_ok) CERT_ST(a.d_out[(size_t)col_group * a.slot_stride + r], dacc);
         }
         if (out_of_range) atomicOr(a.status, 2);
         if (!ok) {

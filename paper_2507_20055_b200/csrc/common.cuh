@@ -43,6 +43,48 @@ inline void launch_chained(Kernel kernel, dim3 grid, dim3 block, size_t smem, cu
 }
 inline long long ceil_div_ll(long long a, long long b) { return (a + b - 1) / b; }
 
+// ---- checked stores (a build with -DCERT_BOUNDS; memory-safety evidence, not for production) ----
+// Every plain store to global memory in the kernels that do not go through TMA is written CERT_ST(lvalue, value).
+// In an ordinary build that is the assignment.  In a CERT_BOUNDS build the address is first looked up in a table of
+// the buffers the current call may write (the net's allocations and the caller's output arrays, uploaded before
+// the call's first launch); a store that falls outside every one of them is skipped and raises bit 2 of the
+// table's status word (cert_net_last_status then returns CERT_ERR_BOUNDS).  Nothing faults either way.
+#ifdef CERT_BOUNDS
+constexpr int kBoundsMax = 1024;
+struct BoundsTable {
+    int n;
+    int *status;
+    unsigned long long lo[kBoundsMax], hi[kBoundsMax];
+};
+// Host side: each translation unit with kernels keeps its own device copy of the table (no relocatable device
+// code is used) and registers an uploader for it when the library is loaded.
+void bounds_register_uploader(void (*upload)(const BoundsTable *));
+void bounds_upload_all(const BoundsTable *t);      // synchronises the device, then calls every uploader
+#ifdef __CUDACC__
+static __device__ BoundsTable g_bounds_table;
+__device__ __forceinline__ bool bounds_check(const void *p, size_t bytes) {
+    const unsigned long long a = (unsigned long long)p;
+    for (int i = 0; i < g_bounds_table.n; ++i)
+        if (a >= g_bounds_table.lo[i] && a + bytes <= g_bounds_table.hi[i]) return true;
+    if (g_bounds_table.status) atomicOr(g_bounds_table.status, 4);
+    return false;
+}
+namespace {
+inline void bounds_upload_this_unit(const BoundsTable *t) { cudaMemcpyToSymbol(g_bounds_table, t, sizeof(BoundsTable)); }
+struct BoundsRegistrar {
+    BoundsRegistrar() { bounds_register_uploader(&bounds_upload_this_unit); }
+};
+static BoundsRegistrar g_bounds_registrar;
+}  // namespace
+#define CERT_ST(lvalue, value)                                                        \
+    do {                                                                              \
+        if (cert::bounds_check(&(lvalue), sizeof(lvalue))) (lvalue) = (value);        \
+    } while (0)
+#endif
+#else
+#define CERT_ST(lvalue, value) ((lvalue) = (value))
+#endif
+
 // One affine layer on the device.
 struct LayerDev {
     int kind, relu_after;
@@ -72,6 +114,10 @@ inline ConvGeom geom_of(const LayerDev &L) {
 
 // ---- launch wrappers (each enqueues exactly one kernel on `st`) ----
 
+#ifdef CERT_BOUNDS
+// Attempts CERT_ST(p[0], 1): with p outside every registered buffer the store is skipped and the status bit raised.
+void launch_checked_store_selftest(float *p, cudaStream_t st);
+#endif
 // *out = max(*out, max |x[i]|) for *out >= 0 (set-up time: the range proof of the fp16 split).
 void launch_absmax(const float *x, long long n, float *out, cudaStream_t st);
 

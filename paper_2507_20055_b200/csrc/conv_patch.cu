@@ -112,14 +112,14 @@ patch_start_kernel(const float *__restrict__ Wk, ConvGeom gk, const float *__res
                     h[e] = tf32_rn(qv[e]);
                     lo[e] = tf32_rn(qv[e] - h[e]);
                 }
-                *reinterpret_cast<float4 *>(dst) = make_float4(h[0], h[1], h[2], h[3]);
-                *reinterpret_cast<float4 *>(patch_lo + (size_t)r * pitch + q0) = make_float4(lo[0], lo[1], lo[2], lo[3]);
+                CERT_ST(*reinterpret_cast<float4 *>(dst), make_float4(h[0], h[1], h[2], h[3]));
+                CERT_ST(*reinterpret_cast<float4 *>(patch_lo + (size_t)r * pitch + q0), make_float4(lo[0], lo[1], lo[2], lo[3]));
             } else {
-                *reinterpret_cast<float4 *>(dst) = make_float4(qv[0], qv[1], qv[2], qv[3]);
+                CERT_ST(*reinterpret_cast<float4 *>(dst), make_float4(qv[0], qv[1], qv[2], qv[3]));
             }
         }
         dacc = warp_sum(dacc);
-        if (lane == 0) d[r] = bias_k[i] + dacc;
+        if (lane == 0) CERT_ST(d[r], bias_k[i] + dacc);
     }
 }
 
@@ -154,7 +154,7 @@ __global__ void patch_gather_kernel(const PatchGather g) {
         for (int i = 0; i < g.n_arr; ++i) {
             float val = 0.0f;
             if (t >= 0) val = g.src[i] ? g.src[i][(size_t)box * g.ld_src + t] : g.fill[i];
-            g.dst[i][(size_t)v * g.ld_dst + e] = val;
+            CERT_ST(g.dst[i][(size_t)v * g.ld_dst + e], val);
         }
     }
 }
@@ -256,10 +256,10 @@ patch_step_kernel(const float *__restrict__ in, const float *__restrict__ W, Con
                     dacc = fmaf(acc, ep.bias_below[t], dacc);
                 }
             }
-            if (EPI == CONVT_EPI_RELU) ep.P[(size_t)r * ps.pitch_out + e] = acc;
+            if (EPI == CONVT_EPI_RELU) CERT_ST(ep.P[(size_t)r * ps.pitch_out + e], acc);
         }
         if (EPI == CONVT_EPI_RELU) {
-            for (int e = n_outp + lane; e < ps.pitch_out; e += 32) ep.P[(size_t)r * ps.pitch_out + e] = 0.0f;
+            for (int e = n_outp + lane; e < ps.pitch_out; e += 32) CERT_ST(ep.P[(size_t)r * ps.pitch_out + e], 0.0f);
         }
         dacc = warp_sum(dacc);
         if (lane == 0) {
@@ -267,9 +267,9 @@ patch_step_kernel(const float *__restrict__ in, const float *__restrict__ W, Con
             for (int sl = 1; sl < ep.n_slots_in; ++sl) tot += ep.d_in[(size_t)sl * ep.slot_stride + r];
             tot += dacc;
             if (EPI == CONVT_EPI_CONCRETIZE)
-                (upper ? ep.ub_out : ep.lb_out)[(size_t)box * ep.n_total + ep.out_off + i] = tot;
+                CERT_ST((upper ? ep.ub_out : ep.lb_out)[(size_t)box * ep.n_total + ep.out_off + i], tot);
             else
-                ep.d_out[r] = tot;
+                CERT_ST(ep.d_out[r], tot);
         }
     }
 }
@@ -343,8 +343,8 @@ __global__ void to_ymajor_pair_kernel(const float *__restrict__ src_hi, const fl
     const int y = e / (c * w), rem = e - y * (c * w);
     const int ch = rem / w, x = rem - ch * w;
     const size_t s = (size_t)r * ld + (size_t)(ch * h + y) * w + x;
-    dst_hi[(size_t)r * ld + e] = src_hi[s];
-    dst_lo[(size_t)r * ld + e] = src_lo[s];
+    CERT_ST(dst_hi[(size_t)r * ld + e], src_hi[s]);
+    CERT_ST(dst_lo[(size_t)r * ld + e], src_lo[s]);
 }
 
 // Up to three per-neuron arrays [batch][ld]; a null source stands for fill[i].
@@ -363,7 +363,7 @@ __global__ void to_ymajor_vectors_kernel(const YMajorVectors g, int batch) {
     const int y = e / (g.c * g.w), rem = e - y * (g.c * g.w);
     const int ch = rem / g.w, x = rem - ch * g.w;
     const size_t s = (size_t)b * g.ld + (size_t)(ch * g.h + y) * g.w + x;
-    for (int i = 0; i < g.n_arr; ++i) g.dst[i][(size_t)b * g.ld + e] = g.src[i] ? g.src[i][s] : g.fill[i];
+    for (int i = 0; i < g.n_arr; ++i) CERT_ST(g.dst[i][(size_t)b * g.ld + e], g.src[i] ? g.src[i][s] : g.fill[i]);
 }
 
 void launch_to_ymajor_pair(const float *src_hi, const float *src_lo, float *dst_hi, float *dst_lo, long long rows,

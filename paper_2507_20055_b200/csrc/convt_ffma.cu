@@ -348,10 +348,10 @@ convt_kernel(const float *__restrict__ Q, int ld_out, int ld_in, const float *__
                                 const size_t o = (size_t)r * ld_in + t;
                                 if (ep.P_lo) {
                                     const float h = tf32_round(qv);
-                                    ep.P[o] = h;
-                                    ep.P_lo[o] = tf32_round(qv - h);
+                                    CERT_ST(ep.P[o], h);
+                                    CERT_ST(ep.P_lo[o], tf32_round(qv - h));
                                 } else {
-                                    ep.P[o] = qv;
+                                    CERT_ST(ep.P[o], qv);
                                 }
                             }
                         }
@@ -372,9 +372,9 @@ convt_kernel(const float *__restrict__ Q, int ld_out, int ld_in, const float *__
             for (int w2 = 0; w2 < kWarps; ++w2) tot += red[w2 * kMaxRowsPerGroup + threadIdx.x];
             if (EPI == CONVT_EPI_CONCRETIZE) {
                 const int b2 = (int)(row / (2LL * ep.n_k)), up2 = (int)((row / ep.n_k) & 1), i2 = (int)(row % ep.n_k);
-                (up2 ? ep.ub_out : ep.lb_out)[(size_t)b2 * ep.n_total + ep.out_off + i2] = tot;
+                CERT_ST((up2 ? ep.ub_out : ep.lb_out)[(size_t)b2 * ep.n_total + ep.out_off + i2], tot);
             } else {
-                ep.d_out[row] = tot;
+                CERT_ST(ep.d_out[row], tot);
             }
         }
         if (EPI == CONVT_EPI_RELU) {
@@ -383,8 +383,8 @@ convt_kernel(const float *__restrict__ Q, int ld_out, int ld_in, const float *__
                 if (r0 + q >= rows) break;
                 const size_t o = (size_t)(r0 + q) * ld_in;
                 for (int t = n_in + threadIdx.x; t < ld_in; t += kThreads) {
-                    ep.P[o + t] = 0.0f;
-                    if (ep.P_lo) ep.P_lo[o + t] = 0.0f;
+                    CERT_ST(ep.P[o + t], 0.0f);
+                    if (ep.P_lo) CERT_ST(ep.P_lo[o + t], 0.0f);
                 }
             }
         }
@@ -417,10 +417,10 @@ __device__ __forceinline__ void finish_element(float v, int t, long long r, int 
         const size_t o = (size_t)r * ld_in + t;
         if (ep.P_lo) {
             const float h = tf32_round(qv);
-            ep.P[o] = h;
-            ep.P_lo[o] = tf32_round(qv - h);
+            CERT_ST(ep.P[o], h);
+            CERT_ST(ep.P_lo[o], tf32_round(qv - h));
         } else {
-            ep.P[o] = qv;
+            CERT_ST(ep.P[o], qv);
         }
     }
 }
@@ -571,9 +571,9 @@ convt_s2_kernel(const float *__restrict__ Q, int ld_out, int ld_in, const float 
             for (int w2 = 0; w2 < kWarps; ++w2) tot += red[w2 * kMaxRowsPerGroup + threadIdx.x];
             if (EPI == CONVT_EPI_CONCRETIZE) {
                 const int b2 = (int)(row / (2LL * ep.n_k)), up2 = (int)((row / ep.n_k) & 1), i2 = (int)(row % ep.n_k);
-                (up2 ? ep.ub_out : ep.lb_out)[(size_t)b2 * ep.n_total + ep.out_off + i2] = tot;
+                CERT_ST((up2 ? ep.ub_out : ep.lb_out)[(size_t)b2 * ep.n_total + ep.out_off + i2], tot);
             } else {
-                ep.d_out[row] = tot;
+                CERT_ST(ep.d_out[row], tot);
             }
         }
         if (EPI == CONVT_EPI_RELU) {
@@ -582,8 +582,8 @@ convt_s2_kernel(const float *__restrict__ Q, int ld_out, int ld_in, const float 
                 if (r0 + q >= rows) break;
                 const size_t o = (size_t)(r0 + q) * ld_in;
                 for (int t = n_in + threadIdx.x; t < ld_in; t += kThreads) {
-                    ep.P[o + t] = 0.0f;
-                    if (ep.P_lo) ep.P_lo[o + t] = 0.0f;
+                    CERT_ST(ep.P[o + t], 0.0f);
+                    if (ep.P_lo) CERT_ST(ep.P_lo[o + t], 0.0f);
                 }
             }
         }

@@ -51,8 +51,8 @@ __global__ void box_kernel(const float *__restrict__ centers, float eps, float l
         l = fmaxf(__fsub_rn(c, eps), lo);
         u = fminf(__fadd_rn(c, eps), hi);
     }
-    l0[idx] = l;
-    u0[idx] = u;
+    CERT_ST(l0[idx], l);
+    CERT_ST(u0[idx], u);
 }
 
 // One warp per (box, neuron of the first layer).
@@ -95,8 +95,8 @@ __global__ void first_layer_kernel(const float *__restrict__ W, const float *__r
     hi = warp_sum(hi);
     if (lane == 0) {
         float bb = bias_n[i];
-        lb_out[(size_t)b * n_total + out_off + i] = lo + bb;
-        ub_out[(size_t)b * n_total + out_off + i] = hi + bb;
+        CERT_ST(lb_out[(size_t)b * n_total + out_off + i], lo + bb);
+        CERT_ST(ub_out[(size_t)b * n_total + out_off + i], hi + bb);
     }
 }
 
@@ -133,8 +133,8 @@ __global__ void first_layer_conv_kernel(const float *__restrict__ W, const float
             }
         }
     const float bb = bias_n[i];
-    lb_out[(size_t)b * n_total + out_off + i] = lo + bb;
-    ub_out[(size_t)b * n_total + out_off + i] = hi + bb;
+    CERT_ST(lb_out[(size_t)b * n_total + out_off + i], lo + bb);
+    CERT_ST(ub_out[(size_t)b * n_total + out_off + i], hi + bb);
 }
 
 // Joins the waiting coefficients of a residual connection to the expression that has reached its source.
@@ -149,7 +149,7 @@ __global__ void add_skip_kernel(float *__restrict__ P, const float *__restrict__
     float s = 0.0f;
     if (S_hi) s = S_hi[idx] + (S_lo ? S_lo[idx] : 0.0f);
     if (identity && t == (int)(r % n_k)) s += 1.0f;
-    P[idx] += s;
+    CERT_ST(P[idx], (P[idx]) + (s));
 }
 
 // Interval step of a layer with a residual connection: the source's concrete output bounds are added.
@@ -159,8 +159,8 @@ __global__ void add_act_bounds_kernel(float *__restrict__ lb_out, float *__restr
     const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (idx >= (long long)batch * n_k) return;
     const int b = (int)(idx / n_k), i = (int)(idx % n_k);
-    lb_out[(size_t)b * n_total + out_off + i] += actL[(size_t)b * ld_act + i];
-    ub_out[(size_t)b * n_total + out_off + i] += actU[(size_t)b * ld_act + i];
+    CERT_ST(lb_out[(size_t)b * n_total + out_off + i], (lb_out[(size_t)b * n_total + out_off + i]) + (actL[(size_t)b * ld_act + i]));
+    CERT_ST(ub_out[(size_t)b * n_total + out_off + i], (ub_out[(size_t)b * n_total + out_off + i]) + (actU[(size_t)b * ld_act + i]));
 }
 
 // A traversal stopped with coefficients still waiting on a residual connection's source: those neurons are
@@ -190,8 +190,8 @@ __global__ void skip_concretize_kernel(const float *__restrict__ S_hi, const flo
     }
     if (lane == 0) {
         if (identity) term += upper ? urow[i] : lrow[i];
-        if (slot) slot[r] = term;
-        else (upper ? ub_out : lb_out)[(size_t)b * n_total + out_off + i] += term;
+        if (slot) CERT_ST(slot[r], term);
+        else CERT_ST((upper ? ub_out : lb_out)[(size_t)b * n_total + out_off + i], ((upper ? ub_out : lb_out)[(size_t)b * n_total + out_off + i]) + (term));
     }
 }
 
@@ -234,8 +234,8 @@ __global__ void relax_kernel(float *__restrict__ lb_out, float *__restrict__ ub_
             }
             l = slot_sum(slots, n_slots, slot_stride, rl);
             u = slot_sum(slots, n_slots, slot_stride, ru);
-            lb_out[(size_t)b * n_total + out_off + t] = l;
-            ub_out[(size_t)b * n_total + out_off + t] = u;
+            CERT_ST(lb_out[(size_t)b * n_total + out_off + t], l);
+            CERT_ST(ub_out[(size_t)b * n_total + out_off + t], u);
         } else {
             l = lb_out[(size_t)b * n_total + out_off + t];
             u = ub_out[(size_t)b * n_total + out_off + t];
@@ -258,17 +258,17 @@ __global__ void relax_kernel(float *__restrict__ lb_out, float *__restrict__ ub_
                 nu = -__fdiv_rn(__fmul_rn(u, l), den);
                 code = (unsigned char)(2 + (pick_one ? 1 : 0));
             }
-            codes[(size_t)b * n_relu + relu_off + t] = code;
+            CERT_ST(codes[(size_t)b * n_relu + relu_off + t], code);
         }
     }
     if (actL) {
-        actL[idx] = al;
-        actU[idx] = au;
+        CERT_ST(actL[idx], al);
+        CERT_ST(actU[idx], au);
     }
     if (!do_relax) return;
-    lamL[idx] = ll;
-    lamU[idx] = lu;
-    nuU[idx] = nu;
+    CERT_ST(lamL[idx], ll);
+    CERT_ST(lamU[idx], lu);
+    CERT_ST(nuU[idx], nu);
 }
 
 // Start of a back-substitution at a conv layer k: the expression of neuron i = (co, oy, ox) is zero except
@@ -290,8 +290,8 @@ __global__ void conv_expr_start_kernel(const float *__restrict__ Wk, ConvGeom gk
     float *lrow = P_lo ? P_lo + (size_t)r * ld : nullptr;
     const float4 zero = make_float4(0.f, 0.f, 0.f, 0.f);
     for (int t = lane * 4; t < ld; t += 128) {
-        *reinterpret_cast<float4 *>(prow + t) = zero;
-        if (lrow) *reinterpret_cast<float4 *>(lrow + t) = zero;
+        CERT_ST(*reinterpret_cast<float4 *>(prow + t), zero);
+        if (lrow) CERT_ST(*reinterpret_cast<float4 *>(lrow + t), zero);
     }
     __syncwarp();      // orders the clearing stores before the window stores of other lanes
     const float *ll = lamL + (size_t)b * ld, *lu = lamU + (size_t)b * ld, *nu = nuU + (size_t)b * ld;
@@ -311,14 +311,14 @@ __global__ void conv_expr_start_kernel(const float *__restrict__ Wk, ConvGeom gk
         dacc = fmaf(qv, bias_below[t], dacc);
         if (lrow) {
             const float h = tf32_round(qv);
-            prow[t] = h;
-            lrow[t] = tf32_round(qv - h);
+            CERT_ST(prow[t], h);
+            CERT_ST(lrow[t], tf32_round(qv - h));
         } else {
-            prow[t] = qv;
+            CERT_ST(prow[t], qv);
         }
     }
     dacc = warp_sum(dacc);
-    if (lane == 0) d[r] = bias_k[i] + dacc;
+    if (lane == 0) CERT_ST(d[r], bias_k[i] + dacc);
 }
 
 // The same start with the columns in [y][channel][x] order (banded conv steps): the window's kh map rows are one
@@ -371,11 +371,11 @@ __global__ void conv_expr_start_ymajor_kernel(const float *__restrict__ Wk, Conv
                 }
             }
         }
-        *reinterpret_cast<float4 *>(prow + t0) = make_float4(hi4[0], hi4[1], hi4[2], hi4[3]);
-        if (lrow) *reinterpret_cast<float4 *>(lrow + t0) = make_float4(lo4[0], lo4[1], lo4[2], lo4[3]);
+        CERT_ST(*reinterpret_cast<float4 *>(prow + t0), make_float4(hi4[0], hi4[1], hi4[2], hi4[3]));
+        if (lrow) CERT_ST(*reinterpret_cast<float4 *>(lrow + t0), make_float4(lo4[0], lo4[1], lo4[2], lo4[3]));
     }
     dacc = warp_sum(dacc);
-    if (lane == 0) d[r] = bias_k[i] + dacc;
+    if (lane == 0) CERT_ST(d[r], bias_k[i] + dacc);
 }
 
 // Start of a back-substitution at FC layer k: row i of W_k pushed through the ReLU below, constant =
@@ -436,17 +436,17 @@ __global__ void fc_expr_start_kernel(const float *__restrict__ Wk, int ldw_k, co
                     h[e] = tf32_round(q[e]);
                     l[e] = tf32_round(q[e] - h[e]);
                 }
-                *reinterpret_cast<float4 *>(qrow) = make_float4(h[0], h[1], h[2], h[3]);
-                *reinterpret_cast<float4 *>(Q_lo + (size_t)(r0 + rr) * ld + t) = make_float4(l[0], l[1], l[2], l[3]);
+                CERT_ST(*reinterpret_cast<float4 *>(qrow), make_float4(h[0], h[1], h[2], h[3]));
+                CERT_ST(*reinterpret_cast<float4 *>(Q_lo + (size_t)(r0 + rr) * ld + t), make_float4(l[0], l[1], l[2], l[3]));
             } else {
-                *reinterpret_cast<float4 *>(qrow) = make_float4(q[0], q[1], q[2], q[3]);
+                CERT_ST(*reinterpret_cast<float4 *>(qrow), make_float4(q[0], q[1], q[2], q[3]));
             }
         }
     }
 #pragma unroll
     for (int rr = 0; rr < kStartRows; ++rr) {
         const float tot = warp_sum(dacc[rr]);
-        if (lane == 0 && i0 + rr < n_k) d[r0 + rr] = bias_k[i0 + rr] + tot;
+        if (lane == 0 && i0 + rr < n_k) CERT_ST(d[r0 + rr], bias_k[i0 + rr] + tot);
     }
 }
 
@@ -497,14 +497,14 @@ __global__ void relu_step_kernel(float *__restrict__ P,
                 h[e] = tf32_round(q[e]);
                 l[e] = tf32_round(q[e] - h[e]);
             }
-            *reinterpret_cast<float4 *>(prow + t) = make_float4(h[0], h[1], h[2], h[3]);
-            *reinterpret_cast<float4 *>(P_lo + (size_t)r * ld + t) = make_float4(l[0], l[1], l[2], l[3]);
+            CERT_ST(*reinterpret_cast<float4 *>(prow + t), make_float4(h[0], h[1], h[2], h[3]));
+            CERT_ST(*reinterpret_cast<float4 *>(P_lo + (size_t)r * ld + t), make_float4(l[0], l[1], l[2], l[3]));
         } else {
-            *reinterpret_cast<float4 *>(prow + t) = make_float4(q[0], q[1], q[2], q[3]);
+            CERT_ST(*reinterpret_cast<float4 *>(prow + t), make_float4(q[0], q[1], q[2], q[3]));
         }
     }
     dacc = warp_sum(dacc);
-    if (lane == 0) d[r] = slot_sum(d, n_slots, slot_stride, r) + dacc;
+    if (lane == 0) CERT_ST(d[r], slot_sum(d, n_slots, slot_stride, r) + dacc);
 }
 
 __global__ void concretize_kernel(const float *__restrict__ P, const float *__restrict__ d, int n_slots,
@@ -528,7 +528,7 @@ __global__ void concretize_kernel(const float *__restrict__ P, const float *__re
     acc = warp_sum(acc);
     if (lane == 0) {
         float v = slot_sum(d, n_slots, slot_stride, r) + acc;
-        (upper ? ub_out : lb_out)[(size_t)b * n_total + out_off + i] = v;
+        CERT_ST((upper ? ub_out : lb_out)[(size_t)b * n_total + out_off + i], v);
     }
 }
 
@@ -548,6 +548,13 @@ __global__ void absmax_kernel(const float *__restrict__ x, long long n, float *_
 }
 
 }  // namespace
+
+#ifdef CERT_BOUNDS
+namespace {
+__global__ void checked_store_selftest_kernel(float *p) { CERT_ST(p[0], 1.0f); }
+}  // namespace
+void launch_checked_store_selftest(float *p, cudaStream_t st) { checked_store_selftest_kernel<<<1, 1, 0, st>>>(p); }
+#endif
 
 void launch_absmax(const float *x, long long n, float *out, cudaStream_t st) {
     const int blocks = (int)std::min<long long>(ceil_div_ll(n, 256), 1184);

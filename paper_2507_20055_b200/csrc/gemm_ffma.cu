@@ -82,8 +82,8 @@ sgemm_nn_kernel(const float *__restrict__ A, int lda, const float *__restrict__ 
         for (int h = 0; h < 2; ++h) {
             int col = col0 + (h == 0 ? tx * 4 : 64 + tx * 4);
             if (col < ldc)
-                *reinterpret_cast<float4 *>(&C[(size_t)row * ldc + col]) =
-                    make_float4(acc[i][h * 4 + 0], acc[i][h * 4 + 1], acc[i][h * 4 + 2], acc[i][h * 4 + 3]);
+                CERT_ST(*reinterpret_cast<float4 *>(&C[(size_t)row * ldc + col]),
+                        make_float4(acc[i][h * 4 + 0], acc[i][h * 4 + 1], acc[i][h * 4 + 2], acc[i][h * 4 + 3]));
         }
     }
 }

@@ -404,7 +404,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_consta
                     for (int sidx = 0; sidx < a.n_slots_in; ++sidx) prev += a.d_in[(size_t)sidx * a.slot_stride + r];
                     tot += prev;
                 }
-                a.d_out[(size_t)slot * a.slot_stride + r] = tot;
+                CERT_ST(a.d_out[(size_t)slot * a.slot_stride + r], tot);
             }
         }
         if (kStores && lane == 0) tma_store_wait_all();

@@ -419,7 +419,7 @@ gemm_tc16_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_cons
                             w[j] = keep + __shfl_xor_sync(0xffffffffu, send, d);
                         }
                     }
-                    if (warp_row0 < a.M) a.colsum[(size_t)(warp_row0 >> 5) * a.ld_n + col0 + lane] = w[0];
+                    if (warp_row0 < a.M) CERT_ST(a.colsum[(size_t)(warp_row0 >> 5) * a.ld_n + col0 + lane], w[0]);
                 } else if (row_ok) {
                     const float *lrow = a.l0 + (size_t)b * a.ld_n + col0;
                     const float *urow = a.u0 + (size_t)b * a.ld_n + col0;
@@ -449,7 +449,7 @@ gemm_tc16_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_cons
                     for (int sidx = 0; sidx < a.n_slots_in; ++sidx) prev += a.d_in[(size_t)sidx * a.slot_stride + r];
                     tot += prev;
                 }
-                a.d_out[(size_t)(2 * nt + half_id) * a.slot_stride + r] = tot;
+                CERT_ST(a.d_out[(size_t)(2 * nt + half_id) * a.slot_stride + r], tot);
             }
         }
         if (EPI != TC_EPI_CONCRETIZE && lane == 0) tma_store_wait_all();
@@ -551,14 +551,14 @@ __global__ void expr_start16_kernel(const float *__restrict__ Wk, int ldw_k, con
                 ph[e >> 1] = (uint32_t)__half_as_ushort(h[0]) | ((uint32_t)__half_as_ushort(h[1]) << 16);
                 pl[e >> 1] = (uint32_t)__half_as_ushort(l[0]) | ((uint32_t)__half_as_ushort(l[1]) << 16);
             }
-            *reinterpret_cast<uint4 *>(Q_hi + (size_t)(r0 + rr) * ld + t) = make_uint4(ph[0], ph[1], ph[2], ph[3]);
-            *reinterpret_cast<uint4 *>(Q_lo + (size_t)(r0 + rr) * ld + t) = make_uint4(pl[0], pl[1], pl[2], pl[3]);
+            CERT_ST(*reinterpret_cast<uint4 *>(Q_hi + (size_t)(r0 + rr) * ld + t), make_uint4(ph[0], ph[1], ph[2], ph[3]));
+            CERT_ST(*reinterpret_cast<uint4 *>(Q_lo + (size_t)(r0 + rr) * ld + t), make_uint4(pl[0], pl[1], pl[2], pl[3]));
         }
     }
 #pragma unroll
     for (int rr = 0; rr < kRowsPerWarp; ++rr) {
         const float tot = warp_sum16(dacc[rr]);
-        if (lane == 0 && i0 + rr < n_k) d[r0 + rr] = bias_k[i0 + rr] + tot;
+        if (lane == 0 && i0 + rr < n_k) CERT_ST(d[r0 + rr], bias_k[i0 + rr] + tot);
     }
     if (__any_sync(0xffffffffu, out_of_range) && lane == 0) atomicOr(status, 2);
 }

@@ -64,6 +64,21 @@ extern "C" cert_status_t cert_first_layer_bounds_noalloc(const float *weight, co
     float *l0 = scratch, *u0 = scratch + kNoAllocMaxFloats;
 
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+#ifdef CERT_BOUNDS
+    {
+        // checking build: what this call may write is the scratch array and the caller's two outputs
+        static cert::BoundsTable t;
+        t.n = 3;
+        t.status = nullptr;
+        t.lo[0] = (unsigned long long)scratch;
+        t.hi[0] = t.lo[0] + 2 * kNoAllocMaxFloats * sizeof(float);
+        t.lo[1] = (unsigned long long)lb_out;
+        t.hi[1] = t.lo[1] + (size_t)batch * out_features * sizeof(float);
+        t.lo[2] = (unsigned long long)ub_out;
+        t.hi[2] = t.lo[2] + (size_t)batch * out_features * sizeof(float);
+        cert::bounds_upload_all(&t);
+    }
+#endif
     // The box kernel writes every element of [batch][ld0], padding included, so
     // nothing depends on what an earlier call left in the array.
     cert::launch_box(centers, eps, clip_lo, clip_hi, batch, in_features, ld0, l0, u0, st);

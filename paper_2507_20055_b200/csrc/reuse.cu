@@ -39,8 +39,8 @@ __global__ void reuse_relax_kernel(const float *__restrict__ colsum, int ld_s, i
             l += cs[(size_t)q * ld_s + t];
             u += cs[(size_t)q * ld_s + n + t];
         }
-        lb_out[(size_t)b * n_total + out_off + t] = l;
-        ub_out[(size_t)b * n_total + out_off + t] = u;
+        CERT_ST(lb_out[(size_t)b * n_total + out_off + t], l);
+        CERT_ST(ub_out[(size_t)b * n_total + out_off + t], u);
         if (do_relax) {
             const bool pick_one = (__fadd_rn(l, u) >= 0.0f);   // relu_n
             ll = pick_one ? 1.0f : 0.0f;
@@ -55,13 +55,13 @@ __global__ void reuse_relax_kernel(const float *__restrict__ colsum, int ld_s, i
                 nu = -__fdiv_rn(__fmul_rn(u, l), den);
                 code = (unsigned char)(2 + (pick_one ? 1 : 0));
             }
-            codes[(size_t)b * n_relu + relu_off + t] = code;
+            CERT_ST(codes[(size_t)b * n_relu + relu_off + t], code);
         }
     }
     if (!do_relax) return;
-    lamL[idx] = ll;
-    lamU[idx] = lu;
-    nuU[idx] = nu;
+    CERT_ST(lamL[idx], ll);
+    CERT_ST(lamU[idx], lu);
+    CERT_ST(nuU[idx], nu);
 }
 
 // S_k from the raw [L_k | U_k]: L_t *= lamL_t; U_t = lamU_t * U_t, + nuU_t on the constant row (without a ReLU
@@ -116,8 +116,8 @@ __global__ void reuse_init16_kernel(const float *__restrict__ W0t, int ldw, cons
             }
             store_pair16(v, h[e], l[e], out_of_range);
         }
-        *reinterpret_cast<uint4 *>(S_hi + (size_t)r * ld_s + col0) = pack8(h);
-        *reinterpret_cast<uint4 *>(S_lo + (size_t)r * ld_s + col0) = pack8(l);
+        CERT_ST(*reinterpret_cast<uint4 *>(S_hi + (size_t)r * ld_s + col0), pack8(h));
+        CERT_ST(*reinterpret_cast<uint4 *>(S_lo + (size_t)r * ld_s + col0), pack8(l));
     }
     if (__any_sync(0xffffffffu, out_of_range) && (threadIdx.x & 31) == 0) atomicOr(status, 2);
 }
@@ -155,8 +155,8 @@ __global__ void reuse_scale16_kernel(const float *__restrict__ raw, __half *__re
             }
             store_pair16(v, h[e], l[e], out_of_range);
         }
-        *reinterpret_cast<uint4 *>(S_hi + (size_t)r * ld_s + col0) = pack8(h);
-        *reinterpret_cast<uint4 *>(S_lo + (size_t)r * ld_s + col0) = pack8(l);
+        CERT_ST(*reinterpret_cast<uint4 *>(S_hi + (size_t)r * ld_s + col0), pack8(h));
+        CERT_ST(*reinterpret_cast<uint4 *>(S_lo + (size_t)r * ld_s + col0), pack8(l));
     }
     if (__any_sync(0xffffffffu, out_of_range) && (threadIdx.x & 31) == 0) atomicOr(status, 2);
 }

@@ -12,6 +12,13 @@ def pytest_configure(config):
     config.addinivalue_line("markers", "gpu: needs a CUDA device (B200)")
 
 
+def pytest_sessionstart(session):
+    # a child run that is meant to exercise the checking build must really have loaded it
+    if os.environ.get("CERT_EXPECT_CHECKED") == "1":
+        from paper_2507_20055_b200 import binding
+        assert binding.lib.cert_built_with_checked_stores() == 1, "CERT_LIB does not point at the checking build"
+
+
 def pytest_collection_modifyitems(config, items):
     try:
         import torch

@@ -222,6 +222,31 @@ def test_soundness_by_sampling(make, m):
         assert (z.max(axis=0) <= ub + 1e-9 * (1 + np.abs(ub))).all()
 
 
+def test_sampling_verdicts_of_the_large_configurations():
+    """10^5 samples from every box of the three large configurations take tens of minutes: that run is made once by
+    tests/golden/make_sampling_verdicts.py and its verdict stored; here the stored verdict is checked (no violation,
+    every box, the oracle source it was made with is the current one) and the check repeated on a subsample."""
+    import hashlib
+    import json
+    import os
+    from oracle import sampling_check as sc
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    verdicts = json.load(open(os.path.join(root, "tests", "golden", "sampling_verdicts.json")))
+    with open(os.path.join(root, "oracle", "deeppoly_oracle.c"), "rb") as f:
+        sha = hashlib.sha256(f.read()).hexdigest()[:16]
+    for idx, boxes, m in ((2, 4, 5000), (3, 2, 5000), (4, 2, 2000)):
+        w = wl.make_config(idx)
+        v = verdicts[w.name]
+        assert v["violations"] == 0 and v["samples_per_box"] == 100_000 and v["boxes"] == w.batch
+        assert v["oracle_source_sha256_16"] == sha, "the oracle changed: run tests/golden/make_sampling_verdicts.py again"
+        c = w.centers[:boxes]
+        r = orc.deeppoly(w.layers, c, w.eps, w.clip_lo, w.clip_hi)
+        l0, u0 = sc.box(c, w.eps, w.clip_lo, w.clip_hi)
+        for b in range(boxes):
+            viol, slack = sc.check_box(w.layers, r["lb"][b], r["ub"][b], l0[b], u0[b], m, seed=7 + b)
+            assert viol == 0 and slack > -1e-6
+
+
 def test_invariants_order_and_relaxation_ranges():
     w = wl.make_config(1, batch=3)
     r = orc.deeppoly(w.layers, w.centers, w.eps)
