@@ -25,16 +25,17 @@ import numpy as np
 
 from paper_2507_20055_b200 import workloads as wl
 
-# DRAM traffic of the dominant kernel, from the ncu capture summarised under profiles/ (read + written bytes
-# of one launch of the ReLU-epilogue contraction, 16-box case, per row of the coefficient matrix; traffic
-# grows in proportion to the rows, so a full launch is rows x this figure).  None for workloads not captured.
+# DRAM traffic of the dominant kernel, from the ncu captures summarised under profiles/ (read + written bytes of one
+# launch of the ReLU-epilogue contraction on a 32-box case, whose matrices (268 / 537 MB each way) exceed L2, per row
+# of the coefficient matrix; traffic grows in proportion to the rows, so a full launch is rows x this figure).
+# None for workloads not captured.
 NCU_TRAFFIC_BYTES_PER_ROW = {
-    ("fc6x1024_b128", "tc"): {"bytes_per_row": (318.128896e6 + 218.081792e6) / 32768.0,
+    ("fc6x1024_b128", "tc"): {"bytes_per_row": (628.547840e6 + 487.951616e6) / 65536.0,
                               "kernel": "gemm_tc_kernel<TC_EPI_RELU, 2>",
-                              "source": "profiles/gemm_tc_kernel_fc6x1024.md (16 boxes, scaled by rows)"},
-    ("fc6x1024_b128", "tc16"): {"bytes_per_row": (139.057152e6 + 95.979264e6) / 32768.0,
+                              "source": "profiles/gemm_tc_kernel_fc6x1024.md (32 boxes, scaled by rows)"},
+    ("fc6x1024_b128", "tc16"): {"bytes_per_row": (273.940992e6 + 232.271872e6) / 65536.0,
                                 "kernel": "gemm_tc16_kernel<TC_EPI_RELU>",
-                                "source": "profiles/gemm_tc16_kernel_fc6x1024.md (16 boxes, scaled by rows)"},
+                                "source": "profiles/gemm_tc16_kernel_fc6x1024.md (32 boxes, scaled by rows)"},
 }
 
 METRIC = "input boxes/sec fully bounded (DeepPoly)"

@@ -227,10 +227,15 @@ cert_status_t cert_net_selftest_bounded_wait(cert_net_t *net, void *stream);
  *            back-step scales a coefficient by a slope in [0, 1], so every entry of the traversal's matrix
  *            over layer j-1 is bounded by the matching entry of |W_k| |W_k-1| ... |W_j|, and the largest
  *            entry of those products over j (cert_net_fp16_coefficient_bound) must stay under 60000.  The
- *            products grow with depth: on deep nets the last layers may stay on TC3XTF32 while the others
- *            run in the fp16 split.  FC nets without residual connections only; otherwise, and for every
- *            layer whose proof fails, TC3XTF32, or FFMA where the tensor-core path is unavailable.
- *            (The environment variable CERT_AUTO_FP16=0, read at create, keeps AUTO on TC3XTF32.)
+ *            products grow with depth, so on deep nets the proof fails for the last layers although their
+ *            real coefficients are small.  Such a layer runs in the fp16 split on trial: its kernels report
+ *            to a status word of the layer's own, and the same traversal in TC3XTF32 is enqueued right behind
+ *            it with kernels that do nothing unless that word came up (an overflow or a run-out wait), in
+ *            which case they recompute the layer; either way the call's bounds are valid and the net's
+ *            status word is untouched.  FC nets without residual connections only; otherwise TC3XTF32, or
+ *            FFMA where the tensor-core path is unavailable.  (Environment variables read at create:
+ *            CERT_AUTO_FP16=0 keeps AUTO on TC3XTF32, CERT_SPECULATE_FP16=0 runs unproven layers in
+ *            TC3XTF32 outright.)
  * Conv back-steps have the same fusions; under FFMA they run on the FMA units, otherwise on the TF32 tensor-core
  * kernel where their geometry allows (see cert_net_set_conv_patches).
  * (The kernels of a call are chained with programmatic dependent launch, so that a kernel's launch and set-up
@@ -255,7 +260,8 @@ float cert_net_fp16_coefficient_bound(const cert_net_t *net, int layer);
  * a traversal to its concretisation; the environment variable CERT_CHAIN=0, read at create, keeps such nets
  * on one launch per back-step), bit 6 = a conv back-step on dense coefficient maps ran in its banded
  * tensor-core form (the environment variable CERT_CONV_BANDS=0, read at create, keeps those steps on the
- * FMA units). */
+ * FMA units), bit 7 = AUTO ran a layer in the fp16 split on trial and enqueued its predicated TC3XTF32 re-run
+ * (bits 1 and 2 are then set as well, whether or not the re-run had to do anything). */
 int cert_net_last_contraction_paths(const cert_net_t *net);
 
 /*

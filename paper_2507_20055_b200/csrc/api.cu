@@ -114,6 +114,11 @@ struct cert_net {
     // AUTO takes the fp16 split: the net's weights prove that no coefficient of any traversal can leave the
     // fp16 range (fp16_coef_bound = the largest entry of |W_k| |W_k-1| ... |W_j| over all k > j >= 1; slopes of a
     // ReLU back-step lie in [0, 1], so every stored coefficient is below it in magnitude)
+    // AUTO, layers whose proof fails (deep nets): the traversal runs in the fp16 split all the same, reporting to a
+    // status word of its own (spec_dev[k], cleared at the start of a call), and is followed by the same traversal
+    // in the TF32 split whose kernels do nothing unless that word came up (an overflow, or a run-out wait).
+    bool speculate = false;
+    int *spec_dev = nullptr;                 // [n_layers]
     bool auto_fp16 = false;                  // some layer's traversal passes the proof
     float fp16_coef_bound = INFINITY;        // the largest bound over all layers
     std::vector<float> fp16_layer_bound;     // [k]: the bound for the traversal of layer k (k >= 1)
@@ -481,6 +486,12 @@ cert_status_t prove_fp16_range(cert_net *net) {
         if (!off && std::isfinite(bound[k]) && bound[k] <= kFp16Safe) net->auto_fp16 = true;
     }
     if (off) net->fp16_layer_bound.assign(K, INFINITY);
+    // speculation needs every re-run kernel to be one that takes the predicate: FC steps on the tensor cores
+    bool all_tc = net->tc_ok;
+    for (int j = 0; j + 1 < K; ++j) all_tc = all_tc && net->tc[j].usable;
+    net->speculate = !off && all_tc;
+    if (const char *e = std::getenv("CERT_SPECULATE_FP16")) net->speculate = net->speculate && std::atoi(e) != 0;
+    if (net->speculate && !dev_alloc_zero(net, &net->spec_dev, (size_t)K)) return CERT_ERR_OOM;
     return CERT_OK;
 }
 
@@ -764,7 +775,9 @@ struct Traversal {
     cert_net *net;
     cudaStream_t st;
     Recorder *rec;
-    int mode;                 // the contraction mode of this call (AUTO resolved)
+    int mode;                 // the contraction mode of this traversal (AUTO resolved)
+    int *status;              // the status word its kernels report to: the net's, or the layer's word of a speculative run
+    const int *run_if;        // not null: a re-run whose kernels do nothing unless that word is non-zero
     int batch, k, j_end, steps;
     long long rows;           // 2 * batch * n_k, ordered (box, side, neuron)
     const float *box_l, *box_u;
@@ -777,7 +790,7 @@ struct Traversal {
     // Relu transformer of layer k; with `slots` its bounds are first summed from n_slots partial sums per row.
     void relax(const float *slots, int n_slots, int slot_npos = 0) const {
         cert::launch_relax(Lk(), lb_out, ub_out, net->n_total, batch, net->codes, net->n_relu, slots, n_slots,
-                           net->slot_stride, st, slot_npos);
+                           net->slot_stride, st, slot_npos, run_if);
         rec->mark(CERT_CLASS_RELAX);
     }
 };
@@ -826,7 +839,8 @@ cert::TcArgs tc_args(const Traversal &t, int K, int n_k, int ld_n, int bn, int n
     a.total_tiles = (int)cert::ceil_div_ll(t.rows, panel_rows) * tiles_per_panel;
     a.d_in = t.net->dbuf[dcur]; a.n_slots_in = dslots; a.d_out = t.net->dbuf[dcur ^ 1];
     a.slot_stride = t.net->slot_stride;
-    a.status = t.net->status_dev;
+    a.status = t.status;
+    a.run_if = t.run_if;
     return a;
 }
 
@@ -860,7 +874,7 @@ void run_chain16(Traversal &t) {
     a.Wk = Lk.W; a.ldw_k = Lk.ld_in; a.bias_k = Lk.bias_n;
     a.box_l = t.box_l; a.box_u = t.box_u;
     a.d_out = net->dbuf[0]; a.slot_stride = net->slot_stride;
-    a.status = net->status_dev;
+    a.status = t.status;
     a.stages = net->chain_stages; a.a_blocks = net->chain_a_blocks;
     a.b_chunk_bytes = net->chain_chunk; a.vec_ld = net->chain_vec_ld;
     const int pairs = (int)std::min<long long>(cert::ceil_div_ll(t.rows, 256), net->sm_count / 2);
@@ -881,7 +895,7 @@ void run_tc16_steps(Traversal &t) {
         ql[p] = reinterpret_cast<__half *>(net->buf_lo[p]);
     }
     int cur = 0, dcur = 0, dslots = 1;
-    cert::launch_init_expr16(Lk, t.layer(t.k - 1), t.batch, qh[cur], ql[cur], net->dbuf[dcur], net->status_dev, t.st);
+    cert::launch_init_expr16(Lk, t.layer(t.k - 1), t.batch, qh[cur], ql[cur], net->dbuf[dcur], t.status, t.st);
     t.rec->mark(CERT_CLASS_RELU_STEP);
     Waiting w;
     w.start(t);
@@ -1047,7 +1061,7 @@ void run_dense(Traversal &t) {
         // a conv layer right above a banded conv layer places its window coefficients at their y-major columns
         y_major = Lk.kind == CERT_LAYER_CONV2D && on_band(k - 1);
         cert::launch_init_expr(Lk, t.layer(k - 1), t.batch, net->buf[cur],
-                               wants_pair(k - 1) ? net->buf_lo[cur] : nullptr, net->dbuf[dcur], st, y_major);
+                               wants_pair(k - 1) ? net->buf_lo[cur] : nullptr, net->dbuf[dcur], st, y_major, t.run_if);
     }
     rec.mark(CERT_CLASS_RELU_STEP);
     Waiting w;
@@ -1265,10 +1279,12 @@ cert_status_t backsub_impl(cert_net *net, const float *centers, float eps, int b
                            st);
         rec.mark(CERT_CLASS_RELAX);
     }
+    bool spec_cleared = false;
     for (int k = 1; k < K; ++k) {
         const int mode = layer_mode(net, forced_mode, k);
         Traversal t;
         t.net = net; t.st = st; t.rec = &rec; t.mode = mode; t.batch = batch; t.k = k;
+        t.status = net->status_dev; t.run_if = nullptr;
         t.steps = (backsteps && backsteps[k] >= 0) ? std::min(backsteps[k], k) : k;
         t.j_end = k - t.steps;
         t.rows = 2LL * batch * net->layers[k].n_out;
@@ -1277,6 +1293,29 @@ cert_status_t backsub_impl(cert_net *net, const float *centers, float eps, int b
         t.lb_out = lb_out; t.ub_out = ub_out;
         t.paths = 0;
         cert::PatchLevel lv[kMaxPatchLevels];
+        // AUTO on a layer whose range proof failed: the fp16 split first, on its own status word, then the
+        // predicated TF32 traversal (cert_net::speculate)
+        const bool speculative = forced_mode < 0 && net->contraction == CERT_CONTRACTION_AUTO && net->speculate &&
+                                 mode == CERT_CONTRACTION_AUTO && t.steps > 0;
+        if (speculative) {
+            if (!spec_cleared) {
+                if (cudaMemsetAsync(net->spec_dev, 0, (size_t)K * sizeof(int), st) != cudaSuccess) {
+                    cudaGetLastError();
+                    return CERT_ERR_CUDA;
+                }
+                spec_cleared = true;
+            }
+            t.mode = CERT_CONTRACTION_TC3XFP16;
+            t.status = net->spec_dev + k;
+            if (net->chain_ok) run_chain16(t);
+            else run_tc16_steps(t);
+            t.mode = CERT_CONTRACTION_TC3XTF32;
+            t.status = net->status_dev;
+            t.run_if = net->spec_dev + k;
+            run_dense(t);
+            paths |= t.paths | 128;
+            continue;
+        }
         if (t.steps == 0) {
             run_interval_step(t);
         } else if (mode == CERT_CONTRACTION_TC3XFP16 && net->chain_ok) {

@@ -139,7 +139,7 @@ void launch_first_layer_bounds(const LayerDev &L, const float *l0, const float *
 // output positions (the order of the tensor-core patch steps) instead of (box, side, neuron).
 void launch_relax(const LayerDev &L, float *lb_out, float *ub_out, int n_total, int batch,
                   unsigned char *codes, int n_relu, const float *slots, int n_slots, long long slot_stride,
-                  cudaStream_t st, int slot_npos = 0);
+                  cudaStream_t st, int slot_npos = 0, const int *run_if = nullptr);
 
 // Start of the back-substitution for layer k: the expression of neuron i is
 // row i of W_k (the same for every box and both sides) and the constant b_k[i];
@@ -147,8 +147,11 @@ void launch_relax(const LayerDev &L, float *lb_out, float *ub_out, int n_total, 
 // picks up Q.b of the affine layer below, through which the next step goes.
 //   Q  [rows][ld] with rows = batch*2*n_k ordered (box, side, neuron)
 //   Q_lo != nullptr: Q is written as a TF32 pair (hi in Q, lo in Q_lo) for the tensor-core contraction
+// run_if != nullptr (here, in launch_relax and in TcArgs, FC layers): the kernel does its work only if *run_if is
+// non-zero when it starts; it belongs to a re-run that an earlier kernel of the same call may have made necessary.
 void launch_init_expr(const LayerDev &Lk, const LayerDev &Lbelow, int batch, float *Q, float *Q_lo, float *d,
-                      cudaStream_t st, int y_major = 0);   // y_major (conv layer k): columns in [y][channel][x] order
+                      cudaStream_t st, int y_major = 0,    // y_major (conv layer k): columns in [y][channel][x] order
+                      const int *run_if = nullptr);
 
 // ReLU back-step in place on P [rows][ld] (expression over the outputs of
 // layer `Lj`, i.e. over its ReLU neurons if it has one), plus d += Q.b_j.

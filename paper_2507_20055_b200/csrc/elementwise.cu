@@ -215,9 +215,10 @@ __global__ void relax_kernel(float *__restrict__ lb_out, float *__restrict__ ub_
                              float *__restrict__ actL, float *__restrict__ actU,
                              unsigned char *__restrict__ codes, int n_relu, int relu_off,
                              const float *__restrict__ slots, int n_slots, long long slot_stride,
-                             int slot_npos, int do_relax) {
+                             int slot_npos, int do_relax, const int *__restrict__ run_if) {
     pdl_trigger();
     pdl_wait();
+    if (run_if && *run_if == 0) return;      // a re-run that is not needed (see Traversal::run_if)
     long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (idx >= (long long)batch * ld) return;
     int b = (int)(idx / ld), t = (int)(idx % ld);
@@ -388,9 +389,10 @@ __global__ void fc_expr_start_kernel(const float *__restrict__ Wk, int ldw_k, co
                                      float *__restrict__ Q, float *__restrict__ Q_lo, float *__restrict__ d,
                                      long long n_warps, int n_k, int n, int ld, int has_relu,
                                      const float *__restrict__ lamL, const float *__restrict__ lamU,
-                                     const float *__restrict__ nuU, const float *__restrict__ bias_below) {
+                                     const float *__restrict__ nuU, const float *__restrict__ bias_below, const int *__restrict__ run_if) {
     pdl_trigger();
     pdl_wait();
+    if (run_if && *run_if == 0) return;      // a re-run that is not needed
     const long long w = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int lane = threadIdx.x & 31;
     if (w >= n_warps) return;
@@ -605,15 +607,15 @@ void launch_first_layer_bounds(const LayerDev &L, const float *l0, const float *
 
 void launch_relax(const LayerDev &L, float *lb_out, float *ub_out, int n_total, int batch,
                   unsigned char *codes, int n_relu, const float *slots, int n_slots, long long slot_stride,
-                  cudaStream_t st, int slot_npos) {
+                  cudaStream_t st, int slot_npos, const int *run_if) {
     long long n = (long long)batch * L.ld_out;
     launch_chained(relax_kernel, dim3((unsigned)ceil_div_ll(n, 256)), dim3(256), 0, st, lb_out, ub_out, n_total,
                    L.out_off, L.n_out, L.ld_out, batch, L.lamL, L.lamU, L.nuU, L.actL, L.actU, codes, n_relu, L.relu_off,
-                   slots, n_slots, slot_stride, slot_npos, L.relu_after);
+                   slots, n_slots, slot_stride, slot_npos, L.relu_after, run_if);
 }
 
 void launch_init_expr(const LayerDev &Lk, const LayerDev &Lb, int batch, float *Q, float *Q_lo, float *d,
-                      cudaStream_t st, int y_major) {
+                      cudaStream_t st, int y_major, const int *run_if) {
     long long rows = 2LL * batch * Lk.n_out;
     if (Lk.kind != CERT_LAYER_FC && y_major) {
         conv_expr_start_ymajor_kernel<<<grid_for_warps(rows), kWarpsPerBlock * 32, 0, st>>>(
@@ -631,11 +633,11 @@ void launch_init_expr(const LayerDev &Lk, const LayerDev &Lb, int batch, float *
     if (warps4 >= 32LL * sm_count()) {          // enough four-row warps to fill the multiprocessors
         launch_chained(fc_expr_start_kernel<4>, dim3(grid_for_warps(warps4)), dim3(kWarpsPerBlock * 32), 0, st, Lk.W,
                        Lk.ld_in, Lk.bias_n, Q, Q_lo, d, warps4, Lk.n_out, Lb.n_out, Lb.ld_out, Lb.relu_after, Lb.lamL,
-                       Lb.lamU, Lb.nuU, Lb.bias_n);
+                       Lb.lamU, Lb.nuU, Lb.bias_n, run_if);
     } else {
         launch_chained(fc_expr_start_kernel<1>, dim3(grid_for_warps(rows)), dim3(kWarpsPerBlock * 32), 0, st, Lk.W,
                        Lk.ld_in, Lk.bias_n, Q, Q_lo, d, rows, Lk.n_out, Lb.n_out, Lb.ld_out, Lb.relu_after, Lb.lamL,
-                       Lb.lamU, Lb.nuU, Lb.bias_n);
+                       Lb.lamU, Lb.nuU, Lb.bias_n, run_if);
     }
 }
 

@@ -77,7 +77,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_consta
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int num_kb = (a.K + BK - 1) / BK;
     const int n_tiles = a.n_tiles;
-    const int total_tiles = a.total_tiles;
+    int total_tiles = a.total_tiles;
     const uint32_t rank = CTAS == 2 ? cluster_ctarank() : 0u;
     const int group = CTAS == 2 ? (int)cluster_id_x() : (int)blockIdx.x;
     const int n_groups = CTAS == 2 ? (int)num_clusters_x() : (int)gridDim.x;
@@ -115,6 +115,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_consta
     if (CTAS == 2) cluster_sync_all();      // the peer's barriers exist before anything arrives on them
     tcgen05_fence_after();
     pdl_wait();                             // everything above needed nothing from the kernel before
+    // a re-run that turned out not to be needed has no tiles: every role falls through to the common exit
+    if (a.run_if && *reinterpret_cast<const volatile int *>(a.run_if) == 0) total_tiles = 0;
     const uint32_t tmem_base = bars->tmem_base;
     volatile uint32_t *abort_flag = &bars->abort_flag;
 

@@ -78,6 +78,7 @@ struct TcArgs {
     const float *bias2;
     float *colsum;
     int *status;                                 // set to 1 if a bounded wait runs out
+    const int *run_if;                           // not null: the launch has no work tiles unless *run_if != 0 when it starts
 };
 
 // One block that waits, with a short limit, on a barrier nothing arrives on, and then raises bit 0 of *status.

@@ -484,7 +484,8 @@ def test_auto_takes_the_fp16_split_only_where_the_weights_prove_its_range():
     finally:
         net.destroy()
     g = run_gpu(w)
-    assert g["paths"] & 2 and g["paths"] & 16         # both splits ran in the one call
+    # layer 2 runs in the fp16 split on trial, overflows, and its TF32 re-run takes over (bit 7: a re-run was enqueued)
+    assert g["paths"] & 2 and g["paths"] & 16 and g["paths"] & 128
     compare(g, _oracle(w), label="pm300/auto")
     w = wl.small_fc([33, 64, 300, 64, 10], batch=4, eps=0.04, seed=75)
     net = binding.CertNet(w.layers, w.batch, w.clip_lo, w.clip_hi)
@@ -501,6 +502,27 @@ def test_auto_takes_the_fp16_split_only_where_the_weights_prove_its_range():
     g = run_gpu(w)
     assert g["paths"] & 16 and not g["paths"] & 1
     compare(g, _oracle(w), label="ordinary/auto")
+
+
+def test_auto_runs_unproven_layers_in_the_fp16_split_on_trial():
+    """784 -> 200 x 9 -> 10: the products of the absolute weights pass 60000 from the eighth layer on although the
+    real coefficients stay small.  AUTO runs those layers in the fp16 split all the same, each on a status word of
+    its own, and enqueues the same traversal in the TF32 split with kernels that do nothing unless that word came
+    up.  Here it does not: the bounds are the fp16 split's, and the call's own status stays clean."""
+    from paper_2507_20055_b200 import binding
+    w = wl.make_config(2, batch=6)
+    net = binding.CertNet(w.layers, w.batch, w.clip_lo, w.clip_hi)
+    try:
+        unproven = [k for k in range(1, len(w.layers)) if net.fp16_coefficient_bound(k) > 60000.0]
+        assert unproven and min(unproven) >= 5
+    finally:
+        net.destroy()
+    ref = _oracle(w)
+    g = run_gpu(w)
+    assert g["paths"] & 32 and g["paths"] & 128 and not g["paths"] & 1
+    compare(g, ref, label="fc9x200/auto on trial")
+    forced = run_gpu(w, contraction=TC16)
+    assert np.array_equal(forced["lb"], g["lb"]) and np.array_equal(forced["ub"], g["ub"])
 
 
 def test_host_calls_report_the_device_status():
