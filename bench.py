@@ -370,18 +370,32 @@ def main():
     torch.cuda.synchronize()
     e2e_s = time.perf_counter() - t0
 
-    # ---- the denominators, measured: micro-kernels that run nothing but the unit in question ----
+    # ---- the denominators, measured: micro-kernels that run nothing but the unit in question.  They run in a
+    #      child process with a time limit: whatever happens there cannot stall or fail the benchmark line (the
+    #      roofline then falls back to the bf16-derived peak) ----
     micro = None
     if rank == 0 and world == 1 and not args.no_microbench:
-        micro = {}
-        for name, kind in (("tcgen05_f16", 0), ("tcgen05_tf32", 1), ("ffma", 2)):
-            try:
-                bt, bmhz, bms = binding.peak_microbench(kind, 5.0, stream.cuda_stream)
-                st_, smhz, sms_ = binding.peak_microbench(kind, 250.0, stream.cuda_stream)
-                micro[name] = {"burst": {"tflops": bt, "sm_mhz": bmhz, "ms": bms},
-                               "sustained": {"tflops": st_, "sm_mhz": smhz, "ms": sms_}}
-            except binding.CertError as e:
-                micro[name] = {"error": str(e)}
+        torch.cuda.synchronize()
+        code = ("import json\nfrom paper_2507_20055_b200 import binding\nout = {}\n"
+                "for name, kind in (('tcgen05_f16', 0), ('tcgen05_tf32', 1), ('ffma', 2)):\n"
+                "    try:\n"
+                "        b = binding.peak_microbench(kind, 5.0)\n"
+                "        s = binding.peak_microbench(kind, 250.0)\n"
+                "        out[name] = {'burst': {'tflops': b[0], 'sm_mhz': b[1], 'ms': b[2]},\n"
+                "                     'sustained': {'tflops': s[0], 'sm_mhz': s[1], 'ms': s[2]}}\n"
+                "    except binding.CertError as e:\n"
+                "        out[name] = {'error': str(e)}\n"
+                "print('MICRO ' + json.dumps(out))\n")
+        try:
+            env = dict(os.environ, CUDA_VISIBLE_DEVICES=os.environ.get("CUDA_VISIBLE_DEVICES", str(local_rank)))
+            r = subprocess.run([sys.executable, "-c", code], cwd=ROOT, env=env, capture_output=True, text=True,
+                               timeout=120)
+            lines = [x for x in r.stdout.splitlines() if x.startswith("MICRO ")]
+            micro = json.loads(lines[-1][6:]) if lines else {"error": (r.stderr or "no output")[-300:]}
+        except subprocess.TimeoutExpired:
+            micro = {"error": "the micro-kernels did not finish within 120 s"}
+        except Exception as e:          # noqa: BLE001  (the benchmark line must come out whatever happens here)
+            micro = {"error": repr(e)[:300]}
 
     # ---- max over ranks ----
     t = torch.tensor([total_ms, e2e_s * 1000.0], dtype=torch.float64, device="cuda")

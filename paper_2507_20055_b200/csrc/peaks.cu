@@ -178,7 +178,11 @@ extern "C" cert_status_t cert_peak_microbench(int kind, double target_ms, double
         cleanup();
         return CERT_ERR_OOM;
     }
-    const int smem = 2 * kTileBytes + 1024 + (int)sizeof(PeakBars);
+    // The kernel needs 34 KB, but it asks for 200 KB so that a multiprocessor holds exactly one of its CTAs, as
+    // with the product kernels: two CTAs on one SM would compete for its tensor memory (an allocation that
+    // cannot be served blocks without a limit), and a CTA pair must sit on two SMs.
+    const int smem = 200 * 1024;
+    static_assert(2 * kTileBytes + 1024 + (int)sizeof(PeakBars) <= 200 * 1024, "operand tiles fit");
     const int pairs = sms / 2;
     double flop_per_unit = 0.0;      // per MMA instruction of one pair, or per loop iteration of the whole grid
     if (kind == 0) flop_per_unit = 2.0 * (kPeakBM * 2) * kPeakBN * 16;
