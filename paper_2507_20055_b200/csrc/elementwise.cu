@@ -100,63 +100,6 @@ __global__ void first_layer_kernel(const float *__restrict__ W, const float *__r
     }
 }
 
-// The FC case tiled: a block owns kIvBoxes boxes x kIvNeurons neurons and walks the inputs in chunks of 32, with the
-// weight tile and the two box tiles in shared memory, so that a weight row is read once per kIvBoxes boxes instead
-// of once per box (the warp-per-output kernel above is bound by its L2 reads on wide layers).  A thread owns two
-// outputs from start to end: fixed summation order, nothing to reduce.
-constexpr int kIvBoxes = 16, kIvNeurons = 32, kIvChunk = 32;
-
-__global__ void __launch_bounds__(256)
-first_layer_tiled_kernel(const float *__restrict__ W, const float *__restrict__ bias_n, int n_in, int ld_in, int n_out,
-                         const float *__restrict__ l0, const float *__restrict__ u0, int ld0, int batch,
-                         float *__restrict__ lb_out, float *__restrict__ ub_out, int n_total, int out_off) {
-    __shared__ float Ws[kIvChunk][kIvNeurons + 1];
-    __shared__ __align__(16) float Ls[kIvBoxes][kIvChunk], Us[kIvBoxes][kIvChunk];
-    pdl_trigger();
-    pdl_wait();
-    const int t = threadIdx.x;
-    const int i0 = blockIdx.x * kIvNeurons, b0 = blockIdx.y * kIvBoxes;
-    const int neuron = t & 31, box_a = t >> 5, box_b = box_a + 8;
-    // loaders: the weight tile as float4 along the inputs (thread -> neuron t / 8, inputs 4 (t % 8) ..), the box
-    // tiles by the lower / upper half of the block
-    const int w_row = t >> 3, w_k = (t & 7) * 4;
-    const int v_box = (t & 127) >> 3, v_k = (t & 7) * 4;
-    const float *vsrc = (t < 128 ? l0 : u0);
-    float lo_a = 0.0f, hi_a = 0.0f, lo_b = 0.0f, hi_b = 0.0f;
-    for (int k0 = 0; k0 < n_in; k0 += kIvChunk) {
-        float4 w4 = make_float4(0.0f, 0.0f, 0.0f, 0.0f), v4 = w4;
-        if (i0 + w_row < n_out && k0 + w_k < ld_in)
-            w4 = *reinterpret_cast<const float4 *>(W + (size_t)(i0 + w_row) * ld_in + k0 + w_k);
-        if (b0 + v_box < batch && k0 + v_k < ld0)
-            v4 = *reinterpret_cast<const float4 *>(vsrc + (size_t)(b0 + v_box) * ld0 + k0 + v_k);
-        __syncthreads();                       // the tiles of the chunk before have been read
-        Ws[w_k + 0][w_row] = w4.x; Ws[w_k + 1][w_row] = w4.y; Ws[w_k + 2][w_row] = w4.z; Ws[w_k + 3][w_row] = w4.w;
-        *reinterpret_cast<float4 *>(t < 128 ? &Ls[v_box][v_k] : &Us[v_box][v_k]) = v4;
-        __syncthreads();
-        const int kmax = n_in - k0 < kIvChunk ? n_in - k0 : kIvChunk;
-        for (int k = 0; k < kmax; ++k) {
-            const float c = Ws[k][neuron];
-            const bool nn = (c >= 0.0f);
-            const float la = Ls[box_a][k], ua = Us[box_a][k], lb = Ls[box_b][k], ub = Us[box_b][k];
-            lo_a = fmaf(c, nn ? la : ua, lo_a);
-            hi_a = fmaf(c, nn ? ua : la, hi_a);
-            lo_b = fmaf(c, nn ? lb : ub, lo_b);
-            hi_b = fmaf(c, nn ? ub : lb, hi_b);
-        }
-    }
-    const int i = i0 + neuron;
-    if (i >= n_out) return;
-    const float bb = bias_n[i];
-    if (b0 + box_a < batch) {
-        CERT_ST(lb_out[(size_t)(b0 + box_a) * n_total + out_off + i], lo_a + bb);
-        CERT_ST(ub_out[(size_t)(b0 + box_a) * n_total + out_off + i], hi_a + bb);
-    }
-    if (b0 + box_b < batch) {
-        CERT_ST(lb_out[(size_t)(b0 + box_b) * n_total + out_off + i], lo_b + bb);
-        CERT_ST(ub_out[(size_t)(b0 + box_b) * n_total + out_off + i], hi_b + bb);
-    }
-}
-
 // The same for a conv layer with one thread per (box, neuron): a neuron has only c_in*kh*kw taps, and
 // the threads of a warp are neighbouring positions of one channel, so the weights are warp-uniform loads.
 __global__ void first_layer_conv_kernel(const float *__restrict__ W, const float *__restrict__ bias_n, ConvGeom g,
@@ -656,16 +599,6 @@ void launch_first_layer_bounds(const LayerDev &L, const float *l0, const float *
     if (L.kind == CERT_LAYER_CONV2D) {
         launch_chained(first_layer_conv_kernel, dim3((unsigned)ceil_div_ll(warps, 128)), dim3(128), 0, st, L.W, L.bias_n,
                        geom_of(L), L.n_out, l0, u0, ld0, batch, lb_out, ub_out, n_total, L.out_off);
-        return;
-    }
-    // rows that can be read as float4 (pitches of 4 floats, 16-byte aligned bases): the tiled kernel
-    const bool vec_ok = L.ld_in % 4 == 0 && ld0 % 4 == 0 && (reinterpret_cast<uintptr_t>(L.W) & 15) == 0 &&
-                        (reinterpret_cast<uintptr_t>(l0) & 15) == 0 && (reinterpret_cast<uintptr_t>(u0) & 15) == 0;
-    if (vec_ok && (long long)ceil_div_ll(batch, kIvBoxes) <= 65535) {
-        launch_chained(first_layer_tiled_kernel, dim3((unsigned)ceil_div_ll(L.n_out, kIvNeurons),
-                                                      (unsigned)ceil_div_ll(batch, kIvBoxes)),
-                       dim3(256), 0, st, L.W, L.bias_n, L.n_in, L.ld_in, L.n_out, l0, u0, ld0, batch, lb_out, ub_out,
-                       n_total, L.out_off);
         return;
     }
     launch_chained(first_layer_kernel, dim3(grid_for_warps(warps)), dim3(kWarpsPerBlock * 32), 0, st, L.W, L.bias_n,
