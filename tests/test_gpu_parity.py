@@ -680,7 +680,7 @@ def _well_conditioned(make, seed):
 @pytest.mark.parametrize("seed", range(10))
 def test_random_fc_shapes_all_contractions(seed):
     w, ref = _well_conditioned(_random_fc, seed)
-    for mode, contraction in (("ffma", 1), ("tc", 2), ("tc16", TC16)):
+    for mode, contraction in (("ffma", 1), ("tc", 2), ("tc16", TC16), ("auto", 0)):
         compare(run_gpu(w, contraction=contraction, max_batch=w.batch + (seed % 3)), ref, min_good_fraction=0.5,
                 label=f"random_fc[{seed}]/{mode}")
 
@@ -799,7 +799,7 @@ def test_random_nets_with_random_traversal_depths(block):
         good = ref["margins"].min(axis=1) >= 1e-5 if ref["margins"].shape[1] else np.ones(w.batch, bool)
         if good.mean() < 0.5:
             continue                      # ill-conditioned branch decisions: not a parity case
-        modes = {"fc": (1, 2, 3), "conv": (1, None), "res": (1, 2)}[kind]
+        modes = {"fc": (1, 2, 3, 0), "conv": (1, None), "res": (1, 2)}[kind]
         for c in modes:
             g = run_gpu(w, contraction=c, backsteps=steps, max_batch=w.batch + block % 2)
             compare(g, ref, label=f"{kind}/{w.name}/mode {c}/depths {steps}")
