@@ -181,7 +181,7 @@ def run_reference(args, w):
     per = {0: 1, 1: 4 * cores, 2: 2 * cores, 3: cores, 4: cores, 5: 2 * cores, 6: cores}
     n_boxes = min(w.batch, args.ref_boxes or per[args.config])
     if args.config == 4 and not args.ref_boxes:
-        n_boxes = max(1, min(cores, 16) // 2)     # about 11 s per box per core
+        n_boxes = max(1, min(cores, 16))          # one box per core, about 11 s per box: every core is busy
     times = []
     for i in range(args.warmup + args.steps):
         base, dt, _ = oracle_sample(w, n_boxes, backsteps=args.backsteps, certifier=args.certifier)

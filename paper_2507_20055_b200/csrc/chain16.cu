@@ -37,13 +37,16 @@ constexpr int kThreadsChain = 64 + kEpiWarps * 32;
 constexpr int kABlockBytes = BM * BKH * 2;       // one 64-column block of the panel (hi or lo): 16 KiB
 constexpr int kAccCols = 256;                    // tensor-memory columns per accumulator
 constexpr int CTAS = 2;
+constexpr int kBlockWriters = 2 * 4;             // warps of a CTA that write a 64-column block: two chunks x four lane quarters
 
 struct __align__(8) BarriersChain {
     uint64_t full[8];
     uint64_t empty[8];
     uint64_t acc_full[2];
     uint64_t acc_empty[2];
-    uint64_t a_ready;           // the panel in shared memory is complete (both CTAs' epilogue warps arrive)
+    uint64_t a_ready[4];        // 64-column block kb of the panel in shared memory is complete (the epilogue warps of
+                                // both CTAs that write its two 32-column chunks arrive): a step's first MMAs start
+                                // on the blocks that are rewritten first while the epilogue still works on the rest
     uint64_t vec_full[2];       // a step's relaxation / bias vectors have landed in staging buffer 0 / 1
     uint64_t vec_empty[2];      // ... and every epilogue warp is done reading them
     uint32_t tmem_base;
@@ -138,7 +141,7 @@ chain16_kernel(const __grid_constant__ ChainParams P, const ChainArgs a) {
             mbar_init(&bars->acc_full[i], 1);
             mbar_init(&bars->acc_empty[i], kEpiWarps * CTAS);
         }
-        mbar_init(&bars->a_ready, kEpiWarps * CTAS);
+        for (int i = 0; i < 4; ++i) mbar_init(&bars->a_ready[i], kBlockWriters * CTAS);
         for (int i = 0; i < 2; ++i) {
             mbar_init(&bars->vec_full[i], 1);
             mbar_init(&bars->vec_empty[i], kEpiWarps);
@@ -252,7 +255,7 @@ chain16_kernel(const __grid_constant__ ChainParams P, const ChainArgs a) {
         // ------------------------------------------------------------ MMA issuer (the leader CTA)
         if (lane == 0 && rank == 0) {
             int s = 0;
-            uint32_t phase = 0, a_phase = 0;
+            uint32_t phase = 0, a_phase = 0;      // a_phase: bit kb = phase of a_ready[kb]
             bool ok = true;
             int lt = 0;
             const uint32_t a_hi0 = smem_u32(A_hi), a_lo0 = smem_u32(A_lo);
@@ -261,10 +264,7 @@ chain16_kernel(const __grid_constant__ ChainParams P, const ChainArgs a) {
                     const ChainLayer &L = P.layer[j];
                     const int num_kb = (L.n_out + BKH - 1) / BKH;
                     const int ksteps = (L.n_out + 15) / 16;       // 16-column MMA steps that hold neurons; the rest of the last block is zero
-                    // the panel over layer j's neurons is in shared memory, in both CTAs
-                    if (!mbar_wait_cluster(&bars->a_ready, a_phase) || *abort_flag) { ok = false; break; }
-                    a_phase ^= 1;
-                    tcgen05_fence_after();
+                    // (the panel over layer j's neurons arrives in shared memory block by block, in both CTAs)
                     // kind::f16: D = f32, A = B = f16 (format 0), both K-major
                     const uint32_t idesc = (1u << 4) | ((uint32_t)(L.bn >> 3) << 17) | ((uint32_t)((BM * CTAS) >> 4) << 24);
                     for (int nt = 0; nt < L.n_tiles && ok; ++nt, ++lt) {
@@ -275,6 +275,11 @@ chain16_kernel(const __grid_constant__ ChainParams P, const ChainArgs a) {
                         const uint32_t d = tmem_base + (uint32_t)(acc * kAccCols);
                         // pass 1: cross terms
                         for (int kb = 0; kb < num_kb; ++kb) {
+                            if (nt == 0) {
+                                // block kb of the panel is complete
+                                if (!mbar_wait_cluster(&bars->a_ready[kb], (a_phase >> kb) & 1u) || *abort_flag) { ok = false; break; }
+                                a_phase ^= 1u << kb;
+                            }
                             if (!mbar_wait(&bars->full[s], phase) || *abort_flag) { ok = false; break; }
                             tcgen05_fence_after();
                             const uint32_t st = smem_u32(Bst + (size_t)s * kStageBytes);
@@ -329,7 +334,7 @@ chain16_kernel(const __grid_constant__ ChainParams P, const ChainArgs a) {
         const int prow = quarter * 32 + lane;               // this thread's row of the CTA's panel
         const uint32_t a_hi0 = smem_u32(A_hi), a_lo0 = smem_u32(A_lo);
         const uint32_t acc_empty_addr0 = map_to_cta(smem_u32(&bars->acc_empty[0]), 0);
-        const uint32_t a_ready_addr = map_to_cta(smem_u32(&bars->a_ready), 0);
+        const uint32_t a_ready_addr = map_to_cta(smem_u32(&bars->a_ready[0]), 0);
         bool ok = true, out_of_range = false;
         int lt = 0, vstep = 0;
         for (long long p = group; p < n_panels && ok; p += n_groups) {
@@ -385,10 +390,10 @@ chain16_kernel(const __grid_constant__ ChainParams P, const ChainArgs a) {
                         for (int e = 0; e < 32; ++e) q[e] = 0.0f;
                     }
                     write_panel_chunk(a_hi0, a_lo0, prow, c0, q, row_ok, out_of_range);
+                    fence_async_smem();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive_cluster(a_ready_addr + (uint32_t)((c0 >> 6) * sizeof(uint64_t)));
                 }
-                fence_async_smem();
-                __syncwarp();
-                if (lane == 0) mbar_arrive_cluster(a_ready_addr);
             }
             // boxes of this CTA's 128 rows (the producer stages the vectors of the first two)
             const long long cta_row0 = p * (BM * CTAS) + (long long)rank * BM;
@@ -467,13 +472,14 @@ chain16_kernel(const __grid_constant__ ChainParams P, const ChainArgs a) {
                                 for (int e = 0; e < 32; ++e) q[e] = 0.0f;
                             }
                             write_panel_chunk(a_hi0, a_lo0, prow, c0, q, row_ok, out_of_range);
+                            fence_async_smem();
+                            __syncwarp();
+                            if (lane == 0) mbar_arrive_cluster(a_ready_addr + (uint32_t)((c0 >> 6) * sizeof(uint64_t)));
                         }
                         tcgen05_fence_before();
-                        fence_async_smem();
                         __syncwarp();
                         if (lane == 0) {
                             mbar_arrive_cluster(acc_empty_addr0 + (uint32_t)(acc * sizeof(uint64_t)));
-                            mbar_arrive_cluster(a_ready_addr);
                             if (vbuf >= 0) mbar_arrive_cluster(map_to_cta(smem_u32(&bars->vec_empty[vbuf]), rank));
                         }
                     } else {
