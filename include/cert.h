@@ -232,8 +232,9 @@ cert_status_t cert_net_selftest_bounded_wait(cert_net_t *net, void *stream);
  *            to a status word of the layer's own, and the same traversal in TC3XTF32 is enqueued right behind
  *            it with kernels that do nothing unless that word came up (an overflow or a run-out wait), in
  *            which case they recompute the layer; either way the call's bounds are valid and the net's
- *            status word is untouched.  FC nets without residual connections only; otherwise TC3XTF32, or
- *            FFMA where the tensor-core path is unavailable.  (Environment variables read at create:
+ *            status word is untouched.  FC nets only (with residual connections no layer has a proof, and
+ *            every full traversal runs on trial); nets with conv layers run in TC3XTF32, or FFMA where the
+ *            tensor-core path is unavailable.  (Environment variables read at create:
  *            CERT_AUTO_FP16=0 keeps AUTO on TC3XTF32, CERT_SPECULATE_FP16=0 runs unproven layers in
  *            TC3XTF32 outright.)
  * Conv back-steps have the same fusions; under FFMA they run on the FMA units, otherwise on the TF32 tensor-core

@@ -417,7 +417,19 @@ cert_status_t prove_fp16_range(cert_net *net) {
     net->auto_fp16 = false;
     net->fp16_coef_bound = INFINITY;
     net->fp16_layer_bound.assign(K, INFINITY);
-    if (!net->tc16_ok || !net->skip_from.empty()) return CERT_OK;
+    if (!net->tc16_ok) return CERT_OK;
+    if (!net->skip_from.empty()) {
+        // residual connections add waiting coefficients to a traversal's matrix, which the products below do not
+        // cover: no layer is proven, every full traversal runs in the fp16 split on trial (see cert_net::speculate)
+        bool all_tc = net->tc_ok;
+        for (int j = 0; j + 1 < K; ++j) all_tc = all_tc && net->tc[j].usable;
+        bool on = all_tc;
+        if (const char *e = std::getenv("CERT_AUTO_FP16")) on = on && std::atoi(e) != 0;
+        if (const char *e = std::getenv("CERT_SPECULATE_FP16")) on = on && std::atoi(e) != 0;
+        net->speculate = on;
+        if (on && !dev_alloc_zero(net, &net->spec_dev, (size_t)K)) return CERT_ERR_OOM;
+        return CERT_OK;
+    }
 #ifdef CERT_BOUNDS
     {
         const cert_status_t bs = bounds_sync(net, nullptr, nullptr, 0);     // the products go through the checked FMA kernel
@@ -1295,8 +1307,9 @@ cert_status_t backsub_impl(cert_net *net, const float *centers, float eps, int b
         cert::PatchLevel lv[kMaxPatchLevels];
         // AUTO on a layer whose range proof failed: the fp16 split first, on its own status word, then the
         // predicated TF32 traversal (cert_net::speculate)
+        // (nets with residual connections: the fp16 schedule covers full traversals only)
         const bool speculative = forced_mode < 0 && net->contraction == CERT_CONTRACTION_AUTO && net->speculate &&
-                                 mode == CERT_CONTRACTION_AUTO && t.steps > 0;
+                                 mode == CERT_CONTRACTION_AUTO && t.steps > 0 && (!residual || t.steps == k);
         if (speculative) {
             if (!spec_cleared) {
                 if (cudaMemsetAsync(net->spec_dev, 0, (size_t)K * sizeof(int), st) != cudaSuccess) {

@@ -567,16 +567,20 @@ RES_NETS = {
 }
 
 
-@pytest.mark.parametrize("mode", ["ffma", "tc", "tc16"])
+@pytest.mark.parametrize("mode", ["ffma", "tc", "tc16", "auto"])
 @pytest.mark.parametrize("name", sorted(RES_NETS))
 def test_residual_nets(name, mode):
     w = RES_NETS[name]()
-    if mode == "tc16" and any(l.kind != "fc" for l in w.layers):
+    all_fc = all(l.kind == "fc" for l in w.layers)
+    if mode == "tc16" and not all_fc:
         pytest.skip("the fp16 split covers FC nets")
     ref = orc.deeppoly(w.layers, w.centers, w.eps, w.clip_lo, w.clip_hi, skip_from=w.skip_from)
-    g = run_gpu(w, contraction={"ffma": 1, "tc": 2, "tc16": 3}[mode], max_batch=w.batch + 1)
+    g = run_gpu(w, contraction={"ffma": 1, "tc": 2, "tc16": 3, "auto": 0}[mode], max_batch=w.batch + 1)
     if mode == "tc16":
         assert g["paths"] & 16 and not g["paths"] & 32      # one launch per back-step, not the chain kernel
+    if mode == "auto":
+        # FC nets with connections: every layer in the fp16 split on trial; conv nets: the TF32 split
+        assert bool(g["paths"] & 128) == all_fc and bool(g["paths"] & 16) == all_fc
     if mode == "tc":
         assert bool(g["paths"] & 64) == (name == "resconv_band")
     compare(g, ref, label=f"{name}/{mode}")
@@ -799,7 +803,7 @@ def test_random_nets_with_random_traversal_depths(block):
         good = ref["margins"].min(axis=1) >= 1e-5 if ref["margins"].shape[1] else np.ones(w.batch, bool)
         if good.mean() < 0.5:
             continue                      # ill-conditioned branch decisions: not a parity case
-        modes = {"fc": (1, 2, 3, 0), "conv": (1, None), "res": (1, 2)}[kind]
+        modes = {"fc": (1, 2, 3, 0), "conv": (1, None), "res": (1, 2, 0)}[kind]
         for c in modes:
             g = run_gpu(w, contraction=c, backsteps=steps, max_batch=w.batch + block % 2)
             compare(g, ref, label=f"{kind}/{w.name}/mode {c}/depths {steps}")
