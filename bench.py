@@ -63,7 +63,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
-                                          "-i", str(self.gpu), "-lms", "100"], stdout=subprocess.PIPE,
+                                          "-i", str(self.gpu), "-lms", "50"], stdout=subprocess.PIPE,
                                          stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
@@ -72,9 +72,10 @@ class ClockSampler:
 
     def _read(self):
         for line in self.proc.stdout:
-            self.rows.append([x.strip() for x in line.split(",")])
+            self.rows.append([x.strip() for x in line.split(",")] + [time.perf_counter()])
 
-    def stop(self):
+    def stop(self, window=None):
+        """window = (t0, t1) in time.perf_counter() terms: only samples read in it count (the timed region)."""
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
         self.proc.terminate()
@@ -84,7 +85,12 @@ class ClockSampler:
             self.proc.kill()
         sm, mx, reasons = [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for r in self.rows:
+        rows = self.rows
+        if window is not None:
+            # a sample is printed up to one period after it was taken
+            inside = [r for r in rows if window[0] + 0.05 <= r[-1] <= window[1] + 0.05]
+            rows = inside or rows
+        for r in rows:
             try:
                 sm.append(float(r[1])); mx.append(float(r[2]))
                 for n, v in zip(names, r[5:9]):
@@ -92,9 +98,7 @@ class ClockSampler:
                         reasons.add(n)
             except Exception:
                 pass
-        # under load = the upper half of the samples
-        load = sorted(sm)[len(sm) // 2:] if sm else []
-        return {"sm_mhz": statistics.median(load) if load else None,
+        return {"sm_mhz": statistics.median(sm) if sm else None,
                 "sm_max_mhz": max(mx) if mx else None, "samples": len(sm), "reasons": sorted(reasons)}
 
 
@@ -307,7 +311,8 @@ def main():
             step_device()
             evs[i][1].record(stream)
     barrier()
-    t_wall = time.perf_counter() - t_wall0
+    t_wall1 = time.perf_counter()
+    t_wall = t_wall1 - t_wall0
     step_ms = [a.elapsed_time(b) for a, b in evs]
     total_ms = sum(step_ms)
     launches = net.last_launch_count() * args.steps
@@ -325,7 +330,7 @@ def main():
                 cls_ms[name] = cls_ms.get(name, 0.0) + ms
                 cls_n[name] = cls_n.get(name, 0) + n
     net.set_profiling(False)
-    clocks = sampler.stop() if rank == 0 else None
+    clocks = sampler.stop((t_wall0, t_wall1)) if rank == 0 else None
 
     # ---- the same steps with the 3xTF32 contraction, for reference, when the fp16 split was timed above ----
     tf32_ref = None

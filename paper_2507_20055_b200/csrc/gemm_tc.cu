@@ -488,22 +488,16 @@ bool tc_driver_init() {
 }
 
 bool tc_prepare_kernels(bool *pair_ok) {
-    cudaError_t e[14];
-    e[12] = cudaFuncSetAttribute(gemm_tc_kernel<TC_EPI_RELU_BAND_SKIP, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemMax);
-    e[13] = cudaFuncSetAttribute(gemm_tc_kernel<TC_EPI_RELU_BAND_SKIP, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemMax);
-    e[8] = cudaFuncSetAttribute(gemm_tc_kernel<TC_EPI_RELU_BAND, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemMax);
-    e[9] = cudaFuncSetAttribute(gemm_tc_kernel<TC_EPI_RELU_BAND, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemMax);
-    e[10] = cudaFuncSetAttribute(gemm_tc_kernel<TC_EPI_CONCRETIZE_BAND, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemMax);
-    e[11] = cudaFuncSetAttribute(gemm_tc_kernel<TC_EPI_CONCRETIZE_BAND, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemMax);
-    e[6] = cudaFuncSetAttribute(gemm_tc_kernel<TC_EPI_RELU_SKIP, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemMax);
-    e[7] = cudaFuncSetAttribute(gemm_tc_kernel<TC_EPI_RELU_SKIP, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemMax);
-    e[0] = cudaFuncSetAttribute(gemm_tc_kernel<TC_EPI_RELU, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemMax);
-    e[1] = cudaFuncSetAttribute(gemm_tc_kernel<TC_EPI_CONCRETIZE, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemMax);
-    e[2] = cudaFuncSetAttribute(gemm_tc_kernel<TC_EPI_RELU, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemMax);
-    e[3] = cudaFuncSetAttribute(gemm_tc_kernel<TC_EPI_CONCRETIZE, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemMax);
-    e[4] = e[5] = cudaSuccess;      // (slots of a variant that no longer exists)
-    for (int i = 0; i < 14; ++i)
-        if (e[i] != cudaSuccess) {
+    const void *kernels[] = {
+        (const void *)gemm_tc_kernel<TC_EPI_RELU, 1>,                (const void *)gemm_tc_kernel<TC_EPI_RELU, 2>,
+        (const void *)gemm_tc_kernel<TC_EPI_CONCRETIZE, 1>,          (const void *)gemm_tc_kernel<TC_EPI_CONCRETIZE, 2>,
+        (const void *)gemm_tc_kernel<TC_EPI_RELU_SKIP, 1>,           (const void *)gemm_tc_kernel<TC_EPI_RELU_SKIP, 2>,
+        (const void *)gemm_tc_kernel<TC_EPI_RELU_BAND, 1>,           (const void *)gemm_tc_kernel<TC_EPI_RELU_BAND, 2>,
+        (const void *)gemm_tc_kernel<TC_EPI_CONCRETIZE_BAND, 1>,     (const void *)gemm_tc_kernel<TC_EPI_CONCRETIZE_BAND, 2>,
+        (const void *)gemm_tc_kernel<TC_EPI_RELU_BAND_SKIP, 1>,      (const void *)gemm_tc_kernel<TC_EPI_RELU_BAND_SKIP, 2>,
+    };
+    for (const void *k : kernels)
+        if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemMax) != cudaSuccess) {
             cudaGetLastError();
             return false;
         }
