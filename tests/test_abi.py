@@ -101,3 +101,29 @@ def test_null_handles_of_the_other_entry_points(lib):
     assert L.cert_net_enable_reusecert(None) == 1
     assert L.cert_net_set_conv_patches(None, 1) == 1
     assert b"fp16" in L.cert_status_string(7)
+
+
+def test_null_handles_and_bad_arguments_of_the_helpers(lib):
+    L = lib.lib
+    assert L.cert_net_check_guards(None, None) == -1
+    assert L.cert_net_auto_contraction(None) == -1
+    assert L.cert_net_fp16_coefficient_bound(None, 0) == -1.0
+    assert L.cert_net_selftest_checked_store(None, None) == 1
+    assert L.cert_built_with_checked_stores() == (1 if os.environ.get("CERT_LIB", "").endswith("_checked.so") else 0)
+    # the peak micro-kernels validate their arguments before they touch the device
+    out = ctypes.c_double()
+    assert L.cert_peak_microbench(3, 5.0, ctypes.byref(out), None, None, None) == 1
+    assert L.cert_peak_microbench(0, 0.0, ctypes.byref(out), None, None, None) == 1
+    assert L.cert_peak_microbench(0, 5000.0, ctypes.byref(out), None, None, None) == 1
+    assert L.cert_peak_microbench(0, 5.0, None, None, None, None) == 1
+    assert b"checked store" in L.cert_status_string(8)
+
+
+def test_the_checking_build_exports_the_same_symbols():
+    """The same sources with -DCERT_BOUNDS (paper_2507_20055_b200/build.py --checked) load and export every symbol."""
+    from paper_2507_20055_b200 import build
+    checked = ctypes.CDLL(build.build_checked())
+    for n in _declared_functions():
+        assert hasattr(checked, n), f"{n} missing from the checking build"
+    checked.cert_built_with_checked_stores.restype = ctypes.c_int
+    assert checked.cert_built_with_checked_stores() == 1
