@@ -55,48 +55,95 @@ __global__ void box_kernel(const float *__restrict__ centers, float eps, float l
     CERT_ST(u0[idx], u);
 }
 
-// One warp per (box, neuron of the first layer).
-__global__ void first_layer_kernel(const float *__restrict__ W, const float *__restrict__ bias_n, int kind,
-                                   ConvGeom g, int n_in, int ld_in, int n_out, const float *__restrict__ l0,
-                                   const float *__restrict__ u0, int ld0, int batch, float *__restrict__ lb_out,
-                                   float *__restrict__ ub_out, int n_total, int out_off) {
+// FC layer: one warp per (box, NEURONS consecutive neurons).  The box row is read once for the warp's neurons
+// (the weight rows come from L2 either way); every output is summed lane-strided and reduced by a shuffle tree.
+template <int NEURONS>
+__global__ void first_layer_kernel(const float *__restrict__ W, const float *__restrict__ bias_n, int n_in, int ld_in,
+                                   int n_out, const float *__restrict__ l0, const float *__restrict__ u0, int ld0,
+                                   int batch, float *__restrict__ lb_out, float *__restrict__ ub_out, int n_total,
+                                   int out_off) {
     pdl_trigger();
     pdl_wait();
-    long long warp = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-    int lane = threadIdx.x & 31;
-    if (warp >= (long long)batch * n_out) return;
-    int b = (int)(warp / n_out), i = (int)(warp % n_out);
+    const long long warp = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int lane = threadIdx.x & 31;
+    const int groups = (n_out + NEURONS - 1) / NEURONS;
+    if (warp >= (long long)batch * groups) return;
+    const int b = (int)(warp / groups), i0 = (int)(warp % groups) * NEURONS;
+    const int n_here = n_out - i0 < NEURONS ? n_out - i0 : NEURONS;
     const float *lrow = l0 + (size_t)b * ld0, *urow = u0 + (size_t)b * ld0;
-    float lo = 0.0f, hi = 0.0f;
-    if (kind == CERT_LAYER_FC) {
-        const float *w = W + (size_t)i * ld_in;
-        for (int s = lane; s < n_in; s += 32) {
-            float c = w[s], l = lrow[s], u = urow[s];
-            bool nn = (c >= 0.0f);
-            lo = fmaf(c, nn ? l : u, lo);
-            hi = fmaf(c, nn ? u : l, hi);
-        }
-    } else {
-        int hw = g.h_out * g.w_out;
-        int co = i / hw, oy = (i / g.w_out) % g.h_out, ox = i % g.w_out;
-        int taps = g.c_in * g.kh * g.kw;
-        for (int q = lane; q < taps; q += 32) {
-            int ci = q / (g.kh * g.kw), ky = (q / g.kw) % g.kh, kx = q % g.kw;
-            int iy = oy * g.stride - g.pad + ky, ix = ox * g.stride - g.pad + kx;
-            if (iy < 0 || iy >= g.h_in || ix < 0 || ix >= g.w_in) continue;
-            int s = (ci * g.h_in + iy) * g.w_in + ix;
-            float c = W[(size_t)co * taps + q], l = lrow[s], u = urow[s];
-            bool nn = (c >= 0.0f);
-            lo = fmaf(c, nn ? l : u, lo);
-            hi = fmaf(c, nn ? u : l, hi);
+    const float *w = W + (size_t)i0 * ld_in;
+    float lo[NEURONS], hi[NEURONS];
+#pragma unroll
+    for (int e = 0; e < NEURONS; ++e) lo[e] = hi[e] = 0.0f;
+    for (int s = lane; s < n_in; s += 32) {
+        const float l = lrow[s], u = urow[s];
+#pragma unroll
+        for (int e = 0; e < NEURONS; ++e) {
+            if (e < n_here) {
+                const float c = w[(size_t)e * ld_in + s];
+                const bool nn = (c >= 0.0f);
+                lo[e] = fmaf(c, nn ? l : u, lo[e]);
+                hi[e] = fmaf(c, nn ? u : l, hi[e]);
+            }
         }
     }
-    lo = warp_sum(lo);
-    hi = warp_sum(hi);
-    if (lane == 0) {
-        float bb = bias_n[i];
-        CERT_ST(lb_out[(size_t)b * n_total + out_off + i], lo + bb);
-        CERT_ST(ub_out[(size_t)b * n_total + out_off + i], hi + bb);
+#pragma unroll
+    for (int e = 0; e < NEURONS; ++e) {
+        const float lo_s = warp_sum(lo[e]), hi_s = warp_sum(hi[e]);
+        if (lane == 0 && e < n_here) {
+            const float bb = bias_n[i0 + e];
+            CERT_ST(lb_out[(size_t)b * n_total + out_off + i0 + e], lo_s + bb);
+            CERT_ST(ub_out[(size_t)b * n_total + out_off + i0 + e], hi_s + bb);
+        }
+    }
+}
+
+// The same with 16-byte loads, for rows whose pitches are multiples of four floats and whose padding up to the
+// next multiple of four is zero (the net's own arrays; a caller's unpadded weights when in_features % 4 == 0).
+template <int NEURONS>
+__global__ void first_layer_vec_kernel(const float *__restrict__ W, const float *__restrict__ bias_n, int n_in, int ld_in,
+                                       int n_out, const float *__restrict__ l0, const float *__restrict__ u0, int ld0,
+                                       int batch, float *__restrict__ lb_out, float *__restrict__ ub_out, int n_total,
+                                       int out_off) {
+    pdl_trigger();
+    pdl_wait();
+    const long long warp = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int lane = threadIdx.x & 31;
+    const int groups = (n_out + NEURONS - 1) / NEURONS;
+    if (warp >= (long long)batch * groups) return;
+    const int b = (int)(warp / groups), i0 = (int)(warp % groups) * NEURONS;
+    const int n_here = n_out - i0 < NEURONS ? n_out - i0 : NEURONS;
+    const float4 *lrow = reinterpret_cast<const float4 *>(l0 + (size_t)b * ld0);
+    const float4 *urow = reinterpret_cast<const float4 *>(u0 + (size_t)b * ld0);
+    float lo[NEURONS], hi[NEURONS];
+#pragma unroll
+    for (int e = 0; e < NEURONS; ++e) lo[e] = hi[e] = 0.0f;
+    const int quads = (n_in + 3) >> 2;
+    for (int q = lane; q < quads; q += 32) {
+        const float4 l4 = lrow[q], u4 = urow[q];
+        const float l[4] = {l4.x, l4.y, l4.z, l4.w}, u[4] = {u4.x, u4.y, u4.z, u4.w};
+#pragma unroll
+        for (int e = 0; e < NEURONS; ++e) {
+            if (e < n_here) {
+                const float4 w4 = *reinterpret_cast<const float4 *>(W + (size_t)(i0 + e) * ld_in + 4 * q);
+                const float c[4] = {w4.x, w4.y, w4.z, w4.w};
+#pragma unroll
+                for (int z = 0; z < 4; ++z) {
+                    const bool nn = (c[z] >= 0.0f);
+                    lo[e] = fmaf(c[z], nn ? l[z] : u[z], lo[e]);
+                    hi[e] = fmaf(c[z], nn ? u[z] : l[z], hi[e]);
+                }
+            }
+        }
+    }
+#pragma unroll
+    for (int e = 0; e < NEURONS; ++e) {
+        const float lo_s = warp_sum(lo[e]), hi_s = warp_sum(hi[e]);
+        if (lane == 0 && e < n_here) {
+            const float bb = bias_n[i0 + e];
+            CERT_ST(lb_out[(size_t)b * n_total + out_off + i0 + e], lo_s + bb);
+            CERT_ST(ub_out[(size_t)b * n_total + out_off + i0 + e], hi_s + bb);
+        }
     }
 }
 
@@ -601,8 +648,19 @@ void launch_first_layer_bounds(const LayerDev &L, const float *l0, const float *
                        geom_of(L), L.n_out, l0, u0, ld0, batch, lb_out, ub_out, n_total, L.out_off);
         return;
     }
-    launch_chained(first_layer_kernel, dim3(grid_for_warps(warps)), dim3(kWarpsPerBlock * 32), 0, st, L.W, L.bias_n,
-                   L.kind, geom_of(L), L.n_in, L.ld_in, L.n_out, l0, u0, ld0, batch, lb_out, ub_out, n_total, L.out_off);
+    // two neurons per warp: the box row is read once for both (measured best of 1, 2, 4, 8 on the 1024-wide layers)
+    constexpr int kPerWarp = 2;
+    const long long fc_warps = (long long)batch * ((L.n_out + kPerWarp - 1) / kPerWarp);
+    const bool vec_ok = L.ld_in % 4 == 0 && ld0 % 4 == 0 && 4 * ((L.n_in + 3) / 4) <= L.ld_in &&
+                        4 * ((L.n_in + 3) / 4) <= ld0 && (reinterpret_cast<uintptr_t>(L.W) & 15) == 0 &&
+                        (reinterpret_cast<uintptr_t>(l0) & 15) == 0 && (reinterpret_cast<uintptr_t>(u0) & 15) == 0;
+    if (vec_ok)
+        launch_chained(first_layer_vec_kernel<kPerWarp>, dim3(grid_for_warps(fc_warps)), dim3(kWarpsPerBlock * 32), 0,
+                       st, L.W, L.bias_n, L.n_in, L.ld_in, L.n_out, l0, u0, ld0, batch, lb_out, ub_out, n_total,
+                       L.out_off);
+    else
+        launch_chained(first_layer_kernel<kPerWarp>, dim3(grid_for_warps(fc_warps)), dim3(kWarpsPerBlock * 32), 0, st,
+                       L.W, L.bias_n, L.n_in, L.ld_in, L.n_out, l0, u0, ld0, batch, lb_out, ub_out, n_total, L.out_off);
 }
 
 void launch_relax(const LayerDev &L, float *lb_out, float *ub_out, int n_total, int batch,
