@@ -721,15 +721,18 @@ def test_bounded_wait_runs_out_and_the_net_stays_usable():
 
 # ---- the call allocates nothing and synchronises nothing: it can be captured into a CUDA graph ----
 
-@pytest.mark.parametrize("mode", ["tc", "tc16"])
+@pytest.mark.parametrize("mode", ["tc", "tc16", "auto_on_trial"])
 def test_call_is_capturable_in_a_cuda_graph(mode):
     import torch
     from paper_2507_20055_b200 import binding
-    w = wl.make_config(1, batch=8)               # 784 -> 100 x 6 -> 10
+    if mode == "auto_on_trial":
+        w = wl.make_config(2, batch=6)           # 784 -> 200 x 9 -> 10: AUTO runs the last layers on trial (a memset
+    else:                                        # and predicated re-runs inside the call)
+        w = wl.make_config(1, batch=8)           # 784 -> 100 x 6 -> 10
     ref = _oracle(w)
     net = binding.CertNet(w.layers, w.batch, w.clip_lo, w.clip_hi)
     try:
-        net.set_contraction({"tc": 2, "tc16": 3}[mode])
+        net.set_contraction({"tc": 2, "tc16": 3, "auto_on_trial": 0}[mode])
         c = torch.from_numpy(w.centers).cuda()
         lb = torch.zeros((w.batch, net.n_total), dtype=torch.float32, device="cuda")
         ub = torch.zeros_like(lb)
@@ -748,6 +751,8 @@ def test_call_is_capturable_in_a_cuda_graph(mode):
         torch.cuda.synchronize()
         g = {"lb": lb.cpu().numpy(), "ub": ub.cpu().numpy(), "codes": net.branch_codes(w.batch).cpu().numpy(),
              "status": net.last_status(), "layers": w.layers}
+        if mode == "auto_on_trial":
+            assert net.last_contraction_paths() & 128
         compare(g, ref, label=f"graph replay/{mode}")
     finally:
         net.destroy()
