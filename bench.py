@@ -33,8 +33,8 @@ NCU_TRAFFIC_BYTES_PER_ROW = {
     ("fc6x1024_b128", "tc"): {"bytes_per_row": (628.547840e6 + 487.951616e6) / 65536.0,
                               "kernel": "gemm_tc_kernel<TC_EPI_RELU, 2>",
                               "source": "profiles/gemm_tc_kernel_fc6x1024.md (32 boxes, scaled by rows)"},
-    ("fc6x1024_b128", "tc16"): {"bytes_per_row": (273.940992e6 + 232.271872e6) / 65536.0,
-                                "kernel": "gemm_tc16_kernel<TC_EPI_RELU>",
+    ("fc6x1024_b128", "tc16"): {"bytes_per_row": (273.501952e6 + 230.443776e6) / 65536.0,
+                                "kernel": "gemm_tc16_kernel<TC_EPI_RELU, one pass>",
                                 "source": "profiles/gemm_tc16_kernel_fc6x1024.md (32 boxes, scaled by rows)"},
 }
 

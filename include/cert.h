@@ -216,12 +216,16 @@ cert_status_t cert_net_selftest_bounded_wait(cert_net_t *net, void *stream);
  *   FFMA:    fp32 FMA units, unfused ReLU step and concretisation kernels.
  *   TC3XTF32: tcgen05 tensor cores with a 3-term TF32 split (fp32-accurate),
  *            ReLU back-step and concretisation fused into the epilogue.
- *   TC3XFP16: the same kernel structure with an fp16 split (x = hi + 2^-11 lo, three fp16
+ *   TC3XFP16: the same kernel structure with an fp16 split (x = hi + lo, three fp16
  *            products per multiply-add, exact in the fp32 accumulators): the accuracy of TC3XTF32 at
  *            twice the tensor-core rate and half the operand bytes, for nets of FC layers only and
  *            coefficients below 65504 in magnitude (beyond that cert_net_last_status reports
  *            CERT_ERR_RANGE and the results are invalid; values under 6.1e-5 are held to 1.5e-11
- *            absolute instead of 2^-22 relative).
+ *            absolute instead of 2^-22 relative).  The coefficients of a traversal travel times a power
+ *            of two, 2^a, so that their lo parts are ordinary fp16 numbers and all three products of a
+ *            k-block come from one staging of its tiles; the range is then |coefficient| 2^a < 65504:
+ *            a = what the layer's proved bound (see AUTO) leaves, at most 8; 4 for a layer that AUTO
+ *            runs on trial; 0 (the whole range) for a layer without a proof when this mode is forced.
  *   AUTO:    decided per affine layer k at create.  TC3XFP16 for the traversal of layer k when the net's
  *            weights prove that none of its coefficients can leave that range on any input: a ReLU
  *            back-step scales a coefficient by a slope in [0, 1], so every entry of the traversal's matrix

@@ -23,6 +23,12 @@ struct Tc16Layer {
     __half *W_hi = nullptr, *W_lo = nullptr;     // W_j transposed, [round_up(n_in, 32)][ld_out]
     cert::TcMap b_hi, b_lo, a_hi[3], a_lo[3], o_hi[3], o_lo[3];   // one per coefficient buffer
     cert::Tc16Plan plan;
+    // One-pass form: W' = 2^w_shift W_j as Wh = fp16(W'), Wl = fp16(W' - Wh), same layout.  w_shift puts the
+    // largest |W'| in [2^14, 2^15), so Wl is a normal fp16 number wherever |W| >= 2^-18 max|W|.
+    bool one_pass = false;
+    __half *Ws_hi = nullptr, *Ws_lo = nullptr;
+    cert::TcMap s_hi, s_lo;
+    float w_unscale = 1.0f;                      // 2^-w_shift
 };
 
 struct TcLayer {
@@ -111,6 +117,7 @@ struct cert_net {
     bool tc_ok = false;                      // tensor-core path usable on this net
     std::vector<TcLayer> tc;                 // per layer: operand maps and tile plan
     bool tc16_ok = false;                    // fp16-split path usable (FC layers only, CTA pairs available)
+    bool tc16_one_pass = false;              // its layers all have the operands of the one-pass form
     // AUTO takes the fp16 split: the net's weights prove that no coefficient of any traversal can leave the
     // fp16 range (fp16_coef_bound = the largest entry of |W_k| |W_k-1| ... |W_j| over all k > j >= 1; slopes of a
     // ReLU back-step lie in [0, 1], so every stored coefficient is below it in magnitude)
@@ -323,8 +330,10 @@ cert_status_t setup_tensor_core_path(cert_net *net, const cert_layer_desc_t *des
     for (int j = 0; j < K; ++j) all_fc = all_fc && net->layers[j].kind == CERT_LAYER_FC;
     net->tc16.assign(K, Tc16Layer());
     if (all_fc && ctas == 2 && cert::tc16_prepare_kernels()) {
-        bool all_ok = true;
+        bool all_ok = true, all_one_pass = true;
         std::vector<__half> h16, l16;
+        bool one_pass_wanted = true;
+        if (const char *e = std::getenv("CERT_TC16_ONE_PASS")) one_pass_wanted = std::atoi(e) != 0;
         for (int j = 0; j < K - 1 && all_ok; ++j) {
             LayerDev &L = net->layers[j];
             Tc16Layer &T = net->tc16[j];
@@ -349,6 +358,33 @@ cert_status_t setup_tensor_core_path(cert_net *net, const cert_layer_desc_t *des
             if (T.plan.stages < 2) { all_ok = false; break; }
             bool ok = cert::tc16_make_map(&T.b_hi, T.W_hi, L.n_out, L.n_in, L.ld_out, 64, T.plan.bn / 2) &&
                       cert::tc16_make_map(&T.b_lo, T.W_lo, L.n_out, L.n_in, L.ld_out, 64, T.plan.bn / 2);
+            if (ok && all_ok && one_pass_wanted) {
+                float wmax = 0.0f;
+                for (size_t i = 0; i < (size_t)L.n_out * L.n_in; ++i) wmax = std::max(wmax, std::fabs(descs[j].weight[i]));
+                int e = 0;
+                if (wmax > 0.0f) std::frexp(wmax, &e);               // wmax = m 2^e, m in [0.5, 1)
+                const int shift = wmax > 0.0f ? std::min(std::max(15 - e, -24), 24) : 0;
+                const float up = std::ldexp(1.0f, shift);
+                std::fill(h16.begin(), h16.end(), __float2half_rn(0.0f));
+                std::fill(l16.begin(), l16.end(), __float2half_rn(0.0f));
+                for (int t = 0; t < L.n_out; ++t)
+                    for (int s2 = 0; s2 < L.n_in; ++s2) {
+                        const float w = descs[j].weight[(size_t)t * L.n_in + s2] * up;   // exact
+                        const __half h = __float2half_rn(w);
+                        h16[(size_t)s2 * L.ld_out + t] = h;
+                        l16[(size_t)s2 * L.ld_out + t] = __float2half_rn(w - __half2float(h));
+                    }
+                if (!dev_alloc(net, (void **)&T.Ws_hi, h16.size() * sizeof(__half)) ||
+                    !dev_alloc(net, (void **)&T.Ws_lo, l16.size() * sizeof(__half)))
+                    return CERT_ERR_OOM;
+                if (cudaMemcpy(T.Ws_hi, h16.data(), h16.size() * sizeof(__half), cudaMemcpyHostToDevice) != cudaSuccess ||
+                    cudaMemcpy(T.Ws_lo, l16.data(), l16.size() * sizeof(__half), cudaMemcpyHostToDevice) != cudaSuccess)
+                    return CERT_ERR_CUDA;
+                T.w_unscale = std::ldexp(1.0f, -shift);
+                T.one_pass = cert::tc16_make_map(&T.s_hi, T.Ws_hi, L.n_out, L.n_in, L.ld_out, 64, T.plan.bn / 2) &&
+                             cert::tc16_make_map(&T.s_lo, T.Ws_lo, L.n_out, L.n_in, L.ld_out, 64, T.plan.bn / 2);
+            }
+            all_one_pass = all_one_pass && T.one_pass;
             long long rows_max = 0;
             for (int k = j + 1; k < K; ++k) rows_max = std::max(rows_max, 2LL * net->max_batch * net->layers[k].n_out);
             for (int p = 0; p < net->n_buf && ok; ++p) {
@@ -365,6 +401,7 @@ cert_status_t setup_tensor_core_path(cert_net *net, const cert_layer_desc_t *des
             if (ok) net->d_slots = std::max(net->d_slots, 2 * T.plan.n_tiles);
         }
         net->tc16_ok = all_ok;
+        net->tc16_one_pass = all_ok && all_one_pass;
         // The chain kernel: every layer a traversal passes through at most kChainMaxWidth neurons wide.
         bool chain = all_ok && net->skip_from.empty() && K <= cert::kChainMaxLayers && cert::chain16_prepare();
         if (const char *e = std::getenv("CERT_CHAIN")) chain = chain && std::atoi(e) != 0;
@@ -410,6 +447,7 @@ cert_status_t setup_tensor_core_path(cert_net *net, const cert_layer_desc_t *des
 #ifdef CERT_BOUNDS
 cert_status_t bounds_sync(cert_net *net, const void *const *extra, const size_t *extra_bytes, int n_extra);
 #endif
+constexpr int kQaMax = 8, kQaTrial = 4;     // exponents of the one-pass fp16 form's coefficient scale (run_tc16_steps)
 constexpr float kFp16Safe = 60000.0f;       // fp16's largest finite value is 65504; the margin covers fp32 rounding here
 
 cert_status_t prove_fp16_range(cert_net *net) {
@@ -789,6 +827,7 @@ struct Traversal {
     Recorder *rec;
     int mode;                 // the contraction mode of this traversal (AUTO resolved)
     int *status;              // the status word its kernels report to: the net's, or the layer's word of a speculative run
+    bool on_trial = false;    // a speculative fp16 run (a flagged range is made good by the re-run behind it)
     const int *run_if;        // not null: a re-run whose kernels do nothing unless that word is non-zero
     int batch, k, j_end, steps;
     long long rows;           // 2 * batch * n_k, ordered (box, side, neuron)
@@ -906,8 +945,26 @@ void run_tc16_steps(Traversal &t) {
         qh[p] = reinterpret_cast<__half *>(net->buf[p]);
         ql[p] = reinterpret_cast<__half *>(net->buf_lo[p]);
     }
+    // One-pass form: the traversal's coefficients travel as pairs of 2^qa Q.  With a range proof the exponent is
+    // what the proved bound leaves of the fp16 range (up to kQaMax: beyond that nothing is gained, lo parts are
+    // normal numbers for every coefficient that matters); without one, a run on trial takes kQaTrial (a flagged
+    // range costs the re-run) and a forced run takes 0 (the whole fp16 range, as the two-pass form).
+    const bool one_pass = net->tc16_one_pass;
+    int qa = 0;
+    if (one_pass) {
+        const float b = t.k < (int)net->fp16_layer_bound.size() ? net->fp16_layer_bound[t.k] : INFINITY;
+        if (std::isfinite(b) && b <= kFp16Safe) {
+            int e = 0;
+            std::frexp(kFp16Safe / std::max(b, 1e-30f), &e);          // ratio = m 2^e, m in [0.5, 1)
+            qa = std::min(std::max(e - 1, 0), kQaMax);
+        } else {
+            qa = t.on_trial ? kQaTrial : 0;
+        }
+    }
+    const float q_scale = std::ldexp(1.0f, qa), q_unscale = std::ldexp(1.0f, -qa);
     int cur = 0, dcur = 0, dslots = 1;
-    cert::launch_init_expr16(Lk, t.layer(t.k - 1), t.batch, qh[cur], ql[cur], net->dbuf[dcur], t.status, t.st);
+    cert::launch_init_expr16(Lk, t.layer(t.k - 1), t.batch, qh[cur], ql[cur], net->dbuf[dcur], t.status,
+                             one_pass ? q_scale : 1.0f, one_pass ? 1.0f : cert::kLoScale, t.st);
     t.rec->mark(CERT_CLASS_RELU_STEP);
     Waiting w;
     w.start(t);
@@ -919,6 +976,8 @@ void run_tc16_steps(Traversal &t) {
         const bool join = j > t.j_end && w.wait_for == j - 1;
         cert::TcArgs a = tc_args(t, Lj.n_out, Lk.n_out, Lj.ld_in, T.plan.bn, T.plan.n_tiles, T.plan.stages,
                                  T.plan.tmem_cols, 256, T.plan.n_tiles, dcur, dslots);
+        a.q_scale = q_scale; a.q_unscale = q_unscale; a.acc_scale = q_unscale * T.w_unscale;
+        const cert::TcMap &b_hi = one_pass ? T.s_hi : T.b_hi, &b_lo = one_pass ? T.s_lo : T.b_lo;
         const int pairs = std::min(a.total_tiles, net->sm_count / 2);
         if (j > t.j_end) {
             tc_relu_epilogue(a, t.layer(j - 1), true);
@@ -927,12 +986,12 @@ void run_tc16_steps(Traversal &t) {
                 a.add_lo = reinterpret_cast<const float *>(ql[w.kept]);
             }
             a.add_identity = (join && w.identity) ? 1 : 0;
-            cert::launch_gemm_tc16(cert::TC_EPI_RELU, pairs, T.a_hi[cur], T.a_lo[cur], T.b_hi, T.b_lo, T.o_hi[nxt],
+            cert::launch_gemm_tc16(cert::TC_EPI_RELU, one_pass, pairs, T.a_hi[cur], T.a_lo[cur], b_hi, b_lo, T.o_hi[nxt],
                                    T.o_lo[nxt], a, T.plan.smem_bytes, t.st);
             if (join) w.joined();
         } else {
             a.l0 = t.box_l; a.u0 = t.box_u;
-            cert::launch_gemm_tc16(cert::TC_EPI_CONCRETIZE, pairs, T.a_hi[cur], T.a_lo[cur], T.b_hi, T.b_lo,
+            cert::launch_gemm_tc16(cert::TC_EPI_CONCRETIZE, one_pass, pairs, T.a_hi[cur], T.a_lo[cur], b_hi, b_lo,
                                    T.a_hi[cur], T.a_lo[cur], a, T.plan.smem_bytes, t.st);
         }
         t.rec->mark(CERT_CLASS_AFFINE);
@@ -1320,8 +1379,10 @@ cert_status_t backsub_impl(cert_net *net, const float *centers, float eps, int b
             }
             t.mode = CERT_CONTRACTION_TC3XFP16;
             t.status = net->spec_dev + k;
+            t.on_trial = true;
             if (net->chain_ok) run_chain16(t);
             else run_tc16_steps(t);
+            t.on_trial = false;
             t.mode = CERT_CONTRACTION_TC3XTF32;
             t.status = net->status_dev;
             t.run_if = net->spec_dev + k;
@@ -1822,7 +1883,7 @@ cert_status_t cert_reusecert_bounds(cert_net_t *net, const float *centers, float
         a.bias2 = RL.bias2; a.colsum = R.colsum;
         a.status = net->status_dev;
         const int pairs = std::min(a.total_tiles, net->sm_count / 2);
-        cert::launch_gemm_tc16(cert::TC_EPI_REUSE, pairs, RL.a16_hi[xa], RL.a16_lo[xa], RL.b16_hi, RL.b16_lo,
+        cert::launch_gemm_tc16(cert::TC_EPI_REUSE, false, pairs, RL.a16_hi[xa], RL.a16_lo[xa], RL.b16_hi, RL.b16_lo,
                                RL.o32[xb], RL.o32[xb], a, RL.plan16.smem_bytes, st);
         rec.mark(CERT_CLASS_AFFINE);
         cert::launch_reuse_relax(R.colsum, RL.ld_s, R.R / 32, Lk, batch, lb_out, ub_out, n_total, net->codes,

@@ -35,6 +35,9 @@ struct TcArgs {
     int n_k;         // neurons of the layer being bounded (decodes a row into box, side, neuron)
     int ld_n;        // padded width of the output (neurons below layer j)
     int bn, n_tiles, stages, tmem_cols;
+    // fp16-split kernel, one-pass form: coefficients travel as pairs of q_scale * Q (q_scale = 2^a, q_unscale = 2^-a);
+    // acc_scale = 2^-(a+s) comes off the accumulator (the weights carry 2^s)
+    float q_scale, q_unscale, acc_scale;
     int total_tiles; // row panels x column tiles (a row panel is 128 rows per CTA of the group)
     // Banded form of a conv back-step on dense coefficient maps (n_bands > 0).  Maps are held row-major by map
     // row ("y-major": [y][channel][x]), so the coefficients of `band_rin` consecutive rows of layer j's output map

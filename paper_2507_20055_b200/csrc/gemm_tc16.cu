@@ -12,6 +12,16 @@
 // pass 2 stages only the hi tiles (two k-blocks per pipeline stage).  A coefficient beyond the fp16 range
 // raises bit 1 of the status word.
 //
+// ONEPASS: both operands carry a power of two, Q' = 2^a Q and W' = 2^s W (a per traversal, s per layer), large
+// enough that the lo parts need no factor of their own to stay normal fp16 numbers: x' = hi + lo with
+// hi = fp16(x'), lo = fp16(x' - hi).  The three products then share one scale,
+//   D += Q_lo * W_hi + Q_hi * W_lo + Q_hi * W_hi,
+// so a k-block is staged once (four tiles) for all of them and the epilogue multiplies by 2^-(a+s).  The two-pass
+// form stages six tiles per k-block.  The kernel is bound by what an SM takes in from L2 per cycle (a plain
+// fp16 GEMM of this tile shape needs the same 64 bytes per cycle and SM as the two-pass form), so fewer staged
+// bytes per product are what raises the tensor pipe's share.  The price is range: |Q| 2^a must stay in the fp16
+// range, where the two-pass form only needs |Q| to.
+//
 // CTA pairs (tcgen05 cta_group::2) on 256-row panels, persistent over (row panel, column tile) work tiles,
 // two accumulators so that the epilogue of a tile overlaps the MMAs of the next, as in gemm_tc.cu.  A tile's
 // MMAs take half the time they take there, so eight epilogue warps (two per TMEM lane quarter, taking
@@ -45,7 +55,7 @@ struct __align__(8) Barriers16 {
     uint32_t abort_flag;
 };
 
-template <int EPI>
+template <int EPI, bool ONEPASS>
 __global__ void __launch_bounds__(kThreads16, 1)
 gemm_tc16_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_constant__ CUtensorMap map_a_lo,
                  const __grid_constant__ CUtensorMap map_b_hi, const __grid_constant__ CUtensorMap map_b_lo,
@@ -124,7 +134,7 @@ gemm_tc16_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_cons
                     if (++s == stages) { s = 0; phase ^= 1; }
                 }
                 // pass 2: the hi tiles of two k-blocks per stage (the second in the slots of the lo tiles)
-                for (int kb = 0; kb < num_kb && ok; kb += 2) {
+                for (int kb = 0; !ONEPASS && kb < num_kb && ok; kb += 2) {
                     if (!mbar_wait(&bars->empty[s], phase ^ 1) || *abort_flag) { ok = false; break; }
                     uint8_t *st = smem + (size_t)s * stage_bytes;
                     const bool two = kb + 1 < num_kb;
@@ -184,12 +194,13 @@ gemm_tc16_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_cons
                         const uint64_t ko = (uint64_t)(k * 2);   // 16 halves = 32 bytes = 2 x 16-byte units
                         mma_f16<CTAS>(d, da_lo + ko, db_hi + ko, idesc, (kb | k) ? 1u : 0u);
                         mma_f16<CTAS>(d, da_hi + ko, db_lo + ko, idesc, 1u);
+                        if (ONEPASS) mma_f16<CTAS>(d, da_hi + ko, db_hi + ko, idesc, 1u);
                     }
                     tcgen05_commit<CTAS>(&bars->empty[s]);
                     if (++s == stages) { s = 0; phase ^= 1; }
                 }
                 // pass 2: hi * hi on top of the cross terms scaled by 2^-11
-                for (int kb = 0; kb < num_kb && ok; kb += 2) {
+                for (int kb = 0; !ONEPASS && kb < num_kb && ok; kb += 2) {
                     if (!mbar_wait(&bars->full[s], phase) || *abort_flag) { ok = false; break; }
                     tcgen05_fence_after();
                     const uint32_t st = smem_u32(smem + (size_t)s * stage_bytes);
@@ -261,6 +272,11 @@ gemm_tc16_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_cons
                 __syncwarp();
                 tmem_ld32(t_addr + (uint32_t)c0, v);
                 tmem_ld_wait();
+                if (ONEPASS) {
+                    // the accumulator holds 2^(a+s) times the product
+#pragma unroll
+                    for (int e = 0; e < 32; ++e) v[e] = __float_as_uint(__uint_as_float(v[e]) * a.acc_scale);
+                }
                 if (EPI == TC_EPI_RELU || EPI == TC_EPI_RELU_SKIP) {
                     // the slab is free again once the previous chunk's stores have read it
                     if (lane == 0) tma_store_wait_read();
@@ -308,9 +324,15 @@ gemm_tc16_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_cons
                                     const __half2 l01 = *reinterpret_cast<const __half2 *>(&sl.x), l23 = *reinterpret_cast<const __half2 *>(&sl.y);
                                     const float2 fh01 = __half22float2(h01), fh23 = __half22float2(h23);
                                     const float2 fl01 = __half22float2(l01), fl23 = __half22float2(l23);
-                                    const float inv = 1.0f / kLoScale;
-                                    s4[0] = fmaf(fl01.x, inv, fh01.x); s4[1] = fmaf(fl01.y, inv, fh01.y);
-                                    s4[2] = fmaf(fl23.x, inv, fh23.x); s4[3] = fmaf(fl23.y, inv, fh23.y);
+                                    if (ONEPASS) {
+                                        // a pair of this traversal: 2^a times the coefficient, lo unscaled
+                                        s4[0] = (fh01.x + fl01.x) * a.q_unscale; s4[1] = (fh01.y + fl01.y) * a.q_unscale;
+                                        s4[2] = (fh23.x + fl23.x) * a.q_unscale; s4[3] = (fh23.y + fl23.y) * a.q_unscale;
+                                    } else {
+                                        const float inv = 1.0f / kLoScale;
+                                        s4[0] = fmaf(fl01.x, inv, fh01.x); s4[1] = fmaf(fl01.y, inv, fh01.y);
+                                        s4[2] = fmaf(fl23.x, inv, fh23.x); s4[3] = fmaf(fl23.y, inv, fh23.y);
+                                    }
                                 }
                                 const int own = a.add_identity ? (int)(rr % a.n_k) : -1;
 #pragma unroll
@@ -344,9 +366,10 @@ gemm_tc16_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_cons
                             __half h[4], l[4];
 #pragma unroll
                             for (int e = 0; e < 4; ++e) {
-                                out_of_range |= row_ok && !(fabsf(q[e]) <= 60000.0f);
-                                h[e] = __float2half_rn(q[e]);
-                                l[e] = __float2half_rn((q[e] - __half2float(h[e])) * kLoScale);
+                                const float x = ONEPASS ? q[e] * a.q_scale : q[e];
+                                out_of_range |= row_ok && !(fabsf(x) <= 60000.0f);
+                                h[e] = __float2half_rn(x);
+                                l[e] = __float2half_rn(ONEPASS ? x - __half2float(h[e]) : (x - __half2float(h[e])) * kLoScale);
                             }
                             ph[g2 * 2 + 0] = (uint32_t)__half_as_ushort(h[0]) | ((uint32_t)__half_as_ushort(h[1]) << 16);
                             ph[g2 * 2 + 1] = (uint32_t)__half_as_ushort(h[2]) | ((uint32_t)__half_as_ushort(h[3]) << 16);
@@ -474,16 +497,18 @@ __device__ __forceinline__ float warp_sum16(float v) {
 }
 
 // Start of a back-substitution at FC layer k as an fp16 pair: row i of W_k pushed through the ReLU below,
-// constant = b_k[i] + the nu terms + Q.b of the layer below.  A warp takes kRowsPerWarp consecutive neurons
+// constant = b_k[i] + the nu terms + Q.b of the layer below.  The pair is hi = fp16(q_scale x),
+// lo = fp16(lo_scale (q_scale x - hi)): (1, 2^11) for the two-pass contraction, (2^a, 1) for the one-pass one.  A warp takes kRowsPerWarp consecutive neurons
 // of one (box, side), 8 columns per lane: the relaxation and bias vectors are read once for those rows.
 constexpr int kRowsPerWarp = 4;
 
-__global__ void expr_start16_kernel(const float *__restrict__ Wk, int ldw_k, const float *__restrict__ bias_k,
+// three 256-thread blocks per SM: the kernel only writes, and needs the warps in flight
+__global__ void __launch_bounds__(256, 3) expr_start16_kernel(const float *__restrict__ Wk, int ldw_k, const float *__restrict__ bias_k,
                                     __half *__restrict__ Q_hi, __half *__restrict__ Q_lo, float *__restrict__ d,
                                     long long n_warps, int n_k, int n, int ld, int has_relu,
                                     const float *__restrict__ lamL, const float *__restrict__ lamU,
                                     const float *__restrict__ nuU, const float *__restrict__ bias_below,
-                                    int *__restrict__ status) {
+                                    int *__restrict__ status, float q_scale, float lo_scale) {
     pdl_trigger();
     pdl_wait();
     const long long w = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
@@ -544,9 +569,10 @@ __global__ void expr_start16_kernel(const float *__restrict__ Wk, int ldw_k, con
 #pragma unroll
                 for (int z = 0; z < 2; ++z) {
                     dacc[rr] = fmaf(q[e + z], bz[e + z], dacc[rr]);
-                    out_of_range |= !(fabsf(q[e + z]) <= 60000.0f);
-                    h[z] = __float2half_rn(q[e + z]);
-                    l[z] = __float2half_rn((q[e + z] - __half2float(h[z])) * kLoScale);
+                    const float x = q[e + z] * q_scale;       // a power of two
+                    out_of_range |= !(fabsf(x) <= 60000.0f);
+                    h[z] = __float2half_rn(x);
+                    l[z] = __float2half_rn((x - __half2float(h[z])) * lo_scale);
                 }
                 ph[e >> 1] = (uint32_t)__half_as_ushort(h[0]) | ((uint32_t)__half_as_ushort(h[1]) << 16);
                 pl[e >> 1] = (uint32_t)__half_as_ushort(l[0]) | ((uint32_t)__half_as_ushort(l[1]) << 16);
@@ -569,7 +595,7 @@ typedef CUresult (*EncodeTiledFn16)(CUtensorMap *, CUtensorMapDataType, cuuint32
                                     CUtensorMapFloatOOBfill);
 EncodeTiledFn16 g_encode16 = nullptr;
 
-template <int EPI>
+template <int EPI, bool ONEPASS>
 void launch_one16(int pairs, const CUtensorMap &ah, const CUtensorMap &al, const CUtensorMap &bh,
                   const CUtensorMap &bl, const CUtensorMap &oh, const CUtensorMap &ol, const TcArgs &args,
                   int smem_bytes, cudaStream_t st) {
@@ -587,7 +613,13 @@ void launch_one16(int pairs, const CUtensorMap &ah, const CUtensorMap &al, const
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = pdl_enabled() ? 2 : 1;
-    cudaLaunchKernelEx(&cfg, gemm_tc16_kernel<EPI>, ah, al, bh, bl, oh, ol, args);
+    cudaLaunchKernelEx(&cfg, gemm_tc16_kernel<EPI, ONEPASS>, ah, al, bh, bl, oh, ol, args);
+}
+
+template <int EPI, bool ONEPASS>
+bool allow_smem16() {
+    return cudaFuncSetAttribute(gemm_tc16_kernel<EPI, ONEPASS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                kTcSmemMax) == cudaSuccess;
 }
 
 }  // namespace
@@ -603,14 +635,10 @@ bool tc16_prepare_kernels() {
         }
         g_encode16 = reinterpret_cast<EncodeTiledFn16>(fn);
     }
-    if (cudaFuncSetAttribute(gemm_tc16_kernel<TC_EPI_RELU_SKIP>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemMax) !=
-            cudaSuccess ||
-        cudaFuncSetAttribute(gemm_tc16_kernel<TC_EPI_RELU>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemMax) !=
-            cudaSuccess ||
-        cudaFuncSetAttribute(gemm_tc16_kernel<TC_EPI_REUSE>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemMax) !=
-            cudaSuccess ||
-        cudaFuncSetAttribute(gemm_tc16_kernel<TC_EPI_CONCRETIZE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             kTcSmemMax) != cudaSuccess) {
+    if (!allow_smem16<TC_EPI_RELU_SKIP, false>() || !allow_smem16<TC_EPI_RELU, false>() ||
+        !allow_smem16<TC_EPI_REUSE, false>() || !allow_smem16<TC_EPI_CONCRETIZE, false>() ||
+        !allow_smem16<TC_EPI_RELU_SKIP, true>() || !allow_smem16<TC_EPI_RELU, true>() ||
+        !allow_smem16<TC_EPI_CONCRETIZE, true>()) {
         cudaGetLastError();
         return false;
     }
@@ -647,8 +675,9 @@ Tc16Plan tc16_tile_plan(int N) {
     return p;
 }
 
-void launch_gemm_tc16(int epi, int pairs, const TcMap &a_hi, const TcMap &a_lo, const TcMap &b_hi, const TcMap &b_lo,
-                      const TcMap &o_hi, const TcMap &o_lo, const TcArgs &args, int smem_bytes, cudaStream_t st) {
+void launch_gemm_tc16(int epi, bool one_pass, int pairs, const TcMap &a_hi, const TcMap &a_lo, const TcMap &b_hi,
+                      const TcMap &b_lo, const TcMap &o_hi, const TcMap &o_lo, const TcArgs &args, int smem_bytes,
+                      cudaStream_t st) {
     const CUtensorMap &ah = reinterpret_cast<const CUtensorMap &>(a_hi);
     const CUtensorMap &al = reinterpret_cast<const CUtensorMap &>(a_lo);
     const CUtensorMap &bh = reinterpret_cast<const CUtensorMap &>(b_hi);
@@ -656,18 +685,24 @@ void launch_gemm_tc16(int epi, int pairs, const TcMap &a_hi, const TcMap &a_lo, 
     const CUtensorMap &oh = reinterpret_cast<const CUtensorMap &>(o_hi);
     const CUtensorMap &ol = reinterpret_cast<const CUtensorMap &>(o_lo);
     const bool skip = args.add_hi || args.add_identity;
-    if (epi == TC_EPI_RELU && skip) launch_one16<TC_EPI_RELU_SKIP>(pairs, ah, al, bh, bl, oh, ol, args, smem_bytes, st);
-    else if (epi == TC_EPI_RELU) launch_one16<TC_EPI_RELU>(pairs, ah, al, bh, bl, oh, ol, args, smem_bytes, st);
-    else if (epi == TC_EPI_REUSE) launch_one16<TC_EPI_REUSE>(pairs, ah, al, bh, bl, oh, ol, args, smem_bytes, st);
-    else launch_one16<TC_EPI_CONCRETIZE>(pairs, ah, al, bh, bl, oh, ol, args, smem_bytes, st);
+    if (one_pass) {
+        if (epi == TC_EPI_RELU && skip) launch_one16<TC_EPI_RELU_SKIP, true>(pairs, ah, al, bh, bl, oh, ol, args, smem_bytes, st);
+        else if (epi == TC_EPI_RELU) launch_one16<TC_EPI_RELU, true>(pairs, ah, al, bh, bl, oh, ol, args, smem_bytes, st);
+        else launch_one16<TC_EPI_CONCRETIZE, true>(pairs, ah, al, bh, bl, oh, ol, args, smem_bytes, st);
+        return;
+    }
+    if (epi == TC_EPI_RELU && skip) launch_one16<TC_EPI_RELU_SKIP, false>(pairs, ah, al, bh, bl, oh, ol, args, smem_bytes, st);
+    else if (epi == TC_EPI_RELU) launch_one16<TC_EPI_RELU, false>(pairs, ah, al, bh, bl, oh, ol, args, smem_bytes, st);
+    else if (epi == TC_EPI_REUSE) launch_one16<TC_EPI_REUSE, false>(pairs, ah, al, bh, bl, oh, ol, args, smem_bytes, st);
+    else launch_one16<TC_EPI_CONCRETIZE, false>(pairs, ah, al, bh, bl, oh, ol, args, smem_bytes, st);
 }
 
 void launch_init_expr16(const LayerDev &Lk, const LayerDev &Lb, int batch, __half *Q_hi, __half *Q_lo, float *d,
-                        int *status, cudaStream_t st) {
+                        int *status, float q_scale, float lo_scale, cudaStream_t st) {
     const long long n_warps = 2LL * batch * ((Lk.n_out + kRowsPerWarp - 1) / kRowsPerWarp);
     launch_chained(expr_start16_kernel, dim3((unsigned)ceil_div_ll(n_warps, 8)), dim3(256), 0, st, Lk.W, Lk.ld_in,
                    Lk.bias_n, Q_hi, Q_lo, d, n_warps, Lk.n_out, Lb.n_out, Lb.ld_out, Lb.relu_after, Lb.lamL, Lb.lamU, Lb.nuU,
-                   Lb.bias_n, status);
+                   Lb.bias_n, status, q_scale, lo_scale);
 }
 
 }  // namespace cert
