@@ -977,6 +977,7 @@ void run_tc16_steps(Traversal &t) {
         cert::TcArgs a = tc_args(t, Lj.n_out, Lk.n_out, Lj.ld_in, T.plan.bn, T.plan.n_tiles, T.plan.stages,
                                  T.plan.tmem_cols, 256, T.plan.n_tiles, dcur, dslots);
         a.q_scale = q_scale; a.q_unscale = q_unscale; a.acc_scale = q_unscale * T.w_unscale;
+        a.n_narrow = T.plan.n_narrow;
         const cert::TcMap &b_hi = one_pass ? T.s_hi : T.b_hi, &b_lo = one_pass ? T.s_lo : T.b_lo;
         const int pairs = std::min(a.total_tiles, net->sm_count / 2);
         if (j > t.j_end) {

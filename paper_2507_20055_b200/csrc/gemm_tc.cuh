@@ -38,6 +38,7 @@ struct TcArgs {
     // fp16-split kernel, one-pass form: coefficients travel as pairs of q_scale * Q (q_scale = 2^a, q_unscale = 2^-a);
     // acc_scale = 2^-(a+s) comes off the accumulator (the weights carry 2^s)
     float q_scale, q_unscale, acc_scale;
+    int n_narrow;    // fp16-split kernel: the last n_narrow column tiles of a row panel are bn - 32 columns wide
     int total_tiles; // row panels x column tiles (a row panel is 128 rows per CTA of the group)
     // Banded form of a conv back-step on dense coefficient maps (n_bands > 0).  Maps are held row-major by map
     // row ("y-major": [y][channel][x]), so the coefficients of `band_rin` consecutive rows of layer j's output map

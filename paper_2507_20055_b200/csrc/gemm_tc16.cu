@@ -118,7 +118,11 @@ gemm_tc16_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_cons
             int armed = 0;
             for (int t = group; t < total_tiles && ok; t += n_groups) {
                 const int row0 = (t / n_tiles) * (BM * CTAS) + (int)rank * BM;
-                const int col0 = (t % n_tiles) * BN + (int)rank * BNL;
+                // the last n_narrow column tiles are 32 columns narrower: this CTA's half of W_j's rows starts
+                // accordingly (the TMA box keeps its size; the rows beyond the half are not read by the MMAs)
+                const int nt = t % n_tiles;
+                const int narrow = nt - (n_tiles - a.n_narrow);
+                const int col0 = nt * BN - (narrow > 0 ? narrow * 32 : 0) + (int)rank * (narrow >= 0 ? BNL - 16 : BNL);
                 // pass 1: all four tiles of a k-block per stage
                 for (int kb = 0; kb < num_kb && ok; ++kb) {
                     if (!mbar_wait(&bars->empty[s], phase ^ 1) || *abort_flag) { ok = false; break; }
@@ -169,7 +173,8 @@ gemm_tc16_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_cons
         // ------------------------------------------------------------ MMA issuer (the leader CTA)
         if (lane == 0 && rank == 0) {
             // kind::f16: D = f32, A = B = f16 (format 0), both K-major
-            const uint32_t idesc = (1u << 4) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)((BM * CTAS) >> 4) << 24);
+            const uint32_t idesc_wide = (1u << 4) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)((BM * CTAS) >> 4) << 24);
+            const uint32_t idesc_narrow = (1u << 4) | ((uint32_t)((BN - 32) >> 3) << 17) | ((uint32_t)((BM * CTAS) >> 4) << 24);
             int s = 0;
             uint32_t phase = 0;
             bool ok = true;
@@ -180,6 +185,7 @@ gemm_tc16_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_cons
                 if (!mbar_wait(&bars->acc_empty[acc], acc_phase ^ 1) || *abort_flag) { ok = false; break; }
                 tcgen05_fence_after();
                 const uint32_t d = tmem_base + (uint32_t)(acc * BN);
+                const uint32_t idesc = (t % n_tiles) >= n_tiles - a.n_narrow ? idesc_narrow : idesc_wide;
                 // pass 1: cross terms
                 for (int kb = 0; kb < num_kb && ok; ++kb) {
                     if (!mbar_wait(&bars->full[s], phase) || *abort_flag) { ok = false; break; }
@@ -250,8 +256,11 @@ gemm_tc16_kernel(const __grid_constant__ CUtensorMap map_a_hi, const __grid_cons
             if (!mbar_wait(&bars->acc_full[acc], acc_phase) || *abort_flag) { ok = false; break; }
             tcgen05_fence_after();
             const uint32_t t_addr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN);
-            for (int c0 = 32 * half_id; c0 < BN; c0 += 64) {
-                const int col0 = nt * BN + c0;
+            const int narrow = nt - (n_tiles - a.n_narrow);
+            const int tile_col0 = nt * BN - (narrow > 0 ? narrow * 32 : 0);
+            const int tile_cols = narrow >= 0 ? BN - 32 : BN;
+            for (int c0 = 32 * half_id; c0 < tile_cols; c0 += 64) {
+                const int col0 = tile_col0 + c0;
                 if (col0 >= a.ld_n) break;                   // warp-uniform; ld_n is a multiple of 32
                 uint32_t v[32];
                 // a residual connection ends on these neurons: its waiting coefficients (an fp16 pair here) for the
@@ -662,8 +671,13 @@ bool tc16_make_map(TcMap *m, const __half *base, long long inner, long long oute
 Tc16Plan tc16_tile_plan(int N) {
     Tc16Plan p;
     p.n_tiles = (N + 255) / 256;
-    int b = ((N + p.n_tiles - 1) / p.n_tiles + 31) / 32 * 32;
+    // 32-column units spread over the tiles: the first tiles take one unit more than the last n_narrow ones
+    const int units = (N + 31) / 32;
+    int b = (units + p.n_tiles - 1) / p.n_tiles * 32;
     p.bn = b;
+    p.n_narrow = (b / 32) * p.n_tiles - units;
+    if (b < 64) p.n_narrow = 0;           // a 32-column tile cannot lose a unit
+    if (p.n_narrow >= p.n_tiles) p.n_narrow = 0;
     const int stage_bytes = 2 * kATileBytes + 2 * (b / 2) * BKH * 2;
     const int fixed = kEpiBytes16 + (int)sizeof(Barriers16) + 1024;
     int st = (kTcSmemMax - fixed) / stage_bytes;

@@ -19,6 +19,7 @@ constexpr float kLoScale = 2048.0f;
 
 struct Tc16Plan {
     int bn, n_tiles, stages, tmem_cols, smem_bytes;
+    int n_narrow;    // the last n_narrow column tiles are bn - 32 wide (N = 784: 224 + 3 x 192 instead of 4 x 224)
 };
 
 bool tc16_prepare_kernels();

@@ -399,6 +399,45 @@ def test_fp16_split_contraction(name, chain, monkeypatch):
     compare(g, _oracle(w), label=f"{name}/tc16/chain={chain}")
 
 
+@pytest.mark.parametrize("name", sorted(FC_NETS))
+def test_fp16_split_two_pass_form(name, monkeypatch):
+    """One launch per back-step with CERT_TC16_ONE_PASS=0 at create: the pair keeps its lo part times 2^11 and a
+    k-block is staged twice (the form ReuseCert's contraction always runs).  The default, one pass over K with both
+    operands times a power of two, is what every other fp16-split test of the per-step kernel runs."""
+    monkeypatch.setenv("CERT_CHAIN", "0")
+    monkeypatch.setenv("CERT_TC16_ONE_PASS", "0")
+    w = FC_NETS[name]()
+    g = run_gpu(w, contraction=TC16)
+    assert g["paths"] & 16 and not g["paths"] & 32
+    compare(g, _oracle(w), label=f"{name}/tc16/two passes")
+
+
+def test_fp16_split_one_pass_scale_follows_the_proved_bound(monkeypatch):
+    """Coefficients of the one-pass form travel times 2^a, a = what the layer's proved bound leaves of the fp16 range
+    (at most 8).  Weights of +-1.5 on 40-wide layers make the bound grow sixtyfold per layer, so a falls from 8 to 3
+    along the net and the output layer, without a proof, runs at a = 0 when the mode is forced: every layer must
+    agree with the oracle, and none may raise the range flag (run_gpu checks the status word)."""
+    from paper_2507_20055_b200 import binding
+    monkeypatch.setenv("CERT_CHAIN", "0")
+    w = wl.small_fc([64, 40, 40, 40, 40, 6], batch=5, eps=0.002, seed=97)
+    for l in w.layers[1:]:
+        l.weight[...] = np.where(l.weight >= 0, 1.5, -1.5).astype(np.float32)
+    net = binding.CertNet(w.layers, w.batch, w.clip_lo, w.clip_hi)
+    try:
+        bounds = [net.fp16_coefficient_bound(k) for k in range(1, len(w.layers))]
+    finally:
+        net.destroy()
+    assert bounds[0] <= 60000.0 / 256                       # a = 8
+    assert 60000.0 / 16 < bounds[2] <= 60000.0              # 0 <= a <= 3
+    assert bounds[3] > 60000.0                              # no proof
+    g = run_gpu(w, contraction=TC16)
+    assert g["paths"] & 16 and not g["paths"] & 32
+    compare(g, _oracle(w), min_good_fraction=0.4, label="pm1.5/tc16 one pass")
+    g = run_gpu(w)                                          # AUTO: the output layer on trial at a = 4
+    assert g["paths"] & 128
+    compare(g, _oracle(w), min_good_fraction=0.4, label="pm1.5/auto")
+
+
 def test_fp16_split_chain_wide_input_and_many_layers():
     """A CIFAR-sized input (14 column tiles in the concretising step) and the deepest net the chain kernel's
     parameter block takes (12 layers); one layer more goes back to one launch per back-step."""
