@@ -438,6 +438,20 @@ def test_fp16_split_one_pass_scale_follows_the_proved_bound(monkeypatch):
     compare(g, _oracle(w), min_good_fraction=0.4, label="pm1.5/auto")
 
 
+@pytest.mark.parametrize("sizes", [[784, 600, 330, 7], [600, 544, 700, 258, 3], [1000, 288, 513, 10]])
+@pytest.mark.parametrize("mode", ["tc16", "tc16_two_pass", "auto"])
+def test_fp16_split_unequal_column_tiles(sizes, mode, monkeypatch):
+    """Layers wider than 256 (one launch per back-step) whose widths make the column tiles of a row panel unequal
+    (600 = 224 + 192 + 192, 784 = 224 + 3 x 192, 330 -> 192 + 160), ragged K blocks and row panels that the
+    2 x batch x n_k rows do not fill."""
+    if mode == "tc16_two_pass":
+        monkeypatch.setenv("CERT_TC16_ONE_PASS", "0")
+    w = wl.small_fc(sizes, batch=3, eps=0.005, seed=sum(sizes))
+    g = run_gpu(w, contraction=0 if mode == "auto" else TC16, max_batch=4)
+    assert g["paths"] & 16 and not g["paths"] & 32
+    compare(g, _oracle(w), min_good_fraction=0.6, label=f"{sizes}/{mode}")
+
+
 def test_fp16_split_chain_wide_input_and_many_layers():
     """A CIFAR-sized input (14 column tiles in the concretising step) and the deepest net the chain kernel's
     parameter block takes (12 layers); one layer more goes back to one launch per back-step."""
