@@ -99,6 +99,32 @@ __global__ void reuse_init16_kernel(const float *__restrict__ W0t, int ldw, cons
     for (int o = lane; r < rows && o < octs; o += 32) {
         const int col0 = o * 8;
         __half h[8], l[8];
+        if ((n & 7) == 0 && (ldw & 3) == 0 && col0 < 2 * n && s <= n0) {
+            // the eight columns lie on one side (n a multiple of 8): 16-byte loads of the weights (or the bias on the
+            // constant row), the slopes and the intercepts
+            const bool upper = col0 >= n;
+            const int t0 = upper ? col0 - n : col0;
+            const float *base_p = s < n0 ? W0t + (size_t)s * ldw + t0 : bias + t0;
+            const float4 b0 = *reinterpret_cast<const float4 *>(base_p), b1 = *reinterpret_cast<const float4 *>(base_p + 4);
+            const float base[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
+            float lam[8] = {1.0f, 1.0f, 1.0f, 1.0f, 1.0f, 1.0f, 1.0f, 1.0f};
+            float nu[8] = {0.0f, 0.0f, 0.0f, 0.0f, 0.0f, 0.0f, 0.0f, 0.0f};
+            if (has_relu) {
+                const float *lam_p = (upper ? lamU : lamL) + (size_t)box * ld_relax + t0;
+                const float4 a0 = *reinterpret_cast<const float4 *>(lam_p), a1 = *reinterpret_cast<const float4 *>(lam_p + 4);
+                lam[0] = a0.x; lam[1] = a0.y; lam[2] = a0.z; lam[3] = a0.w; lam[4] = a1.x; lam[5] = a1.y; lam[6] = a1.z; lam[7] = a1.w;
+                if (upper && s == n0) {
+                    const float *nu_p = nuU + (size_t)box * ld_relax + t0;
+                    const float4 n0v = *reinterpret_cast<const float4 *>(nu_p), n1v = *reinterpret_cast<const float4 *>(nu_p + 4);
+                    nu[0] = n0v.x; nu[1] = n0v.y; nu[2] = n0v.z; nu[3] = n0v.w; nu[4] = n1v.x; nu[5] = n1v.y; nu[6] = n1v.z; nu[7] = n1v.w;
+                }
+            }
+#pragma unroll
+            for (int e = 0; e < 8; ++e) store_pair16(fmaf(lam[e], base[e], nu[e]), h[e], l[e], out_of_range);
+            CERT_ST(*reinterpret_cast<uint4 *>(S_hi + (size_t)r * ld_s + col0), pack8(h));
+            CERT_ST(*reinterpret_cast<uint4 *>(S_lo + (size_t)r * ld_s + col0), pack8(l));
+            continue;
+        }
 #pragma unroll
         for (int e = 0; e < 8; ++e) {
             const int col = col0 + e;
@@ -139,21 +165,39 @@ __global__ void reuse_scale16_kernel(const float *__restrict__ raw, __half *__re
         const float4 r1 = *reinterpret_cast<const float4 *>(raw + (size_t)r * ld_s + col0 + 4);
         const float rv[8] = {r0.x, r0.y, r0.z, r0.w, r1.x, r1.y, r1.z, r1.w};
         __half h[8], l[8];
-#pragma unroll
-        for (int e = 0; e < 8; ++e) {
-            const int col = col0 + e;
-            float v = 0.0f;
-            if (col < 2 * n && s <= n0) {
-                v = rv[e];
-                if (has_relu) {
-                    const bool upper = col >= n;
-                    const int t = upper ? col - n : col;
-                    const float lam = upper ? lamU[(size_t)box * ld_relax + t] : lamL[(size_t)box * ld_relax + t];
-                    const float nu = (upper && s == n0) ? nuU[(size_t)box * ld_relax + t] : 0.0f;
-                    v = fmaf(lam, v, nu);
-                }
+        if ((n & 7) == 0 && col0 < 2 * n && s <= n0 && has_relu) {
+            // the eight columns lie on one side (n a multiple of 8): the slopes, and on the constant row the
+            // intercepts, come as two 16-byte loads each
+            const bool upper = col0 >= n;
+            const float *lam_p = (upper ? lamU : lamL) + (size_t)box * ld_relax + (upper ? col0 - n : col0);
+            const float4 a0 = *reinterpret_cast<const float4 *>(lam_p), a1 = *reinterpret_cast<const float4 *>(lam_p + 4);
+            const float lam[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
+            float nu[8] = {0.0f, 0.0f, 0.0f, 0.0f, 0.0f, 0.0f, 0.0f, 0.0f};
+            if (upper && s == n0) {
+                const float *nu_p = nuU + (size_t)box * ld_relax + (col0 - n);
+                const float4 n0v = *reinterpret_cast<const float4 *>(nu_p), n1v = *reinterpret_cast<const float4 *>(nu_p + 4);
+                nu[0] = n0v.x; nu[1] = n0v.y; nu[2] = n0v.z; nu[3] = n0v.w;
+                nu[4] = n1v.x; nu[5] = n1v.y; nu[6] = n1v.z; nu[7] = n1v.w;
             }
-            store_pair16(v, h[e], l[e], out_of_range);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) store_pair16(fmaf(lam[e], rv[e], nu[e]), h[e], l[e], out_of_range);
+        } else {
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                const int col = col0 + e;
+                float v = 0.0f;
+                if (col < 2 * n && s <= n0) {
+                    v = rv[e];
+                    if (has_relu) {
+                        const bool upper = col >= n;
+                        const int t = upper ? col - n : col;
+                        const float lam = upper ? lamU[(size_t)box * ld_relax + t] : lamL[(size_t)box * ld_relax + t];
+                        const float nu = (upper && s == n0) ? nuU[(size_t)box * ld_relax + t] : 0.0f;
+                        v = fmaf(lam, v, nu);
+                    }
+                }
+                store_pair16(v, h[e], l[e], out_of_range);
+            }
         }
         CERT_ST(*reinterpret_cast<uint4 *>(S_hi + (size_t)r * ld_s + col0), pack8(h));
         CERT_ST(*reinterpret_cast<uint4 *>(S_lo + (size_t)r * ld_s + col0), pack8(l));
