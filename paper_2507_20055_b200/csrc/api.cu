@@ -419,8 +419,10 @@ cert_status_t setup_tensor_core_path(cert_net *net, const cert_layer_desc_t *des
                 cert::ChainLayer &C = net->chain.layer[j];
                 C.n_out = L.n_out; C.n_in = L.n_in; C.ld_in = L.ld_in;
                 if (j + 1 < K) {
-                    net->chain.b_hi[j] = net->tc16[j].b_hi;
-                    net->chain.b_lo[j] = net->tc16[j].b_lo;
+                    // (the one-pass form's pairs of the scaled weights where the net has them)
+                    net->chain.b_hi[j] = net->tc16_one_pass ? net->tc16[j].s_hi : net->tc16[j].b_hi;
+                    net->chain.b_lo[j] = net->tc16_one_pass ? net->tc16[j].s_lo : net->tc16[j].b_lo;
+                    C.w_unscale = net->tc16[j].w_unscale;
                     C.bn = net->tc16[j].plan.bn; C.n_tiles = net->tc16[j].plan.n_tiles;
                 }
                 if (j > 0) {
@@ -915,6 +917,22 @@ void run_interval_step(Traversal &t) {
     if (Lk.relu_after || t.k + 1 < net->n_layers) t.relax(nullptr, 0);
 }
 
+// One-pass form of the fp16 split: the traversal's coefficients travel as pairs of 2^qa Q.  With a range proof the
+// exponent is what the proved bound leaves of the fp16 range (up to kQaMax: beyond that nothing is gained, lo parts
+// are normal numbers for every coefficient that matters); without one, a run on trial takes kQaTrial (a flagged
+// range costs the re-run) and a forced run takes 0 (the whole fp16 range, as the two-pass form).
+int fp16_scale_exponent(const Traversal &t) {
+    const cert_net *net = t.net;
+    if (!net->tc16_one_pass) return 0;
+    const float b = t.k < (int)net->fp16_layer_bound.size() ? net->fp16_layer_bound[t.k] : INFINITY;
+    if (std::isfinite(b) && b <= kFp16Safe) {
+        int e = 0;
+        std::frexp(kFp16Safe / std::max(b, 1e-30f), &e);          // ratio = m 2^e, m in [0.5, 1)
+        return std::min(std::max(e - 1, 0), kQaMax);
+    }
+    return t.on_trial ? kQaTrial : 0;
+}
+
 // fp16 split, narrow FC nets: the whole traversal in one launch, the coefficient panel in shared memory.
 void run_chain16(Traversal &t) {
     cert_net *net = t.net;
@@ -928,6 +946,9 @@ void run_chain16(Traversal &t) {
     a.status = t.status;
     a.stages = net->chain_stages; a.a_blocks = net->chain_a_blocks;
     a.b_chunk_bytes = net->chain_chunk; a.vec_ld = net->chain_vec_ld;
+    const int qa = fp16_scale_exponent(t);
+    a.one_pass = net->tc16_one_pass ? 1 : 0;
+    a.q_scale = std::ldexp(1.0f, qa); a.q_unscale = std::ldexp(1.0f, -qa);
     const int pairs = (int)std::min<long long>(cert::ceil_div_ll(t.rows, 256), net->sm_count / 2);
     cert::launch_chain16(net->chain, a, pairs, net->chain_smem, t.st);
     t.rec->mark(CERT_CLASS_AFFINE);
@@ -945,22 +966,8 @@ void run_tc16_steps(Traversal &t) {
         qh[p] = reinterpret_cast<__half *>(net->buf[p]);
         ql[p] = reinterpret_cast<__half *>(net->buf_lo[p]);
     }
-    // One-pass form: the traversal's coefficients travel as pairs of 2^qa Q.  With a range proof the exponent is
-    // what the proved bound leaves of the fp16 range (up to kQaMax: beyond that nothing is gained, lo parts are
-    // normal numbers for every coefficient that matters); without one, a run on trial takes kQaTrial (a flagged
-    // range costs the re-run) and a forced run takes 0 (the whole fp16 range, as the two-pass form).
     const bool one_pass = net->tc16_one_pass;
-    int qa = 0;
-    if (one_pass) {
-        const float b = t.k < (int)net->fp16_layer_bound.size() ? net->fp16_layer_bound[t.k] : INFINITY;
-        if (std::isfinite(b) && b <= kFp16Safe) {
-            int e = 0;
-            std::frexp(kFp16Safe / std::max(b, 1e-30f), &e);          // ratio = m 2^e, m in [0.5, 1)
-            qa = std::min(std::max(e - 1, 0), kQaMax);
-        } else {
-            qa = t.on_trial ? kQaTrial : 0;
-        }
-    }
+    const int qa = fp16_scale_exponent(t);
     const float q_scale = std::ldexp(1.0f, qa), q_unscale = std::ldexp(1.0f, -qa);
     int cur = 0, dcur = 0, dslots = 1;
     cert::launch_init_expr16(Lk, t.layer(t.k - 1), t.batch, qh[cur], ql[cur], net->dbuf[dcur], t.status,

@@ -8,7 +8,7 @@
 //   start:   Q = rows of W_k through the ReLU of layer k-1, written straight into shared memory
 //            in the swizzled K-major layout the tensor cores read;
 //   step j:  P = Q * W_j on the tensor cores (W_j streamed through a TMA pipeline, accumulator in tensor
-//            memory, two passes as in gemm_tc16.cu), the epilogue applies the ReLU back-step and
+//            memory, one pass or two as in gemm_tc16.cu), the epilogue applies the ReLU back-step and
 //            writes the result over Q as the next step's operand;
 //   end:     the last step's epilogue is map(simplify_lower/upper) against the box (or the stored
 //            bounds of the layer reached); only the bounds leave the kernel.
@@ -84,7 +84,7 @@ __device__ __forceinline__ void bulk_load(uint32_t dst, const void *src, uint32_
 // Writes 32 consecutive columns [c0, c0+32) of panel row `row` as an fp16 pair into the K-major,
 // 128-byte-swizzled blocks the MMA reads (block = c0 / 64; 16-byte chunk g of a row sits at g ^ (row & 7)).
 __device__ __forceinline__ void write_panel_chunk(uint32_t a_hi, uint32_t a_lo, int row, int c0, const float (&q)[32],
-                                                  bool check, bool &out_of_range) {
+                                                  bool check, bool &out_of_range, float lo_scale) {
     const uint32_t off = (uint32_t)(c0 >> 6) * kABlockBytes + (uint32_t)row * 128u;
     const int g0 = (c0 & 63) >> 3;
 #pragma unroll
@@ -98,7 +98,7 @@ __device__ __forceinline__ void write_panel_chunk(uint32_t a_hi, uint32_t a_lo, 
                 const float x = q[g * 8 + e + z];
                 out_of_range |= check && !(fabsf(x) <= 60000.0f);
                 h[z] = __float2half_rn(x);
-                l[z] = __float2half_rn((x - __half2float(h[z])) * kLoScale);
+                l[z] = __float2half_rn((x - __half2float(h[z])) * lo_scale);
             }
             ph[e >> 1] = (uint32_t)__half_as_ushort(h[0]) | ((uint32_t)__half_as_ushort(h[1]) << 16);
             pl[e >> 1] = (uint32_t)__half_as_ushort(l[0]) | ((uint32_t)__half_as_ushort(l[1]) << 16);
@@ -111,8 +111,10 @@ __device__ __forceinline__ void write_panel_chunk(uint32_t a_hi, uint32_t a_lo, 
     }
 }
 
+template <bool ONEPASS>
 __global__ void __launch_bounds__(kThreadsChain, 1)
 chain16_kernel(const __grid_constant__ ChainParams P, const ChainArgs a) {
+    // ONEPASS: see ChainArgs::one_pass (a template parameter so that the two-pass form carries none of its factors)
     pdl_trigger();
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -222,7 +224,7 @@ chain16_kernel(const __grid_constant__ ChainParams P, const ChainArgs a) {
                             if (++s == stages) { s = 0; phase ^= 1; }
                         }
                         // pass 2: the hi tiles of two k-blocks per stage
-                        for (int kb = 0; kb < num_kb && ok; kb += 2) {
+                        for (int kb = 0; !ONEPASS && kb < num_kb && ok; kb += 2) {
                             if (!mbar_wait(&bars->empty[s], phase ^ 1) || *abort_flag) { ok = false; break; }
                             uint8_t *st = Bst + (size_t)s * kStageBytes;
                             const bool two = kb + 1 < num_kb;
@@ -293,12 +295,13 @@ chain16_kernel(const __grid_constant__ ChainParams P, const ChainArgs a) {
                                 const uint64_t ko = (uint64_t)(k * 2);   // 16 halves = 32 bytes = 2 x 16-byte units
                                 mma_f16<CTAS>(d, da_lo + ko, db_hi + ko, idesc, (kb | k) ? 1u : 0u);
                                 mma_f16<CTAS>(d, da_hi + ko, db_lo + ko, idesc, 1u);
+                                if (ONEPASS) mma_f16<CTAS>(d, da_hi + ko, db_hi + ko, idesc, 1u);
                             }
                             tcgen05_commit<CTAS>(&bars->empty[s]);
                             if (++s == stages) { s = 0; phase ^= 1; }
                         }
                         // pass 2: hi * hi on top of the cross terms scaled by 2^-11
-                        for (int kb = 0; kb < num_kb && ok; kb += 2) {
+                        for (int kb = 0; !ONEPASS && kb < num_kb && ok; kb += 2) {
                             if (!mbar_wait(&bars->full[s], phase) || *abort_flag) { ok = false; break; }
                             tcgen05_fence_after();
                             const uint32_t st = smem_u32(Bst + (size_t)s * kStageBytes);
@@ -337,6 +340,10 @@ chain16_kernel(const __grid_constant__ ChainParams P, const ChainArgs a) {
         const uint32_t a_ready_addr = map_to_cta(smem_u32(&bars->a_ready[0]), 0);
         bool ok = true, out_of_range = false;
         int lt = 0, vstep = 0;
+        // one-pass form: the coefficients and the row constant are held times q_scale throughout (every factor is a
+        // power of two, so the results are those of the unscaled arithmetic); the constant is scaled back as it leaves
+        const float q_scale = ONEPASS ? a.q_scale : 1.0f;
+        constexpr float lo_scale = ONEPASS ? 1.0f : kLoScale;
         for (long long p = group; p < n_panels && ok; p += n_groups) {
             const long long r = p * (BM * CTAS) + (long long)rank * BM + prow;
             const bool row_ok = r < a.M;
@@ -344,7 +351,7 @@ chain16_kernel(const __grid_constant__ ChainParams P, const ChainArgs a) {
             const int b = (int)(rr / (2LL * a.n_k));
             const int upper = (int)((rr / a.n_k) & 1);
             const int i = (int)(rr % a.n_k);
-            float dacc = (col_group == 0) ? a.bias_k[i] : 0.0f;
+            float dacc = (col_group == 0) ? a.bias_k[i] * q_scale : 0.0f;
             {
                 // start: row i of W_k through the ReLU of layer k-1; the constant takes the nu terms and Q.b
                 const ChainLayer &Lk = P.layer[a.k];
@@ -375,7 +382,7 @@ chain16_kernel(const __grid_constant__ ChainParams P, const ChainArgs a) {
                             for (int e = 0; e < 4; ++e) {
                                 float x = 0.0f;
                                 if (col + e < n) {
-                                    const float c = c4[e];
+                                    const float c = c4[e] * q_scale;
                                     const bool nonneg = (c >= 0.0f);
                                     const bool use_lower = upper ? !nonneg : nonneg;
                                     x = c * (use_lower ? l4[e] : u4[e]);
@@ -389,7 +396,7 @@ chain16_kernel(const __grid_constant__ ChainParams P, const ChainArgs a) {
 #pragma unroll
                         for (int e = 0; e < 32; ++e) q[e] = 0.0f;
                     }
-                    write_panel_chunk(a_hi0, a_lo0, prow, c0, q, row_ok, out_of_range);
+                    write_panel_chunk(a_hi0, a_lo0, prow, c0, q, row_ok, out_of_range, lo_scale);
                     fence_async_smem();
                     __syncwarp();
                     if (lane == 0) mbar_arrive_cluster(a_ready_addr + (uint32_t)((c0 >> 6) * sizeof(uint64_t)));
@@ -410,6 +417,7 @@ chain16_kernel(const __grid_constant__ ChainParams P, const ChainArgs a) {
                 const int ld_in = L.ld_in, n_in = L.n_in, bn = L.bn, n_tiles = L.n_tiles, relu_below = L.relu_below;
                 const float *lamL = L.lamL + relax_row, *lamU = L.lamU + relax_row, *nuU = L.nuU + relax_row;
                 const float *bias_below = L.bias_below;
+                const float acc_scale = ONEPASS ? L.w_unscale : 1.0f;     // the accumulator holds 2^s times the product
                 // staged copies of these vectors (the producer fetched them while the MMAs ran): the bias always,
                 // the relaxation for rows of the CTA's first two boxes
                 const int vbuf = (a.vec_ld > 0 && !last) ? (vstep & 1) : -1;
@@ -454,7 +462,7 @@ chain16_kernel(const __grid_constant__ ChainParams P, const ChainArgs a) {
                                                     n4[4] = {nu.x, nu.y, nu.z, nu.w};
 #pragma unroll
                                         for (int e = 0; e < 4; ++e) {
-                                            const float c = __uint_as_float(v[g * 4 + e]);
+                                            const float c = __uint_as_float(v[g * 4 + e]) * acc_scale;
                                             const bool nonneg = (c >= 0.0f);
                                             const bool use_lower = upper ? !nonneg : nonneg;
                                             q[g * 4 + e] = c * (use_lower ? l4[e] : u4[e]);
@@ -462,7 +470,7 @@ chain16_kernel(const __grid_constant__ ChainParams P, const ChainArgs a) {
                                         }
                                     } else {
 #pragma unroll
-                                        for (int e = 0; e < 4; ++e) q[g * 4 + e] = __uint_as_float(v[g * 4 + e]);
+                                        for (int e = 0; e < 4; ++e) q[g * 4 + e] = __uint_as_float(v[g * 4 + e]) * acc_scale;
                                     }
 #pragma unroll
                                     for (int e = 0; e < 4; ++e) dacc = fmaf(q[g * 4 + e], b4[e], dacc);
@@ -471,7 +479,7 @@ chain16_kernel(const __grid_constant__ ChainParams P, const ChainArgs a) {
 #pragma unroll
                                 for (int e = 0; e < 32; ++e) q[e] = 0.0f;
                             }
-                            write_panel_chunk(a_hi0, a_lo0, prow, c0, q, row_ok, out_of_range);
+                            write_panel_chunk(a_hi0, a_lo0, prow, c0, q, row_ok, out_of_range, lo_scale);
                             fence_async_smem();
                             __syncwarp();
                             if (lane == 0) mbar_arrive_cluster(a_ready_addr + (uint32_t)((c0 >> 6) * sizeof(uint64_t)));
@@ -500,7 +508,7 @@ chain16_kernel(const __grid_constant__ ChainParams P, const ChainArgs a) {
                                 const float lo4[4] = {l4.x, l4.y, l4.z, l4.w}, up4[4] = {u4.x, u4.y, u4.z, u4.w};
 #pragma unroll
                                 for (int e = 0; e < 4; ++e) {
-                                    const float c = __uint_as_float(v[g * 4 + e]);
+                                    const float c = __uint_as_float(v[g * 4 + e]) * acc_scale;
                                     const bool nonneg = (c >= 0.0f);
                                     dacc = fmaf(c, (nonneg != (upper != 0)) ? lo4[e] : up4[e], dacc);
                                 }
@@ -513,7 +521,7 @@ chain16_kernel(const __grid_constant__ ChainParams P, const ChainArgs a) {
                 }
                 if (vbuf >= 0) ++vstep;
             }
-            if (ok && row_ok) CERT_ST(a.d_out[(size_t)col_group * a.slot_stride + r], dacc);
+            if (ok && row_ok) CERT_ST(a.d_out[(size_t)col_group * a.slot_stride + r], ONEPASS ? dacc * a.q_unscale : dacc);
         }
         if (out_of_range) atomicOr(a.status, 2);
         if (!ok) {
@@ -554,7 +562,8 @@ int chain16_smem_bytes(int a_blocks, int max_bnl, int ld_max, int *stages, int *
 }
 
 bool chain16_prepare() {
-    if (cudaFuncSetAttribute(chain16_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemMax) != cudaSuccess) {
+    if (cudaFuncSetAttribute(chain16_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemMax) != cudaSuccess ||
+        cudaFuncSetAttribute(chain16_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmemMax) != cudaSuccess) {
         cudaGetLastError();
         return false;
     }
@@ -576,7 +585,8 @@ void launch_chain16(const ChainParams &P, const ChainArgs &a, int pairs, int sme
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = pdl_enabled() ? 2 : 1;
-    cudaLaunchKernelEx(&cfg, chain16_kernel, P, a);
+    if (a.one_pass) cudaLaunchKernelEx(&cfg, chain16_kernel<true>, P, a);
+    else cudaLaunchKernelEx(&cfg, chain16_kernel<false>, P, a);
 }
 
 }  // namespace cert

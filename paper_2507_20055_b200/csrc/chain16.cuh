@@ -21,6 +21,7 @@ struct ChainLayer {
     int relu_below;                     // a ReLU sits on the neurons below (j >= 1)
     const float *lamL, *lamU, *nuU;     // relaxation of layer j-1, [batch][ld_in]
     const float *bias_below;            // bias of layer j-1, [ld_in]
+    float w_unscale;                    // one-pass form: 2^-s, the factor the weight pair of this layer carries, inverted
 };
 
 struct ChainParams {
@@ -43,6 +44,11 @@ struct ChainArgs {
     int b_chunk_bytes;                  // room for one CTA's share of a W_j tile k-block (a multiple of 1024)
     int vec_ld;                         // > 0: the relaxation and bias vectors of a step are staged in shared memory
                                         // (two buffers of 7 * vec_ld floats: bias, then lamL, lamU, nuU of two boxes)
+    // One-pass form (see gemm_tc16.cu): the panel holds q_scale * Q (a power of two) as hi + lo with an unscaled lo,
+    // the weight maps hold the pairs of 2^s W_j, a k-block of W_j is streamed once for its three products, and the
+    // row constants are kept times q_scale until they leave (q_unscale = 1 / q_scale).
+    int one_pass;
+    float q_scale, q_unscale;
 };
 
 bool chain16_prepare();

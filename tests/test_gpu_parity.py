@@ -574,8 +574,16 @@ def test_auto_runs_unproven_layers_in_the_fp16_split_on_trial():
     g = run_gpu(w)
     assert g["paths"] & 32 and g["paths"] & 128 and not g["paths"] & 1
     compare(g, ref, label="fc9x200/auto on trial")
+    # forced, the layers without a proof keep the whole fp16 range (coefficients times 1 instead of times 16): the
+    # same bounds up to the rounding of the smallest lo parts
     forced = run_gpu(w, contraction=TC16)
-    assert np.array_equal(forced["lb"], g["lb"]) and np.array_equal(forced["ub"], g["ub"])
+    compare(forced, ref, label="fc9x200/fp16 split forced")
+    for key in ("lb", "ub"):
+        assert np.all(np.abs(forced[key] - g[key]) <= 2e-6 * (1.0 + np.abs(g[key])))
+    # ... and not the TF32 split's: the re-run behind the trial did nothing
+    tf32 = run_gpu(w, contraction=2)
+    last = slice(-w.layers[-1].weight.shape[0], None)
+    assert not np.array_equal(tf32["lb"][:, last], g["lb"][:, last])
 
 
 def test_host_calls_report_the_device_status():
