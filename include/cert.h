@@ -224,7 +224,7 @@ cert_status_t cert_net_selftest_bounded_wait(cert_net_t *net, void *stream);
  *            absolute instead of 2^-22 relative).  The coefficients of a traversal travel times a power
  *            of two, 2^a, so that their lo parts are ordinary fp16 numbers and all three products of a
  *            k-block come from one staging of its tiles; the range is then |coefficient| 2^a < 65504:
- *            a = what the layer's proved bound (see AUTO) leaves, at most 8; 4 for a layer that AUTO
+ *            a = what the layer's proved bound (see AUTO) leaves, at most 14; 4 for a layer that AUTO
  *            runs on trial; 0 (the whole range) for a layer without a proof when this mode is forced.
  *   AUTO:    decided per affine layer k at create.  TC3XFP16 for the traversal of layer k when the net's
  *            weights prove that none of its coefficients can leave that range on any input: a ReLU

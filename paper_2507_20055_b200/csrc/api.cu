@@ -449,7 +449,7 @@ cert_status_t setup_tensor_core_path(cert_net *net, const cert_layer_desc_t *des
 #ifdef CERT_BOUNDS
 cert_status_t bounds_sync(cert_net *net, const void *const *extra, const size_t *extra_bytes, int n_extra);
 #endif
-constexpr int kQaMax = 8, kQaTrial = 4;     // exponents of the one-pass fp16 form's coefficient scale (run_tc16_steps)
+constexpr int kQaMax = 14, kQaTrial = 4;     // exponents of the one-pass fp16 form's coefficient scale (run_tc16_steps)
 constexpr float kFp16Safe = 60000.0f;       // fp16's largest finite value is 65504; the margin covers fp32 rounding here
 
 cert_status_t prove_fp16_range(cert_net *net) {
@@ -918,8 +918,8 @@ void run_interval_step(Traversal &t) {
 }
 
 // One-pass form of the fp16 split: the traversal's coefficients travel as pairs of 2^qa Q.  With a range proof the
-// exponent is what the proved bound leaves of the fp16 range (up to kQaMax: beyond that nothing is gained, lo parts
-// are normal numbers for every coefficient that matters); without one, a run on trial takes kQaTrial (a flagged
+// exponent is what the proved bound leaves of the fp16 range (up to kQaMax; the lo part of a coefficient is a normal
+// fp16 number where |Q| 2^qa >= 2^-3); without one, a run on trial takes kQaTrial (a flagged
 // range costs the re-run) and a forced run takes 0 (the whole fp16 range, as the two-pass form).
 int fp16_scale_exponent(const Traversal &t) {
     const cert_net *net = t.net;

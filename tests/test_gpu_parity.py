@@ -414,7 +414,7 @@ def test_fp16_split_two_pass_form(name, monkeypatch):
 
 def test_fp16_split_one_pass_scale_follows_the_proved_bound(monkeypatch):
     """Coefficients of the one-pass form travel times 2^a, a = what the layer's proved bound leaves of the fp16 range
-    (at most 8).  Weights of +-1.5 on 40-wide layers make the bound grow sixtyfold per layer, so a falls from 8 to 3
+    (at most 14).  Weights of +-1.5 on 40-wide layers make the bound grow sixtyfold per layer, so a falls from 14 to 3
     along the net and the output layer, without a proof, runs at a = 0 when the mode is forced: every layer must
     agree with the oracle, and none may raise the range flag (run_gpu checks the status word)."""
     from paper_2507_20055_b200 import binding
@@ -427,7 +427,7 @@ def test_fp16_split_one_pass_scale_follows_the_proved_bound(monkeypatch):
         bounds = [net.fp16_coefficient_bound(k) for k in range(1, len(w.layers))]
     finally:
         net.destroy()
-    assert bounds[0] <= 60000.0 / 256                       # a = 8
+    assert bounds[0] <= 60000.0 / 16384                     # a = 14
     assert 60000.0 / 16 < bounds[2] <= 60000.0              # 0 <= a <= 3
     assert bounds[3] > 60000.0                              # no proof
     g = run_gpu(w, contraction=TC16)
