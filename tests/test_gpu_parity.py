@@ -452,6 +452,16 @@ def test_fp16_split_unequal_column_tiles(sizes, mode, monkeypatch):
     compare(g, _oracle(w), min_good_fraction=0.6, label=f"{sizes}/{mode}")
 
 
+@pytest.mark.parametrize("mode", ["tc16", "auto"])
+def test_fp16_split_unequal_column_tiles_with_residual_connections(mode):
+    """272-wide layers (column tiles of 160 and 128) in a net with residual connections: the joining epilogue reads the
+    waiting pair at the narrower tile's columns."""
+    w = wl.residual_fc(300, 272, 2, 6, batch=3, eps=0.01, seed=41)
+    g = run_gpu(w, contraction=0 if mode == "auto" else TC16, max_batch=4)
+    assert g["paths"] & 16
+    compare(g, _oracle(w), min_good_fraction=0.6, label=f"residual 272-wide/{mode}")
+
+
 def test_fp16_split_chain_wide_input_and_many_layers():
     """A CIFAR-sized input (14 column tiles in the concretising step) and the deepest net the chain kernel's
     parameter block takes (12 layers); one layer more goes back to one launch per back-step."""
