@@ -390,7 +390,13 @@ def main():
                 "                     'sustained': {'tflops': s[0], 'sm_mhz': s[1], 'ms': s[2]}}\n"
                 "    except binding.CertError as e:\n"
                 "        out[name] = {'error': str(e)}\n"
-                "print('MICRO ' + json.dumps(out))\n")
+                "try:\n"
+                "    t = binding.peak_microbench(3, 5.0)\n"
+                "    out['tma_l2_to_smem'] = {'tb_per_s': t[0], 'sm_mhz': t[1], 'ms': t[2],\n"
+                "                             'bytes_per_cycle_per_sm': t[0] * 1e12 / (t[1] * 1e6) / %d}\n"
+                "except binding.CertError as e:\n"
+                "    out['tma_l2_to_smem'] = {'error': str(e)}\n"
+                "print('MICRO ' + json.dumps(out))\n" % torch.cuda.get_device_properties(local_rank).multi_processor_count)
         try:
             env = dict(os.environ, CUDA_VISIBLE_DEVICES=os.environ.get("CUDA_VISIBLE_DEVICES", str(local_rank)))
             r = subprocess.run([sys.executable, "-c", code], cwd=ROOT, env=env, capture_output=True, text=True,

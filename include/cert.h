@@ -377,6 +377,11 @@ cert_status_t cert_first_layer_bounds_noalloc(const float *weight, const float *
  *   kind 0  tcgen05.mma kind::f16,  CTA pairs, 256 x 256 tiles, both operands resident in shared memory
  *   kind 1  tcgen05.mma kind::tf32, the same shape
  *   kind 2  fp32 fused multiply-adds in registers (one 1024-thread block per multiprocessor)
+ *   kind 3  bulk copies from L2 into shared memory: one block per multiprocessor keeps eight 16 KB copies in flight
+ *           from a 512 KB region of its own (74 MB in all, resident in L2) and nothing reads what lands; this is the
+ *           path the operand tiles of the tensor-core contractions travel.  tflops_out then receives TERABYTES per
+ *           second over all multiprocessors (divide by their number and by sm_mhz_out for bytes per cycle and SM);
+ *           the call allocates and frees that buffer too
  * The kernel is sized by a short calibration run to last about target_ms (0 < target_ms <= 2000); a few ms give
  * a burst figure at boost clocks, a few hundred ms a figure under the power limit.  Outputs (HOST pointers):
  * tflops_out = executed flops / CUDA-event time (2 per multiply-add), sm_mhz_out (may be NULL) = SM cycles per

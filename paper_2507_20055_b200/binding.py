@@ -370,7 +370,7 @@ def first_layer_bounds_noalloc(weight, bias, centers, eps, clip_lo, clip_hi, lb_
 
 def peak_microbench(kind: int, target_ms: float = 5.0, stream_ptr: int = 0):
     """cert_peak_microbench: (TFLOP/s, SM MHz seen by the kernel, ms) for kind 0 = tcgen05 f16, 1 = tcgen05 tf32,
-    2 = fp32 FMA units."""
+    2 = fp32 FMA units; kind 3 = bulk copies from L2 into shared memory, first value in TB/s over all SMs."""
     out = (ctypes.c_double * 3)()
     base = ctypes.addressof(out)
     _check(_lib.cert_peak_microbench(int(kind), float(target_ms), base, base + 8, base + 16, stream_ptr),

@@ -1,13 +1,19 @@
 // Micro-kernels that measure the denominators of the contraction rooflines on the device at hand: the rate of
 // tcgen05.mma kind::f16 and kind::tf32 in the instruction shape the product kernels use (CTA pairs, 256 x 256
 // tiles, both operands resident in shared memory, no loads in the loop), and the rate of the fp32 FMA units on
-// a register-only loop.  (No counterpart in the paper: measurement support.)
+// a register-only loop; and the rate at which the SMs take bulk copies from L2 into shared memory, which is what
+// bounds the fp16-split contraction once its operands are staged more than once.  (No counterpart in the paper:
+// measurement support.)
 //
 // Each kernel also reads the SM cycle counter and the global nanosecond timer at its start and end, so that the
 // rate comes with the SM clock it was measured at (rates are compared per cycle, whatever the power state).
 #include <cmath>
 
+#include <cuda.h>
+#include <cuda_fp16.h>
+
 #include "common.cuh"
+#include "gemm_tc16.cuh"
 #include "tc_ptx.cuh"
 
 namespace cert {
@@ -142,6 +148,58 @@ ffma_peak_kernel(int iters, float *sink, unsigned long long *clocks_out) {
     }
 }
 
+// KIND 3: what the SMs take in from L2 through TMA tile loads into shared memory, the path the contractions' operand
+// tiles travel.  One CTA per SM (it asks for most of the shared memory) keeps eight 16 KB tile loads in flight from
+// a region of its own of a buffer that fits L2 (the tiles of a 128-row panel of a 1024-wide fp16 matrix, over and
+// over), and nothing reads what lands: the rate is the intake alone.  A single thread issues and waits (bounded waits; on a run-out it stops issuing and waits for what is
+// in flight before the CTA gives its shared memory back).
+constexpr int kIntakeSlots = 8;
+constexpr int kIntakeChunk = 16 * 1024;             // the size of an operand tile of the fp16-split kernel
+constexpr int kIntakeTilesPerRow = 16;              // the block's region: 128 rows of 16 x 64 halves (2 KB pitch, 256 KB)
+
+struct __align__(8) IntakeBars {
+    uint64_t full[kIntakeSlots];
+};
+
+__global__ void __launch_bounds__(128, 1)
+l2_intake_kernel(const __grid_constant__ CUtensorMap map, int n_loads, int *status, unsigned long long *clocks_out) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    IntakeBars *bars = reinterpret_cast<IntakeBars *>(smem + kIntakeSlots * kIntakeChunk);
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kIntakeSlots; ++s) mbar_init(&bars->full[s], 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    fence_async_smem();
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        const unsigned long long c0 = (unsigned long long)clock64(), t0 = global_ns();
+        bool ok = true;
+        int issued = 0;
+        for (int i = 0; i < n_loads && ok; ++i) {
+            const int s = i % kIntakeSlots;
+            const int use = i / kIntakeSlots;
+            if (use > 0 && !mbar_wait(&bars->full[s], (uint32_t)((use - 1) & 1))) { ok = false; break; }
+            mbar_arrive_expect_tx(&bars->full[s], kIntakeChunk);
+            // tile i of the block's 128 rows: 64 halves (one 128-byte swizzle row) x 128 rows, as an A tile of the
+            // fp16-split contraction
+            tma_load_2d<1>(smem_u32(smem + (size_t)s * kIntakeChunk), &map, smem_u32(&bars->full[s]),
+                           (i % kIntakeTilesPerRow) * 64, (int)blockIdx.x * 128);
+            issued = i + 1;
+        }
+        // everything in flight lands before the CTA ends
+        const int first = issued > kIntakeSlots ? issued - kIntakeSlots : 0;
+        for (int i = first; i < issued; ++i)
+            if (!mbar_wait(&bars->full[i % kIntakeSlots], (uint32_t)((i / kIntakeSlots) & 1))) ok = false;
+        if (!ok) atomicOr(status, 1);
+        if (blockIdx.x == 0) {
+            clocks_out[0] = (unsigned long long)clock64() - c0;
+            clocks_out[1] = global_ns() - t0;
+        }
+    }
+    __syncthreads();
+}
+
 }  // namespace
 
 }  // namespace cert
@@ -149,7 +207,7 @@ ffma_peak_kernel(int iters, float *sink, unsigned long long *clocks_out) {
 extern "C" cert_status_t cert_peak_microbench(int kind, double target_ms, double *tflops_out, double *sm_mhz_out,
                                               double *ms_out, void *stream) {
     using namespace cert;
-    if (kind < 0 || kind > 2 || !tflops_out || !(target_ms > 0.0) || target_ms > 2000.0) return CERT_ERR_INVALID_ARG;
+    if (kind < 0 || kind > 3 || !tflops_out || !(target_ms > 0.0) || target_ms > 2000.0) return CERT_ERR_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     int dev = 0, sms = 0;
     if (cudaGetDevice(&dev) != cudaSuccess ||
@@ -160,12 +218,15 @@ extern "C" cert_status_t cert_peak_microbench(int kind, double target_ms, double
     int *status = nullptr;
     unsigned long long *clocks = nullptr;
     float *sink = nullptr;
+    uint8_t *l2buf = nullptr;
+    const unsigned long long intake_per_cta = 256ull * 1024ull;     // 128 rows of 2 KB; 148 SMs: 37 MB, inside the 126 MB L2
     cudaEvent_t e0 = nullptr, e1 = nullptr;
     cert_status_t rc = CERT_OK;
     auto cleanup = [&]() {
         if (status) cudaFree(status);
         if (clocks) cudaFree(clocks);
         if (sink) cudaFree(sink);
+        if (l2buf) cudaFree(l2buf);
         if (e0) cudaEventDestroy(e0);
         if (e1) cudaEventDestroy(e1);
     };
@@ -178,17 +239,38 @@ extern "C" cert_status_t cert_peak_microbench(int kind, double target_ms, double
         cleanup();
         return CERT_ERR_OOM;
     }
+    if (kind == 3 && (cudaMalloc(reinterpret_cast<void **>(&l2buf), (size_t)sms * intake_per_cta) != cudaSuccess ||
+                      cudaMemsetAsync(l2buf, 0x3c, (size_t)sms * intake_per_cta, st) != cudaSuccess)) {
+        cudaGetLastError();
+        cleanup();
+        return CERT_ERR_OOM;
+    }
+    TcMap intake_map;
+    if (kind == 3 && (!tc16_prepare_kernels() ||
+                      !tc16_make_map(&intake_map, reinterpret_cast<const __half *>(l2buf), 64 * kIntakeTilesPerRow,
+                                     (long long)sms * 128, 64 * kIntakeTilesPerRow, 64, 128))) {
+        cudaGetLastError();
+        cleanup();
+        return CERT_ERR_UNSUPPORTED;
+    }
     // The kernel needs 34 KB, but it asks for 200 KB so that a multiprocessor holds exactly one of its CTAs, as
     // with the product kernels: two CTAs on one SM would compete for its tensor memory (an allocation that
     // cannot be served blocks without a limit), and a CTA pair must sit on two SMs.
     const int smem = 200 * 1024;
     static_assert(2 * kTileBytes + 1024 + (int)sizeof(PeakBars) <= 200 * 1024, "operand tiles fit");
+    static_assert(kIntakeSlots * kIntakeChunk + 1024 + (int)sizeof(IntakeBars) <= 200 * 1024, "intake ring fits");
     const int pairs = sms / 2;
     double flop_per_unit = 0.0;      // per MMA instruction of one pair, or per loop iteration of the whole grid
     if (kind == 0) flop_per_unit = 2.0 * (kPeakBM * 2) * kPeakBN * 16;
     if (kind == 1) flop_per_unit = 2.0 * (kPeakBM * 2) * kPeakBN * 8;
     const int ffma_blocks = sms;
     if (kind == 2) flop_per_unit = 2.0 * 32.0 * 1024.0 * ffma_blocks;
+    if (kind == 3) flop_per_unit = (double)kIntakeChunk * sms;          // bytes per copy of every CTA
+    if (kind == 3 && cudaFuncSetAttribute(l2_intake_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) {
+        cudaGetLastError();
+        cleanup();
+        return CERT_ERR_CUDA;
+    }
     if (kind < 2 &&
         (cudaFuncSetAttribute(mma_peak_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess ||
          cudaFuncSetAttribute(mma_peak_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)) {
@@ -199,6 +281,10 @@ extern "C" cert_status_t cert_peak_microbench(int kind, double target_ms, double
     auto launch = [&](int units) {
         if (kind == 2) {
             ffma_peak_kernel<<<ffma_blocks, 1024, 0, st>>>(units, sink, clocks);
+            return;
+        }
+        if (kind == 3) {
+            l2_intake_kernel<<<sms, 128, smem, st>>>(reinterpret_cast<const CUtensorMap &>(intake_map), units, status, clocks);
             return;
         }
         cudaLaunchConfig_t cfg = {};
@@ -242,7 +328,7 @@ extern "C" cert_status_t cert_peak_microbench(int kind, double target_ms, double
         rc = CERT_ERR_CUDA;
     if (rc == CERT_OK && flag) rc = CERT_ERR_TIMEOUT;
     if (rc == CERT_OK) {
-        const double total = kind == 2 ? flop_per_unit * units : flop_per_unit * units * pairs;
+        const double total = kind >= 2 ? flop_per_unit * units : flop_per_unit * units * pairs;
         *tflops_out = total / ((double)ms * 1e-3) / 1e12;
         if (sm_mhz_out) *sm_mhz_out = host_clocks[1] ? (double)host_clocks[0] * 1e3 / (double)host_clocks[1] : 0.0;
         if (ms_out) *ms_out = ms;

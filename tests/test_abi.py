@@ -112,7 +112,7 @@ def test_null_handles_and_bad_arguments_of_the_helpers(lib):
     assert L.cert_built_with_checked_stores() == (1 if os.environ.get("CERT_LIB", "").endswith("_checked.so") else 0)
     # the peak micro-kernels validate their arguments before they touch the device
     out = ctypes.c_double()
-    assert L.cert_peak_microbench(3, 5.0, ctypes.byref(out), None, None, None) == 1
+    assert L.cert_peak_microbench(4, 5.0, ctypes.byref(out), None, None, None) == 1
     assert L.cert_peak_microbench(0, 0.0, ctypes.byref(out), None, None, None) == 1
     assert L.cert_peak_microbench(0, 5000.0, ctypes.byref(out), None, None, None) == 1
     assert L.cert_peak_microbench(0, 5.0, None, None, None, None) == 1

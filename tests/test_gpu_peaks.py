@@ -14,8 +14,8 @@ ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 _CODE = r"""
 import json
 from paper_2507_20055_b200 import binding
-out = {k: binding.peak_microbench(k, 3.0) for k in (0, 1, 2)}
-assert binding.lib.cert_peak_microbench(3, 3.0, None, None, None, None) == 1     # bad kind
+out = {k: binding.peak_microbench(k, 3.0) for k in (0, 1, 2, 3)}
+assert binding.lib.cert_peak_microbench(4, 3.0, None, None, None, None) == 1     # bad kind
 assert binding.lib.cert_peak_microbench(0, 0.0, None, None, None, None) == 1     # no output pointer, bad duration
 print("PEAKS " + json.dumps(out))
 """
@@ -31,3 +31,9 @@ def test_peak_microbench_rates_are_the_units_nominal_rates_per_cycle():
         assert 1.0 < ms < 50.0 and 500.0 < mhz < 2100.0
         per_cycle = tflops * 1e12 / (mhz * 1e6) / 148.0
         assert 0.85 * nominal <= per_cycle <= 1.02 * nominal, (kind, per_cycle)
+    # what an SM takes in from L2 through bulk copies: tens of bytes per cycle (the fp16-split contraction in two
+    # passes needs 64 at full MMA rate, in one pass 43)
+    tbs, mhz, ms = peaks["3"]
+    assert 1.0 < ms < 50.0 and 500.0 < mhz < 2100.0
+    per_cycle = tbs * 1e12 / (mhz * 1e6) / 148.0
+    assert 20.0 <= per_cycle <= 200.0, per_cycle
