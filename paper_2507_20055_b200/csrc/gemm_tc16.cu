@@ -507,17 +507,18 @@ __device__ __forceinline__ float warp_sum16(float v) {
 
 // Start of a back-substitution at FC layer k as an fp16 pair: row i of W_k pushed through the ReLU below,
 // constant = b_k[i] + the nu terms + Q.b of the layer below.  The pair is hi = fp16(q_scale x),
-// lo = fp16(lo_scale (q_scale x - hi)): (1, 2^11) for the two-pass contraction, (2^a, 1) for the one-pass one.  A warp takes kRowsPerWarp consecutive neurons
-// of one (box, side), 8 columns per lane: the relaxation and bias vectors are read once for those rows.
+// lo = fp16(lo_scale (q_scale x - hi)): (1, 2^11) for the two-pass contraction, (2^a, 1) for the one-pass one.
+// A warp takes kRowsPerWarp consecutive neurons of one (box, side), 8 columns per lane: the relaxation and bias
+// vectors are read once for those rows.
 constexpr int kRowsPerWarp = 4;
 
 // three 256-thread blocks per SM: the kernel only writes, and needs the warps in flight
-__global__ void __launch_bounds__(256, 3) expr_start16_kernel(const float *__restrict__ Wk, int ldw_k, const float *__restrict__ bias_k,
-                                    __half *__restrict__ Q_hi, __half *__restrict__ Q_lo, float *__restrict__ d,
-                                    long long n_warps, int n_k, int n, int ld, int has_relu,
-                                    const float *__restrict__ lamL, const float *__restrict__ lamU,
-                                    const float *__restrict__ nuU, const float *__restrict__ bias_below,
-                                    int *__restrict__ status, float q_scale, float lo_scale) {
+__global__ void __launch_bounds__(256, 3)
+expr_start16_kernel(const float *__restrict__ Wk, int ldw_k, const float *__restrict__ bias_k, __half *__restrict__ Q_hi,
+                    __half *__restrict__ Q_lo, float *__restrict__ d, long long n_warps, int n_k, int n, int ld,
+                    int has_relu, const float *__restrict__ lamL, const float *__restrict__ lamU,
+                    const float *__restrict__ nuU, const float *__restrict__ bias_below, int *__restrict__ status,
+                    float q_scale, float lo_scale) {
     pdl_trigger();
     pdl_wait();
     const long long w = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
