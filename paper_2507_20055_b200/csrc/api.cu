@@ -29,7 +29,13 @@ struct Tc16Layer {
     __half *Ws_hi = nullptr, *Ws_lo = nullptr;
     cert::TcMap s_hi, s_lo;
     float w_unscale = 1.0f;                      // 2^-w_shift
+    // More, narrower column tiles for launches whose row panels are too few to give every CTA pair a 256-column
+    // tile (small batches, the output layer's traversal): finer[i] has plan.n_tiles + 1 + i column tiles (up to
+    // kMaxFineTiles) and weight maps with the matching box; the output maps are the common ones.
+    struct Finer { cert::Tc16Plan plan; cert::TcMap hi, lo; bool ok = false; };
+    std::vector<Finer> finer;
 };
+constexpr int kMaxFineTiles = 16;
 
 struct TcLayer {
     bool usable = false;
@@ -383,6 +389,16 @@ cert_status_t setup_tensor_core_path(cert_net *net, const cert_layer_desc_t *des
                 T.w_unscale = std::ldexp(1.0f, -shift);
                 T.one_pass = cert::tc16_make_map(&T.s_hi, T.Ws_hi, L.n_out, L.n_in, L.ld_out, 64, T.plan.bn / 2) &&
                              cert::tc16_make_map(&T.s_lo, T.Ws_lo, L.n_out, L.n_in, L.ld_out, 64, T.plan.bn / 2);
+                const int units = (L.n_in + 31) / 32;
+                for (int nt = T.plan.n_tiles + 1; T.one_pass && nt <= std::min(units, kMaxFineTiles); ++nt) {
+                    Tc16Layer::Finer F;
+                    F.plan = cert::tc16_tile_plan(L.n_in, nt);
+                    F.ok = F.plan.stages >= 2 &&
+                           cert::tc16_make_map(&F.hi, T.Ws_hi, L.n_out, L.n_in, L.ld_out, 64, F.plan.bn / 2) &&
+                           cert::tc16_make_map(&F.lo, T.Ws_lo, L.n_out, L.n_in, L.ld_out, 64, F.plan.bn / 2);
+                    if (F.ok) net->d_slots = std::max(net->d_slots, 2 * nt);
+                    T.finer.push_back(F);
+                }
             }
             all_one_pass = all_one_pass && T.one_pass;
             long long rows_max = 0;
@@ -981,11 +997,20 @@ void run_tc16_steps(Traversal &t) {
         w.set_aside(t, j, cur, true);
         const int nxt = next_buffer(t, cur, w.kept);
         const bool join = j > t.j_end && w.wait_for == j - 1;
-        cert::TcArgs a = tc_args(t, Lj.n_out, Lk.n_out, Lj.ld_in, T.plan.bn, T.plan.n_tiles, T.plan.stages,
-                                 T.plan.tmem_cols, 256, T.plan.n_tiles, dcur, dslots);
+        // the tile plan: 256-column tiles unless the row panels are too few to give every CTA pair one; then as many
+        // column tiles as keep the launch one wave of work tiles
+        const cert::Tc16Plan *P = &T.plan;
+        const cert::TcMap *b_hi = one_pass ? &T.s_hi : &T.b_hi, *b_lo = one_pass ? &T.s_lo : &T.b_lo;
+        const long long panels = cert::ceil_div_ll(t.rows, 256);
+        const int want = (int)std::min<long long>((net->sm_count / 2) / panels, kMaxFineTiles);
+        if (one_pass && want > T.plan.n_tiles && !T.finer.empty()) {
+            const int i = std::min(want - T.plan.n_tiles - 1, (int)T.finer.size() - 1);
+            if (T.finer[i].ok) { P = &T.finer[i].plan; b_hi = &T.finer[i].hi; b_lo = &T.finer[i].lo; }
+        }
+        cert::TcArgs a = tc_args(t, Lj.n_out, Lk.n_out, Lj.ld_in, P->bn, P->n_tiles, P->stages, P->tmem_cols, 256,
+                                 P->n_tiles, dcur, dslots);
         a.q_scale = q_scale; a.q_unscale = q_unscale; a.acc_scale = q_unscale * T.w_unscale;
-        a.n_narrow = T.plan.n_narrow;
-        const cert::TcMap &b_hi = one_pass ? T.s_hi : T.b_hi, &b_lo = one_pass ? T.s_lo : T.b_lo;
+        a.n_narrow = P->n_narrow;
         const int pairs = std::min(a.total_tiles, net->sm_count / 2);
         if (j > t.j_end) {
             tc_relu_epilogue(a, t.layer(j - 1), true);
@@ -994,18 +1019,18 @@ void run_tc16_steps(Traversal &t) {
                 a.add_lo = reinterpret_cast<const float *>(ql[w.kept]);
             }
             a.add_identity = (join && w.identity) ? 1 : 0;
-            cert::launch_gemm_tc16(cert::TC_EPI_RELU, one_pass, pairs, T.a_hi[cur], T.a_lo[cur], b_hi, b_lo, T.o_hi[nxt],
-                                   T.o_lo[nxt], a, T.plan.smem_bytes, t.st);
+            cert::launch_gemm_tc16(cert::TC_EPI_RELU, one_pass, pairs, T.a_hi[cur], T.a_lo[cur], *b_hi, *b_lo, T.o_hi[nxt],
+                                   T.o_lo[nxt], a, P->smem_bytes, t.st);
             if (join) w.joined();
         } else {
             a.l0 = t.box_l; a.u0 = t.box_u;
-            cert::launch_gemm_tc16(cert::TC_EPI_CONCRETIZE, one_pass, pairs, T.a_hi[cur], T.a_lo[cur], b_hi, b_lo,
-                                   T.a_hi[cur], T.a_lo[cur], a, T.plan.smem_bytes, t.st);
+            cert::launch_gemm_tc16(cert::TC_EPI_CONCRETIZE, one_pass, pairs, T.a_hi[cur], T.a_lo[cur], *b_hi, *b_lo,
+                                   T.a_hi[cur], T.a_lo[cur], a, P->smem_bytes, t.st);
         }
         t.rec->mark(CERT_CLASS_AFFINE);
         cur = nxt;
         dcur ^= 1;
-        dslots = 2 * T.plan.n_tiles;
+        dslots = 2 * P->n_tiles;
     }
     t.relax(net->dbuf[dcur], dslots);
     t.paths |= 2 | 4 | 16;

@@ -669,9 +669,9 @@ bool tc16_make_map(TcMap *m, const __half *base, long long inner, long long oute
     return r == CUDA_SUCCESS;
 }
 
-Tc16Plan tc16_tile_plan(int N) {
+Tc16Plan tc16_tile_plan(int N, int n_tiles) {
     Tc16Plan p;
-    p.n_tiles = (N + 255) / 256;
+    p.n_tiles = n_tiles > 0 ? n_tiles : (N + 255) / 256;
     // 32-column units spread over the tiles: the first tiles take one unit more than the last n_narrow ones
     const int units = (N + 31) / 32;
     int b = (units + p.n_tiles - 1) / p.n_tiles * 32;

@@ -27,7 +27,9 @@ bool tc16_prepare_kernels();
 // box_inner = 64 -> 128-byte swizzle (operand tiles), 32 -> 64-byte swizzle (epilogue slabs).
 bool tc16_make_map(TcMap *m, const __half *base, long long inner, long long outer, long long pitch_elems,
                    int box_inner, int box_outer);
-Tc16Plan tc16_tile_plan(int N);
+// n_tiles = 0: as few column tiles as 256 columns per tile allow; n_tiles > 0: that many (launches with too few row
+// panels to give every CTA pair a 256-column tile take more, narrower ones)
+Tc16Plan tc16_tile_plan(int N, int n_tiles = 0);
 // CTA pairs only.  TcArgs as for the TF32 kernel; d_out receives 2 * n_tiles slots per row.
 // one_pass == false: both operands are pairs (fp16(x), fp16(2^11 (x - hi))), two passes over K.
 // one_pass == true (not for TC_EPI_REUSE): both operands are pairs with unscaled lo parts of 2^a Q and 2^s W

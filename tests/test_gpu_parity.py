@@ -462,6 +462,18 @@ def test_fp16_split_unequal_column_tiles_with_residual_connections(mode):
     compare(g, _oracle(w), min_good_fraction=0.6, label=f"residual 272-wide/{mode}")
 
 
+@pytest.mark.parametrize("batch", [1, 3])
+def test_fc6x1024_small_batches_take_more_column_tiles(batch):
+    """784 -> 1024 x 6 -> 10 on one and three boxes: 8 and 24 row panels per contraction, too few to give each of the
+    74 CTA pairs a 256-column tile, so the launches take as many narrower column tiles as keep them
+    one wave (the output layer's traversal sixteen); every box against the oracle."""
+    w = wl.make_config(4, batch=batch + 1)
+    w.centers = np.ascontiguousarray(w.centers[1:])          # (the first box has a near-tie neuron)
+    g = run_gpu(w, max_batch=batch + 1)
+    assert g["paths"] & 16
+    compare(g, _oracle(w), label=f"fc6x1024/{batch} boxes")
+
+
 def test_fp16_split_chain_wide_input_and_many_layers():
     """A CIFAR-sized input (14 column tiles in the concretising step) and the deepest net the chain kernel's
     parameter block takes (12 layers); one layer more goes back to one launch per back-step."""
